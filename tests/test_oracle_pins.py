@@ -1,0 +1,347 @@
+"""Pins for the CPU oracle: each part is checked against something other than itself —
+brute force on tiny inputs, closed forms, textbook routines that take another route, and the
+invariants the paper's equations imply (Eq. 4-9, Algorithm 1)."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import pkv_oracle as orc
+from paper_2609_39329_b200 import inputs as gen
+
+
+def tiny_cfg(**kw):
+    base = gen.benchmark_config(2)
+    d = dict(d=32, Hq=4, Hkv=2, hd=8, F=24, L=40, N=12, window=4, budget=10, n_obs=4,
+             rope_theta=1e4, name="pin")
+    d.update(kw)
+    return gen.scaled_config(base, **d)
+
+
+def tiny_problem(cfg, seed=0, scale_w=0.3):
+    r = np.random.default_rng(seed)
+    w = {k: r.standard_normal(s) * scale_w for k, s in {
+        "Wq": (cfg.Dq, cfg.d), "Wk": (cfg.Dkv, cfg.d), "Wv": (cfg.Dkv, cfg.d), "Wo": (cfg.d, cfg.Dq),
+        "Wgate": (cfg.F, cfg.d), "Wup": (cfg.F, cfg.d), "Wdown": (cfg.d, cfg.F)}.items()}
+    w["g_attn"] = 1.0 + 0.1 * r.standard_normal(cfg.d)
+    w["g_mlp"] = 1.0 + 0.1 * r.standard_normal(cfg.d)
+    K = r.standard_normal((cfg.Hkv, cfg.L, cfg.hd))
+    V = r.standard_normal((cfg.Hkv, cfg.L, cfg.hd))
+    x = r.standard_normal((cfg.N, cfg.d))
+    kept = [np.sort(r.choice(cfg.L, size=cfg.budget, replace=False)).astype(np.int32) for _ in range(cfg.Hkv)]
+    return w, K, V, x, kept
+
+
+# ------------------------------------------------------------------ attention ----------
+
+def brute_attention(q, k_new, v_new, K_cache, V_cache, chunk_off):
+    """Literal per-element coding: one query row at a time, python loops, explicit key list."""
+    n, Hq, hd = q.shape
+    g = Hq // k_new.shape[1]
+    out = np.zeros((n, Hq, hd))
+    for c in range(len(chunk_off) - 1):
+        s, e = chunk_off[c], chunk_off[c + 1]
+        for i in range(s, e):
+            for h in range(Hq):
+                kh = h // g
+                keys = [K_cache[kh][r] for r in range(len(K_cache[kh]))] + [k_new[j, kh] for j in range(s, i + 1)]
+                vals = [V_cache[kh][r] for r in range(len(V_cache[kh]))] + [v_new[j, kh] for j in range(s, i + 1)]
+                lg = [sum(q[i, h, t] * kk[t] for t in range(hd)) / math.sqrt(hd) for kk in keys]
+                mx = max(lg)
+                ex = [math.exp(v - mx) for v in lg]
+                den = sum(ex)
+                for t in range(hd):
+                    out[i, h, t] = sum(ex[r] * vals[r][t] for r in range(len(keys))) / den
+    return out.reshape(n, Hq * hd)
+
+
+def rand_attn_inputs(seed=1, n=7, Hq=4, Hkv=2, hd=6, rows=(9, 5)):
+    r = np.random.default_rng(seed)
+    q = r.standard_normal((n, Hq, hd))
+    k = r.standard_normal((n, Hkv, hd))
+    v = r.standard_normal((n, Hkv, hd))
+    Kc = [r.standard_normal((rows[h], hd)) for h in range(Hkv)]
+    Vc = [r.standard_normal((rows[h], hd)) for h in range(Hkv)]
+    return q, k, v, Kc, Vc
+
+
+def test_attention_matches_brute_force_with_chunks_and_ragged_heads():
+    q, k, v, Kc, Vc = rand_attn_inputs()
+    for chunks in ([0, 7], [0, 3, 7], [0, 1, 2, 7]):
+        a = orc.attention(q, k, v, Kc, Vc, chunks)
+        b = brute_attention(q, k, v, Kc, Vc, chunks)
+        np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
+
+
+def test_attention_equal_keys_gives_mean_of_visible_values():
+    q, k, v, Kc, Vc = rand_attn_inputs(rows=(6, 6))
+    one = np.ones(q.shape[2])
+    Kc = [np.tile(one, (6, 1)) for _ in range(2)]
+    k = np.tile(one, (q.shape[0], 2, 1))
+    a = orc.attention(q, k, v, Kc, Vc, [0, q.shape[0]]).reshape(q.shape)
+    for i in range(q.shape[0]):
+        for h in range(q.shape[1]):
+            kh = h // 2
+            want = (Vc[kh].sum(0) + v[:i + 1, kh].sum(0)) / (6 + i + 1)
+            np.testing.assert_allclose(a[i, h], want, rtol=1e-12)
+
+
+def test_attention_dominant_key_returns_its_value():
+    q, k, v, Kc, Vc = rand_attn_inputs()
+    Kc[0][3] = 1e4 * q[2, 0] / np.linalg.norm(q[2, 0])      # aligned with query (token 2, head 0)
+    a = orc.attention(q, k, v, Kc, Vc, [0, 7]).reshape(q.shape)
+    np.testing.assert_allclose(a[2, 0], Vc[0][3], atol=1e-9)
+
+
+def test_attention_invariant_to_cache_permutation_and_logit_shift():
+    q, k, v, Kc, Vc = rand_attn_inputs()
+    a = orc.attention(q, k, v, Kc, Vc, [0, 4, 7])
+    perm = [np.random.default_rng(5).permutation(len(K)) for K in Kc]
+    b = orc.attention(q, k, v, [K[p] for K, p in zip(Kc, perm)], [V[p] for V, p in zip(Vc, perm)], [0, 4, 7])
+    np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
+    # a constant added to every logit of a head: the same bias on every cached key and an
+    # extra key coordinate paired with a constant query coordinate for the chunk keys
+    hd = q.shape[2]
+    q2 = np.concatenate([q, np.ones(q.shape[:2] + (1,))], axis=2) * math.sqrt((hd + 1) / hd)
+    k2 = np.concatenate([k, 3.0 * np.ones(k.shape[:2] + (1,))], axis=2)
+    Kc2 = [np.concatenate([K, 3.0 * np.ones((len(K), 1))], axis=1) for K in Kc]
+    v2 = np.concatenate([v, np.zeros(v.shape[:2] + (1,))], axis=2)
+    Vc2 = [np.concatenate([V, np.zeros((len(V), 1))], axis=1) for V in Vc]
+    c = orc.attention(q2, k2, v2, Kc2, Vc2, [0, 4, 7]).reshape(q.shape[0], q.shape[1], hd + 1)[..., :hd]
+    np.testing.assert_allclose(a, c.reshape(a.shape), rtol=1e-11, atol=1e-12)
+
+
+def test_attention_split_key_sets_merge_back():
+    """Softmax partials (m, l, O) over disjoint key subsets recombine to the whole."""
+    q, k, v, Kc, Vc = rand_attn_inputs(rows=(11, 11))
+    whole = orc.attention(q, k, v, Kc, Vc, [0, 7]).reshape(q.shape)
+    hd = q.shape[2]
+    for i in (0, 3, 6):
+        for h in range(q.shape[1]):
+            kh = h // 2
+            keys = np.concatenate([Kc[kh], k[:i + 1, kh]])
+            vals = np.concatenate([Vc[kh], v[:i + 1, kh]])
+            parts = np.array_split(np.arange(len(keys)), 3)
+            ms, ls, Os = [], [], []
+            for p in parts:
+                lg = keys[p] @ q[i, h] / math.sqrt(hd)
+                m = lg.max()
+                e = np.exp(lg - m)
+                ms.append(m); ls.append(e.sum()); Os.append(e @ vals[p])
+            M = max(ms)
+            num = sum(np.exp(m - M) * O for m, O in zip(ms, Os))
+            den = sum(np.exp(m - M) * l for m, l in zip(ms, ls))
+            np.testing.assert_allclose(whole[i, h], num / den, rtol=1e-12)
+
+
+def test_gqa_equals_mha_with_replicated_kv_heads():
+    q, k, v, Kc, Vc = rand_attn_inputs(rows=(9, 9))
+    a = orc.attention(q, k, v, Kc, Vc, [0, 7])
+    rep = lambda t: np.repeat(t, 2, axis=1)
+    b = orc.attention(q, rep(k), rep(v), [Kc[0], Kc[0], Kc[1], Kc[1]], [Vc[0], Vc[0], Vc[1], Vc[1]], [0, 7])
+    np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
+
+
+def test_kept_gather_equals_full_cache_with_evicted_rows_masked():
+    q, k, v, Kc, Vc = rand_attn_inputs(rows=(9, 9))
+    kept = [np.array([0, 2, 3, 8]), np.array([1, 4, 5, 6, 7])]
+    Kg, Vg = orc.gather_cache(np.stack(Kc), np.stack(Vc), kept)
+    a = orc.attention(q, k, v, Kg, Vg, [0, 7])
+    bias = [np.where(np.isin(np.arange(9), kk), 0.0, -np.inf) for kk in kept]
+    b = orc.attention(q, k, v, Kc, Vc, [0, 7], key_bias=bias)
+    np.testing.assert_allclose(a, b, rtol=1e-12, atol=1e-13)
+
+
+def test_empty_cache_and_first_token_sees_only_itself():
+    q, k, v, _, _ = rand_attn_inputs()
+    empty = [np.zeros((0, q.shape[2]))] * 2
+    a = orc.attention(q, k, v, empty, empty, [0, 3, 7]).reshape(q.shape)
+    for s in (0, 3):                      # first token of a chunk: softmax over one key
+        for h in range(q.shape[1]):
+            np.testing.assert_allclose(a[s, h], v[s, h // 2], rtol=1e-13)
+
+
+# ------------------------------------------------------------------ backbone conventions
+
+def test_rope_is_a_rotation_and_relative():
+    r = np.random.default_rng(0)
+    t = r.standard_normal((5, 3, 8))
+    pos = np.array([0, 1, 7, 100, 4096])
+    rt = orc.rope(t, pos, 1e4)
+    np.testing.assert_allclose(np.linalg.norm(rt, axis=-1), np.linalg.norm(t, axis=-1), rtol=1e-12)
+    np.testing.assert_allclose(rt[0], t[0], rtol=0, atol=0)                 # position 0: identity
+    # inner products depend on position differences only
+    a, b = r.standard_normal((1, 1, 8)), r.standard_normal((1, 1, 8))
+    d1 = np.sum(orc.rope(a, np.array([10]), 1e4) * orc.rope(b, np.array([3]), 1e4))
+    d2 = np.sum(orc.rope(a, np.array([110]), 1e4) * orc.rope(b, np.array([103]), 1e4))
+    assert abs(d1 - d2) < 1e-12
+    # first pair (c = 0, partner hd/2) turns by exactly pos radians
+    e = np.zeros((1, 1, 8)); e[0, 0, 0] = 1.0
+    out = orc.rope(e, np.array([2]), 1e4)[0, 0]
+    np.testing.assert_allclose([out[0], out[4]], [math.cos(2.0), math.sin(2.0)], rtol=1e-13)
+
+
+def test_rmsnorm_and_silu_closed_forms():
+    x = np.array([[3.0, 4.0, 0.0, 0.0]])
+    u = orc.rmsnorm(x, np.array([1.0, 2.0, 1.0, 1.0]), 0.0)
+    np.testing.assert_allclose(u, [[3 / 2.5, 2 * 4 / 2.5, 0, 0]], rtol=1e-14)
+    assert abs(orc.silu(np.array([0.0]))[0]) == 0.0
+    np.testing.assert_allclose(orc.silu(np.array([2.0])), 2.0 / (1 + math.exp(-2.0)), rtol=1e-15)
+
+
+# ------------------------------------------------------------------ ridge regression ---
+
+def rand_XR(seed, N, F, d):
+    r = np.random.default_rng(seed)
+    return r.standard_normal((N, F)), r.standard_normal((N, d))
+
+
+@pytest.mark.parametrize("N,F,d", [(40, 12, 9), (7, 12, 9)])
+def test_ridge_solution_stationarity_and_other_routes(N, F, d):
+    X, R = rand_XR(3, N, F, d)
+    lam = 0.37
+    S_H, S_T = orc.sufficient_statistics(X, R)
+    dW = orc.ridge_solve(S_H, S_T, lam)                       # [d][F]
+    B = dW.T                                                  # [F][d] = G^{-1} C
+    C = X.T @ R
+    grad = X.T @ (X @ B - R) + lam * B                        # stationarity of Eq. 6
+    assert np.linalg.norm(grad) <= 1e-10 * np.linalg.norm(C)
+    # least squares on the augmented system never forms G
+    A = np.vstack([X, math.sqrt(lam) * np.eye(F)])
+    b = np.vstack([R, np.zeros((F, d))])
+    np.testing.assert_allclose(B, np.linalg.lstsq(A, b, rcond=None)[0], rtol=1e-9, atol=1e-11)
+    # dual form
+    np.testing.assert_allclose(B, X.T @ np.linalg.solve(X @ X.T + lam * np.eye(N), R), rtol=1e-9, atol=1e-11)
+    # paper orientation: dW = T^T H' (H'^T H' + lam I)^{-1}
+    np.testing.assert_allclose(dW, R.T @ X @ np.linalg.inv(X.T @ X + lam * np.eye(F)), rtol=1e-9, atol=1e-11)
+    # objective identities and optimality under perturbation
+    J = lambda Bm: np.sum((X @ Bm - R) ** 2) + lam * np.sum(Bm ** 2)
+    np.testing.assert_allclose(J(B), np.sum(R * R) - np.sum(C * B), rtol=1e-10)
+    np.testing.assert_allclose(np.sum((R - X @ B) ** 2), np.sum(R * R) - np.sum(C * B) - lam * np.sum(B * B), rtol=1e-9)
+    r = np.random.default_rng(9)
+    for _ in range(5):
+        assert J(B + 1e-3 * r.standard_normal(B.shape)) > J(B)
+
+
+def test_ridge_single_token_rank_one_closed_form():
+    X, R = rand_XR(4, 1, 10, 6)
+    lam = 0.2
+    S_H, S_T = orc.sufficient_statistics(X, R)
+    dW = orc.ridge_solve(S_H, S_T, lam)
+    want = np.outer(R[0], X[0]) / (X[0] @ X[0] + lam)
+    np.testing.assert_allclose(dW, want, rtol=1e-11)
+
+
+def test_ridge_large_lambda_limit_and_zero_target():
+    X, R = rand_XR(5, 9, 10, 6)
+    S_H, S_T = orc.sufficient_statistics(X, R)
+    lam = 1e9
+    gap = np.linalg.norm(lam * orc.ridge_solve(S_H, S_T, lam) - S_T)      # = O(||S_H|| / lam)
+    assert gap <= 2.0 * np.linalg.norm(S_H, 2) / lam * np.linalg.norm(S_T)
+    assert np.all(orc.ridge_solve(S_H, np.zeros_like(S_T), 0.1) == 0.0)
+    with pytest.raises(ValueError):
+        orc.ridge_solve(S_H, S_T, 0.0)
+
+
+def test_statistics_chunk_additivity():
+    X, R = rand_XR(6, 23, 8, 5)
+    a = orc.sufficient_statistics(X, R)
+    b = orc.sufficient_statistics(X, R, [0, 4, 5, 17, 23])
+    np.testing.assert_allclose(a[0], b[0], rtol=1e-13)
+    np.testing.assert_allclose(a[1], b[1], rtol=1e-13)
+    np.testing.assert_allclose(a[1], R.T @ X, rtol=1e-13)          # S_T = T^T H' is [d][F]
+
+
+def test_adaptive_lambda_is_weighted_eigenvalue_mean():
+    X, _ = rand_XR(7, 6, 10, 1)
+    S = X.T @ X
+    ev = np.linalg.eigvalsh(S)
+    lam = orc.ridge_lambda(S, 0.5)
+    np.testing.assert_allclose(lam, 0.5 * np.sum(ev ** 2) / np.sum(ev), rtol=1e-10)
+    assert np.trace(S) / S.shape[0] <= lam / 0.5 <= ev.max() * (1 + 1e-12)
+    assert orc.ridge_lambda(S, 0.5, orc.LAMBDA_ABSOLUTE) == 0.5
+    np.testing.assert_allclose(orc.ridge_lambda(S, 0.5, orc.LAMBDA_TRACE_MEAN), 0.5 * np.trace(S) / 10)
+    with pytest.raises(ZeroDivisionError):
+        orc.ridge_lambda(np.zeros((3, 3)), 0.1)
+
+
+# ------------------------------------------------------------------ block identities ---
+
+def test_identical_caches_give_zero_target_and_zero_patch():
+    cfg = tiny_cfg()
+    w, K, V, x, _ = tiny_problem(cfg)
+    full = [np.arange(cfg.L, dtype=np.int32)] * cfg.Hkv
+    out = orc.build_patch(w, K, V, full, x, x, [0, cfg.N], cfg.L, 0.1, cfg, keep_intermediates=True)
+    assert np.all(out["T"] == 0.0)
+    assert np.all(out["dW"] == 0.0)
+    np.testing.assert_array_equal(out["xF_next"], out["xC_next"])
+
+
+def test_patched_student_block_output_gap_is_ridge_residual():
+    """Eq. 4: teacher block output minus the patched student's equals T - H' dW^T, where the
+    patched output is obtained by actually running the block with W + dW."""
+    cfg = tiny_cfg()
+    w, K, V, x, kept = tiny_problem(cfg)
+    xC = x + 0.05 * np.random.default_rng(3).standard_normal(x.shape)
+    chunks = [0, 5, cfg.N]
+    out = orc.build_patch(w, K, V, kept, x, xC, chunks, cfg.L, 0.05, cfg, keep_intermediates=True)
+    Kc, Vc = orc.gather_cache(K, V, kept)
+    w2 = dict(w); w2["Wdown"] = w["Wdown"] + out["dW"]
+    stu = orc.block_forward(xC, w2, Kc, Vc, chunks, cfg.L, cfg)
+    tea = orc.block_forward(x, w, list(K), list(V), chunks, cfg.L, cfg)
+    yF = tea["z"] + tea["h"] @ w["Wdown"].T
+    yC = stu["z"] + stu["h"] @ w2["Wdown"].T
+    np.testing.assert_allclose(out["xF_next"], yF, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(out["xC_next"], yC, rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(yF - yC, out["T"] - out["H"] @ out["dW"].T, rtol=1e-8, atol=1e-11)
+    # the ridge-optimal residual reduction: ||T - H'dW^T||^2 = ||T||^2 - <S_T, dW> - lam ||dW||^2
+    want = out["T_fro2"] - np.sum(out["S_T"] * out["dW"]) - out["lam"] * out["dW_fro"] ** 2
+    np.testing.assert_allclose(out["res_fro2"], want, rtol=1e-9)
+    assert out["res_fro2"] < out["T_fro2"]
+
+
+def test_small_lambda_with_fewer_tokens_than_features_reproduces_teacher():
+    cfg = tiny_cfg(N=6, F=24)
+    w, K, V, x, kept = tiny_problem(cfg)
+    out = orc.build_patch(w, K, V, kept, x, x, [0, cfg.N], cfg.L, 1e-9, cfg)
+    assert out["res_fro2"] < 1e-12 * out["T_fro2"]
+    np.testing.assert_allclose(out["xC_next"], out["xF_next"], rtol=1e-5, atol=1e-6)
+
+
+def test_chunks_are_independent_and_restart_positions():
+    cfg = tiny_cfg()
+    w, K, V, x, kept = tiny_problem(cfg)
+    Kc, Vc = orc.gather_cache(K, V, kept)
+    both = orc.block_forward(x, w, Kc, Vc, [0, 5, cfg.N], cfg.L, cfg)
+    second = orc.block_forward(x[5:], w, Kc, Vc, [0, cfg.N - 5], cfg.L, cfg)
+    np.testing.assert_allclose(both["h"][5:], second["h"], rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(both["z"][5:], second["z"], rtol=1e-12, atol=1e-13)
+
+
+def test_build_patch_rejects_bad_index_sets():
+    cfg = tiny_cfg()
+    w, K, V, x, kept = tiny_problem(cfg)
+    for bad in ([3, 3, 5], [5, 4], [-1, 2], [0, cfg.L]):
+        k2 = [np.array(bad, dtype=np.int32), kept[1]]
+        assert orc.check_kept(k2, cfg.L) is not None
+        with pytest.raises(IndexError):
+            orc.build_patch(w, K, V, k2, x, x, [0, cfg.N], cfg.L, 0.1, cfg)
+    assert orc.check_kept(kept, cfg.L) is None
+    assert orc.check_kept([np.zeros(0, dtype=np.int32)] * 2, cfg.L) is None
+
+
+# ------------------------------------------------------------------ merge and formats --
+
+def test_bf16_rounding_and_merge_match_torch():
+    import torch
+    r = np.random.default_rng(0)
+    a = (r.standard_normal(4096) * np.exp(r.uniform(-20, 20, 4096))).astype(np.float32)
+    a[:4] = [1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, -(1.0 + 2 ** -8), 0.0]          # ties
+    want = torch.from_numpy(a).to(torch.bfloat16).to(torch.float32).numpy()
+    np.testing.assert_array_equal(orc.round_bf16(a), want)
+    np.testing.assert_array_equal(gen.round_to_bf16(a), want)
+    W = gen.round_to_bf16(r.standard_normal((8, 8)).astype(np.float32) * 0.02)
+    dW = (r.standard_normal((8, 8)) * 1e-3).astype(np.float32)
+    want = (torch.from_numpy(W) + torch.from_numpy(dW)).to(torch.bfloat16).to(torch.float32).numpy()
+    np.testing.assert_array_equal(orc.merge(W, dW, "bf16"), want)
+    np.testing.assert_array_equal(orc.merge(W, dW, "fp32"), W + dW)
