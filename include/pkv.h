@@ -1,0 +1,222 @@
+/*
+ * pkv.h — C ABI of the PatchKV patch-construction library (libpkv.so, CUDA, sm_100a).
+ *
+ * What the library computes (per transformer block; paper Sec. 2.2-2.3, Algorithm 1):
+ * reference tokens are run through the block twice, once attending to the full KV cache
+ * (teacher) and once to a compressed cache (student); the target t = W(h-h') + (z-z')
+ * (Eq. 5) and the student's MLP features h' give the sufficient statistics
+ * S_H = H'^T H', S_T = T^T H' (Eq. 9); the patch of the MLP down projection is
+ * dW = S_T (S_H + lambda I)^{-1} (Eq. 8) with lambda = lambda0 ||S_H||_F^2 / tr(S_H)
+ * (Eq. 7); the patch is merged as W <- W + dW (Algorithm 1, Merge).
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory owned by the caller (any allocator); the
+ *     library never frees or keeps them after the call returns.  "host" pointers are plain
+ *     host memory.  Inputs are read-only.  Outputs must not alias inputs.
+ *   - All matrices are dense row-major.  Weight matrices are [out][in] (the paper writes the
+ *     down projection as W in R^{d x d_ff}); the patch dW has the layout of W, [d][F].
+ *   - Weights and caches have the element type pkv_dims.dtype (bf16 or fp32).  Residual-stream
+ *     states (xF, xC, next states) and dW are always fp32.
+ *   - Every function returns PKV_OK (0) or a negative pkv_error; nothing throws, aborts or
+ *     traps on the device.  After an error the contents of the outputs are unspecified.
+ *   - Work is enqueued on the CUDA stream given at pkv_create; pkv_build_patch ends with one
+ *     stream synchronisation to read the device status word, so its return code is truthful.
+ *   - A context is not thread-safe; use one per host thread / stream.
+ */
+#ifndef PKV_H_
+#define PKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum pkv_error {
+    PKV_OK = 0,
+    PKV_ERR_INVALID_ARG = -1,  /* null/misaligned pointer, lambda <= 0 or non-finite, N = 0, bad chunk offsets */
+    PKV_ERR_UNSUPPORTED = -2,  /* hd not in {64,128}, Hq % Hkv != 0, F > 8192, sizes the kernels do not cover */
+    PKV_ERR_BAD_INDEX = -3,    /* kept-index set not strictly ascending within [0, L); first offender in stats */
+    PKV_ERR_NOT_PD = -4,       /* Cholesky pivot <= 0 or non-finite; column in stats.err_info */
+    PKV_ERR_DEGENERATE = -5,   /* tr(S_H) = 0 under the adaptive ridge scale (Eq. 7) */
+    PKV_ERR_NONFINITE = -6,    /* NaN/Inf met in the statistics */
+    PKV_ERR_TIMEOUT = -7,      /* a bounded device-side wait (TMA / tensor-core pipeline) expired */
+    PKV_ERR_CUDA = -8,         /* a CUDA runtime call failed; see pkv_last_cuda_error */
+    PKV_ERR_NOMEM = -9         /* workspace allocation failed or caller-provided workspace too small */
+} pkv_error;
+
+enum { PKV_BF16 = 0, PKV_FP32 = 1 };
+
+/* How the ridge coefficient handed to pkv_build_patch is read. */
+enum {
+    PKV_LAMBDA_PAPER = 0,      /* lambda = lambda0 * ||S_H||_F^2 / tr(S_H)   (Eq. 7; default) */
+    PKV_LAMBDA_ABSOLUTE = 1,   /* lambda = lambda0                            (Eq. 6 as written) */
+    PKV_LAMBDA_TRACE_MEAN = 2  /* lambda = lambda0 * tr(S_H) / F              (ridge-scale ablation) */
+};
+
+enum {
+    PKV_ENGINE_AUTO = 0,       /* tcgen05/TMA tensor-core kernels for bf16, SIMT fp32 kernels for fp32 */
+    PKV_ENGINE_SIMT = 1        /* force the SIMT fp32 kernels (on-device cross-check of the tensor path) */
+};
+
+/* Geometry of one block and the capacity the context is sized for. */
+typedef struct pkv_dims {
+    int32_t d;            /* hidden size */
+    int32_t Hq, Hkv, hd;  /* query heads, key/value heads (Hq % Hkv == 0), head dim (64 or 128) */
+    int32_t F;            /* MLP intermediate width (<= 8192) */
+    int32_t L;            /* rows of the full cache per KV head */
+    int32_t N_max;        /* most reference tokens one call may bring */
+    int32_t b_max;        /* most kept rows per KV head in a compressed cache */
+    int32_t dtype;        /* PKV_BF16 | PKV_FP32: element type of weights and caches */
+    float rope_theta;     /* rotary base; 0 disables the rotation */
+    float eps;            /* RMSNorm epsilon */
+} pkv_dims;
+
+typedef struct pkv_opts {
+    int32_t engine;          /* PKV_ENGINE_* */
+    int32_t kv_split;        /* cache rows per attention split; 0 = choose from L and the SM count */
+    void* workspace;         /* optional caller-provided device workspace (256-byte aligned) ... */
+    size_t workspace_bytes;  /* ... of at least pkv_workspace_bytes(); NULL/0: the context allocates */
+} pkv_opts;
+
+/* Block weights, all device, element type dims.dtype except the fp32 norm gains.
+ * Layout [out][in]: Wq[Hq*hd][d] Wk[Hkv*hd][d] Wv[Hkv*hd][d] Wo[d][Hq*hd]
+ *                   Wgate[F][d] Wup[F][d] Wdown[d][F].  Pointers 16-byte aligned. */
+typedef struct pkv_block_weights {
+    const float* g_attn;  /* [d] */
+    const void* Wq;
+    const void* Wk;
+    const void* Wv;
+    const void* Wo;
+    const float* g_mlp;   /* [d] */
+    const void* Wgate;
+    const void* Wup;
+    const void* Wdown;    /* the matrix the patch is built for (unpatched base weights) */
+} pkv_block_weights;
+
+/* Full cache of the block: K, V [Hkv][L][hd], device, keys already rotated. */
+typedef struct pkv_kv {
+    const void* K;
+    const void* V;
+} pkv_kv;
+
+/* Compressed cache, one of two forms (Sec. 2.1: eviction or approximation compressors).
+ *  (a) kept-index set:  idx != NULL.  Head h keeps rows idx[head_off[h] .. head_off[h+1])
+ *      of the full cache, strictly ascending, each in [0, L).  Heads may keep different counts.
+ *  (b) explicit cache:  idx == NULL, Kc/Vc != NULL, packed [head_off[Hkv]][hd] with head h's
+ *      rows at head_off[h]...; optional per-key logit bias (fp32, same packing) or NULL.
+ * head_off is a HOST array of Hkv+1 ints starting at 0; idx/Kc/Vc/bias are device. */
+typedef struct pkv_kv_compressed {
+    const int32_t* head_off;
+    const int32_t* idx;
+    const void* Kc;
+    const void* Vc;
+    const float* bias;
+} pkv_kv_compressed;
+
+/* Reference tokens entering the block (Algorithm 1: states x^F, x^C of every chunk).
+ * xF, xC: device fp32 [N][d] (may alias each other at the first block).  chunk_off: HOST
+ * array of n_chunks+1 strictly increasing offsets, chunk_off[0]=0, chunk_off[n_chunks]=N.
+ * A token attends to the whole cache and causally inside its own chunk; token i of a chunk
+ * starting at s has position pos0 + (i - s) in both streams. */
+typedef struct pkv_ref {
+    const float* xF;
+    const float* xC;
+    int32_t N;
+    int32_t n_chunks;
+    const int32_t* chunk_off;
+    int32_t pos0;
+} pkv_ref;
+
+/* Optional outputs: states entering the next block, device fp32 [N][d].
+ * xF_next = z + W h (teacher, never patched); xC_next = z' + (W + dW) h' (patched student). */
+typedef struct pkv_ref_next {
+    float* xF_next;
+    float* xC_next;
+} pkv_ref_next;
+
+/* Scalars of one build (host). */
+typedef struct pkv_stats {
+    double lambda_eff;   /* ridge coefficient actually added to the diagonal */
+    double trace;        /* tr(S_H) */
+    double fro2;         /* ||S_H||_F^2 */
+    double target_fro2;  /* ||T||_F^2 */
+    double resid_fro2;   /* ||T - H' dW^T||_F^2 (only when next states were requested) */
+    double dW_fro2;      /* ||dW||_F^2 */
+    double min_pivot;    /* smallest Cholesky pivot (squared diagonal of the factor) */
+    int32_t err_info[2]; /* BAD_INDEX: (head, position); NOT_PD: (column, 0); TIMEOUT: (site, 0) */
+    float stage_ms[12];  /* per-stage device time when timing is enabled with pkv_set_timing */
+} pkv_stats;
+
+typedef struct pkv_ctx pkv_ctx;
+
+/* Device bytes a context of these dims needs (Algorithm 1 keeps only one chunk's activations
+ * and the running statistics; here: one call's activations, S_H, S_T, the factor). */
+size_t pkv_workspace_bytes(const pkv_dims* dims, const pkv_opts* opts);
+
+/* Create a context on the current device.  cuda_stream is a cudaStream_t (NULL = default). */
+int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* opts, void* cuda_stream);
+void pkv_destroy(pkv_ctx* ctx);
+
+/* One block of Algorithm 1 (Eq. 4-9): teacher forward with `full`, student forward with `cb`,
+ * targets, statistics, ridge solve.  dW: device fp32 [d][F] out.  next, stats: optional (NULL). */
+int pkv_build_patch(pkv_ctx* ctx, const pkv_block_weights* w, const pkv_kv* full,
+                    const pkv_kv_compressed* cb, const pkv_ref* ref, float lambda, int lambda_mode,
+                    float* dW, const pkv_ref_next* next, pkv_stats* stats);
+
+/* Algorithm 1, Merge: W[i] <- W[i] + dW[i] for the d*F entries, the sum taken in fp32 and
+ * rounded once to W's type (w_dtype = PKV_BF16 | PKV_FP32).  Asynchronous on cuda_stream. */
+int pkv_merge(void* W, int w_dtype, const float* dW, int64_t count, void* cuda_stream);
+
+/* Algorithm 1, outer loop: blocks first_layer..n_layers-1 in sequence, each solved with the
+ * blocks below it already patched in the student (greedy construction, Sec. 2.2).  Arrays are
+ * HOST arrays of n_layers entries.  x0F/x0C enter block first_layer; states are carried in
+ * fp32 inside the context.  dW[l]: device fp32 [d][F].  stats: NULL or n_layers entries.
+ * final: optional states leaving the last block. */
+int pkv_build_stack(pkv_ctx* ctx, int n_layers, int first_layer, const pkv_block_weights* w,
+                    const pkv_kv* full, const pkv_kv_compressed* cb, const pkv_ref* ref0,
+                    float lambda, int lambda_mode, float* const* dW, const pkv_ref_next* final,
+                    pkv_stats* stats);
+
+/* ---- single stages, exported for unit parity tests and per-kernel measurement ---- */
+
+/* Index check + compaction of a kept-index set (bit-exact): Kc[i] = K[h][idx[i]], same for V.
+ * Kc, Vc: device [head_off[Hkv]][hd] out.  Returns PKV_ERR_BAD_INDEX without touching memory
+ * outside the arrays when the set is invalid; bad_head/bad_pos (host, optional) get the first
+ * offender. */
+int pkv_gather_kept(pkv_ctx* ctx, const pkv_kv* full, const int32_t* head_off_host,
+                    const int32_t* idx, void* Kc, void* Vc, int32_t* bad_head, int32_t* bad_pos);
+
+/* Dual-cache attention alone (Sec. 2.2, teacher and student forward passes over the reference
+ * tokens).  q: device fp32 [2][N][Hq*hd] rotated queries of the teacher (0) and student (1)
+ * stream; k_new, v_new: device fp32 [2][N][Hkv*hd] the reference tokens' own keys/values.
+ * Outputs device fp32 [N][Hq*hd]: aF, aC and dA = aF - aC (formed before any rounding). */
+int pkv_attention(pkv_ctx* ctx, const float* q, const float* k_new, const float* v_new,
+                  const pkv_kv* full, const pkv_kv_compressed* cb, int32_t N, int32_t n_chunks,
+                  const int32_t* chunk_off, float* aF, float* aC, float* dA);
+
+/* Sufficient statistics alone (Eq. 9): S_H (+)= X^T X, S_T (+)= R^T X for X [n][F], R [n][d]
+ * device fp32; S_H [F][F], S_T [d][F] device fp32; accumulate != 0 adds to the running sums. */
+int pkv_gram(pkv_ctx* ctx, const float* X, const float* R, int32_t n, float* S_H, float* S_T,
+             int accumulate);
+
+/* Ridge solve alone (Eq. 7-8): dW = S_T (S_H + lambda I)^{-1}.  S_H, S_T are read, not
+ * modified. */
+int pkv_ridge_solve(pkv_ctx* ctx, const float* S_H, const float* S_T, float lambda, int lambda_mode,
+                    float* dW, pkv_stats* stats);
+
+/* Enable (1) / disable (0) per-stage CUDA-event timing into pkv_stats.stage_ms. */
+int pkv_set_timing(pkv_ctx* ctx, int on);
+
+/* Number of kernels the context launched since creation (for launch accounting). */
+int64_t pkv_launch_count(const pkv_ctx* ctx);
+
+const char* pkv_strerror(int code);
+const char* pkv_last_cuda_error(const pkv_ctx* ctx);
+const char* pkv_stage_name(int stage);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PKV_H_ */

@@ -1,0 +1,652 @@
+// C ABI of libpkv.so: context, workspace carving, argument validation and the per-block stage
+// sequence of Algorithm 1 (teacher/student forward, targets, statistics, ridge solve, next
+// states).  All arithmetic happens in the kernels of the other translation units.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "pkv_internal.h"
+#include "pkv_tc.h"
+
+using namespace pkv;
+
+enum Stage { ST_INDEX = 0, ST_QKV, ST_ATTN, ST_OPROJ, ST_MLP, ST_TARGET, ST_GRAM, ST_SOLVE, ST_NEXT, ST_COUNT };
+static const char* kStageNames[ST_COUNT] = {"S0 index check + compaction", "S1-S2 norm + QKV + RoPE",
+                                            "S3 dual-cache attention",     "S4 o-proj + residual",
+                                            "S5 norm + gate/up + SiLU",    "S6 targets",
+                                            "S7 Gram + cross statistics",  "S8 ridge solve",
+                                            "S9 next states"};
+
+struct Carver {
+    char* base;
+    size_t off;
+    template <typename T>
+    T* take(size_t n) {
+        off = (off + 255) & ~(size_t)255;
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+struct Buffers {
+    DevStatus* status;
+    int32_t* head_off;
+    int32_t* tok_cs;
+    float* rope_tab;
+    void* Kc;
+    void* Vc;
+    float* u;       // [2N][d]
+    float* qkv;     // [2N][Dq+2Dkv]
+    float* part_m;
+    float* part_l;
+    float* part_O;
+    float* a2;      // [2N][Dq]: aF rows then dA rows
+    float* aC;      // [N][Dq]
+    float* o;       // [2N][d]
+    float* zF;
+    float* zC;
+    float* dz;
+    float* gu;      // [2N][2F]
+    float* hF;
+    float* hC;
+    float* dh;
+    float* R;       // [N][d]
+    float* XT;      // [F][N]
+    float* RT;      // [d][N]
+    float* S_H;
+    float* S_T;
+    SolveWs solve;
+    float* D;       // [N][d]
+    float* xs[4];   // stack states, ping-pong: xF a/b, xC a/b
+    pkv::TcBuffers tc;
+};
+
+struct pkv_ctx {
+    pkv_dims dims;
+    pkv_opts opts;
+    cudaStream_t st;
+    int engine;
+    int elem_bytes;
+    int kv_split, cap_splitF, cap_splitC;
+    int sm_count;
+    char* ws;
+    bool own_ws;
+    size_t ws_bytes;
+    Buffers b;
+    int32_t* host_stage;     // pinned: head_off + tok_cs
+    DevStatus* host_status;  // pinned
+    int64_t launches;
+    int timing;
+    cudaEvent_t ev[ST_COUNT + 1];
+    char cuda_err[256];
+};
+
+static int choose_engine(const pkv_dims* d, const pkv_opts* o) {
+    if (o && o->engine == PKV_ENGINE_SIMT) return PKV_ENGINE_SIMT;
+    return (d->dtype == PKV_BF16) ? PKV_ENGINE_AUTO : PKV_ENGINE_SIMT;
+}
+
+static void split_plan(const pkv_dims* d, const pkv_opts* o, int sm_count, int* kv_split, int* capF, int* capC) {
+    int g = d->Hq / d->Hkv;
+    long long rows = (long long)d->N_max * g;
+    long long qtiles = (rows + 31) / 32;
+    long long Lt = (long long)d->L + d->N_max;
+    int ks = o ? o->kv_split : 0;
+    if (ks <= 0) {
+        long long want = (4LL * sm_count + qtiles * d->Hkv - 1) / (qtiles * d->Hkv);
+        if (want < 1) want = 1;
+        if (want > 64) want = 64;
+        long long per = (Lt + want - 1) / want;
+        per = ((per + 63) / 64) * 64;
+        if (per < 256) per = 256;
+        ks = (int)per;
+    }
+    ks = ((ks + 31) / 32) * 32;
+    *kv_split = ks;
+    *capF = (int)((Lt + ks - 1) / ks);
+    long long Ls = (long long)d->b_max + d->N_max;
+    *capC = (int)((Ls + ks - 1) / ks);
+    if (*capC < 1) *capC = 1;
+}
+
+static size_t carve(Buffers* b, char* base, const pkv_dims* d, int engine, int elem_bytes, int capF, int capC) {
+    Carver c{base, 0};
+    const size_t N = d->N_max, dm = d->d, F = d->F, Dq = (size_t)d->Hq * d->hd, Dkv = (size_t)d->Hkv * d->hd;
+    const size_t g = d->Hq / d->Hkv, rows = N * g;
+    const size_t tot_kept = (size_t)d->Hkv * d->b_max;
+    b->status = c.take<DevStatus>(1);
+    b->head_off = c.take<int32_t>(d->Hkv + 1);
+    b->tok_cs = c.take<int32_t>(N);
+    b->rope_tab = c.take<float>(N * d->hd);
+    b->Kc = c.take<char>(tot_kept * d->hd * elem_bytes + 256);
+    b->Vc = c.take<char>(tot_kept * d->hd * elem_bytes + 256);
+    b->u = c.take<float>(2 * N * dm);
+    b->qkv = c.take<float>(2 * N * (Dq + 2 * Dkv));
+    size_t nsp = (size_t)capF + capC;
+    b->part_m = c.take<float>(nsp * d->Hkv * rows);
+    b->part_l = c.take<float>(nsp * d->Hkv * rows);
+    b->part_O = c.take<float>(nsp * d->Hkv * rows * d->hd);
+    b->a2 = c.take<float>(2 * N * Dq);
+    b->aC = c.take<float>(N * Dq);
+    b->o = c.take<float>(2 * N * dm);
+    b->zF = c.take<float>(N * dm);
+    b->zC = c.take<float>(N * dm);
+    b->dz = c.take<float>(N * dm);
+    b->gu = c.take<float>(2 * N * 2 * F);
+    b->hF = c.take<float>(N * F);
+    b->hC = c.take<float>(N * F);
+    b->dh = c.take<float>(N * F);
+    b->R = c.take<float>(N * dm);
+    b->XT = c.take<float>(F * N);
+    b->RT = c.take<float>(dm * N);
+    b->S_H = c.take<float>(F * F);
+    b->S_T = c.take<float>(dm * F);
+    size_t nblk = (F + kSolveNb - 1) / kSolveNb;
+    b->solve.G = c.take<float>(F * F);
+    b->solve.Lm = c.take<float>(F * F);
+    b->solve.LT = c.take<float>(F * F);
+    b->solve.inv = c.take<float>(nblk * kSolveNb * kSolveNb);
+    b->solve.invT = c.take<float>(nblk * kSolveNb * kSolveNb);
+    b->solve.Y = c.take<float>(dm * F);
+    b->D = c.take<float>(N * dm);
+    for (int i = 0; i < 4; ++i) b->xs[i] = c.take<float>(N * dm);
+    if (engine != PKV_ENGINE_SIMT) c.off = pkv::tc_carve(&b->tc, base, c.off, d);
+    return (c.off + 255) & ~(size_t)255;
+}
+
+static int dims_ok(const pkv_dims* d) {
+    if (!d) return PKV_ERR_INVALID_ARG;
+    if (d->d <= 0 || d->Hq <= 0 || d->Hkv <= 0 || d->F <= 0 || d->L < 0 || d->N_max <= 0 || d->b_max < 0)
+        return PKV_ERR_INVALID_ARG;
+    if (d->dtype != PKV_BF16 && d->dtype != PKV_FP32) return PKV_ERR_INVALID_ARG;
+    if (!(d->eps >= 0.f) || !(d->rope_theta >= 0.f)) return PKV_ERR_INVALID_ARG;
+    if (d->hd != 64 && d->hd != 128) return PKV_ERR_UNSUPPORTED;
+    if (d->Hq % d->Hkv != 0) return PKV_ERR_UNSUPPORTED;
+    if (d->F > 8192) return PKV_ERR_UNSUPPORTED;
+    if ((long long)d->L + d->N_max > (1LL << 30)) return PKV_ERR_UNSUPPORTED;
+    return PKV_OK;
+}
+
+extern "C" size_t pkv_workspace_bytes(const pkv_dims* dims, const pkv_opts* opts) {
+    if (dims_ok(dims) != PKV_OK) return 0;
+    int ks, cf, cc;
+    split_plan(dims, opts, 148, &ks, &cf, &cc);
+    Buffers b;
+    int engine = choose_engine(dims, opts);
+    return carve(&b, nullptr, dims, engine, dims->dtype == PKV_BF16 ? 2 : 4, cf, cc);
+}
+
+extern "C" int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* opts, void* cuda_stream) {
+    if (!out) return PKV_ERR_INVALID_ARG;
+    *out = nullptr;
+    int rc = dims_ok(dims);
+    if (rc != PKV_OK) return rc;
+    pkv_ctx* c = new (std::nothrow) pkv_ctx();
+    if (!c) return PKV_ERR_NOMEM;
+    memset(c, 0, sizeof(*c));
+    c->dims = *dims;
+    if (opts) c->opts = *opts;
+    c->st = (cudaStream_t)cuda_stream;
+    c->engine = choose_engine(dims, opts);
+    c->elem_bytes = dims->dtype == PKV_BF16 ? 2 : 4;
+    int dev = 0;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        delete c;
+        return PKV_ERR_CUDA;
+    }
+    c->sm_count = prop.multiProcessorCount;
+    if (c->engine != PKV_ENGINE_SIMT) {
+        rc = pkv::tc_supported(dims, prop.major, prop.minor);
+        if (rc != PKV_OK) {
+            delete c;
+            return rc;
+        }
+    }
+    // the split plan uses 148 SMs so that pkv_workspace_bytes (no device needed) agrees with it
+    split_plan(dims, opts, 148, &c->kv_split, &c->cap_splitF, &c->cap_splitC);
+    size_t need = carve(&c->b, nullptr, dims, c->engine, c->elem_bytes, c->cap_splitF, c->cap_splitC);
+    c->ws_bytes = need;
+    if (opts && opts->workspace) {
+        if (opts->workspace_bytes < need || ((uintptr_t)opts->workspace & 255)) {
+            delete c;
+            return PKV_ERR_NOMEM;
+        }
+        c->ws = (char*)opts->workspace;
+        c->own_ws = false;
+    } else {
+        if (cudaMalloc((void**)&c->ws, need) != cudaSuccess) {
+            cudaGetLastError();
+            delete c;
+            return PKV_ERR_NOMEM;
+        }
+        c->own_ws = true;
+    }
+    carve(&c->b, c->ws, dims, c->engine, c->elem_bytes, c->cap_splitF, c->cap_splitC);
+    size_t stage_ints = (size_t)dims->Hkv + 1 + dims->N_max;
+    if (cudaMallocHost((void**)&c->host_stage, stage_ints * sizeof(int32_t)) != cudaSuccess ||
+        cudaMallocHost((void**)&c->host_status, sizeof(DevStatus)) != cudaSuccess) {
+        cudaGetLastError();
+        pkv_destroy(c);
+        return PKV_ERR_NOMEM;
+    }
+    for (int i = 0; i <= ST_COUNT; ++i) cudaEventCreate(&c->ev[i]);
+    if (c->engine != PKV_ENGINE_SIMT) {
+        rc = pkv::tc_init(&c->b.tc, dims);
+        if (rc != PKV_OK) {
+            pkv_destroy(c);
+            return rc;
+        }
+    }
+    *out = c;
+    return PKV_OK;
+}
+
+extern "C" void pkv_destroy(pkv_ctx* c) {
+    if (!c) return;
+    cudaStreamSynchronize(c->st);
+    if (c->own_ws && c->ws) cudaFree(c->ws);
+    if (c->host_stage) cudaFreeHost(c->host_stage);
+    if (c->host_status) cudaFreeHost(c->host_status);
+    for (int i = 0; i <= ST_COUNT; ++i)
+        if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    delete c;
+}
+
+extern "C" int pkv_set_timing(pkv_ctx* c, int on) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    c->timing = on ? 1 : 0;
+    return PKV_OK;
+}
+
+extern "C" int64_t pkv_launch_count(const pkv_ctx* c) { return c ? c->launches : 0; }
+
+extern "C" const char* pkv_strerror(int code) {
+    switch (code) {
+        case PKV_OK: return "ok";
+        case PKV_ERR_INVALID_ARG: return "invalid argument";
+        case PKV_ERR_UNSUPPORTED: return "unsupported shape or device";
+        case PKV_ERR_BAD_INDEX: return "kept-index set is not strictly ascending within [0, L)";
+        case PKV_ERR_NOT_PD: return "ridge matrix is not positive definite in fp32";
+        case PKV_ERR_DEGENERATE: return "tr(S_H) = 0: adaptive ridge scale undefined";
+        case PKV_ERR_NONFINITE: return "non-finite value in the statistics";
+        case PKV_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case PKV_ERR_CUDA: return "CUDA runtime error";
+        case PKV_ERR_NOMEM: return "workspace allocation failed or too small";
+        default: return "unknown error";
+    }
+}
+
+extern "C" const char* pkv_last_cuda_error(const pkv_ctx* c) { return c ? c->cuda_err : ""; }
+extern "C" const char* pkv_stage_name(int s) { return (s >= 0 && s < ST_COUNT) ? kStageNames[s] : ""; }
+
+// ---------------------------------------------------------------------------------------------
+
+static int cuda_fail(pkv_ctx* c, cudaError_t e, const char* where) {
+    snprintf(c->cuda_err, sizeof(c->cuda_err), "%s: %s", where, cudaGetErrorString(e));
+    return PKV_ERR_CUDA;
+}
+
+static void mark(pkv_ctx* c, int i) {
+    if (c->timing) cudaEventRecord(c->ev[i], c->st);
+}
+
+static int check_compressed(const pkv_ctx* c, const pkv_kv_compressed* cb, int* total, int* max_b) {
+    if (!cb || !cb->head_off) return PKV_ERR_INVALID_ARG;
+    const int Hkv = c->dims.Hkv;
+    if (cb->head_off[0] != 0) return PKV_ERR_INVALID_ARG;
+    int mb = 0;
+    for (int h = 0; h < Hkv; ++h) {
+        int bh = cb->head_off[h + 1] - cb->head_off[h];
+        if (bh < 0 || bh > c->dims.b_max) return PKV_ERR_INVALID_ARG;
+        if (bh > mb) mb = bh;
+    }
+    *total = cb->head_off[Hkv];
+    *max_b = mb;
+    if (*total > 0) {
+        if (cb->idx) {
+            if ((uintptr_t)cb->idx & 3) return PKV_ERR_INVALID_ARG;
+        } else {
+            if (!cb->Kc || !cb->Vc) return PKV_ERR_INVALID_ARG;
+            if (((uintptr_t)cb->Kc & 15) || ((uintptr_t)cb->Vc & 15)) return PKV_ERR_INVALID_ARG;
+        }
+    }
+    return PKV_OK;
+}
+
+static int check_chunks(const pkv_ctx* c, int N, int n_chunks, const int32_t* chunk_off) {
+    if (N <= 0 || N > c->dims.N_max || n_chunks <= 0 || !chunk_off) return PKV_ERR_INVALID_ARG;
+    if (chunk_off[0] != 0 || chunk_off[n_chunks] != N) return PKV_ERR_INVALID_ARG;
+    for (int i = 0; i < n_chunks; ++i)
+        if (chunk_off[i + 1] <= chunk_off[i]) return PKV_ERR_INVALID_ARG;
+    return PKV_OK;
+}
+
+// uploads head_off and the per-token chunk starts
+static void upload_meta(pkv_ctx* c, const int32_t* head_off, int N, int n_chunks, const int32_t* chunk_off) {
+    const int Hkv = c->dims.Hkv;
+    int32_t* hs = c->host_stage;
+    for (int h = 0; h <= Hkv; ++h) hs[h] = head_off ? head_off[h] : 0;
+    int32_t* cs = hs + Hkv + 1;
+    for (int ch = 0; ch < n_chunks; ++ch)
+        for (int i = chunk_off[ch]; i < chunk_off[ch + 1]; ++i) cs[i] = chunk_off[ch];
+    cudaMemcpyAsync(c->b.head_off, hs, (Hkv + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, c->st);
+    if (N > 0) cudaMemcpyAsync(c->b.tok_cs, cs, (size_t)N * sizeof(int32_t), cudaMemcpyHostToDevice, c->st);
+}
+
+static void begin_call(pkv_ctx* c) {
+    cudaMemsetAsync(c->b.status, 0, sizeof(DevStatus), c->st);
+}
+
+// reads the status word; fills stats; returns the call's code
+static int end_call(pkv_ctx* c, pkv_stats* stats, const int32_t* head_off) {
+    cudaError_t e = cudaMemcpyAsync(c->host_status, c->b.status, sizeof(DevStatus), cudaMemcpyDeviceToHost, c->st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "status copy");
+    e = cudaStreamSynchronize(c->st);
+    if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronize");
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(c, e, "kernel launch");
+    const DevStatus& s = *c->host_status;
+    if (stats) {
+        stats->lambda_eff = s.lam;
+        stats->trace = s.tr;
+        stats->fro2 = s.fro2;
+        stats->target_fro2 = s.t_fro2;
+        stats->resid_fro2 = s.res_fro2;
+        stats->dW_fro2 = s.dw_fro2;
+        stats->min_pivot = s.min_pivot;
+        stats->err_info[0] = stats->err_info[1] = 0;
+        if (s.code == PKV_ERR_BAD_INDEX && s.bad_index && head_off) {
+            int pos = (int)(s.bad_index - 1), h = 0;
+            while (h + 1 < c->dims.Hkv && head_off[h + 1] <= pos) ++h;
+            stats->err_info[0] = h;
+            stats->err_info[1] = pos - head_off[h];
+        } else if (s.code == PKV_ERR_NOT_PD && s.bad_column) {
+            stats->err_info[0] = (int)(s.bad_column - 1);
+        } else if (s.code == PKV_ERR_TIMEOUT) {
+            stats->err_info[0] = s.info0;
+            stats->err_info[1] = s.info1;
+        }
+        for (int i = 0; i < 12; ++i) stats->stage_ms[i] = 0.f;
+        if (c->timing)
+            for (int i = 0; i < ST_COUNT; ++i) cudaEventElapsedTime(&stats->stage_ms[i], c->ev[i], c->ev[i + 1]);
+    }
+    return s.code;
+}
+
+static AttnArgs attn_args(pkv_ctx* c, const float* q, int64_t ldq, const float* k_new, const float* v_new,
+                          int64_t ldkv, const pkv_kv* full, const void* Kc, const void* Vc, const float* bias,
+                          int N, int max_b) {
+    AttnArgs a;
+    memset(&a, 0, sizeof(a));
+    a.q = q; a.ldq = ldq; a.k_new = k_new; a.v_new = v_new; a.ldkv = ldkv;
+    a.K = full->K; a.V = full->V; a.Kc = Kc; a.Vc = Vc; a.bias = bias;
+    a.head_off = c->b.head_off; a.tok_cs = c->b.tok_cs;
+    a.N = N; a.Hq = c->dims.Hq; a.Hkv = c->dims.Hkv; a.hd = c->dims.hd; a.L = c->dims.L;
+    a.elem_bytes = c->elem_bytes;
+    a.kv_split = c->kv_split;
+    a.nsplitF = (c->dims.L + N + c->kv_split - 1) / c->kv_split;
+    a.nsplitC = (max_b + N + c->kv_split - 1) / c->kv_split;
+    if (a.nsplitC < 1) a.nsplitC = 1;
+    a.part_m = c->b.part_m; a.part_l = c->b.part_l; a.part_O = c->b.part_O;
+    return a;
+}
+
+// S0: returns the compact cache pointers to use
+static void stage_compact(pkv_ctx* c, const Lc& lc, const pkv_kv* full, const pkv_kv_compressed* cb, int total,
+                          const void** Kc, const void** Vc) {
+    if (cb->idx && total > 0) {
+        gather_kept(lc, c->elem_bytes, full->K, full->V, cb->idx, c->b.head_off, c->dims.Hkv, c->dims.L, c->dims.hd,
+                    total, c->b.Kc, c->b.Vc, c->b.status);
+        *Kc = c->b.Kc;
+        *Vc = c->b.Vc;
+    } else {
+        *Kc = cb->Kc ? cb->Kc : c->b.Kc;
+        *Vc = cb->Vc ? cb->Vc : c->b.Vc;
+    }
+}
+
+// Statistics from X [n][F], R [n][d] (Eq. 9), SIMT path.
+static void gram_simt(pkv_ctx* c, const Lc& lc, const float* X, const float* R, int n, float* S_H, float* S_T,
+                      bool accumulate) {
+    const int F = c->dims.F, d = c->dims.d;
+    transpose_f32(lc, X, n, F, c->b.XT);
+    transpose_f32(lc, R, n, d, c->b.RT);
+    gemm_tn_simt(lc, c->b.XT, n, c->b.XT, n, false, S_H, F, F, F, n, 1.f, nullptr, 0, accumulate);
+    gemm_tn_simt(lc, c->b.RT, n, c->b.XT, n, false, S_T, F, d, F, n, 1.f, nullptr, 0, accumulate);
+}
+
+static void solve_stage(pkv_ctx* c, const Lc& lc, const float* S_H, const float* S_T, float lam0, int mode,
+                        float* dW) {
+    const int F = c->dims.F, d = c->dims.d;
+    Buffers& b = c->b;
+    trace_fro2(lc, S_H, F, b.status);
+    make_ridge_matrix(lc, S_H, F, lam0, mode, b.solve.G, b.status);
+    cudaMemcpyAsync(b.solve.Y, S_T, (size_t)d * F * sizeof(float), cudaMemcpyDeviceToDevice, c->st);
+    if (c->engine == PKV_ENGINE_SIMT)
+        ridge_solve_simt(lc, b.solve, F, d, dW, b.status);
+    else
+        pkv::tc_ridge_solve(lc, &b.tc, b.solve, F, d, dW, b.status);
+    sumsq(lc, dW, (int64_t)d * F, &b.status->dw_fro2);
+}
+
+static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv* full,
+                            const pkv_kv_compressed* cb, const pkv_ref* ref, float lambda, int mode, float* dW,
+                            const pkv_ref_next* next, pkv_stats* stats) {
+    if (!c || !w || !full || !cb || !ref || !dW) return PKV_ERR_INVALID_ARG;
+    if (!w->g_attn || !w->Wq || !w->Wk || !w->Wv || !w->Wo || !w->g_mlp || !w->Wgate || !w->Wup || !w->Wdown)
+        return PKV_ERR_INVALID_ARG;
+    if (c->dims.L > 0 && (!full->K || !full->V)) return PKV_ERR_INVALID_ARG;
+    if (!ref->xF || !ref->xC) return PKV_ERR_INVALID_ARG;
+    if (!(lambda > 0.f) || !isfinite(lambda)) return PKV_ERR_INVALID_ARG;
+    if (mode != PKV_LAMBDA_PAPER && mode != PKV_LAMBDA_ABSOLUTE && mode != PKV_LAMBDA_TRACE_MEAN)
+        return PKV_ERR_INVALID_ARG;
+    const void* ptrs[] = {w->Wq, w->Wk, w->Wv, w->Wo, w->Wgate, w->Wup, w->Wdown, full->K, full->V,
+                          ref->xF, ref->xC, dW, w->g_attn, w->g_mlp};
+    for (const void* p : ptrs)
+        if ((uintptr_t)p & 15) return PKV_ERR_INVALID_ARG;
+    if (next && (!next->xF_next || !next->xC_next)) return PKV_ERR_INVALID_ARG;
+    int rc = check_chunks(c, ref->N, ref->n_chunks, ref->chunk_off);
+    if (rc != PKV_OK) return rc;
+    int total = 0, max_b = 0;
+    rc = check_compressed(c, cb, &total, &max_b);
+    if (rc != PKV_OK) return rc;
+
+    const pkv_dims& D = c->dims;
+    const int N = ref->N, d = D.d, F = D.F, hd = D.hd;
+    const int Dq = D.Hq * hd, Dkv = D.Hkv * hd, QKV = Dq + 2 * Dkv;
+    const bool bf = D.dtype == PKV_BF16;
+    Buffers& b = c->b;
+    Lc lc{c->st, &c->launches};
+
+    begin_call(c);
+    upload_meta(c, cb->head_off, N, ref->n_chunks, ref->chunk_off);
+    mark(c, ST_INDEX);
+    const void *Kc, *Vc;
+    stage_compact(c, lc, full, cb, total, &Kc, &Vc);
+    mark(c, ST_QKV);
+
+    if (c->engine == PKV_ENGINE_SIMT) {
+        // S1-S2: both streams stacked, rows [0,N) teacher, [N,2N) student
+        rmsnorm_f32(lc, ref->xF, ref->xC, N, d, w->g_attn, D.eps, b.u);
+        gemm_tn_simt(lc, b.u, d, w->Wq, d, bf, b.qkv, QKV, 2 * N, Dq, d, 1.f, nullptr, 0, false);
+        gemm_tn_simt(lc, b.u, d, w->Wk, d, bf, b.qkv + Dq, QKV, 2 * N, Dkv, d, 1.f, nullptr, 0, false);
+        gemm_tn_simt(lc, b.u, d, w->Wv, d, bf, b.qkv + Dq + Dkv, QKV, 2 * N, Dkv, d, 1.f, nullptr, 0, false);
+        rope_table(lc, b.tok_cs, N, hd, ref->pos0, D.rope_theta, b.rope_tab);
+        rope_apply(lc, b.qkv, QKV, 0, D.Hq + D.Hkv, hd, 2 * N, N, b.rope_tab);
+        mark(c, ST_ATTN);
+        // S3
+        AttnArgs a = attn_args(c, b.qkv, QKV, b.qkv + Dq, b.qkv + Dq + Dkv, QKV, full, Kc, Vc,
+                               cb->idx ? nullptr : cb->bias, N, max_b);
+        a.aF = b.a2; a.aC = b.aC; a.dA = b.a2 + (size_t)N * Dq;
+        attention_simt(lc, a);
+        attention_combine(lc, a);
+        mark(c, ST_OPROJ);
+        // S4: [aF; dA] Wo^T, then zF, dz, zC
+        gemm_tn_simt(lc, b.a2, Dq, w->Wo, Dq, bf, b.o, d, 2 * N, d, Dq, 1.f, nullptr, 0, false);
+        oproj_epilogue(lc, ref->xF, ref->xC, b.o, N, d, b.zF, b.zC, b.dz);
+        mark(c, ST_MLP);
+        // S5
+        rmsnorm_f32(lc, b.zF, b.zC, N, d, w->g_mlp, D.eps, b.u);
+        gemm_tn_simt(lc, b.u, d, w->Wgate, d, bf, b.gu, 2 * F, 2 * N, F, d, 1.f, nullptr, 0, false);
+        gemm_tn_simt(lc, b.u, d, w->Wup, d, bf, b.gu + F, 2 * F, 2 * N, F, d, 1.f, nullptr, 0, false);
+        swiglu(lc, b.gu, N, F, b.hF, b.hC, b.dh);
+        mark(c, ST_TARGET);
+        // S6: R = dh Wdown^T + dz   (Eq. 5)
+        gemm_tn_simt(lc, b.dh, F, w->Wdown, F, bf, b.R, d, N, d, F, 1.f, b.dz, d, false);
+        sumsq(lc, b.R, (int64_t)N * d, &b.status->t_fro2);
+        mark(c, ST_GRAM);
+        // S7 (Eq. 9)
+        gram_simt(c, lc, b.hC, b.R, N, b.S_H, b.S_T, false);
+        mark(c, ST_SOLVE);
+    } else {
+        pkv::TcForwardArgs fa;
+        fa.w = w; fa.full = full; fa.Kc = Kc; fa.Vc = Vc; fa.bias = cb->idx ? nullptr : cb->bias;
+        fa.xF = ref->xF; fa.xC = ref->xC; fa.N = N; fa.pos0 = ref->pos0; fa.max_b = max_b;
+        fa.head_off = b.head_off; fa.tok_cs = b.tok_cs; fa.rope_tab = b.rope_tab;
+        fa.zF = b.zF; fa.zC = b.zC; fa.dz = b.dz; fa.hF = b.hF; fa.hC = b.hC; fa.R = b.R;
+        fa.S_H = b.S_H; fa.S_T = b.S_T; fa.status = b.status;
+        fa.aF = b.a2; fa.aC = b.aC;
+        fa.kv_split = c->kv_split;
+        fa.part_m = b.part_m; fa.part_l = b.part_l; fa.part_O = b.part_O;
+        fa.ev = c->timing ? c->ev : nullptr;
+        rc = pkv::tc_forward(lc, &b.tc, &c->dims, fa);
+        if (rc != PKV_OK) return rc;
+    }
+    // S8 (Eq. 7-8)
+    solve_stage(c, lc, b.S_H, b.S_T, lambda, mode, dW);
+    mark(c, ST_NEXT);
+    // S9: xF_next = zF + hF W^T;  D = R - hC dW^T;  xC_next = xF_next - D
+    if (next) {
+        if (c->engine == PKV_ENGINE_SIMT) {
+            gemm_tn_simt(lc, b.hF, F, w->Wdown, F, bf, next->xF_next, d, N, d, F, 1.f, b.zF, d, false);
+            gemm_tn_simt(lc, b.hC, F, dW, F, false, b.D, d, N, d, F, -1.f, b.R, d, false);
+        } else {
+            pkv::tc_next_states(lc, &b.tc, &c->dims, N, w->Wdown, dW, b.zF, b.R, next->xF_next, b.D);
+        }
+        sumsq(lc, b.D, (int64_t)N * d, &b.status->res_fro2);
+        sub_f32(lc, next->xF_next, b.D, (int64_t)N * d, next->xC_next);
+    }
+    mark(c, ST_COUNT);
+    return end_call(c, stats, cb->head_off);
+}
+
+extern "C" int pkv_build_patch(pkv_ctx* ctx, const pkv_block_weights* w, const pkv_kv* full,
+                               const pkv_kv_compressed* cb, const pkv_ref* ref, float lambda, int lambda_mode,
+                               float* dW, const pkv_ref_next* next, pkv_stats* stats) {
+    return build_patch_impl(ctx, w, full, cb, ref, lambda, lambda_mode, dW, next, stats);
+}
+
+extern "C" int pkv_merge(void* W, int w_dtype, const float* dW, int64_t count, void* cuda_stream) {
+    if (!W || !dW || count < 0) return PKV_ERR_INVALID_ARG;
+    if (w_dtype != PKV_BF16 && w_dtype != PKV_FP32) return PKV_ERR_INVALID_ARG;
+    if (((uintptr_t)W & 15) || ((uintptr_t)dW & 15)) return PKV_ERR_INVALID_ARG;
+    Lc lc{(cudaStream_t)cuda_stream, nullptr};
+    merge_weights(lc, W, w_dtype, dW, count);
+    return cudaGetLastError() == cudaSuccess ? PKV_OK : PKV_ERR_CUDA;
+}
+
+extern "C" int pkv_build_stack(pkv_ctx* c, int n_layers, int first_layer, const pkv_block_weights* w,
+                               const pkv_kv* full, const pkv_kv_compressed* cb, const pkv_ref* ref0, float lambda,
+                               int lambda_mode, float* const* dW, const pkv_ref_next* final, pkv_stats* stats) {
+    if (!c || !w || !full || !cb || !ref0 || !dW || n_layers <= 0 || first_layer < 0 || first_layer >= n_layers)
+        return PKV_ERR_INVALID_ARG;
+    pkv_ref ref = *ref0;
+    for (int l = first_layer; l < n_layers; ++l) {
+        int pp = (l - first_layer) & 1;
+        pkv_ref_next nx;
+        bool last = (l == n_layers - 1);
+        if (last && final) {
+            nx = *final;
+        } else {
+            nx.xF_next = c->b.xs[pp];
+            nx.xC_next = c->b.xs[2 + pp];
+        }
+        const pkv_ref_next* pnx = (last && !final) ? nullptr : &nx;
+        int rc = build_patch_impl(c, &w[l], &full[l], &cb[l], &ref, lambda, lambda_mode, dW[l], pnx,
+                                  stats ? &stats[l] : nullptr);
+        if (rc != PKV_OK) return rc;
+        ref.xF = nx.xF_next;
+        ref.xC = nx.xC_next;
+    }
+    return PKV_OK;
+}
+
+// ---- single stages ------------------------------------------------------------------------------
+
+extern "C" int pkv_gather_kept(pkv_ctx* c, const pkv_kv* full, const int32_t* head_off_host, const int32_t* idx,
+                               void* Kc, void* Vc, int32_t* bad_head, int32_t* bad_pos) {
+    if (!c || !full || !head_off_host) return PKV_ERR_INVALID_ARG;
+    pkv_kv_compressed cb{head_off_host, idx, nullptr, nullptr, nullptr};
+    int total = 0, max_b = 0;
+    int rc = check_compressed(c, &cb, &total, &max_b);
+    if (rc != PKV_OK) return rc;
+    if (total > 0 && (!idx || !Kc || !Vc || !full->K || !full->V)) return PKV_ERR_INVALID_ARG;
+    if (((uintptr_t)Kc & 15) || ((uintptr_t)Vc & 15)) return PKV_ERR_INVALID_ARG;
+    Lc lc{c->st, &c->launches};
+    begin_call(c);
+    int32_t one[2] = {0, 0};
+    upload_meta(c, head_off_host, 0, 0, one);
+    gather_kept(lc, c->elem_bytes, full->K, full->V, idx, c->b.head_off, c->dims.Hkv, c->dims.L, c->dims.hd, total,
+                Kc, Vc, c->b.status);
+    pkv_stats st;
+    rc = end_call(c, &st, head_off_host);
+    if (bad_head) *bad_head = st.err_info[0];
+    if (bad_pos) *bad_pos = st.err_info[1];
+    return rc;
+}
+
+extern "C" int pkv_attention(pkv_ctx* c, const float* q, const float* k_new, const float* v_new,
+                             const pkv_kv* full, const pkv_kv_compressed* cb, int32_t N, int32_t n_chunks,
+                             const int32_t* chunk_off, float* aF, float* aC, float* dA) {
+    if (!c || !q || !k_new || !v_new || !full || !cb || !aF || !aC || !dA) return PKV_ERR_INVALID_ARG;
+    int rc = check_chunks(c, N, n_chunks, chunk_off);
+    if (rc != PKV_OK) return rc;
+    int total = 0, max_b = 0;
+    rc = check_compressed(c, cb, &total, &max_b);
+    if (rc != PKV_OK) return rc;
+    const int Dq = c->dims.Hq * c->dims.hd, Dkv = c->dims.Hkv * c->dims.hd;
+    Lc lc{c->st, &c->launches};
+    begin_call(c);
+    upload_meta(c, cb->head_off, N, n_chunks, chunk_off);
+    const void *Kc, *Vc;
+    stage_compact(c, lc, full, cb, total, &Kc, &Vc);
+    AttnArgs a = attn_args(c, q, Dq, k_new, v_new, Dkv, full, Kc, Vc, cb->idx ? nullptr : cb->bias, N, max_b);
+    a.aF = aF; a.aC = aC; a.dA = dA;
+    if (c->engine == PKV_ENGINE_SIMT) {
+        attention_simt(lc, a);
+        attention_combine(lc, a);
+    } else {
+        rc = pkv::tc_attention(lc, &c->b.tc, &c->dims, a, c->b.status);
+        if (rc != PKV_OK) return rc;
+    }
+    return end_call(c, nullptr, cb->head_off);
+}
+
+extern "C" int pkv_gram(pkv_ctx* c, const float* X, const float* R, int32_t n, float* S_H, float* S_T,
+                        int accumulate) {
+    if (!c || !X || !R || !S_H || !S_T || n <= 0 || n > c->dims.N_max) return PKV_ERR_INVALID_ARG;
+    Lc lc{c->st, &c->launches};
+    begin_call(c);
+    if (c->engine == PKV_ENGINE_SIMT)
+        gram_simt(c, lc, X, R, n, S_H, S_T, accumulate != 0);
+    else
+        pkv::tc_gram(lc, &c->b.tc, &c->dims, X, R, n, S_H, S_T, accumulate != 0, c->b.status);
+    return end_call(c, nullptr, nullptr);
+}
+
+extern "C" int pkv_ridge_solve(pkv_ctx* c, const float* S_H, const float* S_T, float lambda, int lambda_mode,
+                               float* dW, pkv_stats* stats) {
+    if (!c || !S_H || !S_T || !dW) return PKV_ERR_INVALID_ARG;
+    if (!(lambda > 0.f) || !isfinite(lambda)) return PKV_ERR_INVALID_ARG;
+    if (lambda_mode != PKV_LAMBDA_PAPER && lambda_mode != PKV_LAMBDA_ABSOLUTE && lambda_mode != PKV_LAMBDA_TRACE_MEAN)
+        return PKV_ERR_INVALID_ARG;
+    Lc lc{c->st, &c->launches};
+    begin_call(c);
+    solve_stage(c, lc, S_H, S_T, lambda, lambda_mode, dW);
+    return end_call(c, stats, nullptr);
+}

@@ -1,0 +1,94 @@
+// Internal declarations shared by the translation units of libpkv.so.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pkv.h"
+
+namespace pkv {
+
+// Device-resident status and scalar results of one call (zeroed at the start of a call).
+struct DevStatus {
+    int code;                         // first pkv_error raised on the device (0 = none)
+    int info0, info1;                 // see pkv_stats.err_info
+    int pad;
+    unsigned long long bad_index;     // smallest flat position of an invalid kept index (+1), 0 = none
+    unsigned long long bad_column;    // smallest non-positive Cholesky pivot column (+1), 0 = none
+    double tr, fro2, t_fro2, res_fro2, dw_fro2;
+    float lam;
+    float min_pivot;
+};
+
+// Every launcher takes the stream and a launch counter.
+struct Lc {
+    cudaStream_t st;
+    int64_t* launches;
+    void count(int n = 1) const { if (launches) *launches += n; }
+};
+
+// ---- pkv_simt.cu -----------------------------------------------------------------------
+void gather_kept(const Lc& lc, int elem_bytes, const void* K, const void* V, const int32_t* idx,
+                 const int32_t* head_off_dev, int Hkv, int L, int hd, int total, void* Kc, void* Vc,
+                 DevStatus* status);
+// out[r] = x[r] * gain / rms(x[r]) for the rows of x0 (N rows) followed by the rows of x1.
+void rmsnorm_f32(const Lc& lc, const float* x0, const float* x1, int N, int d, const float* gain, float eps,
+                 float* out);
+// C[M][N] = alpha * A[M][K] * B[N][K]^T (+ addend) (+ C if accumulate); B is fp32 or bf16.
+// lower_only: tiles strictly above the diagonal are skipped (symmetric updates).
+void gemm_tn_simt(const Lc& lc, const float* A, int64_t lda, const void* B, int64_t ldb, bool b_bf16, float* C,
+                  int64_t ldc, int M, int N, int K, float alpha, const float* addend, int64_t ldadd,
+                  bool accumulate, bool lower_only = false);
+// cos/sin table [N][hd/2] of pos = pos0 + (i - chunk_start[i]) (double-precision angles).
+void rope_table(const Lc& lc, const int32_t* tok_cs, int N, int hd, int pos0, float theta, float* cs_table);
+// rotate `heads` heads of width hd in rows [0, rows) of buf (row stride ld, column offset col0);
+// token of row r is r % N.
+void rope_apply(const Lc& lc, float* buf, int64_t ld, int col0, int heads, int hd, int rows, int N,
+                const float* cs_table);
+
+struct AttnArgs {
+    const float* q; int64_t ldq;          // [2*N][..] rotated queries, row = stream*N + token
+    const float* k_new; const float* v_new; int64_t ldkv;   // [2*N][..] reference tokens' keys/values
+    const void* K; const void* V;         // full cache [Hkv][L][hd]
+    const void* Kc; const void* Vc;       // compact cache [total][hd]
+    const float* bias;                    // optional logit bias for the compact cache
+    const int32_t* head_off;              // device [Hkv+1]
+    const int32_t* tok_cs;                // device [N] chunk start of each token
+    int N, Hq, Hkv, hd, L, elem_bytes;
+    int kv_split, nsplitF, nsplitC;
+    float* part_m; float* part_l; float* part_O;   // [nsplit][Hkv][N*g] and [..][hd]
+    float* aF; float* aC; float* dA;      // [N][Hq*hd]
+};
+void attention_simt(const Lc& lc, const AttnArgs& a);
+void attention_combine(const Lc& lc, const AttnArgs& a);
+
+// zF = xF + o[0:N]; dz = (xF - xC) + o[N:2N]; zC = zF - dz.   o is [2N][d].
+void oproj_epilogue(const Lc& lc, const float* xF, const float* xC, const float* o, int N, int d, float* zF,
+                    float* zC, float* dz);
+// gu [2N][2F] (gate | up): hF, hC = silu(gate)*up of the two streams, dh = hF - hC.
+void swiglu(const Lc& lc, const float* gu, int N, int F, float* hF, float* hC, float* dh);
+void transpose_f32(const Lc& lc, const float* in, int rows, int cols, float* out);
+// status->tr, fro2 from S [F][F]; optional sum of squares of an arbitrary buffer into *dst.
+void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status);
+void sumsq(const Lc& lc, const float* a, int64_t n, double* dst);
+// lambda from the statistics (mode), G = S_H + lambda I written to G.
+void make_ridge_matrix(const Lc& lc, const float* S_H, int F, float lam0, int mode, float* G, DevStatus* status);
+// out = a - b (n elements); out may alias a.
+void sub_f32(const Lc& lc, const float* a, const float* b, int64_t n, float* out);
+void merge_weights(const Lc& lc, void* W, int w_dtype, const float* dW, int64_t count);
+
+// ---- pkv_solve.cu ----------------------------------------------------------------------
+struct SolveWs {
+    float* G;       // [F][F] ridge matrix, destroyed by the factorisation
+    float* Lm;      // [F][F] lower Cholesky factor (upper part zero)
+    float* LT;      // [F][F] its transpose
+    float* inv;     // [nblk][nb][nb] inverses of the diagonal blocks
+    float* invT;    // [nblk][nb][nb] their transposes
+    float* Y;       // [d][F] right-hand side, overwritten while solving
+};
+constexpr int kSolveNb = 64;
+// dW [d][F] = S_T G^{-1}; ws.G holds G on entry, ws.Y holds a copy of S_T on entry.
+void ridge_solve_simt(const Lc& lc, const SolveWs& ws, int F, int d, float* dW, DevStatus* status);
+
+}  // namespace pkv

@@ -1,0 +1,696 @@
+// SIMT fp32 kernels: index check + compaction, norms, rotary embedding, a tiled fp32 GEMM, a
+// tiled flash-style attention with split-K partials, the split-K combine (which also forms
+// dA = aF - aC before any rounding), element-wise epilogues, reductions and the merge.
+//
+// These kernels are the whole path for fp32 weights/caches and an on-device cross-check of the
+// tensor-core kernels for bf16 (PKV_ENGINE_SIMT).  Nothing here traps: invalid inputs set a
+// status word and the offending access is skipped.
+#include <math.h>
+
+#include "pkv_internal.h"
+
+namespace pkv {
+
+__device__ __forceinline__ float ld_as_float(const float* p) { return *p; }
+__device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+__device__ __forceinline__ void raise(DevStatus* s, int code) { atomicCAS(&s->code, 0, code); }
+
+// ------------------------------------------------------------------------------------------
+// index check + compaction (bit-exact)
+// ------------------------------------------------------------------------------------------
+// One warp per kept row.  Row i of head h is valid iff 0 <= idx[i] < L and it exceeds its
+// predecessor inside the head.  Invalid rows are reported (smallest flat position wins) and not
+// copied.  Copies move 16-byte chunks, so K/V rows must be 16-byte multiples (hd*elem >= 16).
+__global__ void __launch_bounds__(256) k_gather_kept(const uint4* __restrict__ K, const uint4* __restrict__ V,
+                                                     const int32_t* __restrict__ idx,
+                                                     const int32_t* __restrict__ head_off, int Hkv, int L,
+                                                     int row_chunks, int total, uint4* __restrict__ Kc,
+                                                     uint4* __restrict__ Vc, DevStatus* status) {
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (warp >= total) return;
+    int h = 0;
+    while (h + 1 < Hkv && head_off[h + 1] <= warp) ++h;
+    int v = idx[warp];
+    bool ok = v >= 0 && v < L;
+    if (ok && warp > head_off[h]) ok = v > idx[warp - 1];
+    if (!ok) {
+        if (lane == 0) {
+            raise(status, PKV_ERR_BAD_INDEX);
+            unsigned long long key = (unsigned long long)warp + 1ull;
+            unsigned long long old = status->bad_index;
+            while (old == 0ull || key < old) {
+                unsigned long long prev = atomicCAS(&status->bad_index, old, key);
+                if (prev == old) break;
+                old = prev;
+            }
+        }
+        return;
+    }
+    const uint4* ks = K + ((size_t)h * L + v) * row_chunks;
+    const uint4* vs = V + ((size_t)h * L + v) * row_chunks;
+    uint4* kd = Kc + (size_t)warp * row_chunks;
+    uint4* vd = Vc + (size_t)warp * row_chunks;
+    for (int c = lane; c < row_chunks; c += 32) {
+        kd[c] = ks[c];
+        vd[c] = vs[c];
+    }
+}
+
+void gather_kept(const Lc& lc, int elem_bytes, const void* K, const void* V, const int32_t* idx,
+                 const int32_t* head_off_dev, int Hkv, int L, int hd, int total, void* Kc, void* Vc,
+                 DevStatus* status) {
+    if (total <= 0) return;
+    int row_chunks = hd * elem_bytes / 16;
+    int warps_per_block = 8;
+    int blocks = (total + warps_per_block - 1) / warps_per_block;
+    k_gather_kept<<<blocks, 256, 0, lc.st>>>((const uint4*)K, (const uint4*)V, idx, head_off_dev, Hkv, L,
+                                             row_chunks, total, (uint4*)Kc, (uint4*)Vc, status);
+    lc.count();
+}
+
+// ------------------------------------------------------------------------------------------
+// RMSNorm
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float block_sum(float v, float* red) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+    __syncthreads();
+    if (l == 0) red[w] = v;
+    __syncthreads();
+    float t = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
+    if (w == 0) {
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (l == 0) red[0] = t;
+    }
+    __syncthreads();
+    return red[0];
+}
+
+__global__ void __launch_bounds__(256) k_rmsnorm_f32(const float* __restrict__ x0, const float* __restrict__ x1,
+                                                     int N, int d, const float* __restrict__ gain, float eps,
+                                                     float* __restrict__ out) {
+    __shared__ float red[32];
+    int r = blockIdx.x;
+    const float* x = (r < N) ? x0 + (size_t)r * d : x1 + (size_t)(r - N) * d;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        float v = x[c];
+        ss += v * v;
+    }
+    float tot = block_sum(ss, red);
+    float inv = 1.0f / sqrtf(tot / (float)d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) out[(size_t)r * d + c] = x[c] * gain[c] * inv;
+}
+
+void rmsnorm_f32(const Lc& lc, const float* x0, const float* x1, int N, int d, const float* gain, float eps,
+                 float* out) {
+    k_rmsnorm_f32<<<2 * N, 256, 0, lc.st>>>(x0, x1, N, d, gain, eps, out);
+    lc.count();
+}
+
+// ------------------------------------------------------------------------------------------
+// tiled fp32 GEMM, C = alpha * A B^T (+ addend) (+ C)
+// ------------------------------------------------------------------------------------------
+template <typename TB>
+__global__ void __launch_bounds__(256) k_gemm_tn(const float* __restrict__ A, int64_t lda,
+                                                 const TB* __restrict__ B, int64_t ldb, float* C, int64_t ldc,
+                                                 int M, int N, int K, float alpha, const float* addend,
+                                                 int64_t ldadd, int accumulate, int lower_only) {
+    constexpr int BM = 64, BN = 64, BK = 16;
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    int bm = blockIdx.y * BM, bn = blockIdx.x * BN;
+    if (lower_only && bn > bm + BM - 1) return;
+    int tid = threadIdx.x;
+    int tx = tid & 15, ty = tid >> 4;
+    int lr = tid >> 2, lk = (tid & 3) * 4;     // loader: row 0..63, k offset 0,4,8,12
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < K; k0 += BK) {
+        float av[4] = {0.f, 0.f, 0.f, 0.f}, bv[4] = {0.f, 0.f, 0.f, 0.f};
+        int ar = bm + lr, br = bn + lr;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int kk = k0 + lk + i;
+            if (ar < M && kk < K) av[i] = A[(size_t)ar * lda + kk];
+            if (br < N && kk < K) bv[i] = ld_as_float(B + (size_t)br * ldb + kk);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            As[lk + i][lr] = av[i];
+            Bs[lk + i][lr] = bv[i];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        int r = bm + ty * 4 + i;
+        if (r >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int c = bn + tx * 4 + j;
+            if (c >= N) continue;
+            float v = alpha * acc[i][j];
+            if (addend) v += addend[(size_t)r * ldadd + c];
+            if (accumulate) v += C[(size_t)r * ldc + c];
+            C[(size_t)r * ldc + c] = v;
+        }
+    }
+}
+
+void gemm_tn_simt(const Lc& lc, const float* A, int64_t lda, const void* B, int64_t ldb, bool b_bf16, float* C,
+                  int64_t ldc, int M, int N, int K, float alpha, const float* addend, int64_t ldadd,
+                  bool accumulate, bool lower_only) {
+    if (M <= 0 || N <= 0) return;
+    dim3 grid((N + 63) / 64, (M + 63) / 64);
+    if (b_bf16)
+        k_gemm_tn<__nv_bfloat16><<<grid, 256, 0, lc.st>>>(A, lda, (const __nv_bfloat16*)B, ldb, C, ldc, M, N, K,
+                                                          alpha, addend, ldadd, accumulate, lower_only);
+    else
+        k_gemm_tn<float><<<grid, 256, 0, lc.st>>>(A, lda, (const float*)B, ldb, C, ldc, M, N, K, alpha, addend,
+                                                  ldadd, accumulate, lower_only);
+    lc.count();
+}
+
+// ------------------------------------------------------------------------------------------
+// rotary embedding: half-split pairs (c, c + hd/2), angle pos * theta^(-2c/hd)
+// ------------------------------------------------------------------------------------------
+// The angle is formed in double precision: at positions near 2e5 an fp32 product pos*freq
+// would already be off by ~1e-2 rad.
+__global__ void k_rope_table(const int32_t* __restrict__ tok_cs, int N, int hd, int pos0, double theta,
+                             float* __restrict__ tab) {
+    int half = hd / 2;
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N * half) return;
+    int tok = i / half, c = i % half;
+    double pos = (double)pos0 + (double)(tok - tok_cs[tok]);
+    double ang = (theta > 0.0) ? pos * pow(theta, -2.0 * (double)c / (double)hd) : 0.0;
+    double s, co;
+    sincos(ang, &s, &co);
+    tab[2 * (size_t)i] = (float)co;
+    tab[2 * (size_t)i + 1] = (float)s;
+}
+
+void rope_table(const Lc& lc, const int32_t* tok_cs, int N, int hd, int pos0, float theta, float* cs_table) {
+    int n = N * (hd / 2);
+    k_rope_table<<<(n + 255) / 256, 256, 0, lc.st>>>(tok_cs, N, hd, pos0, (double)theta, cs_table);
+    lc.count();
+}
+
+__global__ void k_rope_apply(float* __restrict__ buf, int64_t ld, int col0, int heads, int hd, int rows, int N,
+                             const float* __restrict__ tab) {
+    int half = hd / 2;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t total = (size_t)rows * heads * half;
+    if (i >= total) return;
+    int c = (int)(i % half);
+    int h = (int)((i / half) % heads);
+    int r = (int)(i / ((size_t)half * heads));
+    int tok = r % N;
+    float co = tab[2 * ((size_t)tok * half + c)], s = tab[2 * ((size_t)tok * half + c) + 1];
+    float* p = buf + (size_t)r * ld + col0 + h * hd + c;
+    float lo = p[0], hi = p[half];
+    p[0] = lo * co - hi * s;
+    p[half] = hi * co + lo * s;
+}
+
+void rope_apply(const Lc& lc, float* buf, int64_t ld, int col0, int heads, int hd, int rows, int N,
+                const float* cs_table) {
+    size_t total = (size_t)rows * heads * (hd / 2);
+    k_rope_apply<<<(unsigned)((total + 255) / 256), 256, 0, lc.st>>>(buf, ld, col0, heads, hd, rows, N, cs_table);
+    lc.count();
+}
+
+// ------------------------------------------------------------------------------------------
+// attention, SIMT fp32: tile of 32 query rows x 32 keys, online softmax, split-K partials
+// ------------------------------------------------------------------------------------------
+// Query row r of KV head kh stands for (token r / g, head kh*g + r % g) so that one key/value
+// tile serves the whole GQA group.  The key sequence of a stream is its cache rows followed by
+// the N reference tokens; reference key j is visible to token t iff chunk_start(t) <= j <= t.
+template <typename TC, int HD>
+__global__ void __launch_bounds__(128) k_attn_simt(AttnArgs a) {
+    constexpr int BM = 32, BN = 32;
+    extern __shared__ float sm[];
+    float* Qs = sm;                          // [BM][HD+1]
+    float* Ks = Qs + BM * (HD + 1);          // [BN][HD+1]
+    float* Vs = Ks + BN * (HD + 1);          // [BN][HD]
+    float* Ss = Vs + BN * HD;                // [BM][BN+1]
+    int* row_tok = (int*)(Ss + BM * (BN + 1));   // [BM]
+    int* row_cs = row_tok + BM;                  // [BM]
+
+    const int tid = threadIdx.x;
+    const int kh = blockIdx.y;
+    const int z = blockIdx.z;
+    const int stream = (z >= a.nsplitF) ? 1 : 0;
+    const int split = stream ? z - a.nsplitF : z;
+    const int g = a.Hq / a.Hkv;
+    const int rows = a.N * g;
+    const int r0 = blockIdx.x * BM;
+
+    const TC* Kbase;
+    const TC* Vbase;
+    const float* bias = nullptr;
+    int Lc_rows;
+    if (stream == 0) {
+        Kbase = (const TC*)a.K + (size_t)kh * a.L * HD;
+        Vbase = (const TC*)a.V + (size_t)kh * a.L * HD;
+        Lc_rows = a.L;
+    } else {
+        int off = a.head_off[kh];
+        Kbase = (const TC*)a.Kc + (size_t)off * HD;
+        Vbase = (const TC*)a.Vc + (size_t)off * HD;
+        Lc_rows = a.head_off[kh + 1] - off;
+        if (a.bias) bias = a.bias + off;
+    }
+    const int Lt = Lc_rows + a.N;
+    const int k_begin = split * a.kv_split;
+    const int k_end = min(Lt, k_begin + a.kv_split);
+    const float scale = rsqrtf((float)HD);
+
+    if (tid < BM) {
+        int r = r0 + tid;
+        int tok = (r < rows) ? r / g : 0;
+        row_tok[tid] = (r < rows) ? tok : -1;
+        row_cs[tid] = (r < rows) ? a.tok_cs[tok] : 0;
+    }
+    for (int i = tid; i < BM * HD; i += 128) {
+        int rr = i / HD, c = i % HD;
+        int r = r0 + rr;
+        float v = 0.f;
+        if (r < rows) {
+            int tok = r / g, hg = r % g;
+            v = a.q[((size_t)stream * a.N + tok) * a.ldq + (size_t)(kh * g + hg) * HD + c] * scale;
+        }
+        Qs[rr * (HD + 1) + c] = v;
+    }
+
+    const int row = tid >> 2, sub = tid & 3;
+    float m = -INFINITY, l = 0.f;
+    float O[HD / 4];
+#pragma unroll
+    for (int i = 0; i < HD / 4; ++i) O[i] = 0.f;
+
+    for (int kt = k_begin; kt < k_end; kt += BN) {
+        __syncthreads();
+        for (int i = tid; i < BN * HD; i += 128) {
+            int key = i / HD, c = i % HD;
+            int kk = kt + key;
+            float kv = 0.f, vv = 0.f;
+            if (kk < k_end) {
+                if (kk < Lc_rows) {
+                    kv = ld_as_float(Kbase + (size_t)kk * HD + c);
+                    vv = ld_as_float(Vbase + (size_t)kk * HD + c);
+                } else {
+                    size_t rr = ((size_t)stream * a.N + (kk - Lc_rows)) * a.ldkv + (size_t)kh * HD + c;
+                    kv = a.k_new[rr];
+                    vv = a.v_new[rr];
+                }
+            }
+            Ks[key * (HD + 1) + c] = kv;
+            Vs[key * HD + c] = vv;
+        }
+        __syncthreads();
+        {   // scores: 2 rows x 4 keys per thread
+            int ty = tid >> 3, tx = tid & 7;
+            float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            const float* q0 = Qs + (ty * 2) * (HD + 1);
+            const float* q1 = q0 + (HD + 1);
+            const float* kp = Ks + (tx * 4) * (HD + 1);
+#pragma unroll 8
+            for (int c = 0; c < HD; ++c) {
+                float a0 = q0[c], a1 = q1[c];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float kvv = kp[j * (HD + 1) + c];
+                    s[0][j] = fmaf(a0, kvv, s[0][j]);
+                    s[1][j] = fmaf(a1, kvv, s[1][j]);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                int rr = ty * 2 + i;
+                int tok = row_tok[rr], cs = row_cs[rr];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    int kk = kt + tx * 4 + j;
+                    float v = s[i][j];
+                    bool vis = (kk < k_end) && (tok >= 0);
+                    if (vis) {
+                        if (kk < Lc_rows) {
+                            if (bias) v += bias[kk];
+                        } else {
+                            int jn = kk - Lc_rows;
+                            vis = (jn >= cs) && (jn <= tok);
+                        }
+                    }
+                    Ss[rr * (BN + 1) + tx * 4 + j] = vis ? v : -INFINITY;
+                }
+            }
+        }
+        __syncthreads();
+        {   // online softmax for `row`, 8 keys per thread, 4 threads per row (same warp)
+            float* sr = Ss + row * (BN + 1) + sub * 8;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mx = fmaxf(mx, sr[j]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            float m_new = fmaxf(m, mx);
+            float alpha = 1.f, ps = 0.f;
+            if (m_new == -INFINITY) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) sr[j] = 0.f;
+            } else {
+                alpha = expf(m - m_new);          // m = -inf -> 0
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float p = expf(sr[j] - m_new);
+                    sr[j] = p;
+                    ps += p;
+                }
+            }
+            ps += __shfl_xor_sync(0xffffffffu, ps, 1);
+            ps += __shfl_xor_sync(0xffffffffu, ps, 2);
+            l = l * alpha + ps;
+            m = m_new;
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < HD / 4; ++i) O[i] *= alpha;
+            const float* pr = Ss + row * (BN + 1);
+            for (int k = 0; k < BN; ++k) {
+                float p = pr[k];
+                const float* vr = Vs + k * HD + sub;
+#pragma unroll
+                for (int i = 0; i < HD / 4; ++i) O[i] = fmaf(p, vr[i * 4], O[i]);
+            }
+        }
+    }
+    int r = r0 + row;
+    if (r < rows) {
+        size_t pr = ((size_t)z * a.Hkv + kh) * rows + r;
+        if (sub == 0) {
+            a.part_m[pr] = m;
+            a.part_l[pr] = l;
+        }
+        float* po = a.part_O + pr * HD;
+#pragma unroll
+        for (int i = 0; i < HD / 4; ++i) po[i * 4 + sub] = O[i];
+    }
+}
+
+template <typename TC, int HD>
+static void launch_attn_simt(const Lc& lc, const AttnArgs& a) {
+    int g = a.Hq / a.Hkv;
+    int rows = a.N * g;
+    dim3 grid((rows + 31) / 32, a.Hkv, a.nsplitF + a.nsplitC);
+    size_t smem = (size_t)(32 * (HD + 1) * 2 + 32 * HD + 32 * 33) * sizeof(float) + 64 * sizeof(int);
+    cudaFuncSetAttribute(k_attn_simt<TC, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    k_attn_simt<TC, HD><<<grid, 128, smem, lc.st>>>(a);
+    lc.count();
+}
+
+void attention_simt(const Lc& lc, const AttnArgs& a) {
+    if (a.elem_bytes == 2) {
+        if (a.hd == 128) launch_attn_simt<__nv_bfloat16, 128>(lc, a);
+        else launch_attn_simt<__nv_bfloat16, 64>(lc, a);
+    } else {
+        if (a.hd == 128) launch_attn_simt<float, 128>(lc, a);
+        else launch_attn_simt<float, 64>(lc, a);
+    }
+}
+
+// Split-K combine and residual epilogue: one warp per (kv head, query row); merges the
+// (m, l, O) partials of each stream and writes aF, aC and dA = aF - aC in fp32.
+__global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
+    int g = a.Hq / a.Hkv;
+    int rows = a.N * g;
+    int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (w >= a.Hkv * rows) return;
+    int kh = w / rows, r = w % rows;
+    int tok = r / g, hg = r % g;
+    int hd = a.hd;
+    int per = hd / 32;                       // 2 or 4 columns per lane
+    float res[2][4];
+    for (int s = 0; s < 2; ++s) {
+        int z0 = s ? a.nsplitF : 0;
+        int ns = s ? a.nsplitC : a.nsplitF;
+        float M = -INFINITY;
+        for (int i = 0; i < ns; ++i) M = fmaxf(M, a.part_m[((size_t)(z0 + i) * a.Hkv + kh) * rows + r]);
+        float den = 0.f, num[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int i = 0; i < ns; ++i) {
+            size_t pr = ((size_t)(z0 + i) * a.Hkv + kh) * rows + r;
+            float mi = a.part_m[pr];
+            if (mi == -INFINITY) continue;
+            float wgt = expf(mi - M);
+            den += wgt * a.part_l[pr];
+            const float* po = a.part_O + pr * hd + lane * per;
+            for (int c = 0; c < per; ++c) num[c] += wgt * po[c];
+        }
+        float inv = (den > 0.f) ? 1.f / den : 0.f;
+        for (int c = 0; c < per; ++c) res[s][c] = num[c] * inv;
+    }
+    size_t o = (size_t)tok * a.Hq * hd + (size_t)(kh * g + hg) * hd + lane * per;
+    for (int c = 0; c < per; ++c) {
+        a.aF[o + c] = res[0][c];
+        a.aC[o + c] = res[1][c];
+        a.dA[o + c] = res[0][c] - res[1][c];
+    }
+}
+
+void attention_combine(const Lc& lc, const AttnArgs& a) {
+    int g = a.Hq / a.Hkv;
+    long long warps = (long long)a.Hkv * a.N * g;
+    k_attn_combine<<<(unsigned)((warps + 7) / 8), 256, 0, lc.st>>>(a);
+    lc.count();
+}
+
+// ------------------------------------------------------------------------------------------
+// element-wise epilogues
+// ------------------------------------------------------------------------------------------
+__global__ void k_oproj_epilogue(const float* __restrict__ xF, const float* __restrict__ xC,
+                                 const float* __restrict__ o, size_t n, float* __restrict__ zF,
+                                 float* __restrict__ zC, float* __restrict__ dz) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float f = xF[i], c = xC[i];
+    float zf = f + o[i];
+    float d = (f - c) + o[n + i];
+    zF[i] = zf;
+    dz[i] = d;
+    zC[i] = zf - d;
+}
+
+void oproj_epilogue(const Lc& lc, const float* xF, const float* xC, const float* o, int N, int d, float* zF,
+                    float* zC, float* dz) {
+    size_t n = (size_t)N * d;
+    k_oproj_epilogue<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(xF, xC, o, n, zF, zC, dz);
+    lc.count();
+}
+
+__device__ __forceinline__ float silu_f(float t) { return t / (1.0f + expf(-t)); }
+
+__global__ void k_swiglu(const float* __restrict__ gu, int N, int F, float* __restrict__ hF,
+                         float* __restrict__ hC, float* __restrict__ dh) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t n = (size_t)N * F;
+    if (i >= n) return;
+    size_t r = i / F, c = i % F;
+    const float* a = gu + r * 2 * F;
+    const float* b = gu + (r + N) * 2 * F;
+    float f = silu_f(a[c]) * a[F + c];
+    float s = silu_f(b[c]) * b[F + c];
+    hF[i] = f;
+    hC[i] = s;
+    dh[i] = f - s;
+}
+
+void swiglu(const Lc& lc, const float* gu, int N, int F, float* hF, float* hC, float* dh) {
+    size_t n = (size_t)N * F;
+    k_swiglu<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(gu, N, F, hF, hC, dh);
+    lc.count();
+}
+
+__global__ void k_transpose(const float* __restrict__ in, int rows, int cols, float* __restrict__ out) {
+    __shared__ float t[32][33];
+    int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        int r = r0 + j, c = c0 + threadIdx.x;
+        if (r < rows && c < cols) t[j][threadIdx.x] = in[(size_t)r * cols + c];
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        int c = c0 + j, r = r0 + threadIdx.x;
+        if (r < rows && c < cols) out[(size_t)c * rows + r] = t[threadIdx.x][j];
+    }
+}
+
+void transpose_f32(const Lc& lc, const float* in, int rows, int cols, float* out) {
+    dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
+    k_transpose<<<grid, block, 0, lc.st>>>(in, rows, cols, out);
+    lc.count();
+}
+
+// ------------------------------------------------------------------------------------------
+// reductions and the ridge matrix
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum_d(double v) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__global__ void __launch_bounds__(256) k_trace_fro2(const float* __restrict__ S, int F, DevStatus* status) {
+    size_t n = (size_t)F * F;
+    double fro = 0.0, tr = 0.0;
+    int bad = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float v = S[i];
+        if (!isfinite(v)) bad = 1;
+        fro += (double)v * (double)v;
+        if (i / F == i % F) tr += (double)v;
+    }
+    fro = warp_sum_d(fro);
+    tr = warp_sum_d(tr);
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(&status->fro2, fro);
+        if (tr != 0.0) atomicAdd(&status->tr, tr);
+    }
+    if (bad) raise(status, PKV_ERR_NONFINITE);
+}
+
+void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status) {
+    k_trace_fro2<<<296, 256, 0, lc.st>>>(S, F, status);
+    lc.count();
+}
+
+__global__ void __launch_bounds__(256) k_sumsq(const float* __restrict__ a, size_t n, double* dst) {
+    double s = 0.0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float v = a[i];
+        s += (double)v * (double)v;
+    }
+    s = warp_sum_d(s);
+    if ((threadIdx.x & 31) == 0) atomicAdd(dst, s);
+}
+
+void sumsq(const Lc& lc, const float* a, int64_t n, double* dst) {
+    if (n <= 0) return;
+    k_sumsq<<<296, 256, 0, lc.st>>>(a, (size_t)n, dst);
+    lc.count();
+}
+
+// lambda from the statistics (Eq. 7 or a variant), then G = S_H + lambda I.
+__global__ void k_lambda(int F, float lam0, int mode, DevStatus* status) {
+    double tr = status->tr, fro2 = status->fro2;
+    double lam;
+    if (mode == PKV_LAMBDA_ABSOLUTE) {
+        lam = lam0;
+    } else {
+        if (!(tr > 0.0)) {
+            raise(status, PKV_ERR_DEGENERATE);
+            lam = 1.0;      // keeps the factorisation finite; the call reports the error
+        } else if (mode == PKV_LAMBDA_TRACE_MEAN) {
+            lam = (double)lam0 * tr / (double)F;
+        } else {
+            lam = (double)lam0 * fro2 / tr;
+        }
+    }
+    status->lam = (float)lam;
+    status->min_pivot = INFINITY;
+}
+
+__global__ void k_ridge_matrix(const float* __restrict__ S, int F, float* __restrict__ G,
+                               const DevStatus* __restrict__ status) {
+    size_t n = (size_t)F * F;
+    float lam = status->lam;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float v = S[i];
+        if (i / F == i % F) v += lam;
+        G[i] = v;
+    }
+}
+
+void make_ridge_matrix(const Lc& lc, const float* S_H, int F, float lam0, int mode, float* G, DevStatus* status) {
+    k_lambda<<<1, 1, 0, lc.st>>>(F, lam0, mode, status);
+    k_ridge_matrix<<<592, 256, 0, lc.st>>>(S_H, F, G, status);
+    lc.count(2);
+}
+
+__global__ void k_sub(const float* __restrict__ a, const float* __restrict__ b, size_t n, float* __restrict__ out) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = a[i] - b[i];
+}
+
+void sub_f32(const Lc& lc, const float* a, const float* b, int64_t n, float* out) {
+    if (n <= 0) return;
+    k_sub<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(a, b, (size_t)n, out);
+    lc.count();
+}
+
+// ------------------------------------------------------------------------------------------
+// merge: W <- W + dW, sum in fp32, one rounding to W's type
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_merge_bf16(__nv_bfloat16* __restrict__ W, const float* __restrict__ dW,
+                                                    size_t n) {
+    size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+    if (i + 8 <= n) {
+        uint4 wv = *reinterpret_cast<const uint4*>(W + i);
+        float4 d0 = *reinterpret_cast<const float4*>(dW + i);
+        float4 d1 = *reinterpret_cast<const float4*>(dW + i + 4);
+        __nv_bfloat162* wp = reinterpret_cast<__nv_bfloat162*>(&wv);
+        float2 f;
+        f = __bfloat1622float2(wp[0]); wp[0] = __floats2bfloat162_rn(f.x + d0.x, f.y + d0.y);
+        f = __bfloat1622float2(wp[1]); wp[1] = __floats2bfloat162_rn(f.x + d0.z, f.y + d0.w);
+        f = __bfloat1622float2(wp[2]); wp[2] = __floats2bfloat162_rn(f.x + d1.x, f.y + d1.y);
+        f = __bfloat1622float2(wp[3]); wp[3] = __floats2bfloat162_rn(f.x + d1.z, f.y + d1.w);
+        *reinterpret_cast<uint4*>(W + i) = wv;
+    } else {
+        for (size_t j = i; j < n; ++j) W[j] = __float2bfloat16_rn(__bfloat162float(W[j]) + dW[j]);
+    }
+}
+
+__global__ void __launch_bounds__(256) k_merge_f32(float* __restrict__ W, const float* __restrict__ dW, size_t n) {
+    size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i + 4 <= n) {
+        float4 w = *reinterpret_cast<const float4*>(W + i);
+        float4 d = *reinterpret_cast<const float4*>(dW + i);
+        w.x += d.x; w.y += d.y; w.z += d.z; w.w += d.w;
+        *reinterpret_cast<float4*>(W + i) = w;
+    } else {
+        for (size_t j = i; j < n; ++j) W[j] += dW[j];
+    }
+}
+
+void merge_weights(const Lc& lc, void* W, int w_dtype, const float* dW, int64_t count) {
+    if (count <= 0) return;
+    size_t n = (size_t)count;
+    if (w_dtype == PKV_BF16) {
+        size_t thr = (n + 7) / 8;
+        k_merge_bf16<<<(unsigned)((thr + 255) / 256), 256, 0, lc.st>>>((__nv_bfloat16*)W, dW, n);
+    } else {
+        size_t thr = (n + 3) / 4;
+        k_merge_f32<<<(unsigned)((thr + 255) / 256), 256, 0, lc.st>>>((float*)W, dW, n);
+    }
+    lc.count();
+}
+
+}  // namespace pkv

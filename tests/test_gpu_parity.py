@@ -1,0 +1,343 @@
+"""CUDA path vs the fp64 oracle, element by element on the same seeded inputs, through the C ABI.
+
+Tolerances (stated by the benchmark spec): attention outputs max relative error <= 2e-2
+(relative to max|a| per head), dW relative Frobenius error <= 5e-3, index handling / compaction
+/ merge bit-exact."""
+import numpy as np
+import pytest
+
+from oracle import pkv_oracle as orc
+from paper_2609_39329_b200 import inputs as gen
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+TC_READY = False      # flipped when the tensor-core engine lands
+ATTN_TOL = 2e-2
+DW_TOL = 5e-3
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    from paper_2609_39329_b200 import binding
+    assert torch.cuda.is_available()
+    binding.lib()
+    return binding
+
+
+def small_cfg(dtype="bf16", **kw):
+    base = gen.benchmark_config(2)
+    d = dict(dtype=dtype, d=256, Hq=8, Hkv=2, hd=64, F=192, L=1000, N=70, window=16, budget=100, n_obs=8,
+             name="small")
+    d.update(kw)
+    return gen.scaled_config(base, **d)
+
+
+def engines(B, cfg):
+    """Engines a config must be checked on: fp32 -> SIMT; bf16 -> tensor-core path and SIMT."""
+    if cfg.dtype == "fp32" or not TC_READY:
+        return [B.ENGINE_SIMT]
+    return [B.ENGINE_AUTO, B.ENGINE_SIMT]
+
+
+def gpu_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode=0, kv_split=0, want_next=True):
+    import torch
+    ctx = B.PkvContext(B.dims_from_config(cfg, N_max=xF.shape[0], b_max=max(len(k) for k in lay["kept"])),
+                       engine=engine, kv_split=kv_split)
+    w = B.to_device(lay["weights"], cfg.dtype)
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    off, idx = gen.kept_to_csr(lay["kept"])
+    idx_t = torch.from_numpy(idx).cuda() if len(idx) else None
+    xF_t = torch.from_numpy(np.ascontiguousarray(xF, dtype=np.float32)).cuda()
+    xC_t = xF_t if xC is xF else torch.from_numpy(np.ascontiguousarray(xC, dtype=np.float32)).cuda()
+    if idx_t is None:   # empty compressed cache: explicit form with zero rows
+        dummy = torch.zeros((1, cfg.hd), dtype=kv["K"].dtype, device="cuda")
+        out = ctx.build_patch(w, kv["K"], kv["V"], off, None, xF_t, xC_t, chunk_off, cfg.L, lam0, mode, want_next,
+                              Kc=dummy, Vc=dummy)
+    else:
+        out = ctx.build_patch(w, kv["K"], kv["V"], off, idx_t, xF_t, xC_t, chunk_off, cfg.L, lam0, mode, want_next)
+    res = {k: (v.cpu().numpy() if hasattr(v, "cpu") else v) for k, v in out.items()}
+    res["launches"] = ctx.launch_count()
+    ctx.close()
+    return res
+
+
+def check_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode=0, kv_split=0):
+    ref = H.run_oracle(cfg, lay, xF, xC, chunk_off, lam0, mode)
+    got = gpu_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode, kv_split)
+    e_dw = H.rel_fro(got["dW"], ref["dW"])
+    assert e_dw <= DW_TOL, "dW rel fro %.3e" % e_dw
+    np.testing.assert_allclose(got["stats"]["lambda_eff"], ref["lam"], rtol=2e-3)
+    np.testing.assert_allclose(got["stats"]["trace"], ref["tr"], rtol=2e-3)
+    assert H.rel_fro(got["xF_next"], ref["xF_next"]) <= 1e-3
+    assert H.rel_fro(got["xC_next"], ref["xC_next"]) <= 1e-3
+    # the gap between the next states is the ridge residual (Eq. 4); compare it on its own scale
+    gap_ref = ref["xF_next"] - ref["xC_next"]
+    assert H.rel_fro(got["xF_next"].astype(np.float64) - got["xC_next"], gap_ref) <= 2e-2
+    np.testing.assert_allclose(got["stats"]["target_fro2"], ref["T_fro2"], rtol=2e-2)
+    assert got["launches"] > 0
+    return e_dw
+
+
+# ------------------------------------------------------------------ S0 + merge: bit-exact
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_gather_kept_bit_exact_and_bad_sets_reported(B, dtype):
+    import torch
+    cfg = small_cfg(dtype, hd=128, Hq=6, Hkv=3, L=777)
+    r = np.random.default_rng(0)
+    K = gen._to_dtype(r.standard_normal((cfg.Hkv, cfg.L, cfg.hd)).astype(np.float32), dtype)
+    V = gen._to_dtype(r.standard_normal((cfg.Hkv, cfg.L, cfg.hd)).astype(np.float32), dtype)
+    kept = [np.sort(r.choice(cfg.L, size=b, replace=False)).astype(np.int32) for b in (100, 0, 37)]
+    kept[2][-1] = cfg.L - 1
+    kept[0][0] = 0
+    off, idx = gen.kept_to_csr(kept)
+    ctx = B.PkvContext(B.dims_from_config(cfg, b_max=100), engine=B.ENGINE_SIMT)
+    kv = B.to_device({"K": K, "V": V}, dtype)
+    Kc, Vc = ctx.gather_kept(kv["K"], kv["V"], off, torch.from_numpy(idx).cuda())
+    Ko, Vo = orc.gather_cache(K, V, kept)
+    np.testing.assert_array_equal(Kc.float().cpu().numpy(), np.concatenate(Ko))
+    np.testing.assert_array_equal(Vc.float().cpu().numpy(), np.concatenate(Vo))
+    # invalid sets: duplicate, descending, negative, == L; the first offender is reported
+    for pos, val in ((5, int(idx[4])), (50, int(idx[49]) - 1), (0, -1), (136, cfg.L)):
+        bad = idx.copy()
+        bad[pos] = val
+        badk = [bad[off[h]:off[h + 1]] for h in range(cfg.Hkv)]
+        want = orc.check_kept(badk, cfg.L)
+        with pytest.raises(B.PkvError) as ei:
+            ctx.gather_kept(kv["K"], kv["V"], off, torch.from_numpy(bad).cuda())
+        assert ei.value.code == -3 and tuple(ei.value.info) == want
+    # the context stays usable after an error
+    Kc2, _ = ctx.gather_kept(kv["K"], kv["V"], off, torch.from_numpy(idx).cuda())
+    assert torch.equal(Kc, Kc2)
+    ctx.close()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_merge_bit_exact(B, dtype):
+    import torch
+    r = np.random.default_rng(1)
+    n = (130, 77)      # 10010 entries: not a multiple of the vector width
+    W = gen._to_dtype((r.standard_normal(n) * 0.02).astype(np.float32), dtype)
+    dW = (r.standard_normal(n) * 1e-3).astype(np.float32)
+    want = orc.merge(W, dW, dtype)
+    cfg = small_cfg(dtype)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_SIMT)
+    Wt = torch.from_numpy(W).cuda().to(torch.bfloat16 if dtype == "bf16" else torch.float32)
+    ctx.merge(Wt, torch.from_numpy(dW).cuda())
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(Wt.float().cpu().numpy(), want)
+    ctx.close()
+
+
+# ------------------------------------------------------------------ S3 alone
+
+def attention_case(B, cfg, engine, chunk_off, budgets, kv_split=0, seed=0):
+    import torch
+    r = np.random.default_rng(seed)
+    N = chunk_off[-1]
+    q = r.standard_normal((2, N, cfg.Hq, cfg.hd)).astype(np.float32) * 1.3
+    k = r.standard_normal((2, N, cfg.Hkv, cfg.hd)).astype(np.float32)
+    v = r.standard_normal((2, N, cfg.Hkv, cfg.hd)).astype(np.float32)
+    kvd = gen.gen_cache(cfg, 0) if cfg.dtype == "bf16" else {
+        "K": r.standard_normal((cfg.Hkv, cfg.L, cfg.hd)).astype(np.float32),
+        "V": r.standard_normal((cfg.Hkv, cfg.L, cfg.hd)).astype(np.float32)}
+    kept = gen.select_kept(gen.scaled_config(cfg, kept_rule="random"), 0, per_head_budget=budgets)
+    Kg, Vg = orc.gather_cache(kvd["K"], kvd["V"], kept)
+    aF = orc.attention(q[0], k[0], v[0], list(kvd["K"]), list(kvd["V"]), chunk_off)
+    aC = orc.attention(q[1], k[1], v[1], Kg, Vg, chunk_off)
+    ctx = B.PkvContext(B.dims_from_config(cfg, N_max=N, b_max=max(max(budgets), 1)), engine=engine, kv_split=kv_split)
+    kv = B.to_device({"K": kvd["K"], "V": kvd["V"]}, cfg.dtype)
+    off, idx = gen.kept_to_csr(kept)
+    tq, tk, tv = (torch.from_numpy(t.reshape(2, N, -1)).cuda() for t in (q, k, v))
+    if len(idx):
+        gF, gC, gD = ctx.attention(tq, tk, tv, kv["K"], kv["V"], off, torch.from_numpy(idx).cuda(), chunk_off)
+    else:
+        dummy = torch.zeros((1, cfg.hd), dtype=kv["K"].dtype, device="cuda")
+        gF, gC, gD = ctx.attention(tq, tk, tv, kv["K"], kv["V"], off, None, chunk_off, Kc=dummy, Vc=dummy)
+    gF, gC, gD = (t.cpu().numpy() for t in (gF, gC, gD))
+    ctx.close()
+    assert H.attn_max_rel(gF, aF, cfg.Hq, cfg.hd) <= ATTN_TOL
+    assert H.attn_max_rel(gC, aC, cfg.Hq, cfg.hd) <= ATTN_TOL
+    assert H.attn_max_rel(gD, aF - aC, cfg.Hq, cfg.hd) <= ATTN_TOL
+    np.testing.assert_array_equal(gD, gF - gC)
+    return gF, aF
+
+
+@pytest.mark.parametrize("dtype,hd", [("bf16", 128), ("bf16", 64), ("fp32", 64)])
+def test_attention_parity_ragged_chunks_and_splits(B, dtype, hd):
+    cfg = small_cfg(dtype, hd=hd, Hq=8, Hkv=2, L=1500)
+    for engine in engines(B, cfg):
+        attention_case(B, cfg, engine, [0, 70], [100, 100])
+        attention_case(B, cfg, engine, [0, 13, 14, 70, 131], [257, 31], kv_split=256)   # ragged heads, 4 chunks
+        attention_case(B, cfg, engine, [0, 33], [0, 0])                                  # empty compressed cache
+
+
+def test_attention_group_of_seven_and_odd_lengths(B):
+    cfg = small_cfg("bf16", hd=128, Hq=14, Hkv=2, L=1237)
+    for engine in engines(B, cfg):
+        attention_case(B, cfg, engine, [0, 45], [19, 123], kv_split=320)
+
+
+# ------------------------------------------------------------------ S7, S8 alone
+
+@pytest.mark.parametrize("n,F,d", [(70, 192, 256), (300, 256, 128)])
+def test_gram_parity_and_accumulation(B, n, F, d):
+    import torch
+    cfg = small_cfg("bf16", F=F, d=d, Hq=d // 64, Hkv=1, N=n)
+    r = np.random.default_rng(2)
+    X = (r.standard_normal((n, F)) * np.exp(r.uniform(-1, 1, F))).astype(np.float32)
+    R = (r.standard_normal((n, d)) * 0.1).astype(np.float32)
+    S_H, S_T = orc.sufficient_statistics(X, R)
+    for engine in engines(B, cfg):
+        ctx = B.PkvContext(B.dims_from_config(cfg, N_max=n), engine=engine)
+        Xt, Rt = torch.from_numpy(X).cuda(), torch.from_numpy(R).cuda()
+        gH, gT = ctx.gram(Xt, Rt)
+        assert H.rel_fro(gH.cpu().numpy(), S_H) <= 2e-4
+        assert H.rel_fro(gT.cpu().numpy(), S_T) <= 2e-4
+        # Eq. 9: running sums over chunks
+        h = n // 3
+        aH, aT = ctx.gram(Xt[:h].contiguous(), Rt[:h].contiguous())
+        ctx.gram(Xt[h:].contiguous(), Rt[h:].contiguous(), aH, aT, accumulate=True)
+        assert H.rel_fro(aH.cpu().numpy(), S_H) <= 2e-4
+        assert H.rel_fro(aT.cpu().numpy(), S_T) <= 2e-4
+        ctx.close()
+
+
+@pytest.mark.parametrize("F,d,n", [(192, 256, 70), (200, 64, 500), (64, 64, 10)])
+def test_ridge_solve_parity_modes_and_errors(B, F, d, n):
+    import torch
+    cfg = small_cfg("bf16", F=F, d=d, Hq=max(d // 64, 1), Hkv=1)
+    r = np.random.default_rng(3)
+    X = r.standard_normal((n, F))
+    R = r.standard_normal((n, d))
+    S_H, S_T = orc.sufficient_statistics(X, R)
+    for engine in engines(B, cfg):
+        ctx = B.PkvContext(B.dims_from_config(cfg), engine=engine)
+        tH = torch.from_numpy(S_H.astype(np.float32)).cuda()
+        tT = torch.from_numpy(S_T.astype(np.float32)).cuda()
+        for mode, lam0 in ((B.LAMBDA_PAPER, 0.1), (B.LAMBDA_PAPER, 1e-3), (B.LAMBDA_ABSOLUTE, 5.0),
+                           (B.LAMBDA_TRACE_MEAN, 0.1)):
+            lam = orc.ridge_lambda(S_H, lam0, mode)
+            want = orc.ridge_solve(S_H, S_T, lam)
+            dW, st = ctx.ridge_solve(tH, tT, lam0, mode)
+            assert H.rel_fro(dW.cpu().numpy(), want) <= 1e-3, (mode, lam0)
+            np.testing.assert_allclose(st["lambda_eff"], lam, rtol=1e-4)
+            np.testing.assert_allclose(st["dW_fro2"], np.sum(want * want), rtol=2e-3)
+            assert st["min_pivot"] > 0
+        # not positive definite: a negative diagonal entry that the ridge does not lift
+        bad = S_H.astype(np.float32).copy()
+        bad[5, 5] = -1e6
+        with pytest.raises(B.PkvError) as ei:
+            ctx.ridge_solve(torch.from_numpy(bad).cuda(), tT, 1e-3, B.LAMBDA_ABSOLUTE)
+        assert ei.value.code == -4 and ei.value.info["err_info"][0] == 5
+        with pytest.raises(B.PkvError) as ei:
+            ctx.ridge_solve(torch.zeros_like(tH), tT, 0.1, B.LAMBDA_PAPER)
+        assert ei.value.code == -5
+        with pytest.raises(B.PkvError) as ei:
+            ctx.ridge_solve(tH, tT, 0.0, B.LAMBDA_PAPER)
+        assert ei.value.code == -1
+        dW, _ = ctx.ridge_solve(tH, tT, 0.1, B.LAMBDA_PAPER)      # still usable
+        assert torch.isfinite(dW).all()
+        ctx.close()
+
+
+# ------------------------------------------------------------------ whole block
+
+def test_config1_tiny_fp32_end_to_end(B):
+    cfg = gen.benchmark_config(1)
+    lay = H.make_problem(cfg)
+    x = lay["x0"]
+    check_build(B, cfg, lay, x, x, [0, cfg.N], cfg.lam0, B.ENGINE_SIMT)
+    check_build(B, cfg, lay, x, x, [0, cfg.N], 1e-2, B.ENGINE_SIMT, mode=B.LAMBDA_ABSOLUTE)
+
+
+@pytest.mark.parametrize("hd,Hq,Hkv", [(64, 8, 2), (128, 4, 2)])
+def test_small_bf16_block_chunks_ragged_distinct_states(B, hd, Hq, Hkv):
+    cfg = small_cfg("bf16", hd=hd, Hq=Hq, Hkv=Hkv, d=256, F=192, L=1000, N=150)
+    lay = H.make_problem(cfg, per_head_budget=[100, 37][:Hkv])
+    xF = lay["x0"]
+    xC = (xF + 0.02 * np.random.default_rng(5).standard_normal(xF.shape)).astype(np.float32)
+    for engine in engines(B, cfg):
+        check_build(B, cfg, lay, xF, xC, [0, 40, 41, 150], 0.1, engine, kv_split=256)
+        check_build(B, cfg, lay, xF, xF, [0, 150], 1e-3, engine)
+
+
+def test_identical_caches_give_zero_patch(B):
+    cfg = small_cfg("bf16", L=300, budget=300, N=40)
+    lay = H.make_problem(cfg)
+    lay["kept"] = [np.arange(cfg.L, dtype=np.int32)] * cfg.Hkv
+    for engine in engines(B, cfg):
+        got = gpu_build(B, cfg, lay, lay["x0"], lay["x0"], [0, cfg.N], 0.1, engine)
+        ref = H.run_oracle(cfg, lay, lay["x0"], lay["x0"], [0, cfg.N], 0.1)
+        assert np.all(ref["dW"] == 0.0)
+        # dA, dz, dh are formed as differences of identical numbers: exactly zero, hence dW = 0
+        assert np.all(got["dW"] == 0.0)
+        np.testing.assert_array_equal(got["xF_next"], got["xC_next"])
+
+
+def test_reduced_config2_shape(B):
+    """Llama-3-8B head layout (g = 4, hd = 128) at reduced width and length: several tiles in
+    every dimension and ragged tails."""
+    cfg = small_cfg("bf16", hd=128, Hq=8, Hkv=2, d=512, F=448, L=5000, N=200, window=32, budget=500, n_obs=32,
+                    kept_rule="window_topk")
+    lay = H.make_problem(cfg)
+    for engine in engines(B, cfg):
+        check_build(B, cfg, lay, lay["x0"], lay["x0"], [0, cfg.N], 0.1, engine)
+
+
+def test_two_layer_stack_matches_oracle_chain(B):
+    import torch
+    cfg = small_cfg("bf16", n_layers=2, N=64)
+    lays = [H.make_problem(cfg, layer=l) for l in range(2)]
+    x0 = lays[0]["x0"]
+    xF, xC = x0.astype(np.float64), x0.astype(np.float64)
+    refs = []
+    for l in range(2):
+        o = H.run_oracle(cfg, lays[l], xF, xC, [0, cfg.N], 0.1)
+        refs.append(o)
+        xF, xC = o["xF_next"], o["xC_next"]
+    for engine in engines(B, cfg):
+        ctx = B.PkvContext(B.dims_from_config(cfg), engine=engine)
+        dl = []
+        for l in range(2):
+            off, idx = gen.kept_to_csr(lays[l]["kept"])
+            kv = B.to_device({"K": lays[l]["K"], "V": lays[l]["V"]}, cfg.dtype)
+            dl.append({"w": B.to_device(lays[l]["weights"], cfg.dtype), "K": kv["K"], "V": kv["V"],
+                       "head_off": off, "idx": torch.from_numpy(idx).cuda()})
+        xt = torch.from_numpy(x0).cuda()
+        out = ctx.build_stack(dl, xt, xt, [0, cfg.N], cfg.L, 0.1)
+        for l in range(2):
+            assert H.rel_fro(out["dW"][l].cpu().numpy(), refs[l]["dW"]) <= DW_TOL
+        assert H.rel_fro(out["xC_final"].cpu().numpy(), refs[1]["xC_next"]) <= 1e-3
+        ctx.close()
+
+
+# ------------------------------------------------------------------ boundary
+
+def test_boundary_rejects_bad_arguments(B):
+    import torch
+    cfg = small_cfg("bf16")
+    with pytest.raises(B.PkvError) as ei:
+        B.PkvContext(B.dims_from_config(gen.scaled_config(cfg, hd=96)), engine=B.ENGINE_SIMT)
+    assert ei.value.code == -2
+    with pytest.raises(B.PkvError) as ei:
+        B.PkvContext(B.dims_from_config(gen.scaled_config(cfg, F=9000)), engine=B.ENGINE_SIMT)
+    assert ei.value.code == -2
+    lay = H.make_problem(cfg)
+    x = lay["x0"]
+    for lam in (0.0, -1.0, float("nan"), float("inf")):
+        with pytest.raises(B.PkvError) as ei:
+            gpu_build(B, cfg, lay, x, x, [0, cfg.N], lam, B.ENGINE_SIMT)
+        assert ei.value.code == -1
+    for chunks in ([0, 10, 10, cfg.N], [1, cfg.N], [0, cfg.N - 1]):
+        with pytest.raises(B.PkvError) as ei:
+            gpu_build(B, cfg, lay, x, x, chunks, 0.1, B.ENGINE_SIMT)
+        assert ei.value.code == -1
+    bad = dict(lay)
+    bad["kept"] = [lay["kept"][0].copy(), lay["kept"][1].copy()]
+    bad["kept"][1][7] = bad["kept"][1][6]
+    with pytest.raises(B.PkvError) as ei:
+        gpu_build(B, cfg, bad, x, x, [0, cfg.N], 0.1, B.ENGINE_SIMT)
+    assert ei.value.code == -3 and ei.value.info["err_info"] == (1, 7)
