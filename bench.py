@@ -1,0 +1,335 @@
+#!/usr/bin/env python
+"""Benchmark of PatchKV patch construction (one block of Algorithm 1 per step).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference]
+
+A step is one pass of the whole per-block path (index check + compaction, teacher and student
+forward, targets, statistics, ridge solve, next states, merge) over one synthetic context.
+Prints ONE JSON line.  With --impl reference the fp64 CPU oracle is timed on a bounded sample
+of the same workload instead (host cores; a deliberately slow baseline).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_39329_b200 import inputs as gen  # noqa: E402
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                    "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    "sm_max_mhz": float(d.get("sm_max_mhz", 1965.0)), "source": "measured"}
+        except Exception:
+            pass
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
+
+
+def stage_work(cfg, b_sum, b_max):
+    """Algorithmic work per stage of one block: (name, flops, bytes, bound)."""
+    N, d, F, L, Dq, Dkv, hd = cfg.N, cfg.d, cfg.F, cfg.L, cfg.Dq, cfg.Dkv, cfg.hd
+    eb = 2 if cfg.dtype == "bf16" else 4
+    b_mean = b_sum / cfg.Hkv
+    return [
+        ("S0 index check + compaction", 0.0, 2.0 * (2.0 * b_sum * hd * eb), "hbm"),
+        ("S1-S2 norm + QKV + RoPE", 4.0 * N * d * (Dq + 2 * Dkv), 0.0, "tensor"),
+        ("S3 dual-cache attention", 4.0 * N * L * Dq + 4.0 * N * b_mean * Dq + 4.0 * N * N * Dq,
+         2.0 * (L + b_mean) * Dkv * eb, "tensor"),
+        ("S4 o-proj + residual", 4.0 * N * Dq * d, 0.0, "tensor"),
+        ("S5 norm + gate/up + SiLU", 8.0 * N * d * F, 0.0, "tensor"),
+        ("S6 targets", 2.0 * N * F * d, 0.0, "tensor"),
+        ("S7 Gram + cross statistics", float(N) * F * (F + 1) + 2.0 * N * F * d, 4.0 * (F * F + F * d), "tensor"),
+        ("S8 ridge solve", F ** 3 / 3.0 + 2.0 * F * F * d, 0.0, "alu"),
+        ("S9 next states", 4.0 * N * F * d, 0.0, "tensor"),
+    ]
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for n, v in zip(names, r[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_inputs(cfg, layer=0):
+    lay = gen.gen_layer(cfg, layer)
+    lay["x0"] = gen.gen_reference(cfg)
+    return lay
+
+
+def oracle_sample(cfg, lay, n_sample):
+    """Times the fp64 oracle on the first n_sample reference tokens (full cache, full d x F solve) and
+    scales the token-proportional part to the workload's N.  Returns (ms per context, seconds spent)."""
+    from oracle import pkv_oracle as orc
+    sub = gen.scaled_config(cfg, N=n_sample)
+    x = lay["x0"][:n_sample]
+    t0 = time.perf_counter()
+    out = orc.build_patch(lay["weights"], lay["K"], lay["V"], lay["kept"], x, x, [0, n_sample], cfg.L, cfg.lam0, sub,
+                          keep_intermediates=True)
+    t1 = time.perf_counter()
+    lam = out["lam"]
+    orc.ridge_solve(out["S_H"], out["S_T"], lam)
+    t2 = time.perf_counter()
+    t_solve = t2 - t1
+    t_fwd = (t1 - t0) - t_solve
+    est = t_fwd * (cfg.N / n_sample) + t_solve
+    return est * 1e3, t2 - t0
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = gen.benchmark_config(args.config)
+    lay = build_inputs(cfg)
+    n_sample = min(cfg.N, args.ref_sample)
+    cores = os.cpu_count() or 1
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(cfg, lay, max(n_sample // 4, 4))
+    vals, spent = [], 0.0
+    for _ in range(args.steps):
+        v, s = oracle_sample(cfg, lay, n_sample)
+        vals.append(v); spent += s
+    val = float(np.mean(vals))
+    sample = ("fp64 numpy oracle on the first %d of %d reference tokens (full L=%d cache, full %dx%d solve), "
+              "token-proportional part scaled by %d/%d" % (n_sample, cfg.N, cfg.L, cfg.d, cfg.F, cfg.N, n_sample))
+    line = {"impl": "reference", "metric": "patch_build_ms_per_context", "value": val, "unit": "ms",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": val,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(cfg, lay),
+            "cpu_baseline": {"value": val, "unit": "ms", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_config(cfg, lay):
+    b = [int(len(k)) for k in lay["kept"]]
+    return {"workload": "config %d: %s" % (cfg.cfg_id, cfg.name), "layers_per_step": 1, "d": cfg.d, "F": cfg.F,
+            "Hq": cfg.Hq, "Hkv": cfg.Hkv, "hd": cfg.hd, "L": cfg.L, "n_ref": cfg.N, "kept_per_head": b[0],
+            "lambda0": cfg.lam0, "lambda_mode": "paper (Eq. 7)", "seed": cfg.seed,
+            "l2": "inputs (weights + caches, >300 MB) exceed L2 and a 512 MB buffer is written between steps"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--impl", default="ours")
+    ap.add_argument("--engine", default="auto", choices=["auto", "simt"])
+    ap.add_argument("--ref-sample", type=int, default=32)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_39329_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = measured_peaks()
+    cfg = gen.benchmark_config(args.config)
+    if world > 1:      # replicas only: every rank builds the patch of its own context
+        cfg = gen.scaled_config(cfg, seed=cfg.seed + rank)
+    lay = build_inputs(cfg)
+    b_list = [len(k) for k in lay["kept"]]
+    off, idx = gen.kept_to_csr(lay["kept"])
+
+    engine = B.ENGINE_SIMT if args.engine == "simt" else B.ENGINE_AUTO
+    ctx = B.PkvContext(B.dims_from_config(cfg, b_max=max(b_list)), engine=engine)
+    w = B.to_device(lay["weights"], cfg.dtype)
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    idx_t = torch.from_numpy(idx).cuda()
+    x_t = torch.from_numpy(lay["x0"]).cuda()
+    W_merged = w["Wdown"].clone()
+    dW = torch.empty((cfg.d, cfg.F), dtype=torch.float32, device="cuda")
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    chunk_off = [0, cfg.N]
+
+    def step():
+        out = ctx.build_patch(w, kv["K"], kv["V"], off, idx_t, x_t, x_t, chunk_off, cfg.L, cfg.lam0, B.LAMBDA_PAPER,
+                              True, dW=dW)
+        ctx.merge(W_merged, dW)
+        return out
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    l0 = ctx.launch_count()
+    times = []
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)           # L2 flush, outside the timed events
+        ev[i][0].record()
+        step()
+        ev[i][1].record()
+    barrier()
+    clocks = sampler.stop()
+    launches = ctx.launch_count() - l0 + args.steps      # + one merge kernel per step
+    times = [a.elapsed_time(b) for a, b in ev]
+    ms = float(sum(times) / len(times))
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # per-stage device times (separate pass with the library's stage events)
+    ctx.set_timing(True)
+    stage_acc = None
+    for i in range(5):
+        flush.fill_(i)
+        st = step()["stats"]["stage_ms"][:9]
+        stage_acc = st if stage_acc is None else [a + b for a, b in zip(stage_acc, st)]
+    ctx.set_timing(False)
+    stage_ms = [a / 5 for a in stage_acc]
+    work = stage_work(cfg, sum(b_list), max(b_list))
+    total_flops = sum(wk[1] for wk in work)
+
+    # end to end through the public call with host buffers: H2D of every input, D2H of the patch
+    host = {k: v.cpu().pin_memory() for k, v in {**w, "K": kv["K"], "V": kv["V"], "idx": idx_t, "x": x_t}.items()}
+    dev = {k: torch.empty_like(v, device="cuda") for k, v in host.items()}
+    dW_host = torch.empty((cfg.d, cfg.F), dtype=torch.float32).pin_memory()
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+    d2h = dW_host.numel() * 4
+
+    def e2e_step():
+        for k in host:
+            dev[k].copy_(host[k], non_blocking=True)
+        wd = {k: dev[k] for k in w}
+        ctx.build_patch(wd, dev["K"], dev["V"], off, dev["idx"], dev["x"], dev["x"], chunk_off, cfg.L, cfg.lam0,
+                        B.LAMBDA_PAPER, True, dW=dW)
+        dW_host.copy_(dW, non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_step()
+    barrier()
+    e2e_n = max(3, min(args.steps, 5))
+    t0 = time.perf_counter()
+    for _ in range(e2e_n):
+        e2e_step()
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_n
+    if world > 1:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # roofline of the dominant stage
+    dom = int(np.argmax(stage_ms))
+    name, fl, by, bound = work[dom]
+    dur = stage_ms[dom] * 1e-3
+    if bound == "tensor":
+        peak, unit, ach = peaks["bf16_tflops_sustained"], "TFLOP/s", fl / dur / 1e12
+        peak_note = "bf16 dense, sustained, %s" % peaks["source"]
+    elif bound == "alu":
+        peak = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+        unit, ach = "TFLOP/s", fl / dur / 1e12
+        peak_note = "fp32 FMA: 148 SMs x 128 lanes x 2 x %.0f MHz (derived)" % peaks["sm_max_mhz"]
+    else:
+        peak, unit, ach = peaks["hbm_gbs"], "GB/s", by / dur / 1e9
+        peak_note = "HBM copy, %s" % peaks["source"]
+    roofline = {"kernel": name, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                "traffic": None, "peak_note": peak_note, "stage_ms": stage_ms[dom]}
+    stages = [{"stage": wk[0], "ms": round(t, 4), "algorithmic_tflops": (wk[1] / (t * 1e-3) / 1e12) if t > 0 else None}
+              for wk, t in zip(work, stage_ms)]
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        n_sample = min(cfg.N, args.ref_sample)
+        v, spent = oracle_sample(cfg, lay, n_sample)
+        cpu = {"value": v, "unit": "ms", "cores": os.cpu_count() or 1, "kind": "oracle",
+               "sample": "fp64 numpy oracle, first %d of %d reference tokens, full cache and full solve, token part "
+                         "scaled by %d/%d; %.1f s of CPU wall time" % (n_sample, cfg.N, cfg.N, n_sample, spent)}
+
+    value = ms / world
+    line = {"metric": "patch_build_ms_per_context", "value": value, "unit": "ms", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+            "data": "synthetic", "config": workload_config(cfg, lay),
+            "engine": "simt-fp32" if engine == B.ENGINE_SIMT else "tcgen05",
+            "algorithmic_tflops": total_flops / (ms * 1e-3) / 1e12,
+            "frac_bf16_peak": total_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+            "roofline": roofline, "stages": stages, "cpu_baseline": cpu, "clocks": clocks,
+            "e2e": {"value": e2e_ms / world, "unit": "ms", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
+            "gpu_launches": int(launches), "peaks": peaks}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
