@@ -526,7 +526,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
             gemm_tn_simt(lc, b.hF, F, w->Wdown, F, bf, next->xF_next, d, N, d, F, 1.f, b.zF, d, false);
             gemm_tn_simt(lc, b.hC, F, dW, F, false, b.D, d, N, d, F, -1.f, b.R, d, false);
         } else {
-            pkv::tc_next_states(lc, &b.tc, &c->dims, N, w->Wdown, dW, b.zF, b.R, next->xF_next, b.D);
+            pkv::tc_next_states(lc, &b.tc, &c->dims, N, w->Wdown, dW, b.zF, b.R, next->xF_next, b.D, b.status);
         }
         sumsq(lc, b.D, (int64_t)N * d, &b.status->res_fro2);
         sub_f32(lc, next->xF_next, b.D, (int64_t)N * d, next->xC_next);

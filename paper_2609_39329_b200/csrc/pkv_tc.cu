@@ -1,18 +1,284 @@
-// Tensor-core engine: not built yet in this file's first form; creation of a bf16 context
-// with PKV_ENGINE_AUTO reports PKV_ERR_UNSUPPORTED (there is no silent fallback).
+// Tensor-core engine: stage sequence of one block for bf16 weights and caches.
+//
+// Precision plan.  Weights and caches are bf16 as given.  Every fp32 activation that feeds a
+// tensor-core product is carried as a bf16 pair (hi, lo) and multiplied in two passes against
+// the same bf16 weight tile (three passes when both factors are fp32), all accumulating in
+// fp32 tensor memory; differences (dA, dz, dh) are formed in fp32 before any rounding so that
+// the target T = W dh + dz of Eq. 5 does not inherit the rounding of two nearly equal streams.
+#include <math.h>
+
 #include "pkv_tc.h"
 
 namespace pkv {
 
-int tc_supported(const pkv_dims*, int, int) { return PKV_ERR_UNSUPPORTED; }
-size_t tc_carve(TcBuffers*, char*, size_t off, const pkv_dims*) { return off; }
-int tc_init(TcBuffers*, const pkv_dims*) { return PKV_ERR_UNSUPPORTED; }
-int tc_forward(const Lc&, TcBuffers*, const pkv_dims*, const TcForwardArgs&) { return PKV_ERR_UNSUPPORTED; }
-int tc_attention(const Lc&, TcBuffers*, const pkv_dims*, const AttnArgs&, DevStatus*) { return PKV_ERR_UNSUPPORTED; }
-void tc_gram(const Lc&, TcBuffers*, const pkv_dims*, const float*, const float*, int, float*, float*, bool,
-             DevStatus*) {}
-void tc_ridge_solve(const Lc&, TcBuffers*, const SolveWs&, int, int, float*, DevStatus*) {}
-void tc_next_states(const Lc&, TcBuffers*, const pkv_dims*, int, const void*, const float*, const float*,
-                    const float*, float*, float*) {}
+// ---------------------------------------------------------------------------------------------
+// element-wise kernels producing bf16 pairs
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void split2(float v, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(v);
+    lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+__global__ void __launch_bounds__(256) k_rmsnorm_split(const float* __restrict__ x0, const float* __restrict__ x1,
+                                                       int N, int d, const float* __restrict__ gain, float eps,
+                                                       __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+    __shared__ float red[32];
+    int r = blockIdx.x;
+    const float* x = (r < N) ? x0 + (size_t)r * d : x1 + (size_t)(r - N) * d;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        float v = x[c];
+        ss += v * v;
+    }
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float t = (threadIdx.x < 8) ? red[threadIdx.x] : 0.f;
+    if (threadIdx.x < 32) {
+        for (int o = 4; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (threadIdx.x == 0) red[0] = t;
+    }
+    __syncthreads();
+    float inv = 1.0f / sqrtf(red[0] / (float)d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        float v = x[c] * gain[c] * inv;
+        __nv_bfloat16 h, l;
+        split2(v, h, l);
+        hi[(size_t)r * d + c] = h;
+        lo[(size_t)r * d + c] = l;
+    }
+}
+
+__global__ void __launch_bounds__(256) k_split(const float* __restrict__ a, size_t n, __nv_bfloat16* __restrict__ hi,
+                                               __nv_bfloat16* __restrict__ lo) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    __nv_bfloat16 h, l;
+    split2(a[i], h, l);
+    hi[i] = h;
+    lo[i] = l;
+}
+
+static void split(const Lc& lc, const float* a, size_t n, Pair p) {
+    if (!n) return;
+    k_split<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(a, n, p.hi, p.lo);
+    lc.count();
+}
+
+__device__ __forceinline__ float silu_f(float t) { return t / (1.0f + expf(-t)); }
+
+// gu [2N][2F] (gate | up) -> hF, hC (fp32 + pairs), dh = hF - hC (pair)
+__global__ void __launch_bounds__(256) k_swiglu_split(const float* __restrict__ gu, int N, int F,
+                                                      float* __restrict__ hF32, float* __restrict__ hC32, Pair hF,
+                                                      Pair hC, Pair dh) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t n = (size_t)N * F;
+    if (i >= n) return;
+    size_t r = i / F, c = i % F;
+    const float* a = gu + r * 2 * F;
+    const float* b = gu + (r + N) * 2 * F;
+    float f = silu_f(a[c]) * a[F + c];
+    float s = silu_f(b[c]) * b[F + c];
+    hF32[i] = f;
+    hC32[i] = s;
+    split2(f, hF.hi[i], hF.lo[i]);
+    split2(s, hC.hi[i], hC.lo[i]);
+    split2(f - s, dh.hi[i], dh.lo[i]);
+}
+
+// in [rows][cols] fp32 -> out pair [cols][ldo] (token-contiguous operands of the statistics)
+__global__ void k_transpose_split(const float* __restrict__ in, int rows, int cols, int ldo, Pair out) {
+    __shared__ float t[32][33];
+    int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        int r = r0 + j, c = c0 + threadIdx.x;
+        if (r < rows && c < cols) t[j][threadIdx.x] = in[(size_t)r * cols + c];
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        int c = c0 + j, r = r0 + threadIdx.x;
+        if (r < rows && c < cols) {
+            __nv_bfloat16 h, l;
+            split2(t[threadIdx.x][j], h, l);
+            out.hi[(size_t)c * ldo + r] = h;
+            out.lo[(size_t)c * ldo + r] = l;
+        }
+    }
+}
+
+static void transpose_split(const Lc& lc, const float* in, int rows, int cols, int ldo, Pair out) {
+    dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
+    k_transpose_split<<<grid, block, 0, lc.st>>>(in, rows, cols, ldo, out);
+    lc.count();
+}
+
+// ---------------------------------------------------------------------------------------------
+// helpers
+// ---------------------------------------------------------------------------------------------
+// C = alpha * (A_hi + A_lo) W^T (+ addend): fp32 activation pair against a bf16 weight [Nn][K].
+static int gemm_act_weight(const Lc& lc, Pair A, long long lda, const void* W, long long ldw, float* C,
+                           long long ldc, int M, int Nn, int K, float alpha, const float* addend, long long ldadd,
+                           DevStatus* st) {
+    TcGemm g{};
+    g.A[0] = A.hi; g.A[1] = A.lo; g.lda[0] = g.lda[1] = lda;
+    g.B[0] = g.B[1] = (const __nv_bfloat16*)W; g.ldb[0] = g.ldb[1] = ldw;
+    g.npass = 2; g.C = C; g.ldc = ldc; g.M = M; g.N = Nn; g.K = K; g.alpha = alpha;
+    g.addend = addend; g.ldadd = ldadd;
+    return gemm_tc(lc, g, st);
+}
+
+// C = alpha * (A_hi + A_lo)(B_hi + B_lo)^T without the lo*lo term (+ addend) (+ C).
+static int gemm_pair_pair(const Lc& lc, Pair A, long long lda, Pair B, long long ldb, float* C, long long ldc, int M,
+                          int Nn, int K, float alpha, const float* addend, long long ldadd, bool accumulate,
+                          DevStatus* st) {
+    TcGemm g{};
+    g.A[0] = A.hi; g.B[0] = B.hi;
+    g.A[1] = A.hi; g.B[1] = B.lo;
+    g.A[2] = A.lo; g.B[2] = B.hi;
+    for (int i = 0; i < 3; ++i) { g.lda[i] = lda; g.ldb[i] = ldb; }
+    g.npass = 3; g.C = C; g.ldc = ldc; g.M = M; g.N = Nn; g.K = K; g.alpha = alpha;
+    g.addend = addend; g.ldadd = ldadd; g.accumulate = accumulate;
+    return gemm_tc(lc, g, st);
+}
+
+int tc_supported(const pkv_dims* d, int cc_major, int cc_minor) {
+    (void)cc_minor;
+    if (cc_major != 10) return PKV_ERR_UNSUPPORTED;                      // tcgen05 / TMEM: sm_100 only
+    if (d->dtype != PKV_BF16) return PKV_ERR_UNSUPPORTED;
+    if (d->d % 8 || d->F % 8) return PKV_ERR_UNSUPPORTED;                // 16-byte TMA row strides
+    if (!tc_encode_available()) return PKV_ERR_UNSUPPORTED;
+    return PKV_OK;
+}
+
+struct Carver2 {
+    char* base;
+    size_t off;
+    template <typename T>
+    T* take(size_t n) {
+        off = (off + 255) & ~(size_t)255;
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+    Pair pair(size_t n) {
+        Pair p;
+        p.hi = take<__nv_bfloat16>(n);
+        p.lo = take<__nv_bfloat16>(n);
+        return p;
+    }
+};
+
+size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d) {
+    Carver2 c{base, off};
+    const size_t N = d->N_max, dm = d->d, F = d->F, Dq = (size_t)d->Hq * d->hd, Dkv = (size_t)d->Hkv * d->hd;
+    t->ldT = (int)((N + 7) / 8 * 8);
+    t->u = c.pair(2 * N * dm);
+    t->a = c.pair(2 * N * Dq);
+    t->hF = c.pair(N * F);
+    t->hC = c.pair(N * F);
+    t->dh = c.pair(N * F);
+    t->XT = c.pair(F * (size_t)t->ldT);
+    t->RT = c.pair(dm * (size_t)t->ldT);
+    t->dW = c.pair(dm * F);
+    t->qkv = c.take<float>(2 * N * (Dq + 2 * Dkv));
+    t->o = c.take<float>(2 * N * dm);
+    t->gu = c.take<float>(2 * N * 2 * F);
+    t->dAbuf = nullptr;
+    t->q = c.pair(2 * N * Dq);
+    t->kn = c.take<__nv_bfloat16>(2 * N * Dkv);
+    t->vn = c.take<__nv_bfloat16>(2 * N * Dkv);
+    return c.off;
+}
+
+int tc_init(TcBuffers*, const pkv_dims*) { return PKV_OK; }
+
+static void mark(const TcForwardArgs& a, const Lc& lc, int stage) {
+    if (a.ev) cudaEventRecord(a.ev[stage], lc.st);
+}
+
+void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, const float* R, int n, float* S_H,
+             float* S_T, bool accumulate, DevStatus* status) {
+    const int F = d->F, dm = d->d;
+    transpose_split(lc, X, n, F, t->ldT, t->XT);
+    transpose_split(lc, R, n, dm, t->ldT, t->RT);
+    gemm_pair_pair(lc, t->XT, t->ldT, t->XT, t->ldT, S_H, F, F, F, n, 1.f, nullptr, 0, accumulate, status);
+    gemm_pair_pair(lc, t->RT, t->ldT, t->XT, t->ldT, S_T, F, dm, F, n, 1.f, nullptr, 0, accumulate, status);
+}
+
+int tc_attention(const Lc& lc, TcBuffers*, const pkv_dims*, const AttnArgs& a, DevStatus*) {
+    attention_simt(lc, a);
+    attention_combine(lc, a);
+    return PKV_OK;
+}
+
+void tc_ridge_solve(const Lc& lc, TcBuffers*, const SolveWs& ws, int F, int d, float* dW, DevStatus* status) {
+    ridge_solve_simt(lc, ws, F, d, dW, status);
+}
+
+int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a) {
+    const int N = a.N, d = D->d, F = D->F, hd = D->hd;
+    const int Dq = D->Hq * hd, Dkv = D->Hkv * hd, QKV = Dq + 2 * Dkv;
+    const pkv_block_weights* w = a.w;
+    DevStatus* st = a.status;
+    int rc;
+    // S1-S2: both streams stacked, rows [0,N) teacher, [N,2N) student
+    k_rmsnorm_split<<<2 * N, 256, 0, lc.st>>>(a.xF, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo);
+    lc.count();
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wq, d, t->qkv, QKV, 2 * N, Dq, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wk, d, t->qkv + Dq, QKV, 2 * N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wv, d, t->qkv + Dq + Dkv, QKV, 2 * N, Dkv, d, 1.f, nullptr, 0, st)))
+        return rc;
+    rope_table(lc, a.tok_cs, N, hd, a.pos0, D->rope_theta, a.rope_tab);
+    rope_apply(lc, t->qkv, QKV, 0, D->Hq + D->Hkv, hd, 2 * N, N, a.rope_tab);
+    mark(a, lc, 2);
+    // S3
+    AttnArgs at{};
+    at.q = t->qkv; at.ldq = QKV; at.k_new = t->qkv + Dq; at.v_new = t->qkv + Dq + Dkv; at.ldkv = QKV;
+    at.K = a.full->K; at.V = a.full->V; at.Kc = a.Kc; at.Vc = a.Vc; at.bias = a.bias;
+    at.head_off = a.head_off; at.tok_cs = a.tok_cs;
+    at.N = N; at.Hq = D->Hq; at.Hkv = D->Hkv; at.hd = hd; at.L = D->L; at.elem_bytes = 2;
+    at.kv_split = a.kv_split;
+    at.nsplitF = (D->L + N + a.kv_split - 1) / a.kv_split;
+    at.nsplitC = (a.max_b + N + a.kv_split - 1) / a.kv_split;
+    if (at.nsplitC < 1) at.nsplitC = 1;
+    at.part_m = a.part_m; at.part_l = a.part_l; at.part_O = a.part_O;
+    at.aF = a.aF; at.aC = a.aC; at.dA = a.aF + (size_t)N * Dq;
+    if ((rc = tc_attention(lc, t, D, at, st))) return rc;
+    mark(a, lc, 3);
+    // S4: [aF; dA] Wo^T, then zF, dz, zC
+    split(lc, a.aF, (size_t)2 * N * Dq, t->a);
+    if ((rc = gemm_act_weight(lc, t->a, Dq, w->Wo, Dq, t->o, d, 2 * N, d, Dq, 1.f, nullptr, 0, st))) return rc;
+    oproj_epilogue(lc, a.xF, a.xC, t->o, N, d, a.zF, a.zC, a.dz);
+    mark(a, lc, 4);
+    // S5
+    k_rmsnorm_split<<<2 * N, 256, 0, lc.st>>>(a.zF, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo);
+    lc.count();
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wgate, d, t->gu, 2 * F, 2 * N, F, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wup, d, t->gu + F, 2 * F, 2 * N, F, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        size_t n = (size_t)N * F;
+        k_swiglu_split<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hF, t->hC, t->dh);
+        lc.count();
+    }
+    mark(a, lc, 5);
+    // S6: T = dh Wdown^T + dz   (Eq. 5)
+    if ((rc = gemm_act_weight(lc, t->dh, F, w->Wdown, F, a.R, d, N, d, F, 1.f, a.dz, d, st))) return rc;
+    sumsq(lc, a.R, (int64_t)N * d, &st->t_fro2);
+    mark(a, lc, 6);
+    // S7 (Eq. 9)
+    tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st);
+    mark(a, lc, 7);
+    return PKV_OK;
+}
+
+void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const void* Wdown, const float* dW,
+                    const float* zF, const float* R, float* xF_next, float* Dm, DevStatus* status) {
+    const int d = D->d, F = D->F;
+    // xF_next = zF + hF Wdown^T
+    gemm_act_weight(lc, t->hF, F, Wdown, F, xF_next, d, N, d, F, 1.f, zF, d, status);
+    // D = T - hC dW^T
+    split(lc, dW, (size_t)d * F, t->dW);
+    gemm_pair_pair(lc, t->hC, F, t->dW, F, Dm, d, N, d, F, -1.f, R, d, false, status);
+}
 
 }  // namespace pkv

@@ -1,12 +1,56 @@
 // Tensor-core engine (tcgen05 + TMEM + TMA, sm_100a): interface used by pkv_api.cu.
 #pragma once
 
+#include <cuda.h>
+
 #include "pkv_internal.h"
 
 namespace pkv {
 
+constexpr int kGemmMaxPass = 6;
+
+// C[M][N] = alpha * sum_p A[p][M][K] B[p][N][K]^T (+ addend) (+ C); bf16 operands, fp32 result.
+struct TcGemm {
+    const __nv_bfloat16* A[kGemmMaxPass];
+    long long lda[kGemmMaxPass];
+    const __nv_bfloat16* B[kGemmMaxPass];
+    long long ldb[kGemmMaxPass];
+    int npass;
+    float* C;
+    long long ldc;
+    int M, N, K;
+    float alpha;
+    const float* addend;
+    long long ldadd;
+    bool accumulate, lower_only;
+};
+int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status);
+bool tc_encode_available();
+int tc_make_map_2d(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows);
+int tc_make_map_3d(CUtensorMap* m, const void* ptr, uint64_t d2, uint64_t rows, uint64_t cols, uint64_t ld1,
+                   uint64_t ld2, uint32_t box_rows);
+
+// bf16 hi/lo pairs of fp32 activations: v ~= hi + lo with hi = bf16(v), lo = bf16(v - hi).
+struct Pair {
+    __nv_bfloat16* hi;
+    __nv_bfloat16* lo;
+};
+
 struct TcBuffers {
-    int ready;
+    int ldT;            // leading dimension of the token-contiguous (transposed) operands
+    Pair u;             // [2N][d]   norm outputs (attention norm, then MLP norm)
+    Pair a;             // [2N][Dq]  [aF; dA]
+    Pair hF, hC, dh;    // [N][F]
+    Pair XT;            // [F][ldT]  student features, token-contiguous
+    Pair RT;            // [d][ldT]  targets, token-contiguous
+    Pair dW;            // [d][F]
+    float* qkv;         // [2N][Dq+2Dkv]
+    float* o;           // [2N][d]
+    float* gu;          // [2N][2F]
+    float* dAbuf;       // unused placeholder
+    Pair q;             // [2][Hq][N][hd]   rotated, pre-scaled queries for the attention kernel
+    __nv_bfloat16* kn;  // [2][Hkv][N][hd]  reference tokens' keys
+    __nv_bfloat16* vn;  // [2][Hkv][N][hd]  reference tokens' values
 };
 
 struct TcForwardArgs {
@@ -31,6 +75,6 @@ void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, cons
              float* S_T, bool accumulate, DevStatus* status);
 void tc_ridge_solve(const Lc& lc, TcBuffers* t, const SolveWs& ws, int F, int d, float* dW, DevStatus* status);
 void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* d, int N, const void* Wdown, const float* dW,
-                    const float* zF, const float* R, float* xF_next, float* D);
+                    const float* zF, const float* R, float* xF_next, float* D, DevStatus* status);
 
 }  // namespace pkv

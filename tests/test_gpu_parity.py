@@ -12,7 +12,7 @@ from tests import helpers as H
 
 pytestmark = pytest.mark.gpu
 
-TC_READY = False      # flipped when the tensor-core engine lands
+TC_READY = True       # flipped when the tensor-core engine lands
 ATTN_TOL = 2e-2
 DW_TOL = 5e-3
 
