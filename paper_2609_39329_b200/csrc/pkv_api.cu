@@ -380,9 +380,10 @@ static int end_call(pkv_ctx* c, pkv_stats* stats, const int32_t* head_off) {
 
 static AttnArgs attn_args(pkv_ctx* c, const float* q, int64_t ldq, const float* k_new, const float* v_new,
                           int64_t ldkv, const pkv_kv* full, const void* Kc, const void* Vc, const float* bias,
-                          int N, int max_b) {
+                          int N, int max_b, int total) {
     AttnArgs a;
     memset(&a, 0, sizeof(a));
+    a.total_kept = total; a.max_b = max_b;
     a.q = q; a.ldq = ldq; a.k_new = k_new; a.v_new = v_new; a.ldkv = ldkv;
     a.K = full->K; a.V = full->V; a.Kc = Kc; a.Vc = Vc; a.bias = bias;
     a.head_off = c->b.head_off; a.tok_cs = c->b.tok_cs;
@@ -481,7 +482,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         mark(c, ST_ATTN);
         // S3
         AttnArgs a = attn_args(c, b.qkv, QKV, b.qkv + Dq, b.qkv + Dq + Dkv, QKV, full, Kc, Vc,
-                               cb->idx ? nullptr : cb->bias, N, max_b);
+                               cb->idx ? nullptr : cb->bias, N, max_b, total);
         a.aF = b.a2; a.aC = b.aC; a.dA = b.a2 + (size_t)N * Dq;
         attention_simt(lc, a);
         attention_combine(lc, a);
@@ -506,7 +507,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
     } else {
         pkv::TcForwardArgs fa;
         fa.w = w; fa.full = full; fa.Kc = Kc; fa.Vc = Vc; fa.bias = cb->idx ? nullptr : cb->bias;
-        fa.xF = ref->xF; fa.xC = ref->xC; fa.N = N; fa.pos0 = ref->pos0; fa.max_b = max_b;
+        fa.xF = ref->xF; fa.xC = ref->xC; fa.N = N; fa.pos0 = ref->pos0; fa.max_b = max_b; fa.total_kept = total;
         fa.head_off = b.head_off; fa.tok_cs = b.tok_cs; fa.rope_tab = b.rope_tab;
         fa.zF = b.zF; fa.zC = b.zC; fa.dz = b.dz; fa.hF = b.hF; fa.hC = b.hC; fa.R = b.R;
         fa.S_H = b.S_H; fa.S_T = b.S_T; fa.status = b.status;
@@ -615,7 +616,7 @@ extern "C" int pkv_attention(pkv_ctx* c, const float* q, const float* k_new, con
     upload_meta(c, cb->head_off, N, n_chunks, chunk_off);
     const void *Kc, *Vc;
     stage_compact(c, lc, full, cb, total, &Kc, &Vc);
-    AttnArgs a = attn_args(c, q, Dq, k_new, v_new, Dkv, full, Kc, Vc, cb->idx ? nullptr : cb->bias, N, max_b);
+    AttnArgs a = attn_args(c, q, Dq, k_new, v_new, Dkv, full, Kc, Vc, cb->idx ? nullptr : cb->bias, N, max_b, total);
     a.aF = aF; a.aC = aC; a.dA = dA;
     if (c->engine == PKV_ENGINE_SIMT) {
         attention_simt(lc, a);

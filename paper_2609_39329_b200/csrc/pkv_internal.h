@@ -57,6 +57,7 @@ struct AttnArgs {
     const int32_t* tok_cs;                // device [N] chunk start of each token
     int N, Hq, Hkv, hd, L, elem_bytes;
     int kv_split, nsplitF, nsplitC;
+    int total_kept, max_b;                // rows of the compact cache (all heads), largest head
     float* part_m; float* part_l; float* part_O;   // [nsplit][Hkv][N*g] and [..][hd]
     float* aF; float* aC; float* dA;      // [N][Hq*hd]
 };

@@ -187,6 +187,13 @@ size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d) {
     t->q = c.pair(2 * N * Dq);
     t->kn = c.take<__nv_bfloat16>(2 * N * Dkv);
     t->vn = c.take<__nv_bfloat16>(2 * N * Dkv);
+    int tps, nF, nC;
+    tc_attn_plan(d, d->N_max, d->b_max, &tps, &nF, &nC);
+    const size_t rows = N * (d->Hq / d->Hkv);
+    const size_t nsp = (size_t)nF + nC;
+    t->part_m = c.take<float>(nsp * d->Hkv * rows);
+    t->part_l = c.take<float>(nsp * d->Hkv * rows);
+    t->part_O = c.take<float>(nsp * d->Hkv * rows * d->hd);
     return c.off;
 }
 
@@ -205,10 +212,8 @@ void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, cons
     gemm_pair_pair(lc, t->RT, t->ldT, t->XT, t->ldT, S_T, F, dm, F, n, 1.f, nullptr, 0, accumulate, status);
 }
 
-int tc_attention(const Lc& lc, TcBuffers*, const pkv_dims*, const AttnArgs& a, DevStatus*) {
-    attention_simt(lc, a);
-    attention_combine(lc, a);
-    return PKV_OK;
+int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status) {
+    return attention_tc(lc, t, d, a, nullptr, status);
 }
 
 void tc_ridge_solve(const Lc& lc, TcBuffers*, const SolveWs& ws, int F, int d, float* dW, DevStatus* status) {
@@ -229,7 +234,6 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     if ((rc = gemm_act_weight(lc, t->u, d, w->Wv, d, t->qkv + Dq + Dkv, QKV, 2 * N, Dkv, d, 1.f, nullptr, 0, st)))
         return rc;
     rope_table(lc, a.tok_cs, N, hd, a.pos0, D->rope_theta, a.rope_tab);
-    rope_apply(lc, t->qkv, QKV, 0, D->Hq + D->Hkv, hd, 2 * N, N, a.rope_tab);
     mark(a, lc, 2);
     // S3
     AttnArgs at{};
@@ -237,13 +241,10 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     at.K = a.full->K; at.V = a.full->V; at.Kc = a.Kc; at.Vc = a.Vc; at.bias = a.bias;
     at.head_off = a.head_off; at.tok_cs = a.tok_cs;
     at.N = N; at.Hq = D->Hq; at.Hkv = D->Hkv; at.hd = hd; at.L = D->L; at.elem_bytes = 2;
-    at.kv_split = a.kv_split;
-    at.nsplitF = (D->L + N + a.kv_split - 1) / a.kv_split;
-    at.nsplitC = (a.max_b + N + a.kv_split - 1) / a.kv_split;
-    if (at.nsplitC < 1) at.nsplitC = 1;
-    at.part_m = a.part_m; at.part_l = a.part_l; at.part_O = a.part_O;
+    at.total_kept = a.total_kept; at.max_b = a.max_b;
     at.aF = a.aF; at.aC = a.aC; at.dA = a.aF + (size_t)N * Dq;
-    if ((rc = tc_attention(lc, t, D, at, st))) return rc;
+    // the S2 outputs are not rotated yet: the operand-preparation kernel applies RoPE
+    if ((rc = attention_tc(lc, t, D, at, a.rope_tab, st))) return rc;
     mark(a, lc, 3);
     // S4: [aF; dA] Wo^T, then zF, dz, zC
     split(lc, a.aF, (size_t)2 * N * Dq, t->a);

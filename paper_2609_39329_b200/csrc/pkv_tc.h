@@ -51,6 +51,9 @@ struct TcBuffers {
     Pair q;             // [2][Hq][N][hd]   rotated, pre-scaled queries for the attention kernel
     __nv_bfloat16* kn;  // [2][Hkv][N][hd]  reference tokens' keys
     __nv_bfloat16* vn;  // [2][Hkv][N][hd]  reference tokens' values
+    float* part_m;      // attention split partials [splits][Hkv][N*g]
+    float* part_l;
+    float* part_O;      // [splits][Hkv][N*g][hd]
 };
 
 struct TcForwardArgs {
@@ -58,7 +61,7 @@ struct TcForwardArgs {
     const pkv_kv* full;
     const void* Kc; const void* Vc; const float* bias;
     const float* xF; const float* xC;
-    int N, pos0, max_b, kv_split;
+    int N, pos0, max_b, total_kept, kv_split;
     const int32_t* head_off; const int32_t* tok_cs; float* rope_tab;
     float *zF, *zC, *dz, *hF, *hC, *R, *S_H, *S_T, *aF, *aC;
     float *part_m, *part_l, *part_O;
@@ -66,6 +69,10 @@ struct TcForwardArgs {
     cudaEvent_t* ev;    // stage marks (index = stage) or nullptr
 };
 
+void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, int* nsplitC);
+// q/k_new/v_new of `a` are fp32; rope_tab != nullptr rotates q and k on the way in.
+int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, const float* rope_tab,
+                 DevStatus* status);
 int tc_supported(const pkv_dims* d, int cc_major, int cc_minor);
 size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d);
 int tc_init(TcBuffers* t, const pkv_dims* d);

@@ -1,0 +1,504 @@
+// Dual-cache attention on the 5th-gen tensor cores (sm_100a).
+//
+// A CTA owns one tile of 128 query rows of one KV head of one stream (teacher: full cache,
+// student: compact cache) and one split of that stream's key sequence.  Query row r stands for
+// (token r / g, head kh*g + r % g), so one K/V tile serves the whole GQA group.  The key
+// sequence is the cache, in tiles of 128 rows, followed by the reference tokens' own keys, in
+// tiles of 128, visible causally inside the token's chunk.
+//
+//   warp 0    TMA producer: Q (bf16 hi + lo parts) once, then K and V tiles through 2-stage rings
+//   warp 1    one thread issues tcgen05.mma: S = Q_hi K^T + Q_lo K^T into a double-buffered TMEM
+//             accumulator, then O_tile = P V (V read as an MN-major operand straight from the
+//             cache layout) into a third accumulator
+//   warps 2-5 softmax: each thread owns one query row (one TMEM lane): row max, exp2, P -> bf16
+//             into 128B-swizzled smem for the PV product, running (m, l) in fp32, O kept in
+//             registers as alpha * O + O_tile
+// Partial (m, l, O) per split go to global memory; the combine kernel merges the splits of both
+// streams and forms dA = aF - aC in fp32.
+#include <cuda.h>
+#include <math.h>
+
+#include "pkv_ptx.cuh"
+#include "pkv_tc.h"
+
+namespace pkv {
+
+using namespace ptx;
+
+// ---------------------------------------------------------------------------------------------
+// operand preparation: RoPE (optional), query pre-scaling, bf16 hi/lo split, head-major layouts
+// ---------------------------------------------------------------------------------------------
+// q  -> hi/lo [2][Hkv][N*g][hd] (row = token*g + head-in-group), scaled by log2(e)/sqrt(hd)
+// k,v-> bf16  [2][Hkv][N][hd]
+__global__ void __launch_bounds__(256) k_attn_prep(const float* __restrict__ q, long long ldq,
+                                                   const float* __restrict__ k, const float* __restrict__ v,
+                                                   long long ldkv, const float* __restrict__ rope_tab, int N, int Hq,
+                                                   int Hkv, int hd, __nv_bfloat16* __restrict__ qhi,
+                                                   __nv_bfloat16* __restrict__ qlo, __nv_bfloat16* __restrict__ kn,
+                                                   __nv_bfloat16* __restrict__ vn) {
+    const int half = hd / 2;
+    const int heads = Hq + 2 * Hkv;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    size_t total = (size_t)2 * N * heads * half;
+    if (i >= total) return;
+    int c = (int)(i % half);
+    int h = (int)((i / half) % heads);
+    int row = (int)(i / ((size_t)half * heads));
+    int s = row / N, tok = row % N;
+    float co = 1.f, si = 0.f;
+    if (rope_tab) {
+        co = rope_tab[2 * ((size_t)tok * half + c)];
+        si = rope_tab[2 * ((size_t)tok * half + c) + 1];
+    }
+    if (h < Hq) {
+        const int g = Hq / Hkv;
+        const float* p = q + (size_t)row * ldq + (size_t)h * hd + c;
+        float lo = p[0], hi = p[half];
+        const float sc = 1.4426950408889634f * rsqrtf((float)hd);
+        float a = (lo * co - hi * si) * sc, b = (hi * co + lo * si) * sc;
+        int kh = h / g, hg = h % g;
+        size_t o = (((size_t)s * Hkv + kh) * ((size_t)N * g) + (size_t)tok * g + hg) * hd + c;
+        __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
+        qhi[o] = ah;
+        qhi[o + half] = bh;
+        qlo[o] = __float2bfloat16_rn(a - __bfloat162float(ah));
+        qlo[o + half] = __float2bfloat16_rn(b - __bfloat162float(bh));
+    } else if (h < Hq + Hkv) {
+        int kh = h - Hq;
+        const float* p = k + (size_t)row * ldkv + (size_t)kh * hd + c;
+        float lo = p[0], hi = p[half];
+        size_t o = (((size_t)s * Hkv + kh) * N + tok) * hd + c;
+        kn[o] = __float2bfloat16_rn(lo * co - hi * si);
+        kn[o + half] = __float2bfloat16_rn(hi * co + lo * si);
+    } else {
+        int kh = h - Hq - Hkv;
+        const float* p = v + (size_t)row * ldkv + (size_t)kh * hd + c;
+        size_t o = (((size_t)s * Hkv + kh) * N + tok) * hd + c;
+        vn[o] = __float2bfloat16_rn(p[0]);
+        vn[o + half] = __float2bfloat16_rn(p[half]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// the attention kernel
+// ---------------------------------------------------------------------------------------------
+struct alignas(64) AttnTcParams {
+    CUtensorMap mQhi, mQlo;   // {hd, N*g, 2*Hkv}
+    CUtensorMap mK, mV;       // {hd, L, Hkv}
+    CUtensorMap mKc, mVc;     // {hd, total kept rows}
+    CUtensorMap mKn, mVn;     // {hd, N, 2*Hkv}
+    const int32_t* head_off;
+    const int32_t* tok_cs;
+    const float* bias;
+    int N, g, Hkv, L, rows;
+    int tps, nsplitF, nsplitC;
+    float* part_m;
+    float* part_l;
+    float* part_O;
+    DevStatus* status;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// MN-major operand (V tile: rows = keys, 64 head-dim columns per 128-byte row, 128B swizzle):
+// 64-column blocks `lbo` bytes apart, 8-key groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t smem_addr, uint32_t lbo) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+template <int HD>
+struct AttnSmem {
+    static constexpr int kSub = HD / 64;              // 64-column sub-tiles per row
+    static constexpr int kTile = 128 * HD * 2;        // one 128-row operand tile, bytes
+    static constexpr int kQhi = 0;
+    static constexpr int kQlo = kTile;
+    static constexpr int kK = 2 * kTile;              // 2 stages
+    static constexpr int kV = 4 * kTile;              // 2 stages
+    static constexpr int kP = 6 * kTile;              // [2][128][64] bf16 = 32 KB
+    static constexpr int kBar = kP + 32768;
+    static constexpr int kNumBar = 16;
+    static constexpr int kTotal = kBar + kNumBar * 8 + 16 + 1024;
+};
+
+enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFULL = 9, B_SEMPTY = 11, B_PFULL = 13,
+       B_OFULL = 14, B_OEMPTY = 15 };
+
+template <int HD>
+__global__ void __launch_bounds__(192, 1) k_attn_tc(const __grid_constant__ AttnTcParams p) {
+    using S = AttnSmem<HD>;
+    if (p.status->code != 0) return;      // an earlier stage already failed: the call reports it
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - raw);
+    const uint32_t bars = base + S::kBar;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + S::kBar + S::kNumBar * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int kh = blockIdx.y;
+    const int z = blockIdx.z;
+    const int stream = (z >= p.nsplitF) ? 1 : 0;
+    const int split = stream ? z - p.nsplitF : z;
+    const int r0 = blockIdx.x * 128;
+
+    // key tiles of this CTA: cache tiles [0, nC) then reference-token tiles [nC, nC + nN)
+    int Lc, crow0;
+    if (stream == 0) {
+        Lc = p.L;
+        crow0 = 0;
+    } else {
+        crow0 = p.head_off[kh];
+        Lc = p.head_off[kh + 1] - crow0;
+    }
+    const int nC = (Lc + 127) >> 7;
+    const int tok_max = min(p.N - 1, (r0 + 127) / p.g);
+    const int nN = (tok_max >> 7) + 1;                 // later reference tiles are invisible to this row tile
+    const int t_begin = split * p.tps;
+    const int t_end = min(nC + nN, t_begin + p.tps);
+    const int ntiles = max(0, t_end - t_begin);
+
+    if (threadIdx.x == 0) {
+        mbar_init(bar(B_QFULL), 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(B_KFULL + i), 1);
+            mbar_init(bar(B_KEMPTY + i), 1);
+            mbar_init(bar(B_VFULL + i), 1);
+            mbar_init(bar(B_VEMPTY + i), 1);
+            mbar_init(bar(B_SFULL + i), 1);
+            mbar_init(bar(B_SEMPTY + i), 128);
+        }
+        mbar_init(bar(B_PFULL), 128);
+        mbar_init(bar(B_OFULL), 1);
+        mbar_init(bar(B_OEMPTY), 128);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = *tmem_slot;
+    const uint32_t tS[2] = {tbase, tbase + 128u};
+    const uint32_t tO = tbase + 256u;
+
+    if (warp == 0) {
+        if (lane == 0 && ntiles > 0) {
+            const int zq = stream * p.Hkv + kh;
+            mbar_expect_tx(bar(B_QFULL), 2 * S::kTile);
+#pragma unroll
+            for (int sb = 0; sb < S::kSub; ++sb) {
+                tma_load_3d(base + S::kQhi + sb * 16384, &p.mQhi, bar(B_QFULL), sb * 64, r0, zq);
+                tma_load_3d(base + S::kQlo + sb * 16384, &p.mQlo, bar(B_QFULL), sb * 64, r0, zq);
+            }
+            for (int j = 0; j < ntiles; ++j) {
+                const int t = t_begin + j;
+                const int st = j & 1;
+                const uint32_t ph = ((j >> 1) & 1) ^ 1;
+                if (!mbar_wait(bar(B_KEMPTY + st), ph, abort_flag, p.status, 10)) break;
+                mbar_expect_tx(bar(B_KFULL + st), S::kTile);
+                const uint32_t kd = base + S::kK + st * S::kTile;
+#pragma unroll
+                for (int sb = 0; sb < S::kSub; ++sb) {
+                    if (t >= nC) tma_load_3d(kd + sb * 16384, &p.mKn, bar(B_KFULL + st), sb * 64, (t - nC) * 128, zq);
+                    else if (stream == 0) tma_load_3d(kd + sb * 16384, &p.mK, bar(B_KFULL + st), sb * 64, t * 128, kh);
+                    else tma_load_2d(kd + sb * 16384, &p.mKc, bar(B_KFULL + st), sb * 64, crow0 + t * 128);
+                }
+                if (!mbar_wait(bar(B_VEMPTY + st), ph, abort_flag, p.status, 11)) break;
+                mbar_expect_tx(bar(B_VFULL + st), S::kTile);
+                const uint32_t vd = base + S::kV + st * S::kTile;
+#pragma unroll
+                for (int sb = 0; sb < S::kSub; ++sb) {
+                    if (t >= nC) tma_load_3d(vd + sb * 16384, &p.mVn, bar(B_VFULL + st), sb * 64, (t - nC) * 128, zq);
+                    else if (stream == 0) tma_load_3d(vd + sb * 16384, &p.mV, bar(B_VFULL + st), sb * 64, t * 128, kh);
+                    else tma_load_2d(vd + sb * 16384, &p.mVc, bar(B_VFULL + st), sb * 64, crow0 + t * 128);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && ntiles > 0) {
+            constexpr uint32_t idesc_qk = idesc_bf16(128, 128);
+            constexpr uint32_t idesc_pv = idesc_bf16(128, HD) | (1u << 16);      // B operand MN-major
+            auto issue_qk = [&](int j) {
+                const int st = j & 1;
+                const uint32_t kd = base + S::kK + st * S::kTile;
+#pragma unroll
+                for (int ps = 0; ps < 2; ++ps) {
+                    const uint32_t qd = base + (ps ? S::kQlo : S::kQhi);
+#pragma unroll
+                    for (int ks = 0; ks < HD / 16; ++ks) {
+                        const uint32_t off = (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u;
+                        mma_bf16_ss(tS[st], smem_desc_sw128(qd + off), smem_desc_sw128(kd + off), idesc_qk,
+                                    (ps | ks) != 0);
+                    }
+                }
+                mma_commit(bar(B_SFULL + st));
+                mma_commit(bar(B_KEMPTY + st));
+            };
+            bool ok = mbar_wait(bar(B_QFULL), 0, abort_flag, p.status, 20) &&
+                      mbar_wait(bar(B_KFULL), 0, abort_flag, p.status, 21);
+            if (ok) {
+                tc_fence_after();
+                issue_qk(0);
+            }
+            for (int j = 0; ok && j < ntiles; ++j) {
+                if (j + 1 < ntiles) {
+                    const int n = j + 1, st = n & 1;
+                    ok = mbar_wait(bar(B_KFULL + st), (n >> 1) & 1, abort_flag, p.status, 22) &&
+                         mbar_wait(bar(B_SEMPTY + st), ((n >> 1) & 1) ^ 1, abort_flag, p.status, 23);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_qk(n);
+                }
+                const int st = j & 1;
+                ok = mbar_wait(bar(B_VFULL + st), (j >> 1) & 1, abort_flag, p.status, 24) &&
+                     mbar_wait(bar(B_PFULL), j & 1, abort_flag, p.status, 25) &&
+                     mbar_wait(bar(B_OEMPTY), (j & 1) ^ 1, abort_flag, p.status, 26);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t vd = base + S::kV + st * S::kTile;
+                const uint32_t pd = base + S::kP;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {      // 16 keys per step
+                    const uint64_t da = smem_desc_sw128(pd + (uint32_t)(ks >> 2) * 16384u + (uint32_t)(ks & 3) * 32u);
+                    const uint64_t db = smem_desc_mn_sw128(vd + (uint32_t)ks * 2048u, 16384u);
+                    mma_bf16_ss(tO, da, db, idesc_pv, ks != 0);
+                }
+                mma_commit(bar(B_OFULL));
+                mma_commit(bar(B_VEMPTY + st));
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        const int row_in = q * 32 + lane;
+        const int r = r0 + row_in;
+        const bool valid = r < p.rows;
+        const int tok = valid ? r / p.g : 0;
+        const int cs = valid ? p.tok_cs[tok] : 0;
+        const uint32_t lane_off = (uint32_t)(q * 32) << 16;
+        float m = -INFINITY, l = 0.f, alpha_pend = 1.f;
+        float O[HD];
+#pragma unroll
+        for (int i = 0; i < HD; ++i) O[i] = 0.f;
+        bool ok = true;
+
+        auto accumulate_o = [&](int j) {
+            ok = mbar_wait(bar(B_OFULL), j & 1, abort_flag, p.status, 30);
+            if (!ok) return;
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < HD; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tO + lane_off + (uint32_t)c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) O[c0 + i] = fmaf(alpha_pend, O[c0 + i], __uint_as_float(v[i]));
+            }
+            tc_fence_before();
+            mbar_arrive(bar(B_OEMPTY));
+        };
+
+        for (int j = 0; ok && j < ntiles; ++j) {
+            const int t = t_begin + j;
+            const int st = j & 1;
+            // visible key columns [lo, hi) of this tile for this row
+            int lo = 0, hi = 128;
+            const float* bias = nullptr;
+            if (t < nC) {
+                hi = min(128, Lc - t * 128);
+                if (stream == 1 && p.bias) bias = p.bias + crow0 + t * 128;
+            } else {
+                const int jt = (t - nC) * 128;
+                lo = max(0, cs - jt);
+                hi = min(128, tok - jt + 1);
+            }
+            const bool need_mask = (lo > 0) || (hi < 128) || (bias != nullptr);
+            ok = mbar_wait(bar(B_SFULL + st), (j >> 1) & 1, abort_flag, p.status, 31);
+            if (!ok) break;
+            tc_fence_after();
+            // pass 1: row maximum
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tS[st] + lane_off + (uint32_t)c0, v);
+                tmem_ld_wait();
+                if (need_mask) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int c = c0 + i;
+                        float s = __uint_as_float(v[i]);
+                        if (bias && c < hi) s = fmaf(bias[c], 1.4426950408889634f, s);
+                        mx = fmaxf(mx, (c >= lo && c < hi) ? s : -INFINITY);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+                }
+            }
+            const float m_new = fmaxf(m, mx);
+            const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
+            const float alpha = ex2(m - m_safe);              // m = -inf -> 0
+            // fold in the previous tile's P V product (it also frees the P buffer)
+            if (j > 0) accumulate_o(j - 1);
+            if (!ok) break;
+            // pass 2: P = 2^(S - m) as bf16 into swizzled smem, row sum
+            float ls = 0.f;
+            uint8_t* prow = sm + S::kP + row_in * 128;
+#pragma unroll 1
+            for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(tS[st] + lane_off + (uint32_t)c0, v);
+                tmem_ld_wait();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float s0 = __uint_as_float(v[i]), s1 = __uint_as_float(v[i + 1]);
+                    if (need_mask) {
+                        const int c = c0 + i;
+                        if (bias && c < hi) s0 = fmaf(bias[c], 1.4426950408889634f, s0);
+                        if (bias && c + 1 < hi) s1 = fmaf(bias[c + 1], 1.4426950408889634f, s1);
+                        if (!(c >= lo && c < hi)) s0 = -INFINITY;
+                        if (!(c + 1 >= lo && c + 1 < hi)) s1 = -INFINITY;
+                    }
+                    const float p0 = ex2(s0 - m_safe), p1 = ex2(s1 - m_safe);
+                    ls += p0 + p1;
+                    __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+                    pk[i >> 1] = *reinterpret_cast<uint32_t*>(&b);
+                }
+                // 32 columns = 4 chunks of 16 bytes; chunk index inside the 64-column sub-tile is
+                // XOR-swizzled with the row (128B swizzle), sub-tiles are 16 KB apart
+                uint8_t* psub = prow + (c0 >> 6) * 16384;
+                const int ch0 = (c0 & 63) >> 3;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint4 val = make_uint4(pk[ch * 4], pk[ch * 4 + 1], pk[ch * 4 + 2], pk[ch * 4 + 3]);
+                    *reinterpret_cast<uint4*>(psub + (((ch0 + ch) ^ (row_in & 7)) << 4)) = val;
+                }
+            }
+            l = l * alpha + ls;
+            m = m_new;
+            alpha_pend = alpha;
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(bar(B_PFULL));
+            mbar_arrive(bar(B_SEMPTY + st));
+        }
+        if (ok && ntiles > 0) accumulate_o(ntiles - 1);
+        if (valid && ok) {
+            const size_t pr = ((size_t)z * p.Hkv + kh) * p.rows + r;
+            p.part_m[pr] = (m == -INFINITY) ? -INFINITY : m * 0.6931471805599453f;   // back to natural-log units
+            p.part_l[pr] = l;
+            float4* po = reinterpret_cast<float4*>(p.part_O + pr * HD);
+#pragma unroll
+            for (int i = 0; i < HD / 4; ++i) po[i] = make_float4(O[4 * i], O[4 * i + 1], O[4 * i + 2], O[4 * i + 3]);
+        }
+    }
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tbase, 512);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, int* nsplitC) {
+    const int g = d->Hq / d->Hkv;
+    const long long qtiles = ((long long)d->N_max * g + 127) / 128;
+    const long long base = qtiles * d->Hkv;
+    const long long tilesF = (d->L + 127) / 128 + (d->N_max + 127) / 128;
+    long long want = (6LL * 148 + base - 1) / base;
+    if (want < 1) want = 1;
+    if (want > 64) want = 64;
+    long long t = (tilesF + want - 1) / want;
+    if (t < 4) t = 4;
+    *tps = (int)t;
+    const long long tF = (d->L + 127) / 128 + (N + 127) / 128;
+    const long long tC = (max_b + 127) / 128 + (N + 127) / 128;
+    *nsplitF = (int)((tF + t - 1) / t);
+    *nsplitC = (int)((tC + t - 1) / t);
+    if (*nsplitC < 1) *nsplitC = 1;
+}
+
+template <int HD>
+static int launch_attn(const Lc& lc, const AttnTcParams& p, int qtiles) {
+    using S = AttnSmem<HD>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(k_attn_tc<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess)
+            return PKV_ERR_CUDA;
+        attr_set = true;
+    }
+    dim3 grid(qtiles, p.Hkv, p.nsplitF + p.nsplitC);
+    k_attn_tc<HD><<<grid, 192, S::kTotal, lc.st>>>(p);
+    lc.count();
+    return PKV_OK;
+}
+
+int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, const float* rope_tab,
+                 DevStatus* status) {
+    const int N = a.N, hd = d->hd, Hkv = d->Hkv, g = d->Hq / d->Hkv;
+    const int rows = N * g;
+    {
+        size_t total = (size_t)2 * N * (d->Hq + 2 * Hkv) * (hd / 2);
+        k_attn_prep<<<(unsigned)((total + 255) / 256), 256, 0, lc.st>>>(a.q, a.ldq, a.k_new, a.v_new, a.ldkv, rope_tab, N,
+                                                                        d->Hq, Hkv, hd, t->q.hi, t->q.lo, t->kn, t->vn);
+        lc.count();
+    }
+    AttnTcParams p;
+    int rc;
+    if ((rc = tc_make_map_3d(&p.mQhi, t->q.hi, 2 * Hkv, rows, hd, hd, (uint64_t)rows * hd, 128))) return rc;
+    if ((rc = tc_make_map_3d(&p.mQlo, t->q.lo, 2 * Hkv, rows, hd, hd, (uint64_t)rows * hd, 128))) return rc;
+    if ((rc = tc_make_map_3d(&p.mKn, t->kn, 2 * Hkv, N, hd, hd, (uint64_t)N * hd, 128))) return rc;
+    if ((rc = tc_make_map_3d(&p.mVn, t->vn, 2 * Hkv, N, hd, hd, (uint64_t)N * hd, 128))) return rc;
+    if (d->L > 0) {
+        if ((rc = tc_make_map_3d(&p.mK, a.K, Hkv, d->L, hd, hd, (uint64_t)d->L * hd, 128))) return rc;
+        if ((rc = tc_make_map_3d(&p.mV, a.V, Hkv, d->L, hd, hd, (uint64_t)d->L * hd, 128))) return rc;
+    } else {
+        p.mK = p.mKn;
+        p.mV = p.mVn;
+    }
+    const int total_kept = a.total_kept;
+    if (total_kept > 0) {
+        if ((rc = tc_make_map_2d(&p.mKc, a.Kc, total_kept, hd, hd, 128))) return rc;
+        if ((rc = tc_make_map_2d(&p.mVc, a.Vc, total_kept, hd, hd, 128))) return rc;
+    } else {
+        p.mKc = p.mKn;      // never read: no compact-cache tiles exist
+        p.mVc = p.mVn;
+    }
+    p.head_off = a.head_off; p.tok_cs = a.tok_cs; p.bias = a.bias;
+    p.N = N; p.g = g; p.Hkv = Hkv; p.L = d->L; p.rows = rows;
+    tc_attn_plan(d, N, a.max_b, &p.tps, &p.nsplitF, &p.nsplitC);
+    p.part_m = t->part_m; p.part_l = t->part_l; p.part_O = t->part_O;
+    p.status = status;
+    const int qtiles = (rows + 127) / 128;
+    rc = (hd == 128) ? launch_attn<128>(lc, p, qtiles) : launch_attn<64>(lc, p, qtiles);
+    if (rc != PKV_OK) return rc;
+    AttnArgs c = a;
+    c.nsplitF = p.nsplitF; c.nsplitC = p.nsplitC;
+    c.part_m = t->part_m; c.part_l = t->part_l; c.part_O = t->part_O;
+    attention_combine(lc, c);
+    return PKV_OK;
+}
+
+}  // namespace pkv
