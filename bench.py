@@ -174,6 +174,8 @@ def main():
     ap.add_argument("--engine", default="auto", choices=["auto", "simt"])
     ap.add_argument("--ref-sample", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quick", action="store_true",
+                    help="timed steps only (no stage pass, no end-to-end pass, no CPU baseline): for profiler runs")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -219,7 +221,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(args.warmup if args.quick else max(args.warmup, 3)):
         step()
     barrier()
     sampler = ClockSampler(local)
@@ -241,6 +243,14 @@ def main():
         t = torch.tensor([ms], device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
+
+    if args.quick:
+        if rank == 0:
+            print(json.dumps({"metric": "patch_build_ms_per_context", "value": ms / world, "unit": "ms",
+                              "n_gpus": world, "steps": args.steps, "quick": True, "gpu_launches": int(launches)}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # per-stage device times (separate pass with the library's stage events)
     ctx.set_timing(True)
