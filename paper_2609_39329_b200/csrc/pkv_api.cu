@@ -80,6 +80,7 @@ struct pkv_ctx {
     int32_t* host_stage;     // pinned: head_off + tok_cs
     DevStatus* host_status;  // pinned
     int64_t launches;
+    void* map_cache;
     int timing;
     cudaEvent_t ev[ST_COUNT + 1];
     char cuda_err[256];
@@ -236,6 +237,7 @@ extern "C" int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* o
     }
     for (int i = 0; i <= ST_COUNT; ++i) cudaEventCreate(&c->ev[i]);
     if (c->engine != PKV_ENGINE_SIMT) {
+        c->map_cache = pkv::tc_map_cache_create();
         rc = pkv::tc_init(&c->b.tc, dims);
         if (rc != PKV_OK) {
             pkv_destroy(c);
@@ -252,6 +254,7 @@ extern "C" void pkv_destroy(pkv_ctx* c) {
     if (c->own_ws && c->ws) cudaFree(c->ws);
     if (c->host_stage) cudaFreeHost(c->host_stage);
     if (c->host_status) cudaFreeHost(c->host_status);
+    if (c->map_cache) pkv::tc_map_cache_destroy((pkv::MapCache*)c->map_cache);
     for (int i = 0; i <= ST_COUNT; ++i)
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     delete c;
@@ -431,7 +434,7 @@ static void solve_stage(pkv_ctx* c, const Lc& lc, const float* S_H, const float*
     if (c->engine == PKV_ENGINE_SIMT)
         ridge_solve_simt(lc, b.solve, F, d, dW, b.status);
     else
-        pkv::tc_ridge_solve(lc, &b.tc, b.solve, F, d, dW, b.status);
+        pkv::tc_ridge_solve(lc, &b.tc, b.solve, F, d, dW, lam0, mode, b.status);
     sumsq(lc, dW, (int64_t)d * F, &b.status->dw_fro2);
 }
 
@@ -462,7 +465,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
     const int Dq = D.Hq * hd, Dkv = D.Hkv * hd, QKV = Dq + 2 * Dkv;
     const bool bf = D.dtype == PKV_BF16;
     Buffers& b = c->b;
-    Lc lc{c->st, &c->launches};
+    Lc lc{c->st, &c->launches, c->map_cache};
 
     begin_call(c);
     upload_meta(c, cb->head_off, N, ref->n_chunks, ref->chunk_off);
@@ -588,7 +591,7 @@ extern "C" int pkv_gather_kept(pkv_ctx* c, const pkv_kv* full, const int32_t* he
     if (rc != PKV_OK) return rc;
     if (total > 0 && (!idx || !Kc || !Vc || !full->K || !full->V)) return PKV_ERR_INVALID_ARG;
     if (((uintptr_t)Kc & 15) || ((uintptr_t)Vc & 15)) return PKV_ERR_INVALID_ARG;
-    Lc lc{c->st, &c->launches};
+    Lc lc{c->st, &c->launches, c->map_cache};
     begin_call(c);
     int32_t one[2] = {0, 0};
     upload_meta(c, head_off_host, 0, 0, one);
@@ -611,7 +614,7 @@ extern "C" int pkv_attention(pkv_ctx* c, const float* q, const float* k_new, con
     rc = check_compressed(c, cb, &total, &max_b);
     if (rc != PKV_OK) return rc;
     const int Dq = c->dims.Hq * c->dims.hd, Dkv = c->dims.Hkv * c->dims.hd;
-    Lc lc{c->st, &c->launches};
+    Lc lc{c->st, &c->launches, c->map_cache};
     begin_call(c);
     upload_meta(c, cb->head_off, N, n_chunks, chunk_off);
     const void *Kc, *Vc;
@@ -631,7 +634,7 @@ extern "C" int pkv_attention(pkv_ctx* c, const float* q, const float* k_new, con
 extern "C" int pkv_gram(pkv_ctx* c, const float* X, const float* R, int32_t n, float* S_H, float* S_T,
                         int accumulate) {
     if (!c || !X || !R || !S_H || !S_T || n <= 0 || n > c->dims.N_max) return PKV_ERR_INVALID_ARG;
-    Lc lc{c->st, &c->launches};
+    Lc lc{c->st, &c->launches, c->map_cache};
     begin_call(c);
     if (c->engine == PKV_ENGINE_SIMT)
         gram_simt(c, lc, X, R, n, S_H, S_T, accumulate != 0);
@@ -646,7 +649,7 @@ extern "C" int pkv_ridge_solve(pkv_ctx* c, const float* S_H, const float* S_T, f
     if (!(lambda > 0.f) || !isfinite(lambda)) return PKV_ERR_INVALID_ARG;
     if (lambda_mode != PKV_LAMBDA_PAPER && lambda_mode != PKV_LAMBDA_ABSOLUTE && lambda_mode != PKV_LAMBDA_TRACE_MEAN)
         return PKV_ERR_INVALID_ARG;
-    Lc lc{c->st, &c->launches};
+    Lc lc{c->st, &c->launches, c->map_cache};
     begin_call(c);
     solve_stage(c, lc, S_H, S_T, lambda, lambda_mode, dW);
     return end_call(c, stats, nullptr);

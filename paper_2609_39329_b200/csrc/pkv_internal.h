@@ -25,6 +25,7 @@ struct DevStatus {
 struct Lc {
     cudaStream_t st;
     int64_t* launches;
+    void* map_cache = nullptr;            // tensor-map cache of the tensor-core engine (optional)
     void count(int n = 1) const { if (launches) *launches += n; }
 };
 

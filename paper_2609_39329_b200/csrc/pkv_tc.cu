@@ -115,15 +115,24 @@ static void transpose_split(const Lc& lc, const float* in, int rows, int cols, i
 // ---------------------------------------------------------------------------------------------
 // helpers
 // ---------------------------------------------------------------------------------------------
+static TcGemm plain_gemm(int M, int Nn, int K, float* C, long long ldc, float alpha, const float* addend,
+                         long long ldadd, bool accumulate) {
+    TcGemm g{};
+    g.M = M; g.N = Nn; g.K = K; g.batch = 1;
+    g.C = C; g.ldc = ldc; g.alpha = alpha; g.addend = addend; g.ldadd = ldadd; g.accumulate = accumulate;
+    g.c_rows = M; g.c_cols = Nn;
+    return g;
+}
+
 // C = alpha * (A_hi + A_lo) W^T (+ addend): fp32 activation pair against a bf16 weight [Nn][K].
 static int gemm_act_weight(const Lc& lc, Pair A, long long lda, const void* W, long long ldw, float* C,
                            long long ldc, int M, int Nn, int K, float alpha, const float* addend, long long ldadd,
                            DevStatus* st) {
-    TcGemm g{};
-    g.A[0] = A.hi; g.A[1] = A.lo; g.lda[0] = g.lda[1] = lda;
-    g.B[0] = g.B[1] = (const __nv_bfloat16*)W; g.ldb[0] = g.ldb[1] = ldw;
-    g.npass = 2; g.C = C; g.ldc = ldc; g.M = M; g.N = Nn; g.K = K; g.alpha = alpha;
-    g.addend = addend; g.ldadd = ldadd;
+    TcGemm g = plain_gemm(M, Nn, K, C, ldc, alpha, addend, ldadd, false);
+    g.A[0] = TcMat{A.hi, lda, M, K};
+    g.A[1] = TcMat{A.lo, lda, M, K};
+    g.B[0] = g.B[1] = TcMat{(const __nv_bfloat16*)W, ldw, Nn, K};
+    g.npass = 2;
     return gemm_tc(lc, g, st);
 }
 
@@ -131,13 +140,11 @@ static int gemm_act_weight(const Lc& lc, Pair A, long long lda, const void* W, l
 static int gemm_pair_pair(const Lc& lc, Pair A, long long lda, Pair B, long long ldb, float* C, long long ldc, int M,
                           int Nn, int K, float alpha, const float* addend, long long ldadd, bool accumulate,
                           DevStatus* st) {
-    TcGemm g{};
-    g.A[0] = A.hi; g.B[0] = B.hi;
-    g.A[1] = A.hi; g.B[1] = B.lo;
-    g.A[2] = A.lo; g.B[2] = B.hi;
-    for (int i = 0; i < 3; ++i) { g.lda[i] = lda; g.ldb[i] = ldb; }
-    g.npass = 3; g.C = C; g.ldc = ldc; g.M = M; g.N = Nn; g.K = K; g.alpha = alpha;
-    g.addend = addend; g.ldadd = ldadd; g.accumulate = accumulate;
+    TcGemm g = plain_gemm(M, Nn, K, C, ldc, alpha, addend, ldadd, accumulate);
+    g.A[0] = TcMat{A.hi, lda, M, K}; g.B[0] = TcMat{B.hi, ldb, Nn, K};
+    g.A[1] = TcMat{A.hi, lda, M, K}; g.B[1] = TcMat{B.lo, ldb, Nn, K};
+    g.A[2] = TcMat{A.lo, lda, M, K}; g.B[2] = TcMat{B.hi, ldb, Nn, K};
+    g.npass = 3;
     return gemm_tc(lc, g, st);
 }
 
@@ -194,10 +201,10 @@ size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d) {
     t->part_m = c.take<float>(nsp * d->Hkv * rows);
     t->part_l = c.take<float>(nsp * d->Hkv * rows);
     t->part_O = c.take<float>(nsp * d->Hkv * rows * d->hd);
-    return c.off;
+    return tc_solve_carve(&t->solve, base, c.off, d);
 }
 
-int tc_init(TcBuffers*, const pkv_dims*) { return PKV_OK; }
+int tc_init(TcBuffers* t, const pkv_dims* d) { return tc_solve_init(&t->solve, d); }
 
 static void mark(const TcForwardArgs& a, const Lc& lc, int stage) {
     if (a.ev) cudaEventRecord(a.ev[stage], lc.st);
@@ -216,8 +223,12 @@ int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
     return attention_tc(lc, t, d, a, nullptr, status);
 }
 
-void tc_ridge_solve(const Lc& lc, TcBuffers*, const SolveWs& ws, int F, int d, float* dW, DevStatus* status) {
-    ridge_solve_simt(lc, ws, F, d, dW, status);
+void tc_ridge_solve(const Lc& lc, TcBuffers* t, const SolveWs& ws, int F, int d, float* dW, float lam0, int mode,
+                    DevStatus* status) {
+    // Under the adaptive scale of Eq. 7 cond(G) ~ (tr(S_H)/sigma_max)/lambda0; lambda0 >= 0.05 keeps it
+    // to a few tens.  Absolute and trace-mean coefficients give no such bound.
+    const bool well = (mode == PKV_LAMBDA_PAPER) && (lam0 >= 0.05f);
+    tc_ridge_solve_impl(lc, &t->solve, ws.G, ws.Y, F, d, dW, well, status);
 }
 
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a) {

@@ -9,26 +9,59 @@ namespace pkv {
 
 constexpr int kGemmMaxPass = 6;
 
-// C[M][N] = alpha * sum_p A[p][M][K] B[p][N][K]^T (+ addend) (+ C); bf16 operands, fp32 result.
+// A bf16 matrix as the TMA engine sees it (whole allocation: rows x cols, row stride ld).
+struct TcMat {
+    const __nv_bfloat16* p;
+    long long ld, rows, cols;
+};
+
+// C = alpha * sum_p A_p B_p^T (+ addend) (+ C): bf16 operands, fp32 accumulate.  Operand tiles are
+// addressed by (row0, col0) offsets into whole matrices, with per-batch increments (blockIdx.z);
+// rows/columns past a matrix edge read as zero.  Results go to fp32 C and/or to up to three bf16
+// arrays holding successive roundings of the value (hi, mid, lo).
 struct TcGemm {
-    const __nv_bfloat16* A[kGemmMaxPass];
-    long long lda[kGemmMaxPass];
-    const __nv_bfloat16* B[kGemmMaxPass];
-    long long ldb[kGemmMaxPass];
+    TcMat A[kGemmMaxPass], B[kGemmMaxPass];
     int npass;
+    int a_row0, a_col0, a_zrow, a_zcol;
+    int b_row0, b_col0, b_zrow, b_zcol;
+    int M, N, K, batch;
     float* C;
     long long ldc;
-    int M, N, K;
-    float alpha;
     const float* addend;
     long long ldadd;
+    int c_row0, c_col0, c_zrow, c_zcol, c_rows, c_cols;   // stores are clipped to [0,c_rows) x [0,c_cols)
+    __nv_bfloat16* out[3];
+    long long ldo;
+    int nout;
+    float alpha;
     bool accumulate, lower_only;
+    int k_tri;      // 0: dense; 1: B lower triangular (skip k tiles past the row); 2: B upper triangular
 };
+struct MapCache;
+MapCache* tc_map_cache_create();
+void tc_map_cache_destroy(MapCache* c);
 int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status);
 bool tc_encode_available();
 int tc_make_map_2d(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows);
 int tc_make_map_3d(CUtensorMap* m, const void* ptr, uint64_t d2, uint64_t rows, uint64_t cols, uint64_t ld1,
                    uint64_t ld2, uint32_t box_rows);
+
+// Workspace of the tensor-core ridge solve: bf16 triples (hi, mid, lo) of the factor L, its inverse X,
+// the inverse's transpose, the current panel, the doubling temporaries; pairs of S_T and S_T X^T.
+struct TcSolveBuffers {
+    __nv_bfloat16* L3[3];
+    __nv_bfloat16* X3[3];
+    __nv_bfloat16* XT3[3];
+    __nv_bfloat16* P3[3];
+    __nv_bfloat16* TT3[3];
+    __nv_bfloat16* S2[3];
+    __nv_bfloat16* Z2[3];
+};
+size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, const pkv_dims* d);
+int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d);
+// dW [d][F] = S_T G^{-1}; G [F][F] (lower part read) is destroyed.
+int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int F, int d, float* dW,
+                        bool well_conditioned, DevStatus* status);
 
 // bf16 hi/lo pairs of fp32 activations: v ~= hi + lo with hi = bf16(v), lo = bf16(v - hi).
 struct Pair {
@@ -54,6 +87,7 @@ struct TcBuffers {
     float* part_m;      // attention split partials [splits][Hkv][N*g]
     float* part_l;
     float* part_O;      // [splits][Hkv][N*g][hd]
+    TcSolveBuffers solve;
 };
 
 struct TcForwardArgs {
@@ -80,7 +114,8 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArg
 int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status);
 void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, const float* R, int n, float* S_H,
              float* S_T, bool accumulate, DevStatus* status);
-void tc_ridge_solve(const Lc& lc, TcBuffers* t, const SolveWs& ws, int F, int d, float* dW, DevStatus* status);
+void tc_ridge_solve(const Lc& lc, TcBuffers* t, const SolveWs& ws, int F, int d, float* dW, float lam0, int mode,
+                    DevStatus* status);
 void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* d, int N, const void* Wdown, const float* dW,
                     const float* zF, const float* R, float* xF_next, float* D, DevStatus* status);
 

@@ -11,6 +11,9 @@
 // fp32 product as three or six passes.  Ragged M, N, K are handled by TMA zero fill and
 // predicated stores.
 #include <cuda.h>
+#include <string.h>
+
+#include <new>
 
 #include "pkv_ptx.cuh"
 #include "pkv_tc.h"
@@ -20,45 +23,62 @@ namespace pkv {
 using namespace ptx;
 
 struct alignas(64) GemmTcParams {
-    CUtensorMap mapA[kGemmMaxPass];
-    CUtensorMap mapB[kGemmMaxPass];
-    int npass, M, N, K;
+    CUtensorMap mapA[3];      // distinct A operands (e.g. hi, mid, lo parts)
+    CUtensorMap mapB[3];      // distinct B operands
+    int nA, nB, npass;
+    int pa[kGemmMaxPass], pb[kGemmMaxPass];   // pass i multiplies A operand pa[i] with B operand pb[i]
+    int stages;
+    int M, N, K;
+    int a_row0, a_col0, a_zrow, a_zcol;
+    int b_row0, b_col0, b_zrow, b_zcol;
+    int c_row0, c_col0, c_zrow, c_zcol, c_rows, c_cols;
     float* C;
     long long ldc;
     float alpha;
     const float* addend;
     long long ldadd;
-    int accumulate, lower_only, vec_ok;
+    __nv_bfloat16* out[3];
+    long long ldo;
+    int nout;
+    int accumulate, lower_only, k_tri, vec_ok;
     DevStatus* status;
 };
 
-template <int BN, int STAGES>
-struct GemmSmem {
-    static constexpr int kA = 128 * 64 * 2;
-    static constexpr int kB = BN * 64 * 2;
-    static constexpr int kStage = kA + kB;
-    static constexpr int kBars = 2 * STAGES + 1;
-    static constexpr int kTotal = STAGES * kStage + kBars * 8 + 16 + 1024;   // + alignment slack
-};
+constexpr int kGemmMaxStages = 6;
+constexpr int kGemmBarBytes = (2 * kGemmMaxStages + 1) * 8 + 16;
+constexpr int kGemmStagingBytes = 4 * 32 * 33 * 4;     // aliases the first pipeline stage (free once the MMAs are done)
 
-template <int BN, int STAGES>
+// One k-tile stage holds every distinct operand tile once: nA x [128][64] and nB x [BN][64] bf16,
+// and all passes are issued from it (the shared operand of a split product is not re-read).
+template <int BN>
 __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcParams p) {
-    using S = GemmSmem<BN, STAGES>;
-    const int m0 = blockIdx.y * 128, n0 = blockIdx.x * BN;
+    const int m0 = blockIdx.y * 128, n0 = blockIdx.x * BN, z = blockIdx.z;
     if (p.lower_only && n0 > m0 + 127) return;
     if (p.status->code != 0) return;      // an earlier stage already failed: the call reports it
+    // absolute coordinates of this tile's output; tiles entirely outside the stored region do nothing
+    const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
+    if (crow0 >= p.c_rows || ccol0 >= p.c_cols) return;
 
+    constexpr int kA = 128 * 64 * 2, kB = BN * 64 * 2;
+    const int stage_bytes = p.nA * kA + p.nB * kB;
+    const int STAGES = p.stages;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - raw);
-    const uint32_t bars = base + STAGES * S::kStage;          // full[STAGES], empty[STAGES], tmem_full
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * S::kStage + S::kBars * 8);
+    const uint32_t bars = base + STAGES * stage_bytes;        // full[STAGES], empty[STAGES], tmem_full
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * stage_bytes + (2 * STAGES + 1) * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* staging = reinterpret_cast<float*>(sm);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ktiles = (p.K + 63) / 64;
-    const int total = p.npass * ktiles;
+    // contraction range in 64-wide tiles; a triangular B operand lets whole tiles be skipped:
+    //   k_tri = 1: B[n][k] = 0 for k > n (lower triangular)   -> tiles beyond the tile's last row are zero
+    //   k_tri = 2: B[n][k] = 0 for k < n (upper triangular)   -> tiles before the tile's first row are zero
+    int kt_begin = 0, kt_end = (p.K + 63) / 64;
+    if (p.k_tri == 1) kt_end = min(kt_end, (n0 + BN + 63) / 64);
+    if (p.k_tri == 2) kt_begin = min(kt_end, n0 / 64);
+    const int ktiles = kt_end - kt_begin;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) {
@@ -80,77 +100,127 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int ps = 0; ps < p.npass; ++ps) {
-                prefetch_tmap(&p.mapA[ps]);
-                prefetch_tmap(&p.mapB[ps]);
-            }
-            for (int it = 0; it < total; ++it) {
+            const int ar = p.a_row0 + z * p.a_zrow + m0, ac = p.a_col0 + z * p.a_zcol;
+            const int br = p.b_row0 + z * p.b_zrow + n0, bc = p.b_col0 + z * p.b_zcol;
+            for (int it = 0; it < ktiles; ++it) {
                 const int s = it % STAGES;
                 if (!mbar_wait(bars + 8 * (STAGES + s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, 1)) break;
-                const int ps = it / ktiles, kt = it - ps * ktiles;
+                const int kt = kt_begin + it;
                 const uint32_t full = bars + 8 * s;
-                mbar_expect_tx(full, S::kStage);
-                tma_load_2d(base + s * S::kStage, &p.mapA[ps], full, kt * 64, m0);
-                tma_load_2d(base + s * S::kStage + S::kA, &p.mapB[ps], full, kt * 64, n0);
+                const uint32_t sa = base + s * stage_bytes;
+                mbar_expect_tx(full, stage_bytes);
+                for (int i = 0; i < p.nA; ++i) tma_load_2d(sa + i * kA, &p.mapA[i], full, ac + kt * 64, ar);
+                for (int i = 0; i < p.nB; ++i) tma_load_2d(sa + p.nA * kA + i * kB, &p.mapB[i], full, bc + kt * 64, br);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16(128, BN);
             bool ok = true;
-            for (int it = 0; it < total; ++it) {
+            for (int it = 0; it < ktiles; ++it) {
                 const int s = it % STAGES;
                 if (!mbar_wait(bars + 8 * s, (it / STAGES) & 1, abort_flag, p.status, 2)) { ok = false; break; }
                 tc_fence_after();
-                const uint64_t da = smem_desc_sw128(base + s * S::kStage);
-                const uint64_t db = smem_desc_sw128(base + s * S::kStage + S::kA);
+                const uint32_t sa = base + s * stage_bytes;
+                for (int ps = 0; ps < p.npass; ++ps) {
+                    const uint64_t da = smem_desc_sw128(sa + p.pa[ps] * kA);
+                    const uint64_t db = smem_desc_sw128(sa + p.nA * kA + p.pb[ps] * kB);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
-                    mma_bf16_ss(tbase, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (it | kk) != 0);
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_bf16_ss(tbase, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (it | ps | kk) != 0);
+                }
                 mma_commit(bars + 8 * (STAGES + s));
             }
             if (ok) mma_commit(bars + 8 * (2 * STAGES));
         }
     } else {
+        // epilogue: TMEM -> registers -> per-warp smem tile -> row-contiguous global accesses
         const int q = warp & 3;
-        const bool ok = mbar_wait(bars + 8 * (2 * STAGES), 0, abort_flag, p.status, 3);
-        tc_fence_after();
+        bool ok = true;
+        if (ktiles > 0) {
+            ok = mbar_wait(bars + 8 * (2 * STAGES), 0, abort_flag, p.status, 3);
+            tc_fence_after();
+        }
         if (ok) {
-            const int row = m0 + q * 32 + lane;
+            float* stg = staging + q * (32 * 33);
+            const int rl0 = m0 + q * 32;                 // first row of this warp inside the batch element
+            const int rowa0 = crow0 + q * 32;            // ... and its absolute output row
+            const int nrows = max(0, min(32, min(p.M - rl0, p.c_rows - rowa0)));
+            const bool vec_ok = p.vec_ok != 0;
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
-                tmem_ld32(tbase + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-                tmem_ld_wait();
-                if (row < p.M && n0 + c0 < p.N) {
-                    float* crow = p.C + (size_t)row * p.ldc + n0 + c0;
-                    const float* arow = p.addend ? p.addend + (size_t)row * p.ldadd + n0 + c0 : nullptr;
-                    if (p.vec_ok && n0 + c0 + 32 <= p.N) {
+                if (ktiles > 0) {
+                    tmem_ld32(tbase + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                    tmem_ld_wait();
+                } else {
 #pragma unroll
-                        for (int j = 0; j < 32; j += 4) {
-                            float4 v = make_float4(p.alpha * __uint_as_float(r[j]), p.alpha * __uint_as_float(r[j + 1]),
-                                                   p.alpha * __uint_as_float(r[j + 2]), p.alpha * __uint_as_float(r[j + 3]));
-                            if (arow) {
-                                float4 a = *reinterpret_cast<const float4*>(arow + j);
-                                v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;
+                }
+                const int col = ccol0 + c0;                    // absolute output column of r[0]
+                const int ncol = min(min(32, p.N - (n0 + c0)), p.c_cols - col);
+                if (ncol <= 0) break;
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = p.alpha * __uint_as_float(r[j]);
+                if (p.C && lane < nrows) {
+                    // fp32 output: every lane owns one row; 128 contiguous bytes, loads batched ahead of stores
+                    const size_t row = (size_t)(rowa0 + lane);
+                    float* crow = p.C + row * p.ldc + col;
+                    const float* arow = p.addend ? p.addend + row * p.ldadd + col : nullptr;
+                    if (vec_ok && ncol == 32) {
+                        if (arow) {
+                            float4 a4[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) a4[j] = *reinterpret_cast<const float4*>(arow + 4 * j);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                v[4 * j] += a4[j].x; v[4 * j + 1] += a4[j].y; v[4 * j + 2] += a4[j].z; v[4 * j + 3] += a4[j].w;
                             }
-                            if (p.accumulate) {
-                                float4 c = *reinterpret_cast<const float4*>(crow + j);
-                                v.x += c.x; v.y += c.y; v.z += c.z; v.w += c.w;
-                            }
-                            *reinterpret_cast<float4*>(crow + j) = v;
                         }
+                        if (p.accumulate) {
+                            float4 c4[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) c4[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                v[4 * j] += c4[j].x; v[4 * j + 1] += c4[j].y; v[4 * j + 2] += c4[j].z; v[4 * j + 3] += c4[j].w;
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            *reinterpret_cast<float4*>(crow + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            if (n0 + c0 + j < p.N) {
-                                float v = p.alpha * __uint_as_float(r[j]);
-                                if (arow) v += arow[j];
-                                if (p.accumulate) v += crow[j];
-                                crow[j] = v;
+                            if (j < ncol) {
+                                if (arow) v[j] += arow[j];
+                                if (p.accumulate) v[j] += crow[j];
+                                crow[j] = v[j];
                             }
                         }
                     }
+                }
+                if (p.nout > 0) {
+                    // bf16 parts: through the warp's smem tile so that a warp writes 64 contiguous bytes per row
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = v[j];
+                    __syncwarp();
+                    if (lane < ncol) {
+                        for (int rr = 0; rr < nrows; ++rr) {
+                            const float x = stg[rr * 33 + lane];
+                            const size_t o = (size_t)(rowa0 + rr) * p.ldo + col + lane;
+                            __nv_bfloat16 h = __float2bfloat16_rn(x);
+                            p.out[0][o] = h;
+                            if (p.nout > 1) {
+                                const float r1 = x - __bfloat162float(h);
+                                __nv_bfloat16 m = __float2bfloat16_rn(r1);
+                                p.out[1][o] = m;
+                                if (p.nout > 2) p.out[2][o] = __float2bfloat16_rn(r1 - __bfloat162float(m));
+                            }
+                        }
+                    }
+                    __syncwarp();
                 }
             }
         }
@@ -222,42 +292,127 @@ int tc_make_map_3d(CUtensorMap* m, const void* ptr, uint64_t d2, uint64_t rows, 
     return r == CUDA_SUCCESS ? PKV_OK : PKV_ERR_CUDA;
 }
 
-template <int BN, int STAGES>
-static int launch_gemm(const Lc& lc, const GemmTcParams& p) {
-    using S = GemmSmem<BN, STAGES>;
+// Tensor maps of operands that keep their address and shape (workspace buffers, weights of the
+// current block) are encoded once and reused.
+struct MapCacheEntry {
+    const void* ptr;
+    uint64_t rows, cols, ld;
+    uint32_t box;
+    int valid;
+    CUtensorMap map;
+};
+struct MapCache {
+    static constexpr int kSize = 512;
+    MapCacheEntry e[kSize];
+};
+
+MapCache* tc_map_cache_create() {
+    MapCache* c = new (std::nothrow) MapCache();
+    if (c) memset(c, 0, sizeof(*c));
+    return c;
+}
+void tc_map_cache_destroy(MapCache* c) { delete c; }
+
+static int cached_map(MapCache* cache, CUtensorMap* out, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld,
+                      uint32_t box) {
+    if (!cache) return tc_make_map_2d(out, ptr, rows, cols, ld, box);
+    uint64_t h = (uint64_t)(uintptr_t)ptr * 0x9E3779B97F4A7C15ull ^ (rows * 0xC2B2AE3D27D4EB4Full) ^ (cols << 17) ^
+                 (ld << 33) ^ box;
+    h ^= h >> 29;
+    for (int probe = 0; probe < 4; ++probe) {
+        MapCacheEntry& e = cache->e[(h + probe) % MapCache::kSize];
+        if (e.valid && e.ptr == ptr && e.rows == rows && e.cols == cols && e.ld == ld && e.box == box) {
+            *out = e.map;
+            return PKV_OK;
+        }
+    }
+    int rc = tc_make_map_2d(out, ptr, rows, cols, ld, box);
+    if (rc != PKV_OK) return rc;
+    int slot = -1;
+    for (int probe = 0; probe < 4; ++probe)
+        if (!cache->e[(h + probe) % MapCache::kSize].valid) { slot = (int)((h + probe) % MapCache::kSize); break; }
+    if (slot < 0) slot = (int)(h % MapCache::kSize);
+    MapCacheEntry& e = cache->e[slot];
+    e.ptr = ptr; e.rows = rows; e.cols = cols; e.ld = ld; e.box = box; e.map = *out; e.valid = 1;
+    return PKV_OK;
+}
+
+template <int BN>
+static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     static bool attr_set = false;
+    constexpr int kMaxSmem = 227 * 1024;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(k_gemm_tc<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(k_gemm_tc<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return PKV_ERR_CUDA;
         attr_set = true;
     }
-    dim3 grid((p.N + BN - 1) / BN, (p.M + 127) / 128);
-    k_gemm_tc<BN, STAGES><<<grid, 192, S::kTotal, lc.st>>>(p);
+    const int stage_bytes = p.nA * 128 * 128 + p.nB * BN * 128;
+    const int fixed = kGemmBarBytes + 1024;
+    const int ktiles = (p.K + 63) / 64;
+    // Two CTAs per SM let one tile's epilogue overlap the other's main loop: taken when the contraction
+    // is short (epilogue-bound) or when two stages still fit in half an SM's shared memory.
+    const int half = 112 * 1024 - fixed;
+    int stages;
+    if (ktiles <= 8 || 2 * stage_bytes <= half) stages = half / stage_bytes;
+    else stages = (kMaxSmem - fixed) / stage_bytes;
+    if (stages < 1) stages = 1;
+    if (stages > kGemmMaxStages) stages = kGemmMaxStages;
+    if (stages > ktiles) stages = ktiles > 0 ? ktiles : 1;
+    p.stages = stages;
+    const int smem = stages * stage_bytes + fixed;
+    dim3 grid((p.N + BN - 1) / BN, (p.M + 127) / 128, batch);
+    k_gemm_tc<BN><<<grid, 192, smem, lc.st>>>(p);
     lc.count();
     return PKV_OK;
 }
 
 int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
-    if (g.M <= 0 || g.N <= 0) return PKV_OK;
-    if (g.K <= 0 || g.npass <= 0 || g.npass > kGemmMaxPass) return PKV_ERR_INVALID_ARG;
+    if (g.M <= 0 || g.N <= 0 || g.batch <= 0) return PKV_OK;
+    if (g.K < 0 || g.npass <= 0 || g.npass > kGemmMaxPass || (!g.C && g.nout == 0)) return PKV_ERR_INVALID_ARG;
     GemmTcParams p;
     const int BN = (g.N <= 64) ? 64 : 128;
+    MapCache* cache = (MapCache*)lc.map_cache;
+    // distinct operands
+    const __nv_bfloat16* da[3];
+    const __nv_bfloat16* db[3];
+    p.nA = p.nB = 0;
     for (int i = 0; i < g.npass; ++i) {
-        int rc = tc_make_map_2d(&p.mapA[i], g.A[i], g.M, g.K, g.lda[i], 128);
-        if (rc != PKV_OK) return rc;
-        rc = tc_make_map_2d(&p.mapB[i], g.B[i], g.N, g.K, g.ldb[i], BN);
-        if (rc != PKV_OK) return rc;
+        int ia = -1, ib = -1;
+        for (int k = 0; k < p.nA; ++k) if (da[k] == g.A[i].p) ia = k;
+        for (int k = 0; k < p.nB; ++k) if (db[k] == g.B[i].p) ib = k;
+        if (ia < 0) {
+            if (p.nA == 3) return PKV_ERR_INVALID_ARG;
+            int rc = cached_map(cache, &p.mapA[p.nA], g.A[i].p, g.A[i].rows, g.A[i].cols, g.A[i].ld, 128);
+            if (rc != PKV_OK) return rc;
+            da[p.nA] = g.A[i].p;
+            ia = p.nA++;
+        }
+        if (ib < 0) {
+            if (p.nB == 3) return PKV_ERR_INVALID_ARG;
+            int rc = cached_map(cache, &p.mapB[p.nB], g.B[i].p, g.B[i].rows, g.B[i].cols, g.B[i].ld, BN);
+            if (rc != PKV_OK) return rc;
+            db[p.nB] = g.B[i].p;
+            ib = p.nB++;
+        }
+        p.pa[i] = ia;
+        p.pb[i] = ib;
     }
     p.npass = g.npass; p.M = g.M; p.N = g.N; p.K = g.K;
+    p.a_row0 = g.a_row0; p.a_col0 = g.a_col0; p.a_zrow = g.a_zrow; p.a_zcol = g.a_zcol;
+    p.b_row0 = g.b_row0; p.b_col0 = g.b_col0; p.b_zrow = g.b_zrow; p.b_zcol = g.b_zcol;
+    p.c_row0 = g.c_row0; p.c_col0 = g.c_col0; p.c_zrow = g.c_zrow; p.c_zcol = g.c_zcol;
+    p.c_rows = g.c_rows; p.c_cols = g.c_cols;
     p.C = g.C; p.ldc = g.ldc; p.alpha = g.alpha; p.addend = g.addend; p.ldadd = g.ldadd;
+    for (int i = 0; i < 3; ++i) p.out[i] = g.out[i];
+    p.ldo = g.ldo; p.nout = g.nout;
     p.accumulate = g.accumulate ? 1 : 0;
     p.lower_only = g.lower_only ? 1 : 0;
-    p.vec_ok = (((uintptr_t)g.C & 15) == 0 && g.ldc % 4 == 0 &&
+    p.k_tri = g.k_tri;
+    p.vec_ok = (g.C && ((uintptr_t)g.C & 15) == 0 && g.ldc % 4 == 0 && g.c_col0 % 4 == 0 && g.c_zcol % 4 == 0 &&
                 (!g.addend || (((uintptr_t)g.addend & 15) == 0 && g.ldadd % 4 == 0))) ? 1 : 0;
     p.status = status;
-    if (BN == 64) return launch_gemm<64, 4>(lc, p);
-    return launch_gemm<128, 3>(lc, p);
+    if (BN == 64) return launch_gemm<64>(lc, p, g.batch);
+    return launch_gemm<128>(lc, p, g.batch);
 }
 
 }  // namespace pkv

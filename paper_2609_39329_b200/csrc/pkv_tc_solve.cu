@@ -1,0 +1,397 @@
+// Ridge solve dW = S_T (S_H + lambda I)^{-1} (Eq. 8) with the dense work on the tensor cores.
+//
+// fp32 quantities are carried as bf16 triples (hi, mid, lo: 24 mantissa bits) and multiplied in
+// six passes (hh, hm, mh, hl, lh, mm) into fp32 tensor-memory accumulators, which reproduces an
+// fp32 product to ~2^-24; the two large triangular products at the end use pairs (three passes).
+//
+//   1. blocked right-looking Cholesky G = L L^T, block 128: the diagonal block is factored and
+//      inverted by one CTA in shared memory (k_potrf128), the panel is a GEMM with the block
+//      inverse, the trailing update a GEMM on the lower triangle;
+//   2. X = L^{-1} by recursive doubling from the 128-block inverses:
+//      [A 0; C B]^{-1} = [A^{-1} 0; -B^{-1} C A^{-1}  B^{-1}], every level two batched GEMMs;
+//   3. dW = (S_T X^T) X, two GEMMs that skip the zero tiles of the triangular factor.
+#include <math.h>
+
+#include "pkv_tc.h"
+
+namespace pkv {
+
+constexpr int PB = 128;     // Cholesky block
+constexpr int SB = 16;      // sub-block inside the diagonal kernel
+constexpr int LDS = PB + 1;
+
+__device__ __forceinline__ void split3(float v, __nv_bfloat16& h, __nv_bfloat16& m, __nv_bfloat16& l) {
+    h = __float2bfloat16_rn(v);
+    float r1 = v - __bfloat162float(h);
+    m = __float2bfloat16_rn(r1);
+    l = __float2bfloat16_rn(r1 - __bfloat162float(m));
+}
+
+struct Trip {
+    __nv_bfloat16* a[3];
+};
+
+// Factor the diagonal block at (k0, k0) of G (lower part read), invert the factor, write the
+// inverse (X3) and its transpose (XT3) as bf16 triples.  A pivot that is not positive and finite is
+// reported (smallest column wins) and replaced by 1 so that the call ends finite with
+// PKV_ERR_NOT_PD.
+//
+// The block is processed in 16-column sub-steps: the 16 x 16 diagonal piece is factored by one warp
+// entirely in registers (lane i holds row i, columns are exchanged with shuffles), the rows below
+// it by forward substitution (one row per thread), then the trailing lower triangle is updated.
+constexpr int kPotrfThreads = 512;
+
+__global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restrict__ G, int F, int k0, Trip X3,
+                                                            Trip XT3, DevStatus* status) {
+    extern __shared__ float smf[];
+    float(*A)[LDS] = reinterpret_cast<float(*)[LDS]>(smf);
+    float(*X)[LDS] = reinterpret_cast<float(*)[LDS]>(smf + PB * LDS);
+    float* rd = smf + 2 * PB * LDS;              // [128] reciprocals of the factor's diagonal
+    float(*T)[SB][SB + 1] = reinterpret_cast<float(*)[SB][SB + 1]>(rd + PB);   // [7][16][17]
+    if (status->code != 0) return;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nbk = min(PB, F - k0);
+    for (int i = tid; i < PB * PB; i += kPotrfThreads) {
+        const int r = i >> 7, c = i & 127;
+        float v = (r == c) ? 1.f : 0.f;
+        if (r < nbk && c <= r) v = G[(size_t)(k0 + r) * F + k0 + c];
+        A[r][c] = v;
+        X[r][c] = 0.f;
+    }
+    __syncthreads();
+    float minpiv = INFINITY;
+    for (int c0 = 0; c0 < PB; c0 += SB) {
+        if (warp == 0) {
+            const int li = lane & 15;            // lanes 16..31 mirror lanes 0..15 so every shuffle source is live
+            float a[SB];
+#pragma unroll
+            for (int k = 0; k < SB; ++k) a[k] = A[c0 + li][c0 + k];
+#pragma unroll
+            for (int j = 0; j < SB; ++j) {
+                float piv = __shfl_sync(0xffffffffu, a[j], j);
+                if (!(piv > 0.f) || !isfinite(piv)) {
+                    if (lane == 0 && c0 + j < nbk) {
+                        atomicCAS(&status->code, 0, PKV_ERR_NOT_PD);
+                        unsigned long long key = (unsigned long long)(k0 + c0 + j) + 1ull;
+                        unsigned long long old = status->bad_column;
+                        while (old == 0ull || key < old) {
+                            unsigned long long prev = atomicCAS(&status->bad_column, old, key);
+                            if (prev == old) break;
+                            old = prev;
+                        }
+                    }
+                    piv = 1.f;
+                }
+                if (c0 + j < nbk) minpiv = fminf(minpiv, piv);
+                const float dj = sqrtf(piv), rdj = 1.f / dj;
+                const float lij = (li == j) ? dj : a[j] * rdj;     // column j of the factor, row li
+                a[j] = lij;
+                if (lane == j) rd[c0 + j] = rdj;
+#pragma unroll
+                for (int k = j + 1; k < SB; ++k) {
+                    const float lkj = __shfl_sync(0xffffffffu, lij, k);
+                    a[k] = fmaf(-lij, lkj, a[k]);                  // rows above the diagonal hold unused values
+                }
+            }
+            if (lane < SB) {
+#pragma unroll
+                for (int k = 0; k < SB; ++k)
+                    if (k <= lane) A[c0 + lane][c0 + k] = a[k];
+            }
+        }
+        __syncthreads();
+        const int base = c0 + SB;
+        if (tid < PB - base) {     // rows below: x L_ss^T = a by forward substitution, one row per thread
+            const int r = base + tid;
+            float a[SB];
+#pragma unroll
+            for (int c = 0; c < SB; ++c) a[c] = A[r][c0 + c];
+#pragma unroll
+            for (int c = 0; c < SB; ++c) {
+                float x = a[c];
+#pragma unroll
+                for (int k = 0; k < c; ++k) x = fmaf(-a[k], A[c0 + c][c0 + k], x);
+                a[c] = x * rd[c0 + c];
+            }
+#pragma unroll
+            for (int c = 0; c < SB; ++c) A[r][c0 + c] = a[c];
+        }
+        __syncthreads();
+        {   // trailing update of the lower triangle inside the block; the thread's row stays in registers
+            const int ty = tid >> 4, tx = tid & 15;
+            for (int r = base + ty; r < PB; r += kPotrfThreads / 16) {
+                float ar[SB];
+#pragma unroll
+                for (int c = 0; c < SB; ++c) ar[c] = A[r][c0 + c];
+                for (int k = base + tx; k <= r; k += 16) {
+                    float acc = 0.f;
+#pragma unroll
+                    for (int c = 0; c < SB; ++c) acc = fmaf(ar[c], A[k][c0 + c], acc);
+                    A[r][k] -= acc;
+                }
+            }
+        }
+        __syncthreads();
+    }
+    if (tid == 0) status->min_pivot = fminf(status->min_pivot, minpiv);
+    // ---- inverse of the factor ----
+    if (tid < PB) {      // 16 x 16 diagonal sub-blocks, one column per thread
+        const int o = (tid >> 4) * SB, c = tid & 15;
+        float x[SB];
+#pragma unroll
+        for (int i = 0; i < SB; ++i) {
+            float s = (i == c) ? 1.f : 0.f;
+#pragma unroll
+            for (int k = 0; k < i; ++k) s = fmaf(-A[o + i][o + k], x[k], s);
+            x[i] = (i < c) ? 0.f : s * rd[o + i];
+        }
+#pragma unroll
+        for (int i = 0; i < SB; ++i) X[o + i][o + c] = x[i];
+    }
+    __syncthreads();
+    {   // off-diagonal sub-blocks by distance from the diagonal: X_ij = -X_ii sum_k L_ik X_kj;
+        // the two halves of the CTA take alternate blocks
+        const int grp = tid >> 8, t8 = tid & 255;
+        const int r = t8 >> 4, c = t8 & 15;
+        for (int dd = 1; dd < PB / SB; ++dd) {
+            const int nb = PB / SB - dd;
+            for (int j = grp; j < nb; j += 2) {
+                const int i = j + dd;
+                float t = 0.f;
+                for (int k = j; k < i; ++k)
+#pragma unroll
+                    for (int q = 0; q < SB; ++q) t = fmaf(A[SB * i + r][SB * k + q], X[SB * k + q][SB * j + c], t);
+                T[j][r][c] = t;
+            }
+            __syncthreads();
+            for (int j = grp; j < nb; j += 2) {
+                const int i = j + dd;
+                float x = 0.f;
+#pragma unroll
+                for (int q = 0; q < SB; ++q) x = fmaf(X[SB * i + r][SB * i + q], T[j][q][c], x);
+                X[SB * i + r][SB * j + c] = -x;
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = tid; i < PB * PB; i += kPotrfThreads) {
+        const int r = i >> 7, c = i & 127;
+        if (r < nbk && c < nbk) {
+            const size_t o = (size_t)(k0 + r) * F + k0 + c;
+            __nv_bfloat16 h, m, l;
+            split3((c <= r) ? X[r][c] : 0.f, h, m, l);
+            X3.a[0][o] = h; X3.a[1][o] = m; X3.a[2][o] = l;
+            split3((r <= c) ? X[c][r] : 0.f, h, m, l);
+            XT3.a[0][o] = h; XT3.a[1][o] = m; XT3.a[2][o] = l;
+        }
+    }
+}
+
+// src [rows][cols] fp32 (row stride lds) -> bf16 triple, row stride ldo
+__global__ void __launch_bounds__(256) k_split3(const float* __restrict__ src, long long lds, int rows, int cols,
+                                                Trip out, long long ldo, int nout) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)rows * cols) return;
+    const int r = (int)(i / cols), c = (int)(i % cols);
+    __nv_bfloat16 h, m, l;
+    split3(src[(size_t)r * lds + c], h, m, l);
+    const size_t o = (size_t)r * ldo + c;
+    out.a[0][o] = h;
+    out.a[1][o] = m;
+    if (nout > 2) out.a[2][o] = l;
+}
+
+static void launch_split3(const Lc& lc, const float* src, long long lds, int rows, int cols, Trip out, long long ldo,
+                          int nout) {
+    size_t n = (size_t)rows * cols;
+    if (!n) return;
+    k_split3<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(src, lds, rows, cols, out, ldo, nout);
+    lc.count();
+}
+
+// XT3[2sz + c][s + 2sz + r] = X3[s + 2sz + r][2sz + c]   (r < s clipped to the matrix, c < s)
+__global__ void k_transpose_blocks(Trip X3, Trip XT3, int F, int s) {
+    __shared__ __nv_bfloat16 t[3][32][33];
+    const int z = blockIdx.z;
+    const int r0 = s + 2 * s * z + blockIdx.y * 32, c0 = 2 * s * z + blockIdx.x * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int r = r0 + j, c = c0 + threadIdx.x;
+        if (r < F) {
+#pragma unroll
+            for (int a = 0; a < 3; ++a) t[a][j][threadIdx.x] = X3.a[a][(size_t)r * F + c];
+        }
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int c = c0 + j, r = r0 + threadIdx.x;
+        if (r < F) {
+#pragma unroll
+            for (int a = 0; a < 3; ++a) XT3.a[a][(size_t)c * F + r] = t[a][threadIdx.x][j];
+        }
+    }
+}
+
+static void six_pass(TcGemm& g, const Trip& A, long long lda, long long arows, long long acols, const Trip& B,
+                     long long ldb, long long brows, long long bcols) {
+    // (hi,hi) (hi,mid) (mid,hi) (hi,lo) (lo,hi) (mid,mid)
+    const int ia[6] = {0, 0, 1, 0, 2, 1}, ib[6] = {0, 1, 0, 2, 0, 1};
+    for (int i = 0; i < 6; ++i) {
+        g.A[i] = TcMat{A.a[ia[i]], lda, arows, acols};
+        g.B[i] = TcMat{B.a[ib[i]], ldb, brows, bcols};
+    }
+    g.npass = 6;
+}
+
+static void three_pass(TcGemm& g, const Trip& A, long long lda, long long arows, long long acols, const Trip& B,
+                       long long ldb, long long brows, long long bcols) {
+    const int ia[3] = {0, 0, 1}, ib[3] = {0, 1, 0};
+    for (int i = 0; i < 3; ++i) {
+        g.A[i] = TcMat{A.a[ia[i]], lda, arows, acols};
+        g.B[i] = TcMat{B.a[ib[i]], ldb, brows, bcols};
+    }
+    g.npass = 3;
+}
+
+// largest pairs * s * s over the doubling levels (elements of the TT workspace)
+static size_t tt_elems(int F) {
+    size_t best = (size_t)PB * PB;
+    for (long long s = PB; s < F; s *= 2) {
+        long long P = 0;
+        while ((2 * P + 1) * s < F) ++P;
+        if ((size_t)(P * s * s) > best) best = (size_t)(P * s * s);
+    }
+    return best;
+}
+
+size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, const pkv_dims* d) {
+    const size_t F = d->F, dm = d->d;
+    auto take = [&](size_t bytes) {
+        off = (off + 255) & ~(size_t)255;
+        char* p = base ? base + off : nullptr;
+        off += bytes;
+        return p;
+    };
+    for (int i = 0; i < 3; ++i) {
+        t->L3[i] = (__nv_bfloat16*)take(F * F * 2);
+        t->X3[i] = (__nv_bfloat16*)take(F * F * 2);
+        t->XT3[i] = (__nv_bfloat16*)take(F * F * 2);
+        t->P3[i] = (__nv_bfloat16*)take(F * PB * 2);
+        t->TT3[i] = (__nv_bfloat16*)take(tt_elems((int)F) * 2);
+    }
+    for (int i = 0; i < 3; ++i) {
+        t->S2[i] = (__nv_bfloat16*)take(dm * F * 2);
+        t->Z2[i] = (__nv_bfloat16*)take(dm * F * 2);
+    }
+    return off;
+}
+
+int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d) {
+    // regions of the triangular factors that no kernel writes must read as zero
+    const size_t F = d->F;
+    for (int i = 0; i < 3; ++i) {
+        if (cudaMemset(t->X3[i], 0, F * F * 2) != cudaSuccess) return PKV_ERR_CUDA;
+        if (cudaMemset(t->XT3[i], 0, F * F * 2) != cudaSuccess) return PKV_ERR_CUDA;
+        if (cudaMemset(t->L3[i], 0, F * F * 2) != cudaSuccess) return PKV_ERR_CUDA;
+        if (cudaMemset(t->P3[i], 0, F * PB * 2) != cudaSuccess) return PKV_ERR_CUDA;
+        if (cudaMemset(t->TT3[i], 0, tt_elems((int)F) * 2) != cudaSuccess) return PKV_ERR_CUDA;
+    }
+    static bool attr_set = false;
+    if (!attr_set) {
+        const int smem = (2 * PB * LDS + PB + 7 * SB * (SB + 1)) * (int)sizeof(float);
+        if (cudaFuncSetAttribute(k_potrf128, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+            return PKV_ERR_CUDA;
+        attr_set = true;
+    }
+    return PKV_OK;
+}
+
+int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int F, int d, float* dW,
+                        bool well_conditioned, DevStatus* status) {
+    const int nblk = (F + PB - 1) / PB;
+    const int smem = (2 * PB * LDS + PB + 7 * SB * (SB + 1)) * (int)sizeof(float);
+    Trip L3{{t->L3[0], t->L3[1], t->L3[2]}}, X3{{t->X3[0], t->X3[1], t->X3[2]}}, XT3{{t->XT3[0], t->XT3[1], t->XT3[2]}};
+    Trip P3{{t->P3[0], t->P3[1], t->P3[2]}}, TT3{{t->TT3[0], t->TT3[1], t->TT3[2]}};
+    int rc;
+    // ---- 1. factorisation ----
+    for (int b = 0; b < nblk; ++b) {
+        const int k0 = b * PB, k1 = min(F, k0 + PB), rem = F - k1;
+        k_potrf128<<<1, kPotrfThreads, smem, lc.st>>>(G, F, k0, X3, XT3, status);
+        lc.count();
+        if (rem <= 0) break;
+        // panel L21 = G21 L11^{-T}: split G21, multiply by the block inverse, keep L21 as a triple
+        launch_split3(lc, G + (size_t)k1 * F + k0, F, rem, PB, P3, PB, 3);
+        {
+            TcGemm g{};
+            six_pass(g, P3, PB, F, PB, X3, F, F, F);
+            g.b_row0 = k0; g.b_col0 = k0;
+            g.M = rem; g.N = PB; g.K = PB; g.batch = 1; g.alpha = 1.f;
+            g.c_row0 = k1; g.c_col0 = k0; g.c_rows = F; g.c_cols = F;
+            g.out[0] = L3.a[0]; g.out[1] = L3.a[1]; g.out[2] = L3.a[2]; g.ldo = F; g.nout = 3;
+            if ((rc = gemm_tc(lc, g, status))) return rc;
+        }
+        {   // trailing update G22 -= L21 L21^T on the lower triangle
+            TcGemm g{};
+            six_pass(g, L3, F, F, F, L3, F, F, F);
+            g.a_row0 = k1; g.a_col0 = k0; g.b_row0 = k1; g.b_col0 = k0;
+            g.M = rem; g.N = rem; g.K = PB; g.batch = 1; g.alpha = -1.f;
+            g.C = const_cast<float*>(G); g.ldc = F; g.accumulate = true; g.lower_only = true;
+            g.c_row0 = k1; g.c_col0 = k1; g.c_rows = F; g.c_cols = F;
+            if ((rc = gemm_tc(lc, g, status))) return rc;
+        }
+    }
+    // ---- 2. X = L^{-1} by recursive doubling ----
+    for (int s = PB; s < F; s *= 2) {
+        int P = 0;
+        while ((2 * P + 1) * s < F) ++P;
+        if (P == 0) break;
+        {   // TT_p = A_p^{-T} C_p^T   (A^{-1} the finished top-left inverse, C the block of L below it)
+            TcGemm g{};
+            six_pass(g, XT3, F, F, F, L3, F, F, F);
+            g.a_zrow = 2 * s; g.a_zcol = 2 * s;
+            g.b_row0 = s; g.b_zrow = 2 * s; g.b_zcol = 2 * s;
+            g.M = s; g.N = s; g.K = s; g.batch = P; g.alpha = 1.f;
+            g.c_zrow = s; g.c_rows = P * s; g.c_cols = s;
+            g.out[0] = TT3.a[0]; g.out[1] = TT3.a[1]; g.out[2] = TT3.a[2]; g.ldo = s; g.nout = 3;
+            if ((rc = gemm_tc(lc, g, status))) return rc;
+        }
+        {   // X_p(bottom-left) = -B_p^{-1} TT_p^T
+            TcGemm g{};
+            six_pass(g, X3, F, F, F, TT3, s, (long long)P * s, s);
+            g.a_row0 = s; g.a_col0 = s; g.a_zrow = 2 * s; g.a_zcol = 2 * s;
+            g.b_zrow = s;
+            g.M = s; g.N = s; g.K = s; g.batch = P; g.alpha = -1.f;
+            g.c_row0 = s; g.c_zrow = 2 * s; g.c_zcol = 2 * s; g.c_rows = F; g.c_cols = F;
+            g.out[0] = X3.a[0]; g.out[1] = X3.a[1]; g.out[2] = X3.a[2]; g.ldo = F; g.nout = 3;
+            if ((rc = gemm_tc(lc, g, status))) return rc;
+        }
+        dim3 grid(s / 32, s / 32, P), block(32, 8);
+        k_transpose_blocks<<<grid, block, 0, lc.st>>>(X3, XT3, F, s);
+        lc.count();
+    }
+    // ---- 3. dW = (S_T X^T) X ----
+    // The rounding of these two products is amplified by cond(L): pairs (2^-16, three passes) when
+    // the ridge keeps G well conditioned, triples (2^-24, six passes) otherwise.
+    const int nsp = well_conditioned ? 2 : 3;
+    Trip S2{{t->S2[0], t->S2[1], t->S2[2]}}, Z2{{t->Z2[0], t->Z2[1], t->Z2[2]}};
+    launch_split3(lc, S_T, F, d, F, S2, F, nsp);
+    {
+        TcGemm g{};
+        if (nsp == 2) three_pass(g, S2, F, d, F, X3, F, F, F);
+        else six_pass(g, S2, F, d, F, X3, F, F, F);
+        g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 1;
+        g.c_rows = d; g.c_cols = F;
+        g.out[0] = Z2.a[0]; g.out[1] = Z2.a[1]; g.out[2] = Z2.a[2]; g.ldo = F; g.nout = nsp;
+        if ((rc = gemm_tc(lc, g, status))) return rc;
+    }
+    {
+        TcGemm g{};
+        if (nsp == 2) three_pass(g, Z2, F, d, F, XT3, F, F, F);
+        else six_pass(g, Z2, F, d, F, XT3, F, F, F);
+        g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 2;
+        g.C = dW; g.ldc = F; g.c_rows = d; g.c_cols = F;
+        if ((rc = gemm_tc(lc, g, status))) return rc;
+    }
+    return PKV_OK;
+}
+
+}  // namespace pkv
