@@ -424,17 +424,25 @@ static void gram_simt(pkv_ctx* c, const Lc& lc, const float* X, const float* R, 
     gemm_tn_simt(lc, c->b.RT, n, c->b.XT, n, false, S_T, F, d, F, n, 1.f, nullptr, 0, accumulate);
 }
 
-static void solve_stage(pkv_ctx* c, const Lc& lc, const float* S_H, const float* S_T, float lam0, int mode,
-                        float* dW) {
+// S8.  `S_H_scratch` says that S_H may be overwritten (it is the context's own statistics buffer).
+static void solve_stage(pkv_ctx* c, const Lc& lc, float* S_H, const float* S_T, float lam0, int mode, float* dW,
+                        bool S_H_scratch) {
     const int F = c->dims.F, d = c->dims.d;
     Buffers& b = c->b;
     trace_fro2(lc, S_H, F, b.status);
-    make_ridge_matrix(lc, S_H, F, lam0, mode, b.solve.G, b.status);
-    cudaMemcpyAsync(b.solve.Y, S_T, (size_t)d * F * sizeof(float), cudaMemcpyDeviceToDevice, c->st);
-    if (c->engine == PKV_ENGINE_SIMT)
+    if (c->engine == PKV_ENGINE_SIMT) {
+        make_ridge_matrix(lc, S_H, F, lam0, mode, b.solve.G, b.status);
+        cudaMemcpyAsync(b.solve.Y, S_T, (size_t)d * F * sizeof(float), cudaMemcpyDeviceToDevice, c->st);
         ridge_solve_simt(lc, b.solve, F, d, dW, b.status);
-    else
-        pkv::tc_ridge_solve(lc, &b.tc, b.solve, F, d, dW, lam0, mode, b.status);
+    } else {
+        ridge_lambda(lc, F, lam0, mode, b.status);
+        float* S = S_H;
+        if (!S_H_scratch) {
+            cudaMemcpyAsync(b.solve.G, S_H, (size_t)F * F * sizeof(float), cudaMemcpyDeviceToDevice, c->st);
+            S = b.solve.G;
+        }
+        pkv::tc_ridge_solve(lc, &b.tc, S, S_T, F, d, dW, lam0, mode, b.status);
+    }
     sumsq(lc, dW, (int64_t)d * F, &b.status->dw_fro2);
 }
 
@@ -522,7 +530,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         if (rc != PKV_OK) return rc;
     }
     // S8 (Eq. 7-8)
-    solve_stage(c, lc, b.S_H, b.S_T, lambda, mode, dW);
+    solve_stage(c, lc, b.S_H, b.S_T, lambda, mode, dW, true);
     mark(c, ST_NEXT);
     // S9: xF_next = zF + hF W^T;  D = R - hC dW^T;  xC_next = xF_next - D
     if (next) {
@@ -651,6 +659,6 @@ extern "C" int pkv_ridge_solve(pkv_ctx* c, const float* S_H, const float* S_T, f
         return PKV_ERR_INVALID_ARG;
     Lc lc{c->st, &c->launches, c->map_cache};
     begin_call(c);
-    solve_stage(c, lc, S_H, S_T, lambda, lambda_mode, dW);
+    solve_stage(c, lc, const_cast<float*>(S_H), S_T, lambda, lambda_mode, dW, false);
     return end_call(c, stats, nullptr);
 }

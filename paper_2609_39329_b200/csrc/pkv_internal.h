@@ -74,6 +74,8 @@ void transpose_f32(const Lc& lc, const float* in, int rows, int cols, float* out
 // status->tr, fro2 from S [F][F]; optional sum of squares of an arbitrary buffer into *dst.
 void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status);
 void sumsq(const Lc& lc, const float* a, int64_t n, double* dst);
+// lambda from the statistics (mode) into status->lam (and min_pivot reset).
+void ridge_lambda(const Lc& lc, int F, float lam0, int mode, DevStatus* status);
 // lambda from the statistics (mode), G = S_H + lambda I written to G.
 void make_ridge_matrix(const Lc& lc, const float* S_H, int F, float lam0, int mode, float* G, DevStatus* status);
 // out = a - b (n elements); out may alias a.

@@ -558,43 +558,60 @@ __device__ __forceinline__ double warp_sum_d(double v) {
     return v;
 }
 
+// tr(S) and ||S||_F^2: one row per block iteration, float4 loads, fp32 partial sums per thread
+// (a few hundred terms each), double precision across threads.
 __global__ void __launch_bounds__(256) k_trace_fro2(const float* __restrict__ S, int F, DevStatus* status) {
-    size_t n = (size_t)F * F;
-    double fro = 0.0, tr = 0.0;
+    float fro[4] = {0.f, 0.f, 0.f, 0.f};
+    double tr = 0.0;
     int bad = 0;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        float v = S[i];
-        if (!isfinite(v)) bad = 1;
-        fro += (double)v * (double)v;
-        if (i / F == i % F) tr += (double)v;
+    const bool vec = (F % 4 == 0) && (((uintptr_t)S & 15) == 0);
+    for (int r = blockIdx.x; r < F; r += gridDim.x) {
+        const float* row = S + (size_t)r * F;
+        if (vec) {
+            for (int c = threadIdx.x * 4; c < F; c += 1024) {
+                float4 v = *reinterpret_cast<const float4*>(row + c);
+                fro[0] = fmaf(v.x, v.x, fro[0]); fro[1] = fmaf(v.y, v.y, fro[1]);
+                fro[2] = fmaf(v.z, v.z, fro[2]); fro[3] = fmaf(v.w, v.w, fro[3]);
+            }
+        } else {
+            for (int c = threadIdx.x; c < F; c += 256) fro[0] = fmaf(row[c], row[c], fro[0]);
+        }
+        if (threadIdx.x == 0) tr += (double)row[r];
     }
-    fro = warp_sum_d(fro);
-    tr = warp_sum_d(tr);
-    if ((threadIdx.x & 31) == 0) {
-        atomicAdd(&status->fro2, fro);
-        if (tr != 0.0) atomicAdd(&status->tr, tr);
-    }
+    float f = (fro[0] + fro[1]) + (fro[2] + fro[3]);
+    if (!isfinite(f)) bad = 1;
+    double fd = warp_sum_d((double)f);
+    if ((threadIdx.x & 31) == 0) atomicAdd(&status->fro2, fd);
+    if (threadIdx.x == 0 && tr != 0.0) atomicAdd(&status->tr, tr);
     if (bad) raise(status, PKV_ERR_NONFINITE);
 }
 
 void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status) {
-    k_trace_fro2<<<296, 256, 0, lc.st>>>(S, F, status);
+    k_trace_fro2<<<min(F, 1184), 256, 0, lc.st>>>(S, F, status);
     lc.count();
 }
 
 __global__ void __launch_bounds__(256) k_sumsq(const float* __restrict__ a, size_t n, double* dst) {
-    double s = 0.0;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        float v = a[i];
-        s += (double)v * (double)v;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const size_t n4 = (((uintptr_t)a & 15) == 0) ? n / 4 : 0;
+    const float4* a4 = reinterpret_cast<const float4*>(a);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        float4 v = a4[i];
+        acc[0] = fmaf(v.x, v.x, acc[0]); acc[1] = fmaf(v.y, v.y, acc[1]);
+        acc[2] = fmaf(v.z, v.z, acc[2]); acc[3] = fmaf(v.w, v.w, acc[3]);
     }
-    s = warp_sum_d(s);
+    for (size_t i = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        acc[0] = fmaf(a[i], a[i], acc[0]);
+    double s = warp_sum_d((double)((acc[0] + acc[1]) + (acc[2] + acc[3])));
     if ((threadIdx.x & 31) == 0) atomicAdd(dst, s);
 }
 
 void sumsq(const Lc& lc, const float* a, int64_t n, double* dst) {
     if (n <= 0) return;
-    k_sumsq<<<296, 256, 0, lc.st>>>(a, (size_t)n, dst);
+    int blocks = (int)((n / 4 + 255) / 256);
+    if (blocks > 1184) blocks = 1184;
+    if (blocks < 1) blocks = 1;
+    k_sumsq<<<blocks, 256, 0, lc.st>>>(a, (size_t)n, dst);
     lc.count();
 }
 
@@ -629,10 +646,15 @@ __global__ void k_ridge_matrix(const float* __restrict__ S, int F, float* __rest
     }
 }
 
-void make_ridge_matrix(const Lc& lc, const float* S_H, int F, float lam0, int mode, float* G, DevStatus* status) {
+void ridge_lambda(const Lc& lc, int F, float lam0, int mode, DevStatus* status) {
     k_lambda<<<1, 1, 0, lc.st>>>(F, lam0, mode, status);
+    lc.count();
+}
+
+void make_ridge_matrix(const Lc& lc, const float* S_H, int F, float lam0, int mode, float* G, DevStatus* status) {
+    ridge_lambda(lc, F, lam0, mode, status);
     k_ridge_matrix<<<592, 256, 0, lc.st>>>(S_H, F, G, status);
-    lc.count(2);
+    lc.count();
 }
 
 __global__ void k_sub(const float* __restrict__ a, const float* __restrict__ b, size_t n, float* __restrict__ out) {

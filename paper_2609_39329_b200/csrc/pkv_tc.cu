@@ -223,12 +223,12 @@ int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
     return attention_tc(lc, t, d, a, nullptr, status);
 }
 
-void tc_ridge_solve(const Lc& lc, TcBuffers* t, const SolveWs& ws, int F, int d, float* dW, float lam0, int mode,
-                    DevStatus* status) {
+void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int F, int d, float* dW, float lam0,
+                    int mode, DevStatus* status) {
     // Under the adaptive scale of Eq. 7 cond(G) ~ (tr(S_H)/sigma_max)/lambda0; lambda0 >= 0.05 keeps it
     // to a few tens.  Absolute and trace-mean coefficients give no such bound.
     const bool well = (mode == PKV_LAMBDA_PAPER) && (lam0 >= 0.05f);
-    tc_ridge_solve_impl(lc, &t->solve, ws.G, ws.Y, F, d, dW, well, status);
+    tc_ridge_solve_impl(lc, &t->solve, S, S_T, F, d, dW, well, status);
 }
 
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a) {

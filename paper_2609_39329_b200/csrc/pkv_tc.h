@@ -59,7 +59,7 @@ struct TcSolveBuffers {
 };
 size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, const pkv_dims* d);
 int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d);
-// dW [d][F] = S_T G^{-1}; G [F][F] (lower part read) is destroyed.
+// dW [d][F] = S_T (S + lambda I)^{-1}, lambda = status->lam; S [F][F] (lower part read) is destroyed.
 int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int F, int d, float* dW,
                         bool well_conditioned, DevStatus* status);
 
@@ -114,8 +114,9 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArg
 int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status);
 void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, const float* R, int n, float* S_H,
              float* S_T, bool accumulate, DevStatus* status);
-void tc_ridge_solve(const Lc& lc, TcBuffers* t, const SolveWs& ws, int F, int d, float* dW, float lam0, int mode,
-                    DevStatus* status);
+// S [F][F] is destroyed; S_T is only read.
+void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int F, int d, float* dW, float lam0,
+                    int mode, DevStatus* status);
 void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* d, int N, const void* Wdown, const float* dW,
                     const float* zF, const float* R, float* xF_next, float* D, DevStatus* status);
 

@@ -31,7 +31,8 @@ struct Trip {
     __nv_bfloat16* a[3];
 };
 
-// Factor the diagonal block at (k0, k0) of G (lower part read), invert the factor, write the
+// Factor the diagonal block at (k0, k0) of G = S + lambda I (lower part of S read, lambda from the
+// status word added on the diagonal), invert the factor, write the
 // inverse (X3) and its transpose (XT3) as bf16 triples.  A pivot that is not positive and finite is
 // reported (smallest column wins) and replaced by 1 so that the call ends finite with
 // PKV_ERR_NOT_PD.
@@ -51,10 +52,14 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
     if (status->code != 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nbk = min(PB, F - k0);
+    const float lam = status->lam;
     for (int i = tid; i < PB * PB; i += kPotrfThreads) {
         const int r = i >> 7, c = i & 127;
         float v = (r == c) ? 1.f : 0.f;
-        if (r < nbk && c <= r) v = G[(size_t)(k0 + r) * F + k0 + c];
+        if (r < nbk && c <= r) {
+            v = G[(size_t)(k0 + r) * F + k0 + c];
+            if (r == c) v += lam;                     // G = S_H + lambda I is never materialised
+        }
         A[r][c] = v;
         X[r][c] = 0.f;
     }
