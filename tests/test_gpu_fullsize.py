@@ -1,0 +1,163 @@
+"""Full-size checks in the launch configuration bench.py times (tensor-core engine, default split plan).
+
+Config 2 (the benchmark workload) is compared with the fp64 oracle element by element.  For configs
+3-5 the oracle cannot run a whole block in seconds, so every stage is checked at the full shapes on what
+the oracle can compute one by one (sampled attention rows at full cache length, the full Gram, the full
+ridge solve) and on properties that hold at any size (stationarity of the ridge solution, the ridge
+residual identity between the returned states)."""
+import numpy as np
+import pytest
+
+from oracle import pkv_oracle as orc
+from paper_2609_39329_b200 import inputs as gen
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+ATTN_TOL = 2e-2
+DW_TOL = 5e-3
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    from paper_2609_39329_b200 import binding
+    assert torch.cuda.is_available()
+    return binding
+
+
+def test_config2_whole_block_matches_oracle(B):
+    import torch
+    cfg = gen.benchmark_config(2)
+    lay = gen.gen_layer(cfg, 0)
+    x = gen.gen_reference(cfg)
+    ref = orc.build_patch(lay["weights"], lay["K"], lay["V"], lay["kept"], x, x, [0, cfg.N], cfg.L, cfg.lam0, cfg)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    w = B.to_device(lay["weights"], cfg.dtype)
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    off, idx = gen.kept_to_csr(lay["kept"])
+    xt = torch.from_numpy(x).cuda()
+    out = ctx.build_patch(w, kv["K"], kv["V"], off, torch.from_numpy(idx).cuda(), xt, xt, [0, cfg.N], cfg.L, cfg.lam0)
+    dW = out["dW"].cpu().numpy()
+    err = H.rel_fro(dW, ref["dW"])
+    print("config 2 dW rel fro err %.3e  lambda %.5g (oracle %.5g)" % (err, out["stats"]["lambda_eff"], ref["lam"]))
+    assert err <= DW_TOL
+    np.testing.assert_allclose(out["stats"]["lambda_eff"], ref["lam"], rtol=1e-3)
+    assert H.rel_fro(out["xF_next"].cpu().numpy(), ref["xF_next"]) <= 1e-3
+    assert H.rel_fro(out["xC_next"].cpu().numpy(), ref["xC_next"]) <= 1e-3
+    gap = out["xF_next"].double() - out["xC_next"].double()
+    assert H.rel_fro(gap.cpu().numpy(), ref["xF_next"] - ref["xC_next"]) <= 2e-2
+    np.testing.assert_allclose(out["stats"]["resid_fro2"], float((gap * gap).sum()), rtol=1e-3)
+    np.testing.assert_allclose(out["stats"]["resid_fro2"], ref["res_fro2"], rtol=3e-2)
+    # merge: bit-exact against the two stated roundings
+    Wm = w["Wdown"].clone()
+    ctx.merge(Wm, out["dW"])
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(Wm.float().cpu().numpy(), orc.merge(lay["weights"]["Wdown"], dW, "bf16"))
+    ctx.close()
+
+
+def sampled_attention_check(B, cfg, n_samples=48, seed=0):
+    import torch
+    r = np.random.default_rng(seed)
+    N = cfg.N
+    kvd = gen.gen_cache(cfg, 0)
+    q = (r.standard_normal((2, N, cfg.Hq, cfg.hd)) * 1.3).astype(np.float32)
+    k = r.standard_normal((2, N, cfg.Hkv, cfg.hd)).astype(np.float32)
+    v = r.standard_normal((2, N, cfg.Hkv, cfg.hd)).astype(np.float32)
+    kept = gen.select_kept(cfg, 0, kvd["K"], gen.gen_obs_queries(cfg, 0) if cfg.kept_rule == "window_topk" else None)
+    off, idx = gen.kept_to_csr(kept)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    kv = B.to_device({"K": kvd["K"], "V": kvd["V"]}, cfg.dtype)
+    tq, tk, tv = (torch.from_numpy(t.reshape(2, N, -1)).cuda() for t in (q, k, v))
+    gF, gC, gD = ctx.attention(tq, tk, tv, kv["K"], kv["V"], off, torch.from_numpy(idx).cuda(), [0, N])
+    # compaction is bit-exact on every kept row
+    Kc, Vc = ctx.gather_kept(kv["K"], kv["V"], off, torch.from_numpy(idx).cuda())
+    Ko, Vo = orc.gather_cache(kvd["K"], kvd["V"], kept)
+    np.testing.assert_array_equal(Kc.float().cpu().numpy(), np.concatenate(Ko))
+    np.testing.assert_array_equal(Vc.float().cpu().numpy(), np.concatenate(Vo))
+    gF, gC, gD = (t.cpu().numpy().reshape(N, cfg.Hq, cfg.hd) for t in (gF, gC, gD))
+    ctx.close()
+    toks = np.unique(np.concatenate([[0, 1, N - 1], r.integers(0, N, n_samples)]))
+    worst = 0.0
+    for h in r.choice(cfg.Hq, size=min(cfg.Hq, 6), replace=False):
+        kh = h // cfg.g
+        for stream, got, Kh, Vh in ((0, gF, kvd["K"][kh], kvd["V"][kh]), (1, gC, Ko[kh], Vo[kh])):
+            # one query row at a time: cache rows + causal part of the chunk
+            keys = np.concatenate([Kh.astype(np.float64), k[stream, :, kh].astype(np.float64)])
+            vals = np.concatenate([Vh.astype(np.float64), v[stream, :, kh].astype(np.float64)])
+            rows = len(Kh)
+            want = np.zeros((len(toks), cfg.hd))
+            for n, t in enumerate(toks):
+                lg = keys[:rows + t + 1] @ q[stream, t, h].astype(np.float64) / np.sqrt(cfg.hd)
+                p = np.exp(lg - lg.max())
+                want[n] = (p / p.sum()) @ vals[:rows + t + 1]
+            scale = np.abs(got[:, h]).max()
+            worst = max(worst, np.abs(got[toks, h] - want).max() / scale)
+    np.testing.assert_array_equal(gD, gF - gC)
+    return worst
+
+
+@pytest.mark.parametrize("cfg_id", [2, 3, 4, 5])
+def test_attention_sampled_rows_at_full_cache_length(B, cfg_id):
+    cfg = gen.benchmark_config(cfg_id)
+    worst = sampled_attention_check(B, cfg)
+    print("config %d attention sampled max rel err %.3e" % (cfg_id, worst))
+    assert worst <= ATTN_TOL
+
+
+@pytest.mark.parametrize("cfg_id", [3, 4, 5])
+def test_statistics_and_ridge_solve_at_full_width(B, cfg_id):
+    import torch
+    cfg = gen.benchmark_config(cfg_id)
+    r = np.random.default_rng(cfg_id)
+    N, F, d = cfg.N, cfg.F, cfg.d
+    # features with a decaying spectrum and a dominant direction, targets small differences
+    X = (r.standard_normal((N, F)) * np.exp(r.uniform(-2, 0.5, F)) + 0.5 * r.standard_normal((N, 1))).astype(np.float32)
+    R = (0.05 * r.standard_normal((N, d))).astype(np.float32)
+    S_H, S_T = orc.sufficient_statistics(X, R)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    gH, gT = ctx.gram(torch.from_numpy(X).cuda(), torch.from_numpy(R).cuda())
+    assert H.rel_fro(gH.cpu().numpy(), S_H) <= 2e-4
+    assert H.rel_fro(gT.cpu().numpy(), S_T) <= 2e-4
+    lams = cfg.lam_sweep if cfg.lam_sweep else (cfg.lam0,)
+    for lam0 in lams:
+        lam = orc.ridge_lambda(S_H, lam0)
+        dW, st = ctx.ridge_solve(gH, gT, lam0, B.LAMBDA_PAPER)
+        dWn = dW.cpu().numpy().astype(np.float64)
+        # stationarity of Eq. 6 in fp64 with the GPU's own statistics
+        Hg, Tg = gH.cpu().numpy().astype(np.float64), gT.cpu().numpy().astype(np.float64)
+        lam_g = st["lambda_eff"]
+        stat = np.linalg.norm(dWn @ Hg + lam_g * dWn - Tg) / np.linalg.norm(Tg)
+        want = orc.ridge_solve(S_H, S_T, lam)
+        err = H.rel_fro(dWn, want)
+        print("config %d lambda0 %g: dW rel fro err %.3e, stationarity %.3e, min pivot %.3g" %
+              (cfg_id, lam0, err, stat, st["min_pivot"]))
+        np.testing.assert_allclose(lam_g, lam, rtol=1e-3)
+        assert err <= 2e-3
+        assert stat <= 2e-3
+    ctx.close()
+
+
+@pytest.mark.parametrize("cfg_id", [3, 4, 5])
+def test_whole_block_runs_at_full_size_and_keeps_the_ridge_identities(B, cfg_id):
+    import torch
+    cfg = gen.benchmark_config(cfg_id)
+    lay = gen.gen_layer(cfg, 0)
+    x = gen.gen_reference(cfg)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    w = B.to_device(lay["weights"], cfg.dtype)
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    off, idx = gen.kept_to_csr(lay["kept"])
+    xt = torch.from_numpy(x).cuda()
+    out = ctx.build_patch(w, kv["K"], kv["V"], off, torch.from_numpy(idx).cuda(), xt, xt, [0, cfg.N], cfg.L, cfg.lam0)
+    st = out["stats"]
+    assert torch.isfinite(out["dW"]).all() and st["min_pivot"] > 0
+    np.testing.assert_allclose(st["lambda_eff"], cfg.lam0 * st["fro2"] / st["trace"], rtol=1e-5)    # Eq. 7
+    gap = out["xF_next"].double() - out["xC_next"].double()
+    np.testing.assert_allclose(float((gap * gap).sum()), st["resid_fro2"], rtol=1e-3)
+    assert 0 < st["resid_fro2"] < st["target_fro2"]          # the patch reduces the block-output gap
+    np.testing.assert_allclose(float((out["dW"].double() ** 2).sum()), st["dW_fro2"], rtol=1e-4)
+    print("config %d: lambda %.4g, ||T||^2 %.4g -> residual %.4g" % (cfg_id, st["lambda_eff"], st["target_fro2"],
+                                                                     st["resid_fro2"]))
+    ctx.close()
