@@ -201,6 +201,27 @@ int pkv_attention(pkv_ctx* ctx, const float* q, const float* k_new, const float*
 int pkv_gram(pkv_ctx* ctx, const float* X, const float* R, int32_t n, float* S_H, float* S_T,
              int accumulate);
 
+/* The statistics of pkv_gram for callers that cannot allocate device memory (no counterpart in the
+ * paper: an addition of this library).  Hosts that own all device memory through their own pool, or
+ * that sit in a latency-critical loop where cudaMalloc (a device-wide synchronisation) is not
+ * acceptable, cannot create a pkv_ctx, because a context allocates its workspace.  This call needs no
+ * context: the scratch its kernels use (bf16 operand copies, the status word) lives in a fixed device
+ * array inside the library image, about 4.2 MB, which every GPU that loads the library holds until
+ * the process exits.  It calls no cudaMalloc/cudaFree and no allocating library routine.
+ *   X [n][F], R [n][d], S_H [F][F], S_T [d][F]: device fp32, 16-byte aligned; meaning as in pkv_gram.
+ *   Limits: n <= PKV_NOALLOC_MAX_N, F <= PKV_NOALLOC_MAX_F, d <= PKV_NOALLOC_MAX_D, F % 8 == d % 8 == 0;
+ *   anything larger returns PKV_ERR_UNSUPPORTED (as does a device without tcgen05 tensor cores).
+ *   The first call on a device resolves the array's address and sets kernel attributes: make that
+ *   call before any stream capture begins.  All calls share the one array, which keeps the previous
+ *   call's contents (the call clears what must start at zero): calls whose kernels may overlap on the
+ *   GPU, e.g. from two streams or two host threads, race and must be serialised by the caller.
+ *   The call ends with one synchronisation of cuda_stream to read its status word. */
+#define PKV_NOALLOC_MAX_N 512
+#define PKV_NOALLOC_MAX_F 1024
+#define PKV_NOALLOC_MAX_D 1024
+int pkv_gram_noalloc(const float* X, const float* R, int32_t n, int32_t F, int32_t d, float* S_H, float* S_T,
+                     int accumulate, void* cuda_stream);
+
 /* Ridge solve alone (Eq. 7-8): dW = S_T (S_H + lambda I)^{-1}.  S_H, S_T are read, not
  * modified. */
 int pkv_ridge_solve(pkv_ctx* ctx, const float* S_H, const float* S_T, float lambda, int lambda_mode,

@@ -112,6 +112,9 @@ def lib() -> C.CDLL:
                                 C.c_int32, C.c_int32, P(C.c_int32), C.c_void_p, C.c_void_p, C.c_void_p]
     L.pkv_gram.restype = C.c_int
     L.pkv_gram.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int]
+    L.pkv_gram_noalloc.restype = C.c_int
+    L.pkv_gram_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                   C.c_int, C.c_void_p]
     L.pkv_ridge_solve.restype = C.c_int
     L.pkv_ridge_solve.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_void_p, P(pkv_stats)]
     L.pkv_set_timing.restype = C.c_int
@@ -319,6 +322,23 @@ class PkvContext:
         if rc != 0:
             self._raise(rc, st.as_dict())
         return dW, st.as_dict()
+
+
+def gram_noalloc(X, R, S_H=None, S_T=None, accumulate=False, stream=None):
+    """pkv_gram_noalloc: the Eq. 9 statistics without a context and without any device allocation by the
+    library (the output tensors are the caller's).  For hosts that cannot call cudaMalloc at this point;
+    sizes are limited (n <= 512, F, d <= 1024) and concurrent calls must be serialised by the caller."""
+    import torch
+    n, F = int(X.shape[0]), int(X.shape[1])
+    d = int(R.shape[1])
+    if S_H is None:
+        S_H = torch.zeros((F, F), dtype=torch.float32, device=X.device)
+        S_T = torch.zeros((d, F), dtype=torch.float32, device=X.device)
+    sp = C.c_void_p(stream.cuda_stream if stream is not None else torch.cuda.current_stream().cuda_stream)
+    rc = lib().pkv_gram_noalloc(_ptr(X), _ptr(R), n, F, d, _ptr(S_H), _ptr(S_T), 1 if accumulate else 0, sp)
+    if rc != 0:
+        raise PkvError(rc, lib().pkv_strerror(rc).decode())
+    return S_H, S_T
 
 
 def to_device(arrays: Dict[str, np.ndarray], dtype: str, device="cuda"):

@@ -219,6 +219,17 @@ void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, cons
     gemm_pair_pair(lc, t->RT, t->ldT, t->XT, t->ldT, S_T, F, dm, F, n, 1.f, nullptr, 0, accumulate, status);
 }
 
+// The statistics of Eq. 9 with caller-supplied operand buffers (used by the entry point that owns a
+// fixed device array instead of a context workspace).
+int tc_gram_with_buffers(const Lc& lc, Pair XT, Pair RT, int ldT, const float* X, const float* R, int n, int F, int dm,
+                         float* S_H, float* S_T, bool accumulate, DevStatus* status) {
+    transpose_split(lc, X, n, F, ldT, XT);
+    transpose_split(lc, R, n, dm, ldT, RT);
+    int rc = gemm_pair_pair(lc, XT, ldT, XT, ldT, S_H, F, F, F, n, 1.f, nullptr, 0, accumulate, status);
+    if (rc != PKV_OK) return rc;
+    return gemm_pair_pair(lc, RT, ldT, XT, ldT, S_T, F, dm, F, n, 1.f, nullptr, 0, accumulate, status);
+}
+
 int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status) {
     return attention_tc(lc, t, d, a, nullptr, status);
 }

@@ -114,6 +114,8 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArg
 int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status);
 void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, const float* R, int n, float* S_H,
              float* S_T, bool accumulate, DevStatus* status);
+int tc_gram_with_buffers(const Lc& lc, Pair XT, Pair RT, int ldT, const float* X, const float* R, int n, int F, int dm,
+                         float* S_H, float* S_T, bool accumulate, DevStatus* status);
 // S [F][F] is destroyed; S_T is only read.
 void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int F, int d, float* dW, float lam0,
                     int mode, DevStatus* status);
