@@ -40,7 +40,13 @@ struct Trip {
 // The block is processed in 16-column sub-steps: the 16 x 16 diagonal piece is factored by one warp
 // entirely in registers (lane i holds row i, columns are exchanged with shuffles), the rows below
 // it by forward substitution (one row per thread), then the trailing lower triangle is updated.
-constexpr int kPotrfThreads = 512;
+constexpr int kPotrfThreads = 1024;
+constexpr int kPotrfTElems = 64 * 65;       // largest doubling temporary (one 64 x 64 block, padded)
+constexpr int kPotrfSmemBytes = (2 * PB * LDS + PB + kPotrfTElems) * (int)sizeof(float);
+
+__device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) {
+    return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
+}
 
 __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restrict__ G, int F, int k0, Trip X3,
                                                             Trip XT3, DevStatus* status) {
@@ -48,23 +54,49 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
     float(*A)[LDS] = reinterpret_cast<float(*)[LDS]>(smf);
     float(*X)[LDS] = reinterpret_cast<float(*)[LDS]>(smf + PB * LDS);
     float* rd = smf + 2 * PB * LDS;              // [128] reciprocals of the factor's diagonal
-    float(*T)[SB][SB + 1] = reinterpret_cast<float(*)[SB][SB + 1]>(rd + PB);   // [7][16][17]
+    float* T = rd + PB;                          // doubling temporary
     if (status->code != 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nbk = min(PB, F - k0);
     const float lam = status->lam;
-    for (int i = tid; i < PB * PB; i += kPotrfThreads) {
-        const int r = i >> 7, c = i & 127;
-        float v = (r == c) ? 1.f : 0.f;
-        if (r < nbk && c <= r) {
-            v = G[(size_t)(k0 + r) * F + k0 + c];
-            if (r == c) v += lam;                     // G = S_H + lambda I is never materialised
+    // ---- load the lower part (identity outside the block's extent), lambda on the diagonal ----
+    if (nbk == PB && (F & 3) == 0) {
+        constexpr int kLd = 4096 / kPotrfThreads;
+        float4 v[kLd];
+#pragma unroll
+        for (int u = 0; u < kLd; ++u) {
+            const int i = tid + u * kPotrfThreads;           // 4096 float4 of the block
+            const int r = i >> 5, c4 = (i & 31) * 4;
+            v[u] = (c4 <= r) ? *reinterpret_cast<const float4*>(G + (size_t)(k0 + r) * F + k0 + c4)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        A[r][c] = v;
-        X[r][c] = 0.f;
+#pragma unroll
+        for (int u = 0; u < kLd; ++u) {
+            const int i = tid + u * kPotrfThreads;
+            const int r = i >> 5, c4 = (i & 31) * 4;
+            const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int c = c4 + t;
+                A[r][c] = (c < r) ? e[t] : ((c == r) ? e[t] + lam : 0.f);
+                X[r][c] = 0.f;
+            }
+        }
+    } else {
+        for (int i = tid; i < PB * PB; i += kPotrfThreads) {
+            const int r = i >> 7, c = i & 127;
+            float v = (r == c) ? 1.f : 0.f;
+            if (r < nbk && c <= r) {
+                v = G[(size_t)(k0 + r) * F + k0 + c];
+                if (r == c) v += lam;                     // G = S_H + lambda I is never materialised
+            }
+            A[r][c] = v;
+            X[r][c] = 0.f;
+        }
     }
     __syncthreads();
     float minpiv = INFINITY;
+    int bad_col = -1;
     for (int c0 = 0; c0 < PB; c0 += SB) {
         if (warp == 0) {
             const int li = lane & 15;            // lanes 16..31 mirror lanes 0..15 so every shuffle source is live
@@ -74,22 +106,13 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
 #pragma unroll
             for (int j = 0; j < SB; ++j) {
                 float piv = __shfl_sync(0xffffffffu, a[j], j);
-                if (!(piv > 0.f) || !isfinite(piv)) {
-                    if (lane == 0 && c0 + j < nbk) {
-                        atomicCAS(&status->code, 0, PKV_ERR_NOT_PD);
-                        unsigned long long key = (unsigned long long)(k0 + c0 + j) + 1ull;
-                        unsigned long long old = status->bad_column;
-                        while (old == 0ull || key < old) {
-                            unsigned long long prev = atomicCAS(&status->bad_column, old, key);
-                            if (prev == old) break;
-                            old = prev;
-                        }
-                    }
-                    piv = 1.f;
-                }
+                const bool okp = (piv > 0.f) && (piv < INFINITY);
+                if (!okp && bad_col < 0 && c0 + j < nbk) bad_col = c0 + j;
+                piv = okp ? piv : 1.f;
                 if (c0 + j < nbk) minpiv = fminf(minpiv, piv);
-                const float dj = sqrtf(piv), rdj = 1.f / dj;
-                const float lij = (li == j) ? dj : a[j] * rdj;     // column j of the factor, row li
+                float rdj = rsqrtf(piv);
+                rdj = rdj * fmaf(-0.5f * piv * rdj, rdj, 1.5f);    // one Newton step: full fp32 accuracy
+                const float lij = a[j] * rdj;                       // row li of column j (the pivot row gets sqrt(piv))
                 a[j] = lij;
                 if (lane == j) rd[c0 + j] = rdj;
 #pragma unroll
@@ -138,7 +161,19 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
         }
         __syncthreads();
     }
-    if (tid == 0) status->min_pivot = fminf(status->min_pivot, minpiv);
+    if (tid == 0) {
+        status->min_pivot = fminf(status->min_pivot, minpiv);
+        if (bad_col >= 0) {
+            atomicCAS(&status->code, 0, PKV_ERR_NOT_PD);
+            unsigned long long key = (unsigned long long)(k0 + bad_col) + 1ull;
+            unsigned long long old = status->bad_column;
+            while (old == 0ull || key < old) {
+                unsigned long long prev = atomicCAS(&status->bad_column, old, key);
+                if (prev == old) break;
+                old = prev;
+            }
+        }
+    }
     // ---- inverse of the factor ----
     if (tid < PB) {      // 16 x 16 diagonal sub-blocks, one column per thread
         const int o = (tid >> 4) * SB, c = tid & 15;
@@ -154,40 +189,68 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
         for (int i = 0; i < SB; ++i) X[o + i][o + c] = x[i];
     }
     __syncthreads();
-    {   // off-diagonal sub-blocks by distance from the diagonal: X_ij = -X_ii sum_k L_ik X_kj;
-        // the two halves of the CTA take alternate blocks
-        const int grp = tid >> 8, t8 = tid & 255;
-        const int r = t8 >> 4, c = t8 & 15;
-        for (int dd = 1; dd < PB / SB; ++dd) {
-            const int nb = PB / SB - dd;
-            for (int j = grp; j < nb; j += 2) {
-                const int i = j + dd;
-                float t = 0.f;
-                for (int k = j; k < i; ++k)
-#pragma unroll
-                    for (int q = 0; q < SB; ++q) t = fmaf(A[SB * i + r][SB * k + q], X[SB * k + q][SB * j + c], t);
-                T[j][r][c] = t;
+    // recursive doubling inside the block: [Xa 0; C Xb] -> bottom-left = -Xb (C Xa); every level is two
+    // dense products over all pairs, four output columns per thread
+    for (int s = SB; s < PB; s *= 2) {
+        const int lt = s + 1;
+        const int groups = (PB / (2 * s)) * s * (s / 4);
+        for (int g = tid; g < groups; g += kPotrfThreads) {       // T_p = C_p Xa_p
+            const int cg = g % (s / 4), r = (g / (s / 4)) % s, p = g / ((s / 4) * s);
+            const int o = 2 * p * s, c = cg * 4;
+            float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
+            const float* arow = &A[o + s + r][o];
+#pragma unroll 4
+            for (int k = c; k < s; ++k) {                          // Xa is lower triangular: rows >= column
+                const float av = arow[k];
+                const float* xr = &X[o + k][o + c];
+                t0 = fmaf(av, xr[0], t0); t1 = fmaf(av, xr[1], t1);
+                t2 = fmaf(av, xr[2], t2); t3 = fmaf(av, xr[3], t3);
             }
-            __syncthreads();
-            for (int j = grp; j < nb; j += 2) {
-                const int i = j + dd;
-                float x = 0.f;
-#pragma unroll
-                for (int q = 0; q < SB; ++q) x = fmaf(X[SB * i + r][SB * i + q], T[j][q][c], x);
-                X[SB * i + r][SB * j + c] = -x;
-            }
-            __syncthreads();
+            float* tp = T + (p * s + r) * lt + c;
+            tp[0] = t0; tp[1] = t1; tp[2] = t2; tp[3] = t3;
         }
+        __syncthreads();
+        for (int g = tid; g < groups; g += kPotrfThreads) {       // X_p(bottom-left) = -Xb_p T_p
+            const int cg = g % (s / 4), r = (g / (s / 4)) % s, p = g / ((s / 4) * s);
+            const int o = 2 * p * s, c = cg * 4;
+            float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;
+            const float* xb = &X[o + s + r][o + s];
+#pragma unroll 4
+            for (int k = 0; k <= r; ++k) {                         // Xb is lower triangular
+                const float bv = xb[k];
+                const float* tr = T + (p * s + k) * lt + c;
+                x0 = fmaf(bv, tr[0], x0); x1 = fmaf(bv, tr[1], x1);
+                x2 = fmaf(bv, tr[2], x2); x3 = fmaf(bv, tr[3], x3);
+            }
+            float* xo = &X[o + s + r][o + c];
+            xo[0] = -x0; xo[1] = -x1; xo[2] = -x2; xo[3] = -x3;
+        }
+        __syncthreads();
     }
-    for (int i = tid; i < PB * PB; i += kPotrfThreads) {
-        const int r = i >> 7, c = i & 127;
+    // ---- write the inverse and its transpose as bf16 triples, two columns per thread ----
+    for (int i = tid; i < PB * PB / 2; i += kPotrfThreads) {
+        const int r = i >> 6, c = (i & 63) * 2;
         if (r < nbk && c < nbk) {
             const size_t o = (size_t)(k0 + r) * F + k0 + c;
-            __nv_bfloat16 h, m, l;
-            split3((c <= r) ? X[r][c] : 0.f, h, m, l);
-            X3.a[0][o] = h; X3.a[1][o] = m; X3.a[2][o] = l;
-            split3((r <= c) ? X[c][r] : 0.f, h, m, l);
-            XT3.a[0][o] = h; XT3.a[1][o] = m; XT3.a[2][o] = l;
+            __nv_bfloat16 h0, m0, l0, h1, m1, l1;
+            split3((c <= r) ? X[r][c] : 0.f, h0, m0, l0);
+            split3((c + 1 <= r) ? X[r][c + 1] : 0.f, h1, m1, l1);
+            if (c + 1 < nbk) {
+                *reinterpret_cast<uint32_t*>(X3.a[0] + o) = pack_bf16(h0, h1);
+                *reinterpret_cast<uint32_t*>(X3.a[1] + o) = pack_bf16(m0, m1);
+                *reinterpret_cast<uint32_t*>(X3.a[2] + o) = pack_bf16(l0, l1);
+            } else {
+                X3.a[0][o] = h0; X3.a[1][o] = m0; X3.a[2][o] = l0;
+            }
+            split3((r <= c) ? X[c][r] : 0.f, h0, m0, l0);
+            split3((r <= c + 1) ? X[c + 1][r] : 0.f, h1, m1, l1);
+            if (c + 1 < nbk) {
+                *reinterpret_cast<uint32_t*>(XT3.a[0] + o) = pack_bf16(h0, h1);
+                *reinterpret_cast<uint32_t*>(XT3.a[1] + o) = pack_bf16(m0, m1);
+                *reinterpret_cast<uint32_t*>(XT3.a[2] + o) = pack_bf16(l0, l1);
+            } else {
+                XT3.a[0][o] = h0; XT3.a[1][o] = m0; XT3.a[2][o] = l0;
+            }
         }
     }
 }
@@ -302,8 +365,7 @@ int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d) {
     }
     static bool attr_set = false;
     if (!attr_set) {
-        const int smem = (2 * PB * LDS + PB + 7 * SB * (SB + 1)) * (int)sizeof(float);
-        if (cudaFuncSetAttribute(k_potrf128, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(k_potrf128, cudaFuncAttributeMaxDynamicSharedMemorySize, kPotrfSmemBytes) != cudaSuccess)
             return PKV_ERR_CUDA;
         attr_set = true;
     }
@@ -313,7 +375,7 @@ int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d) {
 int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int F, int d, float* dW,
                         bool well_conditioned, DevStatus* status) {
     const int nblk = (F + PB - 1) / PB;
-    const int smem = (2 * PB * LDS + PB + 7 * SB * (SB + 1)) * (int)sizeof(float);
+    const int smem = kPotrfSmemBytes;
     Trip L3{{t->L3[0], t->L3[1], t->L3[2]}}, X3{{t->X3[0], t->X3[1], t->X3[2]}}, XT3{{t->XT3[0], t->XT3[1], t->XT3[2]}};
     Trip P3{{t->P3[0], t->P3[1], t->P3[2]}}, TT3{{t->TT3[0], t->TT3[1], t->TT3[2]}};
     int rc;
