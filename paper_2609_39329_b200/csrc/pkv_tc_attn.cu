@@ -20,6 +20,7 @@
 
 #include "pkv_ptx.cuh"
 #include "pkv_tc.h"
+#include "pkv_tc_attn2_params.h"
 
 namespace pkv {
 
@@ -424,7 +425,8 @@ __global__ void __launch_bounds__(192, 1) k_attn_tc(const __grid_constant__ Attn
 // ---------------------------------------------------------------------------------------------
 void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, int* nsplitC) {
     const int g = d->Hq / d->Hkv;
-    const long long qtiles = ((long long)d->N_max * g + 127) / 128;
+    const int rows_per_cta = (d->hd == 128) ? 256 : 128;     // the hd = 128 kernel owns two query tiles
+    const long long qtiles = ((long long)d->N_max * g + rows_per_cta - 1) / rows_per_cta;
     const long long base = qtiles * d->Hkv;
     const long long tilesF = (d->L + 127) / 128 + (d->N_max + 127) / 128;
     long long want = (6LL * 148 + base - 1) / base;
@@ -455,6 +457,45 @@ static int launch_attn(const Lc& lc, const AttnTcParams& p, int qtiles) {
     return PKV_OK;
 }
 
+// hd = 128: the two-tile kernel of pkv_tc_attn2.cu (operands already prepared in t->q, t->kn, t->vn)
+int launch_attn2(const Lc& lc, const Attn2Params& p, int qpairs);
+static int attention_tc2(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status) {
+    const int N = a.N, hd = d->hd, Hkv = d->Hkv, g = d->Hq / d->Hkv;
+    const int rows = N * g;
+    Attn2Params p;
+    int rc;
+    if ((rc = tc_make_map_3d(&p.mQhi, t->q.hi, 2 * Hkv, rows, hd, hd, (uint64_t)rows * hd, 128))) return rc;
+    if ((rc = tc_make_map_3d(&p.mQlo, t->q.lo, 2 * Hkv, rows, hd, hd, (uint64_t)rows * hd, 128))) return rc;
+    if ((rc = tc_make_map_3d(&p.mKn, t->kn, 2 * Hkv, N, hd, hd, (uint64_t)N * hd, 128))) return rc;
+    if ((rc = tc_make_map_3d(&p.mVn, t->vn, 2 * Hkv, N, hd, hd, (uint64_t)N * hd, 128))) return rc;
+    if (d->L > 0) {
+        if ((rc = tc_make_map_3d(&p.mK, a.K, Hkv, d->L, hd, hd, (uint64_t)d->L * hd, 128))) return rc;
+        if ((rc = tc_make_map_3d(&p.mV, a.V, Hkv, d->L, hd, hd, (uint64_t)d->L * hd, 128))) return rc;
+    } else {
+        p.mK = p.mKn;
+        p.mV = p.mVn;
+    }
+    if (a.total_kept > 0) {
+        if ((rc = tc_make_map_2d(&p.mKc, a.Kc, a.total_kept, hd, hd, 128))) return rc;
+        if ((rc = tc_make_map_2d(&p.mVc, a.Vc, a.total_kept, hd, hd, 128))) return rc;
+    } else {
+        p.mKc = p.mKn;      // never read: no compact-cache tiles exist
+        p.mVc = p.mVn;
+    }
+    p.head_off = a.head_off; p.tok_cs = a.tok_cs; p.bias = a.bias;
+    p.N = N; p.g = g; p.Hkv = Hkv; p.L = d->L; p.rows = rows;
+    tc_attn_plan(d, N, a.max_b, &p.tps, &p.nsplitF, &p.nsplitC);
+    p.part_m = t->part_m; p.part_l = t->part_l; p.part_O = t->part_O;
+    p.status = status;
+    rc = launch_attn2(lc, p, (rows + 255) / 256);
+    if (rc != PKV_OK) return rc;
+    AttnArgs c = a;
+    c.nsplitF = p.nsplitF; c.nsplitC = p.nsplitC;
+    c.part_m = t->part_m; c.part_l = t->part_l; c.part_O = t->part_O;
+    attention_combine(lc, c);
+    return PKV_OK;
+}
+
 int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, const float* rope_tab,
                  DevStatus* status) {
     const int N = a.N, hd = d->hd, Hkv = d->Hkv, g = d->Hq / d->Hkv;
@@ -465,6 +506,7 @@ int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
                                                                         d->Hq, Hkv, hd, t->q.hi, t->q.lo, t->kn, t->vn);
         lc.count();
     }
+    if (hd == 128) return attention_tc2(lc, t, d, a, status);
     AttnTcParams p;
     int rc;
     if ((rc = tc_make_map_3d(&p.mQhi, t->q.hi, 2 * Hkv, rows, hd, hd, (uint64_t)rows * hd, 128))) return rc;

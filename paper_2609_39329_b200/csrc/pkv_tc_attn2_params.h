@@ -1,0 +1,26 @@
+// Kernel parameters of the two-tile attention kernel (shared by its launcher and its caller).
+#pragma once
+
+#include <cuda.h>
+
+#include "pkv_internal.h"
+
+namespace pkv {
+
+struct alignas(64) Attn2Params {
+    CUtensorMap mQhi, mQlo;   // {hd, N*g, 2*Hkv}
+    CUtensorMap mK, mV;       // {hd, L, Hkv}
+    CUtensorMap mKc, mVc;     // {hd, total kept rows}
+    CUtensorMap mKn, mVn;     // {hd, N, 2*Hkv}
+    const int32_t* head_off;
+    const int32_t* tok_cs;
+    const float* bias;
+    int N, g, Hkv, L, rows;
+    int tps, nsplitF, nsplitC;
+    float* part_m;
+    float* part_l;
+    float* part_O;
+    DevStatus* status;
+};
+
+}  // namespace pkv
