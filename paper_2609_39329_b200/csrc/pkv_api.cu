@@ -255,6 +255,7 @@ extern "C" void pkv_destroy(pkv_ctx* c) {
     if (c->host_stage) cudaFreeHost(c->host_stage);
     if (c->host_status) cudaFreeHost(c->host_status);
     if (c->map_cache) pkv::tc_map_cache_destroy((pkv::MapCache*)c->map_cache);
+    if (c->engine != PKV_ENGINE_SIMT) pkv::tc_destroy(&c->b.tc);
     for (int i = 0; i <= ST_COUNT; ++i)
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
     delete c;

@@ -205,6 +205,7 @@ size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d) {
 }
 
 int tc_init(TcBuffers* t, const pkv_dims* d) { return tc_solve_init(&t->solve, d); }
+void tc_destroy(TcBuffers* t) { tc_solve_destroy(&t->solve); }
 
 static void mark(const TcForwardArgs& a, const Lc& lc, int stage) {
     if (a.ev) cudaEventRecord(a.ev[stage], lc.st);

@@ -33,6 +33,7 @@ struct TcGemm {
     __nv_bfloat16* out[3];
     long long ldo;
     int nout;
+    int out_col_off;   // the bf16 parts are stored at column (absolute column - out_col_off)
     float alpha;
     bool accumulate, lower_only;
     int k_tri;      // 0: dense; 1: B lower triangular (skip k tiles past the row); 2: B upper triangular
@@ -56,7 +57,10 @@ struct TcSolveBuffers {
     __nv_bfloat16* TT3[3];
     __nv_bfloat16* S2[3];
     __nv_bfloat16* Z2[3];
+    cudaStream_t aux;      // high-priority helper stream of the factorisation's critical chain
+    cudaEvent_t ev[3];
 };
+void tc_solve_destroy(TcSolveBuffers* t);
 size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, const pkv_dims* d);
 int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d);
 // dW [d][F] = S_T (S + lambda I)^{-1}, lambda = status->lam; S [F][F] (lower part read) is destroyed.
@@ -110,6 +114,7 @@ int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
 int tc_supported(const pkv_dims* d, int cc_major, int cc_minor);
 size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d);
 int tc_init(TcBuffers* t, const pkv_dims* d);
+void tc_destroy(TcBuffers* t);
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a);
 int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status);
 void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, const float* R, int n, float* S_H,

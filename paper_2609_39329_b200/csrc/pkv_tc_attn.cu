@@ -423,13 +423,17 @@ __global__ void __launch_bounds__(192, 1) k_attn_tc(const __grid_constant__ Attn
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
+// CTAs of the teacher stream ~ kAttnWaves x 148 SMs: enough for balance, few enough that the split
+// partials (m, l, O per row and split) stay small next to the K/V traffic.
+constexpr long long kAttnWaves = 3;
+
 void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, int* nsplitC) {
     const int g = d->Hq / d->Hkv;
     const int rows_per_cta = (d->hd == 128) ? 256 : 128;     // the hd = 128 kernel owns two query tiles
     const long long qtiles = ((long long)d->N_max * g + rows_per_cta - 1) / rows_per_cta;
     const long long base = qtiles * d->Hkv;
     const long long tilesF = (d->L + 127) / 128 + (d->N_max + 127) / 128;
-    long long want = (6LL * 148 + base - 1) / base;
+    long long want = (kAttnWaves * 148 + base - 1) / base;
     if (want < 1) want = 1;
     if (want > 64) want = 64;
     long long t = (tilesF + want - 1) / want;

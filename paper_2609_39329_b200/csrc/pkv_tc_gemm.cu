@@ -39,7 +39,7 @@ struct alignas(64) GemmTcParams {
     long long ldadd;
     __nv_bfloat16* out[3];
     long long ldo;
-    int nout;
+    int nout, out_col_off;
     int accumulate, lower_only, k_tri, vec_ok;
     DevStatus* status;
 };
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                     if (lane < ncol) {
                         for (int rr = 0; rr < nrows; ++rr) {
                             const float x = stg[rr * 33 + lane];
-                            const size_t o = (size_t)(rowa0 + rr) * p.ldo + col + lane;
+                            const size_t o = (size_t)(rowa0 + rr) * p.ldo + (col - p.out_col_off) + lane;
                             __nv_bfloat16 h = __float2bfloat16_rn(x);
                             p.out[0][o] = h;
                             if (p.nout > 1) {
@@ -404,7 +404,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     p.c_rows = g.c_rows; p.c_cols = g.c_cols;
     p.C = g.C; p.ldc = g.ldc; p.alpha = g.alpha; p.addend = g.addend; p.ldadd = g.ldadd;
     for (int i = 0; i < 3; ++i) p.out[i] = g.out[i];
-    p.ldo = g.ldo; p.nout = g.nout;
+    p.ldo = g.ldo; p.nout = g.nout; p.out_col_off = g.out_col_off;
     p.accumulate = g.accumulate ? 1 : 0;
     p.lower_only = g.lower_only ? 1 : 0;
     p.k_tri = g.k_tri;

@@ -363,6 +363,13 @@ int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d) {
         if (cudaMemset(t->P3[i], 0, F * PB * 2) != cudaSuccess) return PKV_ERR_CUDA;
         if (cudaMemset(t->TT3[i], 0, tt_elems((int)F) * 2) != cudaSuccess) return PKV_ERR_CUDA;
     }
+    int least = 0, greatest = 0;
+    cudaDeviceGetStreamPriorityRange(&least, &greatest);
+    // the factorisation's critical chain (diagonal block, panel, next-column update) runs at the highest
+    // priority so that its small kernels are not queued behind the bulk trailing update's CTAs
+    if (cudaStreamCreateWithPriority(&t->aux, cudaStreamNonBlocking, greatest) != cudaSuccess) return PKV_ERR_CUDA;
+    for (int i = 0; i < 3; ++i)
+        if (cudaEventCreateWithFlags(&t->ev[i], cudaEventDisableTiming) != cudaSuccess) return PKV_ERR_CUDA;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(k_potrf128, cudaFuncAttributeMaxDynamicSharedMemorySize, kPotrfSmemBytes) != cudaSuccess)
@@ -372,6 +379,19 @@ int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d) {
     return PKV_OK;
 }
 
+void tc_solve_destroy(TcSolveBuffers* t) {
+    if (t->aux) {
+        cudaStreamSynchronize(t->aux);
+        cudaStreamDestroy(t->aux);
+        t->aux = nullptr;
+    }
+    for (int i = 0; i < 3; ++i)
+        if (t->ev[i]) {
+            cudaEventDestroy(t->ev[i]);
+            t->ev[i] = nullptr;
+        }
+}
+
 int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int F, int d, float* dW,
                         bool well_conditioned, DevStatus* status) {
     const int nblk = (F + PB - 1) / PB;
@@ -379,33 +399,68 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     Trip L3{{t->L3[0], t->L3[1], t->L3[2]}}, X3{{t->X3[0], t->X3[1], t->X3[2]}}, XT3{{t->XT3[0], t->XT3[1], t->XT3[2]}};
     Trip P3{{t->P3[0], t->P3[1], t->P3[2]}}, TT3{{t->TT3[0], t->TT3[1], t->TT3[2]}};
     int rc;
-    // ---- 1. factorisation ----
-    for (int b = 0; b < nblk; ++b) {
+    // ---- 1. factorisation with look-ahead ----
+    // Per block column b:  panel N_b (L21 = G21 L11^{-T});  T1_b = update of the next block column only
+    // (its epilogue also leaves the bf16 triple of the updated column in P3, the next panel's operand);
+    // T2_b = update of everything to the right, on the helper stream, beside the next diagonal block.
+    // sA: critical chain on the high-priority helper stream; sB: bulk updates on the caller's stream
+    cudaStream_t sA = t->aux, sB = lc.st;
+    Lc lcA{sA, lc.launches, lc.map_cache};
+    Lc lcB{sB, lc.launches, lc.map_cache};
+    cudaEventRecord(t->ev[2], sB);
+    cudaStreamWaitEvent(sA, t->ev[2], 0);
+    k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, F, 0, X3, XT3, status);
+    lc.count();
+    if (F > PB) launch_split3(lcA, G + (size_t)PB * F, F, F - PB, PB, Trip{{P3.a[0] + (size_t)PB * PB, P3.a[1] + (size_t)PB * PB, P3.a[2] + (size_t)PB * PB}}, PB, 3);
+    bool t2_pending = false;
+    rc = PKV_OK;
+    for (int b = 0; b < nblk && rc == PKV_OK; ++b) {
         const int k0 = b * PB, k1 = min(F, k0 + PB), rem = F - k1;
-        k_potrf128<<<1, kPotrfThreads, smem, lc.st>>>(G, F, k0, X3, XT3, status);
-        lc.count();
         if (rem <= 0) break;
-        // panel L21 = G21 L11^{-T}: split G21, multiply by the block inverse, keep L21 as a triple
-        launch_split3(lc, G + (size_t)k1 * F + k0, F, rem, PB, P3, PB, 3);
-        {
+        {   // N_b: panel, kept as a bf16 triple in L3
             TcGemm g{};
             six_pass(g, P3, PB, F, PB, X3, F, F, F);
+            g.a_row0 = k1;
             g.b_row0 = k0; g.b_col0 = k0;
             g.M = rem; g.N = PB; g.K = PB; g.batch = 1; g.alpha = 1.f;
             g.c_row0 = k1; g.c_col0 = k0; g.c_rows = F; g.c_cols = F;
             g.out[0] = L3.a[0]; g.out[1] = L3.a[1]; g.out[2] = L3.a[2]; g.ldo = F; g.nout = 3;
-            if ((rc = gemm_tc(lc, g, status))) return rc;
+            if ((rc = gemm_tc(lcA, g, status))) break;
         }
-        {   // trailing update G22 -= L21 L21^T on the lower triangle
+        cudaEventRecord(t->ev[0], sA);
+        cudaStreamWaitEvent(sB, t->ev[0], 0);
+        if (t2_pending) cudaStreamWaitEvent(sA, t->ev[1], 0);      // T2_{b-1} also updated this column
+        {   // T1_b: next block column of G22 -= L21 L21^T, and its bf16 triple for the next panel
             TcGemm g{};
             six_pass(g, L3, F, F, F, L3, F, F, F);
             g.a_row0 = k1; g.a_col0 = k0; g.b_row0 = k1; g.b_col0 = k0;
-            g.M = rem; g.N = rem; g.K = PB; g.batch = 1; g.alpha = -1.f;
-            g.C = const_cast<float*>(G); g.ldc = F; g.accumulate = true; g.lower_only = true;
+            g.M = rem; g.N = min(PB, rem); g.K = PB; g.batch = 1; g.alpha = -1.f;
+            g.C = const_cast<float*>(G); g.ldc = F; g.accumulate = true;
             g.c_row0 = k1; g.c_col0 = k1; g.c_rows = F; g.c_cols = F;
-            if ((rc = gemm_tc(lc, g, status))) return rc;
+            g.out[0] = P3.a[0]; g.out[1] = P3.a[1]; g.out[2] = P3.a[2]; g.ldo = PB; g.nout = 3; g.out_col_off = k1;
+            if ((rc = gemm_tc(lcA, g, status))) break;
         }
+        const int rem2 = rem - PB;
+        if (rem2 > 0) {   // T2_b on the helper stream
+            TcGemm g{};
+            six_pass(g, L3, F, F, F, L3, F, F, F);
+            g.a_row0 = k1 + PB; g.a_col0 = k0; g.b_row0 = k1 + PB; g.b_col0 = k0;
+            g.M = rem2; g.N = rem2; g.K = PB; g.batch = 1; g.alpha = -1.f;
+            g.C = const_cast<float*>(G); g.ldc = F; g.accumulate = true; g.lower_only = true;
+            g.c_row0 = k1 + PB; g.c_col0 = k1 + PB; g.c_rows = F; g.c_cols = F;
+            if ((rc = gemm_tc(lcB, g, status))) break;
+            cudaEventRecord(t->ev[1], sB);
+            t2_pending = true;
+        } else {
+            t2_pending = false;
+        }
+        k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, F, k1, X3, XT3, status);
+        lc.count();
     }
+    // join: the caller's stream continues after the chain's last kernel
+    cudaEventRecord(t->ev[0], sA);
+    cudaStreamWaitEvent(sB, t->ev[0], 0);
+    if (rc != PKV_OK) return rc;
     // ---- 2. X = L^{-1} by recursive doubling ----
     for (int s = PB; s < F; s *= 2) {
         int P = 0;
