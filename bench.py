@@ -71,7 +71,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
@@ -235,7 +235,6 @@ def main():
         step()
         ev[i][1].record()
     barrier()
-    clocks = sampler.stop()
     launches = ctx.launch_count() - l0 + args.steps      # + one merge kernel per step
     times = [a.elapsed_time(b) for a, b in ev]
     ms = float(sum(times) / len(times))
@@ -245,6 +244,7 @@ def main():
         ms = float(t.item())
 
     if args.quick:
+        sampler.stop()
         if rank == 0:
             print(json.dumps({"metric": "patch_build_ms_per_context", "value": ms / world, "unit": "ms",
                               "n_gpus": world, "steps": args.steps, "quick": True, "gpu_launches": int(launches)}))
@@ -288,10 +288,31 @@ def main():
         e2e_step()
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_n
+    clocks = sampler.stop()      # sampled over the timed steps, the stage pass and the end-to-end pass
     if world > 1:
         t = torch.tensor([e2e_ms], device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
+
+    # the same block through the dual (N x N) solver option: same dW, reported beside the headline
+    dual_ms = None
+    if cfg.N <= cfg.F and engine != B.ENGINE_SIMT:
+        ctx_d = B.PkvContext(B.dims_from_config(cfg, b_max=max(b_list)), engine=engine, solver=B.SOLVER_DUAL)
+        def step_d():
+            ctx_d.build_patch(w, kv["K"], kv["V"], off, idx_t, x_t, x_t, chunk_off, cfg.L, cfg.lam0, B.LAMBDA_PAPER,
+                              True, dW=dW)
+            ctx_d.merge(W_merged, dW)
+        for _ in range(3):
+            step_d()
+        evd = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(5)]
+        for i in range(5):
+            flush.fill_(i)
+            evd[i][0].record()
+            step_d()
+            evd[i][1].record()
+        torch.cuda.synchronize()
+        dual_ms = float(sum(a.elapsed_time(b) for a, b in evd) / 5)
+        ctx_d.close()
 
     if rank != 0:
         if world > 1:
@@ -335,7 +356,9 @@ def main():
             "frac_bf16_peak": total_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
             "roofline": roofline, "stages": stages, "cpu_baseline": cpu, "clocks": clocks,
             "e2e": {"value": e2e_ms / world, "unit": "ms", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)},
-            "gpu_launches": int(launches), "peaks": peaks}
+            "gpu_launches": int(launches), "peaks": peaks,
+            "dual_solver_option": {"ms_per_context": dual_ms, "note": "same dW through the N x N system (PKV_SOLVER_DUAL); "
+                                   "the headline value uses the primal F x F solve on the sufficient statistics"}}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

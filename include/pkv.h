@@ -55,6 +55,15 @@ enum {
     PKV_LAMBDA_TRACE_MEAN = 2  /* lambda = lambda0 * tr(S_H) / F              (ridge-scale ablation) */
 };
 
+/* Which linear system the ridge patch is solved through.  Both give the same dW (Woodbury identity):
+ *   primal: dW = S_T (S_H + lambda I)^{-1}, an F x F system on the sufficient statistics (Eq. 8-9);
+ *   dual:   dW = T^T (H' H'^T + lambda I)^{-1} H', an N x N system on the reference tokens of the call.
+ * The dual is cheaper when N < F but needs all reference tokens in one call (no running sums). */
+enum {
+    PKV_SOLVER_PRIMAL = 0,     /* default: the paper's form */
+    PKV_SOLVER_DUAL = 1        /* tensor-core engine only, requires N <= F */
+};
+
 enum {
     PKV_ENGINE_AUTO = 0,       /* tcgen05/TMA tensor-core kernels for bf16, SIMT fp32 kernels for fp32 */
     PKV_ENGINE_SIMT = 1        /* force the SIMT fp32 kernels (on-device cross-check of the tensor path) */
@@ -78,6 +87,7 @@ typedef struct pkv_opts {
     int32_t kv_split;        /* cache rows per attention split; 0 = choose from L and the SM count */
     void* workspace;         /* optional caller-provided device workspace (256-byte aligned) ... */
     size_t workspace_bytes;  /* ... of at least pkv_workspace_bytes(); NULL/0: the context allocates */
+    int32_t solver;          /* PKV_SOLVER_* (used by pkv_build_patch / pkv_build_stack) */
 } pkv_opts;
 
 /* Block weights, all device, element type dims.dtype except the fp32 norm gains.

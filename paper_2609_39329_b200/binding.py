@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(HERE, "libpkv.so")
 PKV_BF16, PKV_FP32 = 0, 1
 LAMBDA_PAPER, LAMBDA_ABSOLUTE, LAMBDA_TRACE_MEAN = 0, 1, 2
 ENGINE_AUTO, ENGINE_SIMT = 0, 1
+SOLVER_PRIMAL, SOLVER_DUAL = 0, 1
 
 ERRORS = {0: "PKV_OK", -1: "PKV_ERR_INVALID_ARG", -2: "PKV_ERR_UNSUPPORTED", -3: "PKV_ERR_BAD_INDEX",
           -4: "PKV_ERR_NOT_PD", -5: "PKV_ERR_DEGENERATE", -6: "PKV_ERR_NONFINITE", -7: "PKV_ERR_TIMEOUT",
@@ -39,7 +40,7 @@ class pkv_dims(C.Structure):
 
 class pkv_opts(C.Structure):
     _fields_ = [("engine", C.c_int32), ("kv_split", C.c_int32), ("workspace", C.c_void_p),
-                ("workspace_bytes", C.c_size_t)]
+                ("workspace_bytes", C.c_size_t), ("solver", C.c_int32)]
 
 
 class pkv_block_weights(C.Structure):
@@ -152,13 +153,14 @@ def dims_from_config(cfg, N_max: Optional[int] = None, b_max: Optional[int] = No
 class PkvContext:
     """Owns one pkv_ctx.  Tensors passed in must live on the context's CUDA device."""
 
-    def __init__(self, dims: pkv_dims, engine: int = ENGINE_AUTO, kv_split: int = 0, stream=None):
+    def __init__(self, dims: pkv_dims, engine: int = ENGINE_AUTO, kv_split: int = 0, stream=None,
+                 solver: int = SOLVER_PRIMAL):
         import torch
         self.torch = torch
         self.dims = dims
         self.L = lib()
         self.stream = stream
-        self.opts = pkv_opts(engine, kv_split, None, 0)
+        self.opts = pkv_opts(engine, kv_split, None, 0, solver)
         h = C.c_void_p()
         sp = C.c_void_p(stream.cuda_stream) if stream is not None else C.c_void_p(torch.cuda.current_stream().cuda_stream)
         rc = self.L.pkv_create(C.byref(h), C.byref(dims), C.byref(self.opts), sp)

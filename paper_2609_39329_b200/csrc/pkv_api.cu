@@ -70,6 +70,7 @@ struct pkv_ctx {
     pkv_opts opts;
     cudaStream_t st;
     int engine;
+    int dual;
     int elem_bytes;
     int kv_split, cap_splitF, cap_splitC;
     int sm_count;
@@ -114,7 +115,8 @@ static void split_plan(const pkv_dims* d, const pkv_opts* o, int sm_count, int* 
     if (*capC < 1) *capC = 1;
 }
 
-static size_t carve(Buffers* b, char* base, const pkv_dims* d, int engine, int elem_bytes, int capF, int capC) {
+static size_t carve(Buffers* b, char* base, const pkv_dims* d, int engine, int elem_bytes, int capF, int capC,
+                    int dual) {
     Carver c{base, 0};
     const size_t N = d->N_max, dm = d->d, F = d->F, Dq = (size_t)d->Hq * d->hd, Dkv = (size_t)d->Hkv * d->hd;
     const size_t g = d->Hq / d->Hkv, rows = N * g;
@@ -155,7 +157,7 @@ static size_t carve(Buffers* b, char* base, const pkv_dims* d, int engine, int e
     b->solve.Y = c.take<float>(dm * F);
     b->D = c.take<float>(N * dm);
     for (int i = 0; i < 4; ++i) b->xs[i] = c.take<float>(N * dm);
-    if (engine != PKV_ENGINE_SIMT) c.off = pkv::tc_carve(&b->tc, base, c.off, d);
+    if (engine != PKV_ENGINE_SIMT) c.off = pkv::tc_carve(&b->tc, base, c.off, d, dual);
     return (c.off + 255) & ~(size_t)255;
 }
 
@@ -178,7 +180,8 @@ extern "C" size_t pkv_workspace_bytes(const pkv_dims* dims, const pkv_opts* opts
     split_plan(dims, opts, 148, &ks, &cf, &cc);
     Buffers b;
     int engine = choose_engine(dims, opts);
-    return carve(&b, nullptr, dims, engine, dims->dtype == PKV_BF16 ? 2 : 4, cf, cc);
+    return carve(&b, nullptr, dims, engine, dims->dtype == PKV_BF16 ? 2 : 4, cf, cc,
+                 (opts && opts->solver == PKV_SOLVER_DUAL && engine != PKV_ENGINE_SIMT) ? 1 : 0);
 }
 
 extern "C" int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* opts, void* cuda_stream) {
@@ -210,7 +213,12 @@ extern "C" int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* o
     }
     // the split plan uses 148 SMs so that pkv_workspace_bytes (no device needed) agrees with it
     split_plan(dims, opts, 148, &c->kv_split, &c->cap_splitF, &c->cap_splitC);
-    size_t need = carve(&c->b, nullptr, dims, c->engine, c->elem_bytes, c->cap_splitF, c->cap_splitC);
+    c->dual = (opts && opts->solver == PKV_SOLVER_DUAL) ? 1 : 0;
+    if (c->dual && (c->engine == PKV_ENGINE_SIMT || dims->N_max > dims->F)) {
+        delete c;
+        return PKV_ERR_UNSUPPORTED;
+    }
+    size_t need = carve(&c->b, nullptr, dims, c->engine, c->elem_bytes, c->cap_splitF, c->cap_splitC, c->dual);
     c->ws_bytes = need;
     if (opts && opts->workspace) {
         if (opts->workspace_bytes < need || ((uintptr_t)opts->workspace & 255)) {
@@ -227,7 +235,7 @@ extern "C" int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* o
         }
         c->own_ws = true;
     }
-    carve(&c->b, c->ws, dims, c->engine, c->elem_bytes, c->cap_splitF, c->cap_splitC);
+    carve(&c->b, c->ws, dims, c->engine, c->elem_bytes, c->cap_splitF, c->cap_splitC, c->dual);
     size_t stage_ints = (size_t)dims->Hkv + 1 + dims->N_max;
     if (cudaMallocHost((void**)&c->host_stage, stage_ints * sizeof(int32_t)) != cudaSuccess ||
         cudaMallocHost((void**)&c->host_status, sizeof(DevStatus)) != cudaSuccess) {
@@ -525,13 +533,20 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         fa.S_H = b.S_H; fa.S_T = b.S_T; fa.status = b.status;
         fa.aF = b.a2; fa.aC = b.aC;
         fa.kv_split = c->kv_split;
+        fa.dual = c->dual;
         fa.part_m = b.part_m; fa.part_l = b.part_l; fa.part_O = b.part_O;
         fa.ev = c->timing ? c->ev : nullptr;
         rc = pkv::tc_forward(lc, &b.tc, &c->dims, fa);
         if (rc != PKV_OK) return rc;
     }
     // S8 (Eq. 7-8)
-    solve_stage(c, lc, b.S_H, b.S_T, lambda, mode, dW, true);
+    if (c->dual) {
+        rc = pkv::tc_dual_solve(lc, &b.tc, &c->dims, N, b.R, lambda, mode, dW, b.status);
+        if (rc != PKV_OK) return rc;
+        sumsq(lc, dW, (int64_t)d * F, &b.status->dw_fro2);
+    } else {
+        solve_stage(c, lc, b.S_H, b.S_T, lambda, mode, dW, true);
+    }
     mark(c, ST_NEXT);
     // S9: xF_next = zF + hF W^T;  D = R - hC dW^T;  xC_next = xF_next - D
     if (next) {

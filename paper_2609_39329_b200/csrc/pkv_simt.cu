@@ -560,13 +560,13 @@ __device__ __forceinline__ double warp_sum_d(double v) {
 
 // tr(S) and ||S||_F^2: one row per block iteration, float4 loads, fp32 partial sums per thread
 // (a few hundred terms each), double precision across threads.
-__global__ void __launch_bounds__(256) k_trace_fro2(const float* __restrict__ S, int F, DevStatus* status) {
+__global__ void __launch_bounds__(256) k_trace_fro2(const float* __restrict__ S, int F, int ld, DevStatus* status) {
     float fro[4] = {0.f, 0.f, 0.f, 0.f};
     double tr = 0.0;
     int bad = 0;
-    const bool vec = (F % 4 == 0) && (((uintptr_t)S & 15) == 0);
+    const bool vec = (F % 4 == 0) && (ld % 4 == 0) && (((uintptr_t)S & 15) == 0);
     for (int r = blockIdx.x; r < F; r += gridDim.x) {
-        const float* row = S + (size_t)r * F;
+        const float* row = S + (size_t)r * ld;
         if (vec) {
             for (int c = threadIdx.x * 4; c < F; c += 1024) {
                 float4 v = *reinterpret_cast<const float4*>(row + c);
@@ -586,8 +586,8 @@ __global__ void __launch_bounds__(256) k_trace_fro2(const float* __restrict__ S,
     if (bad) raise(status, PKV_ERR_NONFINITE);
 }
 
-void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status) {
-    k_trace_fro2<<<min(F, 1184), 256, 0, lc.st>>>(S, F, status);
+void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status, int ld) {
+    k_trace_fro2<<<min(F, 1184), 256, 0, lc.st>>>(S, F, ld > 0 ? ld : F, status);
     lc.count();
 }
 

@@ -175,7 +175,7 @@ struct Carver2 {
     }
 };
 
-size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d) {
+size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d, int dual) {
     Carver2 c{base, off};
     const size_t N = d->N_max, dm = d->d, F = d->F, Dq = (size_t)d->Hq * d->hd, Dkv = (size_t)d->Hkv * d->hd;
     t->ldT = (int)((N + 7) / 8 * 8);
@@ -201,11 +201,73 @@ size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d) {
     t->part_m = c.take<float>(nsp * d->Hkv * rows);
     t->part_l = c.take<float>(nsp * d->Hkv * rows);
     t->part_O = c.take<float>(nsp * d->Hkv * rows * d->hd);
-    return tc_solve_carve(&t->solve, base, c.off, d);
+    c.off = tc_solve_carve(&t->solve, base, c.off, d->F, d->d);
+    t->dual_enabled = dual;
+    t->dual_ld_prev = 0;
+    if (dual) {
+        const size_t ldn = (size_t)t->ldT;
+        t->Gd = c.take<float>(N * ldn);
+        t->RTf = c.take<float>(dm * ldn);
+        t->Yd = c.take<float>(dm * ldn);
+        t->Yp = c.pair(dm * ldn);
+        c.off = tc_solve_carve(&t->dual, base, c.off, (int)ldn, d->d);
+    }
+    return c.off;
 }
 
-int tc_init(TcBuffers* t, const pkv_dims* d) { return tc_solve_init(&t->solve, d); }
-void tc_destroy(TcBuffers* t) { tc_solve_destroy(&t->solve); }
+int tc_init(TcBuffers* t, const pkv_dims*) {
+    int rc = tc_solve_init(&t->solve);
+    if (rc == PKV_OK && t->dual_enabled) rc = tc_solve_init(&t->dual);
+    return rc;
+}
+void tc_destroy(TcBuffers* t) {
+    tc_solve_destroy(&t->solve);
+    if (t->dual_enabled) tc_solve_destroy(&t->dual);
+}
+
+// in [rows][cols] fp32 -> out [cols][ldo] fp32
+__global__ void k_transpose_ld(const float* __restrict__ in, int rows, int cols, int ldo, float* __restrict__ out) {
+    __shared__ float t[32][33];
+    int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        int r = r0 + j, c = c0 + threadIdx.x;
+        if (r < rows && c < cols) t[j][threadIdx.x] = in[(size_t)r * cols + c];
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        int c = c0 + j, r = r0 + threadIdx.x;
+        if (r < rows && c < cols) out[(size_t)c * ldo + r] = t[threadIdx.x][j];
+    }
+}
+
+int tc_dual_solve(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const float* R, float lam0, int mode,
+                  float* dW, DevStatus* status) {
+    const int F = D->F, d = D->d;
+    const int ldn = (N + 7) / 8 * 8;
+    int rc;
+    // G_d = X X^T from the student features (bf16 pair, row-major: the contraction runs over F)
+    if ((rc = gemm_pair_pair(lc, t->hC, F, t->hC, F, t->Gd, ldn, N, N, F, 1.f, nullptr, 0, false, status))) return rc;
+    {
+        dim3 grid((d + 31) / 32, (N + 31) / 32), block(32, 8);
+        k_transpose_ld<<<grid, block, 0, lc.st>>>(R, N, d, ldn, t->RTf);
+        lc.count();
+    }
+    // tr(X X^T) = tr(X^T X) and ||X X^T||_F = ||X^T X||_F: the ridge scale of Eq. 7 is the same number
+    trace_fro2(lc, t->Gd, N, status, ldn);
+    ridge_lambda(lc, F, lam0, mode, status);
+    const bool well = (mode == PKV_LAMBDA_PAPER) && (lam0 >= 0.05f);
+    const bool zero_fill = (ldn != t->dual_ld_prev);
+    t->dual_ld_prev = ldn;
+    if ((rc = tc_ridge_solve_impl(lc, &t->dual, t->Gd, t->RTf, N, ldn, d, t->Yd, well, zero_fill, status))) return rc;
+    // dW = Y X, contraction over the tokens: both operands token-contiguous
+    split(lc, t->Yd, (size_t)d * ldn, t->Yp);
+    TcGemm g = plain_gemm(d, F, N, dW, F, 1.f, nullptr, 0, false);
+    g.A[0] = TcMat{t->Yp.hi, ldn, d, N}; g.B[0] = TcMat{t->XT.hi, t->ldT, F, N};
+    g.A[1] = TcMat{t->Yp.hi, ldn, d, N}; g.B[1] = TcMat{t->XT.lo, t->ldT, F, N};
+    g.A[2] = TcMat{t->Yp.lo, ldn, d, N}; g.B[2] = TcMat{t->XT.hi, t->ldT, F, N};
+    g.npass = 3;
+    return gemm_tc(lc, g, status);
+}
 
 static void mark(const TcForwardArgs& a, const Lc& lc, int stage) {
     if (a.ev) cudaEventRecord(a.ev[stage], lc.st);
@@ -240,7 +302,7 @@ void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int 
     // Under the adaptive scale of Eq. 7 cond(G) ~ (tr(S_H)/sigma_max)/lambda0; lambda0 >= 0.05 keeps it
     // to a few tens.  Absolute and trace-mean coefficients give no such bound.
     const bool well = (mode == PKV_LAMBDA_PAPER) && (lam0 >= 0.05f);
-    tc_ridge_solve_impl(lc, &t->solve, S, S_T, F, d, dW, well, status);
+    tc_ridge_solve_impl(lc, &t->solve, S, S_T, F, F, d, dW, well, false, status);
 }
 
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a) {
@@ -289,8 +351,9 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     if ((rc = gemm_act_weight(lc, t->dh, F, w->Wdown, F, a.R, d, N, d, F, 1.f, a.dz, d, st))) return rc;
     sumsq(lc, a.R, (int64_t)N * d, &st->t_fro2);
     mark(a, lc, 6);
-    // S7 (Eq. 9)
-    tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st);
+    // S7 (Eq. 9); the dual solver only needs the token-contiguous copy of the student features
+    if (a.dual) transpose_split(lc, a.hC, N, F, t->ldT, t->XT);
+    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st);
     mark(a, lc, 7);
     return PKV_OK;
 }

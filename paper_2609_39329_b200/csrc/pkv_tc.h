@@ -57,15 +57,17 @@ struct TcSolveBuffers {
     __nv_bfloat16* TT3[3];
     __nv_bfloat16* S2[3];
     __nv_bfloat16* Z2[3];
+    int nmax;              // largest system the arrays are sized for
     cudaStream_t aux;      // high-priority helper stream of the factorisation's critical chain
     cudaEvent_t ev[3];
 };
 void tc_solve_destroy(TcSolveBuffers* t);
-size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, const pkv_dims* d);
-int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d);
-// dW [d][F] = S_T (S + lambda I)^{-1}, lambda = status->lam; S [F][F] (lower part read) is destroyed.
-int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int F, int d, float* dW,
-                        bool well_conditioned, DevStatus* status);
+size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, int nmax, int dmax);
+int tc_solve_init(TcSolveBuffers* t);
+// dW [d][n] = S_T (S + lambda I)^{-1}, lambda = status->lam; S [n][n] (lower part read) is destroyed.
+// ld: row stride of S, S_T, dW (multiple of 8).  zero_fill: ld differs from the previous call's.
+int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
+                        float* dW, bool well_conditioned, bool zero_fill, DevStatus* status);
 
 // bf16 hi/lo pairs of fp32 activations: v ~= hi + lo with hi = bf16(v), lo = bf16(v - hi).
 struct Pair {
@@ -92,6 +94,13 @@ struct TcBuffers {
     float* part_l;
     float* part_O;      // [splits][Hkv][N*g][hd]
     TcSolveBuffers solve;
+    // dual (N x N) solver: its own work arrays and the fp32 staging of G_d, T^T and Y
+    int dual_enabled, dual_ld_prev;
+    TcSolveBuffers dual;
+    float* Gd;          // [N][ldn]
+    float* RTf;         // [d][ldn]
+    float* Yd;          // [d][ldn]
+    Pair Yp;            // [d][ldn]
 };
 
 struct TcForwardArgs {
@@ -103,6 +112,7 @@ struct TcForwardArgs {
     const int32_t* head_off; const int32_t* tok_cs; float* rope_tab;
     float *zF, *zC, *dz, *hF, *hC, *R, *S_H, *S_T, *aF, *aC;
     float *part_m, *part_l, *part_O;
+    int dual;           // 1: only the token-contiguous copy of the student features is prepared in S7
     DevStatus* status;
     cudaEvent_t* ev;    // stage marks (index = stage) or nullptr
 };
@@ -112,7 +122,10 @@ void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, i
 int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, const float* rope_tab,
                  DevStatus* status);
 int tc_supported(const pkv_dims* d, int cc_major, int cc_minor);
-size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d);
+size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d, int dual);
+// S7'+S8 of the dual form: G_d = X X^T, lambda, Y = T^T (G_d + lambda I)^{-1}, dW = Y X.
+int tc_dual_solve(const Lc& lc, TcBuffers* t, const pkv_dims* d, int N, const float* R, float lam0, int mode,
+                  float* dW, DevStatus* status);
 int tc_init(TcBuffers* t, const pkv_dims* d);
 void tc_destroy(TcBuffers* t);
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a);

@@ -29,6 +29,8 @@ using namespace ptx;
 
 namespace a2 {
 constexpr int HD = 128;
+constexpr float kRescaleThreshold = 0.f;     // log2 units. 0 keeps the exact running maximum: the dominant key then has
+                                             // p = 1, exact in bf16; a stale reference (e.g. 8) triples the output error
 constexpr int kTile = 128 * HD * 2;            // 32 KB: one 128-row operand tile (two 64-column sub-tiles)
 constexpr int kQ = 0;                          // Q0hi Q0lo Q1hi Q1lo
 constexpr int kK = 4 * kTile;                  // one stage
@@ -284,7 +286,7 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
             const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             // reference maximum: moved only when the row maximum outgrew it by more than 2^8
             float alpha = 1.f;
-            const bool move = mx > m_ref + 8.f;          // also true for the first finite maximum (m_ref = -inf)
+            const bool move = mx > m_ref + kRescaleThreshold;         // also true for the first finite maximum (m_ref = -inf)
             if (move) {
                 alpha = ex2f(m_ref - mx);                // m_ref = -inf -> 0
                 m_ref = mx;
@@ -296,10 +298,13 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
             for (int c = 0; c < 128; c += 2) {
                 const float p0 = ex2f(__uint_as_float(s[c]) - m_use);
                 const float p1 = ex2f(__uint_as_float(s[c + 1]) - m_use);
-                l0 += p0;
-                l1 += p1;
                 __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-                s[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
+                const uint32_t pk = *reinterpret_cast<uint32_t*>(&b);
+                // the row sum uses the ROUNDED probabilities, the ones the P V product sees, so that the
+                // rounding of a dominant key cancels between numerator and denominator
+                l0 += __uint_as_float(pk << 16);
+                l1 += __uint_as_float(pk & 0xffff0000u);
+                s[c >> 1] = pk;
             }
             l = l * alpha + (l0 + l1);
             // P overwrites S: the previous P V product must have finished reading it; O is then stable too

@@ -48,7 +48,7 @@ __device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) 
     return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
 }
 
-__global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restrict__ G, int F, int k0, Trip X3,
+__global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restrict__ G, int n, int ld, int k0, Trip X3,
                                                             Trip XT3, DevStatus* status) {
     extern __shared__ float smf[];
     float(*A)[LDS] = reinterpret_cast<float(*)[LDS]>(smf);
@@ -57,17 +57,17 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
     float* T = rd + PB;                          // doubling temporary
     if (status->code != 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int nbk = min(PB, F - k0);
+    const int nbk = min(PB, n - k0);
     const float lam = status->lam;
     // ---- load the lower part (identity outside the block's extent), lambda on the diagonal ----
-    if (nbk == PB && (F & 3) == 0) {
+    if (nbk == PB && (ld & 3) == 0) {
         constexpr int kLd = 4096 / kPotrfThreads;
         float4 v[kLd];
 #pragma unroll
         for (int u = 0; u < kLd; ++u) {
             const int i = tid + u * kPotrfThreads;           // 4096 float4 of the block
             const int r = i >> 5, c4 = (i & 31) * 4;
-            v[u] = (c4 <= r) ? *reinterpret_cast<const float4*>(G + (size_t)(k0 + r) * F + k0 + c4)
+            v[u] = (c4 <= r) ? *reinterpret_cast<const float4*>(G + (size_t)(k0 + r) * ld + k0 + c4)
                              : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
             const int r = i >> 7, c = i & 127;
             float v = (r == c) ? 1.f : 0.f;
             if (r < nbk && c <= r) {
-                v = G[(size_t)(k0 + r) * F + k0 + c];
+                v = G[(size_t)(k0 + r) * ld + k0 + c];
                 if (r == c) v += lam;                     // G = S_H + lambda I is never materialised
             }
             A[r][c] = v;
@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
     for (int i = tid; i < PB * PB / 2; i += kPotrfThreads) {
         const int r = i >> 6, c = (i & 63) * 2;
         if (r < nbk && c < nbk) {
-            const size_t o = (size_t)(k0 + r) * F + k0 + c;
+            const size_t o = (size_t)(k0 + r) * ld + k0 + c;
             __nv_bfloat16 h0, m0, l0, h1, m1, l1;
             split3((c <= r) ? X[r][c] : 0.f, h0, m0, l0);
             split3((c + 1 <= r) ? X[r][c + 1] : 0.f, h1, m1, l1);
@@ -277,24 +277,24 @@ static void launch_split3(const Lc& lc, const float* src, long long lds, int row
     lc.count();
 }
 
-// XT3[2sz + c][s + 2sz + r] = X3[s + 2sz + r][2sz + c]   (r < s clipped to the matrix, c < s)
-__global__ void k_transpose_blocks(Trip X3, Trip XT3, int F, int s) {
+// XT3[2sz + c][s + 2sz + r] = X3[s + 2sz + r][2sz + c]   (r < s clipped to the n x n matrix, c < s); row stride ld
+__global__ void k_transpose_blocks(Trip X3, Trip XT3, int n, int ld, int s) {
     __shared__ __nv_bfloat16 t[3][32][33];
     const int z = blockIdx.z;
     const int r0 = s + 2 * s * z + blockIdx.y * 32, c0 = 2 * s * z + blockIdx.x * 32;
     for (int j = threadIdx.y; j < 32; j += 8) {
         const int r = r0 + j, c = c0 + threadIdx.x;
-        if (r < F) {
+        if (r < n) {
 #pragma unroll
-            for (int a = 0; a < 3; ++a) t[a][j][threadIdx.x] = X3.a[a][(size_t)r * F + c];
+            for (int a = 0; a < 3; ++a) t[a][j][threadIdx.x] = X3.a[a][(size_t)r * ld + c];
         }
     }
     __syncthreads();
     for (int j = threadIdx.y; j < 32; j += 8) {
         const int c = c0 + j, r = r0 + threadIdx.x;
-        if (r < F) {
+        if (r < n) {
 #pragma unroll
-            for (int a = 0; a < 3; ++a) XT3.a[a][(size_t)c * F + r] = t[a][threadIdx.x][j];
+            for (int a = 0; a < 3; ++a) XT3.a[a][(size_t)c * ld + r] = t[a][threadIdx.x][j];
         }
     }
 }
@@ -331,8 +331,9 @@ static size_t tt_elems(int F) {
     return best;
 }
 
-size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, const pkv_dims* d) {
-    const size_t F = d->F, dm = d->d;
+size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, int nmax, int dmax) {
+    const size_t F = (size_t)nmax, dm = (size_t)dmax;
+    t->nmax = nmax;
     auto take = [&](size_t bytes) {
         off = (off + 255) & ~(size_t)255;
         char* p = base ? base + off : nullptr;
@@ -353,9 +354,9 @@ size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, const pkv_dims*
     return off;
 }
 
-int tc_solve_init(TcSolveBuffers* t, const pkv_dims* d) {
+int tc_solve_init(TcSolveBuffers* t) {
     // regions of the triangular factors that no kernel writes must read as zero
-    const size_t F = d->F;
+    const size_t F = (size_t)t->nmax;
     for (int i = 0; i < 3; ++i) {
         if (cudaMemset(t->X3[i], 0, F * F * 2) != cudaSuccess) return PKV_ERR_CUDA;
         if (cudaMemset(t->XT3[i], 0, F * F * 2) != cudaSuccess) return PKV_ERR_CUDA;
@@ -392,13 +393,21 @@ void tc_solve_destroy(TcSolveBuffers* t) {
         }
 }
 
-int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int F, int d, float* dW,
-                        bool well_conditioned, DevStatus* status) {
+int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
+                        float* dW, bool well_conditioned, bool zero_fill, DevStatus* status) {
+    const int F = n;      // dimension of the system; ld is the row stride of G, S_T, dW and of every n x n work array
     const int nblk = (F + PB - 1) / PB;
     const int smem = kPotrfSmemBytes;
     Trip L3{{t->L3[0], t->L3[1], t->L3[2]}}, X3{{t->X3[0], t->X3[1], t->X3[2]}}, XT3{{t->XT3[0], t->XT3[1], t->XT3[2]}};
     Trip P3{{t->P3[0], t->P3[1], t->P3[2]}}, TT3{{t->TT3[0], t->TT3[1], t->TT3[2]}};
     int rc;
+    if (zero_fill) {
+        // the row stride changed since the last call: parts of X / X^T that no kernel writes must read as zero
+        for (int i = 0; i < 3; ++i) {
+            cudaMemsetAsync(t->X3[i], 0, (size_t)n * ld * 2, lc.st);
+            cudaMemsetAsync(t->XT3[i], 0, (size_t)n * ld * 2, lc.st);
+        }
+    }
     // ---- 1. factorisation with look-ahead ----
     // Per block column b:  panel N_b (L21 = G21 L11^{-T});  T1_b = update of the next block column only
     // (its epilogue also leaves the bf16 triple of the updated column in P3, the next panel's operand);
@@ -409,9 +418,9 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     Lc lcB{sB, lc.launches, lc.map_cache};
     cudaEventRecord(t->ev[2], sB);
     cudaStreamWaitEvent(sA, t->ev[2], 0);
-    k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, F, 0, X3, XT3, status);
+    k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, n, ld, 0, X3, XT3, status);
     lc.count();
-    if (F > PB) launch_split3(lcA, G + (size_t)PB * F, F, F - PB, PB, Trip{{P3.a[0] + (size_t)PB * PB, P3.a[1] + (size_t)PB * PB, P3.a[2] + (size_t)PB * PB}}, PB, 3);
+    if (F > PB) launch_split3(lcA, G + (size_t)PB * ld, ld, F - PB, PB, Trip{{P3.a[0] + (size_t)PB * PB, P3.a[1] + (size_t)PB * PB, P3.a[2] + (size_t)PB * PB}}, PB, 3);
     bool t2_pending = false;
     rc = PKV_OK;
     for (int b = 0; b < nblk && rc == PKV_OK; ++b) {
@@ -419,12 +428,12 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         if (rem <= 0) break;
         {   // N_b: panel, kept as a bf16 triple in L3
             TcGemm g{};
-            six_pass(g, P3, PB, F, PB, X3, F, F, F);
+            six_pass(g, P3, PB, F, PB, X3, ld, F, F);
             g.a_row0 = k1;
             g.b_row0 = k0; g.b_col0 = k0;
             g.M = rem; g.N = PB; g.K = PB; g.batch = 1; g.alpha = 1.f;
             g.c_row0 = k1; g.c_col0 = k0; g.c_rows = F; g.c_cols = F;
-            g.out[0] = L3.a[0]; g.out[1] = L3.a[1]; g.out[2] = L3.a[2]; g.ldo = F; g.nout = 3;
+            g.out[0] = L3.a[0]; g.out[1] = L3.a[1]; g.out[2] = L3.a[2]; g.ldo = ld; g.nout = 3;
             if ((rc = gemm_tc(lcA, g, status))) break;
         }
         cudaEventRecord(t->ev[0], sA);
@@ -432,10 +441,10 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         if (t2_pending) cudaStreamWaitEvent(sA, t->ev[1], 0);      // T2_{b-1} also updated this column
         {   // T1_b: next block column of G22 -= L21 L21^T, and its bf16 triple for the next panel
             TcGemm g{};
-            six_pass(g, L3, F, F, F, L3, F, F, F);
+            six_pass(g, L3, ld, F, F, L3, ld, F, F);
             g.a_row0 = k1; g.a_col0 = k0; g.b_row0 = k1; g.b_col0 = k0;
             g.M = rem; g.N = min(PB, rem); g.K = PB; g.batch = 1; g.alpha = -1.f;
-            g.C = const_cast<float*>(G); g.ldc = F; g.accumulate = true;
+            g.C = const_cast<float*>(G); g.ldc = ld; g.accumulate = true;
             g.c_row0 = k1; g.c_col0 = k1; g.c_rows = F; g.c_cols = F;
             g.out[0] = P3.a[0]; g.out[1] = P3.a[1]; g.out[2] = P3.a[2]; g.ldo = PB; g.nout = 3; g.out_col_off = k1;
             if ((rc = gemm_tc(lcA, g, status))) break;
@@ -443,10 +452,10 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         const int rem2 = rem - PB;
         if (rem2 > 0) {   // T2_b on the helper stream
             TcGemm g{};
-            six_pass(g, L3, F, F, F, L3, F, F, F);
+            six_pass(g, L3, ld, F, F, L3, ld, F, F);
             g.a_row0 = k1 + PB; g.a_col0 = k0; g.b_row0 = k1 + PB; g.b_col0 = k0;
             g.M = rem2; g.N = rem2; g.K = PB; g.batch = 1; g.alpha = -1.f;
-            g.C = const_cast<float*>(G); g.ldc = F; g.accumulate = true; g.lower_only = true;
+            g.C = const_cast<float*>(G); g.ldc = ld; g.accumulate = true; g.lower_only = true;
             g.c_row0 = k1 + PB; g.c_col0 = k1 + PB; g.c_rows = F; g.c_cols = F;
             if ((rc = gemm_tc(lcB, g, status))) break;
             cudaEventRecord(t->ev[1], sB);
@@ -454,7 +463,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         } else {
             t2_pending = false;
         }
-        k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, F, k1, X3, XT3, status);
+        k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, n, ld, k1, X3, XT3, status);
         lc.count();
     }
     // join: the caller's stream continues after the chain's last kernel
@@ -468,7 +477,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         if (P == 0) break;
         {   // TT_p = A_p^{-T} C_p^T   (A^{-1} the finished top-left inverse, C the block of L below it)
             TcGemm g{};
-            six_pass(g, XT3, F, F, F, L3, F, F, F);
+            six_pass(g, XT3, ld, F, F, L3, ld, F, F);
             g.a_zrow = 2 * s; g.a_zcol = 2 * s;
             g.b_row0 = s; g.b_zrow = 2 * s; g.b_zcol = 2 * s;
             g.M = s; g.N = s; g.K = s; g.batch = P; g.alpha = 1.f;
@@ -478,16 +487,16 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         }
         {   // X_p(bottom-left) = -B_p^{-1} TT_p^T
             TcGemm g{};
-            six_pass(g, X3, F, F, F, TT3, s, (long long)P * s, s);
+            six_pass(g, X3, ld, F, F, TT3, s, (long long)P * s, s);
             g.a_row0 = s; g.a_col0 = s; g.a_zrow = 2 * s; g.a_zcol = 2 * s;
             g.b_zrow = s;
             g.M = s; g.N = s; g.K = s; g.batch = P; g.alpha = -1.f;
             g.c_row0 = s; g.c_zrow = 2 * s; g.c_zcol = 2 * s; g.c_rows = F; g.c_cols = F;
-            g.out[0] = X3.a[0]; g.out[1] = X3.a[1]; g.out[2] = X3.a[2]; g.ldo = F; g.nout = 3;
+            g.out[0] = X3.a[0]; g.out[1] = X3.a[1]; g.out[2] = X3.a[2]; g.ldo = ld; g.nout = 3;
             if ((rc = gemm_tc(lc, g, status))) return rc;
         }
         dim3 grid(s / 32, s / 32, P), block(32, 8);
-        k_transpose_blocks<<<grid, block, 0, lc.st>>>(X3, XT3, F, s);
+        k_transpose_blocks<<<grid, block, 0, lc.st>>>(X3, XT3, n, ld, s);
         lc.count();
     }
     // ---- 3. dW = (S_T X^T) X ----
@@ -495,22 +504,22 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     // the ridge keeps G well conditioned, triples (2^-24, six passes) otherwise.
     const int nsp = well_conditioned ? 2 : 3;
     Trip S2{{t->S2[0], t->S2[1], t->S2[2]}}, Z2{{t->Z2[0], t->Z2[1], t->Z2[2]}};
-    launch_split3(lc, S_T, F, d, F, S2, F, nsp);
+    launch_split3(lc, S_T, ld, d, F, S2, ld, nsp);
     {
         TcGemm g{};
-        if (nsp == 2) three_pass(g, S2, F, d, F, X3, F, F, F);
-        else six_pass(g, S2, F, d, F, X3, F, F, F);
+        if (nsp == 2) three_pass(g, S2, ld, d, F, X3, ld, F, F);
+        else six_pass(g, S2, ld, d, F, X3, ld, F, F);
         g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 1;
         g.c_rows = d; g.c_cols = F;
-        g.out[0] = Z2.a[0]; g.out[1] = Z2.a[1]; g.out[2] = Z2.a[2]; g.ldo = F; g.nout = nsp;
+        g.out[0] = Z2.a[0]; g.out[1] = Z2.a[1]; g.out[2] = Z2.a[2]; g.ldo = ld; g.nout = nsp;
         if ((rc = gemm_tc(lc, g, status))) return rc;
     }
     {
         TcGemm g{};
-        if (nsp == 2) three_pass(g, Z2, F, d, F, XT3, F, F, F);
-        else six_pass(g, Z2, F, d, F, XT3, F, F, F);
+        if (nsp == 2) three_pass(g, Z2, ld, d, F, XT3, ld, F, F);
+        else six_pass(g, Z2, ld, d, F, XT3, ld, F, F);
         g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 2;
-        g.C = dW; g.ldc = F; g.c_rows = d; g.c_cols = F;
+        g.C = dW; g.ldc = ld; g.c_rows = d; g.c_cols = F;
         if ((rc = gemm_tc(lc, g, status))) return rc;
     }
     return PKV_OK;

@@ -30,7 +30,7 @@ def test_binding_structs_match_header_sizes_and_strerror():
     assert b"ascending" in L.pkv_strerror(-3)
     # workspace sizing needs no device; bad dims give 0
     d = B.make_dims(256, 4, 2, 64, 256, 1024, 64, 128, "fp32", 1e4, 1e-5)
-    o = B.pkv_opts(B.ENGINE_SIMT, 0, None, 0)
+    o = B.pkv_opts(B.ENGINE_SIMT, 0, None, 0, 0)
     assert L.pkv_workspace_bytes(ctypes.byref(d), ctypes.byref(o)) > 0
     d.hd = 96
     assert L.pkv_workspace_bytes(ctypes.byref(d), ctypes.byref(o)) == 0

@@ -26,13 +26,14 @@ def B():
     return binding
 
 
-def test_config2_whole_block_matches_oracle(B):
+@pytest.mark.parametrize("solver", [0, 1])
+def test_config2_whole_block_matches_oracle(B, solver):
     import torch
     cfg = gen.benchmark_config(2)
     lay = gen.gen_layer(cfg, 0)
     x = gen.gen_reference(cfg)
     ref = orc.build_patch(lay["weights"], lay["K"], lay["V"], lay["kept"], x, x, [0, cfg.N], cfg.L, cfg.lam0, cfg)
-    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO, solver=solver)
     w = B.to_device(lay["weights"], cfg.dtype)
     kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
     off, idx = gen.kept_to_csr(lay["kept"])
@@ -40,7 +41,7 @@ def test_config2_whole_block_matches_oracle(B):
     out = ctx.build_patch(w, kv["K"], kv["V"], off, torch.from_numpy(idx).cuda(), xt, xt, [0, cfg.N], cfg.L, cfg.lam0)
     dW = out["dW"].cpu().numpy()
     err = H.rel_fro(dW, ref["dW"])
-    print("config 2 dW rel fro err %.3e  lambda %.5g (oracle %.5g)" % (err, out["stats"]["lambda_eff"], ref["lam"]))
+    print("solver %d:" % solver, "config 2 dW rel fro err %.3e  lambda %.5g (oracle %.5g)" % (err, out["stats"]["lambda_eff"], ref["lam"]))
     assert err <= DW_TOL
     np.testing.assert_allclose(out["stats"]["lambda_eff"], ref["lam"], rtol=1e-3)
     assert H.rel_fro(out["xF_next"].cpu().numpy(), ref["xF_next"]) <= 1e-3

@@ -41,10 +41,10 @@ def engines(B, cfg):
     return [B.ENGINE_AUTO, B.ENGINE_SIMT]
 
 
-def gpu_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode=0, kv_split=0, want_next=True):
+def gpu_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode=0, kv_split=0, want_next=True, solver=0):
     import torch
     ctx = B.PkvContext(B.dims_from_config(cfg, N_max=xF.shape[0], b_max=max(len(k) for k in lay["kept"])),
-                       engine=engine, kv_split=kv_split)
+                       engine=engine, kv_split=kv_split, solver=solver)
     w = B.to_device(lay["weights"], cfg.dtype)
     kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
     off, idx = gen.kept_to_csr(lay["kept"])
@@ -63,9 +63,9 @@ def gpu_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode=0, kv_split=0, 
     return res
 
 
-def check_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode=0, kv_split=0):
+def check_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode=0, kv_split=0, solver=0):
     ref = H.run_oracle(cfg, lay, xF, xC, chunk_off, lam0, mode)
-    got = gpu_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode, kv_split)
+    got = gpu_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode, kv_split, solver=solver)
     e_dw = H.rel_fro(got["dW"], ref["dW"])
     assert e_dw <= DW_TOL, "dW rel fro %.3e" % e_dw
     np.testing.assert_allclose(got["stats"]["lambda_eff"], ref["lam"], rtol=2e-3)
@@ -262,6 +262,22 @@ def test_small_bf16_block_chunks_ragged_distinct_states(B, hd, Hq, Hkv):
     for engine in engines(B, cfg):
         check_build(B, cfg, lay, xF, xC, [0, 40, 41, 150], 0.1, engine, kv_split=256)
         check_build(B, cfg, lay, xF, xF, [0, 150], 1e-3, engine)
+
+
+@pytest.mark.parametrize("N,F", [(150, 192), (70, 448), (128, 128)])
+def test_dual_solver_gives_the_same_patch(B, N, F):
+    """dW through the N x N system (Woodbury) against the oracle's F x F solve, ragged N, several modes."""
+    cfg = small_cfg("bf16", hd=128, Hq=4, Hkv=2, d=256, F=F, L=1000, N=N)
+    lay = H.make_problem(cfg, per_head_budget=[100, 37])
+    xF = lay["x0"]
+    xC = (xF + 0.02 * np.random.default_rng(5).standard_normal(xF.shape)).astype(np.float32)
+    check_build(B, cfg, lay, xF, xC, [0, N // 3, N], 0.1, B.ENGINE_AUTO, solver=B.SOLVER_DUAL)
+    check_build(B, cfg, lay, xF, xF, [0, N], 1e-3, B.ENGINE_AUTO, solver=B.SOLVER_DUAL)
+    check_build(B, cfg, lay, xF, xF, [0, N], 0.05, B.ENGINE_AUTO, mode=B.LAMBDA_TRACE_MEAN, solver=B.SOLVER_DUAL)
+    # the dual form needs N <= F and the tensor-core engine
+    with pytest.raises(B.PkvError) as ei:
+        B.PkvContext(B.dims_from_config(gen.scaled_config(cfg, N=F + 8)), solver=B.SOLVER_DUAL)
+    assert ei.value.code == -2
 
 
 def test_identical_caches_give_zero_patch(B):
