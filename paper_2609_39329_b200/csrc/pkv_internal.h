@@ -61,6 +61,7 @@ struct AttnArgs {
     int total_kept, max_b;                // rows of the compact cache (all heads), largest head
     float* part_m; float* part_l; float* part_O;   // [nsplit][Hkv][N*g] and [..][hd]
     float* aF; float* aC; float* dA;      // [N][Hq*hd]
+    __nv_bfloat16* pair_hi; __nv_bfloat16* pair_lo;   // optional: bf16 hi/lo parts of [aF; dA] as [2N][Hq*hd]
 };
 void attention_simt(const Lc& lc, const AttnArgs& a);
 void attention_combine(const Lc& lc, const AttnArgs& a);

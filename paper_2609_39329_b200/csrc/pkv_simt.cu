@@ -471,9 +471,19 @@ __global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
     }
     size_t o = (size_t)tok * a.Hq * hd + (size_t)(kh * g + hg) * hd + lane * per;
     for (int c = 0; c < per; ++c) {
-        a.aF[o + c] = res[0][c];
+        const float f = res[0][c], dd = res[0][c] - res[1][c];
+        a.aF[o + c] = f;
         a.aC[o + c] = res[1][c];
-        a.dA[o + c] = res[0][c] - res[1][c];
+        a.dA[o + c] = dd;
+        if (a.pair_hi) {        // operands of the o-projection: rows [0,N) aF, rows [N,2N) dA
+            const size_t o2 = o + c + (size_t)a.N * a.Hq * hd;
+            __nv_bfloat16 h = __float2bfloat16_rn(f);
+            a.pair_hi[o + c] = h;
+            a.pair_lo[o + c] = __float2bfloat16_rn(f - __bfloat162float(h));
+            h = __float2bfloat16_rn(dd);
+            a.pair_hi[o2] = h;
+            a.pair_lo[o2] = __float2bfloat16_rn(dd - __bfloat162float(h));
+        }
     }
 }
 

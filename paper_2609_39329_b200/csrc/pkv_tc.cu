@@ -202,6 +202,9 @@ size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d, int dua
     t->part_l = c.take<float>(nsp * d->Hkv * rows);
     t->part_O = c.take<float>(nsp * d->Hkv * rows * d->hd);
     c.off = tc_solve_carve(&t->solve, base, c.off, d->F, d->d);
+    for (int i = 0; i < 3; ++i) t->S3[i] = t->solve.S2[i];     // the solver's S_T operand buffers
+    t->S3_ready = 0;
+    t->own_S_T = nullptr;
     t->dual_enabled = dual;
     t->dual_ld_prev = 0;
     if (dual) {
@@ -258,14 +261,15 @@ int tc_dual_solve(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const fl
     const bool well = (mode == PKV_LAMBDA_PAPER) && (lam0 >= 0.05f);
     const bool zero_fill = (ldn != t->dual_ld_prev);
     t->dual_ld_prev = ldn;
-    if ((rc = tc_ridge_solve_impl(lc, &t->dual, t->Gd, t->RTf, N, ldn, d, t->Yd, well, zero_fill, status))) return rc;
+    if ((rc = tc_ridge_solve_impl(lc, &t->dual, t->Gd, t->RTf, N, ldn, d, t->Yd, well, zero_fill, status, &t->Yp, nullptr)))
+        return rc;
     // dW = Y X, contraction over the tokens: both operands token-contiguous
-    split(lc, t->Yd, (size_t)d * ldn, t->Yp);
     TcGemm g = plain_gemm(d, F, N, dW, F, 1.f, nullptr, 0, false);
     g.A[0] = TcMat{t->Yp.hi, ldn, d, N}; g.B[0] = TcMat{t->XT.hi, t->ldT, F, N};
     g.A[1] = TcMat{t->Yp.hi, ldn, d, N}; g.B[1] = TcMat{t->XT.lo, t->ldT, F, N};
     g.A[2] = TcMat{t->Yp.lo, ldn, d, N}; g.B[2] = TcMat{t->XT.hi, t->ldT, F, N};
     g.npass = 3;
+    g.out[0] = t->dW.hi; g.out[1] = t->dW.lo; g.ldo = F; g.nout = 2;     // operand of the next-state product
     return gemm_tc(lc, g, status);
 }
 
@@ -279,6 +283,18 @@ void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, cons
     transpose_split(lc, X, n, F, t->ldT, t->XT);
     transpose_split(lc, R, n, dm, t->ldT, t->RT);
     gemm_pair_pair(lc, t->XT, t->ldT, t->XT, t->ldT, S_H, F, F, F, n, 1.f, nullptr, 0, accumulate, status);
+    t->S3_ready = 0;
+    if (!accumulate && S_T == t->own_S_T) {
+        // the build's own statistics: also leave the bf16 triple of S_T for the solver's first product
+        TcGemm g = plain_gemm(dm, F, n, S_T, F, 1.f, nullptr, 0, false);
+        g.A[0] = TcMat{t->RT.hi, t->ldT, dm, n}; g.B[0] = TcMat{t->XT.hi, t->ldT, F, n};
+        g.A[1] = TcMat{t->RT.hi, t->ldT, dm, n}; g.B[1] = TcMat{t->XT.lo, t->ldT, F, n};
+        g.A[2] = TcMat{t->RT.lo, t->ldT, dm, n}; g.B[2] = TcMat{t->XT.hi, t->ldT, F, n};
+        g.npass = 3;
+        g.out[0] = t->S3[0]; g.out[1] = t->S3[1]; g.out[2] = t->S3[2]; g.ldo = F; g.nout = 3;
+        if (gemm_tc(lc, g, status) == PKV_OK) t->S3_ready = 1;
+        return;
+    }
     gemm_pair_pair(lc, t->RT, t->ldT, t->XT, t->ldT, S_T, F, dm, F, n, 1.f, nullptr, 0, accumulate, status);
 }
 
@@ -302,7 +318,8 @@ void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int 
     // Under the adaptive scale of Eq. 7 cond(G) ~ (tr(S_H)/sigma_max)/lambda0; lambda0 >= 0.05 keeps it
     // to a few tens.  Absolute and trace-mean coefficients give no such bound.
     const bool well = (mode == PKV_LAMBDA_PAPER) && (lam0 >= 0.05f);
-    tc_ridge_solve_impl(lc, &t->solve, S, S_T, F, F, d, dW, well, false, status);
+    tc_ridge_solve_impl(lc, &t->solve, S, S_T, F, F, d, dW, well, false, status, &t->dW, t->S3_ready ? t->S3 : nullptr);
+    t->S3_ready = 0;
 }
 
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a) {
@@ -328,11 +345,11 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     at.N = N; at.Hq = D->Hq; at.Hkv = D->Hkv; at.hd = hd; at.L = D->L; at.elem_bytes = 2;
     at.total_kept = a.total_kept; at.max_b = a.max_b;
     at.aF = a.aF; at.aC = a.aC; at.dA = a.aF + (size_t)N * Dq;
+    at.pair_hi = t->a.hi; at.pair_lo = t->a.lo;
     // the S2 outputs are not rotated yet: the operand-preparation kernel applies RoPE
     if ((rc = attention_tc(lc, t, D, at, a.rope_tab, st))) return rc;
     mark(a, lc, 3);
     // S4: [aF; dA] Wo^T, then zF, dz, zC
-    split(lc, a.aF, (size_t)2 * N * Dq, t->a);
     if ((rc = gemm_act_weight(lc, t->a, Dq, w->Wo, Dq, t->o, d, 2 * N, d, Dq, 1.f, nullptr, 0, st))) return rc;
     oproj_epilogue(lc, a.xF, a.xC, t->o, N, d, a.zF, a.zC, a.dz);
     mark(a, lc, 4);
@@ -352,6 +369,7 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     sumsq(lc, a.R, (int64_t)N * d, &st->t_fro2);
     mark(a, lc, 6);
     // S7 (Eq. 9); the dual solver only needs the token-contiguous copy of the student features
+    t->own_S_T = a.S_T;
     if (a.dual) transpose_split(lc, a.hC, N, F, t->ldT, t->XT);
     else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st);
     mark(a, lc, 7);
@@ -364,7 +382,7 @@ void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const 
     // xF_next = zF + hF Wdown^T
     gemm_act_weight(lc, t->hF, F, Wdown, F, xF_next, d, N, d, F, 1.f, zF, d, status);
     // D = T - hC dW^T
-    split(lc, dW, (size_t)d * F, t->dW);
+    (void)dW;      // its bf16 pair was written by the solver's last product
     gemm_pair_pair(lc, t->hC, F, t->dW, F, Dm, d, N, d, F, -1.f, R, d, false, status);
 }
 

@@ -47,6 +47,7 @@ int tc_make_map_2d(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols
 int tc_make_map_3d(CUtensorMap* m, const void* ptr, uint64_t d2, uint64_t rows, uint64_t cols, uint64_t ld1,
                    uint64_t ld2, uint32_t box_rows);
 
+struct Pair;
 // Workspace of the tensor-core ridge solve: bf16 triples (hi, mid, lo) of the factor L, its inverse X,
 // the inverse's transpose, the current panel, the doubling temporaries; pairs of S_T and S_T X^T.
 struct TcSolveBuffers {
@@ -67,7 +68,8 @@ int tc_solve_init(TcSolveBuffers* t);
 // dW [d][n] = S_T (S + lambda I)^{-1}, lambda = status->lam; S [n][n] (lower part read) is destroyed.
 // ld: row stride of S, S_T, dW (multiple of 8).  zero_fill: ld differs from the previous call's.
 int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
-                        float* dW, bool well_conditioned, bool zero_fill, DevStatus* status);
+                        float* dW, bool well_conditioned, bool zero_fill, DevStatus* status, const Pair* dW_pair,
+                        __nv_bfloat16* const* S_T_triple);   // optional: dW's bf16 pair out; S_T already split
 
 // bf16 hi/lo pairs of fp32 activations: v ~= hi + lo with hi = bf16(v), lo = bf16(v - hi).
 struct Pair {
@@ -94,6 +96,9 @@ struct TcBuffers {
     float* part_l;
     float* part_O;      // [splits][Hkv][N*g][hd]
     TcSolveBuffers solve;
+    __nv_bfloat16* S3[3];   // bf16 triple of the build's own S_T (aliases solve.S2), written by the Gram epilogue
+    int S3_ready;
+    const float* own_S_T;
     // dual (N x N) solver: its own work arrays and the fp32 staging of G_d, T^T and Y
     int dual_enabled, dual_ld_prev;
     TcSolveBuffers dual;

@@ -394,7 +394,8 @@ void tc_solve_destroy(TcSolveBuffers* t) {
 }
 
 int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
-                        float* dW, bool well_conditioned, bool zero_fill, DevStatus* status) {
+                        float* dW, bool well_conditioned, bool zero_fill, DevStatus* status, const Pair* dW_pair,
+                        __nv_bfloat16* const* S_T_triple) {
     const int F = n;      // dimension of the system; ld is the row stride of G, S_T, dW and of every n x n work array
     const int nblk = (F + PB - 1) / PB;
     const int smem = kPotrfSmemBytes;
@@ -504,7 +505,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     // the ridge keeps G well conditioned, triples (2^-24, six passes) otherwise.
     const int nsp = well_conditioned ? 2 : 3;
     Trip S2{{t->S2[0], t->S2[1], t->S2[2]}}, Z2{{t->Z2[0], t->Z2[1], t->Z2[2]}};
-    launch_split3(lc, S_T, ld, d, F, S2, ld, nsp);
+    if (!S_T_triple) launch_split3(lc, S_T, ld, d, F, S2, ld, nsp);      // else: S2 already holds the triple
     {
         TcGemm g{};
         if (nsp == 2) three_pass(g, S2, ld, d, F, X3, ld, F, F);
@@ -520,6 +521,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         else six_pass(g, Z2, ld, d, F, XT3, ld, F, F);
         g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 2;
         g.C = dW; g.ldc = ld; g.c_rows = d; g.c_cols = F;
+        if (dW_pair) { g.out[0] = dW_pair->hi; g.out[1] = dW_pair->lo; g.ldo = ld; g.nout = 2; }
         if ((rc = gemm_tc(lc, g, status))) return rc;
     }
     return PKV_OK;
