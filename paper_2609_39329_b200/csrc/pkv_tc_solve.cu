@@ -41,6 +41,64 @@ struct Trip {
 // entirely in registers (lane i holds row i, columns are exchanged with shuffles), the rows below
 // it by forward substitution (one row per thread), then the trailing lower triangle is updated.
 constexpr int kPotrfThreads = 1024;
+
+// ---- warp-level TF32 tiles (mma.sync m16n8k8) in split form: each fp32 operand is the sum of three
+// TF32 parts (11 + 11 + 11 significant bits) and six products (hh, hm, mh, hl, lh, mm) are accumulated in
+// fp32, which reproduces the fp32 product to ~2^-24 while the shared-memory traffic is that of one
+// fragment load per operand element.
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ void split_tf32(float x, uint32_t& h, uint32_t& m, uint32_t& l) {
+    h = to_tf32(x);
+    const float r1 = x - __uint_as_float(h);
+    m = to_tf32(r1);
+    l = to_tf32(r1 - __uint_as_float(m));
+}
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+// One 16 x 8 output tile: c += sum over k in [kb, ke) (multiples of 8) of A(i, k) B(k, n).
+// fa(i, k) / fb(k, n) read the operands (shared memory).  Fragment ownership of lane (g = lane/4, t = lane%4):
+// A: (g, t) (g+8, t) (g, t+4) (g+8, t+4);  B: (t, g) (t+4, g);  C: (g, 2t) (g, 2t+1) (g+8, 2t) (g+8, 2t+1).
+// kSix: all six products (fp32-equivalent); otherwise the three leading ones (~2^-21), enough when the
+// ridge keeps the system well conditioned.
+template <bool kSix, typename FA, typename FB>
+__device__ __forceinline__ void warp_tile_tf32(float (&c)[4], int kb, int ke, int lane, FA fa, FB fb) {
+    const int g = lane >> 2, t = lane & 3;
+    // independent accumulators: consecutive mma.sync do not wait on one another
+    float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int k0 = kb; k0 < ke; k0 += 8) {
+        uint32_t ah[4], am[4], al[4], bh[2], bm[2], bl[2];
+        split_tf32(fa(g, k0 + t), ah[0], am[0], al[0]);
+        split_tf32(fa(g + 8, k0 + t), ah[1], am[1], al[1]);
+        split_tf32(fa(g, k0 + t + 4), ah[2], am[2], al[2]);
+        split_tf32(fa(g + 8, k0 + t + 4), ah[3], am[3], al[3]);
+        split_tf32(fb(k0 + t, g), bh[0], bm[0], bl[0]);
+        split_tf32(fb(k0 + t + 4, g), bh[1], bm[1], bl[1]);
+        if (kSix) {
+            mma_tf32(c2, al, bh);
+            mma_tf32(c1, ah, bl);
+            mma_tf32(c2, am, bm);
+        }
+        mma_tf32(c1, am, bh);
+        mma_tf32(c2, ah, bm);
+        mma_tf32(c, ah, bh);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) c[i] += c1[i] + c2[i];
+}
+template <typename FA, typename FB>
+__device__ __forceinline__ void warp_tile_tf32x6(float (&c)[4], int kb, int ke, int lane, bool six, FA fa, FB fb) {
+    if (six) warp_tile_tf32<true>(c, kb, ke, lane, fa, fb);
+    else warp_tile_tf32<false>(c, kb, ke, lane, fa, fb);
+}
 constexpr int kPotrfTElems = 64 * 65;       // largest doubling temporary (one 64 x 64 block, padded)
 constexpr int kPotrfSmemBytes = (2 * PB * LDS + PB + kPotrfTElems) * (int)sizeof(float);
 
@@ -49,7 +107,8 @@ __device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) 
 }
 
 __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restrict__ G, int n, int ld, int k0, Trip X3,
-                                                            Trip XT3, DevStatus* status) {
+                                                            Trip XT3, int six_i, DevStatus* status) {
+    const bool six = six_i != 0;
     extern __shared__ float smf[];
     float(*A)[LDS] = reinterpret_cast<float(*)[LDS]>(smf);
     float(*X)[LDS] = reinterpret_cast<float(*)[LDS]>(smf + PB * LDS);
@@ -145,18 +204,21 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
             for (int c = 0; c < SB; ++c) A[r][c0 + c] = a[c];
         }
         __syncthreads();
-        {   // trailing update of the lower triangle inside the block; the thread's row stays in registers
-            const int ty = tid >> 4, tx = tid & 15;
-            for (int r = base + ty; r < PB; r += kPotrfThreads / 16) {
-                float ar[SB];
-#pragma unroll
-                for (int c = 0; c < SB; ++c) ar[c] = A[r][c0 + c];
-                for (int k = base + tx; k <= r; k += 16) {
-                    float acc = 0.f;
-#pragma unroll
-                    for (int c = 0; c < SB; ++c) acc = fmaf(ar[c], A[k][c0 + c], acc);
-                    A[r][k] -= acc;
-                }
+        {   // trailing update of the lower triangle inside the block: 16 x 8 warp tiles, K = the 16 new columns
+            const int rem = PB - base;
+            const int tm = rem >> 4, tn = rem >> 3;
+            for (int tile = warp; tile < tm * tn; tile += kPotrfThreads / 32) {
+                const int i0 = base + (tile / tn) * 16, n0 = base + (tile % tn) * 8;
+                if (n0 > i0 + 15) continue;                     // entirely above the diagonal
+                float c[4] = {0.f, 0.f, 0.f, 0.f};
+                warp_tile_tf32x6(c, 0, SB, lane, six,
+                                 [&](int i, int k) { return A[i0 + i][c0 + k]; },
+                                 [&](int k, int n) { return A[n0 + n][c0 + k]; });
+                const int g = lane >> 2, t = lane & 3;
+                A[i0 + g][n0 + 2 * t] -= c[0];
+                A[i0 + g][n0 + 2 * t + 1] -= c[1];
+                A[i0 + g + 8][n0 + 2 * t] -= c[2];
+                A[i0 + g + 8][n0 + 2 * t + 1] -= c[3];
             }
         }
         __syncthreads();
@@ -190,40 +252,35 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
     }
     __syncthreads();
     // recursive doubling inside the block: [Xa 0; C Xb] -> bottom-left = -Xb (C Xa); every level is two
-    // dense products over all pairs, four output columns per thread
+    // dense products over all pairs, done as 16 x 8 warp tiles
     for (int s = SB; s < PB; s *= 2) {
         const int lt = s + 1;
-        const int groups = (PB / (2 * s)) * s * (s / 4);
-        for (int g = tid; g < groups; g += kPotrfThreads) {       // T_p = C_p Xa_p
-            const int cg = g % (s / 4), r = (g / (s / 4)) % s, p = g / ((s / 4) * s);
-            const int o = 2 * p * s, c = cg * 4;
-            float t0 = 0.f, t1 = 0.f, t2 = 0.f, t3 = 0.f;
-            const float* arow = &A[o + s + r][o];
-#pragma unroll 4
-            for (int k = c; k < s; ++k) {                          // Xa is lower triangular: rows >= column
-                const float av = arow[k];
-                const float* xr = &X[o + k][o + c];
-                t0 = fmaf(av, xr[0], t0); t1 = fmaf(av, xr[1], t1);
-                t2 = fmaf(av, xr[2], t2); t3 = fmaf(av, xr[3], t3);
-            }
-            float* tp = T + (p * s + r) * lt + c;
-            tp[0] = t0; tp[1] = t1; tp[2] = t2; tp[3] = t3;
+        const int tn = s >> 3, tpp = (s >> 4) * tn, ntile = (PB / (2 * s)) * tpp;
+        for (int tile = warp; tile < ntile; tile += kPotrfThreads / 32) {      // T_p = C_p Xa_p
+            const int p = tile / tpp, i0 = ((tile % tpp) / tn) * 16, n0 = ((tile % tpp) % tn) * 8;
+            const int o = 2 * p * s;
+            float c[4] = {0.f, 0.f, 0.f, 0.f};
+            warp_tile_tf32x6(c, n0, s, lane, six,                  // Xa is lower triangular: rows k >= column n
+                             [&](int i, int k) { return A[o + s + i0 + i][o + k]; },
+                             [&](int k, int n) { return X[o + k][o + n0 + n]; });
+            const int g = lane >> 2, t = lane & 3;
+            float* tp = T + (p * s + i0 + g) * lt + n0 + 2 * t;
+            tp[0] = c[0]; tp[1] = c[1];
+            tp[8 * lt] = c[2]; tp[8 * lt + 1] = c[3];
         }
         __syncthreads();
-        for (int g = tid; g < groups; g += kPotrfThreads) {       // X_p(bottom-left) = -Xb_p T_p
-            const int cg = g % (s / 4), r = (g / (s / 4)) % s, p = g / ((s / 4) * s);
-            const int o = 2 * p * s, c = cg * 4;
-            float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;
-            const float* xb = &X[o + s + r][o + s];
-#pragma unroll 4
-            for (int k = 0; k <= r; ++k) {                         // Xb is lower triangular
-                const float bv = xb[k];
-                const float* tr = T + (p * s + k) * lt + c;
-                x0 = fmaf(bv, tr[0], x0); x1 = fmaf(bv, tr[1], x1);
-                x2 = fmaf(bv, tr[2], x2); x3 = fmaf(bv, tr[3], x3);
-            }
-            float* xo = &X[o + s + r][o + c];
-            xo[0] = -x0; xo[1] = -x1; xo[2] = -x2; xo[3] = -x3;
+        for (int tile = warp; tile < ntile; tile += kPotrfThreads / 32) {      // X_p(bottom-left) = -Xb_p T_p
+            const int p = tile / tpp, i0 = ((tile % tpp) / tn) * 16, n0 = ((tile % tpp) % tn) * 8;
+            const int o = 2 * p * s;
+            float c[4] = {0.f, 0.f, 0.f, 0.f};
+            warp_tile_tf32x6(c, 0, i0 + 16, lane, six,             // Xb is lower triangular: columns k <= row
+                             [&](int i, int k) { return X[o + s + i0 + i][o + s + k]; },
+                             [&](int k, int n) { return T[(p * s + k) * lt + n0 + n]; });
+            const int g = lane >> 2, t = lane & 3;
+            X[o + s + i0 + g][o + n0 + 2 * t] = -c[0];
+            X[o + s + i0 + g][o + n0 + 2 * t + 1] = -c[1];
+            X[o + s + i0 + g + 8][o + n0 + 2 * t] = -c[2];
+            X[o + s + i0 + g + 8][o + n0 + 2 * t + 1] = -c[3];
         }
         __syncthreads();
     }
@@ -419,7 +476,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     Lc lcB{sB, lc.launches, lc.map_cache};
     cudaEventRecord(t->ev[2], sB);
     cudaStreamWaitEvent(sA, t->ev[2], 0);
-    k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, n, ld, 0, X3, XT3, status);
+    k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, n, ld, 0, X3, XT3, well_conditioned ? 0 : 1, status);
     lc.count();
     if (F > PB) launch_split3(lcA, G + (size_t)PB * ld, ld, F - PB, PB, Trip{{P3.a[0] + (size_t)PB * PB, P3.a[1] + (size_t)PB * PB, P3.a[2] + (size_t)PB * PB}}, PB, 3);
     bool t2_pending = false;
@@ -464,7 +521,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         } else {
             t2_pending = false;
         }
-        k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, n, ld, k1, X3, XT3, status);
+        k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, n, ld, k1, X3, XT3, well_conditioned ? 0 : 1, status);
         lc.count();
     }
     // join: the caller's stream continues after the chain's last kernel
