@@ -156,37 +156,51 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
     __syncthreads();
     float minpiv = INFINITY;
     int bad_col = -1;
-    for (int c0 = 0; c0 < PB; c0 += SB) {
-        if (warp == 0) {
-            const int li = lane & 15;            // lanes 16..31 mirror lanes 0..15 so every shuffle source is live
-            float a[SB];
+    // 16 x 16 diagonal piece at c0, factored by warp 0 entirely in registers
+    auto diag16 = [&](int c0) {
+        const int li = lane & 15;            // lanes 16..31 mirror lanes 0..15 so every shuffle source is live
+        float a[SB];
 #pragma unroll
-            for (int k = 0; k < SB; ++k) a[k] = A[c0 + li][c0 + k];
+        for (int k = 0; k < SB; ++k) a[k] = A[c0 + li][c0 + k];
 #pragma unroll
-            for (int j = 0; j < SB; ++j) {
-                float piv = __shfl_sync(0xffffffffu, a[j], j);
-                const bool okp = (piv > 0.f) && (piv < INFINITY);
-                if (!okp && bad_col < 0 && c0 + j < nbk) bad_col = c0 + j;
-                piv = okp ? piv : 1.f;
-                if (c0 + j < nbk) minpiv = fminf(minpiv, piv);
-                float rdj = rsqrtf(piv);
-                rdj = rdj * fmaf(-0.5f * piv * rdj, rdj, 1.5f);    // one Newton step: full fp32 accuracy
-                const float lij = a[j] * rdj;                       // row li of column j (the pivot row gets sqrt(piv))
-                a[j] = lij;
-                if (lane == j) rd[c0 + j] = rdj;
+        for (int j = 0; j < SB; ++j) {
+            float piv = __shfl_sync(0xffffffffu, a[j], j);
+            const bool okp = (piv > 0.f) && (piv < INFINITY);
+            if (!okp && bad_col < 0 && c0 + j < nbk) bad_col = c0 + j;
+            piv = okp ? piv : 1.f;
+            if (c0 + j < nbk) minpiv = fminf(minpiv, piv);
+            float rdj = rsqrtf(piv);
+            rdj = rdj * fmaf(-0.5f * piv * rdj, rdj, 1.5f);    // one Newton step: full fp32 accuracy
+            const float lij = a[j] * rdj;                       // row li of column j (the pivot row gets sqrt(piv))
+            a[j] = lij;
+            if (lane == j) rd[c0 + j] = rdj;
 #pragma unroll
-                for (int k = j + 1; k < SB; ++k) {
-                    const float lkj = __shfl_sync(0xffffffffu, lij, k);
-                    a[k] = fmaf(-lij, lkj, a[k]);                  // rows above the diagonal hold unused values
-                }
-            }
-            if (lane < SB) {
-#pragma unroll
-                for (int k = 0; k < SB; ++k)
-                    if (k <= lane) A[c0 + lane][c0 + k] = a[k];
+            for (int k = j + 1; k < SB; ++k) {
+                const float lkj = __shfl_sync(0xffffffffu, lij, k);
+                a[k] = fmaf(-lij, lkj, a[k]);                  // rows above the diagonal hold unused values
             }
         }
-        __syncthreads();
+        if (lane < SB) {
+#pragma unroll
+            for (int k = 0; k < SB; ++k)
+                if (k <= lane) A[c0 + lane][c0 + k] = a[k];
+        }
+    };
+    // one 16 x 8 tile of the trailing update for the 16 columns at c0
+    auto trail_tile = [&](int c0, int i0, int n0) {
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        warp_tile_tf32x6(c, 0, SB, lane, six,
+                         [&](int i, int k) { return A[i0 + i][c0 + k]; },
+                         [&](int k, int n) { return A[n0 + n][c0 + k]; });
+        const int g = lane >> 2, t = lane & 3;
+        A[i0 + g][n0 + 2 * t] -= c[0];
+        A[i0 + g][n0 + 2 * t + 1] -= c[1];
+        A[i0 + g + 8][n0 + 2 * t] -= c[2];
+        A[i0 + g + 8][n0 + 2 * t + 1] -= c[3];
+    };
+    if (warp == 0) diag16(0);
+    __syncthreads();
+    for (int c0 = 0; c0 < PB; c0 += SB) {
         const int base = c0 + SB;
         if (tid < PB - base) {     // rows below: x L_ss^T = a by forward substitution, one row per thread
             const int r = base + tid;
@@ -204,21 +218,23 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
             for (int c = 0; c < SB; ++c) A[r][c0 + c] = a[c];
         }
         __syncthreads();
-        {   // trailing update of the lower triangle inside the block: 16 x 8 warp tiles, K = the 16 new columns
-            const int rem = PB - base;
-            const int tm = rem >> 4, tn = rem >> 3;
-            for (int tile = warp; tile < tm * tn; tile += kPotrfThreads / 32) {
-                const int i0 = base + (tile / tn) * 16, n0 = base + (tile % tn) * 8;
-                if (n0 > i0 + 15) continue;                     // entirely above the diagonal
-                float c[4] = {0.f, 0.f, 0.f, 0.f};
-                warp_tile_tf32x6(c, 0, SB, lane, six,
-                                 [&](int i, int k) { return A[i0 + i][c0 + k]; },
-                                 [&](int k, int n) { return A[n0 + n][c0 + k]; });
-                const int g = lane >> 2, t = lane & 3;
-                A[i0 + g][n0 + 2 * t] -= c[0];
-                A[i0 + g][n0 + 2 * t + 1] -= c[1];
-                A[i0 + g + 8][n0 + 2 * t] -= c[2];
-                A[i0 + g + 8][n0 + 2 * t + 1] -= c[3];
+        if (base < PB) {
+            // trailing update of the lower triangle inside the block (16 x 8 warp tiles, K = the 16 new
+            // columns).  Warp 0 takes the next diagonal piece first and factors it right away, beside the
+            // other warps' tiles: the serial pivot chain is off the critical path.
+            if (warp == 0) {
+                trail_tile(c0, base, base);
+                trail_tile(c0, base, base + 8);
+                __syncwarp();
+                diag16(base);
+            } else {
+                const int rem = PB - base;
+                const int tm = (rem >> 4) - 1, tn = rem >> 3;          // row tiles below the first one
+                for (int tile = warp - 1; tile < tm * tn; tile += kPotrfThreads / 32 - 1) {
+                    const int i0 = base + 16 + (tile / tn) * 16, n0 = base + (tile % tn) * 8;
+                    if (n0 > i0 + 15) continue;                     // entirely above the diagonal
+                    trail_tile(c0, i0, n0);
+                }
             }
         }
         __syncthreads();
