@@ -50,7 +50,9 @@ constexpr int kGemmStagingBytes = 4 * 32 * 33 * 4;     // aliases the first pipe
 
 // One k-tile stage holds every distinct operand tile once: nA x [128][64] and nB x [BN][64] bf16,
 // and all passes are issued from it (the shared operand of a split product is not re-read).
-template <int BN>
+// PRE: the epilogue warps fetch the fp32 C tile they will add to (read-modify-write products of the
+// factorisation) while the main loop runs, instead of after it.
+template <int BN, bool PRE>
 __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcParams p) {
     const int m0 = blockIdx.y * 128, n0 = blockIdx.x * BN, z = blockIdx.z;
     if (p.lower_only && n0 > m0 + 127) return;
@@ -136,6 +138,20 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     } else {
         // epilogue: TMEM -> registers -> per-warp smem tile -> row-contiguous global accesses
         const int q = warp & 3;
+        const int rl0 = m0 + q * 32;                 // first row of this warp inside the batch element
+        const int rowa0 = crow0 + q * 32;            // ... and its absolute output row
+        const int nrows = max(0, min(32, min(p.M - rl0, p.c_rows - rowa0)));
+        const bool vec_ok = p.vec_ok != 0;
+        // PRE: whole-tile prefetch of C, legal when the tile is full width and vector-aligned
+        constexpr int kPre = PRE ? BN / 4 : 1;
+        float4 cpre[kPre];
+        const bool pre_ok = PRE && p.C && p.accumulate && vec_ok && lane < nrows &&
+                            min(p.N - n0, p.c_cols - ccol0) >= BN;
+        if (PRE && pre_ok) {
+            const float* crow = p.C + (size_t)(rowa0 + lane) * p.ldc + ccol0;
+#pragma unroll
+            for (int j = 0; j < kPre; ++j) cpre[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
+        }
         bool ok = true;
         if (ktiles > 0) {
             ok = mbar_wait(bars + 8 * (2 * STAGES), 0, abort_flag, p.status, 3);
@@ -143,11 +159,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         }
         if (ok) {
             float* stg = staging + q * (32 * 33);
-            const int rl0 = m0 + q * 32;                 // first row of this warp inside the batch element
-            const int rowa0 = crow0 + q * 32;            // ... and its absolute output row
-            const int nrows = max(0, min(32, min(p.M - rl0, p.c_rows - rowa0)));
-            const bool vec_ok = p.vec_ok != 0;
-#pragma unroll 1
+#pragma unroll
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 if (ktiles > 0) {
@@ -180,8 +192,13 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                         }
                         if (p.accumulate) {
                             float4 c4[8];
+                            if (PRE && pre_ok) {
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) c4[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
+                                for (int j = 0; j < 8; ++j) c4[j] = cpre[PRE ? (c0 >> 2) + j : 0];
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) c4[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
+                            }
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
                                 v[4 * j] += c4[j].x; v[4 * j + 1] += c4[j].y; v[4 * j + 2] += c4[j].z; v[4 * j + 3] += c4[j].w;
@@ -337,12 +354,12 @@ static int cached_map(MapCache* cache, CUtensorMap* out, const void* ptr, uint64
     return PKV_OK;
 }
 
-template <int BN>
+template <int BN, bool PRE>
 static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     static bool attr_set = false;
     constexpr int kMaxSmem = 227 * 1024;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(k_gemm_tc<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+        if (cudaFuncSetAttribute(k_gemm_tc<BN, PRE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return PKV_ERR_CUDA;
         attr_set = true;
     }
@@ -352,8 +369,10 @@ static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     // Two CTAs per SM let one tile's epilogue overlap the other's main loop: taken when the contraction
     // is short (epilogue-bound) or when two stages still fit in half an SM's shared memory.
     const int half = 112 * 1024 - fixed;
+    const long long ctas = (long long)((p.N + BN - 1) / BN) * ((p.M + 127) / 128) * batch;
     int stages;
-    if (ktiles <= 8 || 2 * stage_bytes <= half) stages = half / stage_bytes;
+    if (ctas <= 148) stages = (kMaxSmem - fixed) / stage_bytes;      // one wave: occupancy is moot, take the deepest pipeline
+    else if (ktiles <= 8 || 2 * stage_bytes <= half) stages = half / stage_bytes;
     else stages = (kMaxSmem - fixed) / stage_bytes;
     if (stages < 1) stages = 1;
     if (stages > kGemmMaxStages) stages = kGemmMaxStages;
@@ -361,7 +380,7 @@ static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     p.stages = stages;
     const int smem = stages * stage_bytes + fixed;
     dim3 grid((p.N + BN - 1) / BN, (p.M + 127) / 128, batch);
-    k_gemm_tc<BN><<<grid, 192, smem, lc.st>>>(p);
+    k_gemm_tc<BN, PRE><<<grid, 192, smem, lc.st>>>(p);
     lc.count();
     return PKV_OK;
 }
@@ -411,8 +430,9 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     p.vec_ok = (g.C && ((uintptr_t)g.C & 15) == 0 && g.ldc % 4 == 0 && g.c_col0 % 4 == 0 && g.c_zcol % 4 == 0 &&
                 (!g.addend || (((uintptr_t)g.addend & 15) == 0 && g.ldadd % 4 == 0))) ? 1 : 0;
     p.status = status;
-    if (BN == 64) return launch_gemm<64>(lc, p, g.batch);
-    return launch_gemm<128>(lc, p, g.batch);
+    const bool pre = g.C && g.accumulate && p.vec_ok;
+    if (BN == 64) return launch_gemm<64, false>(lc, p, g.batch);
+    return pre ? launch_gemm<128, true>(lc, p, g.batch) : launch_gemm<128, false>(lc, p, g.batch);
 }
 
 }  // namespace pkv
