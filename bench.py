@@ -164,6 +164,120 @@ def workload_config(cfg, lay):
             "l2": "inputs (weights + caches, >300 MB) exceed L2 and a 512 MB buffer is written between steps"}
 
 
+def run_stack(args, cfg, B, torch, dist, world, rank, local, peaks):
+    """Configs 3-5: patches for all blocks of the stack built in sequence (pkv_build_stack); a step is one
+    context = n_layers blocks.  `--distinct-layers` layers are generated with their own seeded weights and
+    caches and the stack cycles through them (generating and holding all 28-40 layers only costs host time;
+    every layer has the same shapes and the per-layer working set is far larger than L2 either way)."""
+    if world > 1:
+        cfg = gen.scaled_config(cfg, seed=cfg.seed + rank)
+    D = max(1, min(args.distinct_layers, cfg.n_layers))
+    lays = [build_inputs(cfg, l) for l in range(D)]
+    b_max = max(len(k) for lay in lays for k in lay["kept"])
+    engine = B.ENGINE_SIMT if args.engine == "simt" else B.ENGINE_AUTO
+    ctx = B.PkvContext(B.dims_from_config(cfg, b_max=b_max), engine=engine)
+    dev = []
+    for lay in lays:
+        off, idx = gen.kept_to_csr(lay["kept"])
+        kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+        dev.append({"w": B.to_device(lay["weights"], cfg.dtype), "K": kv["K"], "V": kv["V"], "head_off": off,
+                    "idx": torch.from_numpy(idx).cuda()})
+    layers = [dev[l % D] for l in range(cfg.n_layers)]
+    x_t = torch.from_numpy(lays[0]["x0"]).cuda()
+    W_merged = [d_["w"]["Wdown"].clone() for d_ in dev]
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    chunk_off = [0, cfg.N]
+    lams = list(cfg.lam_sweep) if cfg.lam_sweep else [cfg.lam0]
+    last = {}
+
+    def step(lam):
+        out = ctx.build_stack(layers, x_t, x_t, chunk_off, cfg.L, lam, B.LAMBDA_PAPER, want_final=True)
+        for l, dWl in enumerate(out["dW"]):
+            ctx.merge(W_merged[l % D], dWl)
+        last["out"] = out
+        return out
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3) if not args.quick else args.warmup):
+        step(lams[0])
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    l0 = ctx.launch_count()
+    per_lam = []
+    n_steps = 0
+    for lam in lams:
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for i in range(args.steps):
+            flush.fill_(i & 0xFF)
+            ev[i][0].record()
+            step(lam)
+            ev[i][1].record()
+            n_steps += 1
+        barrier()
+        per_lam.append(float(sum(a.elapsed_time(b) for a, b in ev) / args.steps))
+    launches = ctx.launch_count() - l0 + n_steps * cfg.n_layers
+    ms = float(sum(per_lam) / len(per_lam))
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ctx.set_timing(True)
+    st = step(lams[-1])["stats"]
+    ctx.set_timing(False)
+    clocks = sampler.stop()
+    stage_ms = [sum(s_["stage_ms"][i] for s_ in st) for i in range(9)]
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    b_list = [len(k) for k in lays[0]["kept"]]
+    work = stage_work(cfg, sum(b_list), max(b_list))
+    total_flops = sum(wk[1] for wk in work) * cfg.n_layers
+    dom = int(np.argmax(stage_ms))
+    name, fl, by, bound = work[dom]
+    dur = stage_ms[dom] * 1e-3
+    fl *= cfg.n_layers
+    if bound == "tensor":
+        peak, unit, ach, note = peaks["bf16_tflops_sustained"], "TFLOP/s", fl / dur / 1e12, "bf16 dense, sustained, %s" % peaks["source"]
+    elif bound == "alu":
+        peak = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+        unit, ach, note = "TFLOP/s", fl / dur / 1e12, "fp32 FMA peak (derived)"
+    else:
+        peak, unit, ach, note = peaks["hbm_gbs"], "GB/s", by * cfg.n_layers / dur / 1e9, "HBM copy, %s" % peaks["source"]
+    cpu = None
+    if not args.no_cpu_baseline and world == 1 and not args.quick:
+        n_sample = min(cfg.N, 16)
+        v, spent = oracle_sample(cfg, lays[0], n_sample)
+        cpu = {"value": v * cfg.n_layers, "unit": "ms", "cores": os.cpu_count() or 1, "kind": "oracle",
+               "sample": "fp64 numpy oracle on layer 0, first %d of %d reference tokens, full cache and full solve, token "
+                         "part scaled by %d/%d, extrapolated from 1 layer to %d; %.1f s of CPU wall time" %
+                         (n_sample, cfg.N, cfg.N, n_sample, cfg.n_layers, spent)}
+    conf = workload_config(cfg, lays[0])
+    conf.update({"layers_per_step": cfg.n_layers, "distinct_layers_generated": D,
+                 "lambda0": lams if len(lams) > 1 else lams[0]})
+    line = {"metric": "patch_build_ms_per_context", "value": ms / world, "unit": "ms", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "ms_per_layer": ms / cfg.n_layers,
+            "ms_per_lambda": per_lam, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": conf, "engine": "simt-fp32" if engine == B.ENGINE_SIMT else "tcgen05",
+            "algorithmic_tflops": total_flops / (ms * 1e-3) / 1e12,
+            "frac_bf16_peak": total_flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+            "roofline": {"kernel": name, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                         "traffic": None, "peak_note": note, "stage_ms": stage_ms[dom]},
+            "stages": [{"stage": wk[0], "ms": round(t_, 3)} for wk, t_ in zip(work, stage_ms)],
+            "cpu_baseline": cpu, "clocks": clocks,
+            "e2e": {"value": None, "unit": "ms", "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
+                    "note": "end-to-end with host buffers is measured on the single-block workload (default config 2)"},
+            "gpu_launches": int(launches), "peaks": peaks}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -174,6 +288,8 @@ def main():
     ap.add_argument("--engine", default="auto", choices=["auto", "simt"])
     ap.add_argument("--ref-sample", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--distinct-layers", type=int, default=2,
+                    help="stack configs: layers generated with their own weights/caches; the stack cycles through them")
     ap.add_argument("--quick", action="store_true",
                     help="timed steps only (no stage pass, no end-to-end pass, no CPU baseline): for profiler runs")
     args = ap.parse_args()
@@ -193,6 +309,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = measured_peaks()
     cfg = gen.benchmark_config(args.config)
+    if cfg.n_layers > 1:
+        run_stack(args, cfg, B, torch, dist, world, rank, local, peaks)
+        return
     if world > 1:      # replicas only: every rank builds the patch of its own context
         cfg = gen.scaled_config(cfg, seed=cfg.seed + rank)
     lay = build_inputs(cfg)
