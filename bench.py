@@ -24,6 +24,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2609_39329_b200 import dist_util as du  # noqa: E402
 from paper_2609_39329_b200 import inputs as gen  # noqa: E402
 
 
@@ -170,7 +171,7 @@ def run_stack(args, cfg, B, torch, dist, world, rank, local, peaks):
     caches and the stack cycles through them (generating and holding all 28-40 layers only costs host time;
     every layer has the same shapes and the per-layer working set is far larger than L2 either way)."""
     if world > 1:
-        cfg = gen.scaled_config(cfg, seed=cfg.seed + rank)
+        cfg = gen.scaled_config(cfg, seed=du.rank_seed(cfg.seed, rank))
     D = max(1, min(args.distinct_layers, cfg.n_layers))
     lays = [build_inputs(cfg, l) for l in range(D)]
     b_max = max(len(k) for lay in lays for k in lay["kept"])
@@ -222,10 +223,7 @@ def run_stack(args, cfg, B, torch, dist, world, rank, local, peaks):
         per_lam.append(float(sum(a.elapsed_time(b) for a, b in ev) / args.steps))
     launches = ctx.launch_count() - l0 + n_steps * cfg.n_layers
     ms = float(sum(per_lam) / len(per_lam))
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = du.max_over_ranks(ms, "cuda")
     ctx.set_timing(True)
     st = step(lams[-1])["stats"]
     ctx.set_timing(False)
@@ -313,7 +311,7 @@ def main():
         run_stack(args, cfg, B, torch, dist, world, rank, local, peaks)
         return
     if world > 1:      # replicas only: every rank builds the patch of its own context
-        cfg = gen.scaled_config(cfg, seed=cfg.seed + rank)
+        cfg = gen.scaled_config(cfg, seed=du.rank_seed(cfg.seed, rank))
     lay = build_inputs(cfg)
     b_list = [len(k) for k in lay["kept"]]
     off, idx = gen.kept_to_csr(lay["kept"])
@@ -357,10 +355,7 @@ def main():
     launches = ctx.launch_count() - l0 + args.steps      # + one merge kernel per step
     times = [a.elapsed_time(b) for a, b in ev]
     ms = float(sum(times) / len(times))
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = du.max_over_ranks(ms, "cuda")
 
     if args.quick:
         sampler.stop()
@@ -408,10 +403,7 @@ def main():
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_n
     clocks = sampler.stop()      # sampled over the timed steps, the stage pass and the end-to-end pass
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = du.max_over_ranks(e2e_ms, "cuda")
 
     # the same block through the dual (N x N) solver option: same dW, reported beside the headline
     dual_ms = None

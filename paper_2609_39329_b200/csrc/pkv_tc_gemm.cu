@@ -389,7 +389,11 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     if (g.M <= 0 || g.N <= 0 || g.batch <= 0) return PKV_OK;
     if (g.K < 0 || g.npass <= 0 || g.npass > kGemmMaxPass || (!g.C && g.nout == 0)) return PKV_ERR_INVALID_ARG;
     GemmTcParams p;
-    const int BN = (g.N <= 64) ? 64 : 128;
+    // 128 x 256 tiles move a third fewer operand bytes per flop than 128 x 128; taken when they still give
+    // at least two waves of CTAs (and the C tile is not prefetched: that variant is 128 wide)
+    const long long tiles256 = (long long)((g.N + 255) / 256) * ((g.M + 127) / 128) * g.batch;
+    const bool wide = g.N >= 512 && tiles256 >= 2 * 148 && !(g.C && g.accumulate) && !g.lower_only && g.k_tri != 2;
+    const int BN = (g.N <= 64) ? 64 : (wide ? 256 : 128);
     MapCache* cache = (MapCache*)lc.map_cache;
     // distinct operands
     const __nv_bfloat16* da[3];
@@ -432,6 +436,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     p.status = status;
     const bool pre = g.C && g.accumulate && p.vec_ok;
     if (BN == 64) return launch_gemm<64, false>(lc, p, g.batch);
+    if (BN == 256) return launch_gemm<256, false>(lc, p, g.batch);
     return pre ? launch_gemm<128, true>(lc, p, g.batch) : launch_gemm<128, false>(lc, p, g.batch);
 }
 
