@@ -237,6 +237,12 @@ int pkv_gram_noalloc(const float* X, const float* R, int32_t n, int32_t F, int32
 int pkv_ridge_solve(pkv_ctx* ctx, const float* S_H, const float* S_T, float lambda, int lambda_mode,
                     float* dW, pkv_stats* stats);
 
+/* Failure-detection self-test: launches one CTA whose pipeline wait is on a barrier that nothing ever
+ * completes, with a short limit (about a millisecond).  The wait must give up, raise the device status
+ * word and let the CTA exit; the call then returns PKV_ERR_TIMEOUT (err site in *site if not NULL) and
+ * the context stays usable.  Nothing faults, traps or spins without a limit. */
+int pkv_selftest_bounded_wait(pkv_ctx* ctx, int32_t* site);
+
 /* Enable (1) / disable (0) per-stage CUDA-event timing into pkv_stats.stage_ms. */
 int pkv_set_timing(pkv_ctx* ctx, int on);
 

@@ -118,6 +118,8 @@ def lib() -> C.CDLL:
                                    C.c_int, C.c_void_p]
     L.pkv_ridge_solve.restype = C.c_int
     L.pkv_ridge_solve.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_void_p, P(pkv_stats)]
+    L.pkv_selftest_bounded_wait.restype = C.c_int
+    L.pkv_selftest_bounded_wait.argtypes = [C.c_void_p, P(C.c_int32)]
     L.pkv_set_timing.restype = C.c_int
     L.pkv_set_timing.argtypes = [C.c_void_p, C.c_int]
     L.pkv_launch_count.restype = C.c_int64
@@ -154,13 +156,15 @@ class PkvContext:
     """Owns one pkv_ctx.  Tensors passed in must live on the context's CUDA device."""
 
     def __init__(self, dims: pkv_dims, engine: int = ENGINE_AUTO, kv_split: int = 0, stream=None,
-                 solver: int = SOLVER_PRIMAL):
+                 solver: int = SOLVER_PRIMAL, workspace=None):
         import torch
         self.torch = torch
         self.dims = dims
         self.L = lib()
         self.stream = stream
-        self.opts = pkv_opts(engine, kv_split, None, 0, solver)
+        self.workspace = workspace      # optional caller-owned uint8 CUDA tensor (kept alive with the context)
+        self.opts = pkv_opts(engine, kv_split, _ptr(workspace) if workspace is not None else None,
+                             int(workspace.numel()) if workspace is not None else 0, solver)
         h = C.c_void_p()
         sp = C.c_void_p(stream.cuda_stream) if stream is not None else C.c_void_p(torch.cuda.current_stream().cuda_stream)
         rc = self.L.pkv_create(C.byref(h), C.byref(dims), C.byref(self.opts), sp)
@@ -192,6 +196,12 @@ class PkvContext:
 
     def launch_count(self) -> int:
         return int(self.L.pkv_launch_count(self.h))
+
+    def selftest_bounded_wait(self):
+        """pkv_selftest_bounded_wait: returns (code, site)."""
+        site = C.c_int32(0)
+        rc = self.L.pkv_selftest_bounded_wait(self.h, C.byref(site))
+        return int(rc), int(site.value)
 
     def set_timing(self, on: bool):
         self.L.pkv_set_timing(self.h, 1 if on else 0)

@@ -269,6 +269,18 @@ extern "C" void pkv_destroy(pkv_ctx* c) {
     delete c;
 }
 
+extern "C" int pkv_selftest_bounded_wait(pkv_ctx* c, int32_t* site) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (c->engine == PKV_ENGINE_SIMT) return PKV_ERR_UNSUPPORTED;      // the SIMT engine has no waits
+    Lc lc{c->st, &c->launches, c->map_cache};
+    cudaMemsetAsync(c->b.status, 0, sizeof(DevStatus), c->st);
+    pkv::tc_selftest_wait(lc, c->b.status);
+    cudaError_t e = cudaMemcpyAsync(c->host_status, c->b.status, sizeof(DevStatus), cudaMemcpyDeviceToHost, c->st);
+    if (e != cudaSuccess || cudaStreamSynchronize(c->st) != cudaSuccess) return PKV_ERR_CUDA;
+    if (site) *site = c->host_status->info0;
+    return c->host_status->code;
+}
+
 extern "C" int pkv_set_timing(pkv_ctx* c, int on) {
     if (!c) return PKV_ERR_INVALID_ARG;
     c->timing = on ? 1 : 0;

@@ -51,7 +51,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 
 // Bounded wait.  `abort_flag` lives in shared memory and is shared by the CTA.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DevStatus* status,
-                                          int site) {
+                                          int site, long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     long long t0 = clock64();
     uint32_t spins = 0;
@@ -59,7 +59,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = 1;
                 if (atomicCAS(&status->code, 0, PKV_ERR_TIMEOUT) == 0) {
                     status->info0 = site;

@@ -43,6 +43,7 @@ MapCache* tc_map_cache_create();
 void tc_map_cache_destroy(MapCache* c);
 int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status);
 bool tc_encode_available();
+void tc_selftest_wait(const Lc& lc, DevStatus* status);
 int tc_make_map_2d(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows);
 int tc_make_map_3d(CUtensorMap* m, const void* ptr, uint64_t d2, uint64_t rows, uint64_t cols, uint64_t ld1,
                    uint64_t ld2, uint32_t box_rows);

@@ -254,6 +254,26 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     }
 }
 
+// Self-test of the bounded wait: the barrier below is initialised and never arrived on.
+__global__ void k_selftest_wait(DevStatus* status) {
+    __shared__ uint64_t bar_mem;
+    __shared__ int abort_flag;
+    const uint32_t bar = smem_u32(&bar_mem);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_wait(bar, 0, &abort_flag, status, 99, 2000000LL);   // ~1 ms
+    __syncthreads();
+}
+
+void tc_selftest_wait(const Lc& lc, DevStatus* status) {
+    k_selftest_wait<<<1, 32, 0, lc.st>>>(status);
+    lc.count();
+}
+
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------

@@ -357,3 +357,48 @@ def test_boundary_rejects_bad_arguments(B):
     with pytest.raises(B.PkvError) as ei:
         gpu_build(B, cfg, bad, x, x, [0, cfg.N], 0.1, B.ENGINE_SIMT)
     assert ei.value.code == -3 and ei.value.info["err_info"] == (1, 7)
+
+
+def test_bounded_wait_gives_timeout_status_and_context_survives(B):
+    """Failure detection without a fault: a pipeline wait on a barrier nothing completes runs out of its
+    (short) limit, the call returns PKV_ERR_TIMEOUT with the wait site, and the context keeps working."""
+    import torch
+    cfg = small_cfg("bf16", hd=128, Hq=4, Hkv=2)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    rc, site = ctx.selftest_bounded_wait()
+    assert rc == -7 and site == 99
+    r = np.random.default_rng(0)
+    X = torch.from_numpy(r.standard_normal((cfg.N, cfg.F)).astype(np.float32)).cuda()
+    R = torch.from_numpy(r.standard_normal((cfg.N, cfg.d)).astype(np.float32)).cuda()
+    gH, _ = ctx.gram(X, R)
+    assert H.rel_fro(gH.cpu().numpy(), X.double().cpu().numpy().T @ X.double().cpu().numpy()) <= 2e-4
+    ctx.close()
+
+
+def test_nonfinite_inputs_are_reported_and_caller_workspace_is_accepted(B):
+    import torch
+    cfg = small_cfg("bf16", hd=128, Hq=4, Hkv=2, N=64)
+    lay = H.make_problem(cfg)
+    x = lay["x0"].copy()
+    x[3, 5] = np.nan
+    with pytest.raises(B.PkvError) as ei:
+        gpu_build(B, cfg, lay, x, x, [0, cfg.N], 0.1, B.ENGINE_AUTO)
+    assert ei.value.code == -6
+    # caller-provided workspace: same result as the context-owned one; an undersized one is refused
+    dims = B.dims_from_config(cfg, b_max=max(len(k) for k in lay["kept"]))
+    probe = B.PkvContext(dims, engine=B.ENGINE_AUTO)
+    need = probe.workspace_bytes()
+    probe.close()
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    ctx = B.PkvContext(dims, engine=B.ENGINE_AUTO, workspace=ws)
+    w = B.to_device(lay["weights"], cfg.dtype)
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    off, idx = gen.kept_to_csr(lay["kept"])
+    xt = torch.from_numpy(lay["x0"]).cuda()
+    out = ctx.build_patch(w, kv["K"], kv["V"], off, torch.from_numpy(idx).cuda(), xt, xt, [0, cfg.N], cfg.L, 0.1)
+    ref = H.run_oracle(cfg, lay, lay["x0"], lay["x0"], [0, cfg.N], 0.1)
+    assert H.rel_fro(out["dW"].cpu().numpy(), ref["dW"]) <= DW_TOL
+    ctx.close()
+    with pytest.raises(B.PkvError) as ei:
+        B.PkvContext(dims, engine=B.ENGINE_AUTO, workspace=ws[:need // 2])
+    assert ei.value.code == -9
