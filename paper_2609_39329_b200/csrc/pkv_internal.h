@@ -26,6 +26,7 @@ struct Lc {
     cudaStream_t st;
     int64_t* launches;
     void* map_cache = nullptr;            // tensor-map cache of the tensor-core engine (optional)
+    bool pdl = false;                     // launch with programmatic stream serialisation (dependent launch)
     void count(int n = 1) const { if (launches) *launches += n; }
 };
 

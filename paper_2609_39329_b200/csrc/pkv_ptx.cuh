@@ -153,6 +153,13 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start
+// before its predecessor in the stream has finished; it must not touch the predecessor's results before
+// pdl_wait().  pdl_launch_dependents() lets the successor start its prologue early.  Both are no-ops for
+// ordinary launches.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
     asm volatile(

@@ -56,7 +56,7 @@ template <int BN, bool PRE>
 __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcParams p) {
     const int m0 = blockIdx.y * 128, n0 = blockIdx.x * BN, z = blockIdx.z;
     if (p.lower_only && n0 > m0 + 127) return;
-    if (p.status->code != 0) return;      // an earlier stage already failed: the call reports it
+    pdl_launch_dependents();
     // absolute coordinates of this tile's output; tiles entirely outside the stored region do nothing
     const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
     if (crow0 >= p.c_rows || ccol0 >= p.c_cols) return;
@@ -99,8 +99,13 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     __syncthreads();
     tc_fence_after();
     const uint32_t tbase = *tmem_slot;
+    // everything above is independent of earlier kernels; from here on their results are read
+    pdl_wait();
+    const bool skip = p.status->code != 0;      // an earlier stage already failed: the call reports it
 
-    if (warp == 0) {
+    if (skip) {
+        // nothing to do: fall through to the teardown
+    } else if (warp == 0) {
         if (lane == 0) {
             const int ar = p.a_row0 + z * p.a_zrow + m0, ac = p.a_col0 + z * p.a_zcol;
             const int br = p.b_row0 + z * p.b_zrow + n0, bc = p.b_col0 + z * p.b_zcol;
@@ -400,7 +405,21 @@ static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     p.stages = stages;
     const int smem = stages * stage_bytes + fixed;
     dim3 grid((p.N + BN - 1) / BN, (p.M + 127) / 128, batch);
-    k_gemm_tc<BN, PRE><<<grid, 192, smem, lc.st>>>(p);
+    if (lc.pdl) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(192);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = lc.st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, k_gemm_tc<BN, PRE>, p) != cudaSuccess) return PKV_ERR_CUDA;
+    } else {
+        k_gemm_tc<BN, PRE><<<grid, 192, smem, lc.st>>>(p);
+    }
     lc.count();
     return PKV_OK;
 }

@@ -12,9 +12,13 @@
 //   3. dW = (S_T X^T) X, two GEMMs that skip the zero tiles of the triangular factor.
 #include <math.h>
 
+#include "pkv_ptx.cuh"
 #include "pkv_tc.h"
 
 namespace pkv {
+
+using ptx::pdl_launch_dependents;
+using ptx::pdl_wait;
 
 constexpr int PB = 128;     // Cholesky block
 constexpr int SB = 16;      // sub-block inside the diagonal kernel
@@ -114,6 +118,8 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
     float(*X)[LDS] = reinterpret_cast<float(*)[LDS]>(smf + PB * LDS);
     float* rd = smf + 2 * PB * LDS;              // [128] reciprocals of the factor's diagonal
     float* T = rd + PB;                          // doubling temporary
+    pdl_launch_dependents();
+    pdl_wait();
     if (status->code != 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nbk = min(PB, n - k0);
@@ -466,6 +472,21 @@ void tc_solve_destroy(TcSolveBuffers* t) {
         }
 }
 
+static void launch_potrf(cudaStream_t st, int smem, const float* G, int n, int ld, int k0, Trip X3, Trip XT3, int six,
+                         DevStatus* status) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(kPotrfThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, k_potrf128, G, n, ld, k0, X3, XT3, six, status);
+}
+
 int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
                         float* dW, bool well_conditioned, bool zero_fill, DevStatus* status, const Pair* dW_pair,
                         __nv_bfloat16* const* S_T_triple) {
@@ -488,11 +509,11 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     // T2_b = update of everything to the right, on the helper stream, beside the next diagonal block.
     // sA: critical chain on the high-priority helper stream; sB: bulk updates on the caller's stream
     cudaStream_t sA = t->aux, sB = lc.st;
-    Lc lcA{sA, lc.launches, lc.map_cache};
+    Lc lcA{sA, lc.launches, lc.map_cache, true};
     Lc lcB{sB, lc.launches, lc.map_cache};
     cudaEventRecord(t->ev[2], sB);
     cudaStreamWaitEvent(sA, t->ev[2], 0);
-    k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, n, ld, 0, X3, XT3, well_conditioned ? 0 : 1, status);
+    launch_potrf(sA, smem, G, n, ld, 0, X3, XT3, well_conditioned ? 0 : 1, status);
     lc.count();
     if (F > PB) launch_split3(lcA, G + (size_t)PB * ld, ld, F - PB, PB, Trip{{P3.a[0] + (size_t)PB * PB, P3.a[1] + (size_t)PB * PB, P3.a[2] + (size_t)PB * PB}}, PB, 3);
     bool t2_pending = false;
@@ -537,7 +558,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         } else {
             t2_pending = false;
         }
-        k_potrf128<<<1, kPotrfThreads, smem, sA>>>(G, n, ld, k1, X3, XT3, well_conditioned ? 0 : 1, status);
+        launch_potrf(sA, smem, G, n, ld, k1, X3, XT3, well_conditioned ? 0 : 1, status);
         lc.count();
     }
     // join: the caller's stream continues after the chain's last kernel
