@@ -165,6 +165,62 @@ def workload_config(cfg, lay):
             "l2": "inputs (weights + caches, >300 MB) exceed L2 and a 512 MB buffer is written between steps"}
 
 
+def run_kernel(args, cfg, B, torch, peaks):
+    """One stage alone, through its single-stage entry point, on the shapes of a benchmark config."""
+    r = np.random.default_rng(cfg.seed)
+    N, F, d = cfg.N, cfg.F, cfg.d
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    if args.kernel == "attention":
+        kvd = gen.gen_cache(cfg, 0)
+        kept = gen.select_kept(cfg, 0, kvd["K"], gen.gen_obs_queries(cfg, 0) if cfg.kept_rule == "window_topk" else None)
+        off, idx = gen.kept_to_csr(kept)
+        ctx = B.PkvContext(B.dims_from_config(cfg, b_max=max(len(k) for k in kept)))
+        kv = B.to_device({"K": kvd["K"], "V": kvd["V"]}, cfg.dtype)
+        q = torch.from_numpy((r.standard_normal((2, N, cfg.Dq)) * 1.3).astype(np.float32)).cuda()
+        k = torch.from_numpy(r.standard_normal((2, N, cfg.Dkv)).astype(np.float32)).cuda()
+        v = torch.from_numpy(r.standard_normal((2, N, cfg.Dkv)).astype(np.float32)).cuda()
+        idx_t = torch.from_numpy(idx).cuda()
+        fn = lambda: ctx.attention(q, k, v, kv["K"], kv["V"], off, idx_t, [0, N])
+        b_mean = sum(len(k_) for k_ in kept) / cfg.Hkv
+        flops = 4.0 * N * cfg.L * cfg.Dq + 4.0 * N * b_mean * cfg.Dq + 4.0 * N * N * cfg.Dq
+        bound, note = "tensor", "prep + k_attn_tc* + combine; Q counted once (it runs as a bf16 hi+lo pair)"
+    elif args.kernel == "gram":
+        ctx = B.PkvContext(B.dims_from_config(cfg, b_max=16))
+        X = torch.from_numpy(r.standard_normal((N, F)).astype(np.float32)).cuda()
+        R = torch.from_numpy((0.1 * r.standard_normal((N, d))).astype(np.float32)).cuda()
+        S_H = torch.zeros((F, F), dtype=torch.float32, device="cuda")
+        S_T = torch.zeros((d, F), dtype=torch.float32, device="cuda")
+        fn = lambda: ctx.gram(X, R, S_H, S_T)
+        flops = float(N) * F * (F + 1) + 2.0 * N * F * d
+        bound, note = "tensor", "2 transposing splits + 2 three-pass k_gemm_tc; symmetric half counted once"
+    else:
+        ctx = B.PkvContext(B.dims_from_config(cfg, b_max=16))
+        X = r.standard_normal((N, F)).astype(np.float32)
+        S_H = torch.from_numpy(X.T @ X).cuda()
+        S_T = torch.from_numpy((0.1 * r.standard_normal((d, F))).astype(np.float32)).cuda()
+        fn = lambda: ctx.ridge_solve(S_H, S_T, cfg.lam0, B.LAMBDA_PAPER)
+        flops = F ** 3 / 3.0 + 2.0 * F * F * d
+        bound, note = "alu", "fp32-equivalent solve executed as multi-pass tensor-core products; fp32 FMA peak as reference"
+    for _ in range(max(args.warmup, 3) if not args.quick else args.warmup):
+        fn()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)
+        ev[i][0].record()
+        fn()
+        ev[i][1].record()
+    torch.cuda.synchronize()
+    ms = float(sum(a.elapsed_time(b) for a, b in ev) / args.steps)
+    peak = peaks["bf16_tflops_sustained"] if bound == "tensor" else 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+    ach = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({"kernel": args.kernel, "config": "config %d: %s" % (cfg.cfg_id, cfg.name), "ms": ms,
+                      "algorithmic_flops": flops,
+                      "roofline": {"bound": bound, "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+                                   "note": note}, "steps": args.steps}))
+    ctx.close()
+
+
 def run_stack(args, cfg, B, torch, dist, world, rank, local, peaks):
     """Configs 3-5: patches for all blocks of the stack built in sequence (pkv_build_stack); a step is one
     context = n_layers blocks.  `--distinct-layers` layers are generated with their own seeded weights and
@@ -288,6 +344,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--distinct-layers", type=int, default=2,
                     help="stack configs: layers generated with their own weights/caches; the stack cycles through them")
+    ap.add_argument("--kernel", default=None, choices=["attention", "gram", "solve"],
+                    help="time one stage alone through its own entry point (pkv_attention / pkv_gram / pkv_ridge_solve) "
+                         "on the shapes of --config, with seeded random operands")
     ap.add_argument("--quick", action="store_true",
                     help="timed steps only (no stage pass, no end-to-end pass, no CPU baseline): for profiler runs")
     args = ap.parse_args()
@@ -307,6 +366,9 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = measured_peaks()
     cfg = gen.benchmark_config(args.config)
+    if args.kernel:
+        run_kernel(args, cfg, B, torch, peaks)
+        return
     if cfg.n_layers > 1:
         run_stack(args, cfg, B, torch, dist, world, rank, local, peaks)
         return

@@ -450,7 +450,8 @@ static void solve_stage(pkv_ctx* c, const Lc& lc, float* S_H, const float* S_T, 
                         bool S_H_scratch) {
     const int F = c->dims.F, d = c->dims.d;
     Buffers& b = c->b;
-    trace_fro2(lc, S_H, F, b.status);
+    // the tensor-core build leaves only the lower triangle of its own S_H
+    trace_fro2(lc, S_H, F, b.status, 0, S_H_scratch && c->engine != PKV_ENGINE_SIMT);
     if (c->engine == PKV_ENGINE_SIMT) {
         make_ridge_matrix(lc, S_H, F, lam0, mode, b.solve.G, b.status);
         cudaMemcpyAsync(b.solve.Y, S_T, (size_t)d * F * sizeof(float), cudaMemcpyDeviceToDevice, c->st);

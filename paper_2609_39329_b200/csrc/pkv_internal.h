@@ -74,7 +74,8 @@ void oproj_epilogue(const Lc& lc, const float* xF, const float* xC, const float*
 void swiglu(const Lc& lc, const float* gu, int N, int F, float* hF, float* hC, float* dh);
 void transpose_f32(const Lc& lc, const float* in, int rows, int cols, float* out);
 // status->tr, fro2 from S [F][F]; optional sum of squares of an arbitrary buffer into *dst.
-void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status, int ld = 0);   // ld = 0: contiguous
+// ld = 0: contiguous.  lower: only entries on or below the diagonal are read (S symmetric).
+void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status, int ld = 0, bool lower = false);
 void sumsq(const Lc& lc, const float* a, int64_t n, double* dst);
 // lambda from the statistics (mode) into status->lam (and min_pivot reset).
 void ridge_lambda(const Lc& lc, int F, float lam0, int mode, DevStatus* status);

@@ -570,14 +570,19 @@ __device__ __forceinline__ double warp_sum_d(double v) {
 
 // tr(S) and ||S||_F^2: one row per block iteration, float4 loads, fp32 partial sums per thread
 // (a few hundred terms each), double precision across threads.
-__global__ void __launch_bounds__(256) k_trace_fro2(const float* __restrict__ S, int F, int ld, DevStatus* status) {
+__global__ void __launch_bounds__(256) k_trace_fro2(const float* __restrict__ S, int F, int ld, int lower,
+                                                    DevStatus* status) {
     float fro[4] = {0.f, 0.f, 0.f, 0.f};
     double tr = 0.0;
     int bad = 0;
     const bool vec = (F % 4 == 0) && (ld % 4 == 0) && (((uintptr_t)S & 15) == 0);
     for (int r = blockIdx.x; r < F; r += gridDim.x) {
         const float* row = S + (size_t)r * ld;
-        if (vec) {
+        if (lower) {
+            // symmetric matrix, lower triangle only: off-diagonal entries count twice
+            for (int c = threadIdx.x; c < r; c += 256) fro[0] = fmaf(2.f * row[c], row[c], fro[0]);
+            if (threadIdx.x == 0) fro[1] = fmaf(row[r], row[r], fro[1]);
+        } else if (vec) {
             for (int c = threadIdx.x * 4; c < F; c += 1024) {
                 float4 v = *reinterpret_cast<const float4*>(row + c);
                 fro[0] = fmaf(v.x, v.x, fro[0]); fro[1] = fmaf(v.y, v.y, fro[1]);
@@ -596,8 +601,8 @@ __global__ void __launch_bounds__(256) k_trace_fro2(const float* __restrict__ S,
     if (bad) raise(status, PKV_ERR_NONFINITE);
 }
 
-void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status, int ld) {
-    k_trace_fro2<<<min(F, 1184), 256, 0, lc.st>>>(S, F, ld > 0 ? ld : F, status);
+void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status, int ld, bool lower) {
+    k_trace_fro2<<<min(F, 1184), 256, 0, lc.st>>>(S, F, ld > 0 ? ld : F, lower ? 1 : 0, status);
     lc.count();
 }
 

@@ -282,9 +282,17 @@ void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, cons
     const int F = d->F, dm = d->d;
     transpose_split(lc, X, n, F, t->ldT, t->XT);
     transpose_split(lc, R, n, dm, t->ldT, t->RT);
-    gemm_pair_pair(lc, t->XT, t->ldT, t->XT, t->ldT, S_H, F, F, F, n, 1.f, nullptr, 0, accumulate, status);
     t->S3_ready = 0;
     if (!accumulate && S_T == t->own_S_T) {
+        // the build's own statistics: S_H is symmetric and its consumers (ridge scale, factorisation)
+        // read the lower triangle only, so only tiles on or below the diagonal are computed
+        TcGemm h = plain_gemm(F, F, n, S_H, F, 1.f, nullptr, 0, false);
+        h.A[0] = TcMat{t->XT.hi, t->ldT, F, n}; h.B[0] = TcMat{t->XT.hi, t->ldT, F, n};
+        h.A[1] = TcMat{t->XT.hi, t->ldT, F, n}; h.B[1] = TcMat{t->XT.lo, t->ldT, F, n};
+        h.A[2] = TcMat{t->XT.lo, t->ldT, F, n}; h.B[2] = TcMat{t->XT.hi, t->ldT, F, n};
+        h.npass = 3;
+        h.lower_only = true;
+        gemm_tc(lc, h, status);
         // the build's own statistics: also leave the bf16 triple of S_T for the solver's first product
         TcGemm g = plain_gemm(dm, F, n, S_T, F, 1.f, nullptr, 0, false);
         g.A[0] = TcMat{t->RT.hi, t->ldT, dm, n}; g.B[0] = TcMat{t->XT.hi, t->ldT, F, n};
@@ -295,6 +303,7 @@ void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, cons
         if (gemm_tc(lc, g, status) == PKV_OK) t->S3_ready = 1;
         return;
     }
+    gemm_pair_pair(lc, t->XT, t->ldT, t->XT, t->ldT, S_H, F, F, F, n, 1.f, nullptr, 0, accumulate, status);
     gemm_pair_pair(lc, t->RT, t->ldT, t->XT, t->ldT, S_T, F, dm, F, n, 1.f, nullptr, 0, accumulate, status);
 }
 
