@@ -81,9 +81,11 @@ struct pkv_ctx {
     int32_t* host_stage;     // pinned: head_off + tok_cs
     DevStatus* host_status;  // pinned
     int64_t launches;
+    int teacher_timed;
     void* map_cache;
     int timing;
     cudaEvent_t ev[ST_COUNT + 1];
+    cudaEvent_t evT[6];      // marks of the teacher half (tensor-core engine)
     char cuda_err[256];
 };
 
@@ -244,6 +246,7 @@ extern "C" int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* o
         return PKV_ERR_NOMEM;
     }
     for (int i = 0; i <= ST_COUNT; ++i) cudaEventCreate(&c->ev[i]);
+    for (int i = 0; i < 6; ++i) cudaEventCreate(&c->evT[i]);
     if (c->engine != PKV_ENGINE_SIMT) {
         c->map_cache = pkv::tc_map_cache_create();
         rc = pkv::tc_init(&c->b.tc, dims);
@@ -266,6 +269,8 @@ extern "C" void pkv_destroy(pkv_ctx* c) {
     if (c->engine != PKV_ENGINE_SIMT) pkv::tc_destroy(&c->b.tc);
     for (int i = 0; i <= ST_COUNT; ++i)
         if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    for (int i = 0; i < 6; ++i)
+        if (c->evT[i]) cudaEventDestroy(c->evT[i]);
     delete c;
 }
 
@@ -396,8 +401,25 @@ static int end_call(pkv_ctx* c, pkv_stats* stats, const int32_t* head_off) {
             stats->err_info[1] = s.info1;
         }
         for (int i = 0; i < 12; ++i) stats->stage_ms[i] = 0.f;
-        if (c->timing)
+        if (c->timing) {
             for (int i = 0; i < ST_COUNT; ++i) cudaEventElapsedTime(&stats->stage_ms[i], c->ev[i], c->ev[i + 1]);
+            if (c->teacher_timed) {
+                // the teacher half ran first, inside the interval the student's marks call "S1-S2":
+                // move its stages to where they belong
+                const int stage_of[5] = {ST_QKV, ST_ATTN, ST_OPROJ, ST_MLP, ST_NEXT};
+                float total = 0.f;
+                for (int i = 0; i < 5; ++i) {
+                    float ms = 0.f;
+                    cudaEventElapsedTime(&ms, c->evT[i], c->evT[i + 1]);
+                    total += ms;
+                    if (stage_of[i] != ST_QKV) stats->stage_ms[stage_of[i]] += ms;
+                }
+                float qkv = 0.f;
+                cudaEventElapsedTime(&qkv, c->evT[0], c->evT[1]);
+                stats->stage_ms[ST_QKV] -= (total - qkv);
+                c->teacher_timed = 0;
+            }
+        }
     }
     return s.code;
 }
@@ -544,11 +566,14 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         fa.head_off = b.head_off; fa.tok_cs = b.tok_cs; fa.rope_tab = b.rope_tab;
         fa.zF = b.zF; fa.zC = b.zC; fa.dz = b.dz; fa.hF = b.hF; fa.hC = b.hC; fa.R = b.R;
         fa.S_H = b.S_H; fa.S_T = b.S_T; fa.status = b.status;
-        fa.aF = b.a2; fa.aC = b.aC;
+        fa.aF = b.a2; fa.aC = b.aC; fa.dA = b.a2 + (size_t)N * Dq;
+        fa.xF_next = next ? next->xF_next : nullptr;
         fa.kv_split = c->kv_split;
         fa.dual = c->dual;
         fa.part_m = b.part_m; fa.part_l = b.part_l; fa.part_O = b.part_O;
         fa.ev = c->timing ? c->ev : nullptr;
+        fa.evT = nullptr;
+        c->teacher_timed = 0;
         rc = pkv::tc_forward(lc, &b.tc, &c->dims, fa);
         if (rc != PKV_OK) return rc;
     }

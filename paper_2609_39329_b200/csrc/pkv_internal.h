@@ -60,6 +60,7 @@ struct AttnArgs {
     int N, Hq, Hkv, hd, L, elem_bytes;
     int kv_split, nsplitF, nsplitC;
     int total_kept, max_b;                // rows of the compact cache (all heads), largest head
+    int mode;                             // 0: both streams; 1: teacher only (aF); 2: student only (aC, dA from a given aF)
     float* part_m; float* part_l; float* part_O;   // [nsplit][Hkv][N*g] and [..][hd]
     float* aF; float* aC; float* dA;      // [N][Hq*hd]
     __nv_bfloat16* pair_hi; __nv_bfloat16* pair_lo;   // optional: bf16 hi/lo parts of [aF; dA] as [2N][Hq*hd]

@@ -451,7 +451,11 @@ __global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
     int hd = a.hd;
     int per = hd / 32;                       // 2 or 4 columns per lane
     float res[2][4];
-    for (int s = 0; s < 2; ++s) {
+    const size_t o = (size_t)tok * a.Hq * hd + (size_t)(kh * g + hg) * hd + lane * per;
+    if (a.mode == 2) {      // the teacher's output was produced earlier
+        for (int c = 0; c < per; ++c) res[0][c] = a.aF[o + c];
+    }
+    for (int s = (a.mode == 2 ? 1 : 0); s < (a.mode == 1 ? 1 : 2); ++s) {
         int z0 = s ? a.nsplitF : 0;
         int ns = s ? a.nsplitC : a.nsplitF;
         float M = -INFINITY;
@@ -469,20 +473,26 @@ __global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
         float inv = (den > 0.f) ? 1.f / den : 0.f;
         for (int c = 0; c < per; ++c) res[s][c] = num[c] * inv;
     }
-    size_t o = (size_t)tok * a.Hq * hd + (size_t)(kh * g + hg) * hd + lane * per;
     for (int c = 0; c < per; ++c) {
-        const float f = res[0][c], dd = res[0][c] - res[1][c];
-        a.aF[o + c] = f;
-        a.aC[o + c] = res[1][c];
-        a.dA[o + c] = dd;
-        if (a.pair_hi) {        // operands of the o-projection: rows [0,N) aF, rows [N,2N) dA
-            const size_t o2 = o + c + (size_t)a.N * a.Hq * hd;
-            __nv_bfloat16 h = __float2bfloat16_rn(f);
-            a.pair_hi[o + c] = h;
-            a.pair_lo[o + c] = __float2bfloat16_rn(f - __bfloat162float(h));
-            h = __float2bfloat16_rn(dd);
-            a.pair_hi[o2] = h;
-            a.pair_lo[o2] = __float2bfloat16_rn(dd - __bfloat162float(h));
+        const float f = res[0][c];
+        if (a.mode != 2) {
+            a.aF[o + c] = f;
+            if (a.pair_hi) {    // operands of the o-projection: rows [0,N) aF, rows [N,2N) dA
+                __nv_bfloat16 h = __float2bfloat16_rn(f);
+                a.pair_hi[o + c] = h;
+                a.pair_lo[o + c] = __float2bfloat16_rn(f - __bfloat162float(h));
+            }
+        }
+        if (a.mode != 1) {
+            const float dd = f - res[1][c];
+            a.aC[o + c] = res[1][c];
+            a.dA[o + c] = dd;
+            if (a.pair_hi) {
+                const size_t o2 = o + c + (size_t)a.N * a.Hq * hd;
+                __nv_bfloat16 h = __float2bfloat16_rn(dd);
+                a.pair_hi[o2] = h;
+                a.pair_lo[o2] = __float2bfloat16_rn(dd - __bfloat162float(h));
+            }
         }
     }
 }

@@ -19,11 +19,13 @@ __device__ __forceinline__ void split2(float v, __nv_bfloat16& hi, __nv_bfloat16
     lo = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
+// rows [row0, row0 + gridDim.x) of the stacked input (rows [0,N) from x0, rows [N,2N) from x1)
 __global__ void __launch_bounds__(256) k_rmsnorm_split(const float* __restrict__ x0, const float* __restrict__ x1,
                                                        int N, int d, const float* __restrict__ gain, float eps,
-                                                       __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo) {
+                                                       __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo,
+                                                       int row0) {
     __shared__ float red[32];
-    int r = blockIdx.x;
+    int r = blockIdx.x + row0;
     const float* x = (r < N) ? x0 + (size_t)r * d : x1 + (size_t)(r - N) * d;
     float ss = 0.f;
     for (int c = threadIdx.x; c < d; c += blockDim.x) {
@@ -84,6 +86,47 @@ __global__ void __launch_bounds__(256) k_swiglu_split(const float* __restrict__ 
     split2(f, hF.hi[i], hF.lo[i]);
     split2(s, hC.hi[i], hC.lo[i]);
     split2(f - s, dh.hi[i], dh.lo[i]);
+}
+
+// teacher half: hF (fp32 + pair) from gu rows [0,N)
+__global__ void __launch_bounds__(256) k_swiglu_teacher(const float* __restrict__ gu, int N, int F,
+                                                        float* __restrict__ hF32, Pair hF) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)N * F) return;
+    size_t r = i / F, c = i % F;
+    const float* a = gu + r * 2 * F;
+    float f = silu_f(a[c]) * a[F + c];
+    hF32[i] = f;
+    split2(f, hF.hi[i], hF.lo[i]);
+}
+// student half: hC (fp32 + pair) from gu rows [N,2N), dh = hF - hC (pair) with the teacher's hF
+__global__ void __launch_bounds__(256) k_swiglu_student(const float* __restrict__ gu, int N, int F,
+                                                        const float* __restrict__ hF32, float* __restrict__ hC32,
+                                                        Pair hC, Pair dh) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)N * F) return;
+    size_t r = i / F, c = i % F;
+    const float* b = gu + (r + N) * 2 * F;
+    float s = silu_f(b[c]) * b[F + c];
+    hC32[i] = s;
+    split2(s, hC.hi[i], hC.lo[i]);
+    split2(hF32[i] - s, dh.hi[i], dh.lo[i]);
+}
+// teacher half of the o-projection epilogue: zF = xF + o[0:N]
+__global__ void k_oproj_teacher(const float* __restrict__ xF, const float* __restrict__ o, size_t n,
+                                float* __restrict__ zF) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) zF[i] = xF[i] + o[i];
+}
+// student half: dz = (xF - xC) + o[N:2N] (the projection of dA); zC = zF - dz
+__global__ void k_oproj_student(const float* __restrict__ xF, const float* __restrict__ xC,
+                                const float* __restrict__ o, const float* __restrict__ zF, size_t n,
+                                float* __restrict__ zC, float* __restrict__ dz) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float dd = (xF[i] - xC[i]) + o[n + i];
+    dz[i] = dd;
+    zC[i] = zF[i] - dd;
 }
 
 // in [rows][cols] fp32 -> out pair [cols][ldo] (token-contiguous operands of the statistics)
@@ -331,6 +374,119 @@ void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int 
     t->S3_ready = 0;
 }
 
+static void fill_attn(AttnArgs& at, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a, int mode) {
+    const int N = a.N, hd = D->hd, Dq = D->Hq * hd, Dkv = D->Hkv * hd, QKV = Dq + 2 * Dkv;
+    at.q = t->qkv; at.ldq = QKV; at.k_new = t->qkv + Dq; at.v_new = t->qkv + Dq + Dkv; at.ldkv = QKV;
+    at.K = a.full->K; at.V = a.full->V; at.Kc = a.Kc; at.Vc = a.Vc; at.bias = a.bias;
+    at.head_off = a.head_off; at.tok_cs = a.tok_cs;
+    at.N = N; at.Hq = D->Hq; at.Hkv = D->Hkv; at.hd = hd; at.L = D->L; at.elem_bytes = 2;
+    at.total_kept = a.total_kept; at.max_b = a.max_b;
+    at.aF = a.aF; at.aC = a.aC; at.dA = a.dA;
+    at.pair_hi = t->a.hi; at.pair_lo = t->a.lo;
+    at.mode = mode;
+}
+
+// Teacher half of one block (Algorithm 1, teacher forward): it reads only xF, the block weights and the full
+// cache, never a patch, and touches only the teacher halves of the stacked scratch buffers (rows [0,N),
+// stream 0 of the attention operands, the teacher's split partials), so that it may run beside the student
+// half / the solve of an earlier block.  Outputs: aF, zF, hF (fp32; hF also as a bf16 pair) and, if asked,
+// xF_next = zF + hF W^T.  The RoPE table must already be there.
+int tc_teacher_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a, float* xF_next) {
+    const int N = a.N, d = D->d, F = D->F, hd = D->hd;
+    const int Dq = D->Hq * hd, Dkv = D->Hkv * hd, QKV = Dq + 2 * Dkv;
+    const pkv_block_weights* w = a.w;
+    DevStatus* st = a.status;
+    int rc;
+    auto markT = [&](int i) { if (a.evT) cudaEventRecord(a.evT[i], lc.st); };
+    markT(0);
+    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.xF, a.xF, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, 0);
+    lc.count();
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wq, d, t->qkv, QKV, N, Dq, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wk, d, t->qkv + Dq, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wv, d, t->qkv + Dq + Dkv, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    markT(1);
+    AttnArgs at{};
+    fill_attn(at, t, D, a, 1);
+    if ((rc = attention_tc(lc, t, D, at, a.rope_tab, st))) return rc;
+    markT(2);
+    // o-projection of aF, residual
+    if ((rc = gemm_act_weight(lc, t->a, Dq, w->Wo, Dq, t->o, d, N, d, Dq, 1.f, nullptr, 0, st))) return rc;
+    {
+        size_t n = (size_t)N * d;
+        k_oproj_teacher<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(a.xF, t->o, n, a.zF);
+        lc.count();
+    }
+    markT(3);
+    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.zF, a.zF, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, 0);
+    lc.count();
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wgate, d, t->gu, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, t->u, d, w->Wup, d, t->gu + F, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        size_t n = (size_t)N * F;
+        k_swiglu_teacher<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, t->hF);
+        lc.count();
+    }
+    markT(4);
+    if (xF_next) rc = gemm_act_weight(lc, t->hF, F, w->Wdown, F, xF_next, d, N, d, F, 1.f, a.zF, d, st);
+    markT(5);
+    return rc;
+}
+
+// Student half (Algorithm 1, student forward + targets + statistics), rows [N,2N) of the stacked buffers.
+// Reads the teacher's aF, zF, hF.  Differences (dA, dz, dh) are formed in fp32 before any rounding.
+int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a) {
+    const int N = a.N, d = D->d, F = D->F, hd = D->hd;
+    const int Dq = D->Hq * hd, Dkv = D->Hkv * hd, QKV = Dq + 2 * Dkv;
+    const pkv_block_weights* w = a.w;
+    DevStatus* st = a.status;
+    int rc;
+    const size_t uo = (size_t)N * d;                   // offsets of the student rows
+    Pair uS{t->u.hi + uo, t->u.lo + uo};
+    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.xF, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, N);
+    lc.count();
+    float* qkvS = t->qkv + (size_t)N * QKV;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wq, d, qkvS, QKV, N, Dq, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wk, d, qkvS + Dq, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wv, d, qkvS + Dq + Dkv, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    mark(a, lc, 2);
+    AttnArgs at{};
+    fill_attn(at, t, D, a, 2);
+    if ((rc = attention_tc(lc, t, D, at, a.rope_tab, st))) return rc;
+    mark(a, lc, 3);
+    // o-projection of dA: dz, zC
+    Pair aS{t->a.hi + (size_t)N * Dq, t->a.lo + (size_t)N * Dq};
+    if ((rc = gemm_act_weight(lc, aS, Dq, w->Wo, Dq, t->o + uo, d, N, d, Dq, 1.f, nullptr, 0, st))) return rc;
+    {
+        size_t n = (size_t)N * d;
+        k_oproj_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(a.xF, a.xC, t->o, a.zF, n, a.zC, a.dz);
+        lc.count();
+    }
+    mark(a, lc, 4);
+    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.zF, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, N);
+    lc.count();
+    float* guS = t->gu + (size_t)N * 2 * F;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wgate, d, guS, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wup, d, guS + F, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        size_t n = (size_t)N * F;
+        k_swiglu_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hC, t->dh);
+        lc.count();
+    }
+    mark(a, lc, 5);
+    // S6: T = dh Wdown^T + dz   (Eq. 5)
+    if ((rc = gemm_act_weight(lc, t->dh, F, w->Wdown, F, a.R, d, N, d, F, 1.f, a.dz, d, st))) return rc;
+    sumsq(lc, a.R, (int64_t)N * d, &st->t_fro2);
+    mark(a, lc, 6);
+    // S7 (Eq. 9); the dual solver only needs the token-contiguous copy of the student features
+    t->own_S_T = a.S_T;
+    if (a.dual) transpose_split(lc, a.hC, N, F, t->ldT, t->XT);
+    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st);
+    mark(a, lc, 7);
+    return PKV_OK;
+}
+
+// One block on one stream with teacher and student fused: every product runs once on the stacked rows
+// (rows [0,N) teacher, [N,2N) student) and the attention is one launch.  Fastest when nothing can overlap.
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a) {
     const int N = a.N, d = D->d, F = D->F, hd = D->hd;
     const int Dq = D->Hq * hd, Dkv = D->Hkv * hd, QKV = Dq + 2 * Dkv;
@@ -338,7 +494,7 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     DevStatus* st = a.status;
     int rc;
     // S1-S2: both streams stacked, rows [0,N) teacher, [N,2N) student
-    k_rmsnorm_split<<<2 * N, 256, 0, lc.st>>>(a.xF, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo);
+    k_rmsnorm_split<<<2 * N, 256, 0, lc.st>>>(a.xF, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, 0);
     lc.count();
     if ((rc = gemm_act_weight(lc, t->u, d, w->Wq, d, t->qkv, QKV, 2 * N, Dq, d, 1.f, nullptr, 0, st))) return rc;
     if ((rc = gemm_act_weight(lc, t->u, d, w->Wk, d, t->qkv + Dq, QKV, 2 * N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
@@ -353,7 +509,7 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     at.head_off = a.head_off; at.tok_cs = a.tok_cs;
     at.N = N; at.Hq = D->Hq; at.Hkv = D->Hkv; at.hd = hd; at.L = D->L; at.elem_bytes = 2;
     at.total_kept = a.total_kept; at.max_b = a.max_b;
-    at.aF = a.aF; at.aC = a.aC; at.dA = a.aF + (size_t)N * Dq;
+    at.aF = a.aF; at.aC = a.aC; at.dA = a.dA;
     at.pair_hi = t->a.hi; at.pair_lo = t->a.lo;
     // the S2 outputs are not rotated yet: the operand-preparation kernel applies RoPE
     if ((rc = attention_tc(lc, t, D, at, a.rope_tab, st))) return rc;
@@ -363,7 +519,7 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     oproj_epilogue(lc, a.xF, a.xC, t->o, N, d, a.zF, a.zC, a.dz);
     mark(a, lc, 4);
     // S5
-    k_rmsnorm_split<<<2 * N, 256, 0, lc.st>>>(a.zF, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo);
+    k_rmsnorm_split<<<2 * N, 256, 0, lc.st>>>(a.zF, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, 0);
     lc.count();
     if ((rc = gemm_act_weight(lc, t->u, d, w->Wgate, d, t->gu, 2 * F, 2 * N, F, d, 1.f, nullptr, 0, st))) return rc;
     if ((rc = gemm_act_weight(lc, t->u, d, w->Wup, d, t->gu + F, 2 * F, 2 * N, F, d, 1.f, nullptr, 0, st))) return rc;
@@ -385,11 +541,13 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     return PKV_OK;
 }
 
+
+
 void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const void* Wdown, const float* dW,
                     const float* zF, const float* R, float* xF_next, float* Dm, DevStatus* status) {
     const int d = D->d, F = D->F;
-    // xF_next = zF + hF Wdown^T
-    gemm_act_weight(lc, t->hF, F, Wdown, F, xF_next, d, N, d, F, 1.f, zF, d, status);
+    // xF_next = zF + hF Wdown^T (skipped when the teacher half already produced it)
+    if (xF_next) gemm_act_weight(lc, t->hF, F, Wdown, F, xF_next, d, N, d, F, 1.f, zF, d, status);
     // D = T - hC dW^T
     (void)dW;      // its bf16 pair was written by the solver's last product
     gemm_pair_pair(lc, t->hC, F, t->dW, F, Dm, d, N, d, F, -1.f, R, d, false, status);

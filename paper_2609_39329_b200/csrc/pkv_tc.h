@@ -116,11 +116,13 @@ struct TcForwardArgs {
     const float* xF; const float* xC;
     int N, pos0, max_b, total_kept, kv_split;
     const int32_t* head_off; const int32_t* tok_cs; float* rope_tab;
-    float *zF, *zC, *dz, *hF, *hC, *R, *S_H, *S_T, *aF, *aC;
+    float *zF, *zC, *dz, *hF, *hC, *R, *S_H, *S_T, *aF, *aC, *dA;
+    float* xF_next;     // optional: teacher state entering the next block
     float *part_m, *part_l, *part_O;
     int dual;           // 1: only the token-contiguous copy of the student features is prepared in S7
     DevStatus* status;
     cudaEvent_t* ev;    // stage marks (index = stage) or nullptr
+    cudaEvent_t* evT;   // 6 marks around the teacher half's stages (S1-2, S3, S4, S5, S9 share) or nullptr
 };
 
 void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, int* nsplitC);
@@ -135,6 +137,8 @@ int tc_dual_solve(const Lc& lc, TcBuffers* t, const pkv_dims* d, int N, const fl
 int tc_init(TcBuffers* t, const pkv_dims* d);
 void tc_destroy(TcBuffers* t);
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a);
+int tc_teacher_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a, float* xF_next);
+int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a);
 int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status);
 void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, const float* R, int n, float* S_H,
              float* S_T, bool accumulate, DevStatus* status);

@@ -34,17 +34,18 @@ using namespace ptx;
 __global__ void __launch_bounds__(256) k_attn_prep(const float* __restrict__ q, long long ldq,
                                                    const float* __restrict__ k, const float* __restrict__ v,
                                                    long long ldkv, const float* __restrict__ rope_tab, int N, int Hq,
-                                                   int Hkv, int hd, __nv_bfloat16* __restrict__ qhi,
+                                                   int Hkv, int hd, int s_begin, int s_count,
+                                                   __nv_bfloat16* __restrict__ qhi,
                                                    __nv_bfloat16* __restrict__ qlo, __nv_bfloat16* __restrict__ kn,
                                                    __nv_bfloat16* __restrict__ vn) {
     const int half = hd / 2;
     const int heads = Hq + 2 * Hkv;
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    size_t total = (size_t)2 * N * heads * half;
+    size_t total = (size_t)s_count * N * heads * half;
     if (i >= total) return;
     int c = (int)(i % half);
     int h = (int)((i / half) % heads);
-    int row = (int)(i / ((size_t)half * heads));
+    int row = (int)(i / ((size_t)half * heads)) + s_begin * N;
     int s = row / N, tok = row % N;
     float co = 1.f, si = 0.f;
     if (rope_tab) {
@@ -93,6 +94,7 @@ struct alignas(64) AttnTcParams {
     const float* bias;
     int N, g, Hkv, L, rows;
     int tps, nsplitF, nsplitC;
+    int z0;
     float* part_m;
     float* part_l;
     float* part_O;
@@ -149,7 +151,7 @@ __global__ void __launch_bounds__(192, 1) k_attn_tc(const __grid_constant__ Attn
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kh = blockIdx.y;
-    const int z = blockIdx.z;
+    const int z = blockIdx.z + p.z0;
     const int stream = (z >= p.nsplitF) ? 1 : 0;
     const int split = stream ? z - p.nsplitF : z;
     const int r0 = blockIdx.x * 128;
@@ -447,7 +449,7 @@ void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, i
 }
 
 template <int HD>
-static int launch_attn(const Lc& lc, const AttnTcParams& p, int qtiles) {
+static int launch_attn(const Lc& lc, const AttnTcParams& p, int qtiles, int zcount) {
     using S = AttnSmem<HD>;
     static bool attr_set = false;
     if (!attr_set) {
@@ -455,14 +457,14 @@ static int launch_attn(const Lc& lc, const AttnTcParams& p, int qtiles) {
             return PKV_ERR_CUDA;
         attr_set = true;
     }
-    dim3 grid(qtiles, p.Hkv, p.nsplitF + p.nsplitC);
+    dim3 grid(qtiles, p.Hkv, zcount);
     k_attn_tc<HD><<<grid, 192, S::kTotal, lc.st>>>(p);
     lc.count();
     return PKV_OK;
 }
 
 // hd = 128: the two-tile kernel of pkv_tc_attn2.cu (operands already prepared in t->q, t->kn, t->vn)
-int launch_attn2(const Lc& lc, const Attn2Params& p, int qpairs);
+int launch_attn2(const Lc& lc, const Attn2Params& p, int qpairs, int zcount);
 static int attention_tc2(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status) {
     const int N = a.N, hd = d->hd, Hkv = d->Hkv, g = d->Hq / d->Hkv;
     const int rows = N * g;
@@ -491,7 +493,9 @@ static int attention_tc2(const Lc& lc, TcBuffers* t, const pkv_dims* d, const At
     tc_attn_plan(d, N, a.max_b, &p.tps, &p.nsplitF, &p.nsplitC);
     p.part_m = t->part_m; p.part_l = t->part_l; p.part_O = t->part_O;
     p.status = status;
-    rc = launch_attn2(lc, p, (rows + 255) / 256);
+    p.z0 = (a.mode == 2) ? p.nsplitF : 0;
+    rc = launch_attn2(lc, p, (rows + 255) / 256,
+                      a.mode == 0 ? p.nsplitF + p.nsplitC : (a.mode == 1 ? p.nsplitF : p.nsplitC));
     if (rc != PKV_OK) return rc;
     AttnArgs c = a;
     c.nsplitF = p.nsplitF; c.nsplitC = p.nsplitC;
@@ -504,10 +508,12 @@ int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
                  DevStatus* status) {
     const int N = a.N, hd = d->hd, Hkv = d->Hkv, g = d->Hq / d->Hkv;
     const int rows = N * g;
+    const int s_begin = (a.mode == 2) ? 1 : 0, s_count = (a.mode == 0) ? 2 : 1;
     {
-        size_t total = (size_t)2 * N * (d->Hq + 2 * Hkv) * (hd / 2);
+        size_t total = (size_t)s_count * N * (d->Hq + 2 * Hkv) * (hd / 2);
         k_attn_prep<<<(unsigned)((total + 255) / 256), 256, 0, lc.st>>>(a.q, a.ldq, a.k_new, a.v_new, a.ldkv, rope_tab, N,
-                                                                        d->Hq, Hkv, hd, t->q.hi, t->q.lo, t->kn, t->vn);
+                                                                        d->Hq, Hkv, hd, s_begin, s_count, t->q.hi, t->q.lo,
+                                                                        t->kn, t->vn);
         lc.count();
     }
     if (hd == 128) return attention_tc2(lc, t, d, a, status);
@@ -538,7 +544,9 @@ int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
     p.part_m = t->part_m; p.part_l = t->part_l; p.part_O = t->part_O;
     p.status = status;
     const int qtiles = (rows + 127) / 128;
-    rc = (hd == 128) ? launch_attn<128>(lc, p, qtiles) : launch_attn<64>(lc, p, qtiles);
+    p.z0 = (a.mode == 2) ? p.nsplitF : 0;
+    const int zcount = a.mode == 0 ? p.nsplitF + p.nsplitC : (a.mode == 1 ? p.nsplitF : p.nsplitC);
+    rc = (hd == 128) ? launch_attn<128>(lc, p, qtiles, zcount) : launch_attn<64>(lc, p, qtiles, zcount);
     if (rc != PKV_OK) return rc;
     AttnArgs c = a;
     c.nsplitF = p.nsplitF; c.nsplitC = p.nsplitC;

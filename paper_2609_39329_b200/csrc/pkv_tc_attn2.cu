@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kh = blockIdx.y;
-    const int z = blockIdx.z;
+    const int z = blockIdx.z + p.z0;
     const int stream = (z >= p.nsplitF) ? 1 : 0;
     const int split = stream ? z - p.nsplitF : z;
     const int r0 = blockIdx.x * 256;
@@ -370,14 +370,14 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
     }
 }
 
-int launch_attn2(const Lc& lc, const Attn2Params& p, int qpairs) {
+int launch_attn2(const Lc& lc, const Attn2Params& p, int qpairs, int zcount) {
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(k_attn_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, a2::kTotal) != cudaSuccess)
             return PKV_ERR_CUDA;
         attr_set = true;
     }
-    dim3 grid(qpairs, p.Hkv, p.nsplitF + p.nsplitC);
+    dim3 grid(qpairs, p.Hkv, zcount);
     k_attn_tc2<<<grid, 320, a2::kTotal, lc.st>>>(p);
     lc.count();
     return PKV_OK;

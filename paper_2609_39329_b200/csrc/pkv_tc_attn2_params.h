@@ -17,6 +17,7 @@ struct alignas(64) Attn2Params {
     const float* bias;
     int N, g, Hkv, L, rows;
     int tps, nsplitF, nsplitC;
+    int z0;                   // first split index of this launch (teacher splits come first, then the student's)
     float* part_m;
     float* part_l;
     float* part_O;
