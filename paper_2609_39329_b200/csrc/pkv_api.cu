@@ -20,6 +20,8 @@ static const char* kStageNames[ST_COUNT] = {"S0 index check + compaction", "S1-S
                                             "S7 Gram + cross statistics",  "S8 ridge solve",
                                             "S9 next states"};
 
+constexpr int kMaxStackLayers = 128;
+
 struct Carver {
     char* base;
     size_t off;
@@ -62,6 +64,15 @@ struct Buffers {
     SolveWs solve;
     float* D;       // [N][d]
     float* xs[4];   // stack states, ping-pong: xF a/b, xC a/b
+    // overlapped stack driver (tensor-core engine): teacher outputs of two blocks in flight, the state
+    // difference xF - xC (ping-pong), per-layer status words and kept-set offsets
+    float* ringA[2];   // aF [N][Dq]
+    float* ringZ[2];   // zF [N][d]
+    float* ringH[2];   // hF [N][F]
+    float* ringX[2];   // xF_next [N][d]
+    float* dxbuf[2];   // [N][d]
+    DevStatus* lstatus;    // [kMaxStackLayers]
+    int32_t* lhead_off;    // [kMaxStackLayers][Hkv+1]
     pkv::TcBuffers tc;
 };
 
@@ -80,6 +91,10 @@ struct pkv_ctx {
     Buffers b;
     int32_t* host_stage;     // pinned: head_off + tok_cs
     DevStatus* host_status;  // pinned
+    int32_t* host_lhead;     // pinned: per-layer kept-set offsets of a stack call
+    DevStatus* host_lstatus; // pinned: per-layer status words of a stack call
+    cudaStream_t tstream;    // teacher stream of the overlapped stack driver
+    cudaEvent_t evTea[2], evStu[2], evSetup;
     int64_t launches;
     int teacher_timed;
     void* map_cache;
@@ -159,7 +174,18 @@ static size_t carve(Buffers* b, char* base, const pkv_dims* d, int engine, int e
     b->solve.Y = c.take<float>(dm * F);
     b->D = c.take<float>(N * dm);
     for (int i = 0; i < 4; ++i) b->xs[i] = c.take<float>(N * dm);
-    if (engine != PKV_ENGINE_SIMT) c.off = pkv::tc_carve(&b->tc, base, c.off, d, dual);
+    if (engine != PKV_ENGINE_SIMT) {
+        for (int i = 0; i < 2; ++i) {
+            b->ringA[i] = c.take<float>(N * Dq);
+            b->ringZ[i] = c.take<float>(N * dm);
+            b->ringH[i] = c.take<float>(N * F);
+            b->ringX[i] = c.take<float>(N * dm);
+            b->dxbuf[i] = c.take<float>(N * dm);
+        }
+        b->lstatus = c.take<DevStatus>(kMaxStackLayers);
+        b->lhead_off = c.take<int32_t>((size_t)kMaxStackLayers * (d->Hkv + 1));
+        c.off = pkv::tc_carve(&b->tc, base, c.off, d, dual);
+    }
     return (c.off + 255) & ~(size_t)255;
 }
 
@@ -245,6 +271,20 @@ extern "C" int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* o
         pkv_destroy(c);
         return PKV_ERR_NOMEM;
     }
+    if (c->engine != PKV_ENGINE_SIMT) {
+        if (cudaMallocHost((void**)&c->host_lhead, (size_t)kMaxStackLayers * (dims->Hkv + 1) * sizeof(int32_t)) != cudaSuccess ||
+            cudaMallocHost((void**)&c->host_lstatus, (size_t)kMaxStackLayers * sizeof(DevStatus)) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&c->tstream, cudaStreamNonBlocking) != cudaSuccess) {
+            cudaGetLastError();
+            pkv_destroy(c);
+            return PKV_ERR_NOMEM;
+        }
+        for (int i = 0; i < 2; ++i) {
+            cudaEventCreateWithFlags(&c->evTea[i], cudaEventDisableTiming);
+            cudaEventCreateWithFlags(&c->evStu[i], cudaEventDisableTiming);
+        }
+        cudaEventCreateWithFlags(&c->evSetup, cudaEventDisableTiming);
+    }
     for (int i = 0; i <= ST_COUNT; ++i) cudaEventCreate(&c->ev[i]);
     for (int i = 0; i < 6; ++i) cudaEventCreate(&c->evT[i]);
     if (c->engine != PKV_ENGINE_SIMT) {
@@ -265,6 +305,14 @@ extern "C" void pkv_destroy(pkv_ctx* c) {
     if (c->own_ws && c->ws) cudaFree(c->ws);
     if (c->host_stage) cudaFreeHost(c->host_stage);
     if (c->host_status) cudaFreeHost(c->host_status);
+    if (c->host_lhead) cudaFreeHost(c->host_lhead);
+    if (c->host_lstatus) cudaFreeHost(c->host_lstatus);
+    if (c->tstream) { cudaStreamSynchronize(c->tstream); cudaStreamDestroy(c->tstream); }
+    for (int i = 0; i < 2; ++i) {
+        if (c->evTea[i]) cudaEventDestroy(c->evTea[i]);
+        if (c->evStu[i]) cudaEventDestroy(c->evStu[i]);
+    }
+    if (c->evSetup) cudaEventDestroy(c->evSetup);
     if (c->map_cache) pkv::tc_map_cache_destroy((pkv::MapCache*)c->map_cache);
     if (c->engine != PKV_ENGINE_SIMT) pkv::tc_destroy(&c->b.tc);
     for (int i = 0; i <= ST_COUNT; ++i)
@@ -445,10 +493,11 @@ static AttnArgs attn_args(pkv_ctx* c, const float* q, int64_t ldq, const float* 
 
 // S0: returns the compact cache pointers to use
 static void stage_compact(pkv_ctx* c, const Lc& lc, const pkv_kv* full, const pkv_kv_compressed* cb, int total,
-                          const void** Kc, const void** Vc) {
+                          const void** Kc, const void** Vc, const int32_t* head_off_dev = nullptr,
+                          DevStatus* status = nullptr) {
     if (cb->idx && total > 0) {
-        gather_kept(lc, c->elem_bytes, full->K, full->V, cb->idx, c->b.head_off, c->dims.Hkv, c->dims.L, c->dims.hd,
-                    total, c->b.Kc, c->b.Vc, c->b.status);
+        gather_kept(lc, c->elem_bytes, full->K, full->V, cb->idx, head_off_dev ? head_off_dev : c->b.head_off,
+                    c->dims.Hkv, c->dims.L, c->dims.hd, total, c->b.Kc, c->b.Vc, status ? status : c->b.status);
         *Kc = c->b.Kc;
         *Vc = c->b.Vc;
     } else {
@@ -469,9 +518,11 @@ static void gram_simt(pkv_ctx* c, const Lc& lc, const float* X, const float* R, 
 
 // S8.  `S_H_scratch` says that S_H may be overwritten (it is the context's own statistics buffer).
 static void solve_stage(pkv_ctx* c, const Lc& lc, float* S_H, const float* S_T, float lam0, int mode, float* dW,
-                        bool S_H_scratch) {
+                        bool S_H_scratch, DevStatus* status = nullptr) {
     const int F = c->dims.F, d = c->dims.d;
-    Buffers& b = c->b;
+    Buffers bl = c->b;
+    if (status) bl.status = status;
+    Buffers& b = bl;
     // the tensor-core build leaves only the lower triangle of its own S_H
     trace_fro2(lc, S_H, F, b.status, 0, S_H_scratch && c->engine != PKV_ENGINE_SIMT);
     if (c->engine == PKV_ENGINE_SIMT) {
@@ -616,11 +667,133 @@ extern "C" int pkv_merge(void* W, int w_dtype, const float* dW, int64_t count, v
     return cudaGetLastError() == cudaSuccess ? PKV_OK : PKV_ERR_CUDA;
 }
 
+static void fill_stats(pkv_ctx* c, const DevStatus& s, pkv_stats* stats, const int32_t* head_off) {
+    memset(stats, 0, sizeof(*stats));
+    stats->lambda_eff = s.lam;
+    stats->trace = s.tr;
+    stats->fro2 = s.fro2;
+    stats->target_fro2 = s.t_fro2;
+    stats->resid_fro2 = s.res_fro2;
+    stats->dW_fro2 = s.dw_fro2;
+    stats->min_pivot = s.min_pivot;
+    if (s.code == PKV_ERR_BAD_INDEX && s.bad_index && head_off) {
+        int pos = (int)(s.bad_index - 1), h = 0;
+        while (h + 1 < c->dims.Hkv && head_off[h + 1] <= pos) ++h;
+        stats->err_info[0] = h;
+        stats->err_info[1] = pos - head_off[h];
+    } else if (s.code == PKV_ERR_NOT_PD && s.bad_column) {
+        stats->err_info[0] = (int)(s.bad_column - 1);
+    } else if (s.code == PKV_ERR_TIMEOUT) {
+        stats->err_info[0] = s.info0;
+        stats->err_info[1] = s.info1;
+    }
+}
+
+// Stack driver with the teacher run ahead (tensor-core engine).  The teacher stream of Algorithm 1 never sees
+// a patch, so the teacher half of block l+1 (and l+2) runs on its own CUDA stream beside the student half and
+// the latency-bound ridge solve of block l.  Teacher outputs live in a ring of two slots; the student carries
+// the state difference xF - xC itself, so that it never reads a teacher state that may already be overwritten.
+static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv_block_weights* w, const pkv_kv* full,
+                                  const pkv_kv_compressed* cb, const pkv_ref* ref0, float lambda, int mode,
+                                  float* const* dW, const pkv_ref_next* final, pkv_stats* stats) {
+    const pkv_dims& D = c->dims;
+    const int N = ref0->N, d = D.d, F = D.F, Hkv = D.Hkv;
+    const int Dq = D.Hq * D.hd;
+    Buffers& b = c->b;
+    int rc = check_chunks(c, N, ref0->n_chunks, ref0->chunk_off);
+    if (rc != PKV_OK) return rc;
+    if (!(lambda > 0.f) || !isfinite(lambda)) return PKV_ERR_INVALID_ARG;
+    if (!ref0->xF || !ref0->xC || (final && (!final->xF_next || !final->xC_next))) return PKV_ERR_INVALID_ARG;
+    std::vector<int> totals(n_layers, 0), maxbs(n_layers, 0);
+    for (int l = first; l < n_layers; ++l) {
+        if ((rc = check_compressed(c, &cb[l], &totals[l], &maxbs[l])) != PKV_OK) return rc;
+        if (!dW[l] || !w[l].Wq || !w[l].Wk || !w[l].Wv || !w[l].Wo || !w[l].Wgate || !w[l].Wup || !w[l].Wdown ||
+            !w[l].g_attn || !w[l].g_mlp || (D.L > 0 && (!full[l].K || !full[l].V)))
+            return PKV_ERR_INVALID_ARG;
+        for (int h = 0; h <= Hkv; ++h) c->host_lhead[(size_t)l * (Hkv + 1) + h] = cb[l].head_off[h];
+    }
+    cudaStream_t S = c->st, T = c->tstream;
+    Lc lcS{S, &c->launches, c->map_cache}, lcT{T, &c->launches, c->map_cache};
+    // set-up on the student stream: status words, kept-set offsets, chunk starts, RoPE table, dx0 = xF0 - xC0
+    cudaMemsetAsync(b.lstatus, 0, (size_t)n_layers * sizeof(DevStatus), S);
+    cudaMemcpyAsync(b.lhead_off + (size_t)first * (Hkv + 1), c->host_lhead + (size_t)first * (Hkv + 1),
+                    (size_t)(n_layers - first) * (Hkv + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, S);
+    upload_meta(c, cb[first].head_off, N, ref0->n_chunks, ref0->chunk_off);
+    rope_table(lcS, b.tok_cs, N, D.hd, ref0->pos0, D.rope_theta, b.rope_tab);
+    sub_f32(lcS, ref0->xF, ref0->xC, (int64_t)N * d, b.dxbuf[0]);
+    cudaEventRecord(c->evSetup, S);
+    cudaStreamWaitEvent(T, c->evSetup, 0);
+
+    const float* xF_in = ref0->xF;
+    const float* xC_in = ref0->xC;
+    for (int l = first; l < n_layers; ++l) {
+        const int k = l - first, slot = k & 1, pp = k & 1;
+        const bool last = (l == n_layers - 1);
+        DevStatus* st = b.lstatus + l;
+        const int32_t* hoff = b.lhead_off + (size_t)l * (Hkv + 1);
+        pkv::TcForwardArgs fa{};
+        fa.w = &w[l]; fa.full = &full[l];
+        fa.N = N; fa.pos0 = ref0->pos0; fa.max_b = maxbs[l]; fa.total_kept = totals[l];
+        fa.head_off = hoff; fa.tok_cs = b.tok_cs; fa.rope_tab = b.rope_tab;
+        fa.aF = b.ringA[slot]; fa.zF = b.ringZ[slot]; fa.hF = b.ringH[slot];
+        fa.aC = b.aC; fa.dA = b.a2 + (size_t)N * Dq;
+        fa.zC = b.zC; fa.dz = b.dz; fa.hC = b.hC; fa.R = b.R; fa.S_H = b.S_H; fa.S_T = b.S_T;
+        fa.status = st; fa.dual = c->dual; fa.kv_split = c->kv_split;
+        // ---- teacher half of block l on the teacher stream ----
+        if (k >= 2) cudaStreamWaitEvent(T, c->evStu[slot], 0);        // slot free: student of block l-2 is done
+        fa.xF = xF_in; fa.xC = xF_in;
+        float* xFn = (last && final) ? final->xF_next : b.ringX[slot];
+        rc = pkv::tc_teacher_forward(lcT, &b.tc, &c->dims, fa, xFn);
+        if (rc != PKV_OK) break;
+        cudaEventRecord(c->evTea[slot], T);
+        // ---- student half, statistics, solve, next student state on the caller's stream ----
+        const void *Kc, *Vc;
+        stage_compact(c, lcS, &full[l], &cb[l], totals[l], &Kc, &Vc, hoff, st);
+        fa.Kc = Kc; fa.Vc = Vc; fa.bias = cb[l].idx ? nullptr : cb[l].bias;
+        fa.xC = xC_in; fa.dx = b.dxbuf[pp];
+        cudaStreamWaitEvent(S, c->evTea[slot], 0);
+        rc = pkv::tc_student_forward(lcS, &b.tc, &c->dims, fa);
+        if (rc != PKV_OK) break;
+        if (c->dual) {
+            rc = pkv::tc_dual_solve(lcS, &b.tc, &c->dims, N, b.R, lambda, mode, dW[l], st);
+            if (rc != PKV_OK) break;
+            sumsq(lcS, dW[l], (int64_t)d * F, &st->dw_fro2);
+        } else {
+            solve_stage(c, lcS, b.S_H, b.S_T, lambda, mode, dW[l], true, st);
+        }
+        float* Dn = b.dxbuf[1 - pp];                                  // xF_next - xC_next = T - hC dW^T
+        pkv::tc_next_states(lcS, &b.tc, &c->dims, N, w[l].Wdown, dW[l], nullptr, b.R, nullptr, Dn, st);
+        sumsq(lcS, Dn, (int64_t)N * d, &st->res_fro2);
+        float* xCn = (last && final) ? final->xC_next : b.xs[2 + (1 - pp)];
+        sub_f32(lcS, xFn, Dn, (int64_t)N * d, xCn);
+        cudaEventRecord(c->evStu[slot], S);
+        xF_in = xFn;
+        xC_in = xCn;
+    }
+    // the last student waited for the last teacher; one copy of all status words, one synchronisation
+    cudaMemcpyAsync(c->host_lstatus, b.lstatus, (size_t)n_layers * sizeof(DevStatus), cudaMemcpyDeviceToHost, S);
+    cudaError_t e = cudaStreamSynchronize(S);
+    cudaError_t e2 = cudaStreamSynchronize(T);
+    if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronize");
+    if (e2 != cudaSuccess) return cuda_fail(c, e2, "teacher stream synchronize");
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(c, e, "kernel launch");
+    if (rc != PKV_OK) return rc;
+    int code = PKV_OK;
+    for (int l = first; l < n_layers; ++l) {
+        if (stats) fill_stats(c, c->host_lstatus[l], &stats[l], cb[l].head_off);
+        if (code == PKV_OK && c->host_lstatus[l].code != 0) code = c->host_lstatus[l].code;
+    }
+    return code;
+}
+
 extern "C" int pkv_build_stack(pkv_ctx* c, int n_layers, int first_layer, const pkv_block_weights* w,
                                const pkv_kv* full, const pkv_kv_compressed* cb, const pkv_ref* ref0, float lambda,
                                int lambda_mode, float* const* dW, const pkv_ref_next* final, pkv_stats* stats) {
     if (!c || !w || !full || !cb || !ref0 || !dW || n_layers <= 0 || first_layer < 0 || first_layer >= n_layers)
         return PKV_ERR_INVALID_ARG;
+    if (c->engine != PKV_ENGINE_SIMT && !c->timing && n_layers - first_layer >= 2 && n_layers <= kMaxStackLayers)
+        return build_stack_overlapped(c, n_layers, first_layer, w, full, cb, ref0, lambda, lambda_mode, dW, final, stats);
     pkv_ref ref = *ref0;
     for (int l = first_layer; l < n_layers; ++l) {
         int pp = (l - first_layer) & 1;

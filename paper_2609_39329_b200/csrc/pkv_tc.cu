@@ -118,13 +118,13 @@ __global__ void k_oproj_teacher(const float* __restrict__ xF, const float* __res
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) zF[i] = xF[i] + o[i];
 }
-// student half: dz = (xF - xC) + o[N:2N] (the projection of dA); zC = zF - dz
-__global__ void k_oproj_student(const float* __restrict__ xF, const float* __restrict__ xC,
-                                const float* __restrict__ o, const float* __restrict__ zF, size_t n,
-                                float* __restrict__ zC, float* __restrict__ dz) {
+// student half: dz = dx + o[N:2N] (dx = xF - xC entering the block, o[N:2N] the projection of dA); zC = zF - dz
+__global__ void k_oproj_student(const float* __restrict__ dx, const float* __restrict__ o,
+                                const float* __restrict__ zF, size_t n, float* __restrict__ zC,
+                                float* __restrict__ dz) {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    float dd = (xF[i] - xC[i]) + o[n + i];
+    float dd = dx[i] + o[n + i];
     dz[i] = dd;
     zC[i] = zF[i] - dd;
 }
@@ -442,7 +442,7 @@ int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     int rc;
     const size_t uo = (size_t)N * d;                   // offsets of the student rows
     Pair uS{t->u.hi + uo, t->u.lo + uo};
-    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.xF, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, N);
+    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.xC, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, N);
     lc.count();
     float* qkvS = t->qkv + (size_t)N * QKV;
     if ((rc = gemm_act_weight(lc, uS, d, w->Wq, d, qkvS, QKV, N, Dq, d, 1.f, nullptr, 0, st))) return rc;
@@ -458,11 +458,11 @@ int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     if ((rc = gemm_act_weight(lc, aS, Dq, w->Wo, Dq, t->o + uo, d, N, d, Dq, 1.f, nullptr, 0, st))) return rc;
     {
         size_t n = (size_t)N * d;
-        k_oproj_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(a.xF, a.xC, t->o, a.zF, n, a.zC, a.dz);
+        k_oproj_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(a.dx, t->o, a.zF, n, a.zC, a.dz);
         lc.count();
     }
     mark(a, lc, 4);
-    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.zF, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, N);
+    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.zC, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, N);
     lc.count();
     float* guS = t->gu + (size_t)N * 2 * F;
     if ((rc = gemm_act_weight(lc, uS, d, w->Wgate, d, guS, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;

@@ -118,6 +118,7 @@ struct TcForwardArgs {
     const int32_t* head_off; const int32_t* tok_cs; float* rope_tab;
     float *zF, *zC, *dz, *hF, *hC, *R, *S_H, *S_T, *aF, *aC, *dA;
     float* xF_next;     // optional: teacher state entering the next block
+    const float* dx;    // student half: xF - xC entering this block (state difference carried between blocks)
     float *part_m, *part_l, *part_O;
     int dual;           // 1: only the token-contiguous copy of the student features is prepared in S7
     DevStatus* status;

@@ -303,30 +303,52 @@ def test_reduced_config2_shape(B):
         check_build(B, cfg, lay, lay["x0"], lay["x0"], [0, cfg.N], 0.1, engine)
 
 
-def test_two_layer_stack_matches_oracle_chain(B):
+@pytest.mark.parametrize("nl,solver,hd", [(2, 0, 64), (5, 0, 128), (4, 1, 128)])
+def test_stack_matches_oracle_chain(B, nl, solver, hd):
+    """Free-running stack: GPU and oracle each propagate their own states through all blocks (the tensor-core
+    engine runs the teacher ahead on its own stream; five blocks exercise the reuse of its two-slot ring)."""
     import torch
-    cfg = small_cfg("bf16", n_layers=2, N=64)
-    lays = [H.make_problem(cfg, layer=l) for l in range(2)]
+    cfg = small_cfg("bf16", n_layers=nl, N=64, hd=hd, Hq=4 if hd == 128 else 8, Hkv=2)
+    lays = [H.make_problem(cfg, layer=l) for l in range(nl)]
     x0 = lays[0]["x0"]
     xF, xC = x0.astype(np.float64), x0.astype(np.float64)
     refs = []
-    for l in range(2):
+    for l in range(nl):
         o = H.run_oracle(cfg, lays[l], xF, xC, [0, cfg.N], 0.1)
         refs.append(o)
         xF, xC = o["xF_next"], o["xC_next"]
-    for engine in engines(B, cfg):
-        ctx = B.PkvContext(B.dims_from_config(cfg), engine=engine)
+    for engine in (engines(B, cfg) if solver == 0 else [B.ENGINE_AUTO]):
+        ctx = B.PkvContext(B.dims_from_config(cfg), engine=engine, solver=solver)
         dl = []
-        for l in range(2):
+        for l in range(nl):
             off, idx = gen.kept_to_csr(lays[l]["kept"])
             kv = B.to_device({"K": lays[l]["K"], "V": lays[l]["V"]}, cfg.dtype)
             dl.append({"w": B.to_device(lays[l]["weights"], cfg.dtype), "K": kv["K"], "V": kv["V"],
                        "head_off": off, "idx": torch.from_numpy(idx).cuda()})
         xt = torch.from_numpy(x0).cuda()
         out = ctx.build_stack(dl, xt, xt, [0, cfg.N], cfg.L, 0.1)
-        for l in range(2):
-            assert H.rel_fro(out["dW"][l].cpu().numpy(), refs[l]["dW"]) <= DW_TOL
-        assert H.rel_fro(out["xC_final"].cpu().numpy(), refs[1]["xC_next"]) <= 1e-3
+        for l in range(nl):
+            assert H.rel_fro(out["dW"][l].cpu().numpy(), refs[l]["dW"]) <= DW_TOL, l
+            np.testing.assert_allclose(out["stats"][l]["lambda_eff"], refs[l]["lam"], rtol=5e-3)
+        assert H.rel_fro(out["xC_final"].cpu().numpy(), refs[-1]["xC_next"]) <= 2e-3
+        assert H.rel_fro(out["xF_final"].cpu().numpy(), refs[-1]["xF_next"]) <= 2e-3
+        # resuming from a later block with the states of the block before gives the same patches
+        if nl >= 4 and engine == B.ENGINE_AUTO:
+            mid = 2
+            xFm = torch.from_numpy(refs[mid - 1]["xF_next"].astype(np.float32)).cuda()
+            xCm = torch.from_numpy(refs[mid - 1]["xC_next"].astype(np.float32)).cuda()
+            out2 = ctx.build_stack(dl, xFm, xCm, [0, cfg.N], cfg.L, 0.1, first_layer=mid)
+            for l in range(mid, nl):
+                assert H.rel_fro(out2["dW"][l].cpu().numpy(), refs[l]["dW"]) <= DW_TOL, l
+        # an invalid kept set in a later block is reported with its position
+        if engine == B.ENGINE_AUTO and solver == 0:
+            bad = dict(dl[-1])
+            bi = dl[-1]["idx"].clone()
+            bi[3] = bi[2]
+            bad["idx"] = bi
+            with pytest.raises(B.PkvError) as ei:
+                ctx.build_stack(dl[:-1] + [bad], xt, xt, [0, cfg.N], cfg.L, 0.1)
+            assert ei.value.code == -3
         ctx.close()
 
 
