@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a pipeline primitives used by the tensor-core kernels:
-// mbarrier, TMA (cp.async.bulk.tensor, no cluster multicast anywhere), tcgen05 (TMEM alloc,
+// mbarrier, TMA (cp.async.bulk.tensor, every load lands in the issuing CTA only), tcgen05 (TMEM alloc,
 // MMA, commit, ld) and the shared-memory / instruction descriptors of the 5th-gen tensor cores.
 //
 // Every wait is bounded: after kWaitCycles the waiter raises PKV_ERR_TIMEOUT in the device

@@ -318,6 +318,55 @@ def test_chunks_are_independent_and_restart_positions():
     np.testing.assert_allclose(both["z"][5:], second["z"], rtol=1e-12, atol=1e-13)
 
 
+def test_greedy_chain_over_blocks_matches_running_the_patched_model():
+    """Algorithm 1 over blocks: feeding each block the states the block below produced must equal
+    (a) for the teacher, the unpatched model run on the full caches, whatever was kept or patched;
+    (b) for the student, the model with every patch merged so far run on the compressed caches."""
+    cfg = tiny_cfg()
+    nl, chunks = 3, [0, 7, 12]
+    blocks = [tiny_problem(cfg, seed=10 + l) for l in range(nl)]
+    x0 = blocks[0][3]
+
+    def chain(kept_of, lam0):
+        xF, xC, outs = x0, x0, []
+        for l, (w, K, V, _, kept) in enumerate(blocks):
+            o = orc.build_patch(w, K, V, kept_of(l, kept), xF, xC, chunks, cfg.L, lam0, cfg)
+            outs.append(o)
+            xF, xC = o["xF_next"], o["xC_next"]
+        return xF, xC, outs
+
+    xF, xC, outs = chain(lambda l, k: k, 0.05)
+    # (a) teacher: plain forward through the unpatched blocks
+    t = x0
+    for w, K, V, _, _ in blocks:
+        f = orc.block_forward(t, w, list(K), list(V), chunks, cfg.L, cfg)
+        t = f["z"] + f["h"] @ w["Wdown"].T
+    np.testing.assert_allclose(xF, t, rtol=1e-11, atol=1e-12)
+    # ... and it does not depend on the kept sets or on lambda
+    xF2, xC2, _ = chain(lambda l, k: [k[0][:3], k[1][2:]], 0.7)
+    np.testing.assert_allclose(xF2, xF, rtol=1e-12, atol=1e-13)
+    assert np.linalg.norm(xC2 - xC) > 1e-3 * np.linalg.norm(xC)
+    # (b) student: forward through the patched blocks on the compressed caches
+    s = x0
+    for (w, K, V, _, kept), o in zip(blocks, outs):
+        Kc, Vc = orc.gather_cache(K, V, kept)
+        f = orc.block_forward(s, w, Kc, Vc, chunks, cfg.L, cfg)
+        s = f["z"] + f["h"] @ (w["Wdown"] + o["dW"]).T
+    np.testing.assert_allclose(xC, s, rtol=1e-9, atol=1e-10)
+    # the patched student ends closer to the teacher than the unpatched one
+    u = x0
+    for w, K, V, _, kept in blocks:
+        Kc, Vc = orc.gather_cache(K, V, kept)
+        f = orc.block_forward(u, w, Kc, Vc, chunks, cfg.L, cfg)
+        u = f["z"] + f["h"] @ w["Wdown"].T
+    assert np.linalg.norm(xF - xC) < np.linalg.norm(xF - u)
+    # full caches in every block: every patch is exactly zero and the streams never part
+    full = [np.arange(cfg.L, dtype=np.int32)] * cfg.Hkv
+    xF3, xC3, outs3 = chain(lambda l, k: full, 0.05)
+    assert all(np.all(o["dW"] == 0.0) for o in outs3)
+    np.testing.assert_array_equal(xF3, xC3)
+
+
 def test_build_patch_rejects_bad_index_sets():
     cfg = tiny_cfg()
     w, K, V, x, kept = tiny_problem(cfg)
