@@ -24,6 +24,7 @@ force on tiny inputs, textbook routines that take another route (QR least square
 augmented system, the dual N x N form, eigenvalues) and the invariants Eq. 4-9 imply.
 The RoPE / norm conventions and the input generators are our own definitions: nothing in
 the paper pins them ("parity unpinned" for those conventions only).
+``low_rank_patch`` (appendix variant) has no CUDA counterpart yet; it is pinned like the rest.
 """
 from __future__ import annotations
 
@@ -189,6 +190,26 @@ def ridge_solve(S_H: np.ndarray, S_T: np.ndarray, lam: float) -> np.ndarray:
     Y = scipy.linalg.solve_triangular(Lc, f64(S_T).T, lower=True)      # Lc Y = S_T^T
     X = scipy.linalg.solve_triangular(Lc.T, Y, lower=False)            # Lc^T X = Y
     return np.ascontiguousarray(X.T)
+
+
+def low_rank_patch(dW: np.ndarray, S_H: np.ndarray, r: int):
+    """Rank-r patch (appendix, low-rank weight patches): with M = dW S_H dW^T  [d][d] and U_r its r
+    leading eigenvectors, dW_r = U_r (U_r^T dW).  Returns (U_r [d][r], B_r = U_r^T dW [r][F],
+    dW_r [d][F], all eigenvalues of M in descending order).  Storage of the factored form is
+    (d + F) r numbers.  Eigenvector signs are arbitrary; dW_r is unique when the r-th and (r+1)-th
+    eigenvalues differ."""
+    dW = f64(dW)
+    d = dW.shape[0]
+    if not (0 <= r <= d):
+        raise ValueError("rank must lie in [0, d]")
+    M = dW @ f64(S_H) @ dW.T
+    M = 0.5 * (M + M.T)
+    evals, evecs = np.linalg.eigh(M)                            # ascending
+    order = np.argsort(evals)[::-1]
+    evals, evecs = evals[order], evecs[:, order]
+    U = np.ascontiguousarray(evecs[:, :r])
+    B = U.T @ dW
+    return U, B, U @ B, evals
 
 
 def round_bf16(a: np.ndarray) -> np.ndarray:

@@ -265,6 +265,52 @@ def test_adaptive_lambda_is_weighted_eigenvalue_mean():
         orc.ridge_lambda(np.zeros((3, 3)), 0.1)
 
 
+def test_low_rank_patch_is_the_reduced_rank_regression_optimum():
+    """Appendix, low-rank patches.  On the reference set the loss of a patch B against the ridge
+    patch is ||H'(dW - B)^T||_F^2 = ||(dW - B) S_H^{1/2}||_F^2, so the best rank-r B is the
+    truncated SVD of dW S_H^{1/2} mapped back (Eckart-Young) -- a route that never forms the
+    d x d eigenproblem the method uses."""
+    r0 = np.random.default_rng(21)
+    N, F, d, r = 40, 14, 9, 3
+    H = r0.standard_normal((N, F)) * (0.2 + r0.random(F))
+    T = r0.standard_normal((N, d)) + H @ r0.standard_normal((F, d))
+    S_H, S_T = H.T @ H, T.T @ H
+    dW = orc.ridge_solve(S_H, S_T, 0.3)
+    U, B, dWr, ev = orc.low_rank_patch(dW, S_H, r)
+    assert U.shape == (d, r) and B.shape == (r, F) and dWr.shape == (d, F)
+    np.testing.assert_allclose(U.T @ U, np.eye(r), atol=1e-12)
+    assert np.linalg.matrix_rank(dWr, tol=1e-9) == r
+    # other route: symmetric square root by eigen-decomposition of S_H, SVD, truncate, map back
+    w, Q = np.linalg.eigh(S_H)
+    root, iroot = (Q * np.sqrt(w)) @ Q.T, (Q / np.sqrt(w)) @ Q.T
+    Us, sv, Vt = np.linalg.svd(dW @ root, full_matrices=False)
+    want = (Us[:, :r] * sv[:r]) @ Vt[:r] @ iroot
+    np.testing.assert_allclose(dWr, want, rtol=1e-8, atol=1e-10)
+    np.testing.assert_allclose(ev[:d], sv ** 2, rtol=1e-9, atol=1e-10)
+    # what the truncation costs on the reference set is the discarded eigenvalues
+    loss = np.linalg.norm(H @ (dW - dWr).T) ** 2
+    np.testing.assert_allclose(loss, ev[r:].sum(), rtol=1e-9)
+    # no random rank-r competitor, nor a plain (unweighted) truncated SVD of dW, does better
+    for _ in range(200):
+        C = dWr + 0.05 * r0.standard_normal((d, r)) @ r0.standard_normal((r, F))
+        A = r0.standard_normal((d, r)) @ r0.standard_normal((r, F))
+        assert np.linalg.norm(H @ (dW - A).T) ** 2 >= loss
+        if np.linalg.matrix_rank(C, tol=1e-9) <= r:
+            assert np.linalg.norm(H @ (dW - C).T) ** 2 >= loss * (1 - 1e-12)
+    Up, sp, Vp = np.linalg.svd(dW, full_matrices=False)
+    plain = (Up[:, :r] * sp[:r]) @ Vp[:r]
+    assert np.linalg.norm(H @ (dW - plain).T) ** 2 > loss
+    # limits: full rank returns the ridge patch, rank 0 the zero patch; the projector is idempotent
+    np.testing.assert_allclose(orc.low_rank_patch(dW, S_H, d)[2], dW, rtol=1e-10, atol=1e-12)
+    assert np.all(orc.low_rank_patch(dW, S_H, 0)[2] == 0.0)
+    np.testing.assert_allclose(orc.low_rank_patch(dWr, S_H, r)[2], dWr, rtol=1e-8, atol=1e-11)
+    # a patch that already has rank r is returned unchanged
+    low = r0.standard_normal((d, r)) @ r0.standard_normal((r, F))
+    np.testing.assert_allclose(orc.low_rank_patch(low, S_H, r)[2], low, rtol=1e-8, atol=1e-10)
+    with pytest.raises(ValueError):
+        orc.low_rank_patch(dW, S_H, d + 1)
+
+
 # ------------------------------------------------------------------ block identities ---
 
 def test_identical_caches_give_zero_target_and_zero_patch():
