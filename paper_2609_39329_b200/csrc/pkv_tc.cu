@@ -51,22 +51,6 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const float* __restrict__
     }
 }
 
-__global__ void __launch_bounds__(256) k_split(const float* __restrict__ a, size_t n, __nv_bfloat16* __restrict__ hi,
-                                               __nv_bfloat16* __restrict__ lo) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    __nv_bfloat16 h, l;
-    split2(a[i], h, l);
-    hi[i] = h;
-    lo[i] = l;
-}
-
-static void split(const Lc& lc, const float* a, size_t n, Pair p) {
-    if (!n) return;
-    k_split<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(a, n, p.hi, p.lo);
-    lc.count();
-}
-
 __device__ __forceinline__ float silu_f(float t) { return t / (1.0f + expf(-t)); }
 
 // gu [2N][2F] (gate | up) -> hF, hC (fp32 + pairs), dh = hF - hC (pair)

@@ -46,7 +46,6 @@ struct alignas(64) GemmTcParams {
 
 constexpr int kGemmMaxStages = 6;
 constexpr int kGemmBarBytes = (2 * kGemmMaxStages + 1) * 8 + 16;
-constexpr int kGemmStagingBytes = 4 * 32 * 33 * 4;     // aliases the first pipeline stage (free once the MMAs are done)
 
 // One k-tile stage holds every distinct operand tile once: nA x [128][64] and nB x [BN][64] bf16,
 // and all passes are issued from it (the shared operand of a split product is not re-read).
