@@ -183,7 +183,15 @@ int pkv_merge(void* W, int w_dtype, const float* dW, int64_t count, void* cuda_s
  * blocks below it already patched in the student (greedy construction, Sec. 2.2).  Arrays are
  * HOST arrays of n_layers entries.  x0F/x0C enter block first_layer; states are carried in
  * fp32 inside the context.  dW[l]: device fp32 [d][F].  stats: NULL or n_layers entries.
- * final: optional states leaving the last block. */
+ * final: optional states leaving the last block.
+ * Scheduling: the teacher of Algorithm 1 never sees a patch, so with the tensor-core engine, two or
+ * more blocks, at most 128 layers and stage timing off, the teacher half of up to two later blocks
+ * runs on a second stream owned by the context, beside the student half and the solve of the
+ * current block; results are the same as block-by-block calls up to rounding order.  That stream is
+ * ordered after the work already queued on the context's stream and is drained before the call
+ * returns; the call returns after one synchronisation.  In this mode stage_ms stays zero.  With
+ * stage timing on, with the SIMT engine or for a single block the blocks run strictly in sequence.
+ * Errors: the status of the first failing block is returned; stats[l].err_info locates it. */
 int pkv_build_stack(pkv_ctx* ctx, int n_layers, int first_layer, const pkv_block_weights* w,
                     const pkv_kv* full, const pkv_kv_compressed* cb, const pkv_ref* ref0,
                     float lambda, int lambda_mode, float* const* dW, const pkv_ref_next* final,
