@@ -35,3 +35,34 @@ def test_binding_structs_match_header_sizes_and_strerror():
     d.hd = 96
     assert L.pkv_workspace_bytes(ctypes.byref(d), ctypes.byref(o)) == 0
     assert L.pkv_merge(None, 0, None, 0, None) == -1
+
+
+def test_workspace_of_every_benchmark_config_fits_one_gpu_beside_its_inputs():
+    """Host arithmetic only: the context's workspace plus the tensors one block keeps resident (weights,
+    full cache, kept indices, states, patch) stays far below 180 GB for all five configs, for both engines
+    and both solvers, and grows with the reference-token capacity."""
+    from paper_2609_39329_b200 import binding as B
+    from paper_2609_39329_b200 import inputs as gen
+    L = B.lib()
+    L.pkv_workspace_bytes.restype = ctypes.c_size_t
+    for cid in range(1, 6):
+        cfg = gen.benchmark_config(cid)
+        eb = 4 if cfg.dtype == "fp32" else 2
+        resident = eb * (cfg.d * (2 * cfg.Dq + 2 * cfg.Dkv) + 3 * cfg.d * cfg.F) + eb * 2 * cfg.Hkv * cfg.L * cfg.hd \
+            + 4 * cfg.Hkv * cfg.budget + 4 * (4 * cfg.N * cfg.d + cfg.d * cfg.F)
+        sizes = {}
+        for engine in (B.ENGINE_AUTO, B.ENGINE_SIMT):
+            for solver in (B.SOLVER_PRIMAL, B.SOLVER_DUAL):
+                if solver == B.SOLVER_DUAL and (engine == B.ENGINE_SIMT or cfg.dtype == "fp32"):
+                    continue
+                d = B.dims_from_config(cfg)
+                o = B.pkv_opts(engine, 0, None, 0, solver)
+                ws = L.pkv_workspace_bytes(ctypes.byref(d), ctypes.byref(o))
+                assert ws > 0, (cid, engine, solver)
+                assert ws % 256 == 0
+                assert ws + resident < 40e9, (cid, engine, solver, ws)
+                sizes[(engine, solver)] = ws
+                d2 = B.dims_from_config(cfg, N_max=2 * cfg.N)
+                assert L.pkv_workspace_bytes(ctypes.byref(d2), ctypes.byref(o)) > ws
+        if cfg.dtype == "bf16":
+            assert sizes[(B.ENGINE_AUTO, B.SOLVER_PRIMAL)] > sizes[(B.ENGINE_SIMT, B.SOLVER_PRIMAL)]
