@@ -161,6 +161,70 @@ def test_empty_cache_and_first_token_sees_only_itself():
             np.testing.assert_allclose(a[s, h], v[s, h // 2], rtol=1e-13)
 
 
+def test_finite_key_bias_is_added_unscaled_to_cached_logits_only():
+    """Approximation-style caches carry one additive logit term per cached key (Sec. 3.1).  A literal
+    per-key loop fixes where it enters: after the 1/sqrt(hd) scaling, on cache keys only, never on the
+    chunk's own keys."""
+    q, k, v, Kc, Vc = rand_attn_inputs(seed=3, rows=(9, 5))
+    r = np.random.default_rng(7)
+    bias = [r.uniform(-2.0, 2.0, len(K)) for K in Kc]
+    n, Hq, hd = q.shape
+    for chunks in ([0, 7], [0, 3, 7]):
+        a = orc.attention(q, k, v, Kc, Vc, chunks, key_bias=bias).reshape(q.shape)
+        for c in range(len(chunks) - 1):
+            s, e = chunks[c], chunks[c + 1]
+            for i in range(s, e):
+                for h in range(Hq):
+                    kh = h // 2
+                    lg = [sum(q[i, h, t] * Kc[kh][j][t] for t in range(hd)) / math.sqrt(hd) + bias[kh][j]
+                          for j in range(len(Kc[kh]))]
+                    lg += [sum(q[i, h, t] * k[j, kh, t] for t in range(hd)) / math.sqrt(hd) for j in range(s, i + 1)]
+                    vals = [Vc[kh][j] for j in range(len(Vc[kh]))] + [v[j, kh] for j in range(s, i + 1)]
+                    mx = max(lg)
+                    ex = [math.exp(x - mx) for x in lg]
+                    want = sum(w_ * val for w_, val in zip(ex, vals)) / sum(ex)
+                    np.testing.assert_allclose(a[i, h], want, rtol=1e-12, atol=1e-13)
+    assert not np.allclose(a, orc.attention(q, k, v, Kc, Vc, chunks).reshape(q.shape))
+
+
+def test_finite_key_bias_closed_form_with_equal_keys():
+    """All keys equal: a cached key with bias beta weighs e^beta, a chunk key weighs 1, whatever hd is
+    (a bias multiplied by 1/sqrt(hd), or applied to the chunk keys too, fails this)."""
+    q, k, v, Kc, Vc = rand_attn_inputs(seed=4, hd=16, rows=(6, 6))
+    one = np.ones(q.shape[2])
+    Kc = [np.tile(one, (6, 1)) for _ in range(2)]
+    k = np.tile(one, (q.shape[0], 2, 1))
+    beta = [np.array([0.0, 1.0, -1.0, 2.0, 0.5, -0.5]), np.array([3.0, 0.0, 0.0, -2.0, 1.5, 0.25])]
+    a = orc.attention(q, k, v, Kc, Vc, [0, q.shape[0]], key_bias=beta).reshape(q.shape)
+    for i in range(q.shape[0]):
+        for h in range(q.shape[1]):
+            kh = h // 2
+            wgt = np.exp(beta[kh])
+            want = (wgt @ Vc[kh] + v[:i + 1, kh].sum(0)) / (wgt.sum() + i + 1)
+            np.testing.assert_allclose(a[i, h], want, rtol=1e-12)
+
+
+def test_prefill_cache_then_cached_forward_equals_one_causal_pass():
+    """prefill_kv pins: the cache it builds from context rows, attended to by reference tokens at
+    positions L.., gives what one causal pass over [context; reference] gives on the reference rows."""
+    cfg = tiny_cfg(L=19, N=6)
+    w, _, _, x, _ = tiny_problem(cfg, seed=9)
+    r = np.random.default_rng(10)
+    ctx = r.standard_normal((cfg.L, cfg.d))
+    K, V, q_ctx = orc.prefill_kv(ctx, w, cfg)
+    assert K.shape == (cfg.Hkv, cfg.L, cfg.hd) and V.shape == K.shape and q_ctx.shape == (cfg.L, cfg.Hq, cfg.hd)
+    cached = orc.block_forward(x, w, list(K), list(V), [0, cfg.N], cfg.L, cfg)
+    empty = [np.zeros((0, cfg.hd))] * cfg.Hkv
+    whole = orc.block_forward(np.concatenate([ctx, x]), w, empty, empty, [0, cfg.L + cfg.N], 0, cfg)
+    np.testing.assert_allclose(cached["a"], whole["a"][cfg.L:], rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(cached["h"], whole["h"][cfg.L:], rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(q_ctx, whole["q"][:cfg.L], rtol=1e-12, atol=1e-13)
+    # a context row moved to another position changes the result: positions matter
+    K2, V2, _ = orc.prefill_kv(ctx[::-1].copy(), w, cfg)
+    assert not np.allclose(orc.block_forward(x, w, list(K2[:, ::-1]), list(V2[:, ::-1]), [0, cfg.N], cfg.L, cfg)["a"],
+                           cached["a"])
+
+
 # ------------------------------------------------------------------ backbone conventions
 
 def test_rope_is_a_rotation_and_relative():
