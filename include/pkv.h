@@ -245,6 +245,17 @@ int pkv_gram_noalloc(const float* X, const float* R, int32_t n, int32_t F, int32
 int pkv_ridge_solve(pkv_ctx* ctx, const float* S_H, const float* S_T, float lambda, int lambda_mode,
                     float* dW, pkv_stats* stats);
 
+/* The product the ridge solve is built from (Eq. 8 needs fp32 accuracy; the tensor cores take bf16): C [M][N]
+ * (+)= alpha * A B^T with A [M][K], B [N][K], C device fp32 row-major, 16-byte aligned.  Each operand is split
+ * into bf16 parts (hi, mid, lo) and multiplied in `passes` passes accumulating in fp32: 6 = fp32-equivalent
+ * (triples), 3 = pairs (about 16 mantissa bits).  accumulate != 0 adds to C.  accumulators = 1, 2 or 4 tensor-
+ * memory accumulators per tile: the tensor core truncates when it adds to an accumulator, so the large hi x hi
+ * pass is kept apart from the cross terms (2) and split in three (4), the parts being added with round to
+ * nearest; the solve uses 4 in its factorisation.  Exported for unit parity tests; tensor-core engine only;
+ * M*K and N*K (K rounded up to 8) must not exceed d*F of the context. */
+int pkv_fp32_product(pkv_ctx* ctx, const float* A, const float* B, int32_t M, int32_t N, int32_t K, float alpha,
+                     float* C, int accumulate, int passes, int accumulators);
+
 /* Failure-detection self-test: launches one CTA whose pipeline wait is on a barrier that nothing ever
  * completes, with a short limit (about a millisecond).  The wait must give up, raise the device status
  * word and let the CTA exit; the call then returns PKV_ERR_TIMEOUT (err site in *site if not NULL) and

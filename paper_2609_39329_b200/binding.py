@@ -118,6 +118,9 @@ def lib() -> C.CDLL:
                                    C.c_int, C.c_void_p]
     L.pkv_ridge_solve.restype = C.c_int
     L.pkv_ridge_solve.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_void_p, P(pkv_stats)]
+    L.pkv_fp32_product.restype = C.c_int
+    L.pkv_fp32_product.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float,
+                                   C.c_void_p, C.c_int, C.c_int, C.c_int]
     L.pkv_selftest_bounded_wait.restype = C.c_int
     L.pkv_selftest_bounded_wait.argtypes = [C.c_void_p, P(C.c_int32)]
     L.pkv_set_timing.restype = C.c_int
@@ -325,6 +328,19 @@ class PkvContext:
         if rc != 0:
             self._raise(rc)
         return S_H, S_T
+
+    def fp32_product(self, A, Bm, alpha=1.0, C_out=None, accumulate=False, passes=6, accumulators=4):
+        """pkv_fp32_product: C (+)= alpha * A Bm^T through the split-bf16 tensor-core product of the solve."""
+        torch = self.torch
+        M, K = int(A.shape[0]), int(A.shape[1])
+        N = int(Bm.shape[0])
+        if C_out is None:
+            C_out = torch.zeros((M, N), dtype=torch.float32, device=A.device)
+        rc = self.L.pkv_fp32_product(self.h, _ptr(A), _ptr(Bm), M, N, K, float(alpha), _ptr(C_out),
+                                     1 if accumulate else 0, int(passes), int(accumulators))
+        if rc != 0:
+            self._raise(rc)
+        return C_out
 
     def ridge_solve(self, S_H, S_T, lam, mode=LAMBDA_PAPER):
         torch = self.torch

@@ -520,25 +520,25 @@ static void gram_simt(pkv_ctx* c, const Lc& lc, const float* X, const float* R, 
 static void solve_stage(pkv_ctx* c, const Lc& lc, float* S_H, const float* S_T, float lam0, int mode, float* dW,
                         bool S_H_scratch, DevStatus* status = nullptr) {
     const int F = c->dims.F, d = c->dims.d;
-    Buffers bl = c->b;
-    if (status) bl.status = status;
-    Buffers& b = bl;
+    Buffers& b = c->b;                 // the context's own buffers: the solver keeps state in b.tc
+    DevStatus* st = status ? status : b.status;
     // the tensor-core build leaves only the lower triangle of its own S_H
-    trace_fro2(lc, S_H, F, b.status, 0, S_H_scratch && c->engine != PKV_ENGINE_SIMT);
+    trace_fro2(lc, S_H, F, st, 0, S_H_scratch && c->engine != PKV_ENGINE_SIMT);
     if (c->engine == PKV_ENGINE_SIMT) {
-        make_ridge_matrix(lc, S_H, F, lam0, mode, b.solve.G, b.status);
+        make_ridge_matrix(lc, S_H, F, lam0, mode, b.solve.G, st);
         cudaMemcpyAsync(b.solve.Y, S_T, (size_t)d * F * sizeof(float), cudaMemcpyDeviceToDevice, c->st);
-        ridge_solve_simt(lc, b.solve, F, d, dW, b.status);
+        ridge_solve_simt(lc, b.solve, F, d, dW, st);
     } else {
-        ridge_lambda(lc, F, lam0, mode, b.status);
+        ridge_lambda(lc, F, lam0, mode, st);
         float* S = S_H;
         if (!S_H_scratch) {
             cudaMemcpyAsync(b.solve.G, S_H, (size_t)F * F * sizeof(float), cudaMemcpyDeviceToDevice, c->st);
             S = b.solve.G;
+            b.tc.S3_ready = 0;         // the caller's S_T, not the one a build's statistics left split in place
         }
-        pkv::tc_ridge_solve(lc, &b.tc, S, S_T, F, d, dW, lam0, mode, b.status);
+        pkv::tc_ridge_solve(lc, &b.tc, S, S_T, F, d, dW, lam0, mode, st);
     }
-    sumsq(lc, dW, (int64_t)d * F, &b.status->dw_fro2);
+    sumsq(lc, dW, (int64_t)d * F, &st->dw_fro2);
 }
 
 static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv* full,
@@ -621,6 +621,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         fa.xF_next = next ? next->xF_next : nullptr;
         fa.kv_split = c->kv_split;
         fa.dual = c->dual;
+        fa.precise_stats = pkv::tc_well_conditioned(lambda, mode) ? 0 : 1;
         fa.part_m = b.part_m; fa.part_l = b.part_l; fa.part_O = b.part_O;
         fa.ev = c->timing ? c->ev : nullptr;
         fa.evT = nullptr;
@@ -739,6 +740,7 @@ static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv
         fa.aC = b.aC; fa.dA = b.a2 + (size_t)N * Dq;
         fa.zC = b.zC; fa.dz = b.dz; fa.hC = b.hC; fa.R = b.R; fa.S_H = b.S_H; fa.S_T = b.S_T;
         fa.status = st; fa.dual = c->dual; fa.kv_split = c->kv_split;
+        fa.precise_stats = pkv::tc_well_conditioned(lambda, mode) ? 0 : 1;
         // ---- teacher half of block l on the teacher stream ----
         if (k >= 2) cudaStreamWaitEvent(T, c->evStu[slot], 0);        // slot free: student of block l-2 is done
         fa.xF = xF_in; fa.xC = xF_in;
@@ -875,6 +877,20 @@ extern "C" int pkv_gram(pkv_ctx* c, const float* X, const float* R, int32_t n, f
         gram_simt(c, lc, X, R, n, S_H, S_T, accumulate != 0);
     else
         pkv::tc_gram(lc, &c->b.tc, &c->dims, X, R, n, S_H, S_T, accumulate != 0, c->b.status);
+    return end_call(c, nullptr, nullptr);
+}
+
+extern "C" int pkv_fp32_product(pkv_ctx* c, const float* A, const float* B, int32_t M, int32_t N, int32_t K, float alpha,
+                                float* C, int accumulate, int passes, int accumulators) {
+    if (!c || !A || !B || !C || M <= 0 || N <= 0 || K <= 0) return PKV_ERR_INVALID_ARG;
+    if (c->engine == PKV_ENGINE_SIMT) return PKV_ERR_UNSUPPORTED;
+    if (((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) return PKV_ERR_INVALID_ARG;
+    Lc lc{c->st, &c->launches, c->map_cache};
+    begin_call(c);
+    c->b.tc.S3_ready = 0;              // the operand buffers of the solver are used as scratch
+    int rc = pkv::tc_fp32_product(lc, &c->b.tc.solve, (size_t)c->dims.d * c->dims.F, A, B, M, N, K, alpha, C,
+                                  accumulate != 0, passes, accumulators, c->b.status);
+    if (rc != PKV_OK) return rc;
     return end_call(c, nullptr, nullptr);
 }
 

@@ -21,6 +21,23 @@ struct DevStatus {
     float min_pivot;
 };
 
+// Kernel attributes (the opt-in to more than 48 KB of dynamic shared memory) belong to the function as
+// loaded on ONE device: a launcher keeps one flag per device ordinal and sets the attribute the first
+// time it runs with that device current.  Two host threads racing on a flag both set the attribute, which
+// is harmless.
+constexpr int kMaxDeviceOrdinals = 64;
+struct PerDeviceOnce {
+    bool done[kMaxDeviceOrdinals] = {};
+    // true when the caller still has to do its once-per-device work; dev gets the current ordinal
+    bool needed(int* dev) {
+        int d = 0;
+        if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDeviceOrdinals) { *dev = -1; return true; }
+        *dev = d;
+        return !done[d];
+    }
+    void mark(int dev) { if (dev >= 0) done[dev] = true; }
+};
+
 // Every launcher takes the stream and a launch counter.
 struct Lc {
     cudaStream_t st;

@@ -1,9 +1,8 @@
 // pkv_gram_noalloc: the sufficient statistics of Eq. 9 for callers that must not allocate.
 //
 // Some hosts of this library cannot call cudaMalloc at the point where they need the statistics:
-// code running between cudaStreamBeginCapture and EndCapture, a plug-in inside a serving engine
-// that owns every byte of device memory through its own pool, or a latency-critical loop where an
-// allocation (an implicit device synchronisation) is not acceptable.  pkv_gram needs a context, and a
+// a plug-in inside a serving engine that owns every byte of device memory through its own pool, or a
+// latency-critical loop where an allocation (an implicit device synchronisation) is not acceptable.  pkv_gram needs a context, and a
 // context allocates its workspace.  This variant keeps the scratch the kernels need — the
 // token-contiguous bf16 hi/lo copies of X and R and the device status word — in a fixed array that is
 // part of the library image, so it needs neither a context nor any allocation.
@@ -59,11 +58,10 @@ extern "C" int pkv_gram_noalloc(const float* X, const float* R, int32_t n, int32
     for (const void* q : ptrs)
         if ((uintptr_t)q & 15) return PKV_ERR_INVALID_ARG;
     int dev = 0;
-    cudaDeviceProp prop;
     if (cudaGetDevice(&dev) != cudaSuccess) return PKV_ERR_CUDA;
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return PKV_ERR_CUDA;
-    (void)prop;
+    const cudaError_t before = cudaPeekAtLastError();      // an error the caller already carries is not this call's
     if (major != 10 || !tc_encode_available()) return PKV_ERR_UNSUPPORTED;
     unsigned char* base = nullptr;
     int rc = setup_device(dev, &base);
@@ -84,6 +82,7 @@ extern "C" int pkv_gram_noalloc(const float* X, const float* R, int32_t n, int32
     DevStatus host;      // plain host memory: the copy below is synchronous with respect to the host
     if (cudaMemcpyAsync(&host, status, sizeof(DevStatus), cudaMemcpyDeviceToHost, st) != cudaSuccess) return PKV_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return PKV_ERR_CUDA;
-    if (cudaGetLastError() != cudaSuccess) return PKV_ERR_CUDA;
+    const cudaError_t after = cudaPeekAtLastError();
+    if (after != cudaSuccess && after != before) return PKV_ERR_CUDA;
     return host.code;
 }

@@ -114,7 +114,8 @@ __global__ void k_oproj_student(const float* __restrict__ dx, const float* __res
 }
 
 // in [rows][cols] fp32 -> out pair [cols][ldo] (token-contiguous operands of the statistics)
-__global__ void k_transpose_split(const float* __restrict__ in, int rows, int cols, int ldo, Pair out) {
+__global__ void k_transpose_split(const float* __restrict__ in, int rows, int cols, int ldo, Pair out,
+                                  __nv_bfloat16* __restrict__ out3) {
     __shared__ float t[32][33];
     int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
     for (int j = threadIdx.y; j < 32; j += 8) {
@@ -126,16 +127,20 @@ __global__ void k_transpose_split(const float* __restrict__ in, int rows, int co
         int c = c0 + j, r = r0 + threadIdx.x;
         if (r < rows && c < cols) {
             __nv_bfloat16 h, l;
-            split2(t[threadIdx.x][j], h, l);
+            const float v = t[threadIdx.x][j];
+            split2(v, h, l);
             out.hi[(size_t)c * ldo + r] = h;
             out.lo[(size_t)c * ldo + r] = l;
+            if (out3) out3[(size_t)c * ldo + r] = __float2bfloat16_rn((v - __bfloat162float(h)) - __bfloat162float(l));
         }
     }
 }
 
-static void transpose_split(const Lc& lc, const float* in, int rows, int cols, int ldo, Pair out) {
+// out3 != nullptr: also the third bf16 part (triples, 24 mantissa bits)
+static void transpose_split(const Lc& lc, const float* in, int rows, int cols, int ldo, Pair out,
+                            __nv_bfloat16* out3 = nullptr) {
     dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
-    k_transpose_split<<<grid, block, 0, lc.st>>>(in, rows, cols, ldo, out);
+    k_transpose_split<<<grid, block, 0, lc.st>>>(in, rows, cols, ldo, out, out3);
     lc.count();
 }
 
@@ -213,6 +218,8 @@ size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d, int dua
     t->dh = c.pair(N * F);
     t->XT = c.pair(F * (size_t)t->ldT);
     t->RT = c.pair(dm * (size_t)t->ldT);
+    t->XT3 = c.take<__nv_bfloat16>(F * (size_t)t->ldT);
+    t->RT3 = c.take<__nv_bfloat16>(dm * (size_t)t->ldT);
     t->dW = c.pair(dm * F);
     t->qkv = c.take<float>(2 * N * (Dq + 2 * Dkv));
     t->o = c.take<float>(2 * N * dm);
@@ -285,7 +292,7 @@ int tc_dual_solve(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const fl
     // tr(X X^T) = tr(X^T X) and ||X X^T||_F = ||X^T X||_F: the ridge scale of Eq. 7 is the same number
     trace_fro2(lc, t->Gd, N, status, ldn);
     ridge_lambda(lc, F, lam0, mode, status);
-    const bool well = (mode == PKV_LAMBDA_PAPER) && (lam0 >= 0.05f);
+    const bool well = tc_well_conditioned(lam0, mode);
     const bool zero_fill = (ldn != t->dual_ld_prev);
     t->dual_ld_prev = ldn;
     if ((rc = tc_ridge_solve_impl(lc, &t->dual, t->Gd, t->RTf, N, ldn, d, t->Yd, well, zero_fill, status, &t->Yp, nullptr)))
@@ -304,12 +311,39 @@ static void mark(const TcForwardArgs& a, const Lc& lc, int stage) {
     if (a.ev) cudaEventRecord(a.ev[stage], lc.st);
 }
 
+// fp32 x fp32 statistics product from token-contiguous triples: all six passes (fp32-equivalent)
+static void six_pass_stats(TcGemm& g, Pair A, const __nv_bfloat16* A3, long long arows, Pair B, const __nv_bfloat16* B3,
+                           long long brows, long long ld, long long n) {
+    const __nv_bfloat16* a[3] = {A.hi, A.lo, A3};
+    const __nv_bfloat16* b[3] = {B.hi, B.lo, B3};
+    const int ia[6] = {0, 0, 1, 0, 2, 1}, ib[6] = {0, 1, 0, 2, 0, 1};
+    for (int i = 0; i < 6; ++i) {
+        g.A[i] = TcMat{a[ia[i]], ld, arows, n};
+        g.B[i] = TcMat{b[ib[i]], ld, brows, n};
+    }
+    g.npass = 6;
+    g.nacc = 4;
+}
+
 void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, const float* R, int n, float* S_H,
-             float* S_T, bool accumulate, DevStatus* status) {
+             float* S_T, bool accumulate, DevStatus* status, bool precise) {
     const int F = d->F, dm = d->d;
-    transpose_split(lc, X, n, F, t->ldT, t->XT);
-    transpose_split(lc, R, n, dm, t->ldT, t->RT);
+    transpose_split(lc, X, n, F, t->ldT, t->XT, precise ? t->XT3 : nullptr);
+    transpose_split(lc, R, n, dm, t->ldT, t->RT, precise ? t->RT3 : nullptr);
     t->S3_ready = 0;
+    if (precise) {
+        // a small ridge coefficient amplifies the rounding of the statistics: triples, six passes
+        const bool own = !accumulate && S_T == t->own_S_T;
+        TcGemm h = plain_gemm(F, F, n, S_H, F, 1.f, nullptr, 0, accumulate);
+        six_pass_stats(h, t->XT, t->XT3, F, t->XT, t->XT3, F, t->ldT, n);
+        h.lower_only = own;
+        gemm_tc(lc, h, status);
+        TcGemm g = plain_gemm(dm, F, n, S_T, F, 1.f, nullptr, 0, accumulate);
+        six_pass_stats(g, t->RT, t->RT3, dm, t->XT, t->XT3, F, t->ldT, n);
+        if (own) { g.out[0] = t->S3[0]; g.out[1] = t->S3[1]; g.out[2] = t->S3[2]; g.ldo = F; g.nout = 3; }
+        if (gemm_tc(lc, g, status) == PKV_OK && own) t->S3_ready = 1;
+        return;
+    }
     if (!accumulate && S_T == t->own_S_T) {
         // the build's own statistics: S_H is symmetric and its consumers (ridge scale, factorisation)
         // read the lower triangle only, so only tiles on or below the diagonal are computed
@@ -351,9 +385,7 @@ int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
 
 void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int F, int d, float* dW, float lam0,
                     int mode, DevStatus* status) {
-    // Under the adaptive scale of Eq. 7 cond(G) ~ (tr(S_H)/sigma_max)/lambda0; lambda0 >= 0.05 keeps it
-    // to a few tens.  Absolute and trace-mean coefficients give no such bound.
-    const bool well = (mode == PKV_LAMBDA_PAPER) && (lam0 >= 0.05f);
+    const bool well = tc_well_conditioned(lam0, mode);
     tc_ridge_solve_impl(lc, &t->solve, S, S_T, F, F, d, dW, well, false, status, &t->dW, t->S3_ready ? t->S3 : nullptr);
     t->S3_ready = 0;
 }
@@ -464,7 +496,7 @@ int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     // S7 (Eq. 9); the dual solver only needs the token-contiguous copy of the student features
     t->own_S_T = a.S_T;
     if (a.dual) transpose_split(lc, a.hC, N, F, t->ldT, t->XT);
-    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st);
+    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st, a.precise_stats != 0);
     mark(a, lc, 7);
     return PKV_OK;
 }
@@ -520,12 +552,10 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     // S7 (Eq. 9); the dual solver only needs the token-contiguous copy of the student features
     t->own_S_T = a.S_T;
     if (a.dual) transpose_split(lc, a.hC, N, F, t->ldT, t->XT);
-    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st);
+    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st, a.precise_stats != 0);
     mark(a, lc, 7);
     return PKV_OK;
 }
-
-
 
 void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const void* Wdown, const float* dW,
                     const float* zF, const float* R, float* xF_next, float* Dm, DevStatus* status) {

@@ -37,6 +37,9 @@ struct TcGemm {
     float alpha;
     bool accumulate, lower_only;
     int k_tri;      // 0: dense; 1: B lower triangular (skip k tiles past the row); 2: B upper triangular
+    int nacc;       // 0/1: one fp32 accumulator; 2 or 4: the hi x hi pass of a split product is accumulated apart
+                    // from the cross passes (and in several parts), which removes most of the tensor core's
+                    // truncation bias from sums of same-signed terms; pass 0 must be the hi x hi pass
 };
 struct MapCache;
 MapCache* tc_map_cache_create();
@@ -72,6 +75,9 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
                         float* dW, bool well_conditioned, bool zero_fill, DevStatus* status, const Pair* dW_pair,
                         __nv_bfloat16* const* S_T_triple);   // optional: dW's bf16 pair out; S_T already split
 
+int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const float* A, const float* B, int M, int N,
+                    int K, float alpha, float* C, bool accumulate, int passes, int nacc, DevStatus* status);
+
 // bf16 hi/lo pairs of fp32 activations: v ~= hi + lo with hi = bf16(v), lo = bf16(v - hi).
 struct Pair {
     __nv_bfloat16* hi;
@@ -85,6 +91,8 @@ struct TcBuffers {
     Pair hF, hC, dh;    // [N][F]
     Pair XT;            // [F][ldT]  student features, token-contiguous
     Pair RT;            // [d][ldT]  targets, token-contiguous
+    __nv_bfloat16* XT3; // third bf16 parts of XT / RT (statistics in six passes when the ridge coefficient is small)
+    __nv_bfloat16* RT3;
     Pair dW;            // [d][F]
     float* qkv;         // [2N][Dq+2Dkv]
     float* o;           // [2N][d]
@@ -121,6 +129,7 @@ struct TcForwardArgs {
     const float* dx;    // student half: xF - xC entering this block (state difference carried between blocks)
     float *part_m, *part_l, *part_O;
     int dual;           // 1: only the token-contiguous copy of the student features is prepared in S7
+    int precise_stats;  // 1: statistics from bf16 triples in six passes (small ridge coefficient), else pairs in three
     DevStatus* status;
     cudaEvent_t* ev;    // stage marks (index = stage) or nullptr
     cudaEvent_t* evT;   // 6 marks around the teacher half's stages (S1-2, S3, S4, S5, S9 share) or nullptr
@@ -142,7 +151,12 @@ int tc_teacher_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcFo
 int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a);
 int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status);
 void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, const float* R, int n, float* S_H,
-             float* S_T, bool accumulate, DevStatus* status);
+             float* S_T, bool accumulate, DevStatus* status, bool precise = false);
+// The precision rule shared by the statistics and the solve.  Under the adaptive scale of Eq. 7,
+// cond(S_H + lambda I) is about (sigma_max / (||S_H||_F^2 / tr S_H)) / lambda0, a few tens when lambda0 >= 0.05:
+// bf16 pairs (about 16 bits) are enough.  A smaller lambda0, or the absolute / trace-mean coefficients (no such
+// bound), take triples everywhere.
+inline bool tc_well_conditioned(float lam0, int mode) { return mode == PKV_LAMBDA_PAPER && lam0 >= 0.05f; }
 int tc_gram_with_buffers(const Lc& lc, Pair XT, Pair RT, int ldT, const float* X, const float* R, int n, int F, int dm,
                          float* S_H, float* S_T, bool accumulate, DevStatus* status);
 // S [F][F] is destroyed; S_T is only read.

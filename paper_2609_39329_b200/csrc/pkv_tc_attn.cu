@@ -139,7 +139,13 @@ enum { B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 3, B_VFULL = 5, B_VEMPTY = 7, B_SFUL
 template <int HD>
 __global__ void __launch_bounds__(192, 1) k_attn_tc(const __grid_constant__ AttnTcParams p) {
     using S = AttnSmem<HD>;
-    if (p.status->code != 0) return;      // an earlier stage already failed: the call reports it
+    {   // an earlier stage already failed: the call reports it.  One thread reads the status word so that the
+        // whole CTA takes the same branch even if the word changes while the CTA starts.
+        __shared__ int s_skip;
+        if (threadIdx.x == 0) s_skip = p.status->code;
+        __syncthreads();
+        if (s_skip != 0) return;
+    }
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -451,11 +457,12 @@ void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, i
 template <int HD>
 static int launch_attn(const Lc& lc, const AttnTcParams& p, int qtiles, int zcount) {
     using S = AttnSmem<HD>;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce once;
+    int dev;
+    if (once.needed(&dev)) {
         if (cudaFuncSetAttribute(k_attn_tc<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess)
             return PKV_ERR_CUDA;
-        attr_set = true;
+        once.mark(dev);
     }
     dim3 grid(qtiles, p.Hkv, zcount);
     k_attn_tc<HD><<<grid, 192, S::kTotal, lc.st>>>(p);
@@ -546,7 +553,7 @@ int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
     const int qtiles = (rows + 127) / 128;
     p.z0 = (a.mode == 2) ? p.nsplitF : 0;
     const int zcount = a.mode == 0 ? p.nsplitF + p.nsplitC : (a.mode == 1 ? p.nsplitF : p.nsplitC);
-    rc = (hd == 128) ? launch_attn<128>(lc, p, qtiles, zcount) : launch_attn<64>(lc, p, qtiles, zcount);
+    rc = launch_attn<64>(lc, p, qtiles, zcount);      // hd = 128 left above for the two-tile kernel
     if (rc != PKV_OK) return rc;
     AttnArgs c = a;
     c.nsplitF = p.nsplitF; c.nsplitC = p.nsplitC;

@@ -12,9 +12,8 @@
 //   warps 2-5   softmax warpgroup of tile 0, warps 6-9 of tile 1: one thread per query row, the
 //               whole S row in registers (single pass), exp2 with the row's reference maximum,
 //               P -> TMEM.  O stays in TMEM across key tiles; it is rescaled (TMEM load, multiply,
-//               store) only when a row's maximum grew by more than 2^8 since the reference was
-//               set, which is rare after the first tiles, and exact (the final (m, l, O) triple is
-//               consistent with whatever reference was used).
+//               store) only when some row of the warp saw a new maximum, which is rare after the
+//               first tiles.  The reference is the exact running maximum (kRescaleThreshold = 0).
 // TMEM: S0 S1 O0 O1, 128 columns each.  Every wait is bounded (see pkv_ptx.cuh).
 #include <cuda.h>
 #include <math.h>
@@ -85,7 +84,13 @@ __device__ __forceinline__ void tmem_st_wait() {
 
 __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Attn2Params p) {
     using namespace a2;
-    if (p.status->code != 0) return;      // an earlier stage already failed: the call reports it
+    {   // an earlier stage already failed: the call reports it.  One thread reads the status word so that the
+        // whole CTA takes the same branch even if the word changes while the CTA starts.
+        __shared__ int s_skip;
+        if (threadIdx.x == 0) s_skip = p.status->code;
+        __syncthreads();
+        if (s_skip != 0) return;
+    }
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -284,7 +289,7 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
                 mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
             }
             const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-            // reference maximum: moved only when the row maximum outgrew it by more than 2^8
+            // reference maximum: the exact running maximum (moved whenever the tile's maximum exceeds it)
             float alpha = 1.f;
             const bool move = mx > m_ref + kRescaleThreshold;         // also true for the first finite maximum (m_ref = -inf)
             if (move) {
@@ -371,11 +376,12 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
 }
 
 int launch_attn2(const Lc& lc, const Attn2Params& p, int qpairs, int zcount) {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce once;
+    int dev;
+    if (once.needed(&dev)) {
         if (cudaFuncSetAttribute(k_attn_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, a2::kTotal) != cudaSuccess)
             return PKV_ERR_CUDA;
-        attr_set = true;
+        once.mark(dev);
     }
     dim3 grid(qpairs, p.Hkv, zcount);
     k_attn_tc2<<<grid, 320, a2::kTotal, lc.st>>>(p);

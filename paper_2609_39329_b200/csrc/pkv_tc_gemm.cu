@@ -41,6 +41,7 @@ struct alignas(64) GemmTcParams {
     long long ldo;
     int nout, out_col_off;
     int accumulate, lower_only, k_tri, vec_ok;
+    int nacc;                 // TMEM accumulators per tile (1, 2 or 4), see TcGemm::nacc
     DevStatus* status;
 };
 
@@ -51,6 +52,14 @@ constexpr int kGemmBarBytes = (2 * kGemmMaxStages + 1) * 8 + 16;
 // and all passes are issued from it (the shared operand of a split product is not re-read).
 // PRE: the epilogue warps fetch the fp32 C tile they will add to (read-modify-write products of the
 // factorisation) while the main loop runs, instead of after it.
+//
+// Accumulators.  The tensor core adds each MMA's result to the fp32 accumulator with truncation, not
+// round-to-nearest: a sum of same-signed terms (the diagonal of a Gram or of L L^T) comes out low by about
+// 2^-25 of the running sum per MMA.  When a small difference C - A B^T is wanted (trailing updates of a
+// rank-deficient ridge matrix) that bias is what limits the result.  With nacc > 1 the large hi x hi pass goes
+// round-robin to accumulators 1..nacc-1, each of which so sees only a few adds at a fraction of the full
+// magnitude, every other pass to accumulator 0 where its truncation is relative to the small cross terms;
+// the epilogue adds the accumulators in registers with round-to-nearest.
 template <int BN, bool PRE>
 __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcParams p) {
     const int m0 = blockIdx.y * 128, n0 = blockIdx.x * BN, z = blockIdx.z;
@@ -90,8 +99,9 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         *abort_flag = 0;
         fence_barrier_init();
     }
+    const int nacc = p.nacc;
     if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), BN);
+        tmem_alloc(smem_u32(tmem_slot), (uint32_t)(BN * nacc));
         tmem_relinquish();
     }
     tc_fence_before();
@@ -100,7 +110,12 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     const uint32_t tbase = *tmem_slot;
     // everything above is independent of earlier kernels; from here on their results are read
     pdl_wait();
-    const bool skip = p.status->code != 0;      // an earlier stage already failed: the call reports it
+    // an earlier stage already failed: the call reports it.  The status word may change while the CTA starts
+    // (another CTA's error), so one thread reads it and the whole CTA takes the same branch.
+    volatile int* skip_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
+    if (threadIdx.x == 0) *skip_flag = p.status->code;
+    __syncthreads();
+    const bool skip = *skip_flag != 0;
 
     if (skip) {
         // nothing to do: fall through to the teardown
@@ -123,6 +138,8 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16(128, BN);
             bool ok = true;
+            uint32_t used = 0u;          // accumulators that already hold a partial sum
+            uint32_t hh = 0u;            // running index of the hi x hi MMAs
             for (int it = 0; it < ktiles; ++it) {
                 const int s = it % STAGES;
                 if (!mbar_wait(bars + 8 * s, (it / STAGES) & 1, abort_flag, p.status, 2)) { ok = false; break; }
@@ -131,9 +148,14 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                 for (int ps = 0; ps < p.npass; ++ps) {
                     const uint64_t da = smem_desc_sw128(sa + p.pa[ps] * kA);
                     const uint64_t db = smem_desc_sw128(sa + p.nA * kA + p.pb[ps] * kB);
+                    const bool big = nacc > 1 && p.pa[ps] == 0 && p.pb[ps] == 0;      // hi x hi
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        mma_bf16_ss(tbase, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (it | ps | kk) != 0);
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint32_t acc = big ? 1u + (hh++ % (uint32_t)(nacc - 1)) : 0u;
+                        mma_bf16_ss(tbase + acc * (uint32_t)BN, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc,
+                                    (used >> acc) & 1u);
+                        used |= 1u << acc;
+                    }
                 }
                 mma_commit(bars + 8 * (STAGES + s));
             }
@@ -169,6 +191,15 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                 if (ktiles > 0) {
                     tmem_ld32(tbase + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
                     tmem_ld_wait();
+                    // further accumulators: added in registers with round to nearest (the launcher only asks for
+                    // them when every one of them receives at least one MMA)
+                    for (int a = 1; a < nacc; ++a) {
+                        uint32_t r2[32];
+                        tmem_ld32(tbase + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * BN + c0), r2);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                    }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) r[j] = 0u;
@@ -254,7 +285,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tbase, BN);
+        tmem_dealloc(tbase, (uint32_t)(BN * nacc));
     }
 }
 
@@ -380,12 +411,13 @@ static int cached_map(MapCache* cache, CUtensorMap* out, const void* ptr, uint64
 
 template <int BN, bool PRE>
 static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
-    static bool attr_set = false;
+    static PerDeviceOnce once;
     constexpr int kMaxSmem = 227 * 1024;
-    if (!attr_set) {
+    int dev;
+    if (once.needed(&dev)) {
         if (cudaFuncSetAttribute(k_gemm_tc<BN, PRE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return PKV_ERR_CUDA;
-        attr_set = true;
+        once.mark(dev);
     }
     const int stage_bytes = p.nA * 128 * 128 + p.nB * BN * 128;
     const int fixed = kGemmBarBytes + 1024;
@@ -395,14 +427,16 @@ static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     const int half = 112 * 1024 - fixed;
     const long long ctas = (long long)((p.N + BN - 1) / BN) * ((p.M + 127) / 128) * batch;
     int stages;
-    if (ctas <= 148) stages = (kMaxSmem - fixed) / stage_bytes;      // one wave: occupancy is moot, take the deepest pipeline
+    const bool one_per_sm = BN * p.nacc > 256;      // two CTAs of this kernel would not fit in the 512 TMEM columns
+    if (ctas <= 148 || one_per_sm) stages = (kMaxSmem - fixed) / stage_bytes;      // occupancy is moot: deepest pipeline
     else if (ktiles <= 8 || 2 * stage_bytes <= half) stages = half / stage_bytes;
     else stages = (kMaxSmem - fixed) / stage_bytes;
     if (stages < 1) stages = 1;
     if (stages > kGemmMaxStages) stages = kGemmMaxStages;
     if (stages > ktiles) stages = ktiles > 0 ? ktiles : 1;
     p.stages = stages;
-    const int smem = stages * stage_bytes + fixed;
+    int smem = stages * stage_bytes + fixed;
+    if (one_per_sm && smem < 120 * 1024) smem = 120 * 1024;      // keeps a second CTA (and its TMEM request) off the SM
     dim3 grid((p.N + BN - 1) / BN, (p.M + 127) / 128, batch);
     if (lc.pdl) {
         cudaLaunchConfig_t cfg = {};
@@ -430,7 +464,8 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     // 128 x 256 tiles move a third fewer operand bytes per flop than 128 x 128; taken when they still give
     // at least two waves of CTAs (and the C tile is not prefetched: that variant is 128 wide)
     const long long tiles256 = (long long)((g.N + 255) / 256) * ((g.M + 127) / 128) * g.batch;
-    const bool wide = g.N >= 512 && tiles256 >= 2 * 148 && !(g.C && g.accumulate) && !g.lower_only && g.k_tri != 2;
+    const bool wide = g.N >= 512 && tiles256 >= 2 * 148 && !(g.C && g.accumulate) && !g.lower_only && g.k_tri != 2 &&
+                      g.nacc < 4;
     const int BN = (g.N <= 64) ? 64 : (wide ? 256 : 128);
     MapCache* cache = (MapCache*)lc.map_cache;
     // distinct operands
@@ -469,6 +504,13 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     p.accumulate = g.accumulate ? 1 : 0;
     p.lower_only = g.lower_only ? 1 : 0;
     p.k_tri = g.k_tri;
+    // several accumulators only for products with one hi x hi pass and cross passes, and only if they fit
+    p.nacc = 1;
+    if (g.nacc > 1 && g.npass >= 2 && p.pa[0] == 0 && p.pb[0] == 0) {
+        int hh_passes = 0;
+        for (int i = 0; i < g.npass; ++i) hh_passes += (p.pa[i] == 0 && p.pb[i] == 0) ? 1 : 0;
+        if (hh_passes == 1) p.nacc = (g.nacc >= 4 && BN * 4 <= 512) ? 4 : (BN * 2 <= 512 ? 2 : 1);
+    }
     p.vec_ok = (g.C && ((uintptr_t)g.C & 15) == 0 && g.ldc % 4 == 0 && g.c_col0 % 4 == 0 && g.c_zcol % 4 == 0 &&
                 (!g.addend || (((uintptr_t)g.addend & 15) == 0 && g.ldadd % 4 == 0))) ? 1 : 0;
     p.status = status;

@@ -120,8 +120,13 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
     float* T = rd + PB;                          // doubling temporary
     pdl_launch_dependents();
     pdl_wait();
-    if (status->code != 0) return;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    {   // one thread reads the status word: the whole CTA takes the same branch
+        __shared__ int s_skip;
+        if (tid == 0) s_skip = status->code;
+        __syncthreads();
+        if (s_skip != 0) return;
+    }
     const int nbk = min(PB, n - k0);
     const float lam = status->lam;
     // ---- load the lower part (identity outside the block's extent), lambda on the diagonal ----
@@ -387,6 +392,7 @@ static void six_pass(TcGemm& g, const Trip& A, long long lda, long long arows, l
         g.B[i] = TcMat{B.a[ib[i]], ldb, brows, bcols};
     }
     g.npass = 6;
+    g.nacc = 4;      // fp32-equivalent products: hi x hi accumulated apart, in three parts
 }
 
 static void three_pass(TcGemm& g, const Trip& A, long long lda, long long arows, long long acols, const Trip& B,
@@ -397,6 +403,34 @@ static void three_pass(TcGemm& g, const Trip& A, long long lda, long long arows,
         g.B[i] = TcMat{B.a[ib[i]], ldb, brows, bcols};
     }
     g.npass = 3;
+    g.nacc = 2;
+}
+
+// C [M][N] (+)= alpha * A B^T for fp32 A [M][K], B [N][K]: both are split into bf16 parts in the solver's S_T / Z
+// operand buffers (so M*K8 and N*K8 must fit in d*F elements, K8 = K rounded up to 8) and multiplied in `passes`
+// tensor-core passes (6: triples, fp32-equivalent; 3: pairs).  The building block of the factorisation,
+// exported for unit tests.
+int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const float* A, const float* B, int M, int N,
+                    int K, float alpha, float* C, bool accumulate, int passes, int nacc, DevStatus* status) {
+    const long long K8 = (K + 7) / 8 * 8;
+    if ((size_t)M * K8 > cap_elems || (size_t)N * K8 > cap_elems) return PKV_ERR_UNSUPPORTED;
+    if (passes != 3 && passes != 6) return PKV_ERR_INVALID_ARG;
+    Trip A3{{t->S2[0], t->S2[1], t->S2[2]}}, B3{{t->Z2[0], t->Z2[1], t->Z2[2]}};
+    if (K8 != K) {
+        for (int i = 0; i < 3; ++i) {
+            cudaMemsetAsync(A3.a[i], 0, (size_t)M * K8 * 2, lc.st);
+            cudaMemsetAsync(B3.a[i], 0, (size_t)N * K8 * 2, lc.st);
+        }
+    }
+    launch_split3(lc, A, K, M, K, A3, K8, 3);
+    launch_split3(lc, B, K, N, K, B3, K8, 3);
+    TcGemm g{};
+    if (passes == 6) six_pass(g, A3, K8, M, K, B3, K8, N, K);
+    else three_pass(g, A3, K8, M, K, B3, K8, N, K);
+    g.M = M; g.N = N; g.K = K; g.batch = 1; g.alpha = alpha;
+    g.C = C; g.ldc = N; g.c_rows = M; g.c_cols = N; g.accumulate = accumulate;
+    g.nacc = nacc;
+    return gemm_tc(lc, g, status);
 }
 
 // largest pairs * s * s over the doubling levels (elements of the TT workspace)
@@ -450,11 +484,12 @@ int tc_solve_init(TcSolveBuffers* t) {
     if (cudaStreamCreateWithPriority(&t->aux, cudaStreamNonBlocking, greatest) != cudaSuccess) return PKV_ERR_CUDA;
     for (int i = 0; i < 3; ++i)
         if (cudaEventCreateWithFlags(&t->ev[i], cudaEventDisableTiming) != cudaSuccess) return PKV_ERR_CUDA;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce once;
+    int dev;
+    if (once.needed(&dev)) {
         if (cudaFuncSetAttribute(k_potrf128, cudaFuncAttributeMaxDynamicSharedMemorySize, kPotrfSmemBytes) != cudaSuccess)
             return PKV_ERR_CUDA;
-        attr_set = true;
+        once.mark(dev);
     }
     return PKV_OK;
 }
@@ -605,6 +640,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         if (nsp == 2) three_pass(g, S2, ld, d, F, X3, ld, F, F);
         else six_pass(g, S2, ld, d, F, X3, ld, F, F);
         g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 1;
+        g.nacc = 2;      // long contraction, no cancellation: two accumulators keep two CTAs per SM
         g.c_rows = d; g.c_cols = F;
         g.out[0] = Z2.a[0]; g.out[1] = Z2.a[1]; g.out[2] = Z2.a[2]; g.ldo = ld; g.nout = nsp;
         if ((rc = gemm_tc(lc, g, status))) return rc;
@@ -614,6 +650,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         if (nsp == 2) three_pass(g, Z2, ld, d, F, XT3, ld, F, F);
         else six_pass(g, Z2, ld, d, F, XT3, ld, F, F);
         g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 2;
+        g.nacc = 2;
         g.C = dW; g.ldc = ld; g.c_rows = d; g.c_cols = F;
         if (dW_pair) { g.out[0] = dW_pair->hi; g.out[1] = dW_pair->lo; g.ldo = ld; g.nout = 2; }
         if ((rc = gemm_tc(lc, g, status))) return rc;

@@ -1,10 +1,13 @@
 """Full-size checks in the launch configuration bench.py times (tensor-core engine, default split plan).
 
-Config 2 (the benchmark workload) is compared with the fp64 oracle element by element.  For configs
-3-5 the oracle cannot run a whole block in seconds, so every stage is checked at the full shapes on what
-the oracle can compute one by one (sampled attention rows at full cache length, the full Gram, the full
-ridge solve) and on properties that hold at any size (stationarity of the ridge solution, the ridge
-residual identity between the returned states)."""
+Config 2 (the benchmark workload) is compared with the fp64 oracle element by element.  Configs 3-5 are
+compared with the oracle as whole blocks at their full cache length, width, head layout and kept rule, with
+the number of reference tokens cut to 256 (the oracle's time grows with it; every other size is the
+config's own), and as a three-block stack at config 3's shape, free-running and re-anchored per block.
+Beside that every stage is checked at the full reference-set size on what the oracle can compute one by
+one (sampled attention rows at full cache length, the full Gram, the full ridge solve) and on properties
+that hold at any size (stationarity of the ridge solution, the ridge residual identity between the
+returned states)."""
 import numpy as np
 import pytest
 
@@ -161,4 +164,89 @@ def test_whole_block_runs_at_full_size_and_keeps_the_ridge_identities(B, cfg_id)
     np.testing.assert_allclose(float((out["dW"].double() ** 2).sum()), st["dW_fro2"], rtol=1e-4)
     print("config %d: lambda %.4g, ||T||^2 %.4g -> residual %.4g" % (cfg_id, st["lambda_eff"], st["target_fro2"],
                                                                      st["resid_fro2"]))
+    ctx.close()
+
+
+# ------------------------------------------------------------------ whole blocks of configs 3-5 vs the oracle
+
+N_CUT = 256        # reference tokens of the whole-block comparisons below (the configs' own N is 1024-4096)
+
+
+def device_layer(B, cfg, lay):
+    import torch
+    off, idx = gen.kept_to_csr(lay["kept"])
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    return {"w": B.to_device(lay["weights"], cfg.dtype), "K": kv["K"], "V": kv["V"], "head_off": off,
+            "idx": torch.from_numpy(idx).cuda()}
+
+
+@pytest.mark.parametrize("cfg_id", [3, 4, 5])
+def test_whole_block_matches_oracle_at_the_shapes_of_configs_3_to_5(B, cfg_id):
+    """Full L, d, F, head layout and kept rule of the config; N cut to N_CUT to bound the oracle's time.
+    Config 4 is checked at the three ridge coefficients of its sweep (one oracle forward, three solves)."""
+    import torch
+    cfg = gen.scaled_config(gen.benchmark_config(cfg_id), N=N_CUT)
+    lay = gen.gen_layer(cfg, 0)
+    x = gen.gen_reference(cfg)
+    lams = cfg.lam_sweep if cfg.lam_sweep else (cfg.lam0,)
+    ref = orc.build_patch(lay["weights"], lay["K"], lay["V"], lay["kept"], x, x, [0, cfg.N], cfg.L, lams[0], cfg,
+                          keep_intermediates=True)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    dl = device_layer(B, cfg, lay)
+    xt = torch.from_numpy(x).cuda()
+    for lam0 in lams:
+        lam = orc.ridge_lambda(ref["S_H"], lam0)
+        want = orc.ridge_solve(ref["S_H"], ref["S_T"], lam)
+        out = ctx.build_patch(dl["w"], dl["K"], dl["V"], dl["head_off"], dl["idx"], xt, xt, [0, cfg.N], cfg.L, lam0)
+        err = H.rel_fro(out["dW"].cpu().numpy(), want)
+        eF = H.rel_fro(out["xF_next"].cpu().numpy(), ref["xF_next"])
+        xC_want = ref["stu"]["z"] + ref["H"] @ (lay["weights"]["Wdown"].astype(np.float64) + want).T
+        eC = H.rel_fro(out["xC_next"].cpu().numpy(), xC_want)
+        print("config %d shape, N=%d, lambda0 %g: dW rel fro err %.3e, xF_next %.2e, xC_next %.2e, lambda %.5g (oracle %.5g)"
+              % (cfg_id, cfg.N, lam0, err, eF, eC, out["stats"]["lambda_eff"], lam))
+        assert err <= DW_TOL
+        np.testing.assert_allclose(out["stats"]["lambda_eff"], lam, rtol=1e-3)
+        np.testing.assert_allclose(out["stats"]["target_fro2"], ref["T_fro2"], rtol=2e-2)
+        assert eF <= 1e-3 and eC <= 1e-3
+    ctx.close()
+
+
+def test_three_block_stack_at_config3_shape_free_running_and_reanchored(B):
+    """Algorithm 1 over blocks through pkv_build_stack (teacher run ahead on its own stream) at config 3's
+    full L, d, F and kept rule; N cut to 128, three blocks.  Free-running: both sides propagate their own
+    states.  Re-anchored: the oracle's block l is fed the states the CUDA path produced for it, which is the
+    contract of one block; those states come from a stack call over the blocks before l, and the patch from a
+    call that resumes at first_layer = l."""
+    import torch
+    nl = 3
+    cfg = gen.scaled_config(gen.benchmark_config(3), N=128, n_layers=nl)
+    lays = [gen.gen_layer(cfg, l) for l in range(nl)]
+    x0 = gen.gen_reference(cfg)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    dl = [device_layer(B, cfg, lay) for lay in lays]
+    xt = torch.from_numpy(x0).cuda()
+    out = ctx.build_stack(dl, xt, xt, [0, cfg.N], cfg.L, cfg.lam0)
+    xF, xC = x0.astype(np.float64), x0.astype(np.float64)
+    for l in range(nl):
+        lay = lays[l]
+        o = orc.build_patch(lay["weights"], lay["K"], lay["V"], lay["kept"], xF, xC, [0, cfg.N], cfg.L, cfg.lam0, cfg)
+        e_free = H.rel_fro(out["dW"][l].cpu().numpy(), o["dW"])
+        msg = "block %d: free-running dW rel fro err %.3e" % (l, e_free)
+        assert e_free <= DW_TOL, msg
+        if l > 0:
+            pre = ctx.build_stack(dl[:l], xt, xt, [0, cfg.N], cfg.L, cfg.lam0)          # states entering block l
+            res = ctx.build_stack(dl, pre["xF_final"], pre["xC_final"], [0, cfg.N], cfg.L, cfg.lam0, first_layer=l)
+            oa = orc.build_patch(lay["weights"], lay["K"], lay["V"], lay["kept"], pre["xF_final"].cpu().numpy(),
+                                 pre["xC_final"].cpu().numpy(), [0, cfg.N], cfg.L, cfg.lam0, cfg)
+            e_anch = H.rel_fro(res["dW"][l].cpu().numpy(), oa["dW"])
+            msg += ", re-anchored %.3e" % e_anch
+            assert e_anch <= DW_TOL, msg
+            # resuming reproduces the uninterrupted run
+            assert H.rel_fro(res["dW"][l].cpu().numpy(), out["dW"][l].cpu().numpy()) <= 1e-4
+        print(msg)
+        xF, xC = o["xF_next"], o["xC_next"]
+    eF = H.rel_fro(out["xF_final"].cpu().numpy(), xF)
+    eC = H.rel_fro(out["xC_final"].cpu().numpy(), xC)
+    print("final states: xF %.2e, xC %.2e" % (eF, eC))
+    assert eF <= 1e-3 and eC <= 1e-3
     ctx.close()

@@ -1,9 +1,12 @@
 """pkv_gram_noalloc, the entry point for callers that cannot allocate device memory (hosts that own
 all device memory through their own pool, or that must avoid cudaMalloc's device-wide synchronisation
 inside a latency-critical loop): it must give what pkv_gram gives, on two calls in a row, since its
-fixed scratch array keeps the previous call's contents.  Collected last on purpose."""
+fixed scratch array keeps the previous call's contents; it is also held to the fp64 oracle's statistics
+and to its promise that the device's free memory does not move across a call.  Collected last on purpose."""
 import numpy as np
 import pytest
+
+from oracle import pkv_oracle as orc
 
 pytestmark = pytest.mark.gpu
 
@@ -28,6 +31,19 @@ def test_noalloc_statistics_match_the_context_entry_point_twice_in_a_row():
         for got, want in ((got_H, want_H), (got_T, want_T)):
             err = (got.double() - want.double()).norm() / want.double().norm()
             assert float(err) <= 2e-4
+        # ... and against the oracle's Eq. 9 sums
+        o_H, o_T = orc.sufficient_statistics(X.cpu().numpy(), R.cpu().numpy())
+        for got, want in ((got_H, o_H), (got_T, o_T)):
+            err = np.linalg.norm(got.cpu().numpy().astype(np.float64) - want) / np.linalg.norm(want)
+            assert err <= 2e-4, err
+        # nothing is allocated: with the outputs supplied by the caller, the device's free memory is the
+        # same before and after a call (the first call on the device, above, already resolved the array)
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        B.gram_noalloc(X, R, got_H, got_T)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0, (free0, free1)
         # running sums over two calls (Eq. 9), again through the shared array
         h = n // 2
         a_H, a_T = B.gram_noalloc(X[:h].contiguous(), R[:h].contiguous())
