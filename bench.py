@@ -232,7 +232,7 @@ def run_stack(args, cfg, B, torch, dist, world, rank, local, peaks):
     lays = [build_inputs(cfg, l) for l in range(D)]
     b_max = max(len(k) for lay in lays for k in lay["kept"])
     engine = B.ENGINE_SIMT if args.engine == "simt" else B.ENGINE_AUTO
-    ctx = B.PkvContext(B.dims_from_config(cfg, b_max=b_max), engine=engine)
+    ctx = B.PkvContext(B.dims_from_config(cfg, b_max=b_max), engine=engine, reserve_sms=args.reserve_sms)
     dev = []
     for lay in lays:
         off, idx = gen.kept_to_csr(lay["kept"])
@@ -326,7 +326,7 @@ def run_stack(args, cfg, B, torch, dist, world, rank, local, peaks):
             "cpu_baseline": cpu, "clocks": clocks,
             "e2e": {"value": None, "unit": "ms", "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
                     "note": "end-to-end with host buffers is measured on the single-block workload (default config 2)"},
-            "gpu_launches": int(launches), "peaks": peaks}
+            "gpu_launches": int(launches), "peaks": peaks, "teacher_sms": ctx.teacher_sm_count()}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -347,6 +347,8 @@ def main():
     ap.add_argument("--kernel", default=None, choices=["attention", "gram", "solve"],
                     help="time one stage alone through its own entry point (pkv_attention / pkv_gram / pkv_ridge_solve) "
                          "on the shapes of --config, with seeded random operands")
+    ap.add_argument("--reserve-sms", type=int, default=0,
+                    help="stack configs: SMs the teacher stream leaves free (0 = library default, negative = none)")
     ap.add_argument("--quick", action="store_true",
                     help="timed steps only (no stage pass, no end-to-end pass, no CPU baseline): for profiler runs")
     args = ap.parse_args()

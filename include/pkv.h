@@ -88,6 +88,8 @@ typedef struct pkv_opts {
     void* workspace;         /* optional caller-provided device workspace (256-byte aligned) ... */
     size_t workspace_bytes;  /* ... of at least pkv_workspace_bytes(); NULL/0: the context allocates */
     int32_t solver;          /* PKV_SOLVER_* (used by pkv_build_patch / pkv_build_stack) */
+    int32_t reserve_sms;     /* pkv_build_stack: SMs the teacher stream leaves free for the student stream and
+                                the ridge solve; 0 = default (12), negative = none (teacher on every SM) */
 } pkv_opts;
 
 /* Block weights, all device, element type dims.dtype except the fp32 norm gains.
@@ -188,6 +190,8 @@ int pkv_merge(void* W, int w_dtype, const float* dW, int64_t count, void* cuda_s
  * more blocks, at most 128 layers and stage timing off, the teacher half of up to two later blocks
  * runs on a second stream owned by the context, beside the student half and the solve of the
  * current block; results are the same as block-by-block calls up to rounding order.  That stream is
+ * confined to all SMs but a small reserve (pkv_opts.reserve_sms) so that its long-running attention
+ * CTAs never starve the student's kernels and the solve.  That stream is
  * ordered after the work already queued on the context's stream and is drained before the call
  * returns; the call returns after one synchronisation.  In this mode stage_ms stays zero.  With
  * stage timing on, with the SIMT engine or for a single block the blocks run strictly in sequence.
@@ -267,6 +271,10 @@ int pkv_set_timing(pkv_ctx* ctx, int on);
 
 /* Number of kernels the context launched since creation (for launch accounting). */
 int64_t pkv_launch_count(const pkv_ctx* ctx);
+
+/* SMs the teacher stream of pkv_build_stack may occupy: the device's SM count minus the reserve when the
+ * driver granted the partition, the full count otherwise. */
+int pkv_teacher_sm_count(const pkv_ctx* ctx);
 
 const char* pkv_strerror(int code);
 const char* pkv_last_cuda_error(const pkv_ctx* ctx);

@@ -40,7 +40,7 @@ class pkv_dims(C.Structure):
 
 class pkv_opts(C.Structure):
     _fields_ = [("engine", C.c_int32), ("kv_split", C.c_int32), ("workspace", C.c_void_p),
-                ("workspace_bytes", C.c_size_t), ("solver", C.c_int32)]
+                ("workspace_bytes", C.c_size_t), ("solver", C.c_int32), ("reserve_sms", C.c_int32)]
 
 
 class pkv_block_weights(C.Structure):
@@ -127,6 +127,8 @@ def lib() -> C.CDLL:
     L.pkv_set_timing.argtypes = [C.c_void_p, C.c_int]
     L.pkv_launch_count.restype = C.c_int64
     L.pkv_launch_count.argtypes = [C.c_void_p]
+    L.pkv_teacher_sm_count.restype = C.c_int
+    L.pkv_teacher_sm_count.argtypes = [C.c_void_p]
     for f in ("pkv_strerror", "pkv_stage_name"):
         getattr(L, f).restype = C.c_char_p
         getattr(L, f).argtypes = [C.c_int]
@@ -159,7 +161,7 @@ class PkvContext:
     """Owns one pkv_ctx.  Tensors passed in must live on the context's CUDA device."""
 
     def __init__(self, dims: pkv_dims, engine: int = ENGINE_AUTO, kv_split: int = 0, stream=None,
-                 solver: int = SOLVER_PRIMAL, workspace=None):
+                 solver: int = SOLVER_PRIMAL, workspace=None, reserve_sms: int = 0):
         import torch
         self.torch = torch
         self.dims = dims
@@ -167,7 +169,7 @@ class PkvContext:
         self.stream = stream
         self.workspace = workspace      # optional caller-owned uint8 CUDA tensor (kept alive with the context)
         self.opts = pkv_opts(engine, kv_split, _ptr(workspace) if workspace is not None else None,
-                             int(workspace.numel()) if workspace is not None else 0, solver)
+                             int(workspace.numel()) if workspace is not None else 0, solver, reserve_sms)
         h = C.c_void_p()
         sp = C.c_void_p(stream.cuda_stream) if stream is not None else C.c_void_p(torch.cuda.current_stream().cuda_stream)
         rc = self.L.pkv_create(C.byref(h), C.byref(dims), C.byref(self.opts), sp)
@@ -199,6 +201,9 @@ class PkvContext:
 
     def launch_count(self) -> int:
         return int(self.L.pkv_launch_count(self.h))
+
+    def teacher_sm_count(self) -> int:
+        return int(self.L.pkv_teacher_sm_count(self.h))
 
     def selftest_bounded_wait(self):
         """pkv_selftest_bounded_wait: returns (code, site)."""

@@ -3,15 +3,97 @@
 // states).  All arithmetic happens in the kernels of the other translation units.
 #include <math.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
 #include <vector>
 
+#include <cuda.h>
+
 #include "pkv_internal.h"
 #include "pkv_tc.h"
 
 using namespace pkv;
+
+// ---------------------------------------------------------------------------------------------
+// SM partition for the teacher stream of the stack driver.
+//
+// The teacher's attention CTAs each hold a whole SM (all of its shared memory and tensor memory) for
+// hundreds of microseconds, and there are several waves of them: while they run, the student's kernels
+// and the latency-bound chain of the ridge solve find no free SM, whatever their stream priority, and
+// the two streams end up running one after the other.  The teacher stream is therefore created inside a
+// green context that owns all SMs but a reserve; the student's kernels and the solve (ordinary streams,
+// all SMs) then always find the reserve free of long-running CTAs.  Driver entry points are looked up at
+// run time; if anything is missing the teacher stream is an ordinary stream (correct, less overlap).
+// ---------------------------------------------------------------------------------------------
+namespace {
+struct GreenApi {
+    CUresult (*DeviceGet)(CUdevice*, int);
+    CUresult (*DeviceGetDevResource)(CUdevice, CUdevResource*, CUdevResourceType);
+    CUresult (*SplitByCount)(CUdevResource*, unsigned int*, const CUdevResource*, CUdevResource*, unsigned int,
+                             unsigned int);
+    CUresult (*GenerateDesc)(CUdevResourceDesc*, CUdevResource*, unsigned int);
+    CUresult (*GreenCtxCreate)(CUgreenCtx*, CUdevResourceDesc, CUdevice, unsigned int);
+    CUresult (*GreenCtxStreamCreate)(CUstream*, CUgreenCtx, unsigned int, int);
+    CUresult (*GreenCtxDestroy)(CUgreenCtx);
+    bool ok;
+};
+
+template <typename Fn>
+bool entry(const char* name, Fn* out) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint(name, &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess || !p) {
+        cudaGetLastError();
+        return false;
+    }
+    *out = reinterpret_cast<Fn>(p);
+    return true;
+}
+
+const GreenApi& green_api() {
+    static GreenApi api = [] {
+        GreenApi a{};
+        a.ok = entry("cuDeviceGet", &a.DeviceGet) && entry("cuDeviceGetDevResource", &a.DeviceGetDevResource) &&
+               entry("cuDevSmResourceSplitByCount", &a.SplitByCount) && entry("cuDevResourceGenerateDesc", &a.GenerateDesc) &&
+               entry("cuGreenCtxCreate", &a.GreenCtxCreate) && entry("cuGreenCtxStreamCreate", &a.GreenCtxStreamCreate) &&
+               entry("cuGreenCtxDestroy", &a.GreenCtxDestroy);
+        return a;
+    }();
+    return api;
+}
+
+// A stream whose kernels run on at least `want_sms` SMs of the current device and leave the rest alone.
+// Returns false (nothing created) when the partition cannot be made.
+bool make_partition_stream(int want_sms, cudaStream_t* stream, void** gctx_out, int* got_sms) {
+    const GreenApi& a = green_api();
+    if (!a.ok || want_sms <= 0) return false;
+    int ord = 0;
+    if (cudaGetDevice(&ord) != cudaSuccess) return false;
+    CUdevice dev;
+    if (a.DeviceGet(&dev, ord) != CUDA_SUCCESS) return false;
+    CUdevResource all, part, rest;
+    if (a.DeviceGetDevResource(dev, &all, CU_DEV_RESOURCE_TYPE_SM) != CUDA_SUCCESS) return false;
+    if ((int)all.sm.smCount <= want_sms) return false;
+    unsigned int groups = 1;
+    if (a.SplitByCount(&part, &groups, &all, &rest, 0, (unsigned int)want_sms) != CUDA_SUCCESS || groups != 1) return false;
+    if (part.sm.smCount >= all.sm.smCount) return false;      // rounding left no reserve
+    CUdevResourceDesc desc;
+    if (a.GenerateDesc(&desc, &part, 1) != CUDA_SUCCESS) return false;
+    CUgreenCtx g;
+    if (a.GreenCtxCreate(&g, desc, dev, CU_GREEN_CTX_DEFAULT_STREAM) != CUDA_SUCCESS) return false;
+    CUstream st;
+    if (a.GreenCtxStreamCreate(&st, g, CU_STREAM_NON_BLOCKING, 0) != CUDA_SUCCESS) {
+        a.GreenCtxDestroy(g);
+        return false;
+    }
+    *stream = (cudaStream_t)st;
+    *gctx_out = (void*)g;
+    *got_sms = (int)part.sm.smCount;
+    return true;
+}
+}  // namespace
 
 enum Stage { ST_INDEX = 0, ST_QKV, ST_ATTN, ST_OPROJ, ST_MLP, ST_TARGET, ST_GRAM, ST_SOLVE, ST_NEXT, ST_COUNT };
 static const char* kStageNames[ST_COUNT] = {"S0 index check + compaction", "S1-S2 norm + QKV + RoPE",
@@ -21,6 +103,9 @@ static const char* kStageNames[ST_COUNT] = {"S0 index check + compaction", "S1-S
                                             "S9 next states"};
 
 constexpr int kMaxStackLayers = 128;
+constexpr int kRing = 3;                    // teacher blocks in flight ahead of the student (ring slots of aF, zF, hF)
+constexpr int kRingX = kRing + 2;           // ring of the teacher's next states: read again after the student's solve
+constexpr int kDefaultReserveSms = 12;      // SMs the teacher stream leaves to the student and the solve (stack driver)
 
 struct Carver {
     char* base;
@@ -66,10 +151,10 @@ struct Buffers {
     float* xs[4];   // stack states, ping-pong: xF a/b, xC a/b
     // overlapped stack driver (tensor-core engine): teacher outputs of two blocks in flight, the state
     // difference xF - xC (ping-pong), per-layer status words and kept-set offsets
-    float* ringA[2];   // aF [N][Dq]
-    float* ringZ[2];   // zF [N][d]
-    float* ringH[2];   // hF [N][F]
-    float* ringX[2];   // xF_next [N][d]
+    float* ringA[kRing];   // aF [N][Dq]
+    float* ringZ[kRing];   // zF [N][d]
+    float* ringH[kRing];   // hF [N][F]
+    float* ringX[kRingX];  // xF_next [N][d]
     float* dxbuf[2];   // [N][d]
     DevStatus* lstatus;    // [kMaxStackLayers]
     int32_t* lhead_off;    // [kMaxStackLayers][Hkv+1]
@@ -94,7 +179,9 @@ struct pkv_ctx {
     int32_t* host_lhead;     // pinned: per-layer kept-set offsets of a stack call
     DevStatus* host_lstatus; // pinned: per-layer status words of a stack call
     cudaStream_t tstream;    // teacher stream of the overlapped stack driver
-    cudaEvent_t evTea[2], evStu[2], evSetup;
+    void* tgreen;            // green context that owns the teacher stream's SM partition (or null)
+    int teacher_sms;         // SMs the teacher stream may use (sm_count when not partitioned)
+    cudaEvent_t evTea[kRing], evStu[kRing], evSetup;
     int64_t launches;
     int teacher_timed;
     void* map_cache;
@@ -175,13 +262,13 @@ static size_t carve(Buffers* b, char* base, const pkv_dims* d, int engine, int e
     b->D = c.take<float>(N * dm);
     for (int i = 0; i < 4; ++i) b->xs[i] = c.take<float>(N * dm);
     if (engine != PKV_ENGINE_SIMT) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kRing; ++i) {
             b->ringA[i] = c.take<float>(N * Dq);
             b->ringZ[i] = c.take<float>(N * dm);
             b->ringH[i] = c.take<float>(N * F);
-            b->ringX[i] = c.take<float>(N * dm);
-            b->dxbuf[i] = c.take<float>(N * dm);
         }
+        for (int i = 0; i < kRingX; ++i) b->ringX[i] = c.take<float>(N * dm);
+        for (int i = 0; i < 2; ++i) b->dxbuf[i] = c.take<float>(N * dm);
         b->lstatus = c.take<DevStatus>(kMaxStackLayers);
         b->lhead_off = c.take<int32_t>((size_t)kMaxStackLayers * (d->Hkv + 1));
         c.off = pkv::tc_carve(&b->tc, base, c.off, d, dual);
@@ -273,13 +360,22 @@ extern "C" int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* o
     }
     if (c->engine != PKV_ENGINE_SIMT) {
         if (cudaMallocHost((void**)&c->host_lhead, (size_t)kMaxStackLayers * (dims->Hkv + 1) * sizeof(int32_t)) != cudaSuccess ||
-            cudaMallocHost((void**)&c->host_lstatus, (size_t)kMaxStackLayers * sizeof(DevStatus)) != cudaSuccess ||
-            cudaStreamCreateWithFlags(&c->tstream, cudaStreamNonBlocking) != cudaSuccess) {
+            cudaMallocHost((void**)&c->host_lstatus, (size_t)kMaxStackLayers * sizeof(DevStatus)) != cudaSuccess) {
             cudaGetLastError();
             pkv_destroy(c);
             return PKV_ERR_NOMEM;
         }
-        for (int i = 0; i < 2; ++i) {
+        // teacher stream: on all SMs but a reserve (see the note at the top of this file), else ordinary
+        c->teacher_sms = c->sm_count;
+        const int reserve = (opts && opts->reserve_sms != 0) ? opts->reserve_sms : kDefaultReserveSms;
+        if (reserve > 0 && reserve < c->sm_count)
+            make_partition_stream(c->sm_count - reserve, &c->tstream, &c->tgreen, &c->teacher_sms);
+        if (!c->tstream && cudaStreamCreateWithFlags(&c->tstream, cudaStreamNonBlocking) != cudaSuccess) {
+            cudaGetLastError();
+            pkv_destroy(c);
+            return PKV_ERR_NOMEM;
+        }
+        for (int i = 0; i < kRing; ++i) {
             cudaEventCreateWithFlags(&c->evTea[i], cudaEventDisableTiming);
             cudaEventCreateWithFlags(&c->evStu[i], cudaEventDisableTiming);
         }
@@ -308,7 +404,8 @@ extern "C" void pkv_destroy(pkv_ctx* c) {
     if (c->host_lhead) cudaFreeHost(c->host_lhead);
     if (c->host_lstatus) cudaFreeHost(c->host_lstatus);
     if (c->tstream) { cudaStreamSynchronize(c->tstream); cudaStreamDestroy(c->tstream); }
-    for (int i = 0; i < 2; ++i) {
+    if (c->tgreen) green_api().GreenCtxDestroy((CUgreenCtx)c->tgreen);
+    for (int i = 0; i < kRing; ++i) {
         if (c->evTea[i]) cudaEventDestroy(c->evTea[i]);
         if (c->evStu[i]) cudaEventDestroy(c->evStu[i]);
     }
@@ -341,6 +438,7 @@ extern "C" int pkv_set_timing(pkv_ctx* c, int on) {
 }
 
 extern "C" int64_t pkv_launch_count(const pkv_ctx* c) { return c ? c->launches : 0; }
+extern "C" int pkv_teacher_sm_count(const pkv_ctx* c) { return c ? c->teacher_sms : 0; }
 
 extern "C" const char* pkv_strerror(int code) {
     switch (code) {
@@ -691,9 +789,12 @@ static void fill_stats(pkv_ctx* c, const DevStatus& s, pkv_stats* stats, const i
 }
 
 // Stack driver with the teacher run ahead (tensor-core engine).  The teacher stream of Algorithm 1 never sees
-// a patch, so the teacher half of block l+1 (and l+2) runs on its own CUDA stream beside the student half and
-// the latency-bound ridge solve of block l.  Teacher outputs live in a ring of two slots; the student carries
-// the state difference xF - xC itself, so that it never reads a teacher state that may already be overwritten.
+// a patch, so the teacher half of blocks l+1 .. l+kRing runs on its own CUDA stream beside the student half and
+// the latency-bound ridge solve of block l.  Teacher outputs aF, zF, hF live in a ring of kRing slots which the
+// student releases as soon as its forward has read them (before its solve); the teacher's next states sit in a
+// longer ring because the student reads them once more after the solve (stream order makes kRing + 2 slots
+// enough: the teacher of block l + kRing + 2 starts after the student forward of block l + 2).  The student
+// carries the state difference xF - xC itself.
 static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv_block_weights* w, const pkv_kv* full,
                                   const pkv_kv_compressed* cb, const pkv_ref* ref0, float lambda, int mode,
                                   float* const* dW, const pkv_ref_next* final, pkv_stats* stats) {
@@ -725,10 +826,19 @@ static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv
     cudaEventRecord(c->evSetup, S);
     cudaStreamWaitEvent(T, c->evSetup, 0);
 
+    // optional timeline (environment variable PKV_STACK_TRACE=1): five timed events per block, printed to stderr
+    const bool trace = getenv("PKV_STACK_TRACE") != nullptr;
+    std::vector<cudaEvent_t> tev;
+    if (trace) {
+        tev.resize((size_t)n_layers * 5);
+        for (auto& e : tev) cudaEventCreate(&e);
+    }
+    auto tmark = [&](int l, int i, cudaStream_t st) { if (trace) cudaEventRecord(tev[(size_t)l * 5 + i], st); };
+
     const float* xF_in = ref0->xF;
     const float* xC_in = ref0->xC;
     for (int l = first; l < n_layers; ++l) {
-        const int k = l - first, slot = k & 1, pp = k & 1;
+        const int k = l - first, slot = k % kRing, pp = k & 1;
         const bool last = (l == n_layers - 1);
         DevStatus* st = b.lstatus + l;
         const int32_t* hoff = b.lhead_off + (size_t)l * (Hkv + 1);
@@ -742,20 +852,25 @@ static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv
         fa.status = st; fa.dual = c->dual; fa.kv_split = c->kv_split;
         fa.precise_stats = pkv::tc_well_conditioned(lambda, mode) ? 0 : 1;
         // ---- teacher half of block l on the teacher stream ----
-        if (k >= 2) cudaStreamWaitEvent(T, c->evStu[slot], 0);        // slot free: student of block l-2 is done
+        if (k >= kRing) cudaStreamWaitEvent(T, c->evStu[slot], 0);    // slot free: student forward of block l-kRing is done
         fa.xF = xF_in; fa.xC = xF_in;
-        float* xFn = (last && final) ? final->xF_next : b.ringX[slot];
+        float* xFn = (last && final) ? final->xF_next : b.ringX[k % kRingX];
+        tmark(l, 0, T);
         rc = pkv::tc_teacher_forward(lcT, &b.tc, &c->dims, fa, xFn);
         if (rc != PKV_OK) break;
         cudaEventRecord(c->evTea[slot], T);
+        tmark(l, 1, T);
         // ---- student half, statistics, solve, next student state on the caller's stream ----
         const void *Kc, *Vc;
         stage_compact(c, lcS, &full[l], &cb[l], totals[l], &Kc, &Vc, hoff, st);
         fa.Kc = Kc; fa.Vc = Vc; fa.bias = cb[l].idx ? nullptr : cb[l].bias;
         fa.xC = xC_in; fa.dx = b.dxbuf[pp];
         cudaStreamWaitEvent(S, c->evTea[slot], 0);
+        tmark(l, 2, S);
         rc = pkv::tc_student_forward(lcS, &b.tc, &c->dims, fa);
         if (rc != PKV_OK) break;
+        cudaEventRecord(c->evStu[slot], S);                           // aF, zF, hF of this slot are no longer needed
+        tmark(l, 3, S);
         if (c->dual) {
             rc = pkv::tc_dual_solve(lcS, &b.tc, &c->dims, N, b.R, lambda, mode, dW[l], st);
             if (rc != PKV_OK) break;
@@ -768,7 +883,7 @@ static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv
         sumsq(lcS, Dn, (int64_t)N * d, &st->res_fro2);
         float* xCn = (last && final) ? final->xC_next : b.xs[2 + (1 - pp)];
         sub_f32(lcS, xFn, Dn, (int64_t)N * d, xCn);
-        cudaEventRecord(c->evStu[slot], S);
+        tmark(l, 4, S);
         xF_in = xFn;
         xC_in = xCn;
     }
@@ -776,6 +891,17 @@ static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv
     cudaMemcpyAsync(c->host_lstatus, b.lstatus, (size_t)n_layers * sizeof(DevStatus), cudaMemcpyDeviceToHost, S);
     cudaError_t e = cudaStreamSynchronize(S);
     cudaError_t e2 = cudaStreamSynchronize(T);
+    if (trace) {
+        if (e == cudaSuccess && e2 == cudaSuccess && rc == PKV_OK) {
+            fprintf(stderr, "block: teacher start..end | student start, forward end, solve+next end (ms since the first teacher)\n");
+            for (int l = first; l < n_layers; ++l) {
+                float t[5];
+                for (int i = 0; i < 5; ++i) cudaEventElapsedTime(&t[i], tev[(size_t)first * 5], tev[(size_t)l * 5 + i]);
+                fprintf(stderr, "%3d: %8.3f .. %8.3f | %8.3f %8.3f %8.3f\n", l, t[0], t[1], t[2], t[3], t[4]);
+            }
+        }
+        for (auto& ev : tev) cudaEventDestroy(ev);
+    }
     if (e != cudaSuccess) return cuda_fail(c, e, "stream synchronize");
     if (e2 != cudaSuccess) return cuda_fail(c, e2, "teacher stream synchronize");
     e = cudaGetLastError();

@@ -37,6 +37,8 @@ struct TcGemm {
     float alpha;
     bool accumulate, lower_only;
     int k_tri;      // 0: dense; 1: B lower triangular (skip k tiles past the row); 2: B upper triangular
+    bool skip_tile00;     // leave the first tile (rows and columns [0,128) of the product) alone
+    bool out_col0_only;   // write the bf16 parts only for the first 128-column block of the product
     int nacc;       // 0/1: one fp32 accumulator; 2 or 4: the hi x hi pass of a split product is accumulated apart
                     // from the cross passes (and in several parts), which removes most of the tensor core's
                     // truncation bias from sums of same-signed terms; pass 0 must be the hi x hi pass
@@ -64,7 +66,10 @@ struct TcSolveBuffers {
     __nv_bfloat16* Z2[3];
     int nmax;              // largest system the arrays are sized for
     cudaStream_t aux;      // high-priority helper stream of the factorisation's critical chain
-    cudaEvent_t ev[3];
+    cudaEvent_t ev[4];
+    CUtensorMap chainP[3], chainX[3];   // tensor maps of the chain kernel's operands, valid for (chain_n, chain_ld)
+    int chain_n, chain_ld;
+    long long* stamps;     // phase marks of the chain kernel (profiling aid)
 };
 void tc_solve_destroy(TcSolveBuffers* t);
 size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, int nmax, int dmax);

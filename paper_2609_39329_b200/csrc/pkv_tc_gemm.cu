@@ -42,6 +42,8 @@ struct alignas(64) GemmTcParams {
     int nout, out_col_off;
     int accumulate, lower_only, k_tri, vec_ok;
     int nacc;                 // TMEM accumulators per tile (1, 2 or 4), see TcGemm::nacc
+    int skip_tile00;          // the tile at (blockIdx.x, blockIdx.y) = (0, 0) is left alone
+    int out_col0_only;        // bf16 parts are written by the tiles of the first block column only
     DevStatus* status;
 };
 
@@ -64,6 +66,7 @@ template <int BN, bool PRE>
 __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcParams p) {
     const int m0 = blockIdx.y * 128, n0 = blockIdx.x * BN, z = blockIdx.z;
     if (p.lower_only && n0 > m0 + 127) return;
+    if (p.skip_tile00 && blockIdx.x == 0 && blockIdx.y == 0) return;
     pdl_launch_dependents();
     // absolute coordinates of this tile's output; tiles entirely outside the stored region do nothing
     const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
@@ -253,7 +256,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                         }
                     }
                 }
-                if (p.nout > 0) {
+                if (p.nout > 0 && (!p.out_col0_only || blockIdx.x == 0)) {
                     // bf16 parts: through the warp's smem tile so that a warp writes 64 contiguous bytes per row
 #pragma unroll
                     for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = v[j];
@@ -466,7 +469,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     const long long tiles256 = (long long)((g.N + 255) / 256) * ((g.M + 127) / 128) * g.batch;
     const bool wide = g.N >= 512 && tiles256 >= 2 * 148 && !(g.C && g.accumulate) && !g.lower_only && g.k_tri != 2 &&
                       g.nacc < 4;
-    const int BN = (g.N <= 64) ? 64 : (wide ? 256 : 128);
+    const int BN = (g.skip_tile00 || g.out_col0_only) ? 128 : ((g.N <= 64) ? 64 : (wide ? 256 : 128));
     MapCache* cache = (MapCache*)lc.map_cache;
     // distinct operands
     const __nv_bfloat16* da[3];
@@ -504,6 +507,8 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     p.accumulate = g.accumulate ? 1 : 0;
     p.lower_only = g.lower_only ? 1 : 0;
     p.k_tri = g.k_tri;
+    p.skip_tile00 = g.skip_tile00 ? 1 : 0;
+    p.out_col0_only = g.out_col0_only ? 1 : 0;
     // several accumulators only for products with one hi x hi pass and cross passes, and only if they fit
     p.nacc = 1;
     if (g.nacc > 1 && g.npass >= 2 && p.pa[0] == 0 && p.pb[0] == 0) {

@@ -4,13 +4,16 @@
 // six passes (hh, hm, mh, hl, lh, mm) into fp32 tensor-memory accumulators, which reproduces an
 // fp32 product to ~2^-24; the two large triangular products at the end use pairs (three passes).
 //
-//   1. blocked right-looking Cholesky G = L L^T, block 128: the diagonal block is factored and
-//      inverted by one CTA in shared memory (k_potrf128), the panel is a GEMM with the block
-//      inverse, the trailing update a GEMM on the lower triangle;
+//   1. blocked right-looking Cholesky G = L L^T, block 128: one CTA per block column (k_chain128)
+//      applies the previous column's update to the diagonal block, factors it and inverts the factor
+//      in shared memory; the panel (a GEMM with the block inverse) and the trailing update (a GEMM on
+//      the lower triangle) of every column run beside that chain;
 //   2. X = L^{-1} by recursive doubling from the 128-block inverses:
 //      [A 0; C B]^{-1} = [A^{-1} 0; -B^{-1} C A^{-1}  B^{-1}], every level two batched GEMMs;
 //   3. dW = (S_T X^T) X, two GEMMs that skip the zero tiles of the triangular factor.
 #include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include "pkv_ptx.cuh"
 #include "pkv_tc.h"
@@ -104,55 +107,240 @@ __device__ __forceinline__ void warp_tile_tf32x6(float (&c)[4], int kb, int ke, 
     else warp_tile_tf32<false>(c, kb, ke, lane, fa, fb);
 }
 constexpr int kPotrfTElems = 64 * 65;       // largest doubling temporary (one 64 x 64 block, padded)
-constexpr int kPotrfSmemBytes = (2 * PB * LDS + PB + kPotrfTElems) * (int)sizeof(float);
 
 __device__ __forceinline__ uint32_t pack_bf16(__nv_bfloat16 a, __nv_bfloat16 b) {
     return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
 }
 
-__global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restrict__ G, int n, int ld, int k0, Trip X3,
-                                                            Trip XT3, int six_i, DevStatus* status) {
-    const bool six = six_i != 0;
-    extern __shared__ float smf[];
-    float(*A)[LDS] = reinterpret_cast<float(*)[LDS]>(smf);
-    float(*X)[LDS] = reinterpret_cast<float(*)[LDS]>(smf + PB * LDS);
-    float* rd = smf + 2 * PB * LDS;              // [128] reciprocals of the factor's diagonal
-    float* T = rd + PB;                          // doubling temporary
-    pdl_launch_dependents();
-    pdl_wait();
+// ---------------------------------------------------------------------------------------------
+// One step of the factorisation's critical chain, one CTA:
+//   L_{k,k-1} = G~_{k,k-1} inv(L_{k-1,k-1})^T                      (tensor cores, bf16 triples from global)
+//   A         = G~_{kk} + lambda I - L_{k,k-1} L_{k,k-1}^T        (tensor cores; G~ updated by columns < k-1)
+//   A = L_kk L_kk^T, inv(L_kk)                                     (shared memory, warp shuffles, TF32 warp tiles)
+// Everything else of block column k-1 (the rest of the panel, the trailing update) runs beside this kernel
+// in ordinary GEMM launches; only this kernel sits between consecutive diagonal blocks.
+//
+// Shared memory (dynamic, 1 KB aligned), reused by phase:
+//   R1  96 KB  operand triple of G~_{k,k-1} (TMA, 128B swizzle)  ->  triple of L_{k,k-1}  ->  X (inverse, fp32) + T
+//   R2  96 KB  triple of inv(L_{k-1,k-1}) (TMA)                 ->  A (fp32) + reciprocal diagonal
+// Tensor memory: four 128-column accumulators (hi x hi pass in three parts, cross passes apart; see the
+// note on truncating accumulation in pkv_tc_gemm.cu).
+// ---------------------------------------------------------------------------------------------
+struct alignas(64) ChainParams {
+    CUtensorMap mP[3];        // panel operand parts  [n][128]  (rows of G~ column k-1)
+    CUtensorMap mX[3];        // parts of the block-diagonal inverse [n][ld]
+    const float* G;
+    int n, ld, k0;
+    Trip X3, XT3;
+    int six;
+    DevStatus* status;
+    long long* stamps;        // optional [blocks][kChainStamps] clock64 marks of thread 0 (phase profile), or null
+};
+
+constexpr int kChainStamps = 16;
+constexpr int kChainR = 3 * 128 * 128 * 2;                 // 96 KB: one operand triple
+constexpr int kChainBar = 2 * kChainR;
+constexpr int kChainSmemBytes = kChainBar + 64 + 1024;
+static_assert(PB * LDS * 4 + kPotrfTElems * 4 <= kChainR, "X and T must fit in R1");
+static_assert(PB * LDS * 4 + PB * 4 <= kChainR, "A and rd must fit in R2");
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+__global__ void __launch_bounds__(kPotrfThreads) k_chain128(const __grid_constant__ ChainParams p) {
+    using namespace ptx;
+    const float* __restrict__ G = p.G;
+    const int n = p.n, ld = p.ld, k0 = p.k0;
+    const Trip X3 = p.X3, XT3 = p.XT3;
+    DevStatus* status = p.status;
+    const bool six = p.six != 0;
+    extern __shared__ uint8_t chain_smem_raw[];
+    const uint32_t raw = smem_u32(chain_smem_raw);
+    const uint32_t sbase = (raw + 1023u) & ~1023u;
+    uint8_t* sm = chain_smem_raw + (sbase - raw);
+    float(*A)[LDS] = reinterpret_cast<float(*)[LDS]>(sm + kChainR);                 // R2
+    float* rd = reinterpret_cast<float*>(sm + kChainR + PB * LDS * 4);              // [128] reciprocals of the factor's diagonal
+    float(*X)[LDS] = reinterpret_cast<float(*)[LDS]>(sm);                           // R1
+    float* T = reinterpret_cast<float*>(sm + PB * LDS * 4);                         // doubling temporary
+    const uint32_t bar_tma = sbase + kChainBar, bar_mma = sbase + kChainBar + 8;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + kChainBar + 16);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* skip_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    {   // one thread reads the status word: the whole CTA takes the same branch
-        __shared__ int s_skip;
-        if (tid == 0) s_skip = status->code;
-        __syncthreads();
-        if (s_skip != 0) return;
+    const bool with_update = k0 > 0;
+    long long* stamps = p.stamps ? p.stamps + (size_t)(k0 / PB) * kChainStamps : nullptr;
+    auto stamp = [&](int i) { if (stamps && tid == 0) stamps[i] = clock64(); };
+    stamp(0);
+
+    pdl_launch_dependents();
+    if (tid == 0) {
+        mbar_init(bar_tma, 1);
+        mbar_init(bar_mma, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
     }
+    if (warp == 1 && with_update) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = with_update ? *tmem_slot : 0u;
+    pdl_wait();
+    if (tid == 0) *skip_flag = status->code;      // one thread reads the status word: the whole CTA takes the same branch
+    __syncthreads();
+    const bool skip = *skip_flag != 0;
+    stamp(1);
     const int nbk = min(PB, n - k0);
     const float lam = status->lam;
-    // ---- load the lower part (identity outside the block's extent), lambda on the diagonal ----
-    if (nbk == PB && (ld & 3) == 0) {
-        constexpr int kLd = 4096 / kPotrfThreads;
-        float4 v[kLd];
+    bool ok = !skip;
+
+    if (ok && with_update) {
+        // ---- operands by TMA: parts of G~_{k,k-1} (rows k0.., the panel operand array) and of inv(L_{k-1,k-1})
+        if (tid == 0) {
+            mbar_expect_tx(bar_tma, 2 * kChainR);
 #pragma unroll
-        for (int u = 0; u < kLd; ++u) {
-            const int i = tid + u * kPotrfThreads;           // 4096 float4 of the block
-            const int r = i >> 5, c4 = (i & 31) * 4;
-            v[u] = (c4 <= r) ? *reinterpret_cast<const float4*>(G + (size_t)(k0 + r) * ld + k0 + c4)
-                             : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int i = 0; i < 3; ++i)
+#pragma unroll
+                for (int sb = 0; sb < 2; ++sb) {
+                    tma_load_2d(sbase + i * 32768 + sb * 16384, &p.mP[i], bar_tma, sb * 64, k0);
+                    tma_load_2d(sbase + kChainR + i * 32768 + sb * 16384, &p.mX[i], bar_tma, k0 - PB + sb * 64, k0 - PB);
+                }
         }
+        const int npass = six ? 6 : 3;
+        const int ia[6] = {0, 0, 1, 0, 2, 1}, ib[6] = {0, 1, 0, 2, 0, 1};
+        constexpr uint32_t idesc = idesc_bf16(128, 128);
+        // product `which`: 0: R1 x R2^T (panel block), 1: R1 x R1^T (its Gram)
+        auto issue = [&](int which) {
+            uint32_t used = 0u, hh = 0u;
+            for (int ps = 0; ps < npass; ++ps) {
+                const uint32_t pa = sbase + ia[ps] * 32768;
+                const uint32_t pb = (which == 0 ? sbase + kChainR : sbase) + ib[ps] * 32768;
+                const bool big = ps == 0;
 #pragma unroll
-        for (int u = 0; u < kLd; ++u) {
-            const int i = tid + u * kPotrfThreads;
-            const int r = i >> 5, c4 = (i & 31) * 4;
-            const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                const int c = c4 + t;
-                A[r][c] = (c < r) ? e[t] : ((c == r) ? e[t] + lam : 0.f);
-                X[r][c] = 0.f;
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (uint32_t)(kk >> 2) * 16384u;
+                    const uint32_t acc = big ? 1u + (hh++ % 3u) : 0u;
+                    mma_bf16_ss(tbase + acc * 128u, smem_desc_sw128(pa + off) + (uint64_t)((kk & 3) * 2),
+                                smem_desc_sw128(pb + off) + (uint64_t)((kk & 3) * 2), idesc, (used >> acc) & 1u);
+                    used |= 1u << acc;
+                }
+            }
+            mma_commit(bar_mma);
+        };
+        if (warp == 1 && lane == 0) {
+            if (mbar_wait(bar_tma, 0, abort_flag, status, 40)) {
+                tc_fence_after();
+                issue(0);
             }
         }
-    } else {
+        // ---- L_{k,k-1}: accumulators -> fp32 -> bf16 triple in R1 (the operand triple there is dead once the
+        //      MMAs have completed).  Warps 0..15: lane quarter = warp & 3, 32 columns each.
+        const int q = warp & 3, cb = warp >> 2;
+        const int row = q * 32 + lane;
+        ok = mbar_wait(bar_mma, 0, abort_flag, status, 41);
+        tc_fence_after();
+        stamp(2);
+        if (ok && warp < 16) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int c0 = cb * 32 + half * 16;
+                uint32_t r[16], r2[16];
+                const uint32_t ta = tbase + ((uint32_t)(q * 32) << 16) + (uint32_t)c0;
+                tmem_ld16(ta, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int a = 1; a < 4; ++a) {
+                    tmem_ld16(ta + (uint32_t)(a * 128), r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                }
+                // 16 columns = two 16-byte chunks per part; chunk index inside the 64-column sub-tile is XOR-swizzled
+                const int sb = c0 >> 6, ch0 = (c0 & 63) >> 3;
+#pragma unroll
+                for (int ch = 0; ch < 2; ++ch) {
+                    uint32_t hv[4], mv[4], lv[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        __nv_bfloat16 h0, m0, l0, h1, m1, l1;
+                        const float v0 = (row < nbk) ? __uint_as_float(r[ch * 8 + 2 * e]) : 0.f;
+                        const float v1 = (row < nbk) ? __uint_as_float(r[ch * 8 + 2 * e + 1]) : 0.f;
+                        split3(v0, h0, m0, l0);
+                        split3(v1, h1, m1, l1);
+                        hv[e] = pack_bf16(h0, h1); mv[e] = pack_bf16(m0, m1); lv[e] = pack_bf16(l0, l1);
+                    }
+                    uint8_t* dst = sm + sb * 16384 + row * 128 + (((ch0 + ch) ^ (row & 7)) << 4);
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(hv[0], hv[1], hv[2], hv[3]);
+                    *reinterpret_cast<uint4*>(dst + 32768) = make_uint4(mv[0], mv[1], mv[2], mv[3]);
+                    *reinterpret_cast<uint4*>(dst + 65536) = make_uint4(lv[0], lv[1], lv[2], lv[3]);
+                }
+            }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        ok = *abort_flag == 0;
+        if (ok && warp == 1 && lane == 0) issue(1);
+        ok = ok && mbar_wait(bar_mma, 1, abort_flag, status, 42);
+        tc_fence_after();
+        stamp(3);
+        // ---- A = G~_kk + lambda I - L L^T (lower part; identity outside the block's extent) into R2
+        if (ok && warp < 16) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int c0 = cb * 32 + half * 16;
+                float g[16];
+                const bool inrow = row < nbk;
+                if (nbk == PB && c0 <= row && (ld & 3) == 0) {   // 16-byte loads; entries right of the diagonal are not used
+                    const float4* gp = reinterpret_cast<const float4*>(G + (size_t)(k0 + row) * ld + k0 + c0);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float4 v = (c0 + 4 * j <= row) ? gp[j] : make_float4(0.f, 0.f, 0.f, 0.f);
+                        g[4 * j] = v.x; g[4 * j + 1] = v.y; g[4 * j + 2] = v.z; g[4 * j + 3] = v.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int c = c0 + j;
+                        g[j] = (inrow && c <= row) ? G[(size_t)(k0 + row) * ld + k0 + c] : 0.f;
+                    }
+                }
+                uint32_t r[16], r2[16];
+                const uint32_t ta = tbase + ((uint32_t)(q * 32) << 16) + (uint32_t)c0;
+                tmem_ld16(ta, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int a = 1; a < 4; ++a) {
+                    tmem_ld16(ta + (uint32_t)(a * 128), r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int c = c0 + j;
+                    float v = (row == c) ? 1.f : 0.f;
+                    if (inrow && c <= row) v = (g[j] - __uint_as_float(r[j])) + ((c == row) ? lam : 0.f);
+                    A[row][c] = v;
+                }
+            }
+        } else if (ok) {
+            // the other warps clear X (R1: the triple of L is dead, its MMAs have completed)
+            for (int i = tid - 512; i < PB * PB; i += kPotrfThreads - 512) X[i >> 7][i & 127] = 0.f;
+        }
+        __syncthreads();
+    } else if (ok) {
+        // ---- first block: the lower part from global memory (identity outside the block's extent), lambda on the diagonal
         for (int i = tid; i < PB * PB; i += kPotrfThreads) {
             const int r = i >> 7, c = i & 127;
             float v = (r == c) ? 1.f : 0.f;
@@ -163,32 +351,46 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
             A[r][c] = v;
             X[r][c] = 0.f;
         }
+        __syncthreads();
     }
-    __syncthreads();
+    stamp(4);
+    if (ok) {
     float minpiv = INFINITY;
     int bad_col = -1;
-    // 16 x 16 diagonal piece at c0, factored by warp 0 entirely in registers
-    auto diag16 = [&](int c0) {
-        const int li = lane & 15;            // lanes 16..31 mirror lanes 0..15 so every shuffle source is live
-        float a[SB];
+    // 16 x 16 diagonal piece at c0 in registers of warp 0: lane i (and its mirror i + 16, so that every shuffle
+    // source is live) holds row i, already loaded into a[].  Two pivots per round: the 2 x 2 leading block is
+    // factored redundantly by every lane from three shuffled values, which halves the number of dependent
+    // shuffle / rsqrt rounds of the pivot chain.
+    auto diag16 = [&](int c0, float (&a)[SB]) {
 #pragma unroll
-        for (int k = 0; k < SB; ++k) a[k] = A[c0 + li][c0 + k];
+        for (int j = 0; j < SB; j += 2) {
+            float p00 = __shfl_sync(0xffffffffu, a[j], j);
+            const float p10 = __shfl_sync(0xffffffffu, a[j], j + 1);
+            const float p11 = __shfl_sync(0xffffffffu, a[j + 1], j + 1);
+            const bool ok0 = (p00 > 0.f) && (p00 < INFINITY);
+            if (!ok0 && bad_col < 0 && c0 + j < nbk) bad_col = c0 + j;
+            p00 = ok0 ? p00 : 1.f;
+            float r0 = rsqrtf(p00);
+            r0 = r0 * fmaf(-0.5f * p00 * r0, r0, 1.5f);         // one Newton step: full fp32 accuracy
+            const float l10 = p10 * r0;
+            float q = fmaf(-l10, l10, p11);
+            const bool ok1 = (q > 0.f) && (q < INFINITY);
+            if (!ok1 && bad_col < 0 && c0 + j + 1 < nbk) bad_col = c0 + j + 1;
+            q = ok1 ? q : 1.f;
+            if (c0 + j < nbk) minpiv = fminf(minpiv, p00);
+            if (c0 + j + 1 < nbk) minpiv = fminf(minpiv, q);
+            float r1 = rsqrtf(q);
+            r1 = r1 * fmaf(-0.5f * q * r1, r1, 1.5f);
+            const float x0 = a[j] * r0;                         // column j of L, this lane's row
+            const float x1 = fmaf(-x0, l10, a[j + 1]) * r1;     // column j + 1 (row j holds an unused value there)
+            a[j] = x0;
+            a[j + 1] = x1;
+            if (lane == j) { rd[c0 + j] = r0; rd[c0 + j + 1] = r1; }
 #pragma unroll
-        for (int j = 0; j < SB; ++j) {
-            float piv = __shfl_sync(0xffffffffu, a[j], j);
-            const bool okp = (piv > 0.f) && (piv < INFINITY);
-            if (!okp && bad_col < 0 && c0 + j < nbk) bad_col = c0 + j;
-            piv = okp ? piv : 1.f;
-            if (c0 + j < nbk) minpiv = fminf(minpiv, piv);
-            float rdj = rsqrtf(piv);
-            rdj = rdj * fmaf(-0.5f * piv * rdj, rdj, 1.5f);    // one Newton step: full fp32 accuracy
-            const float lij = a[j] * rdj;                       // row li of column j (the pivot row gets sqrt(piv))
-            a[j] = lij;
-            if (lane == j) rd[c0 + j] = rdj;
-#pragma unroll
-            for (int k = j + 1; k < SB; ++k) {
-                const float lkj = __shfl_sync(0xffffffffu, lij, k);
-                a[k] = fmaf(-lij, lkj, a[k]);                  // rows above the diagonal hold unused values
+            for (int k = j + 2; k < SB; ++k) {
+                const float y0 = __shfl_sync(0xffffffffu, x0, k);
+                const float y1 = __shfl_sync(0xffffffffu, x1, k);
+                a[k] = fmaf(-x1, y1, fmaf(-x0, y0, a[k]));      // rows above the diagonal hold unused values
             }
         }
         if (lane < SB) {
@@ -209,8 +411,16 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
         A[i0 + g + 8][n0 + 2 * t] -= c[2];
         A[i0 + g + 8][n0 + 2 * t + 1] -= c[3];
     };
-    if (warp == 0) diag16(0);
+    long long d_fs = 0, d_up = 0, d_dg = 0, d_sy = 0, tq = clock64();
+    auto lap = [&](long long& acc) { if (stamps) { const long long now = clock64(); acc += now - tq; tq = now; } };
+    if (warp == 0) {
+        float a[SB];
+#pragma unroll
+        for (int k = 0; k < SB; ++k) a[k] = A[lane & 15][k];
+        diag16(0, a);
+    }
     __syncthreads();
+    lap(d_dg);
     for (int c0 = 0; c0 < PB; c0 += SB) {
         const int base = c0 + SB;
         if (tid < PB - base) {     // rows below: x L_ss^T = a by forward substitution, one row per thread
@@ -229,19 +439,39 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
             for (int c = 0; c < SB; ++c) A[r][c0 + c] = a[c];
         }
         __syncthreads();
+        lap(d_fs);
         if (base < PB) {
-            // trailing update of the lower triangle inside the block (16 x 8 warp tiles, K = the 16 new
-            // columns).  Warp 0 takes the next diagonal piece first and factors it right away, beside the
-            // other warps' tiles: the serial pivot chain is off the critical path.
+            // Trailing update of the lower triangle inside the block (K = the 16 new columns).  Warp 0 owns the
+            // next diagonal piece: it applies the update to that 16 x 16 block in fp32 registers (each half-warp
+            // sums eight of the sixteen columns) and factors it right away, beside the other warps' tiles: the
+            // serial pivot chain never waits for them.
             if (warp == 0) {
-                trail_tile(c0, base, base);
-                trail_tile(c0, base, base + 8);
-                __syncwarp();
-                diag16(base);
-            } else {
+                const int li = lane & 15, kh = (lane >> 4) * 8;
+                float own[8], acc[SB];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) own[k] = A[base + li][c0 + kh + k];
+#pragma unroll
+                for (int m = 0; m < SB; ++m) {
+                    float sacc = 0.f;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) sacc = fmaf(own[k], A[base + m][c0 + kh + k], sacc);
+                    acc[m] = sacc;
+                }
+                float a[SB];
+#pragma unroll
+                for (int m = 0; m < SB; ++m) {
+                    acc[m] += __shfl_xor_sync(0xffffffffu, acc[m], 16);
+                    a[m] = A[base + li][base + m] - acc[m];
+                }
+                lap(d_up);
+                diag16(base, a);
+                lap(d_dg);
+            } else if ((warp & 3) != 0) {
+                // warps 4, 8, ... share warp 0's scheduler: they stay out of the way of the pivot chain
                 const int rem = PB - base;
                 const int tm = (rem >> 4) - 1, tn = rem >> 3;          // row tiles below the first one
-                for (int tile = warp - 1; tile < tm * tn; tile += kPotrfThreads / 32 - 1) {
+                const int wi = warp - 1 - (warp >> 2);                  // index among the 24 working warps
+                for (int tile = wi; tile < tm * tn; tile += 24) {
                     const int i0 = base + 16 + (tile / tn) * 16, n0 = base + (tile % tn) * 8;
                     if (n0 > i0 + 15) continue;                     // entirely above the diagonal
                     trail_tile(c0, i0, n0);
@@ -249,7 +479,9 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
             }
         }
         __syncthreads();
+        lap(d_sy);
     }
+    if (stamps && tid == 0) { stamps[8] = d_fs; stamps[9] = d_up; stamps[10] = d_dg; stamps[11] = d_sy; }
     if (tid == 0) {
         status->min_pivot = fminf(status->min_pivot, minpiv);
         if (bad_col >= 0) {
@@ -263,79 +495,127 @@ __global__ void __launch_bounds__(kPotrfThreads) k_potrf128(const float* __restr
             }
         }
     }
-    // ---- inverse of the factor ----
+    stamp(5);
+    // ---- inverse of the factor (plain fp32 FMAs: exact roundings, no operand splitting) ----
     if (tid < PB) {      // 16 x 16 diagonal sub-blocks, one column per thread
         const int o = (tid >> 4) * SB, c = tid & 15;
         float x[SB];
 #pragma unroll
         for (int i = 0; i < SB; ++i) {
-            float s = (i == c) ? 1.f : 0.f;
+            float sacc = (i == c) ? 1.f : 0.f;
 #pragma unroll
-            for (int k = 0; k < i; ++k) s = fmaf(-A[o + i][o + k], x[k], s);
-            x[i] = (i < c) ? 0.f : s * rd[o + i];
+            for (int k = 0; k < i; ++k) sacc = fmaf(-A[o + i][o + k], x[k], sacc);
+            x[i] = (i < c) ? 0.f : sacc * rd[o + i];
         }
 #pragma unroll
         for (int i = 0; i < SB; ++i) X[o + i][o + c] = x[i];
     }
     __syncthreads();
-    // recursive doubling inside the block: [Xa 0; C Xb] -> bottom-left = -Xb (C Xa); every level is two
-    // dense products over all pairs, done as 16 x 8 warp tiles
-    for (int s = SB; s < PB; s *= 2) {
-        const int lt = s + 1;
-        const int tn = s >> 3, tpp = (s >> 4) * tn, ntile = (PB / (2 * s)) * tpp;
-        for (int tile = warp; tile < ntile; tile += kPotrfThreads / 32) {      // T_p = C_p Xa_p
-            const int p = tile / tpp, i0 = ((tile % tpp) / tn) * 16, n0 = ((tile % tpp) % tn) * 8;
-            const int o = 2 * p * s;
-            float c[4] = {0.f, 0.f, 0.f, 0.f};
-            warp_tile_tf32x6(c, n0, s, lane, six,                  // Xa is lower triangular: rows k >= column n
-                             [&](int i, int k) { return A[o + s + i0 + i][o + k]; },
-                             [&](int k, int n) { return X[o + k][o + n0 + n]; });
-            const int g = lane >> 2, t = lane & 3;
-            float* tp = T + (p * s + i0 + g) * lt + n0 + 2 * t;
-            tp[0] = c[0]; tp[1] = c[1];
-            tp[8 * lt] = c[2]; tp[8 * lt + 1] = c[3];
+    if (stamps && tid == 0) stamps[12] = clock64();
+    // recursive doubling inside the block: [Xa 0; C Xb]^-1 has bottom-left -Xb (C Xa).  Every level is two
+    // products over all pairs; each thread owns a 4 x 4 patch of the output.
+    for (int sz = SB; sz < PB; sz *= 2) {
+        const int lt = sz + 1;
+        const int q4 = sz >> 2;                       // patches per side of one pair's block
+        const int npatch = (PB / (2 * sz)) * q4 * q4;
+        if (tid < npatch) {                           // T_p = C_p Xa_p ; Xa lower triangular: k >= n
+            const int pp = tid / (q4 * q4), rest = tid % (q4 * q4);
+            const int i0 = (rest % q4) * 4, n0 = (rest / q4) * 4, o = 2 * pp * sz;
+            float acc[4][4] = {};
+            for (int k4 = n0; k4 < sz; k4 += 4) {      // n0 and sz are multiples of 4: four steps with all loads up front
+                float av[4][4], bv[4][4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) av[u][r] = A[o + sz + i0 + r][o + k4 + u];
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) bv[u][cc] = X[o + k4 + u][o + n0 + cc];
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int r = 0; r < 4; ++r)
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) acc[r][cc] = fmaf(av[u][r], bv[u][cc], acc[r][cc]);
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) T[(pp * sz + i0 + r) * lt + n0 + cc] = acc[r][cc];
         }
         __syncthreads();
-        for (int tile = warp; tile < ntile; tile += kPotrfThreads / 32) {      // X_p(bottom-left) = -Xb_p T_p
-            const int p = tile / tpp, i0 = ((tile % tpp) / tn) * 16, n0 = ((tile % tpp) % tn) * 8;
-            const int o = 2 * p * s;
-            float c[4] = {0.f, 0.f, 0.f, 0.f};
-            warp_tile_tf32x6(c, 0, i0 + 16, lane, six,             // Xb is lower triangular: columns k <= row
-                             [&](int i, int k) { return X[o + s + i0 + i][o + s + k]; },
-                             [&](int k, int n) { return T[(p * s + k) * lt + n0 + n]; });
-            const int g = lane >> 2, t = lane & 3;
-            X[o + s + i0 + g][o + n0 + 2 * t] = -c[0];
-            X[o + s + i0 + g][o + n0 + 2 * t + 1] = -c[1];
-            X[o + s + i0 + g + 8][o + n0 + 2 * t] = -c[2];
-            X[o + s + i0 + g + 8][o + n0 + 2 * t + 1] = -c[3];
+        if (tid < npatch) {                           // X_p(bottom-left) = -Xb_p T_p ; Xb lower triangular: k <= i
+            const int pp = tid / (q4 * q4), rest = tid % (q4 * q4);
+            const int i0 = (rest % q4) * 4, n0 = (rest / q4) * 4, o = 2 * pp * sz;
+            float acc[4][4] = {};
+            for (int k4 = 0; k4 < i0 + 4; k4 += 4) {
+                float av[4][4], bv[4][4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) av[u][r] = X[o + sz + i0 + r][o + sz + k4 + u];
+#pragma unroll
+                    for (int cc = 0; cc < 4; ++cc) bv[u][cc] = T[(pp * sz + k4 + u) * lt + n0 + cc];
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int r = 0; r < 4; ++r)
+#pragma unroll
+                        for (int cc = 0; cc < 4; ++cc) acc[r][cc] = fmaf(av[u][r], bv[u][cc], acc[r][cc]);
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) X[o + sz + i0 + r][o + n0 + cc] = -acc[r][cc];
         }
         __syncthreads();
+        if (stamps && tid == 0) stamps[12 + (sz == 16 ? 1 : (sz == 32 ? 2 : 3))] = clock64();
     }
-    // ---- write the inverse and its transpose as bf16 triples, two columns per thread ----
-    for (int i = tid; i < PB * PB / 2; i += kPotrfThreads) {
-        const int r = i >> 6, c = (i & 63) * 2;
-        if (r < nbk && c < nbk) {
-            const size_t o = (size_t)(k0 + r) * ld + k0 + c;
-            __nv_bfloat16 h0, m0, l0, h1, m1, l1;
-            split3((c <= r) ? X[r][c] : 0.f, h0, m0, l0);
-            split3((c + 1 <= r) ? X[r][c + 1] : 0.f, h1, m1, l1);
-            if (c + 1 < nbk) {
-                *reinterpret_cast<uint32_t*>(X3.a[0] + o) = pack_bf16(h0, h1);
-                *reinterpret_cast<uint32_t*>(X3.a[1] + o) = pack_bf16(m0, m1);
-                *reinterpret_cast<uint32_t*>(X3.a[2] + o) = pack_bf16(l0, l1);
-            } else {
-                X3.a[0][o] = h0; X3.a[1][o] = m0; X3.a[2][o] = l0;
+    stamp(6);
+    // ---- write the inverse as bf16 triples, eight columns (16 bytes per part) per thread; chunks right of the
+    //      diagonal stay zero (cleared once, never written).  The transposed copy is made off the chain.
+    if (nbk == PB && (ld & 7) == 0) {
+        for (int i = tid; i < PB * PB / 8; i += kPotrfThreads) {
+            const int r = i >> 4, c8 = (i & 15) * 8;
+            if (c8 > r) continue;
+            const size_t o = (size_t)(k0 + r) * ld + k0 + c8;
+            uint32_t hv[4], mv[4], lv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int c = c8 + 2 * e;
+                const float v0 = (c <= r) ? X[r][c] : 0.f, v1 = (c + 1 <= r) ? X[r][c + 1] : 0.f;
+                __nv_bfloat16 h0, m0, l0, h1, m1, l1;
+                split3(v0, h0, m0, l0);
+                split3(v1, h1, m1, l1);
+                hv[e] = pack_bf16(h0, h1); mv[e] = pack_bf16(m0, m1); lv[e] = pack_bf16(l0, l1);
             }
-            split3((r <= c) ? X[c][r] : 0.f, h0, m0, l0);
-            split3((r <= c + 1) ? X[c + 1][r] : 0.f, h1, m1, l1);
-            if (c + 1 < nbk) {
-                *reinterpret_cast<uint32_t*>(XT3.a[0] + o) = pack_bf16(h0, h1);
-                *reinterpret_cast<uint32_t*>(XT3.a[1] + o) = pack_bf16(m0, m1);
-                *reinterpret_cast<uint32_t*>(XT3.a[2] + o) = pack_bf16(l0, l1);
-            } else {
-                XT3.a[0][o] = h0; XT3.a[1][o] = m0; XT3.a[2][o] = l0;
+            *reinterpret_cast<uint4*>(X3.a[0] + o) = make_uint4(hv[0], hv[1], hv[2], hv[3]);
+            *reinterpret_cast<uint4*>(X3.a[1] + o) = make_uint4(mv[0], mv[1], mv[2], mv[3]);
+            *reinterpret_cast<uint4*>(X3.a[2] + o) = make_uint4(lv[0], lv[1], lv[2], lv[3]);
+        }
+    } else {
+        for (int i = tid; i < PB * PB; i += kPotrfThreads) {
+            const int r = i >> 7, c = i & 127;
+            if (r < nbk && c <= r) {
+                const size_t o = (size_t)(k0 + r) * ld + k0 + c;
+                __nv_bfloat16 h, m, l;
+                split3(X[r][c], h, m, l);
+                X3.a[0][o] = h; X3.a[1][o] = m; X3.a[2][o] = l;
             }
         }
+    }
+    }      // ok
+    stamp(7);
+    // teardown: after an abort give copies in flight time to land before the CTA's smem is released
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1 && with_update) {
+        tc_fence_after();
+        tmem_dealloc(tbase, 512);
     }
 }
 
@@ -359,6 +639,28 @@ static void launch_split3(const Lc& lc, const float* src, long long lds, int row
     if (!n) return;
     k_split3<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(src, lds, rows, cols, out, ldo, nout);
     lc.count();
+}
+
+// Diagonal blocks: XT3[k0 + c][k0 + r] = X3[k0 + r][k0 + c] for the 128-blocks on the diagonal (clipped to n x n).
+__global__ void k_transpose_diag(Trip X3, Trip XT3, int n, int ld) {
+    __shared__ __nv_bfloat16 t[3][32][33];
+    const int k0 = blockIdx.z * PB;
+    const int r0 = k0 + blockIdx.y * 32, c0 = k0 + blockIdx.x * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int r = r0 + j, c = c0 + threadIdx.x;
+        if (r < n && c < n) {
+#pragma unroll
+            for (int a = 0; a < 3; ++a) t[a][j][threadIdx.x] = X3.a[a][(size_t)r * ld + c];
+        }
+    }
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int c = c0 + j, r = r0 + threadIdx.x;
+        if (r < n && c < n) {
+#pragma unroll
+            for (int a = 0; a < 3; ++a) XT3.a[a][(size_t)c * ld + r] = t[a][threadIdx.x][j];
+        }
+    }
 }
 
 // XT3[2sz + c][s + 2sz + r] = X3[s + 2sz + r][2sz + c]   (r < s clipped to the n x n matrix, c < s); row stride ld
@@ -464,6 +766,7 @@ size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, int nmax, int d
         t->S2[i] = (__nv_bfloat16*)take(dm * F * 2);
         t->Z2[i] = (__nv_bfloat16*)take(dm * F * 2);
     }
+    t->stamps = (long long*)take(((F + PB - 1) / PB) * kChainStamps * sizeof(long long));
     return off;
 }
 
@@ -482,12 +785,13 @@ int tc_solve_init(TcSolveBuffers* t) {
     // the factorisation's critical chain (diagonal block, panel, next-column update) runs at the highest
     // priority so that its small kernels are not queued behind the bulk trailing update's CTAs
     if (cudaStreamCreateWithPriority(&t->aux, cudaStreamNonBlocking, greatest) != cudaSuccess) return PKV_ERR_CUDA;
-    for (int i = 0; i < 3; ++i)
+    for (int i = 0; i < 4; ++i)
         if (cudaEventCreateWithFlags(&t->ev[i], cudaEventDisableTiming) != cudaSuccess) return PKV_ERR_CUDA;
+    t->chain_n = t->chain_ld = 0;
     static PerDeviceOnce once;
     int dev;
     if (once.needed(&dev)) {
-        if (cudaFuncSetAttribute(k_potrf128, cudaFuncAttributeMaxDynamicSharedMemorySize, kPotrfSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(k_chain128, cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmemBytes) != cudaSuccess)
             return PKV_ERR_CUDA;
         once.mark(dev);
     }
@@ -500,26 +804,25 @@ void tc_solve_destroy(TcSolveBuffers* t) {
         cudaStreamDestroy(t->aux);
         t->aux = nullptr;
     }
-    for (int i = 0; i < 3; ++i)
+    for (int i = 0; i < 4; ++i)
         if (t->ev[i]) {
             cudaEventDestroy(t->ev[i]);
             t->ev[i] = nullptr;
         }
 }
 
-static void launch_potrf(cudaStream_t st, int smem, const float* G, int n, int ld, int k0, Trip X3, Trip XT3, int six,
-                         DevStatus* status) {
+static int launch_chain(cudaStream_t st, const ChainParams& cp) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(1);
     cfg.blockDim = dim3(kPotrfThreads);
-    cfg.dynamicSmemBytes = smem;
+    cfg.dynamicSmemBytes = kChainSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, k_potrf128, G, n, ld, k0, X3, XT3, six, status);
+    return cudaLaunchKernelEx(&cfg, k_chain128, cp) == cudaSuccess ? PKV_OK : PKV_ERR_CUDA;
 }
 
 int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
@@ -527,7 +830,6 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
                         __nv_bfloat16* const* S_T_triple) {
     const int F = n;      // dimension of the system; ld is the row stride of G, S_T, dW and of every n x n work array
     const int nblk = (F + PB - 1) / PB;
-    const int smem = kPotrfSmemBytes;
     Trip L3{{t->L3[0], t->L3[1], t->L3[2]}}, X3{{t->X3[0], t->X3[1], t->X3[2]}}, XT3{{t->XT3[0], t->XT3[1], t->XT3[2]}};
     Trip P3{{t->P3[0], t->P3[1], t->P3[2]}}, TT3{{t->TT3[0], t->TT3[1], t->TT3[2]}};
     int rc;
@@ -538,25 +840,50 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
             cudaMemsetAsync(t->XT3[i], 0, (size_t)n * ld * 2, lc.st);
         }
     }
-    // ---- 1. factorisation with look-ahead ----
-    // Per block column b:  panel N_b (L21 = G21 L11^{-T});  T1_b = update of the next block column only
-    // (its epilogue also leaves the bf16 triple of the updated column in P3, the next panel's operand);
-    // T2_b = update of everything to the right, on the helper stream, beside the next diagonal block.
-    // sA: critical chain on the high-priority helper stream; sB: bulk updates on the caller's stream
+    // ---- 1. factorisation ----
+    // Critical chain (high-priority helper stream sA): one k_chain128 per block column, which applies column
+    // k-1's update to the diagonal block itself, factors it and inverts the factor.  Beside it, on the caller's
+    // stream sB, the bulk of every column: P_k = the panel L_{r,k} = G~_{r,k} inv(L_kk)^T for all rows below
+    // (kept as a bf16 triple), U_k = the trailing update by column k of everything except the next diagonal
+    // block (which the chain kernel does not read back from memory); U_k's first block column also leaves
+    // the bf16 triple of the updated column k+1, the operand of P_{k+1} and of the next chain kernel.
+    //   chain(k)  needs chain(k-1) and U_{k-2};   P_k needs chain(k) and U_{k-1};   U_k needs P_k.
     cudaStream_t sA = t->aux, sB = lc.st;
-    Lc lcA{sA, lc.launches, lc.map_cache, true};
     Lc lcB{sB, lc.launches, lc.map_cache};
-    cudaEventRecord(t->ev[2], sB);
-    cudaStreamWaitEvent(sA, t->ev[2], 0);
-    launch_potrf(sA, smem, G, n, ld, 0, X3, XT3, well_conditioned ? 0 : 1, status);
-    lc.count();
-    if (F > PB) launch_split3(lcA, G + (size_t)PB * ld, ld, F - PB, PB, Trip{{P3.a[0] + (size_t)PB * PB, P3.a[1] + (size_t)PB * PB, P3.a[2] + (size_t)PB * PB}}, PB, 3);
-    bool t2_pending = false;
+    if (t->chain_n != n || t->chain_ld != ld) {
+        for (int i = 0; i < 3; ++i) {
+            if ((rc = tc_make_map_2d(&t->chainP[i], P3.a[i], F, PB, PB, 128))) return rc;
+            if ((rc = tc_make_map_2d(&t->chainX[i], X3.a[i], F, F, ld, 128))) return rc;
+        }
+        t->chain_n = n;
+        t->chain_ld = ld;
+    }
+    ChainParams cp;
+    for (int i = 0; i < 3; ++i) { cp.mP[i] = t->chainP[i]; cp.mX[i] = t->chainX[i]; }
+    cp.G = G; cp.n = n; cp.ld = ld; cp.X3 = X3; cp.XT3 = XT3; cp.six = well_conditioned ? 0 : 1; cp.status = status;
+    // phase profile of the chain kernel (environment variable PKV_SOLVE_TRACE=1): clock64 marks, printed to stderr
+    static const bool trace = getenv("PKV_SOLVE_TRACE") != nullptr;
+    cp.stamps = trace ? t->stamps : nullptr;
+    cudaEvent_t evFork = t->ev[0], evF = t->ev[1];
+    cudaEvent_t evU[2] = {t->ev[2], t->ev[3]};
+    cudaEventRecord(evFork, sB);
+    cudaStreamWaitEvent(sA, evFork, 0);
+    if (F > PB) {
+        launch_split3(lcB, G + (size_t)PB * ld, ld, F - PB, PB,
+                      Trip{{P3.a[0] + (size_t)PB * PB, P3.a[1] + (size_t)PB * PB, P3.a[2] + (size_t)PB * PB}}, PB, 3);
+        cudaEventRecord(evU[1], sB);
+    }
     rc = PKV_OK;
     for (int b = 0; b < nblk && rc == PKV_OK; ++b) {
         const int k0 = b * PB, k1 = min(F, k0 + PB), rem = F - k1;
+        if (b > 0) cudaStreamWaitEvent(sA, evU[b & 1], 0);       // U_{b-2}, or the split of the first column for b = 1
+        cp.k0 = k0;
+        if ((rc = launch_chain(sA, cp))) break;
+        lc.count();
+        cudaEventRecord(evF, sA);
         if (rem <= 0) break;
-        {   // N_b: panel, kept as a bf16 triple in L3
+        cudaStreamWaitEvent(sB, evF, 0);
+        {   // P_b: panel, kept as a bf16 triple in L3
             TcGemm g{};
             six_pass(g, P3, PB, F, PB, X3, ld, F, F);
             g.a_row0 = k1;
@@ -564,50 +891,65 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
             g.M = rem; g.N = PB; g.K = PB; g.batch = 1; g.alpha = 1.f;
             g.c_row0 = k1; g.c_col0 = k0; g.c_rows = F; g.c_cols = F;
             g.out[0] = L3.a[0]; g.out[1] = L3.a[1]; g.out[2] = L3.a[2]; g.ldo = ld; g.nout = 3;
-            if ((rc = gemm_tc(lcA, g, status))) break;
+            if ((rc = gemm_tc(lcB, g, status))) break;
         }
-        cudaEventRecord(t->ev[0], sA);
-        cudaStreamWaitEvent(sB, t->ev[0], 0);
-        if (t2_pending) cudaStreamWaitEvent(sA, t->ev[1], 0);      // T2_{b-1} also updated this column
-        {   // T1_b: next block column of G22 -= L21 L21^T, and its bf16 triple for the next panel
+        if (rem > PB) {   // U_b: G22 -= L21 L21^T on the lower triangle, the first diagonal tile left to the chain
             TcGemm g{};
             six_pass(g, L3, ld, F, F, L3, ld, F, F);
             g.a_row0 = k1; g.a_col0 = k0; g.b_row0 = k1; g.b_col0 = k0;
-            g.M = rem; g.N = min(PB, rem); g.K = PB; g.batch = 1; g.alpha = -1.f;
-            g.C = const_cast<float*>(G); g.ldc = ld; g.accumulate = true;
+            g.M = rem; g.N = rem; g.K = PB; g.batch = 1; g.alpha = -1.f;
+            g.C = const_cast<float*>(G); g.ldc = ld; g.accumulate = true; g.lower_only = true; g.skip_tile00 = true;
             g.c_row0 = k1; g.c_col0 = k1; g.c_rows = F; g.c_cols = F;
             g.out[0] = P3.a[0]; g.out[1] = P3.a[1]; g.out[2] = P3.a[2]; g.ldo = PB; g.nout = 3; g.out_col_off = k1;
-            if ((rc = gemm_tc(lcA, g, status))) break;
-        }
-        const int rem2 = rem - PB;
-        if (rem2 > 0) {   // T2_b on the helper stream
-            TcGemm g{};
-            six_pass(g, L3, ld, F, F, L3, ld, F, F);
-            g.a_row0 = k1 + PB; g.a_col0 = k0; g.b_row0 = k1 + PB; g.b_col0 = k0;
-            g.M = rem2; g.N = rem2; g.K = PB; g.batch = 1; g.alpha = -1.f;
-            g.C = const_cast<float*>(G); g.ldc = ld; g.accumulate = true; g.lower_only = true;
-            g.c_row0 = k1 + PB; g.c_col0 = k1 + PB; g.c_rows = F; g.c_cols = F;
+            g.out_col0_only = true;
             if ((rc = gemm_tc(lcB, g, status))) break;
-            cudaEventRecord(t->ev[1], sB);
-            t2_pending = true;
-        } else {
-            t2_pending = false;
         }
-        launch_potrf(sA, smem, G, n, ld, k1, X3, XT3, well_conditioned ? 0 : 1, status);
-        lc.count();
+        cudaEventRecord(evU[b & 1], sB);
     }
     // join: the caller's stream continues after the chain's last kernel
-    cudaEventRecord(t->ev[0], sA);
-    cudaStreamWaitEvent(sB, t->ev[0], 0);
+    cudaEventRecord(evF, sA);
+    cudaStreamWaitEvent(sB, evF, 0);
     if (rc != PKV_OK) return rc;
+    {   // transposed copies of the diagonal-block inverses (the chain kernel writes only X3)
+        dim3 grid(PB / 32, PB / 32, nblk), block(32, 8);
+        k_transpose_diag<<<grid, block, 0, lc.st>>>(X3, XT3, n, ld);
+        lc.count();
+    }
+    if (trace && nblk <= 64) {
+        static long long host_stamps[64 * kChainStamps];
+        cudaStreamSynchronize(sB);
+        cudaMemcpy(host_stamps, t->stamps, (size_t)nblk * kChainStamps * sizeof(long long), cudaMemcpyDeviceToHost);
+        double acc[kChainStamps] = {0};
+        for (int b = 1; b < nblk; ++b)
+            for (int i = 1; i < kChainStamps; ++i) acc[i] += (double)(host_stamps[b * kChainStamps + i] - host_stamps[b * kChainStamps + i - 1]);
+        fprintf(stderr, "chain kernel phases, mean cycles over blocks 1..%d: setup+wait %.0f | tma+mma1 %.0f | L->smem+mma2 %.0f | "
+                        "A write %.0f | factor %.0f | inverse %.0f | output %.0f ; start-to-start %.0f\n", nblk - 1,
+                acc[1] / (nblk - 1), acc[2] / (nblk - 1), acc[3] / (nblk - 1), acc[4] / (nblk - 1), acc[5] / (nblk - 1),
+                acc[6] / (nblk - 1), acc[7] / (nblk - 1),
+                nblk > 2 ? (double)(host_stamps[(nblk - 1) * kChainStamps] - host_stamps[kChainStamps]) / (nblk - 2) : 0.0);
+        fprintf(stderr, "   start-to-start / busy cycles per block:");
+        for (int b = 1; b < nblk; ++b)
+            fprintf(stderr, " %lld/%lld", (host_stamps[b * kChainStamps] - host_stamps[(b - 1) * kChainStamps]) / 1000,
+                    (host_stamps[b * kChainStamps + 7] - host_stamps[b * kChainStamps]) / 1000);
+        fprintf(stderr, " (thousands)\n");
+        const long long* h1 = host_stamps + kChainStamps;
+        fprintf(stderr, "   block 1, factor phase (cycles): forward substitution+sync %lld | warp 0 update %lld | diagonal pieces %lld | "
+                        "wait for the other warps %lld ; inverse: 16x16 pieces %lld | level 16 %lld | 32 %lld | 64 %lld\n",
+                h1[8], h1[9], h1[10], h1[11], h1[12] - h1[5], h1[13] - h1[12], h1[14] - h1[13], h1[15] - h1[14]);
+
+    }
     // ---- 2. X = L^{-1} by recursive doubling ----
+    // cond(L) = sqrt(cond(G)): with a well-conditioned ridge matrix (a few tens) the rounding of these products
+    // (pairs: 2^-16) reaches dW unamplified and three passes are enough; the factorisation above always takes six
+    // (its trailing updates cancel)
     for (int s = PB; s < F; s *= 2) {
         int P = 0;
         while ((2 * P + 1) * s < F) ++P;
         if (P == 0) break;
         {   // TT_p = A_p^{-T} C_p^T   (A^{-1} the finished top-left inverse, C the block of L below it)
             TcGemm g{};
-            six_pass(g, XT3, ld, F, F, L3, ld, F, F);
+            if (well_conditioned) three_pass(g, XT3, ld, F, F, L3, ld, F, F);
+            else six_pass(g, XT3, ld, F, F, L3, ld, F, F);
             g.a_zrow = 2 * s; g.a_zcol = 2 * s;
             g.b_row0 = s; g.b_zrow = 2 * s; g.b_zcol = 2 * s;
             g.M = s; g.N = s; g.K = s; g.batch = P; g.alpha = 1.f;
@@ -617,7 +959,8 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         }
         {   // X_p(bottom-left) = -B_p^{-1} TT_p^T
             TcGemm g{};
-            six_pass(g, X3, ld, F, F, TT3, s, (long long)P * s, s);
+            if (well_conditioned) three_pass(g, X3, ld, F, F, TT3, s, (long long)P * s, s);
+            else six_pass(g, X3, ld, F, F, TT3, s, (long long)P * s, s);
             g.a_row0 = s; g.a_col0 = s; g.a_zrow = 2 * s; g.a_zcol = 2 * s;
             g.b_zrow = s;
             g.M = s; g.N = s; g.K = s; g.batch = P; g.alpha = -1.f;
@@ -640,7 +983,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         if (nsp == 2) three_pass(g, S2, ld, d, F, X3, ld, F, F);
         else six_pass(g, S2, ld, d, F, X3, ld, F, F);
         g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 1;
-        g.nacc = 2;      // long contraction, no cancellation: two accumulators keep two CTAs per SM
+        g.nacc = well_conditioned ? 1 : 2;      // long contraction, no cancellation; one accumulator keeps two CTAs per SM
         g.c_rows = d; g.c_cols = F;
         g.out[0] = Z2.a[0]; g.out[1] = Z2.a[1]; g.out[2] = Z2.a[2]; g.ldo = ld; g.nout = nsp;
         if ((rc = gemm_tc(lc, g, status))) return rc;
@@ -650,7 +993,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         if (nsp == 2) three_pass(g, Z2, ld, d, F, XT3, ld, F, F);
         else six_pass(g, Z2, ld, d, F, XT3, ld, F, F);
         g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 2;
-        g.nacc = 2;
+        g.nacc = well_conditioned ? 1 : 2;
         g.C = dW; g.ldc = ld; g.c_rows = d; g.c_cols = F;
         if (dW_pair) { g.out[0] = dW_pair->hi; g.out[1] = dW_pair->lo; g.ldo = ld; g.nout = 2; }
         if ((rc = gemm_tc(lc, g, status))) return rc;
