@@ -201,6 +201,20 @@ int pkv_build_stack(pkv_ctx* ctx, int n_layers, int first_layer, const pkv_block
                     float lambda, int lambda_mode, float* const* dW, const pkv_ref_next* final,
                     pkv_stats* stats);
 
+/* Algorithm 1 for several ridge coefficients on the same context and reference set (the ridge-scale ablation
+ * sweeps lambda0).  The teacher stream of Algorithm 1 sees neither a patch nor lambda, so it is run once: its
+ * per-block outputs (attention output, residual term, MLP features, next state: N (Hq hd + 2 d + F) floats per
+ * block) are kept in `teacher_cache`, a caller-owned device buffer of at least pkv_teacher_cache_bytes(), and the
+ * student half, the statistics and the solve of every block are then run once per coefficient.
+ * dW: HOST array of n_lambda * n_layers device pointers, entry [j * n_layers + l] = patch of block l for
+ * lambdas[j]; stats: NULL or n_lambda * n_layers entries in the same order.  Both streams start from ref0->xF
+ * / ref0->xC.  Tensor-core engine only.  Errors as pkv_build_stack; PKV_ERR_NOMEM if the cache is too small. */
+size_t pkv_teacher_cache_bytes(const pkv_dims* dims, int n_layers, int N);
+int pkv_build_stack_sweep(pkv_ctx* ctx, int n_layers, const pkv_block_weights* w, const pkv_kv* full,
+                          const pkv_kv_compressed* cb, const pkv_ref* ref0, int n_lambda, const float* lambdas,
+                          int lambda_mode, float* const* dW, void* teacher_cache, size_t cache_bytes,
+                          pkv_stats* stats);
+
 /* ---- single stages, exported for unit parity tests and per-kernel measurement ---- */
 
 /* Index check + compaction of a kept-index set (bit-exact): Kc[i] = K[h][idx[i]], same for V.
@@ -268,6 +282,15 @@ int pkv_selftest_bounded_wait(pkv_ctx* ctx, int32_t* site);
 
 /* Enable (1) / disable (0) per-stage CUDA-event timing into pkv_stats.stage_ms. */
 int pkv_set_timing(pkv_ctx* ctx, int on);
+
+/* pkv_build_stack scheduling: 0 = default (teacher run ahead where it applies), 1 = strictly block by block on
+ * the context's stream (what stage timing also forces); for measuring one against the other. */
+int pkv_set_stack_schedule(pkv_ctx* ctx, int schedule);
+
+/* Measures the device's fp32 fused-multiply-add rate (TFLOP/s, two flops per FMA) with a register-resident FMA
+ * kernel timed by CUDA events on the context's stream: the denominator for the ridge solve's roofline, which
+ * stands for fp32 arithmetic.  Uses the context's workspace as scratch; synchronises the stream. */
+int pkv_measure_fma_peak(pkv_ctx* ctx, double* tflops);
 
 /* Number of kernels the context launched since creation (for launch accounting). */
 int64_t pkv_launch_count(const pkv_ctx* ctx);

@@ -105,6 +105,12 @@ def lib() -> C.CDLL:
     L.pkv_build_stack.argtypes = [C.c_void_p, C.c_int, C.c_int, P(pkv_block_weights), P(pkv_kv),
                                   P(pkv_kv_compressed), P(pkv_ref), C.c_float, C.c_int, P(C.c_void_p),
                                   P(pkv_ref_next), P(pkv_stats)]
+    L.pkv_teacher_cache_bytes.restype = C.c_size_t
+    L.pkv_teacher_cache_bytes.argtypes = [P(pkv_dims), C.c_int, C.c_int]
+    L.pkv_build_stack_sweep.restype = C.c_int
+    L.pkv_build_stack_sweep.argtypes = [C.c_void_p, C.c_int, P(pkv_block_weights), P(pkv_kv), P(pkv_kv_compressed),
+                                        P(pkv_ref), C.c_int, P(C.c_float), C.c_int, P(C.c_void_p), C.c_void_p,
+                                        C.c_size_t, P(pkv_stats)]
     L.pkv_gather_kept.restype = C.c_int
     L.pkv_gather_kept.argtypes = [C.c_void_p, P(pkv_kv), P(C.c_int32), C.c_void_p, C.c_void_p, C.c_void_p,
                                   P(C.c_int32), P(C.c_int32)]
@@ -127,6 +133,10 @@ def lib() -> C.CDLL:
     L.pkv_set_timing.argtypes = [C.c_void_p, C.c_int]
     L.pkv_launch_count.restype = C.c_int64
     L.pkv_launch_count.argtypes = [C.c_void_p]
+    L.pkv_set_stack_schedule.restype = C.c_int
+    L.pkv_set_stack_schedule.argtypes = [C.c_void_p, C.c_int]
+    L.pkv_measure_fma_peak.restype = C.c_int
+    L.pkv_measure_fma_peak.argtypes = [C.c_void_p, P(C.c_double)]
     L.pkv_teacher_sm_count.restype = C.c_int
     L.pkv_teacher_sm_count.argtypes = [C.c_void_p]
     for f in ("pkv_strerror", "pkv_stage_name"):
@@ -201,6 +211,17 @@ class PkvContext:
 
     def launch_count(self) -> int:
         return int(self.L.pkv_launch_count(self.h))
+
+    def set_stack_schedule(self, sequential: bool):
+        self.L.pkv_set_stack_schedule(self.h, 1 if sequential else 0)
+
+    def measure_fma_peak(self) -> float:
+        """pkv_measure_fma_peak: fp32 FMA TFLOP/s of the device (CUDA-event timed FMA kernel)."""
+        v = C.c_double(0.0)
+        rc = self.L.pkv_measure_fma_peak(self.h, C.byref(v))
+        if rc != 0:
+            self._raise(rc)
+        return float(v.value)
 
     def teacher_sm_count(self) -> int:
         return int(self.L.pkv_teacher_sm_count(self.h))
@@ -293,6 +314,34 @@ class PkvContext:
         if rc != 0:
             self._raise(rc)
         return {"dW": dWs, "xF_final": xFn, "xC_final": xCn, "stats": [s.as_dict() for s in ST]}
+
+    def build_stack_sweep(self, layers, xF0, xC0, chunk_off, pos0, lams, mode=LAMBDA_PAPER, cache=None):
+        """pkv_build_stack_sweep: every block's patch for each ridge coefficient in `lams`, the teacher run once.
+        Returns dict(dW = [per lambda][per layer], stats likewise).  `cache`: optional uint8 CUDA tensor of at
+        least pkv_teacher_cache_bytes (allocated here otherwise)."""
+        torch = self.torch
+        n, nl = len(layers), len(lams)
+        N = int(xF0.shape[0])
+        d, F = self.dims.d, self.dims.F
+        need = int(self.L.pkv_teacher_cache_bytes(C.byref(self.dims), n, N))
+        if cache is None:
+            cache = torch.empty(need, dtype=torch.uint8, device=xF0.device)
+        W = (pkv_block_weights * n)(*[self.weights_struct(l["w"]) for l in layers])
+        KV = (pkv_kv * n)(*[pkv_kv(_ptr(l["K"]), _ptr(l["V"])) for l in layers])
+        cbs = [self.compressed_struct(l["head_off"], l.get("idx"), l.get("Kc"), l.get("Vc"), l.get("bias"))
+               for l in layers]
+        CB = (pkv_kv_compressed * n)(*cbs)
+        co = _i32(chunk_off)
+        ref = pkv_ref(_ptr(xF0), _ptr(xC0), N, len(chunk_off) - 1, C.cast(co, C.POINTER(C.c_int32)), int(pos0))
+        dWs = [[torch.empty((d, F), dtype=torch.float32, device=xF0.device) for _ in range(n)] for _ in range(nl)]
+        DW = (C.c_void_p * (n * nl))(*[_ptr(t) for row in dWs for t in row])
+        ST = (pkv_stats * (n * nl))()
+        LAM = (C.c_float * nl)(*[float(v) for v in lams])
+        rc = self.L.pkv_build_stack_sweep(self.h, n, W, KV, CB, C.byref(ref), nl, LAM, int(mode), DW, _ptr(cache),
+                                          int(cache.numel()), ST)
+        if rc != 0:
+            self._raise(rc)
+        return {"dW": dWs, "stats": [[ST[j * n + l].as_dict() for l in range(n)] for j in range(nl)], "cache": cache}
 
     # ---- single stages ----
     def gather_kept(self, K, V, head_off, idx):

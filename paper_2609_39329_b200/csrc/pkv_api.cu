@@ -183,6 +183,7 @@ struct pkv_ctx {
     int teacher_sms;         // SMs the teacher stream may use (sm_count when not partitioned)
     cudaEvent_t evTea[kRing], evStu[kRing], evSetup;
     int64_t launches;
+    int force_sequential;    // pkv_build_stack: 1 = block by block on one stream even where the overlapped driver applies
     int teacher_timed;
     void* map_cache;
     int timing;
@@ -439,6 +440,19 @@ extern "C" int pkv_set_timing(pkv_ctx* c, int on) {
 
 extern "C" int64_t pkv_launch_count(const pkv_ctx* c) { return c ? c->launches : 0; }
 extern "C" int pkv_teacher_sm_count(const pkv_ctx* c) { return c ? c->teacher_sms : 0; }
+
+extern "C" int pkv_set_stack_schedule(pkv_ctx* c, int schedule) {
+    if (!c || (schedule != 0 && schedule != 1)) return PKV_ERR_INVALID_ARG;
+    c->force_sequential = schedule;
+    return PKV_OK;
+}
+
+extern "C" int pkv_measure_fma_peak(pkv_ctx* c, double* tflops) {
+    if (!c || !tflops) return PKV_ERR_INVALID_ARG;
+    cudaStreamSynchronize(c->st);
+    // scratch: the activation buffer u (2 N d floats) is always large enough for one store per thread
+    return fma_peak_tflops(c->st, c->b.gu, (size_t)2 * c->dims.N_max * 2 * c->dims.F, c->sm_count, tflops);
+}
 
 extern "C" const char* pkv_strerror(int code) {
     switch (code) {
@@ -795,9 +809,19 @@ static void fill_stats(pkv_ctx* c, const DevStatus& s, pkv_stats* stats, const i
 // longer ring because the student reads them once more after the solve (stream order makes kRing + 2 slots
 // enough: the teacher of block l + kRing + 2 starts after the student forward of block l + 2).  The student
 // carries the state difference xF - xC itself.
+//
+// Teacher cache (ridge-coefficient sweeps): with `cache` set, the teacher outputs of every block go to their own
+// slot of that buffer instead of the rings (no slot is reused, so the teacher is never throttled), and a later
+// call with run_teacher = false replays the student half, the statistics and the solve of every block against
+// the cached teacher: the teacher of Algorithm 1 does not depend on the ridge coefficient.
+static size_t teacher_cache_floats_per_layer(const pkv_dims& D, int N) {
+    return (size_t)N * ((size_t)D.Hq * D.hd + 2 * (size_t)D.d + D.F);
+}
+
 static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv_block_weights* w, const pkv_kv* full,
                                   const pkv_kv_compressed* cb, const pkv_ref* ref0, float lambda, int mode,
-                                  float* const* dW, const pkv_ref_next* final, pkv_stats* stats) {
+                                  float* const* dW, const pkv_ref_next* final, pkv_stats* stats,
+                                  float* cache = nullptr, bool run_teacher = true) {
     const pkv_dims& D = c->dims;
     const int N = ref0->N, d = D.d, F = D.F, Hkv = D.Hkv;
     const int Dq = D.Hq * D.hd;
@@ -846,26 +870,35 @@ static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv
         fa.w = &w[l]; fa.full = &full[l];
         fa.N = N; fa.pos0 = ref0->pos0; fa.max_b = maxbs[l]; fa.total_kept = totals[l];
         fa.head_off = hoff; fa.tok_cs = b.tok_cs; fa.rope_tab = b.rope_tab;
-        fa.aF = b.ringA[slot]; fa.zF = b.ringZ[slot]; fa.hF = b.ringH[slot];
+        float* cX = nullptr;
+        if (cache) {
+            float* base_l = cache + (size_t)l * teacher_cache_floats_per_layer(D, N);
+            fa.aF = base_l; fa.zF = base_l + (size_t)N * Dq; fa.hF = fa.zF + (size_t)N * d;
+            cX = fa.hF + (size_t)N * F;
+        } else {
+            fa.aF = b.ringA[slot]; fa.zF = b.ringZ[slot]; fa.hF = b.ringH[slot];
+        }
         fa.aC = b.aC; fa.dA = b.a2 + (size_t)N * Dq;
         fa.zC = b.zC; fa.dz = b.dz; fa.hC = b.hC; fa.R = b.R; fa.S_H = b.S_H; fa.S_T = b.S_T;
         fa.status = st; fa.dual = c->dual; fa.kv_split = c->kv_split;
         fa.precise_stats = pkv::tc_well_conditioned(lambda, mode) ? 0 : 1;
         // ---- teacher half of block l on the teacher stream ----
-        if (k >= kRing) cudaStreamWaitEvent(T, c->evStu[slot], 0);    // slot free: student forward of block l-kRing is done
+        if (k >= kRing && !cache) cudaStreamWaitEvent(T, c->evStu[slot], 0);    // slot free: student forward of block l-kRing is done
         fa.xF = xF_in; fa.xC = xF_in;
-        float* xFn = (last && final) ? final->xF_next : b.ringX[k % kRingX];
+        float* xFn = cache ? cX : ((last && final) ? final->xF_next : b.ringX[k % kRingX]);
         tmark(l, 0, T);
-        rc = pkv::tc_teacher_forward(lcT, &b.tc, &c->dims, fa, xFn);
-        if (rc != PKV_OK) break;
-        cudaEventRecord(c->evTea[slot], T);
+        if (run_teacher) {
+            rc = pkv::tc_teacher_forward(lcT, &b.tc, &c->dims, fa, xFn);
+            if (rc != PKV_OK) break;
+            cudaEventRecord(c->evTea[slot], T);
+        }
         tmark(l, 1, T);
         // ---- student half, statistics, solve, next student state on the caller's stream ----
         const void *Kc, *Vc;
         stage_compact(c, lcS, &full[l], &cb[l], totals[l], &Kc, &Vc, hoff, st);
         fa.Kc = Kc; fa.Vc = Vc; fa.bias = cb[l].idx ? nullptr : cb[l].bias;
         fa.xC = xC_in; fa.dx = b.dxbuf[pp];
-        cudaStreamWaitEvent(S, c->evTea[slot], 0);
+        if (run_teacher) cudaStreamWaitEvent(S, c->evTea[slot], 0);
         tmark(l, 2, S);
         rc = pkv::tc_student_forward(lcS, &b.tc, &c->dims, fa);
         if (rc != PKV_OK) break;
@@ -883,6 +916,8 @@ static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv
         sumsq(lcS, Dn, (int64_t)N * d, &st->res_fro2);
         float* xCn = (last && final) ? final->xC_next : b.xs[2 + (1 - pp)];
         sub_f32(lcS, xFn, Dn, (int64_t)N * d, xCn);
+        if (cache && last && final)
+            cudaMemcpyAsync(final->xF_next, xFn, (size_t)N * d * sizeof(float), cudaMemcpyDeviceToDevice, S);
         tmark(l, 4, S);
         xF_in = xFn;
         xC_in = xCn;
@@ -920,7 +955,8 @@ extern "C" int pkv_build_stack(pkv_ctx* c, int n_layers, int first_layer, const 
                                int lambda_mode, float* const* dW, const pkv_ref_next* final, pkv_stats* stats) {
     if (!c || !w || !full || !cb || !ref0 || !dW || n_layers <= 0 || first_layer < 0 || first_layer >= n_layers)
         return PKV_ERR_INVALID_ARG;
-    if (c->engine != PKV_ENGINE_SIMT && !c->timing && n_layers - first_layer >= 2 && n_layers <= kMaxStackLayers)
+    if (c->engine != PKV_ENGINE_SIMT && !c->timing && !c->force_sequential && n_layers - first_layer >= 2 &&
+        n_layers <= kMaxStackLayers)
         return build_stack_overlapped(c, n_layers, first_layer, w, full, cb, ref0, lambda, lambda_mode, dW, final, stats);
     pkv_ref ref = *ref0;
     for (int l = first_layer; l < n_layers; ++l) {
@@ -939,6 +975,31 @@ extern "C" int pkv_build_stack(pkv_ctx* c, int n_layers, int first_layer, const 
         if (rc != PKV_OK) return rc;
         ref.xF = nx.xF_next;
         ref.xC = nx.xC_next;
+    }
+    return PKV_OK;
+}
+
+extern "C" size_t pkv_teacher_cache_bytes(const pkv_dims* dims, int n_layers, int N) {
+    if (dims_ok(dims) != PKV_OK || n_layers <= 0 || N <= 0) return 0;
+    return (size_t)n_layers * teacher_cache_floats_per_layer(*dims, N) * sizeof(float);
+}
+
+extern "C" int pkv_build_stack_sweep(pkv_ctx* c, int n_layers, const pkv_block_weights* w, const pkv_kv* full,
+                                     const pkv_kv_compressed* cb, const pkv_ref* ref0, int n_lambda,
+                                     const float* lambdas, int lambda_mode, float* const* dW, void* teacher_cache,
+                                     size_t cache_bytes, pkv_stats* stats) {
+    if (!c || !w || !full || !cb || !ref0 || !dW || !lambdas || !teacher_cache || n_layers <= 0 || n_lambda <= 0)
+        return PKV_ERR_INVALID_ARG;
+    if (c->engine == PKV_ENGINE_SIMT || n_layers > kMaxStackLayers) return PKV_ERR_UNSUPPORTED;
+    if (ref0->N <= 0 || ref0->N > c->dims.N_max) return PKV_ERR_INVALID_ARG;
+    if (((uintptr_t)teacher_cache & 15) || cache_bytes < pkv_teacher_cache_bytes(&c->dims, n_layers, ref0->N))
+        return PKV_ERR_NOMEM;
+    for (int j = 0; j < n_lambda; ++j) {
+        // the first coefficient runs the teacher (ahead of its students, filling the cache); the others replay
+        int rc = build_stack_overlapped(c, n_layers, 0, w, full, cb, ref0, lambdas[j], lambda_mode,
+                                        dW + (size_t)j * n_layers, nullptr, stats ? stats + (size_t)j * n_layers : nullptr,
+                                        (float*)teacher_cache, j == 0);
+        if (rc != PKV_OK) return rc;
     }
     return PKV_OK;
 }

@@ -102,6 +102,7 @@ void make_ridge_matrix(const Lc& lc, const float* S_H, int F, float lam0, int mo
 // out = a - b (n elements); out may alias a.
 void sub_f32(const Lc& lc, const float* a, const float* b, int64_t n, float* out);
 void merge_weights(const Lc& lc, void* W, int w_dtype, const float* dW, int64_t count);
+int fma_peak_tflops(cudaStream_t st, float* scratch, size_t scratch_floats, int sm_count, double* tflops);
 
 // ---- pkv_solve.cu ----------------------------------------------------------------------
 struct SolveWs {

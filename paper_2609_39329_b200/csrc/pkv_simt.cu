@@ -740,4 +740,43 @@ void merge_weights(const Lc& lc, void* W, int w_dtype, const float* dW, int64_t 
     lc.count();
 }
 
+// fp32 FMA throughput probe: every thread runs `iters` rounds of 16 independent fused multiply-adds (enough
+// independent chains to cover the pipeline latency); the result is stored so that nothing is optimised away.
+__global__ void __launch_bounds__(256) k_fma_probe(float* __restrict__ out, int iters, float a, float b) {
+    float v[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = (float)(threadIdx.x + i) * 1e-3f;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = fmaf(v[i], a, b);
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) s += v[i];
+    out[(size_t)blockIdx.x * blockDim.x + threadIdx.x] = s;
+}
+
+// Measures the device's sustained fp32 FMA rate (TFLOP/s, 2 flops per FMA) with CUDA events on `st`.
+int fma_peak_tflops(cudaStream_t st, float* scratch, size_t scratch_floats, int sm_count, double* tflops) {
+    const int blocks = sm_count * 8, threads = 256, iters = 4096;
+    if ((size_t)blocks * threads > scratch_floats) return PKV_ERR_NOMEM;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return PKV_ERR_CUDA;
+    double best = 0.0;
+    for (int rep = 0; rep < 5; ++rep) {       // first repetitions warm up; the best of the rest is reported
+        cudaEventRecord(e0, st);
+        k_fma_probe<<<blocks, threads, 0, st>>>(scratch, iters, 0.999f, 1e-4f);
+        cudaEventRecord(e1, st);
+        if (cudaEventSynchronize(e1) != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); return PKV_ERR_CUDA; }
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        const double fl = 2.0 * 16.0 * iters * (double)blocks * threads;
+        if (rep >= 2 && ms > 0.f) best = fmax(best, fl / (ms * 1e-3) / 1e12);
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    *tflops = best;
+    return cudaGetLastError() == cudaSuccess ? PKV_OK : PKV_ERR_CUDA;
+}
+
 }  // namespace pkv

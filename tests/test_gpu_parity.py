@@ -500,6 +500,37 @@ def test_stack_matches_oracle_chain(B, nl, solver, hd):
         ctx.close()
 
 
+def test_lambda_sweep_with_the_teacher_run_once_matches_separate_stacks(B):
+    """pkv_build_stack_sweep (teacher outputs cached, student + solve replayed per ridge coefficient) against
+    one pkv_build_stack per coefficient and against the oracle chain."""
+    import torch
+    nl = 4
+    cfg = small_cfg("bf16", n_layers=nl, N=64, hd=128, Hq=4, Hkv=2)
+    lays = [H.make_problem(cfg, layer=l) for l in range(nl)]
+    x0 = lays[0]["x0"]
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    dl = []
+    for l in range(nl):
+        off, idx = gen.kept_to_csr(lays[l]["kept"])
+        kv = B.to_device({"K": lays[l]["K"], "V": lays[l]["V"]}, cfg.dtype)
+        dl.append({"w": B.to_device(lays[l]["weights"], cfg.dtype), "K": kv["K"], "V": kv["V"], "head_off": off,
+                   "idx": torch.from_numpy(idx).cuda()})
+    xt = torch.from_numpy(x0).cuda()
+    lams = [1e-3, 0.1, 10.0]
+    sweep = ctx.build_stack_sweep(dl, xt, xt, [0, cfg.N], cfg.L, lams)
+    for j, lam0 in enumerate(lams):
+        single = ctx.build_stack(dl, xt, xt, [0, cfg.N], cfg.L, lam0)
+        xF, xC = x0.astype(np.float64), x0.astype(np.float64)
+        for l in range(nl):
+            o = H.run_oracle(cfg, lays[l], xF, xC, [0, cfg.N], lam0)
+            xF, xC = o["xF_next"], o["xC_next"]
+            got = sweep["dW"][j][l].cpu().numpy()
+            assert H.rel_fro(got, single["dW"][l].cpu().numpy()) <= 1e-5, (lam0, l)
+            assert H.rel_fro(got, o["dW"]) <= DW_TOL, (lam0, l)
+            np.testing.assert_allclose(sweep["stats"][j][l]["lambda_eff"], o["lam"], rtol=5e-3)
+    ctx.close()
+
+
 # ------------------------------------------------------------------ boundary
 
 def test_boundary_rejects_bad_arguments(B):
