@@ -358,39 +358,58 @@ __global__ void __launch_bounds__(kPotrfThreads) k_chain128(const __grid_constan
     float minpiv = INFINITY;
     int bad_col = -1;
     // 16 x 16 diagonal piece at c0 in registers of warp 0: lane i (and its mirror i + 16, so that every shuffle
-    // source is live) holds row i, already loaded into a[].  Two pivots per round: the 2 x 2 leading block is
-    // factored redundantly by every lane from three shuffled values, which halves the number of dependent
-    // shuffle / rsqrt rounds of the pivot chain.
+    // source is live) holds row i, already loaded into a[].  Four pivots per round: the 4 x 4 leading block
+    // (ten values, shuffled from lanes j..j+3) is factored redundantly by every lane, so that the dependent
+    // shuffle -> rsqrt -> shuffle round trip is paid four times per piece instead of sixteen.
     auto diag16 = [&](int c0, float (&a)[SB]) {
 #pragma unroll
-        for (int j = 0; j < SB; j += 2) {
-            float p00 = __shfl_sync(0xffffffffu, a[j], j);
-            const float p10 = __shfl_sync(0xffffffffu, a[j], j + 1);
-            const float p11 = __shfl_sync(0xffffffffu, a[j + 1], j + 1);
-            const bool ok0 = (p00 > 0.f) && (p00 < INFINITY);
-            if (!ok0 && bad_col < 0 && c0 + j < nbk) bad_col = c0 + j;
-            p00 = ok0 ? p00 : 1.f;
-            float r0 = rsqrtf(p00);
-            r0 = r0 * fmaf(-0.5f * p00 * r0, r0, 1.5f);         // one Newton step: full fp32 accuracy
-            const float l10 = p10 * r0;
-            float q = fmaf(-l10, l10, p11);
-            const bool ok1 = (q > 0.f) && (q < INFINITY);
-            if (!ok1 && bad_col < 0 && c0 + j + 1 < nbk) bad_col = c0 + j + 1;
-            q = ok1 ? q : 1.f;
-            if (c0 + j < nbk) minpiv = fminf(minpiv, p00);
-            if (c0 + j + 1 < nbk) minpiv = fminf(minpiv, q);
-            float r1 = rsqrtf(q);
-            r1 = r1 * fmaf(-0.5f * q * r1, r1, 1.5f);
-            const float x0 = a[j] * r0;                         // column j of L, this lane's row
-            const float x1 = fmaf(-x0, l10, a[j + 1]) * r1;     // column j + 1 (row j holds an unused value there)
-            a[j] = x0;
-            a[j + 1] = x1;
-            if (lane == j) { rd[c0 + j] = r0; rd[c0 + j + 1] = r1; }
+        for (int j = 0; j < SB; j += 4) {
+            float p[4][4];
 #pragma unroll
-            for (int k = j + 2; k < SB; ++k) {
-                const float y0 = __shfl_sync(0xffffffffu, x0, k);
-                const float y1 = __shfl_sync(0xffffffffu, x1, k);
-                a[k] = fmaf(-x1, y1, fmaf(-x0, y0, a[k]));      // rows above the diagonal hold unused values
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int cc = 0; cc <= r; ++cc) p[r][cc] = __shfl_sync(0xffffffffu, a[j + cc], j + r);
+            float l[4][4], rr[4];
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                float q = p[cc][cc];
+#pragma unroll
+                for (int k = 0; k < cc; ++k) q = fmaf(-l[cc][k], l[cc][k], q);
+                const bool okp = (q > 0.f) && (q < INFINITY);
+                if (!okp && bad_col < 0 && c0 + j + cc < nbk) bad_col = c0 + j + cc;
+                q = okp ? q : 1.f;
+                if (c0 + j + cc < nbk) minpiv = fminf(minpiv, q);
+                float rq = rsqrtf(q);
+                rq = rq * fmaf(-0.5f * q * rq, rq, 1.5f);      // one Newton step: full fp32 accuracy
+                rr[cc] = rq;
+#pragma unroll
+                for (int r = cc + 1; r < 4; ++r) {
+                    float v = p[r][cc];
+#pragma unroll
+                    for (int k = 0; k < cc; ++k) v = fmaf(-l[r][k], l[cc][k], v);
+                    l[r][cc] = v * rq;
+                }
+            }
+            // this lane's row: columns j..j+3 of L (rows j..j+2 hold unused values right of their diagonal)
+            float x[4];
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                float v = a[j + cc];
+#pragma unroll
+                for (int k = 0; k < cc; ++k) v = fmaf(-x[k], l[cc][k], v);
+                x[cc] = v * rr[cc];
+                a[j + cc] = x[cc];
+            }
+            if (lane == j) {
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) rd[c0 + j + cc] = rr[cc];
+            }
+#pragma unroll
+            for (int k = j + 4; k < SB; ++k) {
+                float v = a[k];
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) v = fmaf(-x[cc], __shfl_sync(0xffffffffu, x[cc], k), v);
+                a[k] = v;                                       // rows above the diagonal hold unused values
             }
         }
         if (lane < SB) {
