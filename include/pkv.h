@@ -113,18 +113,28 @@ typedef struct pkv_kv {
     const void* V;
 } pkv_kv;
 
-/* Compressed cache, one of two forms (Sec. 2.1: eviction or approximation compressors).
+/* Compressed cache, one of three forms (Sec. 2.1: eviction or approximation compressors; appendix: quantised caches).
  *  (a) kept-index set:  idx != NULL.  Head h keeps rows idx[head_off[h] .. head_off[h+1])
  *      of the full cache, strictly ascending, each in [0, L).  Heads may keep different counts.
- *  (b) explicit cache:  idx == NULL, Kc/Vc != NULL, packed [head_off[Hkv]][hd] with head h's
- *      rows at head_off[h]...; optional per-key logit bias (fp32, same packing) or NULL.
- * head_off is a HOST array of Hkv+1 ints starting at 0; idx/Kc/Vc/bias are device. */
+ *  (b) explicit cache:  idx == NULL, qbits == 0, Kc/Vc != NULL, packed [head_off[Hkv]][hd] (element type
+ *      dims.dtype) with head h's rows at head_off[h]...; optional per-key logit bias (fp32, same packing) or NULL.
+ *  (c) quantised explicit cache:  idx == NULL, qbits = 8 or 4.  Kc/Vc hold integer codes, same row packing:
+ *      qbits 8: int8 [rows][hd]; qbits 4: bytes [rows][hd/2], element 2j in the low nibble of byte j, element
+ *      2j+1 in the high nibble, 4-bit two's complement.  k_scale/v_scale: fp32 [rows][hd/qgroup], one scale per
+ *      qgroup consecutive elements of a row (qgroup a multiple of 8 that divides hd).  An element decodes to
+ *      scale * code computed in fp32 and rounded to dims.dtype; the student attends to the decoded cache, which
+ *      the library materialises in its workspace during the index/compaction stage.  bias as in (b).
+ * head_off is a HOST array of Hkv+1 ints starting at 0; idx/Kc/Vc/bias/scales are device. */
 typedef struct pkv_kv_compressed {
     const int32_t* head_off;
     const int32_t* idx;
     const void* Kc;
     const void* Vc;
     const float* bias;
+    const float* k_scale;    /* form (c) only */
+    const float* v_scale;
+    int32_t qbits;           /* 0 (forms a, b), 8 or 4 */
+    int32_t qgroup;
 } pkv_kv_compressed;
 
 /* Reference tokens entering the block (Algorithm 1: states x^F, x^C of every chunk).
@@ -223,6 +233,10 @@ int pkv_build_stack_sweep(pkv_ctx* ctx, int n_layers, const pkv_block_weights* w
  * offender. */
 int pkv_gather_kept(pkv_ctx* ctx, const pkv_kv* full, const int32_t* head_off_host,
                     const int32_t* idx, void* Kc, void* Vc, int32_t* bad_head, int32_t* bad_pos);
+
+/* Decode of a quantised compact cache alone (form (c) of pkv_kv_compressed; bit-exact unit check of the student's
+ * load path): Kc, Vc device [head_off[Hkv]][hd] of dims.dtype out. */
+int pkv_dequant_cache(pkv_ctx* ctx, const pkv_kv_compressed* cb, void* Kc, void* Vc);
 
 /* Dual-cache attention alone (Sec. 2.2, teacher and student forward passes over the reference
  * tokens).  q: device fp32 [2][N][Hq*hd] rotated queries of the teacher (0) and student (1)

@@ -24,7 +24,8 @@ force on tiny inputs, textbook routines that take another route (QR least square
 augmented system, the dual N x N form, eigenvalues) and the invariants Eq. 4-9 imply.
 The RoPE / norm conventions and the input generators are our own definitions: nothing in
 the paper pins them ("parity unpinned" for those conventions only).
-``low_rank_patch`` (appendix variant) has no CUDA counterpart yet; it is pinned like the rest.
+``dequantize_cache`` states the storage format of quantised compact caches (ours: the paper names INT8 / INT4
+only); it is pinned on hand-written bytes and closed-form products.
 """
 from __future__ import annotations
 
@@ -246,6 +247,28 @@ def gather_cache(K: np.ndarray, V: np.ndarray, kept: Sequence[np.ndarray]):
     """K'[h][i] = K[h][kept[h][i]] and the same for V — an eviction compressor's cache."""
     return [np.asarray(K[h])[np.asarray(kept[h], dtype=np.int64)] for h in range(len(kept))], \
            [np.asarray(V[h])[np.asarray(kept[h], dtype=np.int64)] for h in range(len(kept))]
+
+
+def dequantize_cache(codes: np.ndarray, scales: np.ndarray, bits: int, group: int, dtype: str) -> np.ndarray:
+    """Decode of a quantised compact cache (appendix, quantised caches: the patch is built against the cache
+    the student will really read).  codes: int8 [rows][hd] for 8 bits; uint8 [rows][hd/2] for 4 bits with element
+    2j in the low nibble of byte j and element 2j+1 in the high nibble, 4-bit two's complement.  scales: fp32
+    [rows][hd/group].  An element is scale * code, the product taken in fp32 and stored in the cache's element
+    type (rounded to bf16 for bf16 caches).  Returns fp32 values [rows][hd]."""
+    scales = np.asarray(scales, dtype=np.float32)
+    if bits == 8:
+        q = np.asarray(codes).astype(np.int8).astype(np.int32)
+    elif bits == 4:
+        b = np.asarray(codes).astype(np.uint8).astype(np.int32)
+        lo, hi = b & 15, b >> 4
+        q = np.stack([lo, hi], axis=-1).reshape(b.shape[0], -1)
+        q = np.where(q >= 8, q - 16, q)
+    else:
+        raise ValueError("bits must be 8 or 4")
+    hd = q.shape[1]
+    s = np.repeat(scales, group, axis=1)[:, :hd]
+    x = (s * q.astype(np.float32)).astype(np.float32)           # fp32 product
+    return round_bf16(x) if dtype == "bf16" else x
 
 
 # ----------------------------------------------------------------------------------------

@@ -54,7 +54,8 @@ class pkv_kv(C.Structure):
 
 class pkv_kv_compressed(C.Structure):
     _fields_ = [("head_off", C.POINTER(C.c_int32)), ("idx", C.c_void_p), ("Kc", C.c_void_p),
-                ("Vc", C.c_void_p), ("bias", C.c_void_p)]
+                ("Vc", C.c_void_p), ("bias", C.c_void_p), ("k_scale", C.c_void_p), ("v_scale", C.c_void_p),
+                ("qbits", C.c_int32), ("qgroup", C.c_int32)]
 
 
 class pkv_ref(C.Structure):
@@ -114,6 +115,8 @@ def lib() -> C.CDLL:
     L.pkv_gather_kept.restype = C.c_int
     L.pkv_gather_kept.argtypes = [C.c_void_p, P(pkv_kv), P(C.c_int32), C.c_void_p, C.c_void_p, C.c_void_p,
                                   P(C.c_int32), P(C.c_int32)]
+    L.pkv_dequant_cache.restype = C.c_int
+    L.pkv_dequant_cache.argtypes = [C.c_void_p, P(pkv_kv_compressed), C.c_void_p, C.c_void_p]
     L.pkv_attention.restype = C.c_int
     L.pkv_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, P(pkv_kv), P(pkv_kv_compressed),
                                 C.c_int32, C.c_int32, P(C.c_int32), C.c_void_p, C.c_void_p, C.c_void_p]
@@ -244,15 +247,18 @@ class PkvContext:
                                    ("g_attn", "Wq", "Wk", "Wv", "Wo", "g_mlp", "Wgate", "Wup", "Wdown")])
 
     @staticmethod
-    def compressed_struct(head_off, idx=None, Kc=None, Vc=None, bias=None):
+    def compressed_struct(head_off, idx=None, Kc=None, Vc=None, bias=None, quant=None):
+        """quant: None or dict(k_scale, v_scale, bits, group) when Kc/Vc hold integer codes."""
         ho = _i32(head_off)
-        s = pkv_kv_compressed(C.cast(ho, C.POINTER(C.c_int32)), _ptr(idx), _ptr(Kc), _ptr(Vc), _ptr(bias))
+        q = quant or {}
+        s = pkv_kv_compressed(C.cast(ho, C.POINTER(C.c_int32)), _ptr(idx), _ptr(Kc), _ptr(Vc), _ptr(bias),
+                              _ptr(q.get("k_scale")), _ptr(q.get("v_scale")), int(q.get("bits", 0)), int(q.get("group", 0)))
         s._keep = ho
         return s
 
     # ---- the path ----
     def build_patch(self, w, K, V, head_off, idx, xF, xC, chunk_off, pos0, lam, mode=LAMBDA_PAPER,
-                    want_next=True, Kc=None, Vc=None, bias=None, dW=None):
+                    want_next=True, Kc=None, Vc=None, bias=None, dW=None, quant=None):
         """pkv_build_patch.  Returns dict(dW, xF_next, xC_next, stats)."""
         torch = self.torch
         N = int(xF.shape[0])
@@ -261,7 +267,7 @@ class PkvContext:
             dW = torch.empty((d, F), dtype=torch.float32, device=xF.device)
         ws = self.weights_struct(w)
         kv = pkv_kv(_ptr(K), _ptr(V))
-        cb = self.compressed_struct(head_off, idx, Kc, Vc, bias)
+        cb = self.compressed_struct(head_off, idx, Kc, Vc, bias, quant)
         co = _i32(chunk_off)
         ref = pkv_ref(_ptr(xF), _ptr(xC), N, len(chunk_off) - 1, C.cast(co, C.POINTER(C.c_int32)), int(pos0))
         st = pkv_stats()
@@ -296,7 +302,7 @@ class PkvContext:
         d, F = self.dims.d, self.dims.F
         W = (pkv_block_weights * n)(*[self.weights_struct(l["w"]) for l in layers])
         KV = (pkv_kv * n)(*[pkv_kv(_ptr(l["K"]), _ptr(l["V"])) for l in layers])
-        cbs = [self.compressed_struct(l["head_off"], l.get("idx"), l.get("Kc"), l.get("Vc"), l.get("bias"))
+        cbs = [self.compressed_struct(l["head_off"], l.get("idx"), l.get("Kc"), l.get("Vc"), l.get("bias"), l.get("quant"))
                for l in layers]
         CB = (pkv_kv_compressed * n)(*cbs)
         co = _i32(chunk_off)
@@ -328,7 +334,7 @@ class PkvContext:
             cache = torch.empty(need, dtype=torch.uint8, device=xF0.device)
         W = (pkv_block_weights * n)(*[self.weights_struct(l["w"]) for l in layers])
         KV = (pkv_kv * n)(*[pkv_kv(_ptr(l["K"]), _ptr(l["V"])) for l in layers])
-        cbs = [self.compressed_struct(l["head_off"], l.get("idx"), l.get("Kc"), l.get("Vc"), l.get("bias"))
+        cbs = [self.compressed_struct(l["head_off"], l.get("idx"), l.get("Kc"), l.get("Vc"), l.get("bias"), l.get("quant"))
                for l in layers]
         CB = (pkv_kv_compressed * n)(*cbs)
         co = _i32(chunk_off)
@@ -358,13 +364,25 @@ class PkvContext:
             self._raise(rc, (bh.value, bp.value))
         return Kc[:total], Vc[:total]
 
-    def attention(self, q, k_new, v_new, K, V, head_off, idx, chunk_off, Kc=None, Vc=None, bias=None):
+    def dequant_cache(self, head_off, Kq, Vq, quant):
+        """pkv_dequant_cache: decoded K', V' [rows][hd] of the context's cache dtype."""
+        torch = self.torch
+        total = int(head_off[-1])
+        Kc = torch.zeros((max(total, 1), self.dims.hd), dtype=self.wdtype, device=Kq.device)
+        Vc = torch.zeros_like(Kc)
+        cb = self.compressed_struct(head_off, None, Kq, Vq, None, quant)
+        rc = self.L.pkv_dequant_cache(self.h, C.byref(cb), _ptr(Kc), _ptr(Vc))
+        if rc != 0:
+            self._raise(rc)
+        return Kc[:total], Vc[:total]
+
+    def attention(self, q, k_new, v_new, K, V, head_off, idx, chunk_off, Kc=None, Vc=None, bias=None, quant=None):
         torch = self.torch
         N = int(q.shape[1])
         Dq = self.dims.Hq * self.dims.hd
         outs = [torch.empty((N, Dq), dtype=torch.float32, device=q.device) for _ in range(3)]
         kv = pkv_kv(_ptr(K), _ptr(V))
-        cb = self.compressed_struct(head_off, idx, Kc, Vc, bias)
+        cb = self.compressed_struct(head_off, idx, Kc, Vc, bias, quant)
         co = _i32(chunk_off)
         rc = self.L.pkv_attention(self.h, _ptr(q), _ptr(k_new), _ptr(v_new), C.byref(kv), C.byref(cb), N,
                                   len(chunk_off) - 1, co, _ptr(outs[0]), _ptr(outs[1]), _ptr(outs[2]))

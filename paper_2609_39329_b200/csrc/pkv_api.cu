@@ -497,7 +497,13 @@ static int check_compressed(const pkv_ctx* c, const pkv_kv_compressed* cb, int* 
     *total = cb->head_off[Hkv];
     *max_b = mb;
     if (*total > 0) {
-        if (cb->idx) {
+        if (cb->qbits != 0) {
+            if (cb->idx) return PKV_ERR_INVALID_ARG;          // a quantised cache is an explicit cache
+            if (cb->qbits != 8 && cb->qbits != 4) return PKV_ERR_UNSUPPORTED;
+            if (cb->qgroup <= 0 || c->dims.hd % cb->qgroup != 0 || cb->qgroup % 8 != 0) return PKV_ERR_UNSUPPORTED;
+            if (!cb->Kc || !cb->Vc || !cb->k_scale || !cb->v_scale) return PKV_ERR_INVALID_ARG;
+            if (((uintptr_t)cb->k_scale & 3) || ((uintptr_t)cb->v_scale & 3)) return PKV_ERR_INVALID_ARG;
+        } else if (cb->idx) {
             if ((uintptr_t)cb->idx & 3) return PKV_ERR_INVALID_ARG;
         } else {
             if (!cb->Kc || !cb->Vc) return PKV_ERR_INVALID_ARG;
@@ -610,6 +616,12 @@ static void stage_compact(pkv_ctx* c, const Lc& lc, const pkv_kv* full, const pk
     if (cb->idx && total > 0) {
         gather_kept(lc, c->elem_bytes, full->K, full->V, cb->idx, head_off_dev ? head_off_dev : c->b.head_off,
                     c->dims.Hkv, c->dims.L, c->dims.hd, total, c->b.Kc, c->b.Vc, status ? status : c->b.status);
+        *Kc = c->b.Kc;
+        *Vc = c->b.Vc;
+    } else if (cb->qbits != 0 && total > 0) {
+        // quantised explicit cache: decoded into the context's compact-cache buffers, the load path of the student
+        dequant_cache(lc, c->elem_bytes, cb->Kc, cb->k_scale, cb->qbits, cb->qgroup, c->dims.hd, total, c->b.Kc);
+        dequant_cache(lc, c->elem_bytes, cb->Vc, cb->v_scale, cb->qbits, cb->qgroup, c->dims.hd, total, c->b.Vc);
         *Kc = c->b.Kc;
         *Vc = c->b.Vc;
     } else {
@@ -1027,6 +1039,20 @@ extern "C" int pkv_gather_kept(pkv_ctx* c, const pkv_kv* full, const int32_t* he
     if (bad_head) *bad_head = st.err_info[0];
     if (bad_pos) *bad_pos = st.err_info[1];
     return rc;
+}
+
+extern "C" int pkv_dequant_cache(pkv_ctx* c, const pkv_kv_compressed* cb, void* Kc, void* Vc) {
+    if (!c || !cb || !Kc || !Vc) return PKV_ERR_INVALID_ARG;
+    int total = 0, max_b = 0;
+    int rc = check_compressed(c, cb, &total, &max_b);
+    if (rc != PKV_OK) return rc;
+    if (cb->qbits == 0) return PKV_ERR_INVALID_ARG;
+    if (((uintptr_t)Kc & 15) || ((uintptr_t)Vc & 15)) return PKV_ERR_INVALID_ARG;
+    Lc lc{c->st, &c->launches, c->map_cache};
+    begin_call(c);
+    dequant_cache(lc, c->elem_bytes, cb->Kc, cb->k_scale, cb->qbits, cb->qgroup, c->dims.hd, total, Kc);
+    dequant_cache(lc, c->elem_bytes, cb->Vc, cb->v_scale, cb->qbits, cb->qgroup, c->dims.hd, total, Vc);
+    return end_call(c, nullptr, nullptr);
 }
 
 extern "C" int pkv_attention(pkv_ctx* c, const float* q, const float* k_new, const float* v_new,

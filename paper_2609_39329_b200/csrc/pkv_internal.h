@@ -52,6 +52,9 @@ struct Lc {
 void gather_kept(const Lc& lc, int elem_bytes, const void* K, const void* V, const int32_t* idx,
                  const int32_t* head_off_dev, int Hkv, int L, int hd, int total, void* Kc, void* Vc,
                  DevStatus* status);
+// out [rows][hd] (element type of the cache) = scale * code for a quantised compact cache (bits 8 or 4).
+void dequant_cache(const Lc& lc, int elem_bytes, const void* codes, const float* scales, int bits, int group, int hd,
+                   int rows, void* out);
 // out[r] = x[r] * gain / rms(x[r]) for the rows of x0 (N rows) followed by the rows of x1.
 void rmsnorm_f32(const Lc& lc, const float* x0, const float* x1, int N, int d, const float* gain, float eps,
                  float* out);

@@ -70,6 +70,55 @@ void gather_kept(const Lc& lc, int elem_bytes, const void* K, const void* V, con
     lc.count();
 }
 
+// Quantised compact cache (appendix, quantised caches): codes are signed integers, 8 bits (one byte per element)
+// or 4 bits (two per byte, even element in the low nibble, two's complement), with one fp32 scale per
+// `group` consecutive elements of a row; an element decodes to scale * code, rounded to the cache's element
+// type.  One thread decodes eight elements (a 16-byte bf16 store or two 16-byte fp32 stores).
+template <typename T>
+__global__ void __launch_bounds__(256) k_dequant_rows(const uint8_t* __restrict__ codes, const float* __restrict__ scales,
+                                                      int bits, int group, int hd, size_t rows, T* __restrict__ out) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // chunk of eight elements
+    const int chunks = hd / 8;
+    if (i >= rows * (size_t)chunks) return;
+    const size_t r = i / chunks;
+    const int c0 = (int)(i % chunks) * 8;
+    const float* sc = scales + r * (size_t)(hd / group);
+    float v[8];
+    if (bits == 8) {
+        const int8_t* q = reinterpret_cast<const int8_t*>(codes) + r * (size_t)hd + c0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = sc[(c0 + e) / group] * (float)q[e];
+    } else {
+        const uint8_t* q = codes + r * (size_t)(hd / 2) + c0 / 2;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const uint8_t byte = q[e >> 1];
+            int nib = (e & 1) ? (byte >> 4) : (byte & 15);
+            nib = (nib ^ 8) - 8;                                 // sign-extend the 4-bit two's complement code
+            v[e] = sc[(c0 + e) / group] * (float)nib;
+        }
+    }
+    T* o = out + r * (size_t)hd + c0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        if constexpr (sizeof(T) == 2) o[e] = __float2bfloat16_rn(v[e]);
+        else o[e] = v[e];
+    }
+}
+
+void dequant_cache(const Lc& lc, int elem_bytes, const void* codes, const float* scales, int bits, int group, int hd,
+                   int rows, void* out) {
+    if (rows <= 0) return;
+    const size_t n = (size_t)rows * (hd / 8);
+    const unsigned blocks = (unsigned)((n + 255) / 256);
+    if (elem_bytes == 2)
+        k_dequant_rows<__nv_bfloat16><<<blocks, 256, 0, lc.st>>>((const uint8_t*)codes, scales, bits, group, hd, (size_t)rows,
+                                                                  (__nv_bfloat16*)out);
+    else
+        k_dequant_rows<float><<<blocks, 256, 0, lc.st>>>((const uint8_t*)codes, scales, bits, group, hd, (size_t)rows, (float*)out);
+    lc.count();
+}
+
 // ------------------------------------------------------------------------------------------
 // RMSNorm
 // ------------------------------------------------------------------------------------------

@@ -259,3 +259,21 @@ def gen_layer(cfg: PkvConfig, layer: int,
         q_obs = gen_obs_queries(cfg, layer) if cfg.kept_rule == "window_topk" else None
     kept = select_kept(cfg, layer, kv["K"], q_obs)
     return {"weights": w, "K": kv["K"], "V": kv["V"], "kept": kept}
+
+
+def quantize_rows(x: np.ndarray, bits: int, group: int):
+    """A storage-side quantiser for compact caches (the compressor's job, off the measured path): symmetric,
+    one fp32 scale per `group` consecutive elements of a row, signed codes of `bits` bits (8: int8 array
+    [rows][hd]; 4: uint8 array [rows][hd/2], even element in the low nibble, two's complement).
+    Returns (codes, scales fp32 [rows][hd/group])."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    rows, hd = x.shape
+    qmax = 127 if bits == 8 else 7
+    g = x.reshape(rows, hd // group, group)
+    amax = np.abs(g).max(axis=2)
+    scales = np.where(amax > 0, amax / qmax, 1.0).astype(np.float32)
+    q = np.clip(np.rint(g / scales[:, :, None]), -qmax, qmax).astype(np.int32).reshape(rows, hd)
+    if bits == 8:
+        return q.astype(np.int8), scales
+    u = (q & 15).astype(np.uint8)
+    return (u[:, 0::2] | (u[:, 1::2] << 4)).astype(np.uint8), scales

@@ -270,6 +270,87 @@ def test_block_with_explicit_cache_and_key_bias_matches_oracle(B, hd, Hq, Hkv):
         ctx.close()
 
 
+@pytest.mark.parametrize("dtype,hd,bits", [("bf16", 128, 8), ("bf16", 128, 4), ("bf16", 64, 4), ("fp32", 64, 8)])
+def test_quantised_compact_cache_decode_bit_exact_and_attention(B, dtype, hd, bits):
+    """INT8 / INT4 compact cache with group scales (appendix, quantised caches): the decode in the student's load
+    path is bit-exact against the oracle's, and attention on the quantised cache matches the oracle's attention on
+    the decoded cache; a finite key bias rides along."""
+    import torch
+    cfg = small_cfg(dtype, hd=hd, Hq=8, Hkv=2, L=700)
+    r = np.random.default_rng(41)
+    budgets, group = [150, 33], 32
+    off = np.zeros(3, dtype=np.int32)
+    off[1:] = np.cumsum(budgets)
+    Kraw = r.standard_normal((sum(budgets), hd)).astype(np.float32) * np.exp(r.uniform(-1, 1, hd)).astype(np.float32)
+    Vraw = r.standard_normal((sum(budgets), hd)).astype(np.float32)
+    Kq, Ks = gen.quantize_rows(Kraw, bits, group)
+    Vq, Vs = gen.quantize_rows(Vraw, bits, group)
+    Kd = orc.dequantize_cache(Kq, Ks, bits, group, dtype)
+    Vd = orc.dequantize_cache(Vq, Vs, bits, group, dtype)
+    bias = r.uniform(-1.0, 1.0, sum(budgets)).astype(np.float32)
+    chunk_off = [0, 40, 97]
+    N = chunk_off[-1]
+    q = r.standard_normal((2, N, cfg.Hq, hd)).astype(np.float32) * 1.3
+    k = r.standard_normal((2, N, cfg.Hkv, hd)).astype(np.float32)
+    v = r.standard_normal((2, N, cfg.Hkv, hd)).astype(np.float32)
+    kvd = gen.gen_cache(cfg, 0) if dtype == "bf16" else {
+        "K": r.standard_normal((cfg.Hkv, cfg.L, hd)).astype(np.float32),
+        "V": r.standard_normal((cfg.Hkv, cfg.L, hd)).astype(np.float32)}
+    split = lambda a: [a[off[h]:off[h + 1]] for h in range(cfg.Hkv)]
+    aC = orc.attention(q[1], k[1], v[1], split(Kd), split(Vd), chunk_off, key_bias=split(bias))
+    quant = {"k_scale": torch.from_numpy(Ks).cuda(), "v_scale": torch.from_numpy(Vs).cuda(), "bits": bits, "group": group}
+    tKq, tVq = torch.from_numpy(Kq).cuda(), torch.from_numpy(Vq).cuda()
+    for engine in engines(B, cfg):
+        ctx = B.PkvContext(B.dims_from_config(cfg, N_max=N, b_max=max(budgets)), engine=engine)
+        gK, gV = ctx.dequant_cache(off, tKq, tVq, quant)
+        np.testing.assert_array_equal(gK.float().cpu().numpy(), Kd)
+        np.testing.assert_array_equal(gV.float().cpu().numpy(), Vd)
+        kv = B.to_device({"K": kvd["K"], "V": kvd["V"]}, cfg.dtype)
+        tq, tk, tv = (torch.from_numpy(t.reshape(2, N, -1)).cuda() for t in (q, k, v))
+        _, gC, _ = ctx.attention(tq, tk, tv, kv["K"], kv["V"], off, None, chunk_off, Kc=tKq, Vc=tVq,
+                                 bias=torch.from_numpy(bias).cuda(), quant=quant)
+        e = H.attn_max_rel(gC.cpu().numpy(), aC, cfg.Hq, hd)
+        print("quantised cache, %s hd %d int%d engine %d: aC err %.2e" % (dtype, hd, bits, engine, e))
+        assert e <= ATTN_TOL
+        # malformed descriptions are refused
+        bad = dict(quant, group=12)
+        with pytest.raises(B.PkvError) as ei:
+            ctx.dequant_cache(off, tKq, tVq, bad)
+        assert ei.value.code == -2
+        ctx.close()
+
+
+def test_block_with_int4_compact_cache_matches_oracle(B):
+    """pkv_build_patch against an INT4 compact cache: the patch is the oracle's patch for the decoded cache."""
+    import torch
+    cfg = small_cfg("bf16", hd=128, Hq=4, Hkv=2, d=256, F=192, L=1000, N=120)
+    lay = H.make_problem(cfg)
+    # the compact cache is a quantised copy of the kept rows of the full cache
+    Kg, Vg = orc.gather_cache(lay["K"], lay["V"], lay["kept"])
+    off, _ = gen.kept_to_csr(lay["kept"])
+    Kq, Ks = gen.quantize_rows(np.concatenate(Kg), 4, 32)
+    Vq, Vs = gen.quantize_rows(np.concatenate(Vg), 4, 32)
+    Kd = orc.dequantize_cache(Kq, Ks, 4, 32, "bf16")
+    Vd = orc.dequantize_cache(Vq, Vs, 4, 32, "bf16")
+    split = lambda a: [a[off[h]:off[h + 1]] for h in range(cfg.Hkv)]
+    x = lay["x0"]
+    ref = orc.build_patch(lay["weights"], lay["K"], lay["V"], None, x, x, [0, cfg.N], cfg.L, 0.1, cfg,
+                          compressed=(split(Kd), split(Vd), None))
+    exact = H.run_oracle(cfg, lay, x, x, [0, cfg.N], 0.1)
+    assert H.rel_fro(exact["dW"], ref["dW"]) > 10 * DW_TOL          # quantisation changes the patch: it must be seen
+    ctx = B.PkvContext(B.dims_from_config(cfg, b_max=max(len(k) for k in lay["kept"])), engine=B.ENGINE_AUTO)
+    w = B.to_device(lay["weights"], cfg.dtype)
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    quant = {"k_scale": torch.from_numpy(Ks).cuda(), "v_scale": torch.from_numpy(Vs).cuda(), "bits": 4, "group": 32}
+    xt = torch.from_numpy(x).cuda()
+    out = ctx.build_patch(w, kv["K"], kv["V"], off, None, xt, xt, [0, cfg.N], cfg.L, 0.1,
+                          Kc=torch.from_numpy(Kq).cuda(), Vc=torch.from_numpy(Vq).cuda(), quant=quant)
+    err = H.rel_fro(out["dW"].cpu().numpy(), ref["dW"])
+    print("block with INT4 compact cache: dW rel fro err %.3e" % err)
+    assert err <= DW_TOL
+    ctx.close()
+
+
 # ------------------------------------------------------------------ S7, S8 alone
 
 @pytest.mark.parametrize("n,F,d", [(70, 192, 256), (300, 256, 128)])

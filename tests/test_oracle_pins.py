@@ -225,6 +225,37 @@ def test_prefill_cache_then_cached_forward_equals_one_causal_pass():
                            cached["a"])
 
 
+def test_quantised_cache_decode_on_hand_written_bytes_and_closed_forms():
+    """The storage format of quantised compact caches: nibble order, sign extension, group scales, and the
+    element type of the decoded value."""
+    # 4 bits: byte 0xA3 holds element 0 = 3 (low nibble) and element 1 = 0xA = -6 (two's complement)
+    codes4 = np.array([[0xA3, 0x7F, 0x80, 0x01]], dtype=np.uint8)           # 8 elements, hd = 8
+    scales = np.array([[0.5]], dtype=np.float32)
+    got = orc.dequantize_cache(codes4, scales, 4, 8, "fp32")
+    np.testing.assert_array_equal(got, np.array([[1.5, -3.0, -0.5, 3.5, 0.0, -4.0, 0.5, 0.0]], dtype=np.float32))
+    # 8 bits, two groups with their own scales
+    codes8 = np.array([[127, -127, 1, 0, -1, 64, -64, 2] * 2], dtype=np.int8)   # hd = 16, group = 8
+    sc = np.array([[0.25, 2.0]], dtype=np.float32)
+    got = orc.dequantize_cache(codes8, sc, 8, 8, "fp32")
+    want = np.concatenate([0.25 * codes8[0, :8].astype(np.float64), 2.0 * codes8[0, 8:].astype(np.float64)])[None]
+    np.testing.assert_array_equal(got.astype(np.float64), want)
+    # bf16 caches: the decoded value is the bf16 rounding of the fp32 product (checked against torch)
+    import torch
+    r = np.random.default_rng(12)
+    c = r.integers(-127, 128, size=(5, 32)).astype(np.int8)
+    s2 = r.uniform(0.01, 0.1, size=(5, 2)).astype(np.float32)
+    got = orc.dequantize_cache(c, s2, 8, 16, "bf16")
+    ref = (torch.from_numpy(np.repeat(s2, 16, axis=1)) * torch.from_numpy(c.astype(np.float32))).to(torch.bfloat16).float().numpy()
+    np.testing.assert_array_equal(got, ref)
+    # a round trip through the harness quantiser is within half a step of every element
+    x = r.standard_normal((6, 64)).astype(np.float32)
+    for bits in (8, 4):
+        q, sc3 = gen.quantize_rows(x, bits, 32)
+        back = orc.dequantize_cache(q, sc3, bits, 32, "fp32")
+        step = np.repeat(sc3, 32, axis=1)
+        assert np.all(np.abs(back - x) <= 0.5 * step * (1 + 1e-6))
+
+
 # ------------------------------------------------------------------ backbone conventions
 
 def test_rope_is_a_rotation_and_relative():
