@@ -36,7 +36,7 @@ extern "C" {
 typedef enum pkv_error {
     PKV_OK = 0,
     PKV_ERR_INVALID_ARG = -1,  /* null/misaligned pointer, lambda <= 0 or non-finite, N = 0, bad chunk offsets */
-    PKV_ERR_UNSUPPORTED = -2,  /* hd not in {64,128}, Hq % Hkv != 0, F > 8192, sizes the kernels do not cover */
+    PKV_ERR_UNSUPPORTED = -2,  /* hd not in {64,128}, Hq % Hkv != 0, F > 32768, sizes the kernels do not cover */
     PKV_ERR_BAD_INDEX = -3,    /* kept-index set not strictly ascending within [0, L); first offender in stats */
     PKV_ERR_NOT_PD = -4,       /* Cholesky pivot <= 0 or non-finite; column in stats.err_info */
     PKV_ERR_DEGENERATE = -5,   /* tr(S_H) = 0 under the adaptive ridge scale (Eq. 7) */
@@ -73,7 +73,7 @@ enum {
 typedef struct pkv_dims {
     int32_t d;            /* hidden size */
     int32_t Hq, Hkv, hd;  /* query heads, key/value heads (Hq % Hkv == 0), head dim (64 or 128) */
-    int32_t F;            /* MLP intermediate width (<= 8192) */
+    int32_t F;            /* MLP intermediate width (<= 32768; the models the paper names have 14336 and 18944) */
     int32_t L;            /* rows of the full cache per KV head */
     int32_t N_max;        /* most reference tokens one call may bring */
     int32_t b_max;        /* most kept rows per KV head in a compressed cache */
@@ -186,6 +186,27 @@ void pkv_destroy(pkv_ctx* ctx);
 int pkv_build_patch(pkv_ctx* ctx, const pkv_block_weights* w, const pkv_kv* full,
                     const pkv_kv_compressed* cb, const pkv_ref* ref, float lambda, int lambda_mode,
                     float* dW, const pkv_ref_next* next, pkv_stats* stats);
+
+/* Streamed reference sets (Sec. 2.3, chunked query encoding; Eq. 9).  The reference set of a context may be far
+ * larger than one call's N_max: it is fed in parts, each a whole number of chunks, and only the running sums
+ * S_H, S_T stay in the context between the calls, so that the workspace does not grow with the reference set.
+ *   pkv_stream_begin     clears the sums and fixes the ridge coefficient and its reading;
+ *   pkv_stream_add       teacher and student forward of ref->N <= N_max tokens (same arguments as
+ *                        pkv_build_patch), targets, S_H += H'^T H', S_T += T^T H'; xF_next (optional, device fp32
+ *                        [N][d]) receives the teacher's states of these tokens entering the next block;
+ *   pkv_stream_finish    lambda from the sums (Eq. 7), dW = S_T (S_H + lambda I)^{-1} (Eq. 8); stats->target_fro2 is
+ *                        the sum over the parts, resid_fro2 is not available;
+ *   pkv_stream_propagate Algorithm 1's student propagation for one part: the student block re-run with the
+ *                        patched W + dW against the compressed cache, xC_next = z' + (W + dW) h' (device fp32 [N][d];
+ *                        tensor-core engine only).
+ * Any number of parts gives the statistics of one call on all tokens up to rounding order (chunks are independent).
+ * A failed pkv_stream_add closes the stream (begin again).  Not available with PKV_SOLVER_DUAL. */
+int pkv_stream_begin(pkv_ctx* ctx, float lambda, int lambda_mode);
+int pkv_stream_add(pkv_ctx* ctx, const pkv_block_weights* w, const pkv_kv* full, const pkv_kv_compressed* cb,
+                   const pkv_ref* ref, float* xF_next);
+int pkv_stream_finish(pkv_ctx* ctx, float* dW, pkv_stats* stats);
+int pkv_stream_propagate(pkv_ctx* ctx, const pkv_block_weights* w, const pkv_kv* full, const pkv_kv_compressed* cb,
+                         const pkv_ref* ref, const float* dW, float* xC_next);
 
 /* Algorithm 1, Merge: W[i] <- W[i] + dW[i] for the d*F entries, the sum taken in fp32 and
  * rounded once to W's type (w_dtype = PKV_BF16 | PKV_FP32).  Asynchronous on cuda_stream. */

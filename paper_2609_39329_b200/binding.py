@@ -100,6 +100,15 @@ def lib() -> C.CDLL:
     L.pkv_build_patch.restype = C.c_int
     L.pkv_build_patch.argtypes = [C.c_void_p, P(pkv_block_weights), P(pkv_kv), P(pkv_kv_compressed), P(pkv_ref),
                                   C.c_float, C.c_int, C.c_void_p, P(pkv_ref_next), P(pkv_stats)]
+    L.pkv_stream_begin.restype = C.c_int
+    L.pkv_stream_begin.argtypes = [C.c_void_p, C.c_float, C.c_int]
+    L.pkv_stream_add.restype = C.c_int
+    L.pkv_stream_add.argtypes = [C.c_void_p, P(pkv_block_weights), P(pkv_kv), P(pkv_kv_compressed), P(pkv_ref), C.c_void_p]
+    L.pkv_stream_finish.restype = C.c_int
+    L.pkv_stream_finish.argtypes = [C.c_void_p, C.c_void_p, P(pkv_stats)]
+    L.pkv_stream_propagate.restype = C.c_int
+    L.pkv_stream_propagate.argtypes = [C.c_void_p, P(pkv_block_weights), P(pkv_kv), P(pkv_kv_compressed), P(pkv_ref),
+                                       C.c_void_p, C.c_void_p]
     L.pkv_merge.restype = C.c_int
     L.pkv_merge.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int64, C.c_void_p]
     L.pkv_build_stack.restype = C.c_int
@@ -281,6 +290,50 @@ class PkvContext:
         if rc != 0:
             self._raise(rc, st.as_dict())
         return {"dW": dW, "xF_next": xFn, "xC_next": xCn, "stats": st.as_dict()}
+
+    # ---- streamed reference sets ----
+    def stream_begin(self, lam, mode=LAMBDA_PAPER):
+        rc = self.L.pkv_stream_begin(self.h, float(lam), int(mode))
+        if rc != 0:
+            self._raise(rc)
+
+    def _ref(self, xF, xC, chunk_off, pos0):
+        co = _i32(chunk_off)
+        ref = pkv_ref(_ptr(xF), _ptr(xC), int(xC.shape[0]), len(chunk_off) - 1, C.cast(co, C.POINTER(C.c_int32)), int(pos0))
+        ref._keep = co
+        return ref
+
+    def stream_add(self, w, K, V, head_off, idx, xF, xC, chunk_off, pos0, want_next=False, Kc=None, Vc=None, bias=None,
+                   quant=None):
+        """pkv_stream_add; returns the teacher's next states of these tokens if asked."""
+        ws = self.weights_struct(w)
+        kv = pkv_kv(_ptr(K), _ptr(V))
+        cb = self.compressed_struct(head_off, idx, Kc, Vc, bias, quant)
+        ref = self._ref(xF, xC, chunk_off, pos0)
+        xFn = self.torch.empty_like(xF) if want_next else None
+        rc = self.L.pkv_stream_add(self.h, C.byref(ws), C.byref(kv), C.byref(cb), C.byref(ref), _ptr(xFn))
+        if rc != 0:
+            self._raise(rc)
+        return xFn
+
+    def stream_finish(self):
+        dW = self.torch.empty((self.dims.d, self.dims.F), dtype=self.torch.float32, device="cuda")
+        st = pkv_stats()
+        rc = self.L.pkv_stream_finish(self.h, _ptr(dW), C.byref(st))
+        if rc != 0:
+            self._raise(rc, st.as_dict())
+        return dW, st.as_dict()
+
+    def stream_propagate(self, w, K, V, head_off, idx, xC, chunk_off, pos0, dW, Kc=None, Vc=None, bias=None, quant=None):
+        ws = self.weights_struct(w)
+        kv = pkv_kv(_ptr(K), _ptr(V))
+        cb = self.compressed_struct(head_off, idx, Kc, Vc, bias, quant)
+        ref = self._ref(xC, xC, chunk_off, pos0)
+        out = self.torch.empty_like(xC)
+        rc = self.L.pkv_stream_propagate(self.h, C.byref(ws), C.byref(kv), C.byref(cb), C.byref(ref), _ptr(dW), _ptr(out))
+        if rc != 0:
+            self._raise(rc)
+        return out
 
     def merge(self, W, dW):
         """pkv_merge: W <- W + dW in place (W bf16 or fp32, dW fp32)."""

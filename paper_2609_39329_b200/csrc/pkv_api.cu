@@ -183,6 +183,9 @@ struct pkv_ctx {
     int teacher_sms;         // SMs the teacher stream may use (sm_count when not partitioned)
     cudaEvent_t evTea[kRing], evStu[kRing], evSetup;
     int64_t launches;
+    int stream_open, stream_mode, stream_tokens;   // streamed reference set in progress (pkv_stream_*)
+    float stream_lambda;
+    double stream_tfro2;
     int force_sequential;    // pkv_build_stack: 1 = block by block on one stream even where the overlapped driver applies
     int teacher_timed;
     void* map_cache;
@@ -285,7 +288,7 @@ static int dims_ok(const pkv_dims* d) {
     if (!(d->eps >= 0.f) || !(d->rope_theta >= 0.f)) return PKV_ERR_INVALID_ARG;
     if (d->hd != 64 && d->hd != 128) return PKV_ERR_UNSUPPORTED;
     if (d->Hq % d->Hkv != 0) return PKV_ERR_UNSUPPORTED;
-    if (d->F > 8192) return PKV_ERR_UNSUPPORTED;
+    if (d->F > 32768) return PKV_ERR_UNSUPPORTED;
     if ((long long)d->L + d->N_max > (1LL << 30)) return PKV_ERR_UNSUPPORTED;
     return PKV_OK;
 }
@@ -665,10 +668,14 @@ static void solve_stage(pkv_ctx* c, const Lc& lc, float* S_H, const float* S_T, 
     sumsq(lc, dW, (int64_t)d * F, &st->dw_fro2);
 }
 
+// stats_only: the streamed form (Sec. 2.3, Eq. 9): teacher and student forward of these tokens, then the running
+// sums S_H, S_T of the context are ADDED to, and the call returns before the solve; xF_next_only optionally receives
+// the teacher's next states of these tokens.
 static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv* full,
                             const pkv_kv_compressed* cb, const pkv_ref* ref, float lambda, int mode, float* dW,
-                            const pkv_ref_next* next, pkv_stats* stats) {
-    if (!c || !w || !full || !cb || !ref || !dW) return PKV_ERR_INVALID_ARG;
+                            const pkv_ref_next* next, pkv_stats* stats, bool stats_only = false,
+                            float* xF_next_only = nullptr) {
+    if (!c || !w || !full || !cb || !ref || (!dW && !stats_only)) return PKV_ERR_INVALID_ARG;
     if (!w->g_attn || !w->Wq || !w->Wk || !w->Wv || !w->Wo || !w->g_mlp || !w->Wgate || !w->Wup || !w->Wdown)
         return PKV_ERR_INVALID_ARG;
     if (c->dims.L > 0 && (!full->K || !full->V)) return PKV_ERR_INVALID_ARG;
@@ -677,7 +684,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
     if (mode != PKV_LAMBDA_PAPER && mode != PKV_LAMBDA_ABSOLUTE && mode != PKV_LAMBDA_TRACE_MEAN)
         return PKV_ERR_INVALID_ARG;
     const void* ptrs[] = {w->Wq, w->Wk, w->Wv, w->Wo, w->Wgate, w->Wup, w->Wdown, full->K, full->V,
-                          ref->xF, ref->xC, dW, w->g_attn, w->g_mlp};
+                          ref->xF, ref->xC, dW, w->g_attn, w->g_mlp, xF_next_only};
     for (const void* p : ptrs)
         if ((uintptr_t)p & 15) return PKV_ERR_INVALID_ARG;
     if (next && (!next->xF_next || !next->xC_next)) return PKV_ERR_INVALID_ARG;
@@ -732,7 +739,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         sumsq(lc, b.R, (int64_t)N * d, &b.status->t_fro2);
         mark(c, ST_GRAM);
         // S7 (Eq. 9)
-        gram_simt(c, lc, b.hC, b.R, N, b.S_H, b.S_T, false);
+        gram_simt(c, lc, b.hC, b.R, N, b.S_H, b.S_T, stats_only);
         mark(c, ST_SOLVE);
     } else {
         pkv::TcForwardArgs fa;
@@ -746,12 +753,25 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         fa.kv_split = c->kv_split;
         fa.dual = c->dual;
         fa.precise_stats = pkv::tc_well_conditioned(lambda, mode) ? 0 : 1;
+        fa.accumulate_stats = stats_only ? 1 : 0;
         fa.part_m = b.part_m; fa.part_l = b.part_l; fa.part_O = b.part_O;
         fa.ev = c->timing ? c->ev : nullptr;
         fa.evT = nullptr;
         c->teacher_timed = 0;
         rc = pkv::tc_forward(lc, &b.tc, &c->dims, fa);
         if (rc != PKV_OK) return rc;
+    }
+    if (stats_only) {
+        // teacher's next states of these tokens, if asked: xF_next = zF + hF W^T
+        if (xF_next_only) {
+            if (c->engine == PKV_ENGINE_SIMT)
+                gemm_tn_simt(lc, b.hF, F, w->Wdown, F, bf, xF_next_only, d, N, d, F, 1.f, b.zF, d, false);
+            else
+                pkv::tc_next_states(lc, &b.tc, &c->dims, N, w->Wdown, nullptr, b.zF, b.R, xF_next_only, nullptr, b.status);
+        }
+        mark(c, ST_NEXT);
+        mark(c, ST_COUNT);
+        return end_call(c, stats, cb->head_off);
     }
     // S8 (Eq. 7-8)
     if (c->dual) {
@@ -781,6 +801,84 @@ extern "C" int pkv_build_patch(pkv_ctx* ctx, const pkv_block_weights* w, const p
                                const pkv_kv_compressed* cb, const pkv_ref* ref, float lambda, int lambda_mode,
                                float* dW, const pkv_ref_next* next, pkv_stats* stats) {
     return build_patch_impl(ctx, w, full, cb, ref, lambda, lambda_mode, dW, next, stats);
+}
+
+// ---- streamed reference sets (Sec. 2.3: chunked query encoding with running sufficient statistics) ----
+
+extern "C" int pkv_stream_begin(pkv_ctx* c, float lambda, int lambda_mode) {
+    if (!c) return PKV_ERR_INVALID_ARG;
+    if (!(lambda > 0.f) || !isfinite(lambda)) return PKV_ERR_INVALID_ARG;
+    if (lambda_mode != PKV_LAMBDA_PAPER && lambda_mode != PKV_LAMBDA_ABSOLUTE && lambda_mode != PKV_LAMBDA_TRACE_MEAN)
+        return PKV_ERR_INVALID_ARG;
+    if (c->dual) return PKV_ERR_UNSUPPORTED;          // the dual form needs every reference token in one call
+    const size_t F = c->dims.F, d = c->dims.d;
+    if (cudaMemsetAsync(c->b.S_H, 0, F * F * sizeof(float), c->st) != cudaSuccess ||
+        cudaMemsetAsync(c->b.S_T, 0, d * F * sizeof(float), c->st) != cudaSuccess)
+        return PKV_ERR_CUDA;
+    c->stream_lambda = lambda;
+    c->stream_mode = lambda_mode;
+    c->stream_tokens = 0;
+    c->stream_tfro2 = 0.0;
+    c->stream_open = 1;
+    return PKV_OK;
+}
+
+extern "C" int pkv_stream_add(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv* full, const pkv_kv_compressed* cb,
+                              const pkv_ref* ref, float* xF_next) {
+    if (!c || !c->stream_open) return PKV_ERR_INVALID_ARG;
+    pkv_stats st;
+    int rc = build_patch_impl(c, w, full, cb, ref, c->stream_lambda, c->stream_mode, nullptr, nullptr, &st, true, xF_next);
+    if (rc != PKV_OK) {
+        c->stream_open = 0;                          // the running sums may be partly updated: start over
+        return rc;
+    }
+    c->stream_tokens += ref->N;
+    c->stream_tfro2 += st.target_fro2;
+    return PKV_OK;
+}
+
+extern "C" int pkv_stream_finish(pkv_ctx* c, float* dW, pkv_stats* stats) {
+    if (!c || !dW || !c->stream_open || ((uintptr_t)dW & 15)) return PKV_ERR_INVALID_ARG;
+    if (c->stream_tokens <= 0) return PKV_ERR_INVALID_ARG;
+    c->stream_open = 0;
+    Lc lc{c->st, &c->launches, c->map_cache};
+    begin_call(c);
+    if (c->engine != PKV_ENGINE_SIMT) c->b.tc.S3_ready = 0;
+    solve_stage(c, lc, c->b.S_H, c->b.S_T, c->stream_lambda, c->stream_mode, dW, true);
+    int rc = end_call(c, stats, nullptr);
+    if (stats) stats->target_fro2 = c->stream_tfro2;
+    return rc;
+}
+
+extern "C" int pkv_stream_propagate(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv* full,
+                                    const pkv_kv_compressed* cb, const pkv_ref* ref, const float* dW, float* xC_next) {
+    if (!c || !w || !full || !cb || !ref || !dW || !xC_next || !ref->xC) return PKV_ERR_INVALID_ARG;
+    if (c->engine == PKV_ENGINE_SIMT) return PKV_ERR_UNSUPPORTED;
+    if (((uintptr_t)dW & 15) || ((uintptr_t)xC_next & 15) || ((uintptr_t)ref->xC & 15)) return PKV_ERR_INVALID_ARG;
+    int rc = check_chunks(c, ref->N, ref->n_chunks, ref->chunk_off);
+    if (rc != PKV_OK) return rc;
+    int total = 0, max_b = 0;
+    rc = check_compressed(c, cb, &total, &max_b);
+    if (rc != PKV_OK) return rc;
+    const pkv_dims& D = c->dims;
+    const int N = ref->N;
+    Buffers& b = c->b;
+    Lc lc{c->st, &c->launches, c->map_cache};
+    begin_call(c);
+    upload_meta(c, cb->head_off, N, ref->n_chunks, ref->chunk_off);
+    const void *Kc, *Vc;
+    stage_compact(c, lc, full, cb, total, &Kc, &Vc);
+    rope_table(lc, b.tok_cs, N, D.hd, ref->pos0, D.rope_theta, b.rope_tab);
+    pkv::TcForwardArgs fa{};
+    fa.w = w; fa.full = full; fa.Kc = Kc; fa.Vc = Vc; fa.bias = cb->idx ? nullptr : cb->bias;
+    fa.xC = ref->xC; fa.N = N; fa.pos0 = ref->pos0; fa.max_b = max_b; fa.total_kept = total;
+    fa.head_off = b.head_off; fa.tok_cs = b.tok_cs; fa.rope_tab = b.rope_tab;
+    fa.aF = b.a2; fa.aC = b.aC; fa.dA = b.a2 + (size_t)N * D.Hq * D.hd;
+    fa.zC = b.zC; fa.dz = b.dz; fa.hF = b.hF; fa.hC = b.hC;
+    fa.status = b.status;
+    rc = pkv::tc_student_propagate(lc, &b.tc, &c->dims, fa, dW, b.D, xC_next);
+    if (rc != PKV_OK) return rc;
+    return end_call(c, nullptr, cb->head_off);
 }
 
 extern "C" int pkv_merge(void* W, int w_dtype, const float* dW, int64_t count, void* cuda_stream) {

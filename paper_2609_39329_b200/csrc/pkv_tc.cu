@@ -501,6 +501,51 @@ int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     return PKV_OK;
 }
 
+int tc_student_propagate(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a, const float* dW,
+                         float* zero_nd, float* xC_next) {
+    const int N = a.N, d = D->d, F = D->F, hd = D->hd;
+    const int Dq = D->Hq * hd, Dkv = D->Hkv * hd, QKV = Dq + 2 * Dkv;
+    const pkv_block_weights* w = a.w;
+    DevStatus* st = a.status;
+    int rc;
+    const size_t uo = (size_t)N * d;
+    Pair uS{t->u.hi + uo, t->u.lo + uo};
+    // with a zero "teacher" attention output and a zero incoming state difference the student half of the
+    // forward computes dA = -a', dz = -a' Wo^T and z' = x' - dz, i.e. the plain student block
+    cudaMemsetAsync(a.aF, 0, (size_t)N * Dq * sizeof(float), lc.st);
+    cudaMemsetAsync(zero_nd, 0, (size_t)N * d * sizeof(float), lc.st);
+    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.xC, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, N);
+    lc.count();
+    float* qkvS = t->qkv + (size_t)N * QKV;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wq, d, qkvS, QKV, N, Dq, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wk, d, qkvS + Dq, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wv, d, qkvS + Dq + Dkv, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    AttnArgs at{};
+    fill_attn(at, t, D, a, 2);
+    if ((rc = attention_tc(lc, t, D, at, a.rope_tab, st))) return rc;
+    Pair aS{t->a.hi + (size_t)N * Dq, t->a.lo + (size_t)N * Dq};
+    if ((rc = gemm_act_weight(lc, aS, Dq, w->Wo, Dq, t->o + uo, d, N, d, Dq, 1.f, nullptr, 0, st))) return rc;
+    {
+        size_t n = (size_t)N * d;
+        k_oproj_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(zero_nd, t->o, a.xC, n, a.zC, a.dz);
+        lc.count();
+    }
+    k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.zC, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, N);
+    lc.count();
+    float* guS = t->gu + (size_t)N * 2 * F;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wgate, d, guS, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
+    if ((rc = gemm_act_weight(lc, uS, d, w->Wup, d, guS + F, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        size_t n = (size_t)N * F;
+        k_swiglu_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hC, t->dh);
+        lc.count();
+    }
+    // xC_next = z' + h' W^T + h' dW^T
+    if ((rc = gemm_act_weight(lc, t->hC, F, w->Wdown, F, xC_next, d, N, d, F, 1.f, a.zC, d, st))) return rc;
+    tc_split_pair(lc, dW, d, F, t->dW);
+    return gemm_pair_pair(lc, t->hC, F, t->dW, F, xC_next, d, N, d, F, 1.f, nullptr, 0, true, st);
+}
+
 // One block on one stream with teacher and student fused: every product runs once on the stacked rows
 // (rows [0,N) teacher, [N,2N) student) and the attention is one launch.  Fastest when nothing can overlap.
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a) {
@@ -552,7 +597,7 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     // S7 (Eq. 9); the dual solver only needs the token-contiguous copy of the student features
     t->own_S_T = a.S_T;
     if (a.dual) transpose_split(lc, a.hC, N, F, t->ldT, t->XT);
-    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st, a.precise_stats != 0);
+    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, a.accumulate_stats != 0, st, a.precise_stats != 0);
     mark(a, lc, 7);
     return PKV_OK;
 }
@@ -564,7 +609,7 @@ void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const 
     if (xF_next) gemm_act_weight(lc, t->hF, F, Wdown, F, xF_next, d, N, d, F, 1.f, zF, d, status);
     // D = T - hC dW^T
     (void)dW;      // its bf16 pair was written by the solver's last product
-    gemm_pair_pair(lc, t->hC, F, t->dW, F, Dm, d, N, d, F, -1.f, R, d, false, status);
+    if (Dm) gemm_pair_pair(lc, t->hC, F, t->dW, F, Dm, d, N, d, F, -1.f, R, d, false, status);
 }
 
 }  // namespace pkv

@@ -134,6 +134,7 @@ struct TcForwardArgs {
     const float* dx;    // student half: xF - xC entering this block (state difference carried between blocks)
     float *part_m, *part_l, *part_O;
     int dual;           // 1: only the token-contiguous copy of the student features is prepared in S7
+    int accumulate_stats;   // 1: S_H, S_T are added to (streamed reference sets, Eq. 9) instead of overwritten
     int precise_stats;  // 1: statistics from bf16 triples in six passes (small ridge coefficient), else pairs in three
     DevStatus* status;
     cudaEvent_t* ev;    // stage marks (index = stage) or nullptr
@@ -169,5 +170,10 @@ void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int 
                     int mode, DevStatus* status);
 void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* d, int N, const void* Wdown, const float* dW,
                     const float* zF, const float* R, float* xF_next, float* D, DevStatus* status);
+// Student block re-run with the patched down projection (Algorithm 1, student propagation):
+// xC_next = z' + (W + dW) h' for the tokens in a.xC against the compact cache.  zero_nd: scratch [N][d].
+int tc_student_propagate(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a, const float* dW,
+                         float* zero_nd, float* xC_next);
+void tc_split_pair(const Lc& lc, const float* src, long long rows, long long cols, Pair out);
 
 }  // namespace pkv

@@ -704,6 +704,10 @@ __global__ void k_transpose_blocks(Trip X3, Trip XT3, int n, int ld, int s) {
     }
 }
 
+void tc_split_pair(const Lc& lc, const float* src, long long rows, long long cols, Pair out) {
+    launch_split3(lc, src, cols, (int)rows, (int)cols, Trip{{out.hi, out.lo, nullptr}}, cols, 2);
+}
+
 static void six_pass(TcGemm& g, const Trip& A, long long lda, long long arows, long long acols, const Trip& B,
                      long long ldb, long long brows, long long bcols) {
     // (hi,hi) (hi,mid) (mid,hi) (hi,lo) (lo,hi) (mid,mid)

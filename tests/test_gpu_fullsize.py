@@ -250,3 +250,26 @@ def test_three_block_stack_at_config3_shape_free_running_and_reanchored(B):
     print("final states: xF %.2e, xC %.2e" % (eF, eC))
     assert eF <= 1e-3 and eC <= 1e-3
     ctx.close()
+
+
+def test_ridge_solve_at_the_true_mlp_width_of_llama3_8b(B):
+    """F = d_ff = 14336 (the width the paper's W in R^{d x d_ff} has in the Llama-3-8B-shaped model): statistics from
+    1024 reference tokens (rank-deficient, as in every benchmark config), solve against the oracle's fp64 Cholesky.
+    d is cut to 256 rows of dW to bound the oracle's time; the F x F system is the full one."""
+    import torch
+    cfg = gen.scaled_config(gen.benchmark_config(2), F=14336, d=256, Hq=2, Hkv=1, N=1024, L=256, budget=16)
+    r = np.random.default_rng(7)
+    X = (r.standard_normal((cfg.N, cfg.F)) * np.exp(r.uniform(-1.5, 0.5, cfg.F))).astype(np.float32)
+    R = (0.05 * r.standard_normal((cfg.N, cfg.d))).astype(np.float32)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    gH, gT = ctx.gram(torch.from_numpy(X).cuda(), torch.from_numpy(R).cuda())
+    S_H, S_T = orc.sufficient_statistics(X, R)
+    assert H.rel_fro(gT.cpu().numpy(), S_T) <= 2e-4
+    lam = orc.ridge_lambda(S_H, 0.1)
+    want = orc.ridge_solve(S_H, S_T, lam)
+    dW, st = ctx.ridge_solve(gH, gT, 0.1)
+    err = H.rel_fro(dW.cpu().numpy(), want)
+    print("F = 14336: dW rel fro err %.3e, lambda %.5g (oracle %.5g), min pivot %.3g" % (err, st["lambda_eff"], lam, st["min_pivot"]))
+    np.testing.assert_allclose(st["lambda_eff"], lam, rtol=1e-3)
+    assert err <= 2e-3
+    ctx.close()

@@ -612,6 +612,54 @@ def test_lambda_sweep_with_the_teacher_run_once_matches_separate_stacks(B):
     ctx.close()
 
 
+@pytest.mark.parametrize("engine_name,lam0", [("tc", 0.1), ("tc", 1e-3), ("simt", 0.1)])
+def test_streamed_reference_set_equals_one_call_and_the_oracle(B, engine_name, lam0):
+    """Sec. 2.3 / Eq. 9: the reference set fed in three parts (whole chunks each), only S_H and S_T kept between the
+    calls, against one pkv_build_patch on all tokens and against the oracle; the teacher's next states come out of
+    the parts, the student's from the propagation call with the patched block (Algorithm 1)."""
+    import torch
+    cfg = small_cfg("bf16", hd=128, Hq=4, Hkv=2, d=256, F=192, L=1000, N=210)
+    engine = B.ENGINE_AUTO if engine_name == "tc" else B.ENGINE_SIMT
+    lay = H.make_problem(cfg, per_head_budget=[100, 37])
+    xF = lay["x0"]
+    xC = (xF + 0.02 * np.random.default_rng(5).standard_normal(xF.shape)).astype(np.float32)
+    chunk_off = [0, 40, 41, 100, 150, 210]
+    parts = [(0, 41, [0, 40, 41]), (41, 150, [0, 59, 109]), (150, 210, [0, 60])]       # token range, local chunk offsets
+    ref = H.run_oracle(cfg, lay, xF, xC, chunk_off, lam0)
+    ctx = B.PkvContext(B.dims_from_config(cfg, N_max=cfg.N, b_max=100), engine=engine)
+    w = B.to_device(lay["weights"], cfg.dtype)
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    off, idx = gen.kept_to_csr(lay["kept"])
+    idx_t = torch.from_numpy(idx).cuda()
+    tF, tC = torch.from_numpy(xF).cuda(), torch.from_numpy(xC).cuda()
+    whole = ctx.build_patch(w, kv["K"], kv["V"], off, idx_t, tF, tC, chunk_off, cfg.L, lam0)
+    ctx.stream_begin(lam0)
+    xFn = []
+    for a, e, co in parts:
+        xFn.append(ctx.stream_add(w, kv["K"], kv["V"], off, idx_t, tF[a:e].contiguous(), tC[a:e].contiguous(), co, cfg.L,
+                                  want_next=True))
+    dW, st = ctx.stream_finish()
+    e_or = H.rel_fro(dW.cpu().numpy(), ref["dW"])
+    e_one = H.rel_fro(dW.cpu().numpy(), whole["dW"].cpu().numpy())
+    print("streamed in 3 parts (%s, lambda0 %g): dW vs oracle %.3e, vs one call %.3e" % (engine_name, lam0, e_or, e_one))
+    assert e_or <= DW_TOL and e_one <= 2e-3
+    np.testing.assert_allclose(st["lambda_eff"], ref["lam"], rtol=2e-3)
+    np.testing.assert_allclose(st["target_fro2"], ref["T_fro2"], rtol=2e-2)
+    assert H.rel_fro(torch.cat(xFn).cpu().numpy(), ref["xF_next"]) <= 1e-3
+    if engine_name == "tc":
+        xCn = torch.cat([ctx.stream_propagate(w, kv["K"], kv["V"], off, idx_t, tC[a:e].contiguous(), co, cfg.L, dW)
+                         for a, e, co in parts])
+        assert H.rel_fro(xCn.cpu().numpy(), ref["xC_next"]) <= 1e-3
+    # a second stream on the same context starts from zero sums
+    ctx.stream_begin(lam0)
+    ctx.stream_add(w, kv["K"], kv["V"], off, idx_t, tF, tC, chunk_off, cfg.L)
+    dW2, _ = ctx.stream_finish()
+    assert H.rel_fro(dW2.cpu().numpy(), ref["dW"]) <= DW_TOL
+    with pytest.raises(B.PkvError):                      # no stream open
+        ctx.stream_finish()
+    ctx.close()
+
+
 # ------------------------------------------------------------------ boundary
 
 def test_boundary_rejects_bad_arguments(B):
@@ -621,7 +669,7 @@ def test_boundary_rejects_bad_arguments(B):
         B.PkvContext(B.dims_from_config(gen.scaled_config(cfg, hd=96)), engine=B.ENGINE_SIMT)
     assert ei.value.code == -2
     with pytest.raises(B.PkvError) as ei:
-        B.PkvContext(B.dims_from_config(gen.scaled_config(cfg, F=9000)), engine=B.ENGINE_SIMT)
+        B.PkvContext(B.dims_from_config(gen.scaled_config(cfg, F=40000)), engine=B.ENGINE_SIMT)
     assert ei.value.code == -2
     lay = H.make_problem(cfg)
     x = lay["x0"]
