@@ -293,6 +293,18 @@ int pkv_gram(pkv_ctx* ctx, const float* X, const float* R, int32_t n, float* S_H
 int pkv_gram_noalloc(const float* X, const float* R, int32_t n, int32_t F, int32_t d, float* S_H, float* S_T,
                      int accumulate, void* cuda_stream);
 
+/* Rank-r patch (appendix, low-rank weight patches): with M = dW S_H dW^T (d x d) and U_r its r leading
+ * eigenvectors, the patch is stored as U_r [d][r] and B_r = U_r^T dW [r][F] ((d + F) r numbers), dW_r = U_r B_r.
+ * dW [d][F] and S_H [F][F] (full symmetric matrix): device fp32, read only.  U, Br: device fp32 out; dW_r: optional
+ * device fp32 [d][F] out (the expanded rank-r patch) or NULL; ritz_values: optional device fp32 [r + 8] out, the
+ * leading approximate eigenvalues of M in descending order (the gap after the r-th says how well U_r is determined;
+ * eigenvector signs are arbitrary).  M is formed on the tensor cores (fp32-equivalent products), the eigenvectors by
+ * `iterations` sweeps (0 = 24) of subspace iteration with Rayleigh-Ritz on r + 8 vectors in fp64.  scratch: caller-
+ * owned device memory of pkv_low_rank_scratch_bytes().  Tensor-core engine; r <= 40 and r + 8 <= d.  Synchronises. */
+size_t pkv_low_rank_scratch_bytes(const pkv_dims* dims, int r);
+int pkv_low_rank(pkv_ctx* ctx, const float* dW, const float* S_H, int32_t r, int32_t iterations, void* scratch,
+                 size_t scratch_bytes, float* U, float* Br, float* dW_r, float* ritz_values);
+
 /* Ridge solve alone (Eq. 7-8): dW = S_T (S_H + lambda I)^{-1}.  S_H, S_T are read, not
  * modified. */
 int pkv_ridge_solve(pkv_ctx* ctx, const float* S_H, const float* S_T, float lambda, int lambda_mode,

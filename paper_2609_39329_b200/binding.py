@@ -134,6 +134,11 @@ def lib() -> C.CDLL:
     L.pkv_gram_noalloc.restype = C.c_int
     L.pkv_gram_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                    C.c_int, C.c_void_p]
+    L.pkv_low_rank_scratch_bytes.restype = C.c_size_t
+    L.pkv_low_rank_scratch_bytes.argtypes = [P(pkv_dims), C.c_int]
+    L.pkv_low_rank.restype = C.c_int
+    L.pkv_low_rank.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t,
+                               C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     L.pkv_ridge_solve.restype = C.c_int
     L.pkv_ridge_solve.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_void_p, P(pkv_stats)]
     L.pkv_fp32_product.restype = C.c_int
@@ -466,6 +471,22 @@ class PkvContext:
         if rc != 0:
             self._raise(rc)
         return C_out
+
+    def low_rank(self, dW, S_H, r, iterations=0, want_expanded=True):
+        """pkv_low_rank: returns dict(U [d][r], Br [r][F], dW_r [d][F] or None, ritz [r + 8])."""
+        torch = self.torch
+        d, F = self.dims.d, self.dims.F
+        need = int(self.L.pkv_low_rank_scratch_bytes(C.byref(self.dims), int(r)))
+        scratch = torch.empty(need, dtype=torch.uint8, device=dW.device)
+        U = torch.empty((d, r), dtype=torch.float32, device=dW.device)
+        Br = torch.empty((r, F), dtype=torch.float32, device=dW.device)
+        dWr = torch.empty((d, F), dtype=torch.float32, device=dW.device) if want_expanded else None
+        ritz = torch.empty(r + 8, dtype=torch.float32, device=dW.device)
+        rc = self.L.pkv_low_rank(self.h, _ptr(dW), _ptr(S_H), int(r), int(iterations), _ptr(scratch), need, _ptr(U),
+                                 _ptr(Br), _ptr(dWr), _ptr(ritz))
+        if rc != 0:
+            self._raise(rc)
+        return {"U": U, "Br": Br, "dW_r": dWr, "ritz": ritz}
 
     def ridge_solve(self, S_H, S_T, lam, mode=LAMBDA_PAPER):
         torch = self.torch

@@ -1206,6 +1206,27 @@ extern "C" int pkv_fp32_product(pkv_ctx* c, const float* A, const float* B, int3
     return end_call(c, nullptr, nullptr);
 }
 
+extern "C" size_t pkv_low_rank_scratch_bytes(const pkv_dims* dims, int r) {
+    if (dims_ok(dims) != PKV_OK || r <= 0) return 0;
+    return pkv::tc_lowrank_scratch_bytes(dims->d, dims->F, r);
+}
+
+extern "C" int pkv_low_rank(pkv_ctx* c, const float* dW, const float* S_H, int32_t r, int32_t iterations, void* scratch,
+                            size_t scratch_bytes, float* U, float* Br, float* dW_r, float* ritz_values) {
+    if (!c || !dW || !S_H || !scratch || !U || !Br || r <= 0) return PKV_ERR_INVALID_ARG;
+    if (c->engine == PKV_ENGINE_SIMT) return PKV_ERR_UNSUPPORTED;
+    const void* ptrs[] = {dW, S_H, scratch, U, Br, dW_r, ritz_values};
+    for (const void* q : ptrs)
+        if ((uintptr_t)q & 15) return PKV_ERR_INVALID_ARG;
+    if (scratch_bytes < pkv::tc_lowrank_scratch_bytes(c->dims.d, c->dims.F, r)) return PKV_ERR_NOMEM;
+    Lc lc{c->st, &c->launches, c->map_cache};
+    begin_call(c);
+    int rc = pkv::tc_lowrank(lc, &c->b.tc, &c->dims, dW, S_H, r, iterations > 0 ? iterations : 24, scratch, U, Br, dW_r,
+                             ritz_values, c->b.status);
+    if (rc != PKV_OK) return rc;
+    return end_call(c, nullptr, nullptr);
+}
+
 extern "C" int pkv_ridge_solve(pkv_ctx* c, const float* S_H, const float* S_T, float lambda, int lambda_mode,
                                float* dW, pkv_stats* stats) {
     if (!c || !S_H || !S_T || !dW) return PKV_ERR_INVALID_ARG;

@@ -81,7 +81,9 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
                         __nv_bfloat16* const* S_T_triple);   // optional: dW's bf16 pair out; S_T already split
 
 int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const float* A, const float* B, int M, int N,
-                    int K, float alpha, float* C, bool accumulate, int passes, int nacc, DevStatus* status);
+                    int K, float alpha, float* C, bool accumulate, int passes, int nacc, DevStatus* status,
+                    bool b_in_factor_buffer = false);
+
 
 // bf16 hi/lo pairs of fp32 activations: v ~= hi + lo with hi = bf16(v), lo = bf16(v - hi).
 struct Pair {
@@ -140,6 +142,11 @@ struct TcForwardArgs {
     cudaEvent_t* ev;    // stage marks (index = stage) or nullptr
     cudaEvent_t* evT;   // 6 marks around the teacher half's stages (S1-2, S3, S4, S5, S9 share) or nullptr
 };
+
+// Rank-r patch (appendix): U [d][r], Br [r][F] = U^T dW, optional dWr [d][F] = U Br, optional evals [r + 8].
+size_t tc_lowrank_scratch_bytes(int d, int F, int r);
+int tc_lowrank(const Lc& lc, TcBuffers* t, const pkv_dims* D, const float* dW, const float* S_H, int r, int iters,
+               void* scratch, float* U, float* Br, float* dWr, float* evals_out, DevStatus* status);
 
 void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, int* nsplitC);
 // q/k_new/v_new of `a` are fp32; rope_tab != nullptr rotates q and k on the way in.

@@ -736,11 +736,16 @@ static void three_pass(TcGemm& g, const Trip& A, long long lda, long long arows,
 // tensor-core passes (6: triples, fp32-equivalent; 3: pairs).  The building block of the factorisation,
 // exported for unit tests.
 int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const float* A, const float* B, int M, int N,
-                    int K, float alpha, float* C, bool accumulate, int passes, int nacc, DevStatus* status) {
+                    int K, float alpha, float* C, bool accumulate, int passes, int nacc, DevStatus* status,
+                    bool b_in_factor_buffer) {
     const long long K8 = (K + 7) / 8 * 8;
-    if ((size_t)M * K8 > cap_elems || (size_t)N * K8 > cap_elems) return PKV_ERR_UNSUPPORTED;
+    // B's parts go to the S_T X^T operand buffer, or (a square operand as large as the system) to the factor's
+    // buffer, which is cleared again afterwards: parts of it that no kernel of the solve writes must read as zero
+    const size_t capB = b_in_factor_buffer ? (size_t)t->nmax * t->nmax : cap_elems;
+    if ((size_t)M * K8 > cap_elems || (size_t)N * K8 > capB) return PKV_ERR_UNSUPPORTED;
     if (passes != 3 && passes != 6) return PKV_ERR_INVALID_ARG;
     Trip A3{{t->S2[0], t->S2[1], t->S2[2]}}, B3{{t->Z2[0], t->Z2[1], t->Z2[2]}};
+    if (b_in_factor_buffer) B3 = Trip{{t->L3[0], t->L3[1], t->L3[2]}};
     if (K8 != K) {
         for (int i = 0; i < 3; ++i) {
             cudaMemsetAsync(A3.a[i], 0, (size_t)M * K8 * 2, lc.st);
@@ -755,7 +760,10 @@ int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const flo
     g.M = M; g.N = N; g.K = K; g.batch = 1; g.alpha = alpha;
     g.C = C; g.ldc = N; g.c_rows = M; g.c_cols = N; g.accumulate = accumulate;
     g.nacc = nacc;
-    return gemm_tc(lc, g, status);
+    const int rc = gemm_tc(lc, g, status);
+    if (b_in_factor_buffer)
+        for (int i = 0; i < 3; ++i) cudaMemsetAsync(t->L3[i], 0, (size_t)t->nmax * t->nmax * 2, lc.st);
+    return rc;
 }
 
 // largest pairs * s * s over the doubling levels (elements of the TT workspace)

@@ -273,3 +273,33 @@ def test_ridge_solve_at_the_true_mlp_width_of_llama3_8b(B):
     np.testing.assert_allclose(st["lambda_eff"], lam, rtol=1e-3)
     assert err <= 2e-3
     ctx.close()
+
+
+def test_low_rank_patch_at_config2_width(B):
+    """Rank-32 patch (appendix) at d = F = 4096: the weighted truncation loss tr((dW - dW_r) S_H (dW - dW_r)^T) equals
+    the sum of the discarded eigenvalues of dW S_H dW^T (the oracle's), the leading eigenvalues agree, and the
+    factors have orthonormal columns.  The loss is insensitive to the order inside eigenvalue clusters, so this
+    holds whether or not the 32nd gap is open."""
+    import torch
+    cfg = gen.benchmark_config(2)
+    r, n = 32, 512
+    rng = np.random.default_rng(61)
+    X = rng.standard_normal((n, cfg.F)).astype(np.float32)
+    basis = rng.standard_normal((cfg.F, 64)).astype(np.float32)
+    mix = rng.standard_normal((64, cfg.d)).astype(np.float32)
+    R = ((X @ basis) * (0.9 ** np.arange(64, dtype=np.float32))[None, :]) @ mix * np.float32(1e-2)
+    S_H, S_T = orc.sufficient_statistics(X, R)
+    dW = orc.ridge_solve(S_H, S_T, orc.ridge_lambda(S_H, 0.1))
+    _, _, _, ev_o = orc.low_rank_patch(dW, S_H, r)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    out = ctx.low_rank(torch.from_numpy(dW.astype(np.float32)).cuda(), torch.from_numpy(S_H.astype(np.float32)).cuda(), r)
+    dWr = out["dW_r"].cpu().numpy().astype(np.float64)
+    E = dW - dWr
+    loss = float(np.sum((E @ S_H) * E))
+    U = out["U"].cpu().numpy().astype(np.float64)
+    print("rank-32 patch at d = F = 4096: weighted loss %.6g vs discarded eigenvalues %.6g (kept %.6g)"
+          % (loss, ev_o[r:].sum(), ev_o[:r].sum()))
+    np.testing.assert_allclose(loss, ev_o[r:].sum(), rtol=5e-3)
+    np.testing.assert_allclose(out["ritz"].cpu().numpy()[:8], ev_o[:8], rtol=2e-3)
+    np.testing.assert_allclose(U.T @ U, np.eye(r), atol=1e-5)
+    ctx.close()

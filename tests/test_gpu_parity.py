@@ -472,6 +472,43 @@ def test_fp32_equivalent_product_and_its_accumulation_bias(B, M, N, K):
     ctx.close()
 
 
+@pytest.mark.parametrize("d,F,n,r", [(256, 192, 500, 32), (128, 128, 60, 8)])
+def test_low_rank_patch_matches_oracle(B, d, F, n, r):
+    """Appendix, low-rank weight patches: dW_r = U_r U_r^T dW with U_r the leading eigenvectors of dW S_H dW^T,
+    against the oracle's eigendecomposition; the weighted loss of the truncation is the sum of the discarded
+    eigenvalues; the stored factors have (d + F) r numbers."""
+    import torch
+    cfg = small_cfg("bf16", F=F, d=d, Hq=max(d // 64, 1), Hkv=1)
+    rng = np.random.default_rng(51)
+    X = rng.standard_normal((n, F))
+    # targets with a decaying spectrum so that the r-th eigenvalue gap is open
+    basis = rng.standard_normal((F, d))
+    R = (X @ basis) * (0.85 ** np.arange(d))[None, :] + 1e-3 * rng.standard_normal((n, d))
+    S_H, S_T = orc.sufficient_statistics(X, R)
+    dW = orc.ridge_solve(S_H, S_T, orc.ridge_lambda(S_H, 0.1))
+    U_o, B_o, dWr_o, ev_o = orc.low_rank_patch(dW, S_H, r)
+    assert ev_o[r - 1] > 1.3 * ev_o[r]                       # an open gap: dW_r is then well determined
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    t_dW = torch.from_numpy(dW.astype(np.float32)).cuda()
+    t_SH = torch.from_numpy(S_H.astype(np.float32)).cuda()
+    out = ctx.low_rank(t_dW, t_SH, r)
+    dWr = out["dW_r"].cpu().numpy().astype(np.float64)
+    err = H.rel_fro(dWr, dWr_o)
+    # loss identity: tr((dW - dW_r) S_H (dW - dW_r)^T) = sum of the discarded eigenvalues
+    E = dW - dWr
+    loss = np.trace(E @ S_H @ E.T)
+    print("rank-%d patch (d %d, F %d): dW_r rel fro err %.3e; weighted loss %.6g vs discarded eigenvalues %.6g"
+          % (r, d, F, err, loss, ev_o[r:].sum()))
+    assert err <= DW_TOL
+    np.testing.assert_allclose(loss, ev_o[r:].sum(), rtol=2e-3)
+    np.testing.assert_allclose(out["ritz"].cpu().numpy()[:r], ev_o[:r], rtol=2e-3)
+    U = out["U"].cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(U.T @ U, np.eye(r), atol=1e-5)                      # orthonormal columns
+    np.testing.assert_allclose(out["Br"].cpu().numpy(), U.T @ dW, rtol=0, atol=1e-4 * np.abs(dW).max() * np.sqrt(d))
+    np.testing.assert_allclose(dWr, U @ out["Br"].cpu().numpy().astype(np.float64), rtol=0, atol=1e-5 * np.abs(dW).max())
+    ctx.close()
+
+
 # ------------------------------------------------------------------ whole block
 
 def test_config1_tiny_fp32_end_to_end(B):
