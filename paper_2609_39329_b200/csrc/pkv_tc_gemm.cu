@@ -46,11 +46,37 @@ struct alignas(64) GemmTcParams {
     int skip_tile00;          // the tile at (blockIdx.x, blockIdx.y) = (0, 0) is left alone
     int out_col0_only;        // bf16 parts are written by the tiles of the first block column only
     int tiles_m, tiles_n, batch, nbuf;   // persistent kernel: tile grid and accumulator buffers in tensor memory
+    int out_vec;              // the bf16 parts can be stored 16 bytes at a time (alignment of pointers, stride, offsets)
     DevStatus* status;
 };
 
 constexpr int kGemmMaxStages = 6;
+
+__device__ __forceinline__ uint32_t pack2_bf16(__nv_bfloat16 a, __nv_bfloat16 b) {
+    return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
+}
 constexpr int kGemmBarBytes = (2 * kGemmMaxStages + 1) * 8 + 16;
+
+// 32 consecutive values of one output row as up to three bf16 parts (successive roundings), 16-byte stores
+__device__ __forceinline__ void store_parts_row(const GemmTcParams& p, const float (&v)[32], size_t o) {
+#pragma unroll
+    for (int c8 = 0; c8 < 4; ++c8) {
+        uint32_t h[4], m[4], l[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float x0 = v[c8 * 8 + 2 * e], x1 = v[c8 * 8 + 2 * e + 1];
+            const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+            const float r0 = x0 - __bfloat162float(h0), r1 = x1 - __bfloat162float(h1);
+            const __nv_bfloat16 m0 = __float2bfloat16_rn(r0), m1 = __float2bfloat16_rn(r1);
+            h[e] = pack2_bf16(h0, h1);
+            m[e] = pack2_bf16(m0, m1);
+            l[e] = pack2_bf16(__float2bfloat16_rn(r0 - __bfloat162float(m0)), __float2bfloat16_rn(r1 - __bfloat162float(m1)));
+        }
+        *reinterpret_cast<uint4*>(p.out[0] + o + c8 * 8) = make_uint4(h[0], h[1], h[2], h[3]);
+        if (p.nout > 1) *reinterpret_cast<uint4*>(p.out[1] + o + c8 * 8) = make_uint4(m[0], m[1], m[2], m[3]);
+        if (p.nout > 2) *reinterpret_cast<uint4*>(p.out[2] + o + c8 * 8) = make_uint4(l[0], l[1], l[2], l[3]);
+    }
+}
 
 // One k-tile stage holds every distinct operand tile once: nA x [128][64] and nB x [BN][64] bf16,
 // and all passes are issued from it (the shared operand of a split product is not re-read).
@@ -258,7 +284,11 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                         }
                     }
                 }
-                if (p.nout > 0 && (!p.out_col0_only || blockIdx.x == 0)) {
+                if (p.nout > 0 && (!p.out_col0_only || blockIdx.x == 0) && p.out_vec && ncol == 32) {
+                    // bf16 parts straight from the registers: the lane owns 32 consecutive columns of its row,
+                    // four 16-byte stores per part
+                    if (lane < nrows) store_parts_row(p, v, (size_t)(rowa0 + lane) * p.ldo + (col - p.out_col_off));
+                } else if (p.nout > 0 && (!p.out_col0_only || blockIdx.x == 0)) {
                     // bf16 parts: through the warp's smem tile so that a warp writes 64 contiguous bytes per row
 #pragma unroll
                     for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = v[j];
@@ -520,7 +550,9 @@ __global__ void __launch_bounds__(192) k_gemm_tcp(const __grid_constant__ GemmTc
                         }
                     }
                 }
-                if (p.nout > 0 && (!p.out_col0_only || (first_col && c0 < 128))) {
+                if (p.nout > 0 && (!p.out_col0_only || (first_col && c0 < 128)) && p.out_vec && ncol == 32) {
+                    if (lane < nrows) store_parts_row(p, v, (size_t)(rowa0 + lane) * p.ldo + (col - p.out_col_off));
+                } else if (p.nout > 0 && (!p.out_col0_only || (first_col && c0 < 128))) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = v[j];
                     __syncwarp();
@@ -841,6 +873,13 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     p.vec_ok = (g.C && ((uintptr_t)g.C & 15) == 0 && g.ldc % 4 == 0 && g.c_col0 % 4 == 0 && g.c_zcol % 4 == 0 &&
                 (!g.addend || (((uintptr_t)g.addend & 15) == 0 && g.ldadd % 4 == 0))) ? 1 : 0;
     p.status = status;
+    p.out_vec = 0;
+    if (g.nout > 0) {
+        bool ok = g.ldo % 8 == 0 && (g.c_col0 - g.out_col_off) % 8 == 0 && g.c_zcol % 8 == 0;
+        for (int i = 0; i < g.nout; ++i) ok = ok && (((uintptr_t)g.out[i]) & 15) == 0;
+        // every row offset (c_row0 + z c_zrow + ...) * ldo is then a multiple of 8 elements as well
+        p.out_vec = ok ? 1 : 0;
+    }
     if (gemm_persistent()) {
         if (BN == 64) return launch_gemm_p<64>(lc, p, g.batch);
         if (BN == 256) return launch_gemm_p<256>(lc, p, g.batch);
