@@ -47,7 +47,7 @@ struct Trip {
 // The block is processed in 16-column sub-steps: the 16 x 16 diagonal piece is factored by one warp
 // entirely in registers (lane i holds row i, columns are exchanged with shuffles), the rows below
 // it by forward substitution (one row per thread), then the trailing lower triangle is updated.
-constexpr int kPotrfThreads = 1024;
+constexpr int kPotrfThreads = 512;       // 16 warps: up to 128 registers per thread keep the pivot chain free of spills
 
 // ---- warp-level TF32 tiles (mma.sync m16n8k8) in split form: each fp32 operand is the sum of three
 // TF32 parts (11 + 11 + 11 significant bits) and six products (hh, hm, mh, hl, lh, mm) are accumulated in
@@ -334,10 +334,10 @@ __global__ void __launch_bounds__(kPotrfThreads) k_chain128(const __grid_constan
                     A[row][c] = v;
                 }
             }
-        } else if (ok) {
-            // the other warps clear X (R1: the triple of L is dead, its MMAs have completed)
-            for (int i = tid - 512; i < PB * PB; i += kPotrfThreads - 512) X[i >> 7][i & 127] = 0.f;
         }
+        // clear X (R1: the triple of L is dead, its MMAs have completed)
+        if (ok)
+            for (int i = tid; i < PB * PB; i += kPotrfThreads) X[i >> 7][i & 127] = 0.f;
         __syncthreads();
     } else if (ok) {
         // ---- first block: the lower part from global memory (identity outside the block's extent), lambda on the diagonal
@@ -489,8 +489,9 @@ __global__ void __launch_bounds__(kPotrfThreads) k_chain128(const __grid_constan
                 // warps 4, 8, ... share warp 0's scheduler: they stay out of the way of the pivot chain
                 const int rem = PB - base;
                 const int tm = (rem >> 4) - 1, tn = rem >> 3;          // row tiles below the first one
-                const int wi = warp - 1 - (warp >> 2);                  // index among the 24 working warps
-                for (int tile = wi; tile < tm * tn; tile += 24) {
+                constexpr int kWork = (kPotrfThreads / 32) - (kPotrfThreads / 128);   // warps with (warp & 3) != 0
+                const int wi = warp - 1 - (warp >> 2);                  // index among the working warps
+                for (int tile = wi; tile < tm * tn; tile += kWork) {
                     const int i0 = base + 16 + (tile / tn) * 16, n0 = base + (tile % tn) * 8;
                     if (n0 > i0 + 15) continue;                     // entirely above the diagonal
                     trail_tile(c0, i0, n0);
