@@ -917,7 +917,8 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         cudaStreamWaitEvent(sB, evF, 0);
         {   // P_b: panel, kept as a bf16 triple in L3
             TcGemm g{};
-            six_pass(g, P3, PB, F, PB, X3, ld, F, F);
+            if (well_conditioned) three_pass(g, P3, PB, F, PB, X3, ld, F, F);
+            else six_pass(g, P3, PB, F, PB, X3, ld, F, F);
             g.a_row0 = k1;
             g.b_row0 = k0; g.b_col0 = k0;
             g.M = rem; g.N = PB; g.K = PB; g.batch = 1; g.alpha = 1.f;
@@ -927,7 +928,8 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         }
         if (rem > PB) {   // U_b: G22 -= L21 L21^T on the lower triangle, the first diagonal tile left to the chain
             TcGemm g{};
-            six_pass(g, L3, ld, F, F, L3, ld, F, F);
+            if (well_conditioned) three_pass(g, L3, ld, F, F, L3, ld, F, F);
+            else six_pass(g, L3, ld, F, F, L3, ld, F, F);
             g.a_row0 = k1; g.a_col0 = k0; g.b_row0 = k1; g.b_col0 = k0;
             g.M = rem; g.N = rem; g.K = PB; g.batch = 1; g.alpha = -1.f;
             g.C = const_cast<float*>(G); g.ldc = ld; g.accumulate = true; g.lower_only = true; g.skip_tile00 = true;
@@ -972,8 +974,9 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     }
     // ---- 2. X = L^{-1} by recursive doubling ----
     // cond(L) = sqrt(cond(G)): with a well-conditioned ridge matrix (a few tens) the rounding of these products
-    // (pairs: 2^-16) reaches dW unamplified and three passes are enough; the factorisation above always takes six
-    // (its trailing updates cancel)
+    // (pairs: 2^-16) reaches dW unamplified and three passes are enough.  The same holds for the factorisation
+    // above: lambda is then of the order of the diagonal of S_H and the trailing updates do not cancel; with a small
+    // lambda0 they do, and everything takes triples in six passes with separated accumulators.
     for (int s = PB; s < F; s *= 2) {
         int P = 0;
         while ((2 * P + 1) * s < F) ++P;
