@@ -228,6 +228,11 @@ size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d, int dua
     t->q = c.pair(2 * N * Dq);
     t->kn = c.take<__nv_bfloat16>(2 * N * Dkv);
     t->vn = c.take<__nv_bfloat16>(2 * N * Dkv);
+    t->K16 = t->Kc16 = nullptr;
+    if (d->hd == 128) {
+        t->K16 = c.take<__nv_bfloat16>((size_t)d->Hkv * d->L * d->hd + 8);
+        t->Kc16 = c.take<__nv_bfloat16>((size_t)d->Hkv * d->b_max * d->hd + 128 * d->hd);
+    }
     int tps, nF, nC;
     tc_attn_plan(d, d->N_max, d->b_max, &tps, &nF, &nC);
     const size_t rows = N * (d->Hq / d->Hkv);

@@ -108,6 +108,8 @@ struct TcBuffers {
     Pair q;             // [2][Hq][N][hd]   rotated, pre-scaled queries for the attention kernel
     __nv_bfloat16* kn;  // [2][Hkv][N][hd]  reference tokens' keys
     __nv_bfloat16* vn;  // [2][Hkv][N][hd]  reference tokens' values
+    void* K16;          // fp16 copy of the full cache's keys [Hkv][L][hd] (hd = 128 attention, fp16 key operands)
+    void* Kc16;         // fp16 copy of the compact cache's keys [Hkv * b_max][hd]
     float* part_m;      // attention split partials [splits][Hkv][N*g]
     float* part_l;
     float* part_O;      // [splits][Hkv][N*g][hd]

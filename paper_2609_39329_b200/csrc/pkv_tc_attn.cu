@@ -16,6 +16,7 @@
 // Partial (m, l, O) per split go to global memory; the combine kernel merges the splits of both
 // streams and forms dA = aF - aC in fp32.
 #include <cuda.h>
+#include <stdlib.h>
 #include <math.h>
 
 #include "pkv_ptx.cuh"
@@ -34,7 +35,7 @@ using namespace ptx;
 __global__ void __launch_bounds__(256) k_attn_prep(const float* __restrict__ q, long long ldq,
                                                    const float* __restrict__ k, const float* __restrict__ v,
                                                    long long ldkv, const float* __restrict__ rope_tab, int N, int Hq,
-                                                   int Hkv, int hd, int s_begin, int s_count,
+                                                   int Hkv, int hd, int s_begin, int s_count, int q_f16,
                                                    __nv_bfloat16* __restrict__ qhi,
                                                    __nv_bfloat16* __restrict__ qlo, __nv_bfloat16* __restrict__ kn,
                                                    __nv_bfloat16* __restrict__ vn) {
@@ -60,18 +61,31 @@ __global__ void __launch_bounds__(256) k_attn_prep(const float* __restrict__ q, 
         float a = (lo * co - hi * si) * sc, b = (hi * co + lo * si) * sc;
         int kh = h / g, hg = h % g;
         size_t o = (((size_t)s * Hkv + kh) * ((size_t)N * g) + (size_t)tok * g + hg) * hd + c;
-        __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
-        qhi[o] = ah;
-        qhi[o + half] = bh;
-        qlo[o] = __float2bfloat16_rn(a - __bfloat162float(ah));
-        qlo[o + half] = __float2bfloat16_rn(b - __bfloat162float(bh));
+        if (q_f16) {
+            // one fp16 part (11 significant bits): the attention kernel multiplies it with the bf16 keys in one pass
+            __half* qh = reinterpret_cast<__half*>(qhi);
+            qh[o] = __float2half_rn(a);
+            qh[o + half] = __float2half_rn(b);
+        } else {
+            __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
+            qhi[o] = ah;
+            qhi[o + half] = bh;
+            qlo[o] = __float2bfloat16_rn(a - __bfloat162float(ah));
+            qlo[o + half] = __float2bfloat16_rn(b - __bfloat162float(bh));
+        }
     } else if (h < Hq + Hkv) {
         int kh = h - Hq;
         const float* p = k + (size_t)row * ldkv + (size_t)kh * hd + c;
         float lo = p[0], hi = p[half];
         size_t o = (((size_t)s * Hkv + kh) * N + tok) * hd + c;
-        kn[o] = __float2bfloat16_rn(lo * co - hi * si);
-        kn[o + half] = __float2bfloat16_rn(hi * co + lo * si);
+        if (q_f16) {
+            __half* kh16 = reinterpret_cast<__half*>(kn);
+            kh16[o] = __float2half_rn(lo * co - hi * si);
+            kh16[o + half] = __float2half_rn(hi * co + lo * si);
+        } else {
+            kn[o] = __float2bfloat16_rn(lo * co - hi * si);
+            kn[o + half] = __float2bfloat16_rn(hi * co + lo * si);
+        }
     } else {
         int kh = h - Hq - Hkv;
         const float* p = v + (size_t)row * ldkv + (size_t)kh * hd + c;
@@ -79,6 +93,30 @@ __global__ void __launch_bounds__(256) k_attn_prep(const float* __restrict__ q, 
         vn[o] = __float2bfloat16_rn(p[0]);
         vn[o + half] = __float2bfloat16_rn(p[half]);
     }
+}
+
+// bf16 -> fp16, eight elements per thread.  Exact for every bf16 value of magnitude in [2^-14, 65504] (8 significant
+// bits fit in fp16's 11); smaller magnitudes round to fp16 subnormals (absolute error below 3e-8).
+__global__ void __launch_bounds__(256) k_bf16_to_f16(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n8) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n8) return;
+    const uint4 v = src[i];
+    const uint32_t in[4] = {v.x, v.y, v.z, v.w};
+    uint32_t out[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float lo = __uint_as_float(in[e] << 16), hi = __uint_as_float(in[e] & 0xffff0000u);
+        const __half2 h = __floats2half2_rn(lo, hi);
+        out[e] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    dst[i] = make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+static void to_f16(const Lc& lc, const void* src, void* dst, size_t elems) {
+    const size_t n8 = elems / 8;
+    if (!n8) return;
+    k_bf16_to_f16<<<(unsigned)((n8 + 255) / 256), 256, 0, lc.st>>>((const uint4*)src, (uint4*)dst, n8);
+    lc.count();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -470,6 +508,12 @@ static int launch_attn(const Lc& lc, const AttnTcParams& p, int qtiles, int zcou
     return PKV_OK;
 }
 
+// Query operand of the hd = 128 kernel: one fp16 part (default) or a bf16 hi + lo pair (PKV_ATTN_Q=pair)
+static bool attn_q_f16() {
+    static const bool v = [] { const char* e = getenv("PKV_ATTN_Q"); return !(e && e[0] == 'p'); }();
+    return v;
+}
+
 // hd = 128: the two-tile kernel of pkv_tc_attn2.cu (operands already prepared in t->q, t->kn, t->vn)
 int launch_attn2(const Lc& lc, const Attn2Params& p, int qpairs, int zcount);
 static int attention_tc2(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status) {
@@ -481,15 +525,29 @@ static int attention_tc2(const Lc& lc, TcBuffers* t, const pkv_dims* d, const At
     if ((rc = tc_make_map_3d(&p.mQlo, t->q.lo, 2 * Hkv, rows, hd, hd, (uint64_t)rows * hd, 128))) return rc;
     if ((rc = tc_make_map_3d(&p.mKn, t->kn, 2 * Hkv, N, hd, hd, (uint64_t)N * hd, 128))) return rc;
     if ((rc = tc_make_map_3d(&p.mVn, t->vn, 2 * Hkv, N, hd, hd, (uint64_t)N * hd, 128))) return rc;
+    // fp16 mode: the key operands are fp16 copies of the (bf16) caches, made here; values stay bf16
+    const bool f16 = attn_q_f16();
+    const void* Kfull = a.K;
+    const void* Kcomp = a.Kc;
+    if (f16) {
+        if (d->L > 0 && a.mode != 2) {
+            to_f16(lc, a.K, t->K16, (size_t)Hkv * d->L * hd);
+            Kfull = t->K16;
+        } else {
+            Kfull = t->K16;
+        }
+        if (a.total_kept > 0 && a.mode != 1) to_f16(lc, a.Kc, t->Kc16, (size_t)a.total_kept * hd);
+        Kcomp = t->Kc16;
+    }
     if (d->L > 0) {
-        if ((rc = tc_make_map_3d(&p.mK, a.K, Hkv, d->L, hd, hd, (uint64_t)d->L * hd, 128))) return rc;
+        if ((rc = tc_make_map_3d(&p.mK, Kfull, Hkv, d->L, hd, hd, (uint64_t)d->L * hd, 128))) return rc;
         if ((rc = tc_make_map_3d(&p.mV, a.V, Hkv, d->L, hd, hd, (uint64_t)d->L * hd, 128))) return rc;
     } else {
         p.mK = p.mKn;
         p.mV = p.mVn;
     }
     if (a.total_kept > 0) {
-        if ((rc = tc_make_map_2d(&p.mKc, a.Kc, a.total_kept, hd, hd, 128))) return rc;
+        if ((rc = tc_make_map_2d(&p.mKc, Kcomp, a.total_kept, hd, hd, 128))) return rc;
         if ((rc = tc_make_map_2d(&p.mVc, a.Vc, a.total_kept, hd, hd, 128))) return rc;
     } else {
         p.mKc = p.mKn;      // never read: no compact-cache tiles exist
@@ -501,6 +559,7 @@ static int attention_tc2(const Lc& lc, TcBuffers* t, const pkv_dims* d, const At
     p.part_m = t->part_m; p.part_l = t->part_l; p.part_O = t->part_O;
     p.status = status;
     p.z0 = (a.mode == 2) ? p.nsplitF : 0;
+    p.q_f16 = f16 ? 1 : 0;
     rc = launch_attn2(lc, p, (rows + 255) / 256,
                       a.mode == 0 ? p.nsplitF + p.nsplitC : (a.mode == 1 ? p.nsplitF : p.nsplitC));
     if (rc != PKV_OK) return rc;
@@ -519,7 +578,8 @@ int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
     {
         size_t total = (size_t)s_count * N * (d->Hq + 2 * Hkv) * (hd / 2);
         k_attn_prep<<<(unsigned)((total + 255) / 256), 256, 0, lc.st>>>(a.q, a.ldq, a.k_new, a.v_new, a.ldkv, rope_tab, N,
-                                                                        d->Hq, Hkv, hd, s_begin, s_count, t->q.hi, t->q.lo,
+                                                                        d->Hq, Hkv, hd, s_begin, s_count,
+                                                                        (hd == 128 && attn_q_f16()) ? 1 : 0, t->q.hi, t->q.lo,
                                                                         t->kn, t->vn);
         lc.count();
     }

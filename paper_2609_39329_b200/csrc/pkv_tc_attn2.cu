@@ -149,13 +149,14 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
     if (warp == 0) {
         if (lane == 0 && ntiles > 0) {
             const int zq = stream * p.Hkv + kh;
-            mbar_expect_tx(bar(B_QFULL), 4 * kTile);
+            mbar_expect_tx(bar(B_QFULL), (p.q_f16 ? 2 : 4) * kTile);
 #pragma unroll
             for (int t = 0; t < 2; ++t)
 #pragma unroll
                 for (int sb = 0; sb < 2; ++sb) {
                     tma_load_3d(base + kQ + (2 * t) * kTile + sb * 16384, &p.mQhi, bar(B_QFULL), sb * 64, r0 + t * 128, zq);
-                    tma_load_3d(base + kQ + (2 * t + 1) * kTile + sb * 16384, &p.mQlo, bar(B_QFULL), sb * 64, r0 + t * 128, zq);
+                    if (!p.q_f16)
+                        tma_load_3d(base + kQ + (2 * t + 1) * kTile + sb * 16384, &p.mQlo, bar(B_QFULL), sb * 64, r0 + t * 128, zq);
                 }
             for (int j = 0; j < ntiles; ++j) {
                 const int t = t_begin + j;
@@ -182,12 +183,14 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
         }
     } else if (warp == 1) {
         if (lane == 0 && ntiles > 0) {
-            constexpr uint32_t idesc_qk = idesc_bf16(128, 128);
+            // fp16 mode: queries AND keys are fp16 (both operand format fields 0); the two operands of one MMA must
+            // have the same 16-bit type
+            const uint32_t idesc_qk = p.q_f16 ? (idesc_bf16(128, 128) & ~((7u << 7) | (7u << 10))) : idesc_bf16(128, 128);
+            const int q_passes = p.q_f16 ? 1 : 2;
             constexpr uint32_t idesc_pv = idesc_bf16(128, HD) | (1u << 16);      // B operand MN-major
             auto issue_qk = [&](int gq) {
                 const uint32_t kd = base + kK;
-#pragma unroll
-                for (int ps = 0; ps < 2; ++ps) {
+                for (int ps = 0; ps < q_passes; ++ps) {
                     const uint32_t qd = base + kQ + (2 * gq + ps) * kTile;
 #pragma unroll
                     for (int ks = 0; ks < HD / 16; ++ks) {

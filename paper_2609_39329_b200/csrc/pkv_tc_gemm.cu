@@ -821,7 +821,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     // 128 x 256 tiles move a third fewer operand bytes per flop than 128 x 128; taken when they still give
     // at least two waves of CTAs (and the C tile is not prefetched: that variant is 128 wide)
     const long long tiles256 = (long long)((g.N + 255) / 256) * ((g.M + 127) / 128) * g.batch;
-    const bool wide = g.N >= 512 && tiles256 >= 2 * 148 && !(g.C && g.accumulate) && !g.lower_only && g.k_tri != 2 &&
+    const bool wide = g.N >= 512 && tiles256 >= 2 * 148 && !(g.C && g.accumulate) && !g.lower_only &&
                       g.nacc < 4;
     const int BN = (g.skip_tile00 || g.out_col0_only) ? 128 : ((g.N <= 64) ? 64 : (wide ? 256 : 128));
     MapCache* cache = (MapCache*)lc.map_cache;
