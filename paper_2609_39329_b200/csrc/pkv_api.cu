@@ -64,9 +64,12 @@ const GreenApi& green_api() {
     return api;
 }
 
-// A stream whose kernels run on at least `want_sms` SMs of the current device and leave the rest alone.
+}  // namespace
+
+namespace pkv {
+// A green context that owns at least `want_sms` SMs of the current device and leaves the rest alone.
 // Returns false (nothing created) when the partition cannot be made.
-bool make_partition_stream(int want_sms, cudaStream_t* stream, void** gctx_out, int* got_sms) {
+bool green_partition_create(int want_sms, void** gctx_out, int* got_sms) {
     const GreenApi& a = green_api();
     if (!a.ok || want_sms <= 0) return false;
     int ord = 0;
@@ -83,14 +86,34 @@ bool make_partition_stream(int want_sms, cudaStream_t* stream, void** gctx_out, 
     if (a.GenerateDesc(&desc, &part, 1) != CUDA_SUCCESS) return false;
     CUgreenCtx g;
     if (a.GreenCtxCreate(&g, desc, dev, CU_GREEN_CTX_DEFAULT_STREAM) != CUDA_SUCCESS) return false;
-    CUstream st;
-    if (a.GreenCtxStreamCreate(&st, g, CU_STREAM_NON_BLOCKING, 0) != CUDA_SUCCESS) {
-        a.GreenCtxDestroy(g);
-        return false;
-    }
-    *stream = (cudaStream_t)st;
     *gctx_out = (void*)g;
     *got_sms = (int)part.sm.smCount;
+    return true;
+}
+
+// A stream of that partition: its kernels run on the partition's SMs only.
+bool green_partition_stream(void* gctx, int priority, cudaStream_t* stream) {
+    CUstream st;
+    if (!gctx || green_api().GreenCtxStreamCreate(&st, (CUgreenCtx)gctx, CU_STREAM_NON_BLOCKING, priority) != CUDA_SUCCESS)
+        return false;
+    *stream = (cudaStream_t)st;
+    return true;
+}
+
+void green_partition_destroy(void* gctx) {
+    if (gctx) green_api().GreenCtxDestroy((CUgreenCtx)gctx);
+}
+}  // namespace pkv
+
+namespace {
+bool make_partition_stream(int want_sms, cudaStream_t* stream, void** gctx_out, int* got_sms) {
+    void* g = nullptr;
+    if (!green_partition_create(want_sms, &g, got_sms)) return false;
+    if (!green_partition_stream(g, 0, stream)) {
+        green_partition_destroy(g);
+        return false;
+    }
+    *gctx_out = g;
     return true;
 }
 }  // namespace
@@ -408,7 +431,7 @@ extern "C" void pkv_destroy(pkv_ctx* c) {
     if (c->host_lhead) cudaFreeHost(c->host_lhead);
     if (c->host_lstatus) cudaFreeHost(c->host_lstatus);
     if (c->tstream) { cudaStreamSynchronize(c->tstream); cudaStreamDestroy(c->tstream); }
-    if (c->tgreen) green_api().GreenCtxDestroy((CUgreenCtx)c->tgreen);
+    green_partition_destroy(c->tgreen);
     for (int i = 0; i < kRing; ++i) {
         if (c->evTea[i]) cudaEventDestroy(c->evTea[i]);
         if (c->evStu[i]) cudaEventDestroy(c->evStu[i]);

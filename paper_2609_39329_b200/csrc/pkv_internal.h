@@ -48,6 +48,11 @@ struct Lc {
     void count(int n = 1) const { if (launches) *launches += n; }
 };
 
+// ---- SM partitions (pkv_api.cu): a green context owning a subset of the SMs, and streams inside it ----
+bool green_partition_create(int want_sms, void** gctx_out, int* got_sms);
+bool green_partition_stream(void* gctx, int priority, cudaStream_t* stream);
+void green_partition_destroy(void* gctx);
+
 // ---- pkv_simt.cu -----------------------------------------------------------------------
 void gather_kept(const Lc& lc, int elem_bytes, const void* K, const void* V, const int32_t* idx,
                  const int32_t* head_off_dev, int Hkv, int L, int hd, int total, void* Kc, void* Vc,

@@ -26,6 +26,7 @@ struct TcGemm {
     int b_row0, b_col0, b_zrow, b_zcol;
     int M, N, K, batch;
     float* C;
+    float* const* C_ind;   // optional: device location holding the fp32 output base (C then only gives the alignment)
     long long ldc;
     const float* addend;
     long long ldadd;
@@ -37,8 +38,10 @@ struct TcGemm {
     float alpha;
     bool accumulate, lower_only;
     int k_tri;      // 0: dense; 1: B lower triangular (skip k tiles past the row); 2: B upper triangular
+    int a_tri;      // the same for the A operand (1: A[m][k] = 0 for k > m; 2: A[m][k] = 0 for k < m)
     bool skip_tile00;     // leave the first tile (rows and columns [0,128) of the product) alone
     bool out_col0_only;   // write the bf16 parts only for the first 128-column block of the product
+    unsigned long long* stamps;   // optional device array of 8 global-timer marks (phases of the first CTA)
     int nacc;       // 0/1: one fp32 accumulator; 2 or 4: the hi x hi pass of a split product is accumulated apart
                     // from the cross passes (and in several parts), which removes most of the tensor core's
                     // truncation bias from sums of same-signed terms; pass 0 must be the hi x hi pass
@@ -56,6 +59,18 @@ int tc_make_map_3d(CUtensorMap* m, const void* ptr, uint64_t d2, uint64_t rows, 
 struct Pair;
 // Workspace of the tensor-core ridge solve: bf16 triples (hi, mid, lo) of the factor L, its inverse X,
 // the inverse's transpose, the current panel, the doubling temporaries; pairs of S_T and S_T X^T.
+constexpr int kSolveEvents = 6;
+constexpr int kSolveGraphs = 4;
+// One captured solve: replayed when the operands, the shape and the precision plan are the same.
+struct SolveGraph {
+    const float *G, *S_T;
+    int n, ld, d;
+    bool well, triple, aligned;
+    const void *pair_hi, *pair_lo;
+    cudaGraphExec_t exec;
+    int64_t launches;
+    unsigned long long used;
+};
 struct TcSolveBuffers {
     __nv_bfloat16* L3[3];
     __nv_bfloat16* X3[3];
@@ -66,10 +81,18 @@ struct TcSolveBuffers {
     __nv_bfloat16* Z2[3];
     int nmax;              // largest system the arrays are sized for
     cudaStream_t aux;      // high-priority helper stream of the factorisation's critical chain
-    cudaEvent_t ev[4];
+    cudaStream_t bulk;     // helper stream: panels and trailing updates
+    cudaStream_t aux2;     // helper stream: the doubling levels of the inverse beside the factorisation
+    cudaEvent_t ev[kSolveEvents];
     CUtensorMap chainP[3], chainX[3];   // tensor maps of the chain kernel's operands, valid for (chain_n, chain_ld)
     int chain_n, chain_ld;
     long long* stamps;     // phase marks of the chain kernel (profiling aid)
+    float** slot;          // device location of the result's address, read by a captured solve's final products
+    DevStatus* gstatus;    // status word of a captured solve (copied from / to the caller's)
+    cudaStream_t origin;   // stream the solve is captured on
+    SolveGraph graphs[kSolveGraphs];
+    int n_graphs, graph_off;
+    unsigned long long graph_clock;
 };
 void tc_solve_destroy(TcSolveBuffers* t);
 size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, int nmax, int dmax);

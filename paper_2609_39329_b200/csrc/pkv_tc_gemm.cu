@@ -34,6 +34,7 @@ struct alignas(64) GemmTcParams {
     int b_row0, b_col0, b_zrow, b_zcol;
     int c_row0, c_col0, c_zrow, c_zcol, c_rows, c_cols;
     float* C;
+    float* const* C_ind;      // if set, the fp32 output base is read from this device location instead of C
     long long ldc;
     float alpha;
     const float* addend;
@@ -41,13 +42,14 @@ struct alignas(64) GemmTcParams {
     __nv_bfloat16* out[3];
     long long ldo;
     int nout, out_col_off;
-    int accumulate, lower_only, k_tri, vec_ok;
+    int accumulate, lower_only, k_tri, a_tri, vec_ok;
     int nacc;                 // TMEM accumulators per tile (1, 2 or 4), see TcGemm::nacc
     int skip_tile00;          // the tile at (blockIdx.x, blockIdx.y) = (0, 0) is left alone
     int out_col0_only;        // bf16 parts are written by the tiles of the first block column only
     int tiles_m, tiles_n, batch, nbuf;   // persistent kernel: tile grid and accumulator buffers in tensor memory
     int out_vec;              // the bf16 parts can be stored 16 bytes at a time (alignment of pointers, stride, offsets)
     DevStatus* status;
+    unsigned long long* stamps;   // optional: global-timer marks of the first CTA's phases (profiling aid)
 };
 
 constexpr int kGemmMaxStages = 6;
@@ -78,6 +80,14 @@ __device__ __forceinline__ void store_parts_row(const GemmTcParams& p, const flo
     }
 }
 
+__device__ __forceinline__ void gemm_stamp(const GemmTcParams& p, int i) {
+    if (p.stamps && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) {
+        unsigned long long ns;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns));
+        p.stamps[i] = ns;
+    }
+}
+
 // One k-tile stage holds every distinct operand tile once: nA x [128][64] and nB x [BN][64] bf16,
 // and all passes are issued from it (the shared operand of a split product is not re-read).
 // PRE: the epilogue warps fetch the fp32 C tile they will add to (read-modify-write products of the
@@ -96,6 +106,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     if (p.lower_only && n0 > m0 + 127) return;
     if (p.skip_tile00 && blockIdx.x == 0 && blockIdx.y == 0) return;
     pdl_launch_dependents();
+    if (threadIdx.x == 0) gemm_stamp(p, 0);
     // absolute coordinates of this tile's output; tiles entirely outside the stored region do nothing
     const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
     if (crow0 >= p.c_rows || ccol0 >= p.c_cols) return;
@@ -119,6 +130,9 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     int kt_begin = 0, kt_end = (p.K + 63) / 64;
     if (p.k_tri == 1) kt_end = min(kt_end, (n0 + BN + 63) / 64);
     if (p.k_tri == 2) kt_begin = min(kt_end, n0 / 64);
+    //   a_tri: the same for a triangular A operand (1: A[m][k] = 0 for k > m; 2: A[m][k] = 0 for k < m)
+    if (p.a_tri == 1) kt_end = min(kt_end, (m0 + 128 + 63) / 64);
+    if (p.a_tri == 2) kt_begin = max(kt_begin, min(kt_end, m0 / 64));
     const int ktiles = kt_end - kt_begin;
 
     if (threadIdx.x == 0) {
@@ -144,9 +158,10 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     // an earlier stage already failed: the call reports it.  The status word may change while the CTA starts
     // (another CTA's error), so one thread reads it and the whole CTA takes the same branch.
     volatile int* skip_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
-    if (threadIdx.x == 0) *skip_flag = p.status->code;
+    if (threadIdx.x == 0) { gemm_stamp(p, 1); *skip_flag = p.status->code; }
     __syncthreads();
     const bool skip = *skip_flag != 0;
+    if (threadIdx.x == 0) gemm_stamp(p, 2);
 
     if (skip) {
         // nothing to do: fall through to the teardown
@@ -175,6 +190,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                 const int s = it % STAGES;
                 if (!mbar_wait(bars + 8 * s, (it / STAGES) & 1, abort_flag, p.status, 2)) { ok = false; break; }
                 tc_fence_after();
+                if (it == 0) gemm_stamp(p, 3);
                 const uint32_t sa = base + s * stage_bytes;
                 for (int ps = 0; ps < p.npass; ++ps) {
                     const uint64_t da = smem_desc_sw128(sa + p.pa[ps] * kA);
@@ -191,6 +207,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                 mma_commit(bars + 8 * (STAGES + s));
             }
             if (ok) mma_commit(bars + 8 * (2 * STAGES));
+            gemm_stamp(p, 4);
         }
     } else {
         // epilogue: TMEM -> registers -> per-warp smem tile -> row-contiguous global accesses
@@ -199,13 +216,14 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         const int rowa0 = crow0 + q * 32;            // ... and its absolute output row
         const int nrows = max(0, min(32, min(p.M - rl0, p.c_rows - rowa0)));
         const bool vec_ok = p.vec_ok != 0;
+        float* const Cp = p.C_ind ? *p.C_ind : p.C;
         // PRE: whole-tile prefetch of C, legal when the tile is full width and vector-aligned
         constexpr int kPre = PRE ? BN / 4 : 1;
         float4 cpre[kPre];
-        const bool pre_ok = PRE && p.C && p.accumulate && vec_ok && lane < nrows &&
+        const bool pre_ok = PRE && Cp && p.accumulate && vec_ok && lane < nrows &&
                             min(p.N - n0, p.c_cols - ccol0) >= BN;
         if (PRE && pre_ok) {
-            const float* crow = p.C + (size_t)(rowa0 + lane) * p.ldc + ccol0;
+            const float* crow = Cp + (size_t)(rowa0 + lane) * p.ldc + ccol0;
 #pragma unroll
             for (int j = 0; j < kPre; ++j) cpre[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
         }
@@ -214,6 +232,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
             ok = mbar_wait(bars + 8 * (2 * STAGES), 0, abort_flag, p.status, 3);
             tc_fence_after();
         }
+        if (warp == 2 && lane == 0) gemm_stamp(p, 5);
         if (ok) {
             float* stg = staging + q * (32 * 33);
 #pragma unroll
@@ -241,10 +260,10 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = p.alpha * __uint_as_float(r[j]);
-                if (p.C && lane < nrows) {
+                if (Cp && lane < nrows) {
                     // fp32 output: every lane owns one row; 128 contiguous bytes, loads batched ahead of stores
                     const size_t row = (size_t)(rowa0 + lane);
-                    float* crow = p.C + row * p.ldc + col;
+                    float* crow = Cp + row * p.ldc + col;
                     const float* arow = p.addend ? p.addend + row * p.ldadd + col : nullptr;
                     if (vec_ok && ncol == 32) {
                         if (arow) {
@@ -313,6 +332,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         }
     }
     // teardown: after an abort give copies in flight time to land before the CTA's smem is released
+    if (warp == 2 && lane == 0) gemm_stamp(p, 6);
     if (*abort_flag) {
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
     }
@@ -322,6 +342,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         tc_fence_after();
         tmem_dealloc(tbase, (uint32_t)(BN * nacc));
     }
+    if (threadIdx.x == 0) gemm_stamp(p, 7);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -399,11 +420,13 @@ __global__ void __launch_bounds__(192) k_gemm_tcp(const __grid_constant__ GemmTc
         const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
         return crow0 < p.c_rows && ccol0 < p.c_cols;
     };
-    auto k_range = [&](int n0, int& kt_begin, int& kt_end) {
+    auto k_range = [&](int m0, int n0, int& kt_begin, int& kt_end) {
         kt_begin = 0;
         kt_end = (p.K + 63) / 64;
         if (p.k_tri == 1) kt_end = min(kt_end, (n0 + BN + 63) / 64);
         if (p.k_tri == 2) kt_begin = min(kt_end, n0 / 64);
+        if (p.a_tri == 1) kt_end = min(kt_end, (m0 + 128 + 63) / 64);
+        if (p.a_tri == 2) kt_begin = max(kt_begin, min(kt_end, m0 / 64));
     };
 
     if (skip) {
@@ -415,7 +438,7 @@ __global__ void __launch_bounds__(192) k_gemm_tcp(const __grid_constant__ GemmTc
             for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
                 int z, m0, n0, kb, ke;
                 if (!decode(t, z, m0, n0)) continue;
-                k_range(n0, kb, ke);
+                k_range(m0, n0, kb, ke);
                 const int ar = p.a_row0 + z * p.a_zrow + m0, ac = p.a_col0 + z * p.a_zcol;
                 const int br = p.b_row0 + z * p.b_zrow + n0, bc = p.b_col0 + z * p.b_zcol;
                 for (int kt = kb; kt < ke; ++kt, ++it) {
@@ -437,7 +460,7 @@ __global__ void __launch_bounds__(192) k_gemm_tcp(const __grid_constant__ GemmTc
             for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
                 int z, m0, n0, kb, ke;
                 if (!decode(t, z, m0, n0)) continue;
-                k_range(n0, kb, ke);
+                k_range(m0, n0, kb, ke);
                 const uint32_t buf = tcount % (uint32_t)nbuf;
                 // the epilogue must have drained this accumulator buffer (first use: passes at once)
                 if (!mbar_wait(bar_acce + 8 * buf, ((tcount / nbuf) & 1) ^ 1, abort_flag, p.status, 4)) { ok = false; break; }
@@ -473,12 +496,13 @@ __global__ void __launch_bounds__(192) k_gemm_tcp(const __grid_constant__ GemmTc
         const int q = warp & 3;
         float* stg = staging + q * (32 * 33);
         const bool vec_ok = p.vec_ok != 0;
+        float* const Cp = p.C_ind ? *p.C_ind : p.C;
         uint32_t tcount = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
             int z, m0, n0, kb, ke;
             if (!decode(t, z, m0, n0)) continue;
-            k_range(n0, kb, ke);
+            k_range(m0, n0, kb, ke);
             const bool has_acc = ke > kb;
             const uint32_t buf = tcount % (uint32_t)nbuf;
             const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
@@ -513,9 +537,9 @@ __global__ void __launch_bounds__(192) k_gemm_tcp(const __grid_constant__ GemmTc
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = p.alpha * __uint_as_float(r[j]);
-                if (p.C && lane < nrows) {
+                if (Cp && lane < nrows) {
                     const size_t row = (size_t)(rowa0 + lane);
-                    float* crow = p.C + row * p.ldc + col;
+                    float* crow = Cp + row * p.ldc + col;
                     const float* arow = p.addend ? p.addend + row * p.ldadd + col : nullptr;
                     if (vec_ok && ncol == 32) {
                         if (arow) {
@@ -855,12 +879,13 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     p.b_row0 = g.b_row0; p.b_col0 = g.b_col0; p.b_zrow = g.b_zrow; p.b_zcol = g.b_zcol;
     p.c_row0 = g.c_row0; p.c_col0 = g.c_col0; p.c_zrow = g.c_zrow; p.c_zcol = g.c_zcol;
     p.c_rows = g.c_rows; p.c_cols = g.c_cols;
-    p.C = g.C; p.ldc = g.ldc; p.alpha = g.alpha; p.addend = g.addend; p.ldadd = g.ldadd;
+    p.C = g.C; p.C_ind = g.C_ind; p.ldc = g.ldc; p.alpha = g.alpha; p.addend = g.addend; p.ldadd = g.ldadd;
     for (int i = 0; i < 3; ++i) p.out[i] = g.out[i];
     p.ldo = g.ldo; p.nout = g.nout; p.out_col_off = g.out_col_off;
     p.accumulate = g.accumulate ? 1 : 0;
     p.lower_only = g.lower_only ? 1 : 0;
     p.k_tri = g.k_tri;
+    p.a_tri = g.a_tri;
     p.skip_tile00 = g.skip_tile00 ? 1 : 0;
     p.out_col0_only = g.out_col0_only ? 1 : 0;
     // several accumulators only for products with one hi x hi pass and cross passes, and only if they fit
@@ -873,6 +898,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     p.vec_ok = (g.C && ((uintptr_t)g.C & 15) == 0 && g.ldc % 4 == 0 && g.c_col0 % 4 == 0 && g.c_zcol % 4 == 0 &&
                 (!g.addend || (((uintptr_t)g.addend & 15) == 0 && g.ldadd % 4 == 0))) ? 1 : 0;
     p.status = status;
+    p.stamps = g.stamps;
     p.out_vec = 0;
     if (g.nout > 0) {
         bool ok = g.ldo % 8 == 0 && (g.c_col0 - g.out_col_off) % 8 == 0 && g.c_zcol % 8 == 0;

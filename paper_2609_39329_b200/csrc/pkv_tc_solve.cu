@@ -9,13 +9,18 @@
 //      in shared memory; the panel (a GEMM with the block inverse) and the trailing update (a GEMM on
 //      the lower triangle) of every column run beside that chain;
 //   2. X = L^{-1} by recursive doubling from the 128-block inverses:
-//      [A 0; C B]^{-1} = [A^{-1} 0; -B^{-1} C A^{-1}  B^{-1}], every level two batched GEMMs;
+//      [A 0; C B]^{-1} = [A^{-1} 0; -B^{-1} C A^{-1}  B^{-1}], two GEMMs per pair of blocks, issued on a
+//      third stream as soon as a pair's columns are factored (only the pairs that contain the last column
+//      remain after the factorisation);
 //   3. dW = (S_T X^T) X, two GEMMs that skip the zero tiles of the triangular factor.
+// The launches of one solve (about 150 on three streams) are captured into a CUDA graph per operand set and
+// replayed, see tc_ridge_solve_impl.
 #include <math.h>
 #include <stdio.h>
 #include <stdlib.h>
 
 #include "pkv_ptx.cuh"
+#include <time.h>
 #include "pkv_tc.h"
 
 namespace pkv {
@@ -137,7 +142,7 @@ struct alignas(64) ChainParams {
     long long* stamps;        // optional [blocks][kChainStamps] clock64 marks of thread 0 (phase profile), or null
 };
 
-constexpr int kChainStamps = 16;
+constexpr int kChainStamps = 18;     // 16 clock64 marks + the global timer (ns) at the kernel's start and end
 constexpr int kChainR = 3 * 128 * 128 * 2;                 // 96 KB: one operand triple
 constexpr int kChainBar = 2 * kChainR;
 constexpr int kChainSmemBytes = kChainBar + 64 + 1024;
@@ -177,7 +182,15 @@ __global__ void __launch_bounds__(kPotrfThreads) k_chain128(const __grid_constan
     const bool with_update = k0 > 0;
     long long* stamps = p.stamps ? p.stamps + (size_t)(k0 / PB) * kChainStamps : nullptr;
     auto stamp = [&](int i) { if (stamps && tid == 0) stamps[i] = clock64(); };
+    auto wall = [&](int i) {
+        if (stamps && tid == 0) {
+            unsigned long long ns;
+            asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns));
+            stamps[i] = (long long)ns;
+        }
+    };
     stamp(0);
+    wall(16);
 
     pdl_launch_dependents();
     if (tid == 0) {
@@ -627,6 +640,7 @@ __global__ void __launch_bounds__(kPotrfThreads) k_chain128(const __grid_constan
     }
     }      // ok
     stamp(7);
+    wall(17);
     // teardown: after an abort give copies in flight time to land before the CTA's smem is released
     if (*abort_flag) {
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
@@ -662,9 +676,9 @@ static void launch_split3(const Lc& lc, const float* src, long long lds, int row
 }
 
 // Diagonal blocks: XT3[k0 + c][k0 + r] = X3[k0 + r][k0 + c] for the 128-blocks on the diagonal (clipped to n x n).
-__global__ void k_transpose_diag(Trip X3, Trip XT3, int n, int ld) {
+__global__ void k_transpose_diag(Trip X3, Trip XT3, int n, int ld, int blk0) {
     __shared__ __nv_bfloat16 t[3][32][33];
-    const int k0 = blockIdx.z * PB;
+    const int k0 = (blk0 + blockIdx.z) * PB;
     const int r0 = k0 + blockIdx.y * 32, c0 = k0 + blockIdx.x * 32;
     for (int j = threadIdx.y; j < 32; j += 8) {
         const int r = r0 + j, c = c0 + threadIdx.x;
@@ -684,9 +698,9 @@ __global__ void k_transpose_diag(Trip X3, Trip XT3, int n, int ld) {
 }
 
 // XT3[2sz + c][s + 2sz + r] = X3[s + 2sz + r][2sz + c]   (r < s clipped to the n x n matrix, c < s); row stride ld
-__global__ void k_transpose_blocks(Trip X3, Trip XT3, int n, int ld, int s) {
+__global__ void k_transpose_blocks(Trip X3, Trip XT3, int n, int ld, int s, int pair0) {
     __shared__ __nv_bfloat16 t[3][32][33];
-    const int z = blockIdx.z;
+    const int z = pair0 + blockIdx.z;
     const int r0 = s + 2 * s * z + blockIdx.y * 32, c0 = 2 * s * z + blockIdx.x * 32;
     for (int j = threadIdx.y; j < 32; j += 8) {
         const int r = r0 + j, c = c0 + threadIdx.x;
@@ -761,20 +775,39 @@ int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const flo
     g.M = M; g.N = N; g.K = K; g.batch = 1; g.alpha = alpha;
     g.C = C; g.ldc = N; g.c_rows = M; g.c_cols = N; g.accumulate = accumulate;
     g.nacc = nacc;
+    // PKV_GEMM_TRACE=1: phase times of the product's first CTA, and the launch-to-launch time around it
+    static const bool gtrace = getenv("PKV_GEMM_TRACE") != nullptr;
+    static unsigned long long* dstamps = nullptr;
+    if (gtrace) {
+        if (!dstamps) cudaMalloc(&dstamps, 3 * 8 * sizeof(unsigned long long));
+        cudaMemsetAsync(dstamps, 0, 3 * 8 * sizeof(unsigned long long), lc.st);
+        for (int rep = 0; rep < 2; ++rep) { g.stamps = dstamps + 8 * rep; gemm_tc(lc, g, status); }
+        g.stamps = dstamps + 16;
+    }
     const int rc = gemm_tc(lc, g, status);
+    if (gtrace) {
+        unsigned long long h[24];
+        cudaStreamSynchronize(lc.st);
+        cudaMemcpy(h, dstamps, sizeof(h), cudaMemcpyDeviceToHost);
+        for (int rep = 0; rep < 3; ++rep) {
+            const unsigned long long* s = h + 8 * rep;
+            fprintf(stderr, "gemm %dx%dx%d passes %d acc %d, launch %d: entry +0 | dependencies met %.2f | status read %.2f | first k-tile "
+                            "landed %.2f | last MMA issued %.2f | accumulator ready %.2f | epilogue done %.2f | exit %.2f us",
+                    M, N, K, passes, nacc, rep, (s[1] - s[0]) * 1e-3, (s[2] - s[0]) * 1e-3, (s[3] - s[0]) * 1e-3, (s[4] - s[0]) * 1e-3,
+                    (s[5] - s[0]) * 1e-3, (s[6] - s[0]) * 1e-3, (s[7] - s[0]) * 1e-3);
+            if (rep > 0) fprintf(stderr, " ; entry %.2f us after the previous launch's exit", ((double)s[0] - (double)h[8 * (rep - 1) + 7]) * 1e-3);
+            fprintf(stderr, "\n");
+        }
+    }
     if (b_in_factor_buffer)
         for (int i = 0; i < 3; ++i) cudaMemsetAsync(t->L3[i], 0, (size_t)t->nmax * t->nmax * 2, lc.st);
     return rc;
 }
 
-// largest pairs * s * s over the doubling levels (elements of the TT workspace)
+// elements of the doubling's temporary TT
 static size_t tt_elems(int F) {
-    size_t best = (size_t)PB * PB;
-    for (long long s = PB; s < F; s *= 2) {
-        long long P = 0;
-        while ((2 * P + 1) * s < F) ++P;
-        if ((size_t)(P * s * s) > best) best = (size_t)(P * s * s);
-    }
+    size_t best = (size_t)PB * PB;      // one pair at a time: the largest level below F
+    for (long long s = PB; s < F; s *= 2) best = (size_t)(s * s);
     return best;
 }
 
@@ -799,6 +832,8 @@ size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, int nmax, int d
         t->Z2[i] = (__nv_bfloat16*)take(dm * F * 2);
     }
     t->stamps = (long long*)take(((F + PB - 1) / PB) * kChainStamps * sizeof(long long));
+    t->slot = (float**)take(256);
+    t->gstatus = (DevStatus*)take(256);
     return off;
 }
 
@@ -817,7 +852,16 @@ int tc_solve_init(TcSolveBuffers* t) {
     // the factorisation's critical chain (diagonal block, panel, next-column update) runs at the highest
     // priority so that its small kernels are not queued behind the bulk trailing update's CTAs
     if (cudaStreamCreateWithPriority(&t->aux, cudaStreamNonBlocking, greatest) != cudaSuccess) return PKV_ERR_CUDA;
-    for (int i = 0; i < 4; ++i)
+    // ... the panels and trailing updates (needed two chain steps later) below it, and the doubling levels of the
+    // inverse (needed only at the end) below those, filling the SMs the others leave idle
+    const int mid = (least + greatest) / 2;
+    if (cudaStreamCreateWithPriority(&t->bulk, cudaStreamNonBlocking, mid) != cudaSuccess) return PKV_ERR_CUDA;
+    if (cudaStreamCreateWithPriority(&t->aux2, cudaStreamNonBlocking, least) != cudaSuccess) return PKV_ERR_CUDA;
+    if (cudaStreamCreateWithFlags(&t->origin, cudaStreamNonBlocking) != cudaSuccess) return PKV_ERR_CUDA;
+    t->n_graphs = 0;
+    t->graph_off = 0;
+    t->graph_clock = 0;
+    for (int i = 0; i < kSolveEvents; ++i)
         if (cudaEventCreateWithFlags(&t->ev[i], cudaEventDisableTiming) != cudaSuccess) return PKV_ERR_CUDA;
     t->chain_n = t->chain_ld = 0;
     static PerDeviceOnce once;
@@ -836,7 +880,15 @@ void tc_solve_destroy(TcSolveBuffers* t) {
         cudaStreamDestroy(t->aux);
         t->aux = nullptr;
     }
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < t->n_graphs; ++i) cudaGraphExecDestroy(t->graphs[i].exec);
+    t->n_graphs = 0;
+    for (cudaStream_t* st : {&t->origin, &t->bulk, &t->aux2})
+        if (*st) {
+            cudaStreamSynchronize(*st);
+            cudaStreamDestroy(*st);
+            *st = nullptr;
+        }
+    for (int i = 0; i < kSolveEvents; ++i)
         if (t->ev[i]) {
             cudaEventDestroy(t->ev[i]);
             t->ev[i] = nullptr;
@@ -857,9 +909,16 @@ static int launch_chain(cudaStream_t st, const ChainParams& cp) {
     return cudaLaunchKernelEx(&cfg, k_chain128, cp) == cudaSuccess ? PKV_OK : PKV_ERR_CUDA;
 }
 
-int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
-                        float* dW, bool well_conditioned, bool zero_fill, DevStatus* status, const Pair* dW_pair,
-                        __nv_bfloat16* const* S_T_triple) {
+static bool solve_trace() {
+    static const bool v = getenv("PKV_SOLVE_TRACE") != nullptr;
+    return v;
+}
+
+// The whole solve, issued from lc.st.  dW is the result's address, or, with dW_ind set, only has its alignment,
+// the address being read on the device from *dW_ind (the form a captured graph replays with another destination).
+static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
+                      float* dW, float* const* dW_ind, bool well_conditioned, bool zero_fill,
+                      DevStatus* status, const Pair* dW_pair, __nv_bfloat16* const* S_T_triple) {
     const int F = n;      // dimension of the system; ld is the row stride of G, S_T, dW and of every n x n work array
     const int nblk = (F + PB - 1) / PB;
     Trip L3{{t->L3[0], t->L3[1], t->L3[2]}}, X3{{t->X3[0], t->X3[1], t->X3[2]}}, XT3{{t->XT3[0], t->XT3[1], t->XT3[2]}};
@@ -880,7 +939,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     // block (which the chain kernel does not read back from memory); U_k's first block column also leaves
     // the bf16 triple of the updated column k+1, the operand of P_{k+1} and of the next chain kernel.
     //   chain(k)  needs chain(k-1) and U_{k-2};   P_k needs chain(k) and U_{k-1};   U_k needs P_k.
-    cudaStream_t sA = t->aux, sB = lc.st;
+    cudaStream_t sA = t->aux, sB = t->bulk;      // priorities: chain > bulk (sB) > the inverse's doubling (sC)
     Lc lcB{sB, lc.launches, lc.map_cache};
     if (t->chain_n != n || t->chain_ld != ld) {
         for (int i = 0; i < 3; ++i) {
@@ -894,12 +953,61 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     for (int i = 0; i < 3; ++i) { cp.mP[i] = t->chainP[i]; cp.mX[i] = t->chainX[i]; }
     cp.G = G; cp.n = n; cp.ld = ld; cp.X3 = X3; cp.XT3 = XT3; cp.six = well_conditioned ? 0 : 1; cp.status = status;
     // phase profile of the chain kernel (environment variable PKV_SOLVE_TRACE=1): clock64 marks, printed to stderr
-    static const bool trace = getenv("PKV_SOLVE_TRACE") != nullptr;
+    const bool trace = solve_trace();
     cp.stamps = trace ? t->stamps : nullptr;
     cudaEvent_t evFork = t->ev[0], evF = t->ev[1];
     cudaEvent_t evU[2] = {t->ev[2], t->ev[3]};
-    cudaEventRecord(evFork, sB);
+    cudaEvent_t evP = t->ev[4], evC = t->ev[5];
+    // Third stream sC: X = L^{-1} by recursive doubling, [A 0; C B]^{-1} = [A^{-1} 0; -B^{-1} C A^{-1}  B^{-1}],
+    // pair by pair as soon as a pair's columns are factored, beside the factorisation (whose panel products and
+    // chain kernels leave most SMs idle); only the levels that need the last columns remain for the end.
+    cudaStream_t sC = t->aux2;
+    Lc lcC{sC, lc.launches, lc.map_cache};
+    auto pass_plan = [&](TcGemm& g, const Trip& A, long long lda, long long ar, long long ac, const Trip& B, long long ldb,
+                         long long br, long long bc) {
+        if (well_conditioned) three_pass(g, A, lda, ar, ac, B, ldb, br, bc);
+        else six_pass(g, A, lda, ar, ac, B, ldb, br, bc);
+    };
+    // pair p of level s: rows/columns [o, o + 2s) clipped to F, o = 2 s p; top-left inverse (s x s) and
+    // bottom-right inverse (bot x bot) are finished, the bottom-left block of L is the panel's
+    auto doubling_pair = [&](int s, int p) -> int {
+        const int o = 2 * s * p, bot = min(s, F - (o + s));
+        {   // TT [s][bot] = A^{-T} C^T   (A^{-T} upper triangular: contraction index >= row)
+            TcGemm g{};
+            pass_plan(g, XT3, ld, F, F, L3, ld, F, F);
+            g.a_row0 = o; g.a_col0 = o; g.a_tri = 2;
+            g.b_row0 = o + s; g.b_col0 = o;
+            g.M = s; g.N = bot; g.K = s; g.batch = 1; g.alpha = 1.f;
+            g.c_rows = s; g.c_cols = s;
+            g.out[0] = TT3.a[0]; g.out[1] = TT3.a[1]; g.out[2] = TT3.a[2]; g.ldo = s; g.nout = 3;
+            const int r = gemm_tc(lcC, g, status);
+            if (r) return r;
+        }
+        {   // X(bottom-left) [bot][s] = -B^{-1} TT^T   (B^{-1} lower triangular: contraction index <= row)
+            TcGemm g{};
+            pass_plan(g, X3, ld, F, F, TT3, s, s, s);
+            g.a_row0 = o + s; g.a_col0 = o + s; g.a_tri = 1;
+            g.M = bot; g.N = s; g.K = bot; g.batch = 1; g.alpha = -1.f;
+            g.c_row0 = o + s; g.c_col0 = o; g.c_rows = F; g.c_cols = F;
+            g.out[0] = X3.a[0]; g.out[1] = X3.a[1]; g.out[2] = X3.a[2]; g.ldo = ld; g.nout = 3;
+            const int r = gemm_tc(lcC, g, status);
+            if (r) return r;
+        }
+        dim3 grid(s / 32, s / 32, 1), block(32, 8);
+        k_transpose_blocks<<<grid, block, 0, sC>>>(X3, XT3, n, ld, s, p);
+        lc.count();
+        return PKV_OK;
+    };
+    const int nsp = well_conditioned ? 2 : 3;
+    Trip S2{{t->S2[0], t->S2[1], t->S2[2]}}, Z2{{t->Z2[0], t->Z2[1], t->Z2[2]}};
+    static cudaEvent_t tev[5];      // trace mode only: stream timeline of the call
+    if (trace && !tev[0]) for (auto& e : tev) cudaEventCreate(&e);
+    timespec ts0{};
+    if (trace) { cudaEventRecord(tev[0], lc.st); clock_gettime(CLOCK_MONOTONIC, &ts0); }
+    cudaEventRecord(evFork, lc.st);
     cudaStreamWaitEvent(sA, evFork, 0);
+    cudaStreamWaitEvent(sB, evFork, 0);
+    cudaStreamWaitEvent(sC, evFork, 0);
     if (F > PB) {
         launch_split3(lcB, G + (size_t)PB * ld, ld, F - PB, PB,
                       Trip{{P3.a[0] + (size_t)PB * PB, P3.a[1] + (size_t)PB * PB, P3.a[2] + (size_t)PB * PB}}, PB, 3);
@@ -913,12 +1021,25 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         if ((rc = launch_chain(sA, cp))) break;
         lc.count();
         cudaEventRecord(evF, sA);
+        {   // sC: transposed copy of this block's inverse, then every pair that block b completes, lowest level first
+            cudaStreamWaitEvent(sC, evF, 0);
+            if (b > 0) cudaStreamWaitEvent(sC, evP, 0);          // P_{b-1}: the last panel such a pair reads
+            dim3 grid(PB / 32, PB / 32, 1), block(32, 8);
+            k_transpose_diag<<<grid, block, 0, sC>>>(X3, XT3, n, ld, b);
+            lc.count();
+            for (long long s = PB; s < F && rc == PKV_OK; s *= 2) {
+                const int per = (int)(2 * s / PB), p = b / per;
+                if ((2LL * p + 1) * s >= F) continue;            // no bottom half: nothing to do at this level
+                if (b + 1 != min(nblk, (p + 1) * per)) continue; // the pair's last block is not b
+                rc = doubling_pair((int)s, p);
+            }
+            if (rc != PKV_OK) break;
+        }
         if (rem <= 0) break;
         cudaStreamWaitEvent(sB, evF, 0);
         {   // P_b: panel, kept as a bf16 triple in L3
             TcGemm g{};
-            if (well_conditioned) three_pass(g, P3, PB, F, PB, X3, ld, F, F);
-            else six_pass(g, P3, PB, F, PB, X3, ld, F, F);
+            pass_plan(g, P3, PB, F, PB, X3, ld, F, F);
             g.a_row0 = k1;
             g.b_row0 = k0; g.b_col0 = k0;
             g.M = rem; g.N = PB; g.K = PB; g.batch = 1; g.alpha = 1.f;
@@ -926,10 +1047,10 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
             g.out[0] = L3.a[0]; g.out[1] = L3.a[1]; g.out[2] = L3.a[2]; g.ldo = ld; g.nout = 3;
             if ((rc = gemm_tc(lcB, g, status))) break;
         }
+        cudaEventRecord(evP, sB);
         if (rem > PB) {   // U_b: G22 -= L21 L21^T on the lower triangle, the first diagonal tile left to the chain
             TcGemm g{};
-            if (well_conditioned) three_pass(g, L3, ld, F, F, L3, ld, F, F);
-            else six_pass(g, L3, ld, F, F, L3, ld, F, F);
+            pass_plan(g, L3, ld, F, F, L3, ld, F, F);
             g.a_row0 = k1; g.a_col0 = k0; g.b_row0 = k1; g.b_col0 = k0;
             g.M = rem; g.N = rem; g.K = PB; g.batch = 1; g.alpha = -1.f;
             g.C = const_cast<float*>(G); g.ldc = ld; g.accumulate = true; g.lower_only = true; g.skip_tile00 = true;
@@ -940,78 +1061,48 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         }
         cudaEventRecord(evU[b & 1], sB);
     }
-    // join: the caller's stream continues after the chain's last kernel
-    cudaEventRecord(evF, sA);
-    cudaStreamWaitEvent(sB, evF, 0);
-    if (rc != PKV_OK) return rc;
-    {   // transposed copies of the diagonal-block inverses (the chain kernel writes only X3)
-        dim3 grid(PB / 32, PB / 32, nblk), block(32, 8);
-        k_transpose_diag<<<grid, block, 0, lc.st>>>(X3, XT3, n, ld);
-        lc.count();
+    if (trace) {
+        timespec ts; clock_gettime(CLOCK_MONOTONIC, &ts);
+        fprintf(stderr, "host: factorisation loop issued in %.3f ms\n", (ts.tv_sec - ts0.tv_sec) * 1e3 + (ts.tv_nsec - ts0.tv_nsec) * 1e-6);
     }
+    // join: the caller's stream continues after the chain's last kernel and the last doubling level
+    cudaEventRecord(evF, sA);
+    cudaEventRecord(evP, sB);
+    cudaEventRecord(evC, sC);
+    if (trace) { cudaEventRecord(tev[1], sA); cudaEventRecord(tev[2], sC); }
+    for (cudaEvent_t e : {evF, evP, evC}) cudaStreamWaitEvent(lc.st, e, 0);
+    if (rc != PKV_OK) return rc;
     if (trace && nblk <= 64) {
         static long long host_stamps[64 * kChainStamps];
-        cudaStreamSynchronize(sB);
+        cudaStreamSynchronize(lc.st);
         cudaMemcpy(host_stamps, t->stamps, (size_t)nblk * kChainStamps * sizeof(long long), cudaMemcpyDeviceToHost);
         double acc[kChainStamps] = {0};
         for (int b = 1; b < nblk; ++b)
-            for (int i = 1; i < kChainStamps; ++i) acc[i] += (double)(host_stamps[b * kChainStamps + i] - host_stamps[b * kChainStamps + i - 1]);
+            for (int i = 1; i < 8; ++i) acc[i] += (double)(host_stamps[b * kChainStamps + i] - host_stamps[b * kChainStamps + i - 1]);
         fprintf(stderr, "chain kernel phases, mean cycles over blocks 1..%d: setup+wait %.0f | tma+mma1 %.0f | L->smem+mma2 %.0f | "
-                        "A write %.0f | factor %.0f | inverse %.0f | output %.0f ; start-to-start %.0f\n", nblk - 1,
+                        "A write %.0f | factor %.0f | inverse %.0f | output %.0f ; start-to-start %.0f ns\n", nblk - 1,
                 acc[1] / (nblk - 1), acc[2] / (nblk - 1), acc[3] / (nblk - 1), acc[4] / (nblk - 1), acc[5] / (nblk - 1),
                 acc[6] / (nblk - 1), acc[7] / (nblk - 1),
-                nblk > 2 ? (double)(host_stamps[(nblk - 1) * kChainStamps] - host_stamps[kChainStamps]) / (nblk - 2) : 0.0);
-        fprintf(stderr, "   start-to-start / busy cycles per block:");
+                nblk > 2 ? (double)(host_stamps[(nblk - 1) * kChainStamps + 16] - host_stamps[kChainStamps + 16]) / (nblk - 2) : 0.0);
+        fprintf(stderr, "   start-to-start / busy per block (us, global timer):");
         for (int b = 1; b < nblk; ++b)
-            fprintf(stderr, " %lld/%lld", (host_stamps[b * kChainStamps] - host_stamps[(b - 1) * kChainStamps]) / 1000,
-                    (host_stamps[b * kChainStamps + 7] - host_stamps[b * kChainStamps]) / 1000);
-        fprintf(stderr, " (thousands)\n");
+            fprintf(stderr, " %.1f/%.1f", (host_stamps[b * kChainStamps + 16] - host_stamps[(b - 1) * kChainStamps + 16]) * 1e-3,
+                    (host_stamps[b * kChainStamps + 17] - host_stamps[b * kChainStamps + 16]) * 1e-3);
+        fprintf(stderr, "\n");
         const long long* h1 = host_stamps + kChainStamps;
         fprintf(stderr, "   block 1, factor phase (cycles): forward substitution+sync %lld | warp 0 update %lld | diagonal pieces %lld | "
                         "wait for the other warps %lld ; inverse: 16x16 pieces %lld | level 16 %lld | 32 %lld | 64 %lld\n",
                 h1[8], h1[9], h1[10], h1[11], h1[12] - h1[5], h1[13] - h1[12], h1[14] - h1[13], h1[15] - h1[14]);
 
     }
-    // ---- 2. X = L^{-1} by recursive doubling ----
-    // cond(L) = sqrt(cond(G)): with a well-conditioned ridge matrix (a few tens) the rounding of these products
-    // (pairs: 2^-16) reaches dW unamplified and three passes are enough.  The same holds for the factorisation
-    // above: lambda is then of the order of the diagonal of S_H and the trailing updates do not cancel; with a small
-    // lambda0 they do, and everything takes triples in six passes with separated accumulators.
-    for (int s = PB; s < F; s *= 2) {
-        int P = 0;
-        while ((2 * P + 1) * s < F) ++P;
-        if (P == 0) break;
-        {   // TT_p = A_p^{-T} C_p^T   (A^{-1} the finished top-left inverse, C the block of L below it)
-            TcGemm g{};
-            if (well_conditioned) three_pass(g, XT3, ld, F, F, L3, ld, F, F);
-            else six_pass(g, XT3, ld, F, F, L3, ld, F, F);
-            g.a_zrow = 2 * s; g.a_zcol = 2 * s;
-            g.b_row0 = s; g.b_zrow = 2 * s; g.b_zcol = 2 * s;
-            g.M = s; g.N = s; g.K = s; g.batch = P; g.alpha = 1.f;
-            g.c_zrow = s; g.c_rows = P * s; g.c_cols = s;
-            g.out[0] = TT3.a[0]; g.out[1] = TT3.a[1]; g.out[2] = TT3.a[2]; g.ldo = s; g.nout = 3;
-            if ((rc = gemm_tc(lc, g, status))) return rc;
-        }
-        {   // X_p(bottom-left) = -B_p^{-1} TT_p^T
-            TcGemm g{};
-            if (well_conditioned) three_pass(g, X3, ld, F, F, TT3, s, (long long)P * s, s);
-            else six_pass(g, X3, ld, F, F, TT3, s, (long long)P * s, s);
-            g.a_row0 = s; g.a_col0 = s; g.a_zrow = 2 * s; g.a_zcol = 2 * s;
-            g.b_zrow = s;
-            g.M = s; g.N = s; g.K = s; g.batch = P; g.alpha = -1.f;
-            g.c_row0 = s; g.c_zrow = 2 * s; g.c_zcol = 2 * s; g.c_rows = F; g.c_cols = F;
-            g.out[0] = X3.a[0]; g.out[1] = X3.a[1]; g.out[2] = X3.a[2]; g.ldo = ld; g.nout = 3;
-            if ((rc = gemm_tc(lc, g, status))) return rc;
-        }
-        dim3 grid(s / 32, s / 32, P), block(32, 8);
-        k_transpose_blocks<<<grid, block, 0, lc.st>>>(X3, XT3, n, ld, s);
-        lc.count();
-    }
+    // (2. X = L^{-1} was built beside the factorisation, see sC above.)  cond(L) = sqrt(cond(G)): with a
+    // well-conditioned ridge matrix (a few tens) the rounding of those products (pairs: 2^-16) reaches dW
+    // unamplified and three passes are enough.  The same holds for the factorisation: lambda is then of the order
+    // of the diagonal of S_H and the trailing updates do not cancel; with a small lambda0 they do, and everything
+    // takes triples in six passes with separated accumulators.
     // ---- 3. dW = (S_T X^T) X ----
     // The rounding of these two products is amplified by cond(L): pairs (2^-16, three passes) when
     // the ridge keeps G well conditioned, triples (2^-24, six passes) otherwise.
-    const int nsp = well_conditioned ? 2 : 3;
-    Trip S2{{t->S2[0], t->S2[1], t->S2[2]}}, Z2{{t->Z2[0], t->Z2[1], t->Z2[2]}};
     if (!S_T_triple) launch_split3(lc, S_T, ld, d, F, S2, ld, nsp);      // else: S2 already holds the triple
     {
         TcGemm g{};
@@ -1023,16 +1114,104 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         g.out[0] = Z2.a[0]; g.out[1] = Z2.a[1]; g.out[2] = Z2.a[2]; g.ldo = ld; g.nout = nsp;
         if ((rc = gemm_tc(lc, g, status))) return rc;
     }
+    if (trace) cudaEventRecord(tev[3], lc.st);
     {
         TcGemm g{};
         if (nsp == 2) three_pass(g, Z2, ld, d, F, XT3, ld, F, F);
         else six_pass(g, Z2, ld, d, F, XT3, ld, F, F);
         g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 2;
         g.nacc = well_conditioned ? 1 : 2;
-        g.C = dW; g.ldc = ld; g.c_rows = d; g.c_cols = F;
+        g.C = dW; g.C_ind = dW_ind; g.ldc = ld; g.c_rows = d; g.c_cols = F;
         if (dW_pair) { g.out[0] = dW_pair->hi; g.out[1] = dW_pair->lo; g.ldo = ld; g.nout = 2; }
         if ((rc = gemm_tc(lc, g, status))) return rc;
     }
+    if (trace) {
+        cudaEventRecord(tev[4], lc.st);
+        cudaEventSynchronize(tev[4]);
+        float a, b, c2, e;
+        cudaEventElapsedTime(&a, tev[0], tev[1]);
+        cudaEventElapsedTime(&b, tev[0], tev[2]);
+        cudaEventElapsedTime(&c2, tev[0], tev[3]);
+        cudaEventElapsedTime(&e, tev[0], tev[4]);
+        fprintf(stderr, "solve timeline (ms from the start): last chain kernel %.3f | last doubling level %.3f | S_T X^T %.3f | dW %.3f\n",
+                a, b, c2, e);
+    }
+    return PKV_OK;
+}
+
+__global__ void k_solve_begin(float** slot, float* dW, DevStatus* gstatus, const DevStatus* status) {
+    if (threadIdx.x == 0) {
+        *slot = dW;
+        *gstatus = *status;
+    }
+}
+__global__ void k_solve_end(DevStatus* status, const DevStatus* gstatus) {
+    if (threadIdx.x == 0) *status = *gstatus;
+}
+
+// The solve is some hundreds of small dependent launches on four streams: issued one by one they cost the host
+// more than a millisecond and the device several microseconds of stream bookkeeping each.  The body is therefore
+// captured once per (operands, shape, precision plan) into a CUDA graph on an internal stream and replayed;
+// what changes from call to call goes through device memory: the result's address (a pointer slot the final
+// products read) and the status word (copied in before, out after).  PKV_SOLVE_GRAPH=0 in the environment, the
+// phase trace, a changed row stride or any failure to capture select the launch-by-launch path.
+int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
+                        float* dW, bool well_conditioned, bool zero_fill, DevStatus* status, const Pair* dW_pair,
+                        __nv_bfloat16* const* S_T_triple) {
+    static const bool graphs_on = [] { const char* e = getenv("PKV_SOLVE_GRAPH"); return !e || atoi(e) != 0; }();
+    if (!graphs_on || t->graph_off || solve_trace() || zero_fill)
+        return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple);
+    const bool aligned = ((uintptr_t)dW & 15) == 0;
+    SolveGraph* e = nullptr;
+    for (int i = 0; i < t->n_graphs; ++i) {
+        SolveGraph& c = t->graphs[i];
+        if (c.G == G && c.S_T == S_T && c.n == n && c.ld == ld && c.d == d && c.well == well_conditioned &&
+            c.triple == (S_T_triple != nullptr) && c.aligned == aligned && c.pair_hi == (dW_pair ? dW_pair->hi : nullptr) &&
+            c.pair_lo == (dW_pair ? dW_pair->lo : nullptr))
+            e = &c;
+    }
+    k_solve_begin<<<1, 32, 0, lc.st>>>(t->slot, dW, t->gstatus, status);
+    lc.count();
+    if (!e) {
+        const int64_t before = lc.launches ? *lc.launches : 0;
+        if (cudaStreamBeginCapture(t->origin, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
+            cudaGetLastError();
+            t->graph_off = 1;
+            return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple);
+        }
+        Lc lco{t->origin, lc.launches, lc.map_cache};
+        const int rc = solve_body(lco, t, G, S_T, n, ld, d, dW, t->slot, well_conditioned, false, t->gstatus, dW_pair,
+                                  S_T_triple);
+        cudaGraph_t gr = nullptr;
+        const cudaError_t ce = cudaStreamEndCapture(t->origin, &gr);
+        cudaGraphExec_t exec = nullptr;
+        if (rc == PKV_OK && ce == cudaSuccess && gr && cudaGraphInstantiate(&exec, gr, 0) != cudaSuccess) exec = nullptr;
+        if (gr) cudaGraphDestroy(gr);
+        if (rc != PKV_OK) { cudaGetLastError(); return rc; }
+        if (!exec) {      // capture is not available here: stay on the launch-by-launch path from now on
+            cudaGetLastError();
+            t->graph_off = 1;
+            if (lc.launches) *lc.launches = before;
+            return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple);
+        }
+        int slot = t->n_graphs;
+        if (slot == kSolveGraphs) {      // evict the least recently used
+            slot = 0;
+            for (int i = 1; i < kSolveGraphs; ++i) if (t->graphs[i].used < t->graphs[slot].used) slot = i;
+            cudaGraphExecDestroy(t->graphs[slot].exec);
+        } else {
+            ++t->n_graphs;
+        }
+        e = &t->graphs[slot];
+        *e = SolveGraph{G, S_T, n, ld, d, well_conditioned, S_T_triple != nullptr, aligned, dW_pair ? dW_pair->hi : nullptr,
+                        dW_pair ? dW_pair->lo : nullptr, exec, (lc.launches ? *lc.launches : 0) - before, 0};
+    } else {
+        lc.count((int)e->launches);
+    }
+    e->used = ++t->graph_clock;
+    if (cudaGraphLaunch(e->exec, lc.st) != cudaSuccess) return PKV_ERR_CUDA;
+    k_solve_end<<<1, 32, 0, lc.st>>>(status, t->gstatus);
+    lc.count();
     return PKV_OK;
 }
 
