@@ -169,6 +169,18 @@ typedef struct pkv_stats {
     double min_pivot;    /* smallest Cholesky pivot (squared diagonal of the factor) */
     int32_t err_info[2]; /* BAD_INDEX: (head, position); NOT_PD: (column, 0); TIMEOUT: (site, 0) */
     float stage_ms[12];  /* per-stage device time when timing is enabled with pkv_set_timing */
+    /* Conditioning of the ridge matrix G = S_H + lambda I (ridge-scale ablation: a small coefficient makes the solve
+     * ill conditioned).  lambda_max(G) lies between the weighted eigenvalue mean ||S_H||_F^2 / tr(S_H) + lambda and
+     * ||S_H||_F + lambda; lambda_min(G) between lambda and the smallest pivot.  Hence
+     *   cond_lower_bound = (fro2 / trace + lambda_eff) / min_pivot  <=  cond(G)  <=
+     *   cond_upper_bound = (sqrt(fro2) + lambda_eff) / lambda_eff.
+     * cond_warning = 1 when the lower bound exceeds 1e4: the fp32-equivalent factorisation (relative rounding
+     * 2^-24, amplified by cond(G)) may then miss the 5e-3 tolerance the build is checked to; the patch is still
+     * returned.  All three are 0 when the solve did not run. */
+    double cond_lower_bound;
+    double cond_upper_bound;
+    int32_t cond_warning;
+    int32_t reserved;
 } pkv_stats;
 
 typedef struct pkv_ctx pkv_ctx;

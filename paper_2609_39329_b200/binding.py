@@ -70,13 +70,16 @@ class pkv_ref_next(C.Structure):
 class pkv_stats(C.Structure):
     _fields_ = [("lambda_eff", C.c_double), ("trace", C.c_double), ("fro2", C.c_double),
                 ("target_fro2", C.c_double), ("resid_fro2", C.c_double), ("dW_fro2", C.c_double),
-                ("min_pivot", C.c_double), ("err_info", C.c_int32 * 2), ("stage_ms", C.c_float * 12)]
+                ("min_pivot", C.c_double), ("err_info", C.c_int32 * 2), ("stage_ms", C.c_float * 12),
+                ("cond_lower_bound", C.c_double), ("cond_upper_bound", C.c_double), ("cond_warning", C.c_int32),
+                ("reserved", C.c_int32)]
 
     def as_dict(self) -> Dict[str, object]:
         return {"lambda_eff": self.lambda_eff, "trace": self.trace, "fro2": self.fro2,
                 "target_fro2": self.target_fro2, "resid_fro2": self.resid_fro2, "dW_fro2": self.dW_fro2,
                 "min_pivot": self.min_pivot, "err_info": (self.err_info[0], self.err_info[1]),
-                "stage_ms": [float(x) for x in self.stage_ms]}
+                "stage_ms": [float(x) for x in self.stage_ms], "cond_lower_bound": self.cond_lower_bound,
+                "cond_upper_bound": self.cond_upper_bound, "cond_warning": int(self.cond_warning)}
 
 
 _lib = None

@@ -563,6 +563,16 @@ static void begin_call(pkv_ctx* c) {
     cudaMemsetAsync(c->b.status, 0, sizeof(DevStatus), c->st);
 }
 
+// bounds on cond(S_H + lambda I) from what the solve leaves in the status word (see pkv_stats)
+static void fill_cond(const DevStatus& s, pkv_stats* stats) {
+    stats->cond_lower_bound = stats->cond_upper_bound = 0.0;
+    stats->cond_warning = stats->reserved = 0;
+    if (!(s.lam > 0.f) || !(s.min_pivot > 0.f) || !(s.tr > 0.0)) return;
+    stats->cond_lower_bound = (s.fro2 / s.tr + (double)s.lam) / (double)s.min_pivot;
+    stats->cond_upper_bound = (sqrt(s.fro2) + (double)s.lam) / (double)s.lam;
+    stats->cond_warning = stats->cond_lower_bound > 1e4 ? 1 : 0;
+}
+
 // reads the status word; fills stats; returns the call's code
 static int end_call(pkv_ctx* c, pkv_stats* stats, const int32_t* head_off) {
     cudaError_t e = cudaMemcpyAsync(c->host_status, c->b.status, sizeof(DevStatus), cudaMemcpyDeviceToHost, c->st);
@@ -580,6 +590,7 @@ static int end_call(pkv_ctx* c, pkv_stats* stats, const int32_t* head_off) {
         stats->resid_fro2 = s.res_fro2;
         stats->dW_fro2 = s.dw_fro2;
         stats->min_pivot = s.min_pivot;
+        fill_cond(s, stats);
         stats->err_info[0] = stats->err_info[1] = 0;
         if (s.code == PKV_ERR_BAD_INDEX && s.bad_index && head_off) {
             int pos = (int)(s.bad_index - 1), h = 0;
@@ -922,6 +933,7 @@ static void fill_stats(pkv_ctx* c, const DevStatus& s, pkv_stats* stats, const i
     stats->resid_fro2 = s.res_fro2;
     stats->dW_fro2 = s.dw_fro2;
     stats->min_pivot = s.min_pivot;
+    fill_cond(s, stats);
     if (s.code == PKV_ERR_BAD_INDEX && s.bad_index && head_off) {
         int pos = (int)(s.bad_index - 1), h = 0;
         while (h + 1 < c->dims.Hkv && head_off[h + 1] <= pos) ++h;

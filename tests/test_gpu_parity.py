@@ -397,6 +397,15 @@ def test_ridge_solve_parity_modes_and_errors(B, F, d, n):
             np.testing.assert_allclose(st["lambda_eff"], lam, rtol=1e-4)
             np.testing.assert_allclose(st["dW_fro2"], np.sum(want * want), rtol=2e-3)
             assert st["min_pivot"] > 0
+            # the reported bounds bracket the condition number of the ridge matrix
+            ev = np.linalg.eigvalsh(S_H + lam * np.eye(F))
+            cond = ev[-1] / ev[0]
+            assert st["cond_lower_bound"] <= cond * (1 + 1e-3) and cond <= st["cond_upper_bound"] * (1 + 1e-3), (mode, lam0)
+            assert st["cond_warning"] == 0
+        # a ridge far below the spectrum of a rank-deficient S_H (n < F): flagged, the patch is still returned
+        if n < F:
+            dW, st = ctx.ridge_solve(tH, tT, 2e-3, B.LAMBDA_ABSOLUTE)
+            assert st["cond_warning"] == 1 and st["cond_lower_bound"] > 1e4 and torch.isfinite(dW).all()
         # not positive definite: a negative diagonal entry that the ridge does not lift
         bad = S_H.astype(np.float32).copy()
         bad[5, 5] = -1e6
