@@ -25,7 +25,7 @@ def test_library_builds_loads_and_exports_every_declared_symbol():
 def test_binding_structs_match_header_sizes_and_strerror():
     from paper_2609_39329_b200 import binding as B
     L = B.lib()
-    assert ctypes.sizeof(B.pkv_dims) == 44 and ctypes.sizeof(B.pkv_stats) == 7 * 8 + 8 + 48
+    assert ctypes.sizeof(B.pkv_dims) == 44 and ctypes.sizeof(B.pkv_stats) == 7 * 8 + 8 + 48 + 2 * 8 + 2 * 4
     assert L.pkv_strerror(0) == b"ok"
     assert b"ascending" in L.pkv_strerror(-3)
     # workspace sizing needs no device; bad dims give 0
