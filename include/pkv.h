@@ -40,7 +40,7 @@ typedef enum pkv_error {
     PKV_ERR_BAD_INDEX = -3,    /* kept-index set not strictly ascending within [0, L); first offender in stats */
     PKV_ERR_NOT_PD = -4,       /* Cholesky pivot <= 0 or non-finite; column in stats.err_info */
     PKV_ERR_DEGENERATE = -5,   /* tr(S_H) = 0 under the adaptive ridge scale (Eq. 7) */
-    PKV_ERR_NONFINITE = -6,    /* NaN/Inf met in the statistics */
+    PKV_ERR_NONFINITE = -6,    /* NaN/Inf met in the statistics, or a cached key outside fp16's range (hd = 128) */
     PKV_ERR_TIMEOUT = -7,      /* a bounded device-side wait (TMA / tensor-core pipeline) expired */
     PKV_ERR_CUDA = -8,         /* a CUDA runtime call failed; see pkv_last_cuda_error */
     PKV_ERR_NOMEM = -9         /* workspace allocation failed or caller-provided workspace too small */

@@ -97,25 +97,32 @@ __global__ void __launch_bounds__(256) k_attn_prep(const float* __restrict__ q, 
 
 // bf16 -> fp16, eight elements per thread.  Exact for every bf16 value of magnitude in [2^-14, 65504] (8 significant
 // bits fit in fp16's 11); smaller magnitudes round to fp16 subnormals (absolute error below 3e-8).
-__global__ void __launch_bounds__(256) k_bf16_to_f16(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n8) {
+// A bf16 value is exact in fp16 when its magnitude is inside fp16's range (keys of a cache are; below 6e-8 they
+// flush towards zero, which no logit notices).  A key beyond 65504 or not finite would turn into an infinity:
+// the call reports PKV_ERR_NONFINITE instead (such a cache needs the bf16-pair path, PKV_ATTN_Q=pair).
+__global__ void __launch_bounds__(256) k_bf16_to_f16(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n8,
+                                                     DevStatus* status) {
     const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n8) return;
     const uint4 v = src[i];
     const uint32_t in[4] = {v.x, v.y, v.z, v.w};
     uint32_t out[4];
+    bool bad = false;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         const float lo = __uint_as_float(in[e] << 16), hi = __uint_as_float(in[e] & 0xffff0000u);
+        bad = bad || !(fabsf(lo) <= 65504.f) || !(fabsf(hi) <= 65504.f);
         const __half2 h = __floats2half2_rn(lo, hi);
         out[e] = *reinterpret_cast<const uint32_t*>(&h);
     }
     dst[i] = make_uint4(out[0], out[1], out[2], out[3]);
+    if (bad) atomicCAS(&status->code, 0, PKV_ERR_NONFINITE);
 }
 
-static void to_f16(const Lc& lc, const void* src, void* dst, size_t elems) {
+static void to_f16(const Lc& lc, const void* src, void* dst, size_t elems, DevStatus* status) {
     const size_t n8 = elems / 8;
     if (!n8) return;
-    k_bf16_to_f16<<<(unsigned)((n8 + 255) / 256), 256, 0, lc.st>>>((const uint4*)src, (uint4*)dst, n8);
+    k_bf16_to_f16<<<(unsigned)((n8 + 255) / 256), 256, 0, lc.st>>>((const uint4*)src, (uint4*)dst, n8, status);
     lc.count();
 }
 
@@ -531,12 +538,12 @@ static int attention_tc2(const Lc& lc, TcBuffers* t, const pkv_dims* d, const At
     const void* Kcomp = a.Kc;
     if (f16) {
         if (d->L > 0 && a.mode != 2) {
-            to_f16(lc, a.K, t->K16, (size_t)Hkv * d->L * hd);
+            to_f16(lc, a.K, t->K16, (size_t)Hkv * d->L * hd, status);
             Kfull = t->K16;
         } else {
             Kfull = t->K16;
         }
-        if (a.total_kept > 0 && a.mode != 1) to_f16(lc, a.Kc, t->Kc16, (size_t)a.total_kept * hd);
+        if (a.total_kept > 0 && a.mode != 1) to_f16(lc, a.Kc, t->Kc16, (size_t)a.total_kept * hd, status);
         Kcomp = t->Kc16;
     }
     if (d->L > 0) {

@@ -760,6 +760,13 @@ def test_nonfinite_inputs_are_reported_and_caller_workspace_is_accepted(B):
     with pytest.raises(B.PkvError) as ei:
         gpu_build(B, cfg, lay, x, x, [0, cfg.N], 0.1, B.ENGINE_AUTO)
     assert ei.value.code == -6
+    # a cached key beyond fp16's range cannot go through the fp16 key copies of the hd-128 attention: reported
+    lay2 = dict(lay)
+    lay2["K"] = lay["K"].copy()
+    lay2["K"][0, 7, 3] = 1.0e5
+    with pytest.raises(B.PkvError) as ei:
+        gpu_build(B, cfg, lay2, lay["x0"], lay["x0"], [0, cfg.N], 0.1, B.ENGINE_AUTO)
+    assert ei.value.code == -6
     # caller-provided workspace: same result as the context-owned one; an undersized one is refused
     dims = B.dims_from_config(cfg, b_max=max(len(k) for k in lay["kept"]))
     probe = B.PkvContext(dims, engine=B.ENGINE_AUTO)
