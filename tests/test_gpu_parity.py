@@ -578,10 +578,11 @@ def test_reduced_config2_shape(B):
         check_build(B, cfg, lay, lay["x0"], lay["x0"], [0, cfg.N], 0.1, engine)
 
 
-@pytest.mark.parametrize("nl,solver,hd", [(2, 0, 64), (5, 0, 128), (4, 1, 128)])
+@pytest.mark.parametrize("nl,solver,hd", [(2, 0, 64), (5, 0, 128), (4, 1, 128), (8, 0, 128)])
 def test_stack_matches_oracle_chain(B, nl, solver, hd):
     """Free-running stack: GPU and oracle each propagate their own states through all blocks (the tensor-core
-    engine runs the teacher ahead on its own stream; five blocks exercise the reuse of its two-slot ring)."""
+    engine runs the teacher ahead on its own stream; five blocks reuse its three-slot ring of teacher outputs, eight
+    blocks go round it twice and once round the five-slot ring of the teacher's next states)."""
     import torch
     cfg = small_cfg("bf16", n_layers=nl, N=64, hd=hd, Hq=4 if hd == 128 else 8, Hkv=2)
     lays = [H.make_problem(cfg, layer=l) for l in range(nl)]
