@@ -90,8 +90,9 @@ __device__ __forceinline__ void gemm_stamp(const GemmTcParams& p, int i) {
 
 // One k-tile stage holds every distinct operand tile once: nA x [128][64] and nB x [BN][64] bf16,
 // and all passes are issued from it (the shared operand of a split product is not re-read).
-// PRE: the epilogue warps fetch the fp32 C tile they will add to (read-modify-write products of the
-// factorisation) while the main loop runs, instead of after it.
+// (A variant whose epilogue warps prefetched the fp32 C tile of a read-modify-write product during the main loop
+// needed 240 registers per thread, one CTA per SM; without it two or three CTAs share an SM and hide the
+// read's latency better: the solve went from 2.51 to 2.45 ms at F = 4096 and from 3.66 to 3.55 ms at F = 5120.)
 //
 // Accumulators.  The tensor core adds each MMA's result to the fp32 accumulator with truncation, not
 // round-to-nearest: a sum of same-signed terms (the diagonal of a Gram or of L L^T) comes out low by about
@@ -100,7 +101,7 @@ __device__ __forceinline__ void gemm_stamp(const GemmTcParams& p, int i) {
 // round-robin to accumulators 1..nacc-1, each of which so sees only a few adds at a fraction of the full
 // magnitude, every other pass to accumulator 0 where its truncation is relative to the small cross terms;
 // the epilogue adds the accumulators in registers with round-to-nearest.
-template <int BN, bool PRE>
+template <int BN>
 __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcParams p) {
     const int m0 = blockIdx.y * 128, n0 = blockIdx.x * BN, z = blockIdx.z;
     if (p.lower_only && n0 > m0 + 127) return;
@@ -217,16 +218,6 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         const int nrows = max(0, min(32, min(p.M - rl0, p.c_rows - rowa0)));
         const bool vec_ok = p.vec_ok != 0;
         float* const Cp = p.C_ind ? *p.C_ind : p.C;
-        // PRE: whole-tile prefetch of C, legal when the tile is full width and vector-aligned
-        constexpr int kPre = PRE ? BN / 4 : 1;
-        float4 cpre[kPre];
-        const bool pre_ok = PRE && Cp && p.accumulate && vec_ok && lane < nrows &&
-                            min(p.N - n0, p.c_cols - ccol0) >= BN;
-        if (PRE && pre_ok) {
-            const float* crow = Cp + (size_t)(rowa0 + lane) * p.ldc + ccol0;
-#pragma unroll
-            for (int j = 0; j < kPre; ++j) cpre[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
-        }
         bool ok = true;
         if (ktiles > 0) {
             ok = mbar_wait(bars + 8 * (2 * STAGES), 0, abort_flag, p.status, 3);
@@ -277,13 +268,8 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                         }
                         if (p.accumulate) {
                             float4 c4[8];
-                            if (PRE && pre_ok) {
 #pragma unroll
-                                for (int j = 0; j < 8; ++j) c4[j] = cpre[PRE ? (c0 >> 2) + j : 0];
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) c4[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
-                            }
+                            for (int j = 0; j < 8; ++j) c4[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
                                 v[4 * j] += c4[j].x; v[4 * j + 1] += c4[j].y; v[4 * j + 2] += c4[j].z; v[4 * j + 3] += c4[j].w;
@@ -736,13 +722,13 @@ static int cached_map(MapCache* cache, CUtensorMap* out, const void* ptr, uint64
     return PKV_OK;
 }
 
-template <int BN, bool PRE>
+template <int BN>
 static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     static PerDeviceOnce once;
     constexpr int kMaxSmem = 227 * 1024;
     int dev;
     if (once.needed(&dev)) {
-        if (cudaFuncSetAttribute(k_gemm_tc<BN, PRE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+        if (cudaFuncSetAttribute(k_gemm_tc<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
             return PKV_ERR_CUDA;
         once.mark(dev);
     }
@@ -776,9 +762,9 @@ static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
         at[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = at;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, k_gemm_tc<BN, PRE>, p) != cudaSuccess) return PKV_ERR_CUDA;
+        if (cudaLaunchKernelEx(&cfg, k_gemm_tc<BN>, p) != cudaSuccess) return PKV_ERR_CUDA;
     } else {
-        k_gemm_tc<BN, PRE><<<grid, 192, smem, lc.st>>>(p);
+        k_gemm_tc<BN><<<grid, 192, smem, lc.st>>>(p);
     }
     lc.count();
     return PKV_OK;
@@ -843,7 +829,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     if (g.K < 0 || g.npass <= 0 || g.npass > kGemmMaxPass || (!g.C && g.nout == 0)) return PKV_ERR_INVALID_ARG;
     GemmTcParams p;
     // 128 x 256 tiles move a third fewer operand bytes per flop than 128 x 128; taken when they still give
-    // at least two waves of CTAs (and the C tile is not prefetched: that variant is 128 wide)
+    // at least two waves of CTAs
     const long long tiles256 = (long long)((g.N + 255) / 256) * ((g.M + 127) / 128) * g.batch;
     const bool wide = g.N >= 512 && tiles256 >= 2 * 148 && !(g.C && g.accumulate) && !g.lower_only &&
                       g.nacc < 4;
@@ -911,10 +897,9 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
         if (BN == 256) return launch_gemm_p<256>(lc, p, g.batch);
         return launch_gemm_p<128>(lc, p, g.batch);
     }
-    const bool pre = g.C && g.accumulate && p.vec_ok;
-    if (BN == 64) return launch_gemm<64, false>(lc, p, g.batch);
-    if (BN == 256) return launch_gemm<256, false>(lc, p, g.batch);
-    return pre ? launch_gemm<128, true>(lc, p, g.batch) : launch_gemm<128, false>(lc, p, g.batch);
+    if (BN == 64) return launch_gemm<64>(lc, p, g.batch);
+    if (BN == 256) return launch_gemm<256>(lc, p, g.batch);
+    return launch_gemm<128>(lc, p, g.batch);
 }
 
 }  // namespace pkv
