@@ -41,7 +41,7 @@ struct TcGemm {
     int a_tri;      // the same for the A operand (1: A[m][k] = 0 for k > m; 2: A[m][k] = 0 for k < m)
     bool skip_tile00;     // leave the first tile (rows and columns [0,128) of the product) alone
     bool out_col0_only;   // write the bf16 parts only for the first 128-column block of the product
-    unsigned long long* stamps;   // optional device array of 8 global-timer marks (phases of the first CTA)
+    unsigned long long* stamps;   // optional device array of 16 global-timer marks (phases of the first CTA, epilogue chunks)
     int nacc;       // 0/1: one fp32 accumulator; 2 or 4: the hi x hi pass of a split product is accumulated apart
                     // from the cross passes (and in several parts), which removes most of the tensor core's
                     // truncation bias from sums of same-signed terms; pass 0 must be the hi x hi pass

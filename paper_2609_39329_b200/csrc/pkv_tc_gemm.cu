@@ -226,12 +226,14 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         if (warp == 2 && lane == 0) gemm_stamp(p, 5);
         if (ok) {
             float* stg = staging + q * (32 * 33);
-#pragma unroll
+            // not unrolled: a CTA runs each chunk's code once, and a short-K tile's time is mostly instruction fetch
+#pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 if (ktiles > 0) {
                     tmem_ld32(tbase + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
                     tmem_ld_wait();
+                    if (warp == 2 && lane == 0 && c0 < 128) gemm_stamp(p, 8 + (c0 >> 5) * 2);
                     // further accumulators: added in registers with round to nearest (the launcher only asks for
                     // them when every one of them receives at least one MMA)
                     for (int a = 1; a < nacc; ++a) {
@@ -245,6 +247,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
 #pragma unroll
                     for (int j = 0; j < 32; ++j) r[j] = 0u;
                 }
+                if (warp == 2 && lane == 0 && c0 < 128) gemm_stamp(p, 9 + (c0 >> 5) * 2);
                 const int col = ccol0 + c0;                    // absolute output column of r[0]
                 const int ncol = min(min(32, p.N - (n0 + c0)), p.c_cols - col);
                 if (ncol <= 0) break;

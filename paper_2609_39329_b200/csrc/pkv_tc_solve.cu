@@ -779,23 +779,25 @@ int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const flo
     static const bool gtrace = getenv("PKV_GEMM_TRACE") != nullptr;
     static unsigned long long* dstamps = nullptr;
     if (gtrace) {
-        if (!dstamps) cudaMalloc(&dstamps, 3 * 8 * sizeof(unsigned long long));
-        cudaMemsetAsync(dstamps, 0, 3 * 8 * sizeof(unsigned long long), lc.st);
-        for (int rep = 0; rep < 2; ++rep) { g.stamps = dstamps + 8 * rep; gemm_tc(lc, g, status); }
-        g.stamps = dstamps + 16;
+        if (!dstamps) cudaMalloc(&dstamps, 3 * 16 * sizeof(unsigned long long));
+        cudaMemsetAsync(dstamps, 0, 3 * 16 * sizeof(unsigned long long), lc.st);
+        for (int rep = 0; rep < 2; ++rep) { g.stamps = dstamps + 16 * rep; gemm_tc(lc, g, status); }
+        g.stamps = dstamps + 32;
     }
     const int rc = gemm_tc(lc, g, status);
     if (gtrace) {
-        unsigned long long h[24];
+        unsigned long long h[48];
         cudaStreamSynchronize(lc.st);
         cudaMemcpy(h, dstamps, sizeof(h), cudaMemcpyDeviceToHost);
         for (int rep = 0; rep < 3; ++rep) {
-            const unsigned long long* s = h + 8 * rep;
+            const unsigned long long* s = h + 16 * rep;
             fprintf(stderr, "gemm %dx%dx%d passes %d acc %d, launch %d: entry +0 | dependencies met %.2f | status read %.2f | first k-tile "
                             "landed %.2f | last MMA issued %.2f | accumulator ready %.2f | epilogue done %.2f | exit %.2f us",
                     M, N, K, passes, nacc, rep, (s[1] - s[0]) * 1e-3, (s[2] - s[0]) * 1e-3, (s[3] - s[0]) * 1e-3, (s[4] - s[0]) * 1e-3,
                     (s[5] - s[0]) * 1e-3, (s[6] - s[0]) * 1e-3, (s[7] - s[0]) * 1e-3);
-            if (rep > 0) fprintf(stderr, " ; entry %.2f us after the previous launch's exit", ((double)s[0] - (double)h[8 * (rep - 1) + 7]) * 1e-3);
+            if (rep > 0) fprintf(stderr, " ; entry %.2f us after the previous launch's exit", ((double)s[0] - (double)h[16 * (rep - 1) + 7]) * 1e-3);
+            fprintf(stderr, " ; chunks (loaded/summed):");
+            for (int c = 0; c < 8; ++c) fprintf(stderr, " %.2f", (s[8 + c] - s[0]) * 1e-3);
             fprintf(stderr, "\n");
         }
     }
