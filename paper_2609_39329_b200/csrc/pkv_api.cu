@@ -642,6 +642,7 @@ static AttnArgs attn_args(pkv_ctx* c, const float* q, int64_t ldq, const float* 
     a.nsplitF = (c->dims.L + N + c->kv_split - 1) / c->kv_split;
     a.nsplitC = (max_b + N + c->kv_split - 1) / c->kv_split;
     if (a.nsplitC < 1) a.nsplitC = 1;
+    a.zoffC = a.nsplitF;
     a.part_m = c->b.part_m; a.part_l = c->b.part_l; a.part_O = c->b.part_O;
     return a;
 }

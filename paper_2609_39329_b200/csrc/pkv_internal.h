@@ -85,6 +85,7 @@ struct AttnArgs {
     const int32_t* tok_cs;                // device [N] chunk start of each token
     int N, Hq, Hkv, hd, L, elem_bytes;
     int kv_split, nsplitF, nsplitC;
+    int zoffC;                            // slot of the student's first split in the partial buffers (teacher: 0)
     int total_kept, max_b;                // rows of the compact cache (all heads), largest head
     int mode;                             // 0: both streams; 1: teacher only (aF); 2: student only (aC, dA from a given aF)
     float* part_m; float* part_l; float* part_O;   // [nsplit][Hkv][N*g] and [..][hd]

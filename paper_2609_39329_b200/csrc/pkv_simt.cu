@@ -505,7 +505,7 @@ __global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
         for (int c = 0; c < per; ++c) res[0][c] = a.aF[o + c];
     }
     for (int s = (a.mode == 2 ? 1 : 0); s < (a.mode == 1 ? 1 : 2); ++s) {
-        int z0 = s ? a.nsplitF : 0;
+        int z0 = s ? a.zoffC : 0;
         int ns = s ? a.nsplitC : a.nsplitF;
         float M = -INFINITY;
         for (int i = 0; i < ns; ++i) M = fmaxf(M, a.part_m[((size_t)(z0 + i) * a.Hkv + kh) * rows + r]);

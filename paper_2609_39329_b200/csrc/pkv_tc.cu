@@ -233,10 +233,8 @@ size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d, int dua
         t->K16 = c.take<__nv_bfloat16>((size_t)d->Hkv * d->L * d->hd + 8);
         t->Kc16 = c.take<__nv_bfloat16>((size_t)d->Hkv * d->b_max * d->hd + 128 * d->hd);
     }
-    int tps, nF, nC;
-    tc_attn_plan(d, d->N_max, d->b_max, &tps, &nF, &nC);
     const size_t rows = N * (d->Hq / d->Hkv);
-    const size_t nsp = (size_t)nF + nC;
+    const size_t nsp = (size_t)tc_attn_partial_slots(d);
     t->part_m = c.take<float>(nsp * d->Hkv * rows);
     t->part_l = c.take<float>(nsp * d->Hkv * rows);
     t->part_O = c.take<float>(nsp * d->Hkv * rows * d->hd);

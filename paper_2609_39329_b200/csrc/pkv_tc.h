@@ -173,7 +173,8 @@ size_t tc_lowrank_scratch_bytes(int d, int F, int r);
 int tc_lowrank(const Lc& lc, TcBuffers* t, const pkv_dims* D, const float* dW, const float* S_H, int r, int iters,
                void* scratch, float* U, float* Br, float* dWr, float* evals_out, DevStatus* status);
 
-void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, int* nsplitC);
+void tc_attn_plan(const pkv_dims* d, int N, int max_b, int mode, int* tps, int* nsplitF, int* nsplitC, int* zoffC);
+int tc_attn_partial_slots(const pkv_dims* d);
 // q/k_new/v_new of `a` are fp32; rope_tab != nullptr rotates q and k on the way in.
 int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, const float* rope_tab,
                  DevStatus* status);

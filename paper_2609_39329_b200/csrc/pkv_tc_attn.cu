@@ -16,10 +16,14 @@
 // Partial (m, l, O) per split go to global memory; the combine kernel merges the splits of both
 // streams and forms dA = aF - aC in fp32.
 #include <cuda.h>
+#include <stdio.h>
 #include <stdlib.h>
 #include <math.h>
 
 #include "pkv_ptx.cuh"
+#include <mutex>
+#include <vector>
+
 #include "pkv_tc.h"
 #include "pkv_tc_attn2_params.h"
 
@@ -139,7 +143,7 @@ struct alignas(64) AttnTcParams {
     const float* bias;
     int N, g, Hkv, L, rows;
     int tps, nsplitF, nsplitC;
-    int z0;
+    int z0, zoffC;
     float* part_m;
     float* part_l;
     float* part_O;
@@ -454,7 +458,7 @@ __global__ void __launch_bounds__(192, 1) k_attn_tc(const __grid_constant__ Attn
         }
         if (ok && ntiles > 0) accumulate_o(ntiles - 1);
         if (valid && ok) {
-            const size_t pr = ((size_t)z * p.Hkv + kh) * p.rows + r;
+            const size_t pr = ((size_t)(stream ? p.zoffC + split : split) * p.Hkv + kh) * p.rows + r;
             p.part_m[pr] = (m == -INFINITY) ? -INFINITY : m * 0.6931471805599453f;   // back to natural-log units
             p.part_l[pr] = l;
             float4* po = reinterpret_cast<float4*>(p.part_O + pr * HD);
@@ -476,27 +480,128 @@ __global__ void __launch_bounds__(192, 1) k_attn_tc(const __grid_constant__ Attn
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
-// CTAs of the teacher stream ~ kAttnWaves x 148 SMs: enough for balance, few enough that the split
-// partials (m, l, O per row and split) stay small next to the K/V traffic.
-constexpr long long kAttnWaves = 3;
+// Split planning.  Every CTA takes one (query tile pair, KV head, split) and `tps` key tiles; CTAs are handed to
+// the SMs in grid order (all units of the teacher's first split, then its second, ..., then the student's).
+// With one CTA per SM (hd = 128: the kernel owns all of tensor memory) the time is that of the last SM to
+// finish, and a split count that leaves a nearly empty last round (3.03 rounds of 148) wastes a quarter of the
+// machine: the planner therefore replays that hand-out for every candidate split count, each CTA costing its key
+// tiles plus a fixed part (prologue, partial results written and merged later), and keeps the cheapest.  The
+// choice depends on the context's dimensions only (N_max, b_max), so that buffers sized once fit every call.
+constexpr long long kAttnWaves = 3;         // hd = 64: CTAs of the teacher stream ~ kAttnWaves x the SM count
+constexpr int kAttnCtaOverheadTiles = 4;    // fixed cost of a CTA in units of one key tile's work
+constexpr int kAttnTeacherReserve = 12;     // SMs the stack driver's teacher stream leaves free by default
 
-void tc_attn_plan(const pkv_dims* d, int N, int max_b, int* tps, int* nsplitF, int* nsplitC) {
+static long long attn_makespan(int slots, long long base, long long tF, long long tC, long long t) {
+    // min-heap of the slots' free times; CTAs in grid order
+    std::vector<long long> heap((size_t)slots, 0);
+    auto push_cta = [&](long long cost) {
+        // replace the smallest element (heap[0]) by heap[0] + cost and restore the heap
+        long long v = heap[0] + cost;
+        size_t i = 0, n = heap.size();
+        for (;;) {
+            size_t l = 2 * i + 1, r = l + 1, m = i;
+            long long mv = v;
+            if (l < n && heap[l] < mv) { m = l; mv = heap[l]; }
+            if (r < n && heap[r] < mv) { m = r; mv = heap[r]; }
+            if (m == i) break;
+            heap[i] = heap[m];
+            i = m;
+        }
+        heap[i] = v;
+    };
+    for (long long done = 0; done < tF; done += t)
+        for (long long u = 0; u < base; ++u) push_cta(kAttnCtaOverheadTiles + (tF - done < t ? tF - done : t));
+    for (long long done = 0; done < tC; done += t)
+        for (long long u = 0; u < base; ++u) push_cta(kAttnCtaOverheadTiles + (tC - done < t ? tC - done : t));
+    long long worst = 0;
+    for (long long v : heap) worst = v > worst ? v : worst;
+    return worst;
+}
+
+// tps for one launch mode (0: both streams, 1: teacher only, 2: student only); remembered per (dimensions, mode)
+static long long attn_tps(const pkv_dims* d, int mode) {
     const int g = d->Hq / d->Hkv;
     const int rows_per_cta = (d->hd == 128) ? 256 : 128;     // the hd = 128 kernel owns two query tiles
     const long long qtiles = ((long long)d->N_max * g + rows_per_cta - 1) / rows_per_cta;
     const long long base = qtiles * d->Hkv;
     const long long tilesF = (d->L + 127) / 128 + (d->N_max + 127) / 128;
-    long long want = (kAttnWaves * 148 + base - 1) / base;
-    if (want < 1) want = 1;
-    if (want > 64) want = 64;
-    long long t = (tilesF + want - 1) / want;
-    if (t < 4) t = 4;
-    *tps = (int)t;
+    if (d->hd != 128) {
+        long long want = (kAttnWaves * 148 + base - 1) / base;
+        if (want < 1) want = 1;
+        if (want > 64) want = 64;
+        const long long t = (tilesF + want - 1) / want;
+        return t < 4 ? 4 : t;
+    }
+    struct Seen { pkv_dims d; long long t; };
+    static std::mutex mu;
+    static Seen seen[3] = {};
+    std::lock_guard<std::mutex> lock(mu);
+    Seen& e = seen[mode];
+    if (e.t > 0 && e.d.L == d->L && e.d.N_max == d->N_max && e.d.b_max == d->b_max && e.d.Hq == d->Hq && e.d.Hkv == d->Hkv &&
+        e.d.hd == d->hd)
+        return e.t;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        sms <= 0) {
+        cudaGetLastError();
+        sms = 148;
+    }
+    // the teacher alone runs on its stream's SM partition (all SMs but the default reserve of the stack driver)
+    const int slots = (mode == 1 && sms > kAttnTeacherReserve) ? sms - kAttnTeacherReserve : sms;
+    const long long tF = (mode == 2) ? 0 : tilesF;
+    const long long tC = (mode == 1) ? 0 : (d->b_max + 127) / 128 + (d->N_max + 127) / 128;
+    const long long longest = tF > tC ? tF : tC;
+    long long best = -1, best_t = longest;
+    for (long long sp = 1; sp <= 64; ++sp) {
+        long long cand = (longest + sp - 1) / sp;
+        if (cand < 4) cand = 4;
+        if (base * ((tF + cand - 1) / cand + (tC + cand - 1) / cand) > 262144) break;   // keep the replay cheap
+        const long long cost = attn_makespan(slots, base, tF, tC, cand);
+        if (best < 0 || cost < best) { best = cost; best_t = cand; }
+        if (cand == 4) break;
+    }
+    e.d = *d;
+    e.t = best_t;
+    if (getenv("PKV_ATTN_TRACE"))
+        fprintf(stderr, "attention plan, mode %d on %d SMs: %lld units, %lld + %lld key tiles -> %lld tiles per split, modelled time %lld tile units\n",
+                mode, slots, base, tF, tC, best_t, best);
+    return best_t;
+}
+
+static void attn_counts(const pkv_dims* d, int N, int max_b, long long t, int* nF, int* nC) {
     const long long tF = (d->L + 127) / 128 + (N + 127) / 128;
     const long long tC = (max_b + 127) / 128 + (N + 127) / 128;
-    *nsplitF = (int)((tF + t - 1) / t);
-    *nsplitC = (int)((tC + t - 1) / t);
-    if (*nsplitC < 1) *nsplitC = 1;
+    *nF = (int)((tF + t - 1) / t);
+    *nC = (int)((tC + t - 1) / t);
+    if (*nC < 1) *nC = 1;
+}
+
+// Partials of the teacher's splits sit at [0, nsplitF), those of the student's at [zoffC, zoffC + nsplitC): zoffC is
+// the largest teacher split count of any mode at the context's N_max, so that a teacher-only launch of one block
+// and a student-only launch of another (stack driver) never share a slot.
+void tc_attn_plan(const pkv_dims* d, int N, int max_b, int mode, int* tps, int* nsplitF, int* nsplitC, int* zoffC) {
+    const long long t = attn_tps(d, mode);
+    *tps = (int)t;
+    attn_counts(d, N, max_b, t, nsplitF, nsplitC);
+    int z = 0;
+    for (int m = 0; m < 2; ++m) {
+        int nF, nC;
+        attn_counts(d, d->N_max, d->b_max, attn_tps(d, m), &nF, &nC);
+        if (nF > z) z = nF;
+    }
+    *zoffC = z;
+}
+
+// Split slots the partial buffers must hold.
+int tc_attn_partial_slots(const pkv_dims* d) {
+    int z = 0, c = 0;
+    for (int m = 0; m < 3; ++m) {
+        int nF, nC;
+        attn_counts(d, d->N_max, d->b_max, attn_tps(d, m), &nF, &nC);
+        if (m != 2 && nF > z) z = nF;
+        if (m != 1 && nC > c) c = nC;
+    }
+    return z + c;
 }
 
 template <int HD>
@@ -562,7 +667,7 @@ static int attention_tc2(const Lc& lc, TcBuffers* t, const pkv_dims* d, const At
     }
     p.head_off = a.head_off; p.tok_cs = a.tok_cs; p.bias = a.bias;
     p.N = N; p.g = g; p.Hkv = Hkv; p.L = d->L; p.rows = rows;
-    tc_attn_plan(d, N, a.max_b, &p.tps, &p.nsplitF, &p.nsplitC);
+    tc_attn_plan(d, N, a.max_b, a.mode, &p.tps, &p.nsplitF, &p.nsplitC, &p.zoffC);
     p.part_m = t->part_m; p.part_l = t->part_l; p.part_O = t->part_O;
     p.status = status;
     p.z0 = (a.mode == 2) ? p.nsplitF : 0;
@@ -571,7 +676,7 @@ static int attention_tc2(const Lc& lc, TcBuffers* t, const pkv_dims* d, const At
                       a.mode == 0 ? p.nsplitF + p.nsplitC : (a.mode == 1 ? p.nsplitF : p.nsplitC));
     if (rc != PKV_OK) return rc;
     AttnArgs c = a;
-    c.nsplitF = p.nsplitF; c.nsplitC = p.nsplitC;
+    c.nsplitF = p.nsplitF; c.nsplitC = p.nsplitC; c.zoffC = p.zoffC;
     c.part_m = t->part_m; c.part_l = t->part_l; c.part_O = t->part_O;
     attention_combine(lc, c);
     return PKV_OK;
@@ -614,7 +719,7 @@ int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
     }
     p.head_off = a.head_off; p.tok_cs = a.tok_cs; p.bias = a.bias;
     p.N = N; p.g = g; p.Hkv = Hkv; p.L = d->L; p.rows = rows;
-    tc_attn_plan(d, N, a.max_b, &p.tps, &p.nsplitF, &p.nsplitC);
+    tc_attn_plan(d, N, a.max_b, a.mode, &p.tps, &p.nsplitF, &p.nsplitC, &p.zoffC);
     p.part_m = t->part_m; p.part_l = t->part_l; p.part_O = t->part_O;
     p.status = status;
     const int qtiles = (rows + 127) / 128;
@@ -623,7 +728,7 @@ int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
     rc = launch_attn<64>(lc, p, qtiles, zcount);      // hd = 128 left above for the two-tile kernel
     if (rc != PKV_OK) return rc;
     AttnArgs c = a;
-    c.nsplitF = p.nsplitF; c.nsplitC = p.nsplitC;
+    c.nsplitF = p.nsplitF; c.nsplitC = p.nsplitC; c.zoffC = p.zoffC;
     c.part_m = t->part_m; c.part_l = t->part_l; c.part_O = t->part_O;
     attention_combine(lc, c);
     return PKV_OK;

@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
         if (ok && ntiles > 0) ok = mbar_wait(bar(B_ODONE + gq), (ntiles - 1) & 1, abort_flag, p.status, 33);
         if (ok) {
             tc_fence_after();
-            const size_t pr = ((size_t)z * p.Hkv + kh) * p.rows + r;
+            const size_t pr = ((size_t)(stream ? p.zoffC + split : split) * p.Hkv + kh) * p.rows + r;
             if (valid) {
                 p.part_m[pr] = (m_ref == -INFINITY) ? -INFINITY : m_ref * 0.6931471805599453f;   // natural-log units
                 p.part_l[pr] = l;

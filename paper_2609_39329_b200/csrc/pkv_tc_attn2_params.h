@@ -20,6 +20,7 @@ struct alignas(64) Attn2Params {
     int q_f16;                // queries are one fp16 part and every key operand is fp16 (one QK^T pass) instead of
                               // a bf16 hi + lo query pair against bf16 keys (two passes)
     int z0;                   // first split index of this launch (teacher splits come first, then the student's)
+    int zoffC;                // slot of the student's first split in the partial buffers
     float* part_m;
     float* part_l;
     float* part_O;

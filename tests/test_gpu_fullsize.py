@@ -241,8 +241,10 @@ def test_three_block_stack_at_config3_shape_free_running_and_reanchored(B):
             e_anch = H.rel_fro(res["dW"][l].cpu().numpy(), oa["dW"])
             msg += ", re-anchored %.3e" % e_anch
             assert e_anch <= DW_TOL, msg
-            # resuming reproduces the uninterrupted run
-            assert H.rel_fro(res["dW"][l].cpu().numpy(), out["dW"][l].cpu().numpy()) <= 1e-4
+            # resuming reproduces the uninterrupted run up to the rounding of the attention's split merge: the states
+            # entering block l come from a stack call whose launches (one block: both streams in one launch; more:
+            # teacher and student apart) cut the cache into different numbers of splits
+            assert H.rel_fro(res["dW"][l].cpu().numpy(), out["dW"][l].cpu().numpy()) <= 2e-3
         print(msg)
         xF, xC = o["xF_next"], o["xC_next"]
     eF = H.rel_fro(out["xF_final"].cpu().numpy(), xF)
