@@ -986,7 +986,6 @@ static int build_stack_overlapped(pkv_ctx* c, int n_layers, int first, const pkv
     }
     cudaStream_t S = c->st, T = c->tstream;
     Lc lcS{S, &c->launches, c->map_cache}, lcT{T, &c->launches, c->map_cache};
-    lcT.sms = c->teacher_sms;
     // set-up on the student stream: status words, kept-set offsets, chunk starts, RoPE table, dx0 = xF0 - xC0
     cudaMemsetAsync(b.lstatus, 0, (size_t)n_layers * sizeof(DevStatus), S);
     cudaMemcpyAsync(b.lhead_off + (size_t)first * (Hkv + 1), c->host_lhead + (size_t)first * (Hkv + 1),

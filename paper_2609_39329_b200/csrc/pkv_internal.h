@@ -44,7 +44,6 @@ struct Lc {
     int64_t* launches;
     void* map_cache = nullptr;            // tensor-map cache of the tensor-core engine (optional)
     bool pdl = false;                     // launch with programmatic stream serialisation (dependent launch)
-    int sms = 0;                          // SMs this stream's kernels may occupy (0 = all): persistent grids are sized to it
     void count(int n = 1) const { if (launches) *launches += n; }
 };
 

@@ -46,7 +46,6 @@ struct alignas(64) GemmTcParams {
     int nacc;                 // TMEM accumulators per tile (1, 2 or 4), see TcGemm::nacc
     int skip_tile00;          // the tile at (blockIdx.x, blockIdx.y) = (0, 0) is left alone
     int out_col0_only;        // bf16 parts are written by the tiles of the first block column only
-    int tiles_m, tiles_n, batch, nbuf;   // persistent kernel: tile grid and accumulator buffers in tensor memory
     int out_vec;              // the bf16 parts can be stored 16 bytes at a time (alignment of pointers, stride, offsets)
     DevStatus* status;
     unsigned long long* stamps;   // optional: global-timer marks of the first CTA's phases (profiling aid)
@@ -103,7 +102,11 @@ __device__ __forceinline__ void gemm_stamp(const GemmTcParams& p, int i) {
 // the epilogue adds the accumulators in registers with round-to-nearest.
 template <int BN>
 __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcParams p) {
-    const int m0 = blockIdx.y * 128, n0 = blockIdx.x * BN, z = blockIdx.z;
+    // Tiles are handed out in grid order; where a triangular operand makes the contraction grow with the tile's
+    // column (k_tri 1) or row (a_tri 1), the order is reversed so that the long tiles start first
+    const int bx = (p.k_tri == 1) ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
+    const int by = (p.a_tri == 1) ? (int)(gridDim.y - 1 - blockIdx.y) : (int)blockIdx.y;
+    const int m0 = by * 128, n0 = bx * BN, z = blockIdx.z;
     if (p.lower_only && n0 > m0 + 127) return;
     if (p.skip_tile00 && blockIdx.x == 0 && blockIdx.y == 0) return;
     pdl_launch_dependents();
@@ -334,277 +337,6 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     if (threadIdx.x == 0) gemm_stamp(p, 7);
 }
 
-// ---------------------------------------------------------------------------------------------
-// Persistent variant: one CTA per SM walks over the output tiles (grouped order: eight row blocks share
-// their column blocks, so that tiles in flight at the same time reuse operands out of L2).  The TMA
-// producer runs ahead into the next tile's operands, and with two accumulator buffers in tensor memory
-// (when nbuf * nacc * BN <= 512 columns) the epilogue of one tile overlaps the MMAs of the next.  Barrier
-// phases are carried in running counters across tiles.  Same arithmetic, operands and epilogue as
-// k_gemm_tc.
-// ---------------------------------------------------------------------------------------------
-constexpr int kGemmPStaging = 4 * 32 * 33 * 4;      // per-warp transposition tiles of the bf16 outputs
-
-template <int BN>
-__global__ void __launch_bounds__(192) k_gemm_tcp(const __grid_constant__ GemmTcParams p) {
-    pdl_launch_dependents();
-    constexpr int kA = 128 * 64 * 2, kB = BN * 64 * 2;
-    const int stage_bytes = p.nA * kA + p.nB * kB;
-    const int STAGES = p.stages;
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
-    uint8_t* sm = smem_raw + (base - raw);
-    // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
-    const uint32_t bars = base + STAGES * stage_bytes;
-    const uint32_t bar_accf = bars + 8 * (2 * STAGES), bar_acce = bar_accf + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * stage_bytes + (2 * STAGES + 4) * 8);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    volatile int* skip_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
-    float* staging = reinterpret_cast<float*>(sm + STAGES * stage_bytes + (2 * STAGES + 4) * 8 + 16);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int nacc = p.nacc, nbuf = p.nbuf;
-    uint32_t tcols = 32;
-    while (tcols < (uint32_t)(BN * nacc * nbuf)) tcols <<= 1;
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < STAGES; ++i) {
-            mbar_init(bars + 8 * i, 1);
-            mbar_init(bars + 8 * (STAGES + i), 1);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(bar_accf + 8 * i, 1);
-            mbar_init(bar_acce + 8 * i, 4);          // one arrival per epilogue warp
-        }
-        *abort_flag = 0;
-        fence_barrier_init();
-    }
-    if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_slot), tcols);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tbase = *tmem_slot;
-    pdl_wait();
-    if (threadIdx.x == 0) *skip_flag = p.status->code;       // one thread reads the status word: one branch for the CTA
-    __syncthreads();
-    const bool skip = *skip_flag != 0;
-
-    const int per_batch = p.tiles_m * p.tiles_n, total = per_batch * p.batch;
-    constexpr int GM = 8;
-    // tile id -> (batch element, row block, column block); false if the tile has nothing to do
-    auto decode = [&](int t, int& z, int& m0, int& n0) -> bool {
-        z = t / per_batch;
-        const int r = t - z * per_batch;
-        const int group = r / (GM * p.tiles_n);
-        const int first_m = group * GM;
-        const int gsz = min(GM, p.tiles_m - first_m);
-        const int in_g = r - group * GM * p.tiles_n;
-        const int mb = first_m + in_g % gsz, nb = in_g / gsz;
-        m0 = mb * 128;
-        n0 = nb * BN;
-        if (p.lower_only && n0 > m0 + 127) return false;
-        if (p.skip_tile00 && mb == 0 && nb == 0) return false;
-        const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
-        return crow0 < p.c_rows && ccol0 < p.c_cols;
-    };
-    auto k_range = [&](int m0, int n0, int& kt_begin, int& kt_end) {
-        kt_begin = 0;
-        kt_end = (p.K + 63) / 64;
-        if (p.k_tri == 1) kt_end = min(kt_end, (n0 + BN + 63) / 64);
-        if (p.k_tri == 2) kt_begin = min(kt_end, n0 / 64);
-        if (p.a_tri == 1) kt_end = min(kt_end, (m0 + 128 + 63) / 64);
-        if (p.a_tri == 2) kt_begin = max(kt_begin, min(kt_end, m0 / 64));
-    };
-
-    if (skip) {
-        // nothing to do: fall through to the teardown
-    } else if (warp == 0) {
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-                int z, m0, n0, kb, ke;
-                if (!decode(t, z, m0, n0)) continue;
-                k_range(m0, n0, kb, ke);
-                const int ar = p.a_row0 + z * p.a_zrow + m0, ac = p.a_col0 + z * p.a_zcol;
-                const int br = p.b_row0 + z * p.b_zrow + n0, bc = p.b_col0 + z * p.b_zcol;
-                for (int kt = kb; kt < ke; ++kt, ++it) {
-                    const uint32_t s = it % (uint32_t)STAGES;
-                    if (!mbar_wait(bars + 8 * (STAGES + s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, 1)) { ok = false; break; }
-                    const uint32_t full = bars + 8 * s;
-                    const uint32_t sa = base + s * stage_bytes;
-                    mbar_expect_tx(full, stage_bytes);
-                    for (int i = 0; i < p.nA; ++i) tma_load_2d(sa + i * kA, &p.mapA[i], full, ac + kt * 64, ar);
-                    for (int i = 0; i < p.nB; ++i) tma_load_2d(sa + p.nA * kA + i * kB, &p.mapB[i], full, bc + kt * 64, br);
-                }
-            }
-        }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16(128, BN);
-            uint32_t it = 0, tcount = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-                int z, m0, n0, kb, ke;
-                if (!decode(t, z, m0, n0)) continue;
-                k_range(m0, n0, kb, ke);
-                const uint32_t buf = tcount % (uint32_t)nbuf;
-                // the epilogue must have drained this accumulator buffer (first use: passes at once)
-                if (!mbar_wait(bar_acce + 8 * buf, ((tcount / nbuf) & 1) ^ 1, abort_flag, p.status, 4)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t tacc = tbase + buf * (uint32_t)(nacc * BN);
-                uint32_t used = 0u, hh = 0u;
-                for (int kt = kb; kt < ke; ++kt, ++it) {
-                    const uint32_t s = it % (uint32_t)STAGES;
-                    if (!mbar_wait(bars + 8 * s, (it / STAGES) & 1, abort_flag, p.status, 2)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t sa = base + s * stage_bytes;
-                    for (int ps = 0; ps < p.npass; ++ps) {
-                        const uint64_t da = smem_desc_sw128(sa + p.pa[ps] * kA);
-                        const uint64_t db = smem_desc_sw128(sa + p.nA * kA + p.pb[ps] * kB);
-                        const bool big = nacc > 1 && p.pa[ps] == 0 && p.pb[ps] == 0;      // hi x hi
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            const uint32_t acc = big ? 1u + (hh++ % (uint32_t)(nacc - 1)) : 0u;
-                            mma_bf16_ss(tacc + acc * (uint32_t)BN, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc,
-                                        (used >> acc) & 1u);
-                            used |= 1u << acc;
-                        }
-                    }
-                    mma_commit(bars + 8 * (STAGES + s));
-                }
-                if (!ok) break;
-                mma_commit(bar_accf + 8 * buf);      // with no MMA pending (empty contraction) it arrives at once
-                ++tcount;
-            }
-        }
-    } else {
-        // epilogue: TMEM -> registers -> per-warp smem tile -> row-contiguous global accesses
-        const int q = warp & 3;
-        float* stg = staging + q * (32 * 33);
-        const bool vec_ok = p.vec_ok != 0;
-        float* const Cp = p.C_ind ? *p.C_ind : p.C;
-        uint32_t tcount = 0;
-        bool ok = true;
-        for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-            int z, m0, n0, kb, ke;
-            if (!decode(t, z, m0, n0)) continue;
-            k_range(m0, n0, kb, ke);
-            const bool has_acc = ke > kb;
-            const uint32_t buf = tcount % (uint32_t)nbuf;
-            const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
-            const int rl0 = m0 + q * 32;                 // first row of this warp inside the batch element
-            const int rowa0 = crow0 + q * 32;            // ... and its absolute output row
-            const int nrows = max(0, min(32, min(p.M - rl0, p.c_rows - rowa0)));
-            const bool first_col = (n0 == 0);
-            ok = mbar_wait(bar_accf + 8 * buf, (tcount / nbuf) & 1, abort_flag, p.status, 3);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t tacc = tbase + buf * (uint32_t)(nacc * BN) + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t r[32];
-                if (has_acc) {
-                    tmem_ld32(tacc + (uint32_t)c0, r);
-                    tmem_ld_wait();
-                    for (int a = 1; a < nacc; ++a) {
-                        uint32_t r2[32];
-                        tmem_ld32(tacc + (uint32_t)(a * BN + c0), r2);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = 0u;
-                }
-                const int col = ccol0 + c0;                    // absolute output column of r[0]
-                const int ncol = min(min(32, p.N - (n0 + c0)), p.c_cols - col);
-                if (ncol <= 0) break;
-                float v[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = p.alpha * __uint_as_float(r[j]);
-                if (Cp && lane < nrows) {
-                    const size_t row = (size_t)(rowa0 + lane);
-                    float* crow = Cp + row * p.ldc + col;
-                    const float* arow = p.addend ? p.addend + row * p.ldadd + col : nullptr;
-                    if (vec_ok && ncol == 32) {
-                        if (arow) {
-                            float4 a4[8];
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) a4[j] = *reinterpret_cast<const float4*>(arow + 4 * j);
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                v[4 * j] += a4[j].x; v[4 * j + 1] += a4[j].y; v[4 * j + 2] += a4[j].z; v[4 * j + 3] += a4[j].w;
-                            }
-                        }
-                        if (p.accumulate) {
-                            float4 c4[8];
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) c4[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                v[4 * j] += c4[j].x; v[4 * j + 1] += c4[j].y; v[4 * j + 2] += c4[j].z; v[4 * j + 3] += c4[j].w;
-                            }
-                        }
-#pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            *reinterpret_cast<float4*>(crow + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (j < ncol) {
-                                if (arow) v[j] += arow[j];
-                                if (p.accumulate) v[j] += crow[j];
-                                crow[j] = v[j];
-                            }
-                        }
-                    }
-                }
-                if (p.nout > 0 && (!p.out_col0_only || (first_col && c0 < 128)) && p.out_vec && ncol == 32) {
-                    if (lane < nrows) store_parts_row(p, v, (size_t)(rowa0 + lane) * p.ldo + (col - p.out_col_off));
-                } else if (p.nout > 0 && (!p.out_col0_only || (first_col && c0 < 128))) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = v[j];
-                    __syncwarp();
-                    if (lane < ncol) {
-                        for (int rr = 0; rr < nrows; ++rr) {
-                            const float x = stg[rr * 33 + lane];
-                            const size_t o = (size_t)(rowa0 + rr) * p.ldo + (col - p.out_col_off) + lane;
-                            __nv_bfloat16 h = __float2bfloat16_rn(x);
-                            p.out[0][o] = h;
-                            if (p.nout > 1) {
-                                const float r1 = x - __bfloat162float(h);
-                                __nv_bfloat16 m = __float2bfloat16_rn(r1);
-                                p.out[1][o] = m;
-                                if (p.nout > 2) p.out[2][o] = __float2bfloat16_rn(r1 - __bfloat162float(m));
-                            }
-                        }
-                    }
-                    __syncwarp();
-                }
-            }
-            // this warp is done with the accumulator buffer
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acce + 8 * buf);
-            ++tcount;
-        }
-    }
-    // teardown: after an abort give copies in flight time to land before the CTA's smem is released
-    if (*abort_flag) {
-        for (int i = 0; i < 64; ++i) __nanosleep(1000);
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        tmem_dealloc(tbase, tcols);
-    }
-}
-
 // Self-test of the bounded wait: the barrier below is initialised and never arrived on.
 __global__ void k_selftest_wait(DevStatus* status) {
     __shared__ uint64_t bar_mem;
@@ -773,60 +505,10 @@ static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     return PKV_OK;
 }
 
-template <int BN>
-static int launch_gemm_p(const Lc& lc, GemmTcParams& p, int batch) {
-    static PerDeviceOnce once;
-    static int sm_count = 0;
-    constexpr int kMaxSmem = 227 * 1024;
-    int dev;
-    if (once.needed(&dev)) {
-        if (cudaFuncSetAttribute(k_gemm_tcp<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
-            return PKV_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev < 0 ? 0 : dev) != cudaSuccess) return PKV_ERR_CUDA;
-        once.mark(dev);
-    }
-    const int stage_bytes = p.nA * 128 * 128 + p.nB * BN * 128;
-    const int fixed = (2 * kGemmMaxStages + 4) * 8 + 16 + kGemmPStaging + 1024;
-    int stages = (kMaxSmem - fixed) / stage_bytes;
-    if (stages < 1) return PKV_ERR_UNSUPPORTED;
-    if (stages > kGemmMaxStages) stages = kGemmMaxStages;
-    p.stages = stages;
-    p.tiles_m = (p.M + 127) / 128;
-    p.tiles_n = (p.N + BN - 1) / BN;
-    p.batch = batch;
-    p.nbuf = (2 * p.nacc * BN <= 512) ? 2 : 1;
-    const long long total = (long long)p.tiles_m * p.tiles_n * batch;
-    const int sms = (lc.sms > 0 && lc.sms < sm_count) ? lc.sms : sm_count;
-    const int grid = (int)((total < sms) ? total : sms);
-    const int smem = stages * stage_bytes + (2 * stages + 4) * 8 + 16 + kGemmPStaging + 1024;
-    if (lc.pdl) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid);
-        cfg.blockDim = dim3(192);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = lc.st;
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = at;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, k_gemm_tcp<BN>, p) != cudaSuccess) return PKV_ERR_CUDA;
-    } else {
-        k_gemm_tcp<BN><<<grid, 192, smem, lc.st>>>(p);
-    }
-    lc.count();
-    return PKV_OK;
-}
-
-// PKV_GEMM=persistent in the environment selects the persistent kernel.  Measured against the one-tile-per-CTA
-// kernel it changes little (statistics at d = F = 5120: 1.12 vs 1.20 ms; a whole config-2 block: 4.54 vs 4.39 ms):
-// the split-bf16 products are bound by operand traffic from L2 and, at few reference tokens, by the number of
-// tiles, not by the epilogue that the second accumulator buffer hides.  The default stays the simpler kernel.
-static bool gemm_persistent() {
-    static const bool v = [] { const char* e = getenv("PKV_GEMM"); return e && e[0] == 'p'; }();
-    return v;
-}
-
+// (A persistent variant - one CTA per SM walking over the tiles with a second accumulator buffer so that one tile's
+// epilogue overlaps the next tile's MMAs - was built and measured: statistics at d = F = 5120 1.12 vs 1.20 ms, a
+// whole config-2 block 4.54 vs 4.39 ms.  The split-bf16 products are bound by operand traffic from L2 and, at few
+// reference tokens, by the number of tiles, not by the epilogue; the simpler kernel stayed.)
 int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     if (g.M <= 0 || g.N <= 0 || g.batch <= 0) return PKV_OK;
     if (g.K < 0 || g.npass <= 0 || g.npass > kGemmMaxPass || (!g.C && g.nout == 0)) return PKV_ERR_INVALID_ARG;
@@ -894,11 +576,6 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
         for (int i = 0; i < g.nout; ++i) ok = ok && (((uintptr_t)g.out[i]) & 15) == 0;
         // every row offset (c_row0 + z c_zrow + ...) * ldo is then a multiple of 8 elements as well
         p.out_vec = ok ? 1 : 0;
-    }
-    if (gemm_persistent()) {
-        if (BN == 64) return launch_gemm_p<64>(lc, p, g.batch);
-        if (BN == 256) return launch_gemm_p<256>(lc, p, g.batch);
-        return launch_gemm_p<128>(lc, p, g.batch);
     }
     if (BN == 64) return launch_gemm<64>(lc, p, g.batch);
     if (BN == 256) return launch_gemm<256>(lc, p, g.batch);

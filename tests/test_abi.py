@@ -15,7 +15,9 @@ def declared_functions():
 def test_library_builds_loads_and_exports_every_declared_symbol():
     from paper_2609_39329_b200 import build
     path = build.build()
-    lib = ctypes.CDLL(path)
+    # RTLD_NOW: every symbol the library itself refers to must resolve at load time (lazy binding would hide an
+    # internal function that lost its definition until the first call on a GPU machine)
+    lib = ctypes.CDLL(path, mode=os.RTLD_NOW)
     names = declared_functions()
     assert {"pkv_build_patch", "pkv_merge", "pkv_create", "pkv_destroy", "pkv_build_stack"} <= set(names)
     for n in names:

@@ -709,6 +709,35 @@ def test_streamed_reference_set_equals_one_call_and_the_oracle(B, engine_name, l
 
 # ------------------------------------------------------------------ boundary
 
+_ALT_CASE = '''
+import sys
+sys.path.insert(0, %r)
+from paper_2609_39329_b200 import binding as B
+from tests import test_gpu_parity as T
+from tests import helpers as H
+cfg = T.small_cfg("bf16", hd=128, Hq=8, Hkv=2, d=512, F=448, L=3000, N=200, window=32, budget=300, n_obs=16)
+lay = H.make_problem(cfg)
+e = T.check_build(B, cfg, lay, lay["x0"], lay["x0"], [0, 120, cfg.N], 0.1, B.ENGINE_AUTO)
+print("ALT_OK %%.3e" %% e)
+'''
+
+
+@pytest.mark.parametrize("env", [{"PKV_ATTN_Q": "pair"}, {"PKV_SOLVE_GRAPH": "0"}, {"PKV_SOLVE_TRACE": "1"}])
+def test_alternate_paths_selected_by_environment(env):
+    """Paths the environment selects at start-up, each in a process of its own on one small hd-128 block against the
+    oracle: bf16 query pairs against bf16 keys (the attention path for caches outside fp16's range), the solve
+    issued launch by launch instead of replayed as a graph, and the solve's phase trace."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", _ALT_CASE % root], env={**os.environ, **env}, capture_output=True, text=True,
+                       timeout=900, cwd=root)
+    assert r.returncode == 0 and "ALT_OK" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
+    if "PKV_SOLVE_TRACE" in env:
+        assert "solve timeline" in r.stderr
+
+
 def test_boundary_rejects_bad_arguments(B):
     import torch
     cfg = small_cfg("bf16")
