@@ -272,18 +272,30 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                                 v[4 * j] += a4[j].x; v[4 * j + 1] += a4[j].y; v[4 * j + 2] += a4[j].z; v[4 * j + 3] += a4[j].w;
                             }
                         }
-                        if (p.accumulate) {
-                            float4 c4[8];
+                        // C += v.  Where this tile does not also have to write bf16 parts of the sum, the addition is
+                        // left to the memory system (a vector reduction: same single rounding of C + v, no load, and so
+                        // no DRAM round trip per chunk inside the epilogue); every element has one writer per launch.
+                        const bool parts_here = p.nout > 0 && (!p.out_col0_only || blockIdx.x == 0);
+                        if (p.accumulate && !parts_here) {
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) c4[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
+                            for (int j = 0; j < 8; ++j)
+                                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(crow + 4 * j), "f"(v[4 * j]),
+                                             "f"(v[4 * j + 1]), "f"(v[4 * j + 2]), "f"(v[4 * j + 3])
+                                             : "memory");
+                        } else {
+                            if (p.accumulate) {
+                                float4 c4[8];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                v[4 * j] += c4[j].x; v[4 * j + 1] += c4[j].y; v[4 * j + 2] += c4[j].z; v[4 * j + 3] += c4[j].w;
+                                for (int j = 0; j < 8; ++j) c4[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    v[4 * j] += c4[j].x; v[4 * j + 1] += c4[j].y; v[4 * j + 2] += c4[j].z; v[4 * j + 3] += c4[j].w;
+                                }
                             }
-                        }
 #pragma unroll
-                        for (int j = 0; j < 8; ++j)
-                            *reinterpret_cast<float4*>(crow + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                            for (int j = 0; j < 8; ++j)
+                                *reinterpret_cast<float4*>(crow + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                        }
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {

@@ -911,8 +911,14 @@ static int launch_chain(cudaStream_t st, const ChainParams& cp) {
     return cudaLaunchKernelEx(&cfg, k_chain128, cp) == cudaSuccess ? PKV_OK : PKV_ERR_CUDA;
 }
 
+// PKV_SOLVE_TRACE=1: launch-by-launch issue with the chain kernel's phase profile and the stream timeline;
+// PKV_SOLVE_TRACE=graph: the replayed graph, with only the chain kernels' start and end times
+static bool solve_trace_graph() {
+    static const bool v = [] { const char* e = getenv("PKV_SOLVE_TRACE"); return e && e[0] == 'g'; }();
+    return v;
+}
 static bool solve_trace() {
-    static const bool v = getenv("PKV_SOLVE_TRACE") != nullptr;
+    static const bool v = getenv("PKV_SOLVE_TRACE") != nullptr && !solve_trace_graph();
     return v;
 }
 
@@ -956,7 +962,7 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
     cp.G = G; cp.n = n; cp.ld = ld; cp.X3 = X3; cp.XT3 = XT3; cp.six = well_conditioned ? 0 : 1; cp.status = status;
     // phase profile of the chain kernel (environment variable PKV_SOLVE_TRACE=1): clock64 marks, printed to stderr
     const bool trace = solve_trace();
-    cp.stamps = trace ? t->stamps : nullptr;
+    cp.stamps = (trace || solve_trace_graph()) ? t->stamps : nullptr;
     cudaEvent_t evFork = t->ev[0], evF = t->ev[1];
     cudaEvent_t evU[2] = {t->ev[2], t->ev[3]};
     cudaEvent_t evP = t->ev[4], evC = t->ev[5];
@@ -1214,6 +1220,20 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     if (cudaGraphLaunch(e->exec, lc.st) != cudaSuccess) return PKV_ERR_CUDA;
     k_solve_end<<<1, 32, 0, lc.st>>>(status, t->gstatus);
     lc.count();
+    if (solve_trace_graph()) {
+        const int nblk = (n + PB - 1) / PB;
+        static long long hs[64 * kChainStamps];
+        if (nblk <= 64) {
+            cudaStreamSynchronize(lc.st);
+            cudaMemcpy(hs, t->stamps, (size_t)nblk * kChainStamps * sizeof(long long), cudaMemcpyDeviceToHost);
+            fprintf(stderr, "chain kernels of the replayed solve, start-to-start / busy per block (us, global timer):");
+            for (int b = 1; b < nblk; ++b)
+                fprintf(stderr, " %.1f/%.1f", (hs[b * kChainStamps + 16] - hs[(b - 1) * kChainStamps + 16]) * 1e-3,
+                        (hs[b * kChainStamps + 17] - hs[b * kChainStamps + 16]) * 1e-3);
+            fprintf(stderr, " ; first start to last end %.1f us\n",
+                    (hs[(nblk - 1) * kChainStamps + 17] - hs[16]) * 1e-3);
+        }
+    }
     return PKV_OK;
 }
 
