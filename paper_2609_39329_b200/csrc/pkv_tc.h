@@ -59,7 +59,7 @@ int tc_make_map_3d(CUtensorMap* m, const void* ptr, uint64_t d2, uint64_t rows, 
 struct Pair;
 // Workspace of the tensor-core ridge solve: bf16 triples (hi, mid, lo) of the factor L, its inverse X,
 // the inverse's transpose, the current panel, the doubling temporaries; pairs of S_T and S_T X^T.
-constexpr int kSolveEvents = 6;
+constexpr int kSolveEvents = 9;
 constexpr int kSolveGraphs = 4;
 // One captured solve: replayed when the operands, the shape and the precision plan are the same.
 struct SolveGraph {
@@ -81,7 +81,8 @@ struct TcSolveBuffers {
     __nv_bfloat16* Z2[3];
     int nmax;              // largest system the arrays are sized for
     cudaStream_t aux;      // high-priority helper stream of the factorisation's critical chain
-    cudaStream_t bulk;     // helper stream: panels and trailing updates
+    cudaStream_t bulk;     // helper stream: panels and the first two block columns of every trailing update
+    cudaStream_t bulk2;    // helper stream: the rest of every trailing update
     cudaStream_t aux2;     // helper stream: the doubling levels of the inverse beside the factorisation
     cudaEvent_t ev[kSolveEvents];
     CUtensorMap chainP[3], chainX[3];   // tensor maps of the chain kernel's operands, valid for (chain_n, chain_ld)

@@ -857,7 +857,9 @@ int tc_solve_init(TcSolveBuffers* t) {
     // ... the panels and trailing updates (needed two chain steps later) below it, and the doubling levels of the
     // inverse (needed only at the end) below those, filling the SMs the others leave idle
     const int mid = (least + greatest) / 2;
-    if (cudaStreamCreateWithPriority(&t->bulk, cudaStreamNonBlocking, mid) != cudaSuccess) return PKV_ERR_CUDA;
+    if (cudaStreamCreateWithPriority(&t->bulk, cudaStreamNonBlocking, greatest < least ? greatest + 1 : greatest) != cudaSuccess)
+        return PKV_ERR_CUDA;
+    if (cudaStreamCreateWithPriority(&t->bulk2, cudaStreamNonBlocking, mid) != cudaSuccess) return PKV_ERR_CUDA;
     if (cudaStreamCreateWithPriority(&t->aux2, cudaStreamNonBlocking, least) != cudaSuccess) return PKV_ERR_CUDA;
     if (cudaStreamCreateWithFlags(&t->origin, cudaStreamNonBlocking) != cudaSuccess) return PKV_ERR_CUDA;
     t->n_graphs = 0;
@@ -884,7 +886,7 @@ void tc_solve_destroy(TcSolveBuffers* t) {
     }
     for (int i = 0; i < t->n_graphs; ++i) cudaGraphExecDestroy(t->graphs[i].exec);
     t->n_graphs = 0;
-    for (cudaStream_t* st : {&t->origin, &t->bulk, &t->aux2})
+    for (cudaStream_t* st : {&t->origin, &t->bulk, &t->bulk2, &t->aux2})
         if (*st) {
             cudaStreamSynchronize(*st);
             cudaStreamDestroy(*st);
@@ -947,8 +949,9 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
     // block (which the chain kernel does not read back from memory); U_k's first block column also leaves
     // the bf16 triple of the updated column k+1, the operand of P_{k+1} and of the next chain kernel.
     //   chain(k)  needs chain(k-1) and U_{k-2};   P_k needs chain(k) and U_{k-1};   U_k needs P_k.
-    cudaStream_t sA = t->aux, sB = t->bulk;      // priorities: chain > bulk (sB) > the inverse's doubling (sC)
-    Lc lcB{sB, lc.launches, lc.map_cache};
+    // priorities: chain (sA) > panel + first columns of the update (sB) > rest of the update (sE) > the inverse's doubling (sC)
+    cudaStream_t sA = t->aux, sB = t->bulk, sE = t->bulk2;
+    Lc lcB{sB, lc.launches, lc.map_cache}, lcE{sE, lc.launches, lc.map_cache};
     if (t->chain_n != n || t->chain_ld != ld) {
         for (int i = 0; i < 3; ++i) {
             if ((rc = tc_make_map_2d(&t->chainP[i], P3.a[i], F, PB, PB, 128))) return rc;
@@ -966,6 +969,7 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
     cudaEvent_t evFork = t->ev[0], evF = t->ev[1];
     cudaEvent_t evU[2] = {t->ev[2], t->ev[3]};
     cudaEvent_t evP = t->ev[4], evC = t->ev[5];
+    cudaEvent_t evUb[3] = {t->ev[6], t->ev[7], t->ev[8]};
     // Third stream sC: X = L^{-1} by recursive doubling, [A 0; C B]^{-1} = [A^{-1} 0; -B^{-1} C A^{-1}  B^{-1}],
     // pair by pair as soon as a pair's columns are factored, beside the factorisation (whose panel products and
     // chain kernels leave most SMs idle); only the levels that need the last columns remain for the end.
@@ -1015,6 +1019,7 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
     cudaEventRecord(evFork, lc.st);
     cudaStreamWaitEvent(sA, evFork, 0);
     cudaStreamWaitEvent(sB, evFork, 0);
+    cudaStreamWaitEvent(sE, evFork, 0);
     cudaStreamWaitEvent(sC, evFork, 0);
     if (F > PB) {
         launch_split3(lcB, G + (size_t)PB * ld, ld, F - PB, PB,
@@ -1024,7 +1029,8 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
     rc = PKV_OK;
     for (int b = 0; b < nblk && rc == PKV_OK; ++b) {
         const int k0 = b * PB, k1 = min(F, k0 + PB), rem = F - k1;
-        if (b > 0) cudaStreamWaitEvent(sA, evU[b & 1], 0);       // U_{b-2}, or the split of the first column for b = 1
+        if (b > 0) cudaStreamWaitEvent(sA, evU[b & 1], 0);       // U^a_{b-2}, or the split of the first column for b = 1
+        if (b > 2) cudaStreamWaitEvent(sA, evUb[(b - 3) % 3], 0); // U^b_{b-3}: the last bulk part that touches block column b
         cp.k0 = k0;
         if ((rc = launch_chain(sA, cp))) break;
         lc.count();
@@ -1056,17 +1062,36 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
             if ((rc = gemm_tc(lcB, g, status))) break;
         }
         cudaEventRecord(evP, sB);
-        if (rem > PB) {   // U_b: G22 -= L21 L21^T on the lower triangle, the first diagonal tile left to the chain
+        // U_b: G22 -= L21 L21^T on the lower triangle, in two launches.  U^a_b, the first two block columns (on sB):
+        // column b+1 gets its last update here and leaves the bf16 triple of the next panel operand, column b+2
+        // holds the next-but-one diagonal block; the first diagonal tile is left to the chain kernel.  U^b_b, all
+        // further columns (on sE), has two chain steps to finish.  Updates of one tile by U^a and U^b of different
+        // steps may overlap in time: both add through the memory system's reductions; the one launch that reads a
+        // column back (U^a's first column) waits for the bulk parts that touched it.
+        if (rem > PB) {
+            if (b > 1) cudaStreamWaitEvent(sB, evUb[(b - 2) % 3], 0);
             TcGemm g{};
             pass_plan(g, L3, ld, F, F, L3, ld, F, F);
             g.a_row0 = k1; g.a_col0 = k0; g.b_row0 = k1; g.b_col0 = k0;
-            g.M = rem; g.N = rem; g.K = PB; g.batch = 1; g.alpha = -1.f;
+            g.M = rem; g.N = min(rem, 2 * PB); g.K = PB; g.batch = 1; g.alpha = -1.f;
             g.C = const_cast<float*>(G); g.ldc = ld; g.accumulate = true; g.lower_only = true; g.skip_tile00 = true;
             g.c_row0 = k1; g.c_col0 = k1; g.c_rows = F; g.c_cols = F;
             g.out[0] = P3.a[0]; g.out[1] = P3.a[1]; g.out[2] = P3.a[2]; g.ldo = PB; g.nout = 3; g.out_col_off = k1;
             g.out_col0_only = true;
             if ((rc = gemm_tc(lcB, g, status))) break;
         }
+        if (rem > 2 * PB) {
+            const int o = k1 + 2 * PB;
+            cudaStreamWaitEvent(sE, evP, 0);
+            TcGemm g{};
+            pass_plan(g, L3, ld, F, F, L3, ld, F, F);
+            g.a_row0 = o; g.a_col0 = k0; g.b_row0 = o; g.b_col0 = k0;
+            g.M = F - o; g.N = F - o; g.K = PB; g.batch = 1; g.alpha = -1.f;
+            g.C = const_cast<float*>(G); g.ldc = ld; g.accumulate = true; g.lower_only = true;
+            g.c_row0 = o; g.c_col0 = o; g.c_rows = F; g.c_cols = F;
+            if ((rc = gemm_tc(lcE, g, status))) break;
+        }
+        cudaEventRecord(evUb[b % 3], sE);
         cudaEventRecord(evU[b & 1], sB);
     }
     if (trace) {
@@ -1078,7 +1103,8 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
     cudaEventRecord(evP, sB);
     cudaEventRecord(evC, sC);
     if (trace) { cudaEventRecord(tev[1], sA); cudaEventRecord(tev[2], sC); }
-    for (cudaEvent_t e : {evF, evP, evC}) cudaStreamWaitEvent(lc.st, e, 0);
+    cudaEventRecord(evUb[0], sE);
+    for (cudaEvent_t e : {evF, evP, evC, evUb[0]}) cudaStreamWaitEvent(lc.st, e, 0);
     if (rc != PKV_OK) return rc;
     if (trace && nblk <= 64) {
         static long long host_stamps[64 * kChainStamps];
