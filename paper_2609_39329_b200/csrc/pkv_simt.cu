@@ -627,37 +627,55 @@ __device__ __forceinline__ double warp_sum_d(double v) {
     return v;
 }
 
+// Sum of a double over the block: warp shuffles, then one value per warp through shared memory.  Returns the
+// total in thread 0 (other threads: unspecified).
+__device__ __forceinline__ double block_sum_d(double v) {
+    __shared__ double part[32];
+    v = warp_sum_d(v);
+    const int w = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    if ((threadIdx.x & 31) == 0) part[w] = v;
+    __syncthreads();
+    double t = 0.0;
+    if (threadIdx.x < 32) {
+        t = (threadIdx.x < nw) ? part[threadIdx.x] : 0.0;
+        t = warp_sum_d(t);
+    }
+    __syncthreads();
+    return t;
+}
+
 // tr(S) and ||S||_F^2: one row per block iteration, float4 loads, fp32 partial sums per thread
-// (a few hundred terms each), double precision across threads.
+// (a few hundred terms each), double precision across threads; one atomic per block.
 __global__ void __launch_bounds__(256) k_trace_fro2(const float* __restrict__ S, int F, int ld, int lower,
                                                     DevStatus* status) {
     float fro[4] = {0.f, 0.f, 0.f, 0.f};
     double tr = 0.0;
-    int bad = 0;
-    const bool vec = (F % 4 == 0) && (ld % 4 == 0) && (((uintptr_t)S & 15) == 0);
+    const bool vec = (ld % 4 == 0) && (((uintptr_t)S & 15) == 0);
     for (int r = blockIdx.x; r < F; r += gridDim.x) {
         const float* row = S + (size_t)r * ld;
-        if (lower) {
-            // symmetric matrix, lower triangle only: off-diagonal entries count twice
-            for (int c = threadIdx.x; c < r; c += 256) fro[0] = fmaf(2.f * row[c], row[c], fro[0]);
-            if (threadIdx.x == 0) fro[1] = fmaf(row[r], row[r], fro[1]);
-        } else if (vec) {
-            for (int c = threadIdx.x * 4; c < F; c += 1024) {
-                float4 v = *reinterpret_cast<const float4*>(row + c);
-                fro[0] = fmaf(v.x, v.x, fro[0]); fro[1] = fmaf(v.y, v.y, fro[1]);
-                fro[2] = fmaf(v.z, v.z, fro[2]); fro[3] = fmaf(v.w, v.w, fro[3]);
-            }
-        } else {
-            for (int c = threadIdx.x; c < F; c += 256) fro[0] = fmaf(row[c], row[c], fro[0]);
+        // symmetric matrix of which only the lower triangle is valid: entries left of the diagonal count twice
+        const int ncol = lower ? r : F;
+        const float w = lower ? 2.f : 1.f;
+        const int n4 = vec ? (ncol & ~3) : 0;
+        for (int c = threadIdx.x * 4; c < n4; c += 1024) {
+            float4 v = *reinterpret_cast<const float4*>(row + c);
+            fro[0] = fmaf(w * v.x, v.x, fro[0]); fro[1] = fmaf(w * v.y, v.y, fro[1]);
+            fro[2] = fmaf(w * v.z, v.z, fro[2]); fro[3] = fmaf(w * v.w, v.w, fro[3]);
         }
-        if (threadIdx.x == 0) tr += (double)row[r];
+        for (int c = n4 + threadIdx.x; c < ncol; c += 256) fro[0] = fmaf(w * row[c], row[c], fro[0]);
+        if (threadIdx.x == 0) {
+            if (lower) fro[1] = fmaf(row[r], row[r], fro[1]);
+            tr += (double)row[r];
+        }
     }
-    float f = (fro[0] + fro[1]) + (fro[2] + fro[3]);
-    if (!isfinite(f)) bad = 1;
-    double fd = warp_sum_d((double)f);
-    if ((threadIdx.x & 31) == 0) atomicAdd(&status->fro2, fd);
-    if (threadIdx.x == 0 && tr != 0.0) atomicAdd(&status->tr, tr);
-    if (bad) raise(status, PKV_ERR_NONFINITE);
+    const float f = (fro[0] + fro[1]) + (fro[2] + fro[3]);
+    const int bad = __syncthreads_or(!isfinite(f));
+    const double fd = block_sum_d((double)f);
+    if (threadIdx.x == 0) {
+        atomicAdd(&status->fro2, fd);
+        if (tr != 0.0) atomicAdd(&status->tr, tr);
+        if (bad) raise(status, PKV_ERR_NONFINITE);
+    }
 }
 
 void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status, int ld, bool lower) {
@@ -665,19 +683,29 @@ void trace_fro2(const Lc& lc, const float* S, int F, DevStatus* status, int ld, 
     lc.count();
 }
 
+// Sum of squares: four independent 16-byte loads in flight per thread, one atomic per block.
 __global__ void __launch_bounds__(256) k_sumsq(const float* __restrict__ a, size_t n, double* dst) {
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     const size_t n4 = (((uintptr_t)a & 15) == 0) ? n / 4 : 0;
     const float4* a4 = reinterpret_cast<const float4*>(a);
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
-        float4 v = a4[i];
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < n4; i += 4 * stride) {
+        const float4 v0 = a4[i], v1 = a4[i + stride], v2 = a4[i + 2 * stride], v3 = a4[i + 3 * stride];
+        acc[0] = fmaf(v0.x, v0.x, acc[0]); acc[1] = fmaf(v0.y, v0.y, acc[1]); acc[2] = fmaf(v0.z, v0.z, acc[2]); acc[3] = fmaf(v0.w, v0.w, acc[3]);
+        acc[0] = fmaf(v1.x, v1.x, acc[0]); acc[1] = fmaf(v1.y, v1.y, acc[1]); acc[2] = fmaf(v1.z, v1.z, acc[2]); acc[3] = fmaf(v1.w, v1.w, acc[3]);
+        acc[0] = fmaf(v2.x, v2.x, acc[0]); acc[1] = fmaf(v2.y, v2.y, acc[1]); acc[2] = fmaf(v2.z, v2.z, acc[2]); acc[3] = fmaf(v2.w, v2.w, acc[3]);
+        acc[0] = fmaf(v3.x, v3.x, acc[0]); acc[1] = fmaf(v3.y, v3.y, acc[1]); acc[2] = fmaf(v3.z, v3.z, acc[2]); acc[3] = fmaf(v3.w, v3.w, acc[3]);
+    }
+    for (; i < n4; i += stride) {
+        const float4 v = a4[i];
         acc[0] = fmaf(v.x, v.x, acc[0]); acc[1] = fmaf(v.y, v.y, acc[1]);
         acc[2] = fmaf(v.z, v.z, acc[2]); acc[3] = fmaf(v.w, v.w, acc[3]);
     }
-    for (size_t i = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
-        acc[0] = fmaf(a[i], a[i], acc[0]);
-    double s = warp_sum_d((double)((acc[0] + acc[1]) + (acc[2] + acc[3])));
-    if ((threadIdx.x & 31) == 0) atomicAdd(dst, s);
+    for (size_t k = n4 * 4 + (size_t)blockIdx.x * blockDim.x + threadIdx.x; k < n; k += stride)
+        acc[0] = fmaf(a[k], a[k], acc[0]);
+    const double s = block_sum_d((double)((acc[0] + acc[1]) + (acc[2] + acc[3])));
+    if (threadIdx.x == 0) atomicAdd(dst, s);
 }
 
 void sumsq(const Lc& lc, const float* a, int64_t n, double* dst) {
