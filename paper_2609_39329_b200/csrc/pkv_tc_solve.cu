@@ -6,14 +6,15 @@
 //
 //   1. blocked right-looking Cholesky G = L L^T, block 128: one CTA per block column (k_chain128)
 //      applies the previous column's update to the diagonal block, factors it and inverts the factor
-//      in shared memory; the panel (a GEMM with the block inverse) and the trailing update (a GEMM on
-//      the lower triangle) of every column run beside that chain;
+//      in shared memory; the panel (a GEMM with the block inverse) and the trailing update (two GEMMs on
+//      the lower triangle: the two block columns that the next steps wait for, and the rest) of every
+//      column run beside that chain on two further streams;
 //   2. X = L^{-1} by recursive doubling from the 128-block inverses:
 //      [A 0; C B]^{-1} = [A^{-1} 0; -B^{-1} C A^{-1}  B^{-1}], two GEMMs per pair of blocks, issued on a
-//      third stream as soon as a pair's columns are factored (only the pairs that contain the last column
+//      fourth stream as soon as a pair's columns are factored (only the pairs that contain the last column
 //      remain after the factorisation);
 //   3. dW = (S_T X^T) X, two GEMMs that skip the zero tiles of the triangular factor.
-// The launches of one solve (about 150 on three streams) are captured into a CUDA graph per operand set and
+// The launches of one solve (about 260 on four streams) are captured into a CUDA graph per operand set and
 // replayed, see tc_ridge_solve_impl.
 #include <math.h>
 #include <stdio.h>
