@@ -235,7 +235,7 @@ def measure_kernel(kind, cfg, B, torch, peaks, fma_tflops, steps, warmup, flush)
         fn = lambda: ctx.attention(q, k, v, kv["K"], kv["V"], off, idx_t, [0, N])
         b_mean = sum(len(k_) for k_ in kept) / cfg.Hkv
         flops = 4.0 * N * cfg.L * cfg.Dq + 4.0 * N * b_mean * cfg.Dq + 4.0 * N * N * cfg.Dq
-        bound, note = "tensor", "operand preparation + attention kernel + combine; Q counted once (it runs as a bf16 hi+lo pair)"
+        bound, note = "tensor", "key conversion to fp16 + operand preparation + attention kernel + combine; executed MMA work = algorithmic work (fp16 Q against fp16 K, bf16 P against bf16 V)"
     elif kind == "gram":
         ctx = B.PkvContext(B.dims_from_config(cfg, b_max=16))
         X = torch.from_numpy(r.standard_normal((N, F)).astype(np.float32)).cuda()
