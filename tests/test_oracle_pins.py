@@ -535,3 +535,24 @@ def test_bf16_rounding_and_merge_match_torch():
     want = (torch.from_numpy(W) + torch.from_numpy(dW)).to(torch.bfloat16).to(torch.float32).numpy()
     np.testing.assert_array_equal(orc.merge(W, dW, "bf16"), want)
     np.testing.assert_array_equal(orc.merge(W, dW, "fp32"), W + dW)
+
+
+def test_oracle_reproduces_its_stored_values_on_config1():
+    """Drift guard, not a pin: the stored numbers are the oracle's own (the paper prints none), written by
+    tests/golden/make_oracle_fixture.py.  An unintended change of the oracle or of the input recipe shows here."""
+    import importlib.util
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_oracle_fixture", os.path.join(here, "make_oracle_fixture.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    stored = {}
+    for line in open(os.path.join(here, "config1_oracle.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        name, v = line.rstrip("\n").split("\t")
+        stored[name] = float(v)
+    now = dict(mod.values())
+    assert set(now) == set(stored)
+    for name, v in now.items():
+        np.testing.assert_allclose(v, stored[name], rtol=1e-9, err_msg=name)
