@@ -168,6 +168,35 @@ static int gemm_act_weight(const Lc& lc, Pair A, long long lda, const void* W, l
     return gemm_tc(lc, g, st);
 }
 
+// The same for two or three weight matrices applied to the same activations, their outputs side by side in C
+// (q | k | v, gate | up): one launch when every width is a multiple of 256, else one per matrix.
+static int gemm_act_weights(const Lc& lc, Pair A, long long lda, const void* const* W, const int* widths, int nw,
+                            long long ldw, float* C, long long ldc, int M, int K, DevStatus* st) {
+    bool grouped = nw > 1 && nw <= 3;
+    int total = 0;
+    for (int k = 0; k < nw; ++k) { grouped = grouped && widths[k] % 256 == 0; total += widths[k]; }
+    if (!grouped) {
+        int off = 0;
+        for (int k = 0; k < nw; ++k) {
+            const int rc = gemm_act_weight(lc, A, lda, W[k], ldw, C + off, ldc, M, widths[k], K, 1.f, nullptr, 0, st);
+            if (rc != PKV_OK) return rc;
+            off += widths[k];
+        }
+        return PKV_OK;
+    }
+    TcGemm g = plain_gemm(M, total, K, C, ldc, 1.f, nullptr, 0, false);
+    g.A[0] = TcMat{A.hi, lda, M, K};
+    g.A[1] = TcMat{A.lo, lda, M, K};
+    g.B[0] = g.B[1] = TcMat{(const __nv_bfloat16*)W[0], ldw, widths[0], K};
+    g.npass = 2;
+    g.ngrp = nw;
+    for (int k = 0; k < nw; ++k) {
+        g.Bgrp[k] = TcMat{(const __nv_bfloat16*)W[k], ldw, widths[k], K};
+        g.grp_n[k] = widths[k];
+    }
+    return gemm_tc(lc, g, st);
+}
+
 // C = alpha * (A_hi + A_lo)(B_hi + B_lo)^T without the lo*lo term (+ addend) (+ C).
 static int gemm_pair_pair(const Lc& lc, Pair A, long long lda, Pair B, long long ldb, float* C, long long ldc, int M,
                           int Nn, int K, float alpha, const float* addend, long long ldadd, bool accumulate,
@@ -420,9 +449,11 @@ int tc_teacher_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     markT(0);
     k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.xF, a.xF, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, 0);
     lc.count();
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wq, d, t->qkv, QKV, N, Dq, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wk, d, t->qkv + Dq, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wv, d, t->qkv + Dq + Dkv, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        const void* const Ws[3] = {w->Wq, w->Wk, w->Wv};
+        const int widths[3] = {Dq, Dkv, Dkv};
+        if ((rc = gemm_act_weights(lc, t->u, d, Ws, widths, 3, d, t->qkv, QKV, N, d, st))) return rc;
+    }
     markT(1);
     AttnArgs at{};
     fill_attn(at, t, D, a, 1);
@@ -438,8 +469,11 @@ int tc_teacher_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     markT(3);
     k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.zF, a.zF, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, 0);
     lc.count();
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wgate, d, t->gu, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wup, d, t->gu + F, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        const void* const Ws[2] = {w->Wgate, w->Wup};
+        const int widths[2] = {F, F};
+        if ((rc = gemm_act_weights(lc, t->u, d, Ws, widths, 2, d, t->gu, 2 * F, N, d, st))) return rc;
+    }
     {
         size_t n = (size_t)N * F;
         k_swiglu_teacher<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, t->hF);
@@ -464,9 +498,11 @@ int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.xC, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, N);
     lc.count();
     float* qkvS = t->qkv + (size_t)N * QKV;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wq, d, qkvS, QKV, N, Dq, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wk, d, qkvS + Dq, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wv, d, qkvS + Dq + Dkv, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        const void* const Ws[3] = {w->Wq, w->Wk, w->Wv};
+        const int widths[3] = {Dq, Dkv, Dkv};
+        if ((rc = gemm_act_weights(lc, uS, d, Ws, widths, 3, d, qkvS, QKV, N, d, st))) return rc;
+    }
     mark(a, lc, 2);
     AttnArgs at{};
     fill_attn(at, t, D, a, 2);
@@ -484,8 +520,11 @@ int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.zC, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, N);
     lc.count();
     float* guS = t->gu + (size_t)N * 2 * F;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wgate, d, guS, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wup, d, guS + F, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        const void* const Ws[2] = {w->Wgate, w->Wup};
+        const int widths[2] = {F, F};
+        if ((rc = gemm_act_weights(lc, uS, d, Ws, widths, 2, d, guS, 2 * F, N, d, st))) return rc;
+    }
     {
         size_t n = (size_t)N * F;
         k_swiglu_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hC, t->dh);
@@ -520,9 +559,11 @@ int tc_student_propagate(const Lc& lc, TcBuffers* t, const pkv_dims* D, const Tc
     k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.xC, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, N);
     lc.count();
     float* qkvS = t->qkv + (size_t)N * QKV;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wq, d, qkvS, QKV, N, Dq, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wk, d, qkvS + Dq, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wv, d, qkvS + Dq + Dkv, QKV, N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        const void* const Ws[3] = {w->Wq, w->Wk, w->Wv};
+        const int widths[3] = {Dq, Dkv, Dkv};
+        if ((rc = gemm_act_weights(lc, uS, d, Ws, widths, 3, d, qkvS, QKV, N, d, st))) return rc;
+    }
     AttnArgs at{};
     fill_attn(at, t, D, a, 2);
     if ((rc = attention_tc(lc, t, D, at, a.rope_tab, st))) return rc;
@@ -536,8 +577,11 @@ int tc_student_propagate(const Lc& lc, TcBuffers* t, const pkv_dims* D, const Tc
     k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.zC, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, N);
     lc.count();
     float* guS = t->gu + (size_t)N * 2 * F;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wgate, d, guS, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, uS, d, w->Wup, d, guS + F, 2 * F, N, F, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        const void* const Ws[2] = {w->Wgate, w->Wup};
+        const int widths[2] = {F, F};
+        if ((rc = gemm_act_weights(lc, uS, d, Ws, widths, 2, d, guS, 2 * F, N, d, st))) return rc;
+    }
     {
         size_t n = (size_t)N * F;
         k_swiglu_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hC, t->dh);
@@ -560,10 +604,11 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     // S1-S2: both streams stacked, rows [0,N) teacher, [N,2N) student
     k_rmsnorm_split<<<2 * N, 256, 0, lc.st>>>(a.xF, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, 0);
     lc.count();
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wq, d, t->qkv, QKV, 2 * N, Dq, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wk, d, t->qkv + Dq, QKV, 2 * N, Dkv, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wv, d, t->qkv + Dq + Dkv, QKV, 2 * N, Dkv, d, 1.f, nullptr, 0, st)))
-        return rc;
+    {
+        const void* const Ws[3] = {w->Wq, w->Wk, w->Wv};
+        const int widths[3] = {Dq, Dkv, Dkv};
+        if ((rc = gemm_act_weights(lc, t->u, d, Ws, widths, 3, d, t->qkv, QKV, 2 * N, d, st))) return rc;
+    }
     rope_table(lc, a.tok_cs, N, hd, a.pos0, D->rope_theta, a.rope_tab);
     mark(a, lc, 2);
     // S3
@@ -585,8 +630,11 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     // S5
     k_rmsnorm_split<<<2 * N, 256, 0, lc.st>>>(a.zF, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, 0);
     lc.count();
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wgate, d, t->gu, 2 * F, 2 * N, F, d, 1.f, nullptr, 0, st))) return rc;
-    if ((rc = gemm_act_weight(lc, t->u, d, w->Wup, d, t->gu + F, 2 * F, 2 * N, F, d, 1.f, nullptr, 0, st))) return rc;
+    {
+        const void* const Ws[2] = {w->Wgate, w->Wup};
+        const int widths[2] = {F, F};
+        if ((rc = gemm_act_weights(lc, t->u, d, Ws, widths, 2, d, t->gu, 2 * F, 2 * N, d, st))) return rc;
+    }
     {
         size_t n = (size_t)N * F;
         k_swiglu_split<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hF, t->hC, t->dh);

@@ -22,6 +22,11 @@ struct TcMat {
 struct TcGemm {
     TcMat A[kGemmMaxPass], B[kGemmMaxPass];
     int npass;
+    // Grouped B: the product's columns are the concatenation of ngrp (2 or 3) matrices Bgrp[k] [grp_n[k]][K]
+    // (separately stored weights applied to the same activations: Wq | Wk | Wv, Wgate | Wup), every pass taking
+    // the group's matrix as its B operand (B[] is then ignored); each grp_n[k] must be a multiple of the tile width
+    TcMat Bgrp[3];
+    int ngrp, grp_n[3];
     int a_row0, a_col0, a_zrow, a_zcol;
     int b_row0, b_col0, b_zrow, b_zcol;
     int M, N, K, batch;

@@ -27,6 +27,7 @@ struct alignas(64) GemmTcParams {
     CUtensorMap mapA[3];      // distinct A operands (e.g. hi, mid, lo parts)
     CUtensorMap mapB[3];      // distinct B operands
     int nA, nB, npass;
+    int ngrp, grp_end[3];     // grouped B (see TcGemm): mapB[k] serves output columns [grp_end[k-1], grp_end[k])
     int pa[kGemmMaxPass], pb[kGemmMaxPass];   // pass i multiplies A operand pa[i] with B operand pb[i]
     int stages;
     int M, N, K;
@@ -172,7 +173,13 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     } else if (warp == 0) {
         if (lane == 0) {
             const int ar = p.a_row0 + z * p.a_zrow + m0, ac = p.a_col0 + z * p.a_zcol;
-            const int br = p.b_row0 + z * p.b_zrow + n0, bc = p.b_col0 + z * p.b_zcol;
+            int br = p.b_row0 + z * p.b_zrow + n0;
+            const int bc = p.b_col0 + z * p.b_zcol;
+            int gsel = 0;      // grouped B: the matrix this tile's columns belong to, rows counted from its start
+            if (p.ngrp > 1) {
+                while (gsel + 1 < p.ngrp && n0 >= p.grp_end[gsel]) ++gsel;
+                if (gsel > 0) br -= p.grp_end[gsel - 1];
+            }
             for (int it = 0; it < ktiles; ++it) {
                 const int s = it % STAGES;
                 if (!mbar_wait(bars + 8 * (STAGES + s), ((it / STAGES) & 1) ^ 1, abort_flag, p.status, 1)) break;
@@ -181,7 +188,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                 const uint32_t sa = base + s * stage_bytes;
                 mbar_expect_tx(full, stage_bytes);
                 for (int i = 0; i < p.nA; ++i) tma_load_2d(sa + i * kA, &p.mapA[i], full, ac + kt * 64, ar);
-                for (int i = 0; i < p.nB; ++i) tma_load_2d(sa + p.nA * kA + i * kB, &p.mapB[i], full, bc + kt * 64, br);
+                for (int i = 0; i < p.nB; ++i) tma_load_2d(sa + p.nA * kA + i * kB, &p.mapB[p.ngrp > 1 ? gsel : i], full, bc + kt * 64, br);
             }
         }
     } else if (warp == 1) {
@@ -556,6 +563,21 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
         }
         p.pa[i] = ia;
         p.pb[i] = ib;
+    }
+    p.ngrp = 0;
+    if (g.ngrp > 1) {
+        // grouped B: one operand slot in shared memory, one tensor map per group
+        if (g.ngrp > 3 || p.nB != 1) return PKV_ERR_INVALID_ARG;
+        int end = 0;
+        for (int k = 0; k < g.ngrp; ++k) {
+            if (g.grp_n[k] <= 0 || g.grp_n[k] % BN != 0) return PKV_ERR_INVALID_ARG;
+            int rc = cached_map(cache, &p.mapB[k], g.Bgrp[k].p, g.Bgrp[k].rows, g.Bgrp[k].cols, g.Bgrp[k].ld, BN);
+            if (rc != PKV_OK) return rc;
+            end += g.grp_n[k];
+            p.grp_end[k] = end;
+        }
+        if (end != g.N) return PKV_ERR_INVALID_ARG;
+        p.ngrp = g.ngrp;
     }
     p.npass = g.npass; p.M = g.M; p.N = g.N; p.K = g.K;
     p.a_row0 = g.a_row0; p.a_col0 = g.a_col0; p.a_zrow = g.a_zrow; p.a_zcol = g.a_zcol;
