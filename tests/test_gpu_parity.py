@@ -423,6 +423,30 @@ def test_ridge_solve_parity_modes_and_errors(B, F, d, n):
         ctx.close()
 
 
+def test_solve_with_more_operand_sets_than_cached_graphs(B):
+    """The solve is replayed from a graph captured per operand set, a few of which are kept: six different S_T
+    buffers in turn (older graphs are dropped), then the first again, each against the oracle; the result address
+    changes from call to call as well."""
+    import torch
+    F, d, n = 320, 256, 90
+    cfg = small_cfg("bf16", F=F, d=d, Hq=4, Hkv=1)
+    r = np.random.default_rng(11)
+    X = r.standard_normal((n, F))
+    S_H, _ = orc.sufficient_statistics(X, r.standard_normal((n, d)))
+    lam = orc.ridge_lambda(S_H, 0.1, B.LAMBDA_PAPER)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    tH = torch.from_numpy(S_H.astype(np.float32)).cuda()
+    sets = []
+    for i in range(6):
+        _, S_T = orc.sufficient_statistics(X, r.standard_normal((n, d)))
+        sets.append((S_T, torch.from_numpy(S_T.astype(np.float32)).cuda()))
+    for i in list(range(6)) + [0, 3]:
+        S_T, tT = sets[i]
+        dW, _ = ctx.ridge_solve(tH, tT, 0.1, B.LAMBDA_PAPER)
+        assert H.rel_fro(dW.cpu().numpy(), orc.ridge_solve(S_H, S_T, lam)) <= 1e-3, i
+    ctx.close()
+
+
 def test_standalone_solve_after_a_build_uses_the_callers_statistics(B):
     """A build leaves its own S_T split into bf16 parts inside the context; a later pkv_ridge_solve must take the
     S_T it is handed."""
