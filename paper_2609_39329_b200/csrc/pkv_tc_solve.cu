@@ -809,9 +809,9 @@ int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const flo
 
 // elements of the doubling's temporary TT
 static size_t tt_elems(int F) {
-    size_t best = (size_t)PB * PB;      // one pair at a time: the largest level below F
-    for (long long s = PB; s < F; s *= 2) best = (size_t)(s * s);
-    return best;
+    size_t sum = (size_t)PB * PB;       // one s x s region per doubling level s = 128, 256, ... below F
+    for (long long s = PB; s < F; s *= 2) sum += (size_t)(s * s);
+    return sum;
 }
 
 size_t tc_solve_carve(TcSolveBuffers* t, char* base, size_t off, int nmax, int dmax) {
@@ -981,31 +981,38 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
         if (well_conditioned) three_pass(g, A, lda, ar, ac, B, ldb, br, bc);
         else six_pass(g, A, lda, ar, ac, B, ldb, br, bc);
     };
-    // pair p of level s: rows/columns [o, o + 2s) clipped to F, o = 2 s p; top-left inverse (s x s) and
-    // bottom-right inverse (bot x bot) are finished, the bottom-left block of L is the panel's
-    auto doubling_pair = [&](int s, int p) -> int {
+    // Pair p of level s: rows/columns [o, o + 2s) clipped to F, o = 2 s p.  Its first product needs only the top
+    // half (inverse A^{-1} and the block C of L below it) and is issued as soon as that half is factored; the
+    // second one waits for the bottom-right inverse.  Every level has its own TT region (a pair's first product
+    // precedes its second, and the next pair of the level starts after that).
+    auto tt_level = [&](int s) {
+        size_t off = 0;
+        for (long long q = PB; q < s; q *= 2) off += (size_t)(q * q);
+        return Trip{{TT3.a[0] + off, TT3.a[1] + off, TT3.a[2] + off}};
+    };
+    auto pair_first = [&](int s, int p) -> int {      // TT [s][bot] = A^{-T} C^T   (A^{-T} upper triangular: k >= row)
         const int o = 2 * s * p, bot = min(s, F - (o + s));
-        {   // TT [s][bot] = A^{-T} C^T   (A^{-T} upper triangular: contraction index >= row)
-            TcGemm g{};
-            pass_plan(g, XT3, ld, F, F, L3, ld, F, F);
-            g.a_row0 = o; g.a_col0 = o; g.a_tri = 2;
-            g.b_row0 = o + s; g.b_col0 = o;
-            g.M = s; g.N = bot; g.K = s; g.batch = 1; g.alpha = 1.f;
-            g.c_rows = s; g.c_cols = s;
-            g.out[0] = TT3.a[0]; g.out[1] = TT3.a[1]; g.out[2] = TT3.a[2]; g.ldo = s; g.nout = 3;
-            const int r = gemm_tc(lcC, g, status);
-            if (r) return r;
-        }
-        {   // X(bottom-left) [bot][s] = -B^{-1} TT^T   (B^{-1} lower triangular: contraction index <= row)
-            TcGemm g{};
-            pass_plan(g, X3, ld, F, F, TT3, s, s, s);
-            g.a_row0 = o + s; g.a_col0 = o + s; g.a_tri = 1;
-            g.M = bot; g.N = s; g.K = bot; g.batch = 1; g.alpha = -1.f;
-            g.c_row0 = o + s; g.c_col0 = o; g.c_rows = F; g.c_cols = F;
-            g.out[0] = X3.a[0]; g.out[1] = X3.a[1]; g.out[2] = X3.a[2]; g.ldo = ld; g.nout = 3;
-            const int r = gemm_tc(lcC, g, status);
-            if (r) return r;
-        }
+        const Trip TT = tt_level(s);
+        TcGemm g{};
+        pass_plan(g, XT3, ld, F, F, L3, ld, F, F);
+        g.a_row0 = o; g.a_col0 = o; g.a_tri = 2;
+        g.b_row0 = o + s; g.b_col0 = o;
+        g.M = s; g.N = bot; g.K = s; g.batch = 1; g.alpha = 1.f;
+        g.c_rows = s; g.c_cols = s;
+        g.out[0] = TT.a[0]; g.out[1] = TT.a[1]; g.out[2] = TT.a[2]; g.ldo = s; g.nout = 3;
+        return gemm_tc(lcC, g, status);
+    };
+    auto pair_second = [&](int s, int p) -> int {     // X(bottom-left) [bot][s] = -B^{-1} TT^T   (B^{-1} lower triangular: k <= row)
+        const int o = 2 * s * p, bot = min(s, F - (o + s));
+        const Trip TT = tt_level(s);
+        TcGemm g{};
+        pass_plan(g, X3, ld, F, F, TT, s, s, s);
+        g.a_row0 = o + s; g.a_col0 = o + s; g.a_tri = 1;
+        g.M = bot; g.N = s; g.K = bot; g.batch = 1; g.alpha = -1.f;
+        g.c_row0 = o + s; g.c_col0 = o; g.c_rows = F; g.c_cols = F;
+        g.out[0] = X3.a[0]; g.out[1] = X3.a[1]; g.out[2] = X3.a[2]; g.ldo = ld; g.nout = 3;
+        const int r = gemm_tc(lcC, g, status);
+        if (r) return r;
         dim3 grid(s / 32, s / 32, 1), block(32, 8);
         k_transpose_blocks<<<grid, block, 0, sC>>>(X3, XT3, n, ld, s, p);
         lc.count();
@@ -1042,11 +1049,18 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
             dim3 grid(PB / 32, PB / 32, 1), block(32, 8);
             k_transpose_diag<<<grid, block, 0, sC>>>(X3, XT3, n, ld, b);
             lc.count();
+            // first products of the pairs whose top half ended with block b - 1 (its panel P_{b-1} is the block C)
+            for (long long s = PB; s < F && rc == PKV_OK; s *= 2) {
+                const int per = (int)(2 * s / PB), p = b / per;
+                if (b % per != per / 2 || (2LL * p + 1) * s >= F) continue;
+                rc = pair_first((int)s, p);
+            }
+            // second products of the pairs that block b completes, lowest level first
             for (long long s = PB; s < F && rc == PKV_OK; s *= 2) {
                 const int per = (int)(2 * s / PB), p = b / per;
                 if ((2LL * p + 1) * s >= F) continue;            // no bottom half: nothing to do at this level
                 if (b + 1 != min(nblk, (p + 1) * per)) continue; // the pair's last block is not b
-                rc = doubling_pair((int)s, p);
+                rc = pair_second((int)s, p);
             }
             if (rc != PKV_OK) break;
         }
