@@ -129,6 +129,10 @@ constexpr int kMaxStackLayers = 128;
 constexpr int kRing = 3;                    // teacher blocks in flight ahead of the student (ring slots of aF, zF, hF)
 constexpr int kRingX = kRing + 2;           // ring of the teacher's next states: read again after the student's solve
 constexpr int kDefaultReserveSms = 12;      // SMs the teacher stream leaves to the student and the solve (stack driver)
+// Single-block build with a light teacher half (see build_teacher_stream): SMs its partition leaves to the solve.
+// Measured at d = F = 4096, N = 512, L = 32768: 3.24 ms per block without the overlap, 3.07 / 2.94 / 2.92 / 2.91 / 3.35
+// with 32 / 56 / 76 / 90 / 104 SMs left to the solve.
+constexpr int kBuildReserveSms = 80;
 
 struct Carver {
     char* base;
@@ -204,6 +208,9 @@ struct pkv_ctx {
     cudaStream_t tstream;    // teacher stream of the overlapped stack driver
     void* tgreen;            // green context that owns the teacher stream's SM partition (or null)
     int teacher_sms;         // SMs the teacher stream may use (sm_count when not partitioned)
+    cudaStream_t bstream;    // single-block build: stream of a smaller partition for a light teacher half (or null)
+    void* bgreen;
+    int build_teacher_sms;
     cudaEvent_t evTea[kRing], evStu[kRing], evSetup;
     int64_t launches;
     int stream_open, stream_mode, stream_tokens;   // streamed reference set in progress (pkv_stream_*)
@@ -402,6 +409,13 @@ extern "C" int pkv_create(pkv_ctx** out, const pkv_dims* dims, const pkv_opts* o
             pkv_destroy(c);
             return PKV_ERR_NOMEM;
         }
+        {
+            int keep = kBuildReserveSms;
+            if (const char* e = getenv("PKV_BUILD_RESERVE_SMS")) keep = atoi(e);
+            c->build_teacher_sms = 0;
+            if (keep > 0 && keep + 8 <= c->sm_count)
+                make_partition_stream(c->sm_count - keep, &c->bstream, &c->bgreen, &c->build_teacher_sms);
+        }
         for (int i = 0; i < kRing; ++i) {
             cudaEventCreateWithFlags(&c->evTea[i], cudaEventDisableTiming);
             cudaEventCreateWithFlags(&c->evStu[i], cudaEventDisableTiming);
@@ -430,8 +444,11 @@ extern "C" void pkv_destroy(pkv_ctx* c) {
     if (c->host_status) cudaFreeHost(c->host_status);
     if (c->host_lhead) cudaFreeHost(c->host_lhead);
     if (c->host_lstatus) cudaFreeHost(c->host_lstatus);
+    if (c->engine != PKV_ENGINE_SIMT && c->b.tc.side) cudaStreamSynchronize(c->b.tc.side);
     if (c->tstream) { cudaStreamSynchronize(c->tstream); cudaStreamDestroy(c->tstream); }
     green_partition_destroy(c->tgreen);
+    if (c->bstream) { cudaStreamSynchronize(c->bstream); cudaStreamDestroy(c->bstream); }
+    green_partition_destroy(c->bgreen);
     for (int i = 0; i < kRing; ++i) {
         if (c->evTea[i]) cudaEventDestroy(c->evTea[i]);
         if (c->evStu[i]) cudaEventDestroy(c->evStu[i]);
@@ -647,6 +664,21 @@ static AttnArgs attn_args(pkv_ctx* c, const float* q, int64_t ldq, const float* 
     return a;
 }
 
+// Single-block build, teacher half beside the solve: which stream it runs on.  The solve's factorisation is a chain of
+// about 45 us per 128 columns that leaves most SMs idle but stalls when its trailing updates are starved.  A teacher
+// half that fits into that idle time gets the small partition (it must not crowd the updates out); a heavier one is
+// the bottleneck itself and gets the stack driver's partition (all SMs but a small reserve).
+static cudaStream_t build_teacher_stream(const pkv_ctx* c, int N) {
+    const pkv_dims& D = c->dims;
+    const double Dq = (double)D.Hq * D.hd, Dkv = (double)D.Hkv * D.hd, d = D.d, F = D.F;
+    const double attn = 4.0 * N * Dq * ((double)D.L + N);
+    const double gemm = 2.0 * N * (d * (Dq + 2 * Dkv) + Dq * d + 2 * d * F + 2 * F * d) * 2.0;     // two passes each
+    const double teacher_ms = (attn / 0.9e15 + gemm / 1.0e15) * 1e3;
+    const double chain_ms = (F / 128.0) * 0.045;
+    if (c->bstream && teacher_ms < 0.6 * chain_ms) return c->bstream;
+    return c->tstream;
+}
+
 // S0: returns the compact cache pointers to use
 static void stage_compact(pkv_ctx* c, const Lc& lc, const pkv_kv* full, const pkv_kv_compressed* cb, int total,
                           const void** Kc, const void** Vc, const int32_t* head_off_dev = nullptr,
@@ -793,8 +825,12 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         fa.ev = c->timing ? c->ev : nullptr;
         fa.evT = nullptr;
         c->teacher_timed = 0;
-        rc = pkv::tc_forward(lc, &b.tc, &c->dims, fa);
-        if (rc != PKV_OK) return rc;
+        if (pkv::tc_forward_overlapped_applies(&b.tc, fa)) rc = pkv::tc_forward_overlapped(lc, &b.tc, &c->dims, fa, build_teacher_stream(c, N));
+        else rc = pkv::tc_forward(lc, &b.tc, &c->dims, fa);
+        if (rc != PKV_OK) {
+            pkv::tc_side_quiesce(&b.tc);
+            return rc;
+        }
     }
     if (stats_only) {
         // teacher's next states of these tokens, if asked: xF_next = zF + hF W^T
@@ -809,12 +845,17 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         return end_call(c, stats, cb->head_off);
     }
     // S8 (Eq. 7-8)
+    bool next_async = false;
     if (c->dual) {
         rc = pkv::tc_dual_solve(lc, &b.tc, &c->dims, N, b.R, lambda, mode, dW, b.status);
         if (rc != PKV_OK) return rc;
         sumsq(lc, dW, (int64_t)d * F, &b.status->dw_fro2);
     } else {
+        // the teacher's next state does not depend on the patch: beside the solve where the side stream is in use
+        if (next && c->engine != PKV_ENGINE_SIMT)
+            next_async = pkv::tc_teacher_next_async(lc, &b.tc, &c->dims, N, w->Wdown, b.zF, next->xF_next, b.status);
         solve_stage(c, lc, b.S_H, b.S_T, lambda, mode, dW, true);
+        if (c->engine != PKV_ENGINE_SIMT) pkv::tc_build_trace_mark(&b.tc, 4, c->st);
     }
     mark(c, ST_NEXT);
     // S9: xF_next = zF + hF W^T;  D = R - hC dW^T;  xC_next = xF_next - D
@@ -823,13 +864,18 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
             gemm_tn_simt(lc, b.hF, F, w->Wdown, F, bf, next->xF_next, d, N, d, F, 1.f, b.zF, d, false);
             gemm_tn_simt(lc, b.hC, F, dW, F, false, b.D, d, N, d, F, -1.f, b.R, d, false);
         } else {
-            pkv::tc_next_states(lc, &b.tc, &c->dims, N, w->Wdown, dW, b.zF, b.R, next->xF_next, b.D, b.status);
+            pkv::tc_next_states(lc, &b.tc, &c->dims, N, w->Wdown, dW, b.zF, b.R, next_async ? nullptr : next->xF_next,
+                                b.D, b.status);
+            pkv::tc_side_join(lc, &b.tc);
         }
         sumsq(lc, b.D, (int64_t)N * d, &b.status->res_fro2);
         sub_f32(lc, next->xF_next, b.D, (int64_t)N * d, next->xC_next);
     }
     mark(c, ST_COUNT);
-    return end_call(c, stats, cb->head_off);
+    if (c->engine != PKV_ENGINE_SIMT && !c->dual) pkv::tc_build_trace_mark(&b.tc, 5, c->st);
+    rc = end_call(c, stats, cb->head_off);
+    if (c->engine != PKV_ENGINE_SIMT && !c->dual) pkv::tc_build_trace_print(&b.tc);
+    return rc;
 }
 
 extern "C" int pkv_build_patch(pkv_ctx* ctx, const pkv_block_weights* w, const pkv_kv* full,

@@ -90,6 +90,11 @@ struct AttnArgs {
     float* part_m; float* part_l; float* part_O;   // [nsplit][Hkv][N*g] and [..][hd]
     float* aF; float* aC; float* dA;      // [N][Hq*hd]
     __nv_bfloat16* pair_hi; __nv_bfloat16* pair_lo;   // optional: bf16 hi/lo parts of [aF; dA] as [2N][Hq*hd]
+    // Student before teacher (a build whose teacher half runs beside the solve).  With mode 2 the combine writes aC
+    // and its pair into rows [N,2N) and no difference; with mode 1 it reads that aC, writes aF and dA = aF - aC and
+    // puts the pair of dA (not of aF) into rows [0,N).
+    int student_first;
+    void* combine_wait;                   // host side only: a cudaEvent_t the combine's stream waits for first
 };
 void attention_simt(const Lc& lc, const AttnArgs& a);
 void attention_combine(const Lc& lc, const AttnArgs& a);

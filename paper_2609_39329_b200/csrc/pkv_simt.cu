@@ -501,7 +501,7 @@ __global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
     int per = hd / 32;                       // 2 or 4 columns per lane
     float res[2][4];
     const size_t o = (size_t)tok * a.Hq * hd + (size_t)(kh * g + hg) * hd + lane * per;
-    if (a.mode == 2) {      // the teacher's output was produced earlier
+    if (a.mode == 2 && !a.student_first) {      // the teacher's output was produced earlier
         for (int c = 0; c < per; ++c) res[0][c] = a.aF[o + c];
     }
     for (int s = (a.mode == 2 ? 1 : 0); s < (a.mode == 1 ? 1 : 2); ++s) {
@@ -521,6 +521,31 @@ __global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
         }
         float inv = (den > 0.f) ? 1.f / den : 0.f;
         for (int c = 0; c < per; ++c) res[s][c] = num[c] * inv;
+    }
+    if (a.student_first) {
+        for (int c = 0; c < per; ++c) {
+            if (a.mode == 2) {          // student alone: aC and its pair in rows [N,2N)
+                const float v = res[1][c];
+                a.aC[o + c] = v;
+                if (a.pair_hi) {
+                    const size_t o2 = o + c + (size_t)a.N * a.Hq * hd;
+                    __nv_bfloat16 h = __float2bfloat16_rn(v);
+                    a.pair_hi[o2] = h;
+                    a.pair_lo[o2] = __float2bfloat16_rn(v - __bfloat162float(h));
+                }
+            } else {                    // teacher after the student: aF, dA = aF - aC, pair of dA in rows [0,N)
+                const float f = res[0][c];
+                const float dd = f - a.aC[o + c];
+                a.aF[o + c] = f;
+                a.dA[o + c] = dd;
+                if (a.pair_hi) {
+                    __nv_bfloat16 h = __float2bfloat16_rn(dd);
+                    a.pair_hi[o + c] = h;
+                    a.pair_lo[o + c] = __float2bfloat16_rn(dd - __bfloat162float(h));
+                }
+            }
+        }
+        return;
     }
     for (int c = 0; c < per; ++c) {
         const float f = res[0][c];
@@ -549,6 +574,7 @@ __global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
 void attention_combine(const Lc& lc, const AttnArgs& a) {
     int g = a.Hq / a.Hkv;
     long long warps = (long long)a.Hkv * a.N * g;
+    if (a.combine_wait) cudaStreamWaitEvent(lc.st, (cudaEvent_t)a.combine_wait, 0);
     k_attn_combine<<<(unsigned)((warps + 7) / 8), 256, 0, lc.st>>>(a);
     lc.count();
 }

@@ -6,6 +6,8 @@
 // fp32 tensor memory; differences (dA, dz, dh) are formed in fp32 before any rounding so that
 // the target T = W dh + dz of Eq. 5 does not inherit the rounding of two nearly equal streams.
 #include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include "pkv_tc.h"
 
@@ -111,6 +113,30 @@ __global__ void k_oproj_student(const float* __restrict__ dx, const float* __res
     float dd = dx[i] + o[n + i];
     dz[i] = dd;
     zC[i] = zF[i] - dd;
+}
+
+// teacher half after the student's: dz = (xF - xC) + o[0:N] (the projection of dA), zF = zC + dz
+__global__ void k_oproj_teacher_diff(const float* __restrict__ xF, const float* __restrict__ xC,
+                                     const float* __restrict__ o, const float* __restrict__ zC, size_t n,
+                                     float* __restrict__ zF, float* __restrict__ dz) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float dd = (xF[i] - xC[i]) + o[i];
+    dz[i] = dd;
+    zF[i] = zC[i] + dd;
+}
+// teacher half after the student's: hF (fp32 + pair) from gu rows [0,N), dh = hF - hC (pair) with the student's hC
+__global__ void __launch_bounds__(256) k_swiglu_teacher_diff(const float* __restrict__ gu, int N, int F,
+                                                             const float* __restrict__ hC32, float* __restrict__ hF32,
+                                                             Pair hF, Pair dh) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)N * F) return;
+    size_t r = i / F, c = i % F;
+    const float* a = gu + r * 2 * F;
+    float f = silu_f(a[c]) * a[F + c];
+    hF32[i] = f;
+    split2(f, hF.hi[i], hF.lo[i]);
+    split2(f - hC32[i], dh.hi[i], dh.lo[i]);
 }
 
 // in [rows][cols] fp32 -> out pair [cols][ldo] (token-contiguous operands of the statistics)
@@ -287,9 +313,36 @@ size_t tc_carve(TcBuffers* t, char* base, size_t off, const pkv_dims* d, int dua
 int tc_init(TcBuffers* t, const pkv_dims*) {
     int rc = tc_solve_init(&t->solve);
     if (rc == PKV_OK && t->dual_enabled) rc = tc_solve_init(&t->dual);
-    return rc;
+    if (rc != PKV_OK) return rc;
+    int least = 0, greatest = 0;
+    cudaDeviceGetStreamPriorityRange(&least, &greatest);
+    if (cudaStreamCreateWithPriority(&t->side, cudaStreamNonBlocking, least) != cudaSuccess ||
+        cudaEventCreateWithFlags(&t->evSide, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&t->evSideDone, cudaEventDisableTiming) != cudaSuccess)
+        return PKV_ERR_CUDA;
+    t->S_T_async = t->next_async = 0;
+    if (cudaStreamCreateWithPriority(&t->fast, cudaStreamNonBlocking, greatest) != cudaSuccess) return PKV_ERR_CUDA;
+    for (cudaEvent_t& e : t->evq)
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return PKV_ERR_CUDA;
+    return PKV_OK;
 }
 void tc_destroy(TcBuffers* t) {
+    if (t->side) {
+        cudaStreamSynchronize(t->side);
+        cudaStreamDestroy(t->side);
+        t->side = nullptr;
+    }
+    if (t->fast) {
+        cudaStreamSynchronize(t->fast);
+        cudaStreamDestroy(t->fast);
+        t->fast = nullptr;
+    }
+    for (cudaEvent_t& e : t->evq)
+        if (e) { cudaEventDestroy(e); e = nullptr; }
+    for (cudaEvent_t& e : t->tr)
+        if (e) { cudaEventDestroy(e); e = nullptr; }
+    if (t->evSide) { cudaEventDestroy(t->evSide); t->evSide = nullptr; }
+    if (t->evSideDone) { cudaEventDestroy(t->evSideDone); t->evSideDone = nullptr; }
     tc_solve_destroy(&t->solve);
     if (t->dual_enabled) tc_solve_destroy(&t->dual);
 }
@@ -357,47 +410,146 @@ static void six_pass_stats(TcGemm& g, Pair A, const __nv_bfloat16* A3, long long
     g.nacc = 4;
 }
 
+// The build's own statistics (Eq. 9).  S_H is symmetric and its consumers (ridge scale, factorisation) read the
+// lower triangle only, so only tiles on or below the diagonal are computed; S_T is also left as the bf16 triple the
+// solver's first product reads.  precise: a small ridge coefficient amplifies the rounding of the statistics:
+// triples, six passes.  The operands are the token-contiguous copies t->XT, t->RT.
+static int gram_self_own(const Lc& lc, TcBuffers* t, int F, int n, float* S_H, bool precise, DevStatus* status) {
+    TcGemm h = plain_gemm(F, F, n, S_H, F, 1.f, nullptr, 0, false);
+    if (precise) {
+        six_pass_stats(h, t->XT, t->XT3, F, t->XT, t->XT3, F, t->ldT, n);
+    } else {
+        h.A[0] = TcMat{t->XT.hi, t->ldT, F, n}; h.B[0] = TcMat{t->XT.hi, t->ldT, F, n};
+        h.A[1] = TcMat{t->XT.hi, t->ldT, F, n}; h.B[1] = TcMat{t->XT.lo, t->ldT, F, n};
+        h.A[2] = TcMat{t->XT.lo, t->ldT, F, n}; h.B[2] = TcMat{t->XT.hi, t->ldT, F, n};
+        h.npass = 3;
+    }
+    h.lower_only = true;
+    return gemm_tc(lc, h, status);
+}
+static int gram_cross_own(const Lc& lc, TcBuffers* t, int F, int dm, int n, float* S_T, bool precise, DevStatus* status) {
+    TcGemm g = plain_gemm(dm, F, n, S_T, F, 1.f, nullptr, 0, false);
+    if (precise) {
+        six_pass_stats(g, t->RT, t->RT3, dm, t->XT, t->XT3, F, t->ldT, n);
+    } else {
+        g.A[0] = TcMat{t->RT.hi, t->ldT, dm, n}; g.B[0] = TcMat{t->XT.hi, t->ldT, F, n};
+        g.A[1] = TcMat{t->RT.hi, t->ldT, dm, n}; g.B[1] = TcMat{t->XT.lo, t->ldT, F, n};
+        g.A[2] = TcMat{t->RT.lo, t->ldT, dm, n}; g.B[2] = TcMat{t->XT.hi, t->ldT, F, n};
+        g.npass = 3;
+    }
+    g.out[0] = t->S3[0]; g.out[1] = t->S3[1]; g.out[2] = t->S3[2]; g.ldo = F; g.nout = 3;
+    const int rc = gemm_tc(lc, g, status);
+    if (rc == PKV_OK) t->S3_ready = 1;
+    return rc;
+}
+
 void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, const float* R, int n, float* S_H,
              float* S_T, bool accumulate, DevStatus* status, bool precise) {
     const int F = d->F, dm = d->d;
     transpose_split(lc, X, n, F, t->ldT, t->XT, precise ? t->XT3 : nullptr);
     transpose_split(lc, R, n, dm, t->ldT, t->RT, precise ? t->RT3 : nullptr);
     t->S3_ready = 0;
+    if (!accumulate && S_T == t->own_S_T) {
+        gram_self_own(lc, t, F, n, S_H, precise, status);
+        gram_cross_own(lc, t, F, dm, n, S_T, precise, status);
+        return;
+    }
     if (precise) {
-        // a small ridge coefficient amplifies the rounding of the statistics: triples, six passes
-        const bool own = !accumulate && S_T == t->own_S_T;
         TcGemm h = plain_gemm(F, F, n, S_H, F, 1.f, nullptr, 0, accumulate);
         six_pass_stats(h, t->XT, t->XT3, F, t->XT, t->XT3, F, t->ldT, n);
-        h.lower_only = own;
         gemm_tc(lc, h, status);
         TcGemm g = plain_gemm(dm, F, n, S_T, F, 1.f, nullptr, 0, accumulate);
         six_pass_stats(g, t->RT, t->RT3, dm, t->XT, t->XT3, F, t->ldT, n);
-        if (own) { g.out[0] = t->S3[0]; g.out[1] = t->S3[1]; g.out[2] = t->S3[2]; g.ldo = F; g.nout = 3; }
-        if (gemm_tc(lc, g, status) == PKV_OK && own) t->S3_ready = 1;
-        return;
-    }
-    if (!accumulate && S_T == t->own_S_T) {
-        // the build's own statistics: S_H is symmetric and its consumers (ridge scale, factorisation)
-        // read the lower triangle only, so only tiles on or below the diagonal are computed
-        TcGemm h = plain_gemm(F, F, n, S_H, F, 1.f, nullptr, 0, false);
-        h.A[0] = TcMat{t->XT.hi, t->ldT, F, n}; h.B[0] = TcMat{t->XT.hi, t->ldT, F, n};
-        h.A[1] = TcMat{t->XT.hi, t->ldT, F, n}; h.B[1] = TcMat{t->XT.lo, t->ldT, F, n};
-        h.A[2] = TcMat{t->XT.lo, t->ldT, F, n}; h.B[2] = TcMat{t->XT.hi, t->ldT, F, n};
-        h.npass = 3;
-        h.lower_only = true;
-        gemm_tc(lc, h, status);
-        // the build's own statistics: also leave the bf16 triple of S_T for the solver's first product
-        TcGemm g = plain_gemm(dm, F, n, S_T, F, 1.f, nullptr, 0, false);
-        g.A[0] = TcMat{t->RT.hi, t->ldT, dm, n}; g.B[0] = TcMat{t->XT.hi, t->ldT, F, n};
-        g.A[1] = TcMat{t->RT.hi, t->ldT, dm, n}; g.B[1] = TcMat{t->XT.lo, t->ldT, F, n};
-        g.A[2] = TcMat{t->RT.lo, t->ldT, dm, n}; g.B[2] = TcMat{t->XT.hi, t->ldT, F, n};
-        g.npass = 3;
-        g.out[0] = t->S3[0]; g.out[1] = t->S3[1]; g.out[2] = t->S3[2]; g.ldo = F; g.nout = 3;
-        if (gemm_tc(lc, g, status) == PKV_OK) t->S3_ready = 1;
+        gemm_tc(lc, g, status);
         return;
     }
     gemm_pair_pair(lc, t->XT, t->ldT, t->XT, t->ldT, S_H, F, F, F, n, 1.f, nullptr, 0, accumulate, status);
     gemm_pair_pair(lc, t->RT, t->ldT, t->XT, t->ldT, S_T, F, dm, F, n, 1.f, nullptr, 0, accumulate, status);
+}
+
+static bool side_stream_on() {
+    static const bool v = [] { const char* e = getenv("PKV_SIDE_STREAM"); return !e || atoi(e) != 0; }();
+    return v;
+}
+
+// S6 (targets, Eq. 5) and S7 (statistics, Eq. 9) at the end of a forward.  Only S_H is needed to start the
+// factorisation, so where the build's own solve follows (not the dual form, not a streamed accumulation, no stage
+// marks) the caller's stream makes the student features' token-contiguous copy and S_H, and everything that involves
+// the targets - T = dh Wdown^T + dz, its norm, its copy, S_T - goes to the side stream: the solve picks it up at its
+// last two products.
+static int targets_and_stats(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a, bool accumulate) {
+    const int N = a.N, d = D->d, F = D->F;
+    DevStatus* st = a.status;
+    const bool precise = a.precise_stats != 0;
+    int rc;
+    t->own_S_T = a.S_T;
+    if (!side_stream_on() || !t->side || a.ev || a.dual || accumulate) {
+        if ((rc = gemm_act_weight(lc, t->dh, F, a.w->Wdown, F, a.R, d, N, d, F, 1.f, a.dz, d, st))) return rc;
+        sumsq(lc, a.R, (int64_t)N * d, &st->t_fro2);
+        mark(a, lc, 6);
+        if (a.dual) transpose_split(lc, a.hC, N, F, t->ldT, t->XT);
+        else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, accumulate, st, precise);
+        mark(a, lc, 7);
+        return PKV_OK;
+    }
+    t->S3_ready = 0;
+    transpose_split(lc, a.hC, N, F, t->ldT, t->XT, precise ? t->XT3 : nullptr);
+    cudaEventRecord(t->evSide, lc.st);
+    cudaStreamWaitEvent(t->side, t->evSide, 0);
+    const Lc ls{t->side, lc.launches, lc.map_cache};
+    rc = gemm_act_weight(ls, t->dh, F, a.w->Wdown, F, a.R, d, N, d, F, 1.f, a.dz, d, st);
+    if (rc == PKV_OK) {
+        sumsq(ls, a.R, (int64_t)N * d, &st->t_fro2);
+        transpose_split(ls, a.R, N, d, t->ldT, t->RT, precise ? t->RT3 : nullptr);
+        rc = gram_cross_own(ls, t, F, d, N, a.S_T, precise, st);
+    }
+    // recorded in every case, so that the solve's wait ends
+    cudaEventRecord(t->solve.st_ready, t->side);
+    t->S_T_async = 1;
+    t->next_async = 0;
+    if (rc != PKV_OK) return rc;
+    return gram_self_own(lc, t, F, N, a.S_H, precise, st);
+}
+
+bool tc_teacher_next_async(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const void* Wdown, const float* zF,
+                           float* xF_next, DevStatus* status) {
+    if (!t->S_T_async) return false;
+    const Lc ls{t->side, lc.launches, lc.map_cache};
+    cudaStreamWaitEvent(t->side, t->solve.st_ready, 0);      // the teacher half may have run on another stream
+    gemm_act_weight(ls, t->hF, D->F, Wdown, D->F, xF_next, D->d, N, D->d, D->F, 1.f, zF, D->d, status);
+    cudaEventRecord(t->evSideDone, t->side);
+    t->next_async = 1;
+    return true;
+}
+
+static bool build_trace_on() {
+    static const bool v = getenv("PKV_BUILD_TRACE") != nullptr;
+    return v;
+}
+void tc_build_trace_mark(TcBuffers* t, int i, cudaStream_t st) {
+    if (!build_trace_on()) return;
+    if (!t->tr[0])
+        for (cudaEvent_t& e : t->tr) cudaEventCreate(&e);
+    cudaEventRecord(t->tr[i], st);
+}
+void tc_build_trace_print(TcBuffers* t) {
+    if (!build_trace_on() || !t->tr[0]) return;
+    float ms[6] = {};
+    for (int i = 1; i < 6; ++i)
+        if (cudaEventElapsedTime(&ms[i], t->tr[0], t->tr[i]) != cudaSuccess) { cudaGetLastError(); ms[i] = -1.f; }
+    fprintf(stderr, "build timeline (ms from the start): S_H %.3f | teacher attention %.3f | S_T %.3f | solve %.3f | end %.3f\n",
+            ms[1], ms[2], ms[3], ms[4], ms[5]);
+}
+
+void tc_side_quiesce(TcBuffers* t) {
+    if (t->fast) cudaStreamSynchronize(t->fast);
+    if (t->side) cudaStreamSynchronize(t->side);
+    t->S_T_async = t->next_async = 0;
+}
+
+void tc_side_join(const Lc& lc, TcBuffers* t) {
+    if (t->next_async) cudaStreamWaitEvent(lc.st, t->evSideDone, 0);
+    t->next_async = 0;
 }
 
 // The statistics of Eq. 9 with caller-supplied operand buffers (used by the entry point that owns a
@@ -418,8 +570,10 @@ int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
 void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int F, int d, float* dW, float lam0,
                     int mode, DevStatus* status) {
     const bool well = tc_well_conditioned(lam0, mode);
-    tc_ridge_solve_impl(lc, &t->solve, S, S_T, F, F, d, dW, well, false, status, &t->dW, t->S3_ready ? t->S3 : nullptr);
+    tc_ridge_solve_impl(lc, &t->solve, S, S_T, F, F, d, dW, well, false, status, &t->dW, t->S3_ready ? t->S3 : nullptr,
+                        t->S_T_async != 0);
     t->S3_ready = 0;
+    t->S_T_async = 0;
 }
 
 static void fill_attn(AttnArgs& at, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a, int mode) {
@@ -531,16 +685,9 @@ int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
         lc.count();
     }
     mark(a, lc, 5);
-    // S6: T = dh Wdown^T + dz   (Eq. 5)
-    if ((rc = gemm_act_weight(lc, t->dh, F, w->Wdown, F, a.R, d, N, d, F, 1.f, a.dz, d, st))) return rc;
-    sumsq(lc, a.R, (int64_t)N * d, &st->t_fro2);
-    mark(a, lc, 6);
-    // S7 (Eq. 9); the dual solver only needs the token-contiguous copy of the student features
-    t->own_S_T = a.S_T;
-    if (a.dual) transpose_split(lc, a.hC, N, F, t->ldT, t->XT);
-    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, false, st, a.precise_stats != 0);
-    mark(a, lc, 7);
-    return PKV_OK;
+    // S6: T = dh Wdown^T + dz (Eq. 5); S7 (Eq. 9); the dual solver only needs the token-contiguous copy of the
+    // student features
+    return targets_and_stats(lc, t, D, a, false);
 }
 
 int tc_student_propagate(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a, const float* dW,
@@ -641,16 +788,130 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
         lc.count();
     }
     mark(a, lc, 5);
-    // S6: T = dh Wdown^T + dz   (Eq. 5)
-    if ((rc = gemm_act_weight(lc, t->dh, F, w->Wdown, F, a.R, d, N, d, F, 1.f, a.dz, d, st))) return rc;
-    sumsq(lc, a.R, (int64_t)N * d, &st->t_fro2);
-    mark(a, lc, 6);
-    // S7 (Eq. 9); the dual solver only needs the token-contiguous copy of the student features
+    // S6: T = dh Wdown^T + dz (Eq. 5); S7 (Eq. 9)
+    return targets_and_stats(lc, t, D, a, a.accumulate_stats != 0);
+}
+
+static bool build_overlap_on() {
+    static const bool v = [] { const char* e = getenv("PKV_BUILD_OVERLAP"); return !e || atoi(e) != 0; }();
+    return v;
+}
+
+bool tc_forward_overlapped_applies(const TcBuffers* t, const TcForwardArgs& a) {
+    return side_stream_on() && build_overlap_on() && t->side && t->fast && !a.ev && !a.dual && !a.accumulate_stats;
+}
+
+// One block, student first.  The ridge solve needs S_H = H'^T H' (student only) for its long, latency-bound
+// factorisation and S_T only for its last two products, and the teacher half of Algorithm 1 is about two thirds of the
+// forward's work.  So: the student half and S_H run first on a high-priority stream and the caller's stream goes on to
+// the solve; the teacher half, the differences, the targets (Eq. 5) and S_T (Eq. 9) run on the low-priority side stream
+// in the SMs the factorisation leaves idle.  The differences are still formed in fp32 before any rounding: the
+// attention combine of the teacher subtracts the student's aC, dz = (xF - xC) + dA Wo^T, the teacher's residual state
+// is zF = zC + dz (so that zF - zC is dz exactly), dh = hF - hC from the two fp32 activations.
+// Events: evq[0] set-up done (caller's stream -> student); evq[1] aC, evq[2] zC, evq[3] hC (student -> teacher);
+// evSide token-contiguous student features; evq[4] S_H (student -> caller's stream and -> the teacher's start);
+// solve.st_ready S_T.  teacher_stream is normally a stream of an SM partition, so that the teacher's long-running
+// CTAs cannot occupy every SM while the factorisation's short dependent kernels wait for a slot.
+int tc_forward_overlapped(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArgs& a,
+                          cudaStream_t teacher_stream) {
+    const int N = a.N, d = D->d, F = D->F, hd = D->hd;
+    const int Dq = D->Hq * hd, Dkv = D->Hkv * hd, QKV = Dq + 2 * Dkv;
+    const pkv_block_weights* w = a.w;
+    DevStatus* st = a.status;
+    const bool precise = a.precise_stats != 0;
+    int rc;
+    tc_build_trace_mark(t, 0, lc.st);
+    rope_table(lc, a.tok_cs, N, hd, a.pos0, D->rope_theta, a.rope_tab);
+    cudaEventRecord(t->evq[0], lc.st);
+    cudaStreamWaitEvent(t->fast, t->evq[0], 0);
+    cudaStream_t ts = teacher_stream ? teacher_stream : t->side;
+    const Lc lf{t->fast, lc.launches, lc.map_cache}, ls{ts, lc.launches, lc.map_cache};
+    const void* const Wqkv[3] = {w->Wq, w->Wk, w->Wv};
+    const int wqkv[3] = {Dq, Dkv, Dkv};
+    const void* const Wgu[2] = {w->Wgate, w->Wup};
+    const int wgu[2] = {F, F};
     t->own_S_T = a.S_T;
-    if (a.dual) transpose_split(lc, a.hC, N, F, t->ldT, t->XT);
-    else tc_gram(lc, t, D, a.hC, a.R, N, a.S_H, a.S_T, a.accumulate_stats != 0, st, a.precise_stats != 0);
-    mark(a, lc, 7);
-    return PKV_OK;
+    t->S3_ready = 0;
+
+    // ---- student half (rows [N,2N) of the stacked buffers) and S_H ----
+    {
+        const size_t uo = (size_t)N * d;
+        Pair uS{t->u.hi + uo, t->u.lo + uo};
+        k_rmsnorm_split<<<N, 256, 0, lf.st>>>(a.xC, a.xC, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, N);
+        lf.count();
+        if ((rc = gemm_act_weights(lf, uS, d, Wqkv, wqkv, 3, d, t->qkv + (size_t)N * QKV, QKV, N, d, st))) return rc;
+        AttnArgs at{};
+        fill_attn(at, t, D, a, 2);
+        at.student_first = 1;
+        if ((rc = attention_tc(lf, t, D, at, a.rope_tab, st))) return rc;
+        cudaEventRecord(t->evq[1], lf.st);
+        Pair aS{t->a.hi + (size_t)N * Dq, t->a.lo + (size_t)N * Dq};
+        if ((rc = gemm_act_weight(lf, aS, Dq, w->Wo, Dq, t->o + uo, d, N, d, Dq, 1.f, nullptr, 0, st))) return rc;
+        k_oproj_teacher<<<(unsigned)((uo + 255) / 256), 256, 0, lf.st>>>(a.xC, t->o + uo, uo, a.zC);      // zC = xC + aC Wo^T
+        lf.count();
+        cudaEventRecord(t->evq[2], lf.st);
+        k_rmsnorm_split<<<N, 256, 0, lf.st>>>(a.zC, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, N);
+        lf.count();
+        float* guS = t->gu + (size_t)N * 2 * F;
+        if ((rc = gemm_act_weights(lf, uS, d, Wgu, wgu, 2, d, guS, 2 * F, N, d, st))) return rc;
+        const size_t n = (size_t)N * F;
+        k_swiglu_teacher<<<(unsigned)((n + 255) / 256), 256, 0, lf.st>>>(guS, N, F, a.hC, t->hC);
+        lf.count();
+        cudaEventRecord(t->evq[3], lf.st);
+        transpose_split(lf, a.hC, N, F, t->ldT, t->XT, precise ? t->XT3 : nullptr);
+        cudaEventRecord(t->evSide, lf.st);
+        if ((rc = gram_self_own(lf, t, F, N, a.S_H, precise, st))) return rc;
+        tc_build_trace_mark(t, 1, lf.st);
+        cudaEventRecord(t->evq[4], lf.st);
+        cudaStreamWaitEvent(lc.st, t->evq[4], 0);
+    }
+
+    // ---- teacher half (rows [0,N)), differences, targets and S_T on the side stream ----
+    {
+        // not before S_H is done: whatever share of the SMs the teacher takes earlier delays the start of the solve
+        cudaStreamWaitEvent(ls.st, t->evq[4], 0);
+        k_rmsnorm_split<<<N, 256, 0, ls.st>>>(a.xF, a.xF, N, d, w->g_attn, D->eps, t->u.hi, t->u.lo, 0);
+        ls.count();
+        rc = gemm_act_weights(ls, t->u, d, Wqkv, wqkv, 3, d, t->qkv, QKV, N, d, st);
+        if (rc == PKV_OK) {
+            AttnArgs at{};
+            fill_attn(at, t, D, a, 1);
+            at.student_first = 1;
+            at.combine_wait = t->evq[1];
+            rc = attention_tc(ls, t, D, at, a.rope_tab, st);
+            tc_build_trace_mark(t, 2, ls.st);
+        }
+        if (rc == PKV_OK) rc = gemm_act_weight(ls, t->a, Dq, w->Wo, Dq, t->o, d, N, d, Dq, 1.f, nullptr, 0, st);
+        if (rc == PKV_OK) {
+            const size_t n = (size_t)N * d;
+            cudaStreamWaitEvent(ls.st, t->evq[2], 0);
+            k_oproj_teacher_diff<<<(unsigned)((n + 255) / 256), 256, 0, ls.st>>>(a.xF, a.xC, t->o, a.zC, n, a.zF, a.dz);
+            ls.count();
+            k_rmsnorm_split<<<N, 256, 0, ls.st>>>(a.zF, a.zF, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, 0);
+            ls.count();
+            rc = gemm_act_weights(ls, t->u, d, Wgu, wgu, 2, d, t->gu, 2 * F, N, d, st);
+        }
+        if (rc == PKV_OK) {
+            const size_t n = (size_t)N * F;
+            cudaStreamWaitEvent(ls.st, t->evq[3], 0);
+            k_swiglu_teacher_diff<<<(unsigned)((n + 255) / 256), 256, 0, ls.st>>>(t->gu, N, F, a.hC, a.hF, t->hF, t->dh);
+            ls.count();
+            // S6 (Eq. 5), S_T (Eq. 9)
+            rc = gemm_act_weight(ls, t->dh, F, w->Wdown, F, a.R, d, N, d, F, 1.f, a.dz, d, st);
+        }
+        if (rc == PKV_OK) {
+            sumsq(ls, a.R, (int64_t)N * d, &st->t_fro2);
+            transpose_split(ls, a.R, N, d, t->ldT, t->RT, precise ? t->RT3 : nullptr);
+            cudaStreamWaitEvent(ls.st, t->evSide, 0);
+            rc = gram_cross_own(ls, t, F, d, N, a.S_T, precise, st);
+        }
+        tc_build_trace_mark(t, 3, ls.st);
+        // recorded in every case, so that the solve's wait ends
+        cudaEventRecord(t->solve.st_ready, ls.st);
+        t->S_T_async = 1;
+        t->next_async = 0;
+    }
+    return rc;
 }
 
 void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* D, int N, const void* Wdown, const float* dW,

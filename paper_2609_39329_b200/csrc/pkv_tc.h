@@ -70,7 +70,7 @@ constexpr int kSolveGraphs = 4;
 struct SolveGraph {
     const float *G, *S_T;
     int n, ld, d;
-    bool well, triple, aligned;
+    bool well, triple, aligned, wait;
     const void *pair_hi, *pair_lo;
     cudaGraphExec_t exec;
     int64_t launches;
@@ -90,6 +90,7 @@ struct TcSolveBuffers {
     cudaStream_t bulk2;    // helper stream: the rest of every trailing update
     cudaStream_t aux2;     // helper stream: the doubling levels of the inverse beside the factorisation
     cudaEvent_t ev[kSolveEvents];
+    cudaEvent_t st_ready;  // recorded by a caller that produces S_T on another stream beside the factorisation
     CUtensorMap chainP[3], chainX[3];   // tensor maps of the chain kernel's operands, valid for (chain_n, chain_ld)
     int chain_n, chain_ld;
     long long* stamps;     // phase marks of the chain kernel (profiling aid)
@@ -107,7 +108,8 @@ int tc_solve_init(TcSolveBuffers* t);
 // ld: row stride of S, S_T, dW (multiple of 8).  zero_fill: ld differs from the previous call's.
 int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
                         float* dW, bool well_conditioned, bool zero_fill, DevStatus* status, const Pair* dW_pair,
-                        __nv_bfloat16* const* S_T_triple);   // optional: dW's bf16 pair out; S_T already split
+                        __nv_bfloat16* const* S_T_triple,    // optional: dW's bf16 pair out; S_T already split
+                        bool wait_S_T = false);              // S_T is complete only once t->st_ready has fired
 
 int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const float* A, const float* B, int M, int N,
                     int K, float alpha, float* C, bool accumulate, int passes, int nacc, DevStatus* status,
@@ -146,6 +148,18 @@ struct TcBuffers {
     __nv_bfloat16* S3[3];   // bf16 triple of the build's own S_T (aliases solve.S2), written by the Gram epilogue
     int S3_ready;
     const float* own_S_T;
+    // Side stream: S_T needs the targets, the factorisation of S_H + lambda I does not.  The target product (S6),
+    // the cross statistics S_T and the teacher's next state are issued on `side` (lowest priority) and run in the
+    // SMs the latency-bound factorisation leaves idle; the solve waits for solve.st_ready before its first use of
+    // S_T.  S_T_async: such work is in flight for the next solve; next_async: the teacher's next state as well.
+    cudaStream_t side;
+    cudaEvent_t evSide, evSideDone;
+    int S_T_async, next_async;
+    // Single-block build with the whole teacher half beside the solve (tc_forward_overlapped): the student half runs
+    // first, on `fast` (high priority), the teacher half on `side`; evq orders the two (see there).
+    cudaStream_t fast;
+    cudaEvent_t evq[6];
+    cudaEvent_t tr[6];  // PKV_BUILD_TRACE=1: timed marks (start, S_H, teacher attention, S_T, solve, end), else null
     // dual (N x N) solver: its own work arrays and the fp32 staging of G_d, T^T and Y
     int dual_enabled, dual_ld_prev;
     TcSolveBuffers dual;
@@ -192,6 +206,13 @@ int tc_dual_solve(const Lc& lc, TcBuffers* t, const pkv_dims* d, int N, const fl
 int tc_init(TcBuffers* t, const pkv_dims* d);
 void tc_destroy(TcBuffers* t);
 int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a);
+// Same results as tc_forward up to rounding, scheduled for one block with nothing else to overlap: student half and
+// S_H first, so that the factorisation can start; teacher half, targets and S_T on the side stream beside it.
+// Returns false (nothing issued) where that schedule does not apply (stage marks, dual form, accumulation, switched
+// off by PKV_SIDE_STREAM=0 or PKV_BUILD_OVERLAP=0).
+bool tc_forward_overlapped_applies(const TcBuffers* t, const TcForwardArgs& a);
+int tc_forward_overlapped(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a,
+                          cudaStream_t teacher_stream);   // stream of the teacher half (nullptr: the side stream)
 int tc_teacher_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a, float* xF_next);
 int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a);
 int tc_attention(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& a, DevStatus* status);
@@ -209,6 +230,16 @@ void tc_ridge_solve(const Lc& lc, TcBuffers* t, float* S, const float* S_T, int 
                     int mode, DevStatus* status);
 void tc_next_states(const Lc& lc, TcBuffers* t, const pkv_dims* d, int N, const void* Wdown, const float* dW,
                     const float* zF, const float* R, float* xF_next, float* D, DevStatus* status);
+// xF_next = zF + hF Wdown^T on the side stream (only while S_T_async is set: returns false otherwise, nothing issued);
+// tc_side_join makes lc.st wait for it.
+bool tc_teacher_next_async(const Lc& lc, TcBuffers* t, const pkv_dims* d, int N, const void* Wdown, const float* zF,
+                           float* xF_next, DevStatus* status);
+void tc_side_join(const Lc& lc, TcBuffers* t);
+// after a failed issue: waits (host) for whatever the internal streams still hold
+void tc_side_quiesce(TcBuffers* t);
+// PKV_BUILD_TRACE=1: mark i on a stream; tc_build_trace_print after the call's synchronisation
+void tc_build_trace_mark(TcBuffers* t, int i, cudaStream_t st);
+void tc_build_trace_print(TcBuffers* t);
 // Student block re-run with the patched down projection (Algorithm 1, student propagation):
 // xC_next = z' + (W + dW) h' for the tokens in a.xC against the compact cache.  zero_nd: scratch [N][d].
 int tc_student_propagate(const Lc& lc, TcBuffers* t, const pkv_dims* d, const TcForwardArgs& a, const float* dW,

@@ -863,6 +863,7 @@ int tc_solve_init(TcSolveBuffers* t) {
     if (cudaStreamCreateWithPriority(&t->bulk2, cudaStreamNonBlocking, mid) != cudaSuccess) return PKV_ERR_CUDA;
     if (cudaStreamCreateWithPriority(&t->aux2, cudaStreamNonBlocking, least) != cudaSuccess) return PKV_ERR_CUDA;
     if (cudaStreamCreateWithFlags(&t->origin, cudaStreamNonBlocking) != cudaSuccess) return PKV_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&t->st_ready, cudaEventDisableTiming) != cudaSuccess) return PKV_ERR_CUDA;
     t->n_graphs = 0;
     t->graph_off = 0;
     t->graph_clock = 0;
@@ -898,6 +899,10 @@ void tc_solve_destroy(TcSolveBuffers* t) {
             cudaEventDestroy(t->ev[i]);
             t->ev[i] = nullptr;
         }
+    if (t->st_ready) {
+        cudaEventDestroy(t->st_ready);
+        t->st_ready = nullptr;
+    }
 }
 
 static int launch_chain(cudaStream_t st, const ChainParams& cp) {
@@ -929,7 +934,7 @@ static bool solve_trace() {
 // the address being read on the device from *dW_ind (the form a captured graph replays with another destination).
 static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
                       float* dW, float* const* dW_ind, bool well_conditioned, bool zero_fill,
-                      DevStatus* status, const Pair* dW_pair, __nv_bfloat16* const* S_T_triple) {
+                      DevStatus* status, const Pair* dW_pair, __nv_bfloat16* const* S_T_triple, bool wait_S_T) {
     const int F = n;      // dimension of the system; ld is the row stride of G, S_T, dW and of every n x n work array
     const int nblk = (F + PB - 1) / PB;
     Trip L3{{t->L3[0], t->L3[1], t->L3[2]}}, X3{{t->X3[0], t->X3[1], t->X3[2]}}, XT3{{t->XT3[0], t->XT3[1], t->XT3[2]}};
@@ -1152,6 +1157,10 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
     // ---- 3. dW = (S_T X^T) X ----
     // The rounding of these two products is amplified by cond(L): pairs (2^-16, three passes) when
     // the ridge keeps G well conditioned, triples (2^-24, six passes) otherwise.
+    // S_T produced on another stream beside the factorisation: its event was recorded (by the host) before this
+    // solve was issued; in a captured solve the wait becomes an event-wait node on that same event object
+    if (wait_S_T && cudaStreamWaitEvent(lc.st, t->st_ready, dW_ind ? cudaEventWaitExternal : 0) != cudaSuccess)
+        return PKV_ERR_CUDA;
     if (!S_T_triple) launch_split3(lc, S_T, ld, d, F, S2, ld, nsp);      // else: S2 already holds the triple
     {
         TcGemm g{};
@@ -1195,7 +1204,18 @@ __global__ void k_solve_begin(float** slot, float* dW, DevStatus* gstatus, const
     }
 }
 __global__ void k_solve_end(DevStatus* status, const DevStatus* gstatus) {
-    if (threadIdx.x == 0) *status = *gstatus;
+    if (threadIdx.x == 0) {
+        DevStatus s = *gstatus;
+        // what another stream put into the caller's word while the solve ran (the targets' norm, a raised code):
+        // the solve itself never touches t_fro2
+        s.t_fro2 = status->t_fro2;
+        if (s.code == 0 && status->code != 0) {
+            s.code = status->code;
+            s.info0 = status->info0;
+            s.info1 = status->info1;
+        }
+        *status = s;
+    }
 }
 
 // The solve is some hundreds of small dependent launches on four streams: issued one by one they cost the host
@@ -1206,16 +1226,16 @@ __global__ void k_solve_end(DevStatus* status, const DevStatus* gstatus) {
 // phase trace, a changed row stride or any failure to capture select the launch-by-launch path.
 int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
                         float* dW, bool well_conditioned, bool zero_fill, DevStatus* status, const Pair* dW_pair,
-                        __nv_bfloat16* const* S_T_triple) {
+                        __nv_bfloat16* const* S_T_triple, bool wait_S_T) {
     static const bool graphs_on = [] { const char* e = getenv("PKV_SOLVE_GRAPH"); return !e || atoi(e) != 0; }();
     if (!graphs_on || t->graph_off || solve_trace() || zero_fill)
-        return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple);
+        return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple, wait_S_T);
     const bool aligned = ((uintptr_t)dW & 15) == 0;
     SolveGraph* e = nullptr;
     for (int i = 0; i < t->n_graphs; ++i) {
         SolveGraph& c = t->graphs[i];
         if (c.G == G && c.S_T == S_T && c.n == n && c.ld == ld && c.d == d && c.well == well_conditioned &&
-            c.triple == (S_T_triple != nullptr) && c.aligned == aligned && c.pair_hi == (dW_pair ? dW_pair->hi : nullptr) &&
+            c.triple == (S_T_triple != nullptr) && c.aligned == aligned && c.wait == wait_S_T && c.pair_hi == (dW_pair ? dW_pair->hi : nullptr) &&
             c.pair_lo == (dW_pair ? dW_pair->lo : nullptr))
             e = &c;
     }
@@ -1226,11 +1246,11 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
         if (cudaStreamBeginCapture(t->origin, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
             cudaGetLastError();
             t->graph_off = 1;
-            return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple);
+            return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple, wait_S_T);
         }
         Lc lco{t->origin, lc.launches, lc.map_cache};
         const int rc = solve_body(lco, t, G, S_T, n, ld, d, dW, t->slot, well_conditioned, false, t->gstatus, dW_pair,
-                                  S_T_triple);
+                                  S_T_triple, wait_S_T);
         cudaGraph_t gr = nullptr;
         const cudaError_t ce = cudaStreamEndCapture(t->origin, &gr);
         cudaGraphExec_t exec = nullptr;
@@ -1241,7 +1261,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
             cudaGetLastError();
             t->graph_off = 1;
             if (lc.launches) *lc.launches = before;
-            return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple);
+            return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple, wait_S_T);
         }
         int slot = t->n_graphs;
         if (slot == kSolveGraphs) {      // evict the least recently used
@@ -1252,7 +1272,7 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
             ++t->n_graphs;
         }
         e = &t->graphs[slot];
-        *e = SolveGraph{G, S_T, n, ld, d, well_conditioned, S_T_triple != nullptr, aligned, dW_pair ? dW_pair->hi : nullptr,
+        *e = SolveGraph{G, S_T, n, ld, d, well_conditioned, S_T_triple != nullptr, aligned, wait_S_T, dW_pair ? dW_pair->hi : nullptr,
                         dW_pair ? dW_pair->lo : nullptr, exec, (lc.launches ? *lc.launches : 0) - before, 0};
     } else {
         lc.count((int)e->launches);
