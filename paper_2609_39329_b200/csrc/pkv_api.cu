@@ -809,7 +809,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         gram_simt(c, lc, b.hC, b.R, N, b.S_H, b.S_T, stats_only);
         mark(c, ST_SOLVE);
     } else {
-        pkv::TcForwardArgs fa;
+        pkv::TcForwardArgs fa{};
         fa.w = w; fa.full = full; fa.Kc = Kc; fa.Vc = Vc; fa.bias = cb->idx ? nullptr : cb->bias;
         fa.xF = ref->xF; fa.xC = ref->xC; fa.N = N; fa.pos0 = ref->pos0; fa.max_b = max_b; fa.total_kept = total;
         fa.head_off = b.head_off; fa.tok_cs = b.tok_cs; fa.rope_tab = b.rope_tab;

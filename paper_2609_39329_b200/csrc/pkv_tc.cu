@@ -115,13 +115,15 @@ __global__ void k_oproj_student(const float* __restrict__ dx, const float* __res
     zC[i] = zF[i] - dd;
 }
 
-// teacher half after the student's: dz = (xF - xC) + o[0:N] (the projection of dA), zF = zC + dz
+// teacher half after the student's: dz = (xF - xC) + o[0:N] (the projection of dA), zF = zC + dz; dx, if given, is
+// the incoming state difference carried between the blocks of a stack
 __global__ void k_oproj_teacher_diff(const float* __restrict__ xF, const float* __restrict__ xC,
-                                     const float* __restrict__ o, const float* __restrict__ zC, size_t n,
-                                     float* __restrict__ zF, float* __restrict__ dz) {
+                                     const float* __restrict__ dx, const float* __restrict__ o,
+                                     const float* __restrict__ zC, size_t n, float* __restrict__ zF,
+                                     float* __restrict__ dz) {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    float dd = (xF[i] - xC[i]) + o[i];
+    float dd = (dx ? dx[i] : xF[i] - xC[i]) + o[i];
     dz[i] = dd;
     zF[i] = zC[i] + dd;
 }
@@ -885,7 +887,7 @@ int tc_forward_overlapped(const Lc& lc, TcBuffers* t, const pkv_dims* D, const T
         if (rc == PKV_OK) {
             const size_t n = (size_t)N * d;
             cudaStreamWaitEvent(ls.st, t->evq[2], 0);
-            k_oproj_teacher_diff<<<(unsigned)((n + 255) / 256), 256, 0, ls.st>>>(a.xF, a.xC, t->o, a.zC, n, a.zF, a.dz);
+            k_oproj_teacher_diff<<<(unsigned)((n + 255) / 256), 256, 0, ls.st>>>(a.xF, a.xC, a.dx, t->o, a.zC, n, a.zF, a.dz);
             ls.count();
             k_rmsnorm_split<<<N, 256, 0, ls.st>>>(a.zF, a.zF, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, 0);
             ls.count();

@@ -73,6 +73,7 @@ struct SolveGraph {
     bool well, triple, aligned, wait;
     const void *pair_hi, *pair_lo;
     cudaGraphExec_t exec;
+    cudaGraphExec_t exec2;     // final products, where the solve waits for S_T between two graphs (else null)
     int64_t launches;
     unsigned long long used;
 };

@@ -886,7 +886,10 @@ void tc_solve_destroy(TcSolveBuffers* t) {
         cudaStreamDestroy(t->aux);
         t->aux = nullptr;
     }
-    for (int i = 0; i < t->n_graphs; ++i) cudaGraphExecDestroy(t->graphs[i].exec);
+    for (int i = 0; i < t->n_graphs; ++i) {
+        cudaGraphExecDestroy(t->graphs[i].exec);
+        if (t->graphs[i].exec2) cudaGraphExecDestroy(t->graphs[i].exec2);
+    }
     t->n_graphs = 0;
     for (cudaStream_t* st : {&t->origin, &t->bulk, &t->bulk2, &t->aux2})
         if (*st) {
@@ -934,13 +937,14 @@ static bool solve_trace() {
 // the address being read on the device from *dW_ind (the form a captured graph replays with another destination).
 static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
                       float* dW, float* const* dW_ind, bool well_conditioned, bool zero_fill,
-                      DevStatus* status, const Pair* dW_pair, __nv_bfloat16* const* S_T_triple, bool wait_S_T) {
+                      DevStatus* status, const Pair* dW_pair, __nv_bfloat16* const* S_T_triple, bool wait_S_T,
+                      int phase = 0) {      // 0: the whole solve; 1: factorisation and inverse only; 2: final products only
     const int F = n;      // dimension of the system; ld is the row stride of G, S_T, dW and of every n x n work array
     const int nblk = (F + PB - 1) / PB;
     Trip L3{{t->L3[0], t->L3[1], t->L3[2]}}, X3{{t->X3[0], t->X3[1], t->X3[2]}}, XT3{{t->XT3[0], t->XT3[1], t->XT3[2]}};
     Trip P3{{t->P3[0], t->P3[1], t->P3[2]}}, TT3{{t->TT3[0], t->TT3[1], t->TT3[2]}};
     int rc;
-    if (zero_fill) {
+    if (zero_fill && phase != 2) {
         // the row stride changed since the last call: parts of X / X^T that no kernel writes must read as zero
         for (int i = 0; i < 3; ++i) {
             cudaMemsetAsync(t->X3[i], 0, (size_t)n * ld * 2, lc.st);
@@ -1028,6 +1032,7 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
     static cudaEvent_t tev[5];      // trace mode only: stream timeline of the call
     if (trace && !tev[0]) for (auto& e : tev) cudaEventCreate(&e);
     timespec ts0{};
+    if (phase != 2) {
     if (trace) { cudaEventRecord(tev[0], lc.st); clock_gettime(CLOCK_MONOTONIC, &ts0); }
     cudaEventRecord(evFork, lc.st);
     cudaStreamWaitEvent(sA, evFork, 0);
@@ -1149,6 +1154,8 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
                 h1[8], h1[9], h1[10], h1[11], h1[12] - h1[5], h1[13] - h1[12], h1[14] - h1[13], h1[15] - h1[14]);
 
     }
+    }
+    if (phase == 1) return PKV_OK;
     // (2. X = L^{-1} was built beside the factorisation, see sC above.)  cond(L) = sqrt(cond(G)): with a
     // well-conditioned ridge matrix (a few tens) the rounding of those products (pairs: 2^-16) reaches dW
     // unamplified and three passes are enough.  The same holds for the factorisation: lambda is then of the order
@@ -1158,9 +1165,8 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
     // The rounding of these two products is amplified by cond(L): pairs (2^-16, three passes) when
     // the ridge keeps G well conditioned, triples (2^-24, six passes) otherwise.
     // S_T produced on another stream beside the factorisation: its event was recorded (by the host) before this
-    // solve was issued; in a captured solve the wait becomes an event-wait node on that same event object
-    if (wait_S_T && cudaStreamWaitEvent(lc.st, t->st_ready, dW_ind ? cudaEventWaitExternal : 0) != cudaSuccess)
-        return PKV_ERR_CUDA;
+    // solve was issued.  (A captured solve is split in two graphs at this point and waits between them.)
+    if (wait_S_T && cudaStreamWaitEvent(lc.st, t->st_ready, 0) != cudaSuccess) return PKV_ERR_CUDA;
     if (!S_T_triple) launch_split3(lc, S_T, ld, d, F, S2, ld, nsp);      // else: S2 already holds the triple
     {
         TcGemm g{};
@@ -1243,22 +1249,33 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
     lc.count();
     if (!e) {
         const int64_t before = lc.launches ? *lc.launches : 0;
-        if (cudaStreamBeginCapture(t->origin, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
-            cudaGetLastError();
-            t->graph_off = 1;
-            return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple, wait_S_T);
+        const Lc lco{t->origin, lc.launches, lc.map_cache};
+        // S_T arriving from another stream: two graphs, split where the final products begin, and an ordinary wait
+        // for the producer's event between them
+        const int n_parts = wait_S_T ? 2 : 1;
+        cudaGraphExec_t exec[2] = {nullptr, nullptr};
+        int rc = PKV_OK;
+        bool captured = true;
+        for (int part = 0; part < n_parts && captured && rc == PKV_OK; ++part) {
+            if (cudaStreamBeginCapture(t->origin, cudaStreamCaptureModeRelaxed) != cudaSuccess) {
+                captured = false;
+                break;
+            }
+            rc = solve_body(lco, t, G, S_T, n, ld, d, dW, t->slot, well_conditioned, false, t->gstatus, dW_pair, S_T_triple,
+                            false, wait_S_T ? part + 1 : 0);
+            cudaGraph_t gr = nullptr;
+            const cudaError_t ce = cudaStreamEndCapture(t->origin, &gr);
+            if (rc == PKV_OK && (ce != cudaSuccess || !gr || cudaGraphInstantiate(&exec[part], gr, 0) != cudaSuccess)) {
+                exec[part] = nullptr;
+                captured = false;
+            }
+            if (gr) cudaGraphDestroy(gr);
         }
-        Lc lco{t->origin, lc.launches, lc.map_cache};
-        const int rc = solve_body(lco, t, G, S_T, n, ld, d, dW, t->slot, well_conditioned, false, t->gstatus, dW_pair,
-                                  S_T_triple, wait_S_T);
-        cudaGraph_t gr = nullptr;
-        const cudaError_t ce = cudaStreamEndCapture(t->origin, &gr);
-        cudaGraphExec_t exec = nullptr;
-        if (rc == PKV_OK && ce == cudaSuccess && gr && cudaGraphInstantiate(&exec, gr, 0) != cudaSuccess) exec = nullptr;
-        if (gr) cudaGraphDestroy(gr);
-        if (rc != PKV_OK) { cudaGetLastError(); return rc; }
-        if (!exec) {      // capture is not available here: stay on the launch-by-launch path from now on
+        if (rc != PKV_OK || !captured) {
+            for (cudaGraphExec_t x : exec) if (x) cudaGraphExecDestroy(x);
             cudaGetLastError();
+            if (rc != PKV_OK) return rc;
+            // capture is not available here: stay on the launch-by-launch path from now on
             t->graph_off = 1;
             if (lc.launches) *lc.launches = before;
             return solve_body(lc, t, G, S_T, n, ld, d, dW, nullptr, well_conditioned, zero_fill, status, dW_pair, S_T_triple, wait_S_T);
@@ -1268,17 +1285,22 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
             slot = 0;
             for (int i = 1; i < kSolveGraphs; ++i) if (t->graphs[i].used < t->graphs[slot].used) slot = i;
             cudaGraphExecDestroy(t->graphs[slot].exec);
+            if (t->graphs[slot].exec2) cudaGraphExecDestroy(t->graphs[slot].exec2);
         } else {
             ++t->n_graphs;
         }
         e = &t->graphs[slot];
         *e = SolveGraph{G, S_T, n, ld, d, well_conditioned, S_T_triple != nullptr, aligned, wait_S_T, dW_pair ? dW_pair->hi : nullptr,
-                        dW_pair ? dW_pair->lo : nullptr, exec, (lc.launches ? *lc.launches : 0) - before, 0};
+                        dW_pair ? dW_pair->lo : nullptr, exec[0], exec[1], (lc.launches ? *lc.launches : 0) - before, 0};
     } else {
         lc.count((int)e->launches);
     }
     e->used = ++t->graph_clock;
     if (cudaGraphLaunch(e->exec, lc.st) != cudaSuccess) return PKV_ERR_CUDA;
+    if (e->exec2) {
+        if (cudaStreamWaitEvent(lc.st, t->st_ready, 0) != cudaSuccess || cudaGraphLaunch(e->exec2, lc.st) != cudaSuccess)
+            return PKV_ERR_CUDA;
+    }
     k_solve_end<<<1, 32, 0, lc.st>>>(status, t->gstatus);
     lc.count();
     if (solve_trace_graph()) {

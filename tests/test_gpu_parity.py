@@ -731,6 +731,40 @@ def test_streamed_reference_set_equals_one_call_and_the_oracle(B, engine_name, l
     ctx.close()
 
 
+def test_timed_build_uses_the_stacked_schedule_and_agrees(B):
+    """With stage timing on, a block runs teacher and student stacked on one stream (so that the stage marks mean
+    something); without, the student half runs first and the teacher half beside the solve.  Same patch either way,
+    and both against the oracle."""
+    import torch
+    cfg = small_cfg("bf16", hd=128, Hq=8, Hkv=2, d=512, F=448, L=3000, N=200, window=32, budget=300, n_obs=16)
+    lay = H.make_problem(cfg)
+    rng = np.random.default_rng(5)
+    xF = lay["x0"]
+    xC = (xF + 0.05 * rng.standard_normal(xF.shape)).astype(np.float32)
+    chunk_off = [0, 120, cfg.N]
+    ref = H.run_oracle(cfg, lay, xF, xC, chunk_off, 0.1, 0)
+    ctx = B.PkvContext(B.dims_from_config(cfg, N_max=cfg.N, b_max=max(len(k) for k in lay["kept"])), engine=B.ENGINE_AUTO)
+    w = B.to_device(lay["weights"], cfg.dtype)
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    off, idx = gen.kept_to_csr(lay["kept"])
+    idx_t = torch.from_numpy(idx).cuda()
+    tF, tC = torch.from_numpy(xF).cuda(), torch.from_numpy(xC).cuda()
+    outs = []
+    for timed in (False, True, False):
+        ctx.set_timing(timed)
+        o = ctx.build_patch(w, kv["K"], kv["V"], off, idx_t, tF, tC, chunk_off, cfg.L, 0.1, 0, True)
+        outs.append({k: (v.cpu().numpy() if hasattr(v, "cpu") else v) for k, v in o.items()})
+    ctx.close()
+    errs = [H.rel_fro(o["dW"], ref["dW"]) for o in outs]
+    cross = H.rel_fro(outs[1]["dW"], outs[0]["dW"])
+    print("untimed / timed / untimed vs oracle: %.3e %.3e %.3e; timed vs untimed %.3e" % (*errs, cross))
+    assert max(errs) <= DW_TOL and cross <= 2e-3
+    assert sum(outs[1]["stats"]["stage_ms"]) > 0 and sum(outs[0]["stats"]["stage_ms"]) == 0
+    for o in outs:
+        assert H.rel_fro(o["xF_next"], ref["xF_next"]) <= 1e-3 and H.rel_fro(o["xC_next"], ref["xC_next"]) <= 1e-3
+        np.testing.assert_allclose(o["stats"]["target_fro2"], ref["T_fro2"], rtol=2e-2)
+
+
 # ------------------------------------------------------------------ boundary
 
 _ALT_CASE = '''
@@ -746,11 +780,15 @@ print("ALT_OK %%.3e" %% e)
 '''
 
 
-@pytest.mark.parametrize("env", [{"PKV_ATTN_Q": "pair"}, {"PKV_SOLVE_GRAPH": "0"}, {"PKV_SOLVE_TRACE": "1"}])
+@pytest.mark.parametrize("env", [{"PKV_ATTN_Q": "pair"}, {"PKV_SOLVE_GRAPH": "0"}, {"PKV_SOLVE_TRACE": "1"},
+                                 {"PKV_BUILD_OVERLAP": "0"}, {"PKV_SIDE_STREAM": "0"}, {"PKV_BUILD_RESERVE_SMS": "0"},
+                                 {"PKV_BUILD_TRACE": "1"}])
 def test_alternate_paths_selected_by_environment(env):
     """Paths the environment selects at start-up, each in a process of its own on one small hd-128 block against the
     oracle: bf16 query pairs against bf16 keys (the attention path for caches outside fp16's range), the solve
-    issued launch by launch instead of replayed as a graph, and the solve's phase trace."""
+    issued launch by launch instead of replayed as a graph, the solve's phase trace, the block with teacher and
+    student stacked on one stream (no teacher half beside the solve), nothing at all beside the solve, the teacher
+    half on the stack driver's partition instead of the build's own, and the build's timeline."""
     import os
     import subprocess
     import sys
@@ -760,6 +798,8 @@ def test_alternate_paths_selected_by_environment(env):
     assert r.returncode == 0 and "ALT_OK" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
     if "PKV_SOLVE_TRACE" in env:
         assert "solve timeline" in r.stderr
+    if "PKV_BUILD_TRACE" in env:
+        assert "build timeline" in r.stderr
 
 
 def test_boundary_rejects_bad_arguments(B):
