@@ -72,6 +72,10 @@ namespace pkv {
 bool green_partition_create(int want_sms, void** gctx_out, int* got_sms) {
     const GreenApi& a = green_api();
     if (!a.ok || want_sms <= 0) return false;
+    // PKV_SM_PARTITIONS=0: ordinary streams everywhere (a profiler that cannot prepare kernels launched into a green
+    // context can still list every launch; the schedules stay the same, only the SM split is gone)
+    static const bool off = [] { const char* e = getenv("PKV_SM_PARTITIONS"); return e && atoi(e) == 0; }();
+    if (off) return false;
     int ord = 0;
     if (cudaGetDevice(&ord) != cudaSuccess) return false;
     CUdevice dev;
