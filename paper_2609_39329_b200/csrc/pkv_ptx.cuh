@@ -153,6 +153,25 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// fp16 x fp16 -> fp32: the operand format fields (bits 7-9, 10-12) zero
+__host__ __device__ constexpr uint32_t idesc_f16(int M, int N) {
+    return idesc_bf16(M, N) & ~((7u << 7) | (7u << 10));
+}
+
+// Power-of-two scale that brings an fp32 array with max|x| = m (given by its bit pattern) into fp16's upper range:
+// m * scale lies in [8192, 16384), so nothing overflows and values down to 2^-27 of the maximum keep their eleven
+// bits.  A zero or non-finite maximum gives 1.
+__device__ __forceinline__ float f16_scale_from_max(unsigned max_bits) {
+    const int e = (int)((max_bits >> 23) & 0xffu);
+    if (e < 20 || e == 255) return 1.f;                                  // (an all-but-zero array stays as it is)
+    return __uint_as_float((unsigned)(127 + 13 - (e - 127)) << 23);      // 2^(13 - floor(log2 m))
+}
+__device__ __forceinline__ float f16_inv_scale_from_max(unsigned max_bits) {
+    const int e = (int)((max_bits >> 23) & 0xffu);
+    if (e < 20 || e == 255) return 1.f;
+    return __uint_as_float((unsigned)(127 - 13 + (e - 127)) << 23);
+}
+
 // Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start
 // before its predecessor in the stream has finished; it must not touch the predecessor's results before
 // pdl_wait().  pdl_launch_dependents() lets the successor start its prologue early.  Both are no-ops for

@@ -47,6 +47,11 @@ struct TcGemm {
     bool skip_tile00;     // leave the first tile (rows and columns [0,128) of the product) alone
     bool out_col0_only;   // write the bf16 parts only for the first 128-column block of the product
     unsigned long long* stamps;   // optional device array of 16 global-timer marks (phases of the first CTA, epilogue chunks)
+    bool f16;       // the operands are fp16 (same 16-bit containers; both operands of a pass must share the type)
+    // optional: device words holding the bit pattern of max|x| of the fp32 arrays the A / B operands were made from
+    // by scaled_f16_from_max (pkv_ptx.cuh); the product is divided by the two power-of-two scales
+    const unsigned* amax_a;
+    const unsigned* amax_b;
     int nacc;       // 0/1: one fp32 accumulator; 2 or 4: the hi x hi pass of a split product is accumulated apart
                     // from the cross passes (and in several parts), which removes most of the tensor core's
                     // truncation bias from sums of same-signed terms; pass 0 must be the hi x hi pass
@@ -130,6 +135,8 @@ struct TcBuffers {
     Pair hF, hC, dh;    // [N][F]
     Pair XT;            // [F][ldT]  student features, token-contiguous
     Pair RT;            // [d][ldT]  targets, token-contiguous
+    unsigned* stat;     // [0], [1]: bit patterns of max|H'|, max|T| of the current statistics (fp16 single-pass form)
+    int stats_f16;      // the operands in XT.hi / RT.hi are scaled fp16 copies (else bf16 pairs)
     __nv_bfloat16* XT3; // third bf16 parts of XT / RT (statistics in six passes when the ridge coefficient is small)
     __nv_bfloat16* RT3;
     Pair dW;            // [d][F]

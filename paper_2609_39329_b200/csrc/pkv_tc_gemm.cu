@@ -38,6 +38,9 @@ struct alignas(64) GemmTcParams {
     float* const* C_ind;      // if set, the fp32 output base is read from this device location instead of C
     long long ldc;
     float alpha;
+    const unsigned* amax_a;   // optional power-of-two operand scales to divide out, see TcGemm
+    const unsigned* amax_b;
+    int f16;                  // fp16 operands
     const float* addend;
     long long ldadd;
     __nv_bfloat16* out[3];
@@ -193,7 +196,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16(128, BN);
+            const uint32_t idesc = p.f16 ? idesc_f16(128, BN) : idesc_bf16(128, BN);
             bool ok = true;
             uint32_t used = 0u;          // accumulators that already hold a partial sum
             uint32_t hh = 0u;            // running index of the hi x hi MMAs
@@ -235,6 +238,9 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
         }
         if (warp == 2 && lane == 0) gemm_stamp(p, 5);
         if (ok) {
+            float alpha = p.alpha;
+            if (p.amax_a) alpha *= f16_inv_scale_from_max(*p.amax_a);
+            if (p.amax_b) alpha *= f16_inv_scale_from_max(*p.amax_b);
             float* stg = staging + q * (32 * 33);
             // not unrolled: a CTA runs each chunk's code once, and a short-K tile's time is mostly instruction fetch
 #pragma unroll 1
@@ -263,7 +269,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
                 if (ncol <= 0) break;
                 float v[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = p.alpha * __uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j) v[j] = alpha * __uint_as_float(r[j]);
                 if (Cp && lane < nrows) {
                     // fp32 output: every lane owns one row; 128 contiguous bytes, loads batched ahead of stores
                     const size_t row = (size_t)(rowa0 + lane);
@@ -585,6 +591,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     p.c_row0 = g.c_row0; p.c_col0 = g.c_col0; p.c_zrow = g.c_zrow; p.c_zcol = g.c_zcol;
     p.c_rows = g.c_rows; p.c_cols = g.c_cols;
     p.C = g.C; p.C_ind = g.C_ind; p.ldc = g.ldc; p.alpha = g.alpha; p.addend = g.addend; p.ldadd = g.ldadd;
+    p.amax_a = g.amax_a; p.amax_b = g.amax_b; p.f16 = g.f16 ? 1 : 0;
     for (int i = 0; i < 3; ++i) p.out[i] = g.out[i];
     p.ldo = g.ldo; p.nout = g.nout; p.out_col_off = g.out_col_off;
     p.accumulate = g.accumulate ? 1 : 0;

@@ -731,6 +731,24 @@ def test_streamed_reference_set_equals_one_call_and_the_oracle(B, engine_name, l
     ctx.close()
 
 
+def test_statistics_survive_massive_activations(B):
+    """The build's statistics take one pass over fp16 copies scaled by a power of two from each array's maximum.
+    A few features 256 times larger than the rest (rows of Wup scaled by a power of two, so that they stay bf16
+    values) must not cost the others their bits: same tolerance against the oracle as everywhere."""
+    cfg = small_cfg("bf16", hd=128, Hq=8, Hkv=2, d=512, F=448, L=3000, N=200, window=32, budget=300, n_obs=16)
+    lay = H.make_problem(cfg)
+    w = dict(lay["weights"])
+    wu = np.array(w["Wup"], dtype=np.float32, copy=True)
+    wu[::37] *= 256.0
+    w["Wup"] = wu
+    lay = dict(lay, weights=w)
+    rng = np.random.default_rng(11)
+    xF = lay["x0"]
+    xC = (xF + 0.05 * rng.standard_normal(xF.shape)).astype(np.float32)
+    e = check_build(B, cfg, lay, xF, xC, [0, 120, cfg.N], 0.1, B.ENGINE_AUTO)
+    print("features x256: dW rel fro err %.3e" % e)
+
+
 def test_timed_build_uses_the_stacked_schedule_and_agrees(B):
     """With stage timing on, a block runs teacher and student stacked on one stream (so that the stage marks mean
     something); without, the student half runs first and the teacher half beside the solve.  Same patch either way,
@@ -782,13 +800,14 @@ print("ALT_OK %%.3e" %% e)
 
 @pytest.mark.parametrize("env", [{"PKV_ATTN_Q": "pair"}, {"PKV_SOLVE_GRAPH": "0"}, {"PKV_SOLVE_TRACE": "1"},
                                  {"PKV_BUILD_OVERLAP": "0"}, {"PKV_SIDE_STREAM": "0"}, {"PKV_BUILD_RESERVE_SMS": "0"},
-                                 {"PKV_BUILD_TRACE": "1"}])
+                                 {"PKV_BUILD_TRACE": "1"}, {"PKV_STATS_F16": "0"}])
 def test_alternate_paths_selected_by_environment(env):
     """Paths the environment selects at start-up, each in a process of its own on one small hd-128 block against the
     oracle: bf16 query pairs against bf16 keys (the attention path for caches outside fp16's range), the solve
     issued launch by launch instead of replayed as a graph, the solve's phase trace, the block with teacher and
     student stacked on one stream (no teacher half beside the solve), nothing at all beside the solve, the teacher
-    half on the stack driver's partition instead of the build's own, and the build's timeline."""
+    half on the stack driver's partition instead of the build's own, the build's timeline, and the statistics from
+    bf16 pairs in three passes instead of one scaled fp16 pass."""
     import os
     import subprocess
     import sys
