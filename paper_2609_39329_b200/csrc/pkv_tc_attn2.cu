@@ -82,6 +82,28 @@ __device__ __forceinline__ void tmem_st_wait() {
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
+// Fewer issue slots per score (the softmax warps are bound by instruction issue, not by any one pipe): the
+// subtraction of the reference maximum as one packed instruction per pair, the running maximum three inputs at a
+// time, the row sum straight from the packed bf16 pair (fp32 + bf16 -> fp32).
+__device__ __forceinline__ uint64_t pack_f32x2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void sub_f32x2(uint32_t a0, uint32_t a1, uint64_t mm, float& r0, float& r1) {
+    asm("{ .reg .b64 t; mov.b64 t, {%2, %3}; sub.f32x2 t, t, %4; mov.b64 {%0, %1}, t; }"
+        : "=f"(r0), "=f"(r1) : "r"(a0), "r"(a1), "l"(mm));
+}
+__device__ __forceinline__ float max3f(float a, uint32_t b, uint32_t c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(__uint_as_float(b)), "f"(__uint_as_float(c)));
+    return r;
+}
+__device__ __forceinline__ void add_bf16x2(float& l0, float& l1, uint32_t pk) {
+    asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; add.rn.f32.bf16 %0, lo, %0; add.rn.f32.bf16 %1, hi, %1; }"
+        : "+f"(l0), "+f"(l1) : "r"(pk));
+}
+
 __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Attn2Params p) {
     using namespace a2;
     {   // an earlier stage already failed: the call reports it.  One thread reads the status word so that the
@@ -285,11 +307,11 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
             }
             float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 128; c += 4) {
-                mx0 = fmaxf(mx0, __uint_as_float(s[c]));
-                mx1 = fmaxf(mx1, __uint_as_float(s[c + 1]));
-                mx2 = fmaxf(mx2, __uint_as_float(s[c + 2]));
-                mx3 = fmaxf(mx3, __uint_as_float(s[c + 3]));
+            for (int c = 0; c < 128; c += 8) {
+                mx0 = max3f(mx0, s[c], s[c + 1]);
+                mx1 = max3f(mx1, s[c + 2], s[c + 3]);
+                mx2 = max3f(mx2, s[c + 4], s[c + 5]);
+                mx3 = max3f(mx3, s[c + 6], s[c + 7]);
             }
             const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             // reference maximum: the exact running maximum (moved whenever the tile's maximum exceeds it)
@@ -302,16 +324,17 @@ __global__ void __launch_bounds__(320, 1) k_attn_tc2(const __grid_constant__ Att
             const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
             float l0 = 0.f, l1 = 0.f;
             // P as packed bf16 pairs, written over the first half of s[] (entry c/2 is dead by then)
+            const uint64_t mm = pack_f32x2(m_use, m_use);
 #pragma unroll
             for (int c = 0; c < 128; c += 2) {
-                const float p0 = ex2f(__uint_as_float(s[c]) - m_use);
-                const float p1 = ex2f(__uint_as_float(s[c + 1]) - m_use);
+                float x0, x1;
+                sub_f32x2(s[c], s[c + 1], mm, x0, x1);
+                const float p0 = ex2f(x0), p1 = ex2f(x1);
                 __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
                 const uint32_t pk = *reinterpret_cast<uint32_t*>(&b);
                 // the row sum uses the ROUNDED probabilities, the ones the P V product sees, so that the
                 // rounding of a dominant key cancels between numerator and denominator
-                l0 += __uint_as_float(pk << 16);
-                l1 += __uint_as_float(pk & 0xffff0000u);
+                add_bf16x2(l0, l1, pk);
                 s[c >> 1] = pk;
             }
             l = l * alpha + (l0 + l1);
