@@ -19,8 +19,13 @@
  *     states (xF, xC, next states) and dW are always fp32.
  *   - Every function returns PKV_OK (0) or a negative pkv_error; nothing throws, aborts or
  *     traps on the device.  After an error the contents of the outputs are unspecified.
- *   - Work is enqueued on the CUDA stream given at pkv_create; pkv_build_patch ends with one
- *     stream synchronisation to read the device status word, so its return code is truthful.
+ *   - Work is ordered after whatever is already queued on the CUDA stream given at pkv_create and is
+ *     complete when a call returns: pkv_build_patch and the other building calls end with one stream
+ *     synchronisation to read the device status word, so the return code is truthful.  Inside a call
+ *     the tensor-core engine also uses streams of its own (the teacher half of a block, the targets and
+ *     S_T run beside the ridge solve; the solve itself spans four streams), all forked from and joined
+ *     back into the context's stream before the call returns; none of this may be issued while the
+ *     caller's stream is being captured.
  *   - A context is not thread-safe; use one per host thread / stream.
  */
 #ifndef PKV_H_
