@@ -800,14 +800,14 @@ print("ALT_OK %%.3e" %% e)
 
 @pytest.mark.parametrize("env", [{"PKV_ATTN_Q": "pair"}, {"PKV_SOLVE_GRAPH": "0"}, {"PKV_SOLVE_TRACE": "1"},
                                  {"PKV_BUILD_OVERLAP": "0"}, {"PKV_SIDE_STREAM": "0"}, {"PKV_BUILD_RESERVE_SMS": "0"},
-                                 {"PKV_BUILD_TRACE": "1"}, {"PKV_STATS_F16": "0"}])
+                                 {"PKV_BUILD_TRACE": "1"}, {"PKV_STATS_F16": "0"}, {"PKV_SM_PARTITIONS": "0"}])
 def test_alternate_paths_selected_by_environment(env):
     """Paths the environment selects at start-up, each in a process of its own on one small hd-128 block against the
     oracle: bf16 query pairs against bf16 keys (the attention path for caches outside fp16's range), the solve
     issued launch by launch instead of replayed as a graph, the solve's phase trace, the block with teacher and
     student stacked on one stream (no teacher half beside the solve), nothing at all beside the solve, the teacher
-    half on the stack driver's partition instead of the build's own, the build's timeline, and the statistics from
-    bf16 pairs in three passes instead of one scaled fp16 pass."""
+    half on the stack driver's partition instead of the build's own, the build's timeline, the statistics from
+    bf16 pairs in three passes instead of one scaled fp16 pass, and ordinary streams in place of SM partitions."""
     import os
     import subprocess
     import sys
