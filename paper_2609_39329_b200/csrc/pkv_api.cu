@@ -831,8 +831,10 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         c->teacher_timed = 0;
         if (pkv::tc_forward_overlapped_applies(&b.tc, fa)) rc = pkv::tc_forward_overlapped(lc, &b.tc, &c->dims, fa, build_teacher_stream(c, N));
         else rc = pkv::tc_forward(lc, &b.tc, &c->dims, fa);
-        if (rc != PKV_OK) {
+        if (rc != PKV_OK) {      // issue failed half-way: let every internal stream run dry before reporting
             pkv::tc_side_quiesce(&b.tc);
+            if (c->tstream) cudaStreamSynchronize(c->tstream);
+            if (c->bstream) cudaStreamSynchronize(c->bstream);
             return rc;
         }
     }
