@@ -400,7 +400,8 @@ def run_stack(args, cfg, B, torch, dist, world, rank, local, peaks):
     work = stage_work(cfg, sum(b_list))
     dom = int(np.argmax(stage_ms))
     name, fl, by, bound = work[dom]
-    dur = stage_ms[dom] * 1e-3
+    dur_ms = s8_timed_schedule if (dom == 7 and s8_timed_schedule > 0) else stage_ms[dom]
+    dur = dur_ms * 1e-3
     fl *= cfg.n_layers
     if bound == "tensor":
         peak, unit, ach, note = peaks["bf16_tflops_sustained"], "TFLOP/s", fl / dur / 1e12, "bf16 dense, sustained, %s" % peaks["source"]
@@ -558,8 +559,16 @@ def main():
         flush.fill_(i)
         st = step()["stats"]["stage_ms"][:9]
         stage_acc = st if stage_acc is None else [a + b for a, b in zip(stage_acc, st)]
-    ctx.set_timing(False)
     stage_ms = [a / 5 for a in stage_acc]
+    # the ridge solve's interval inside the schedule that `value` is timed on (the teacher half runs beside it)
+    ctx.set_timing(2)
+    step()
+    s8_acc = 0.0
+    for i in range(5):
+        flush.fill_(i)
+        s8_acc += step()["stats"]["stage_ms"][7]
+    s8_timed_schedule = s8_acc / 5
+    ctx.set_timing(False)
     work = stage_work(cfg, sum(b_list))
     total_flops = sum(wk[1] for wk in work)
     fma = ctx.measure_fma_peak()
@@ -615,7 +624,8 @@ def main():
     # roofline of the dominant stage
     dom = int(np.argmax(stage_ms))
     name, fl, by, bound = work[dom]
-    dur = stage_ms[dom] * 1e-3
+    dur_ms = s8_timed_schedule if (dom == 7 and s8_timed_schedule > 0) else stage_ms[dom]
+    dur = dur_ms * 1e-3
     traffic = None
     if bound == "tensor":
         peak, unit, ach = peaks["bf16_tflops_sustained"], "TFLOP/s", fl / dur / 1e12
@@ -626,7 +636,9 @@ def main():
         peak_note = ("fp32 FMA rate measured in this run (register-resident FMA kernel, CUDA events); the stage stands "
                      "for fp32 arithmetic but runs as multi-pass tensor-core products plus a chain of %d single-CTA factor "
                      "kernels, one per 128 columns: it is bound by that chain's latency (%.1f us per step if the whole stage "
-                     "were chain), not by FMA throughput" % (nsteps, stage_ms[dom] * 1e3 / nsteps))
+                     "were chain), not by FMA throughput; the stage is timed inside the schedule of `value`, with the "
+                     "teacher half running beside it (%.3f ms; %.3f ms with nothing beside it, stacked schedule)"
+                     % (nsteps, dur_ms * 1e3 / nsteps, dur_ms, stage_ms[dom]))
         if cfg.cfg_id == 2:
             traffic = SOLVE_STAGE_TRAFFIC_CONFIG2
     else:
@@ -634,7 +646,8 @@ def main():
         peak_note = "HBM copy, %s" % peaks["source"]
     roofline = {"kernel": name + " (stage: k_chain128 chain + k_gemm_tc products)" if bound == "alu" else name,
                 "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                "traffic": traffic, "peak_note": peak_note, "stage_ms": stage_ms[dom]}
+                "traffic": traffic, "peak_note": peak_note, "stage_ms": dur_ms,
+                "stage_ms_stacked_schedule": stage_ms[dom]}
     stages = [{"stage": wk[0], "ms": round(t, 4), "algorithmic_tflops": (wk[1] / (t * 1e-3) / 1e12) if t > 0 else None}
               for wk, t in zip(work, stage_ms)]
     tensor_flops = sum(wk[1] for wk in work if wk[3] == "tensor")

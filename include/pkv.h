@@ -344,7 +344,9 @@ int pkv_fp32_product(pkv_ctx* ctx, const float* A, const float* B, int32_t M, in
  * the context stays usable.  Nothing faults, traps or spins without a limit. */
 int pkv_selftest_bounded_wait(pkv_ctx* ctx, int32_t* site);
 
-/* Enable (1) / disable (0) per-stage CUDA-event timing into pkv_stats.stage_ms. */
+/* Per-stage CUDA-event timing into pkv_stats.stage_ms.  0: off.  1: every stage; a block then runs teacher and student
+ * stacked on one stream and a stack block by block, so that every stage has an interval of its own.  2: only the ridge
+ * solve's interval (stage_ms[7]) on the caller's stream, without changing the schedule. */
 int pkv_set_timing(pkv_ctx* ctx, int on);
 
 /* pkv_build_stack scheduling: 0 = default (teacher run ahead where it applies), 1 = strictly block by block on

@@ -252,8 +252,9 @@ class PkvContext:
         rc = self.L.pkv_selftest_bounded_wait(self.h, C.byref(site))
         return int(rc), int(site.value)
 
-    def set_timing(self, on: bool):
-        self.L.pkv_set_timing(self.h, 1 if on else 0)
+    def set_timing(self, on):
+        """False/0: off; True/1: every stage (stacked schedule); 2: the solve's interval only, default schedule."""
+        self.L.pkv_set_timing(self.h, 2 if on == 2 else (1 if on else 0))
 
     def stage_names(self) -> List[str]:
         return [self.L.pkv_stage_name(i).decode() for i in range(9)]

@@ -481,7 +481,7 @@ extern "C" int pkv_selftest_bounded_wait(pkv_ctx* c, int32_t* site) {
 
 extern "C" int pkv_set_timing(pkv_ctx* c, int on) {
     if (!c) return PKV_ERR_INVALID_ARG;
-    c->timing = on ? 1 : 0;
+    c->timing = (on == 2) ? 2 : (on ? 1 : 0);
     return PKV_OK;
 }
 
@@ -528,7 +528,7 @@ static int cuda_fail(pkv_ctx* c, cudaError_t e, const char* where) {
 }
 
 static void mark(pkv_ctx* c, int i) {
-    if (c->timing) cudaEventRecord(c->ev[i], c->st);
+    if (c->timing == 1 || (c->timing == 2 && (i == ST_SOLVE || i == ST_NEXT))) cudaEventRecord(c->ev[i], c->st);
 }
 
 static int check_compressed(const pkv_ctx* c, const pkv_kv_compressed* cb, int* total, int* max_b) {
@@ -625,7 +625,9 @@ static int end_call(pkv_ctx* c, pkv_stats* stats, const int32_t* head_off) {
             stats->err_info[1] = s.info1;
         }
         for (int i = 0; i < 12; ++i) stats->stage_ms[i] = 0.f;
-        if (c->timing) {
+        if (c->timing == 2) {      // the solve's interval on the caller's stream, default schedule
+            cudaEventElapsedTime(&stats->stage_ms[ST_SOLVE], c->ev[ST_SOLVE], c->ev[ST_NEXT]);
+        } else if (c->timing) {
             for (int i = 0; i < ST_COUNT; ++i) cudaEventElapsedTime(&stats->stage_ms[i], c->ev[i], c->ev[i + 1]);
             if (c->teacher_timed) {
                 // the teacher half ran first, inside the interval the student's marks call "S1-S2":
@@ -826,7 +828,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         fa.precise_stats = pkv::tc_well_conditioned(lambda, mode) ? 0 : 1;
         fa.accumulate_stats = stats_only ? 1 : 0;
         fa.part_m = b.part_m; fa.part_l = b.part_l; fa.part_O = b.part_O;
-        fa.ev = c->timing ? c->ev : nullptr;
+        fa.ev = (c->timing == 1) ? c->ev : nullptr;
         fa.evT = nullptr;
         c->teacher_timed = 0;
         if (pkv::tc_forward_overlapped_applies(&b.tc, fa)) rc = pkv::tc_forward_overlapped(lc, &b.tc, &c->dims, fa, build_teacher_stream(c, N));
@@ -858,6 +860,7 @@ static int build_patch_impl(pkv_ctx* c, const pkv_block_weights* w, const pkv_kv
         sumsq(lc, dW, (int64_t)d * F, &b.status->dw_fro2);
     } else {
         // the teacher's next state does not depend on the patch: beside the solve where the side stream is in use
+        if (c->timing == 2) mark(c, ST_SOLVE);
         if (next && c->engine != PKV_ENGINE_SIMT)
             next_async = pkv::tc_teacher_next_async(lc, &b.tc, &c->dims, N, w->Wdown, b.zF, next->xF_next, b.status);
         solve_stage(c, lc, b.S_H, b.S_T, lambda, mode, dW, true);
@@ -1153,7 +1156,7 @@ extern "C" int pkv_build_stack(pkv_ctx* c, int n_layers, int first_layer, const 
                                int lambda_mode, float* const* dW, const pkv_ref_next* final, pkv_stats* stats) {
     if (!c || !w || !full || !cb || !ref0 || !dW || n_layers <= 0 || first_layer < 0 || first_layer >= n_layers)
         return PKV_ERR_INVALID_ARG;
-    if (c->engine != PKV_ENGINE_SIMT && !c->timing && !c->force_sequential && n_layers - first_layer >= 2 &&
+    if (c->engine != PKV_ENGINE_SIMT && c->timing != 1 && !c->force_sequential && n_layers - first_layer >= 2 &&
         n_layers <= kMaxStackLayers)
         return build_stack_overlapped(c, n_layers, first_layer, w, full, cb, ref0, lambda, lambda_mode, dW, final, stats);
     pkv_ref ref = *ref0;

@@ -768,14 +768,18 @@ def test_timed_build_uses_the_stacked_schedule_and_agrees(B):
     idx_t = torch.from_numpy(idx).cuda()
     tF, tC = torch.from_numpy(xF).cuda(), torch.from_numpy(xC).cuda()
     outs = []
-    for timed in (False, True, False):
+    for timed in (False, True, False, 2):
         ctx.set_timing(timed)
         o = ctx.build_patch(w, kv["K"], kv["V"], off, idx_t, tF, tC, chunk_off, cfg.L, 0.1, 0, True)
         outs.append({k: (v.cpu().numpy() if hasattr(v, "cpu") else v) for k, v in o.items()})
     ctx.close()
     errs = [H.rel_fro(o["dW"], ref["dW"]) for o in outs]
     cross = H.rel_fro(outs[1]["dW"], outs[0]["dW"])
-    print("untimed / timed / untimed vs oracle: %.3e %.3e %.3e; timed vs untimed %.3e" % (*errs, cross))
+    print("untimed / timed / untimed / solve-only timing vs oracle: %.3e %.3e %.3e %.3e; timed vs untimed %.3e" % (*errs, cross))
+    # mode 2 times the solve alone and leaves the schedule as it is
+    sm = outs[3]["stats"]["stage_ms"]
+    assert sm[7] > 0 and sum(sm) == sm[7]
+    assert H.rel_fro(outs[3]["dW"], outs[0]["dW"]) <= 1e-5
     assert max(errs) <= DW_TOL and cross <= 2e-3
     assert sum(outs[1]["stats"]["stage_ms"]) > 0 and sum(outs[0]["stats"]["stage_ms"]) == 0
     for o in outs:
