@@ -749,6 +749,46 @@ def test_statistics_survive_massive_activations(B):
     print("features x256: dW rel fro err %.3e" % e)
 
 
+def test_repeated_builds_on_one_context_are_stable(B):
+    """The build spreads one block over several internal streams (student half, teacher half on an SM partition,
+    targets and S_T beside the solve, the solve's own four).  Forty builds back to back on one context, alternating
+    between two problems, must each reproduce the first result of their problem: an ordering hole between the
+    streams would show up as a result that depends on what ran before."""
+    import torch
+    cfg = small_cfg("bf16", hd=128, Hq=8, Hkv=2, d=512, F=448, L=3000, N=200, window=32, budget=300, n_obs=16)
+    lay = H.make_problem(cfg)
+    rng = np.random.default_rng(17)
+    xF = lay["x0"]
+    xCs = [(xF + s_ * rng.standard_normal(xF.shape)).astype(np.float32) for s_ in (0.05, 0.2)]
+    chunk_off = [0, 120, cfg.N]
+    ctx = B.PkvContext(B.dims_from_config(cfg, N_max=cfg.N, b_max=max(len(k) for k in lay["kept"])), engine=B.ENGINE_AUTO)
+    w = B.to_device(lay["weights"], cfg.dtype)
+    kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
+    off, idx = gen.kept_to_csr(lay["kept"])
+    idx_t = torch.from_numpy(idx).cuda()
+    tF = torch.from_numpy(xF).cuda()
+    tCs = [torch.from_numpy(x).cuda() for x in xCs]
+    first = [None, None]
+    worst = 0.0
+    for i in range(40):
+        k = i & 1
+        o = ctx.build_patch(w, kv["K"], kv["V"], off, idx_t, tF, tCs[k], chunk_off, cfg.L, 0.1, 0, True)
+        got = {n: o[n].cpu().numpy() for n in ("dW", "xF_next", "xC_next")}
+        got["t"] = o["stats"]["target_fro2"]
+        if first[k] is None:
+            first[k] = got
+            ref = H.run_oracle(cfg, lay, xF, xCs[k], chunk_off, 0.1, 0)
+            assert H.rel_fro(got["dW"], ref["dW"]) <= DW_TOL
+            continue
+        for n in ("dW", "xF_next", "xC_next"):
+            e = H.rel_fro(got[n], first[k][n])
+            worst = max(worst, e)
+            assert e <= 1e-5, (i, n, e)
+        np.testing.assert_allclose(got["t"], first[k]["t"], rtol=1e-6)
+    ctx.close()
+    print("40 alternating builds: largest deviation from the first result %.2e" % worst)
+
+
 def test_timed_build_uses_the_stacked_schedule_and_agrees(B):
     """With stage timing on, a block runs teacher and student stacked on one stream (so that the stage marks mean
     something); without, the student half runs first and the teacher half beside the solve.  Same patch either way,
