@@ -510,7 +510,8 @@ static int gram_cross_own(const Lc& lc, TcBuffers* t, int F, int dm, int n, floa
         g.A[2] = TcMat{t->RT.lo, t->ldT, dm, n}; g.B[2] = TcMat{t->XT.hi, t->ldT, F, n};
         g.npass = 3;
     }
-    g.out[0] = t->S3[0]; g.out[1] = t->S3[1]; g.out[2] = t->S3[2]; g.ldo = F; g.nout = 3;
+    // the solver's first product reads two parts of S_T on the well-conditioned plan, three otherwise
+    g.out[0] = t->S3[0]; g.out[1] = t->S3[1]; g.out[2] = t->S3[2]; g.ldo = F; g.nout = precise ? 3 : 2;
     const int rc = gemm_tc(lc, g, status);
     if (rc == PKV_OK) t->S3_ready = 1;
     return rc;
