@@ -327,6 +327,25 @@ int pkv_low_rank(pkv_ctx* ctx, const float* dW, const float* S_H, int32_t r, int
 int pkv_ridge_solve(pkv_ctx* ctx, const float* S_H, const float* S_T, float lambda, int lambda_mode,
                     float* dW, pkv_stats* stats);
 
+/* Ridge solve with iterative refinement (Eq. 6 read with lambda as written, and the small coefficients of the
+ * ridge-scale ablation: S_H + lambda I is then ill conditioned, and the rounding of the factorisation and of the
+ * explicit inverse factor reaches dW amplified by its condition number).  After the solve of pkv_ridge_solve,
+ * `steps` times: R = S_T - dW (S_H + lambda I) as an fp32-equivalent product against the caller's S_H, then
+ * dW += R (S_H + lambda I)^{-1} through the factor already computed.  Each step costs one d x F x F product in six
+ * passes and the two triangular products of Eq. 8 again; what it cannot remove is the rounding of the fp32 residual
+ * itself (about 2^-24 cond(G)), so one step is normally all that helps.  steps = 0 is pkv_ridge_solve; at most 8.
+ * S_H must be the full symmetric matrix.  stats->resid_fro2 = ||S_T - dW (S_H + lambda I)||_F^2 of the iterate
+ * BEFORE the last correction (0 for steps = 0); dW_fro2 is the final iterate's.  Tensor-core engine only
+ * (PKV_ERR_UNSUPPORTED otherwise); pointers 16-byte aligned. */
+int pkv_ridge_solve_refined(pkv_ctx* ctx, const float* S_H, const float* S_T, float lambda, int lambda_mode,
+                            int32_t steps, float* dW, pkv_stats* stats);
+
+/* The same refinement after every ridge solve the context runs from now on (pkv_build_patch, pkv_build_stack and
+ * its sweep, pkv_stream_finish, pkv_ridge_solve): steps = 0 (default) switches it off.  A build keeps a full
+ * symmetric copy of S_H beside the matrix it factors in place; the student's next state is formed with the
+ * refined patch.  Tensor-core engine with the primal solver only (PKV_ERR_UNSUPPORTED otherwise). */
+int pkv_set_refinement(pkv_ctx* ctx, int steps);
+
 /* The product the ridge solve is built from (Eq. 8 needs fp32 accuracy; the tensor cores take bf16): C [M][N]
  * (+)= alpha * A B^T with A [M][K], B [N][K], C device fp32 row-major, 16-byte aligned.  Each operand is split
  * into bf16 parts (hi, mid, lo) and multiplied in `passes` passes accumulating in fp32: 6 = fp32-equivalent

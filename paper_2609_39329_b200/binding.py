@@ -144,6 +144,9 @@ def lib() -> C.CDLL:
                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     L.pkv_ridge_solve.restype = C.c_int
     L.pkv_ridge_solve.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_void_p, P(pkv_stats)]
+    L.pkv_ridge_solve_refined.restype = C.c_int
+    L.pkv_ridge_solve_refined.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_int32, C.c_void_p,
+                                          P(pkv_stats)]
     L.pkv_fp32_product.restype = C.c_int
     L.pkv_fp32_product.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_float,
                                    C.c_void_p, C.c_int, C.c_int, C.c_int]
@@ -153,6 +156,8 @@ def lib() -> C.CDLL:
     L.pkv_set_timing.argtypes = [C.c_void_p, C.c_int]
     L.pkv_launch_count.restype = C.c_int64
     L.pkv_launch_count.argtypes = [C.c_void_p]
+    L.pkv_set_refinement.restype = C.c_int
+    L.pkv_set_refinement.argtypes = [C.c_void_p, C.c_int]
     L.pkv_set_stack_schedule.restype = C.c_int
     L.pkv_set_stack_schedule.argtypes = [C.c_void_p, C.c_int]
     L.pkv_measure_fma_peak.restype = C.c_int
@@ -251,6 +256,12 @@ class PkvContext:
         site = C.c_int32(0)
         rc = self.L.pkv_selftest_bounded_wait(self.h, C.byref(site))
         return int(rc), int(site.value)
+
+    def set_refinement(self, steps):
+        """Corrections of iterative refinement after every ridge solve of this context (0 = off)."""
+        rc = self.L.pkv_set_refinement(self.h, int(steps))
+        if rc != 0:
+            self._raise(rc, {})
 
     def set_timing(self, on):
         """False/0: off; True/1: every stage (stacked schedule); 2: the solve's interval only, default schedule."""
@@ -492,11 +503,15 @@ class PkvContext:
             self._raise(rc)
         return {"U": U, "Br": Br, "dW_r": dWr, "ritz": ritz}
 
-    def ridge_solve(self, S_H, S_T, lam, mode=LAMBDA_PAPER):
+    def ridge_solve(self, S_H, S_T, lam, mode=LAMBDA_PAPER, refine_steps=0):
         torch = self.torch
         dW = torch.empty((self.dims.d, self.dims.F), dtype=torch.float32, device=S_H.device)
         st = pkv_stats()
-        rc = self.L.pkv_ridge_solve(self.h, _ptr(S_H), _ptr(S_T), float(lam), int(mode), _ptr(dW), C.byref(st))
+        if refine_steps:
+            rc = self.L.pkv_ridge_solve_refined(self.h, _ptr(S_H), _ptr(S_T), float(lam), int(mode), int(refine_steps),
+                                                _ptr(dW), C.byref(st))
+        else:
+            rc = self.L.pkv_ridge_solve(self.h, _ptr(S_H), _ptr(S_T), float(lam), int(mode), _ptr(dW), C.byref(st))
         if rc != 0:
             self._raise(rc, st.as_dict())
         return dW, st.as_dict()

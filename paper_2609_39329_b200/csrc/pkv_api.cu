@@ -220,6 +220,7 @@ struct pkv_ctx {
     int stream_open, stream_mode, stream_tokens;   // streamed reference set in progress (pkv_stream_*)
     float stream_lambda;
     double stream_tfro2;
+    int refine_steps;        // corrections of iterative refinement after every ridge solve of a build (pkv_set_refinement)
     int force_sequential;    // pkv_build_stack: 1 = block by block on one stream even where the overlapped driver applies
     int teacher_timed;
     void* map_cache;
@@ -494,6 +495,13 @@ extern "C" int pkv_set_stack_schedule(pkv_ctx* c, int schedule) {
     return PKV_OK;
 }
 
+extern "C" int pkv_set_refinement(pkv_ctx* c, int steps) {
+    if (!c || steps < 0 || steps > 8) return PKV_ERR_INVALID_ARG;
+    if (steps > 0 && (c->engine == PKV_ENGINE_SIMT || c->dual)) return PKV_ERR_UNSUPPORTED;
+    c->refine_steps = steps;
+    return PKV_OK;
+}
+
 extern "C" int pkv_measure_fma_peak(pkv_ctx* c, double* tflops) {
     if (!c || !tflops) return PKV_ERR_INVALID_ARG;
     cudaStreamSynchronize(c->st);
@@ -717,11 +725,36 @@ static void gram_simt(pkv_ctx* c, const Lc& lc, const float* X, const float* R, 
 }
 
 // S8.  `S_H_scratch` says that S_H may be overwritten (it is the context's own statistics buffer).
-static void solve_stage(pkv_ctx* c, const Lc& lc, float* S_H, const float* S_T, float lam0, int mode, float* dW,
-                        bool S_H_scratch, DevStatus* status = nullptr) {
+// Iterative refinement of dW = S_T (S_H + lambda I)^{-1} after a tensor-core solve: `steps` times the residual
+// R = S_T - dW (S_full + lambda I) as an fp32-equivalent product, then dW += (R X^T) X with the inverse factor the
+// solve left behind.  S_full: the full symmetric S_H, untouched by the factorisation.
+static int refine_solution(pkv_ctx* c, const Lc& lc, const float* S_full, const float* S_T, float lam0, int mode,
+                           float* dW, DevStatus* st, int steps, bool report_residual) {
+    const int F = c->dims.F, d = c->dims.d;
+    Buffers& b = c->b;
+    const bool well = pkv::tc_well_conditioned(lam0, mode);
+    float* P = b.solve.Y;      // [d][F]: dW S_H, then the residual
+    for (int s = 0; s < steps; ++s) {
+        int rc = pkv::tc_fp32_product(lc, &b.tc.solve, (size_t)d * F, dW, S_full, d, F, F, 1.f, P, false, 6, 4, st, true);
+        if (rc != PKV_OK) return rc;
+        refine_residual(lc, S_T, dW, P, (int64_t)d * F, st, report_residual);
+        if (report_residual) sumsq(lc, P, (int64_t)d * F, &st->res_fro2);
+        if ((rc = pkv::tc_solve_apply_add(lc, &b.tc.solve, P, F, F, d, dW, well, st)) != PKV_OK) return rc;
+        sumsq(lc, dW, (int64_t)d * F, &st->dw_fro2);
+    }
+    // the next-state product of a build reads dW as a bf16 pair, which the solve's last product wrote
+    if (steps > 0) pkv::tc_split_pair(lc, dW, d, F, b.tc.dW);
+    return PKV_OK;
+}
+
+// refine < 0: the context's setting (pkv_set_refinement); the standalone refined solve passes its own count and
+// reports the residual's norm.
+static int solve_stage(pkv_ctx* c, const Lc& lc, float* S_H, const float* S_T, float lam0, int mode, float* dW,
+                       bool S_H_scratch, DevStatus* status = nullptr, int refine = -1) {
     const int F = c->dims.F, d = c->dims.d;
     Buffers& b = c->b;                 // the context's own buffers: the solver keeps state in b.tc
     DevStatus* st = status ? status : b.status;
+    const int steps = refine >= 0 ? refine : c->refine_steps;
     // the tensor-core build leaves only the lower triangle of its own S_H
     trace_fro2(lc, S_H, F, st, 0, S_H_scratch && c->engine != PKV_ENGINE_SIMT);
     if (c->engine == PKV_ENGINE_SIMT) {
@@ -731,14 +764,23 @@ static void solve_stage(pkv_ctx* c, const Lc& lc, float* S_H, const float* S_T, 
     } else {
         ridge_lambda(lc, F, lam0, mode, st);
         float* S = S_H;
+        const float* S_full = S_H;     // what a refinement step multiplies by: never the factored copy
         if (!S_H_scratch) {
-            cudaMemcpyAsync(b.solve.G, S_H, (size_t)F * F * sizeof(float), cudaMemcpyDeviceToDevice, c->st);
+            cudaMemcpyAsync(b.solve.G, S_H, (size_t)F * F * sizeof(float), cudaMemcpyDeviceToDevice, lc.st);
             S = b.solve.G;
             b.tc.S3_ready = 0;         // the caller's S_T, not the one a build's statistics left split in place
+        } else if (steps > 0) {
+            symmetric_from_lower(lc, S_H, b.solve.G, F);     // S_H itself is factored in place
+            S_full = b.solve.G;
         }
         pkv::tc_ridge_solve(lc, &b.tc, S, S_T, F, d, dW, lam0, mode, st);
+        if (steps > 0) {
+            sumsq(lc, dW, (int64_t)d * F, &st->dw_fro2);     // (cleared again by the first step; keeps the code path uniform)
+            return refine_solution(c, lc, S_full, S_T, lam0, mode, dW, st, steps, refine >= 0);
+        }
     }
     sumsq(lc, dW, (int64_t)d * F, &st->dw_fro2);
+    return PKV_OK;
 }
 
 // stats_only: the streamed form (Sec. 2.3, Eq. 9): teacher and student forward of these tokens, then the running
@@ -1280,6 +1322,21 @@ extern "C" int pkv_gram(pkv_ctx* c, const float* X, const float* R, int32_t n, f
     else
         pkv::tc_gram(lc, &c->b.tc, &c->dims, X, R, n, S_H, S_T, accumulate != 0, c->b.status);
     return end_call(c, nullptr, nullptr);
+}
+
+extern "C" int pkv_ridge_solve_refined(pkv_ctx* c, const float* S_H, const float* S_T, float lambda, int lambda_mode,
+                                       int32_t steps, float* dW, pkv_stats* stats) {
+    if (!c || !S_H || !S_T || !dW || steps < 0 || steps > 8) return PKV_ERR_INVALID_ARG;
+    if (!(lambda > 0.f) || !isfinite(lambda)) return PKV_ERR_INVALID_ARG;
+    if (lambda_mode != PKV_LAMBDA_PAPER && lambda_mode != PKV_LAMBDA_ABSOLUTE && lambda_mode != PKV_LAMBDA_TRACE_MEAN)
+        return PKV_ERR_INVALID_ARG;
+    if (((uintptr_t)S_H & 15) || ((uintptr_t)S_T & 15) || ((uintptr_t)dW & 15)) return PKV_ERR_INVALID_ARG;
+    if (c->engine == PKV_ENGINE_SIMT) return PKV_ERR_UNSUPPORTED;
+    Lc lc{c->st, &c->launches, c->map_cache};
+    begin_call(c);
+    const int rc = solve_stage(c, lc, const_cast<float*>(S_H), S_T, lambda, lambda_mode, dW, false, nullptr, steps);
+    if (rc != PKV_OK) return rc;
+    return end_call(c, stats, nullptr);
 }
 
 extern "C" int pkv_fp32_product(pkv_ctx* c, const float* A, const float* B, int32_t M, int32_t N, int32_t K, float alpha,

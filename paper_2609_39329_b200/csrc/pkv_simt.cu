@@ -796,6 +796,56 @@ void sub_f32(const Lc& lc, const float* a, const float* b, int64_t n, float* out
     lc.count();
 }
 
+// Residual of the ridge system for iterative refinement: R = S_T - lambda dW - P with P = dW S_H given (in place:
+// R overwrites P); lambda is the coefficient the solve used (status->lam).  The norm of dW is reported anew after the
+// correction and is cleared here, the residual's norm too where the caller reports it.
+__global__ void k_refine_residual(const float* __restrict__ S_T, const float* __restrict__ dW, float* __restrict__ P, size_t n,
+                                  DevStatus* status) {
+    const float lam = status->lam;
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) P[i] = (S_T[i] - P[i]) - lam * dW[i];
+}
+__global__ void k_clear_refine_norms(DevStatus* status, int clear_res) {
+    if (clear_res) status->res_fro2 = 0.0;
+    status->dw_fro2 = 0.0;
+}
+
+void refine_residual(const Lc& lc, const float* S_T, const float* dW, float* P, int64_t n, DevStatus* status, bool clear_res) {
+    if (n <= 0) return;
+    k_clear_refine_norms<<<1, 1, 0, lc.st>>>(status, clear_res ? 1 : 0);
+    k_refine_residual<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(S_T, dW, P, (size_t)n, status);
+    lc.count(2);
+}
+
+// G (full symmetric) from the lower triangle of S: G[i][j] = S[max(i,j)][min(i,j)].
+__global__ void k_symmetric_from_lower(const float* __restrict__ S, float* __restrict__ G, int F) {
+    __shared__ float t[32][33];
+    const int bi = blockIdx.y, bj = blockIdx.x;
+    if (bj > bi) return;
+    const int r0 = bi * 32, c0 = bj * 32;
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int r = r0 + j, c = c0 + threadIdx.x;
+        float v = 0.f;
+        if (r < F && c < F) {
+            v = c <= r ? S[(size_t)r * F + c] : S[(size_t)c * F + r];      // diagonal tiles: mirror inside the tile
+            G[(size_t)r * F + c] = v;
+        }
+        t[j][threadIdx.x] = v;
+    }
+    if (bj == bi) return;
+    __syncthreads();
+    for (int j = threadIdx.y; j < 32; j += 8) {
+        const int r = c0 + j, c = r0 + threadIdx.x;      // the mirrored tile
+        if (r < F && c < F) G[(size_t)r * F + c] = t[threadIdx.x][j];
+    }
+}
+
+void symmetric_from_lower(const Lc& lc, const float* S, float* G, int F) {
+    dim3 grid((F + 31) / 32, (F + 31) / 32), block(32, 8);
+    k_symmetric_from_lower<<<grid, block, 0, lc.st>>>(S, G, F);
+    lc.count();
+}
+
 // ------------------------------------------------------------------------------------------
 // merge: W <- W + dW, sum in fp32, one rounding to W's type
 // ------------------------------------------------------------------------------------------

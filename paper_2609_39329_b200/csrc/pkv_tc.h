@@ -117,6 +117,11 @@ int tc_ridge_solve_impl(const Lc& lc, TcSolveBuffers* t, const float* G, const f
                         __nv_bfloat16* const* S_T_triple,    // optional: dW's bf16 pair out; S_T already split
                         bool wait_S_T = false);              // S_T is complete only once t->st_ready has fired
 
+// dW [d][n] += (R X^T) X with the inverse factor X of the system solved last on t (one correction of iterative
+// refinement); R [d][n] fp32, row stride ld.
+int tc_solve_apply_add(const Lc& lc, TcSolveBuffers* t, const float* R, int n, int ld, int d, float* dW,
+                       bool well_conditioned, DevStatus* status);
+
 int tc_fp32_product(const Lc& lc, TcSolveBuffers* t, size_t cap_elems, const float* A, const float* B, int M, int N,
                     int K, float alpha, float* C, bool accumulate, int passes, int nacc, DevStatus* status,
                     bool b_in_factor_buffer = false);

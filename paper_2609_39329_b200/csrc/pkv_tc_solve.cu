@@ -938,7 +938,8 @@ static bool solve_trace() {
 static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const float* S_T, int n, int ld, int d,
                       float* dW, float* const* dW_ind, bool well_conditioned, bool zero_fill,
                       DevStatus* status, const Pair* dW_pair, __nv_bfloat16* const* S_T_triple, bool wait_S_T,
-                      int phase = 0) {      // 0: the whole solve; 1: factorisation and inverse only; 2: final products only
+                      int phase = 0,        // 0: the whole solve; 1: factorisation and inverse only; 2: final products only
+                      bool add_to_dW = false) {      // the last product adds to dW instead of overwriting it
     const int F = n;      // dimension of the system; ld is the row stride of G, S_T, dW and of every n x n work array
     const int nblk = (F + PB - 1) / PB;
     Trip L3{{t->L3[0], t->L3[1], t->L3[2]}}, X3{{t->X3[0], t->X3[1], t->X3[2]}}, XT3{{t->XT3[0], t->XT3[1], t->XT3[2]}};
@@ -1185,7 +1186,7 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
         else six_pass(g, Z2, ld, d, F, XT3, ld, F, F);
         g.M = d; g.N = F; g.K = F; g.batch = 1; g.alpha = 1.f; g.k_tri = 2;
         g.nacc = well_conditioned ? 1 : 2;
-        g.C = dW; g.C_ind = dW_ind; g.ldc = ld; g.c_rows = d; g.c_cols = F;
+        g.C = dW; g.C_ind = dW_ind; g.ldc = ld; g.c_rows = d; g.c_cols = F; g.accumulate = add_to_dW;
         if (dW_pair) { g.out[0] = dW_pair->hi; g.out[1] = dW_pair->lo; g.ldo = ld; g.nout = 2; }
         if ((rc = gemm_tc(lc, g, status))) return rc;
     }
@@ -1201,6 +1202,14 @@ static int solve_body(const Lc& lc, TcSolveBuffers* t, const float* G, const flo
                 a, b, c2, e);
     }
     return PKV_OK;
+}
+
+// One correction of iterative refinement: dW += (R X^T) X with the inverse factor X = L^{-1} that the last solve of
+// this system left in the solver's buffers (Eq. 8 applied to a residual R [d][n] instead of S_T).
+int tc_solve_apply_add(const Lc& lc, TcSolveBuffers* t, const float* R, int n, int ld, int d, float* dW,
+                       bool well_conditioned, DevStatus* status) {
+    return solve_body(lc, t, nullptr, R, n, ld, d, dW, nullptr, well_conditioned, false, status, nullptr, nullptr, false, 2,
+                      true);
 }
 
 __global__ void k_solve_begin(float** slot, float* dW, DevStatus* gstatus, const DevStatus* status) {

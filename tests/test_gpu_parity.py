@@ -39,10 +39,12 @@ def engines(B, cfg):
     return [B.ENGINE_AUTO, B.ENGINE_SIMT]
 
 
-def gpu_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode=0, kv_split=0, want_next=True, solver=0):
+def gpu_build(B, cfg, lay, xF, xC, chunk_off, lam0, engine, mode=0, kv_split=0, want_next=True, solver=0, refine=0):
     import torch
     ctx = B.PkvContext(B.dims_from_config(cfg, N_max=xF.shape[0], b_max=max(len(k) for k in lay["kept"])),
                        engine=engine, kv_split=kv_split, solver=solver)
+    if refine:
+        ctx.set_refinement(refine)
     w = B.to_device(lay["weights"], cfg.dtype)
     kv = B.to_device({"K": lay["K"], "V": lay["V"]}, cfg.dtype)
     off, idx = gen.kept_to_csr(lay["kept"])
@@ -423,6 +425,64 @@ def test_ridge_solve_parity_modes_and_errors(B, F, d, n):
         ctx.close()
 
 
+def ill_conditioned_statistics(F, d, n, seed=5):
+    r = np.random.default_rng(seed)
+    S_H, S_T = orc.sufficient_statistics(r.standard_normal((n, F)), r.standard_normal((n, d)))
+    # what the device is handed is the fp32 rounding; the oracle solves exactly that system in fp64
+    return S_H.astype(np.float32), S_T.astype(np.float32)
+
+
+def test_iterative_refinement_for_a_small_absolute_ridge(B):
+    """Eq. 6 with lambda as written (absolute mode) on a rank-deficient S_H (n < F): cond(G) = 4.6e4, the plain
+    fp32-equivalent solve misses the 5e-3 tolerance, one correction brings it inside; the reported residual norm falls
+    from step to step; zero steps is the plain solve bit for bit."""
+    import torch
+    F = d = 2048
+    cfg = small_cfg("bf16", F=F, d=d, Hq=16, Hkv=2, hd=128, N=64)
+    S_H, S_T = ill_conditioned_statistics(F, d, 512)
+    want = orc.ridge_solve(S_H.astype(np.float64), S_T.astype(np.float64), 0.1)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    tH, tT = torch.from_numpy(S_H).cuda(), torch.from_numpy(S_T).cuda()
+    plain, st0 = ctx.ridge_solve(tH, tT, 0.1, B.LAMBDA_ABSOLUTE)
+    assert st0["cond_warning"] == 1
+    errs, resid = [H.rel_fro(plain.cpu().numpy(), want)], []
+    for steps in (1, 2):
+        dW, st = ctx.ridge_solve(tH, tT, 0.1, B.LAMBDA_ABSOLUTE, refine_steps=steps)
+        errs.append(H.rel_fro(dW.cpu().numpy(), want))
+        resid.append(np.sqrt(st["resid_fro2"]) / np.linalg.norm(S_T))
+        np.testing.assert_allclose(st["dW_fro2"], np.sum(want * want), rtol=1e-2)
+    print("refinement at cond 4.6e4: error %.2e -> %.2e -> %.2e, residual before the last step %.1e, %.1e" %
+          (errs[0], errs[1], errs[2], resid[0], resid[1]))
+    assert errs[0] > DW_TOL > errs[1] and errs[1] <= errs[0] / 4 and errs[2] <= DW_TOL
+    assert resid[1] < resid[0] / 4
+    # the context's own setting applies the same correction to a plain solve call; switched off again it is gone
+    ctx.set_refinement(1)
+    dW1, _ = ctx.ridge_solve(tH, tT, 0.1, B.LAMBDA_ABSOLUTE)
+    assert H.rel_fro(dW1.cpu().numpy(), want) <= DW_TOL
+    ctx.set_refinement(0)
+    again, _ = ctx.ridge_solve(tH, tT, 0.1, B.LAMBDA_ABSOLUTE)
+    assert torch.equal(again, plain)
+    with pytest.raises(B.PkvError):
+        ctx.set_refinement(9)
+    ctx.close()
+    # well conditioned (Eq. 7, lambda0 = 0.1): refinement changes nothing that matters
+    S_H, S_T = ill_conditioned_statistics(448, 256, 900, seed=6)
+    cfg = small_cfg("bf16", F=448, d=256, Hq=4, Hkv=1)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    lam = orc.ridge_lambda(S_H.astype(np.float64), 0.1, B.LAMBDA_PAPER)
+    want = orc.ridge_solve(S_H.astype(np.float64), S_T.astype(np.float64), lam)
+    for steps in (0, 1):
+        dW, _ = ctx.ridge_solve(torch.from_numpy(S_H).cuda(), torch.from_numpy(S_T).cuda(), 0.1, B.LAMBDA_PAPER,
+                                refine_steps=steps)
+        assert H.rel_fro(dW.cpu().numpy(), want) <= 1e-4, steps
+    ctx.close()
+    simt = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_SIMT)
+    with pytest.raises(B.PkvError) as ei:
+        simt.set_refinement(1)
+    assert ei.value.code == -2
+    simt.close()
+
+
 def test_solve_with_more_operand_sets_than_cached_graphs(B):
     """The solve is replayed from a graph captured per operand set, a few of which are kept: six different S_T
     buffers in turn (older graphs are dropped), then the first again, each against the oracle; the result address
@@ -577,6 +637,55 @@ def test_dual_solver_gives_the_same_patch(B, N, F):
     with pytest.raises(B.PkvError) as ei:
         B.PkvContext(B.dims_from_config(gen.scaled_config(cfg, N=F + 8)), solver=B.SOLVER_DUAL)
     assert ei.value.code == -2
+
+
+def test_block_and_stack_with_refinement_match_the_oracle(B):
+    """pkv_set_refinement on the building calls: a block in absolute-lambda mode with fewer reference tokens than
+    features (ill conditioned: the condition warning is raised) and a three-block stack, each with one correction,
+    against the oracle; the student's next state is formed with the refined patch."""
+    import torch
+    cfg = small_cfg("bf16", hd=128, Hq=4, Hkv=2, d=256, F=448, L=700, N=70)
+    lay = H.make_problem(cfg)
+    x = lay["x0"]
+    # the absolute coefficient: 5e-5 of the eigenvalue mean of S_H (the oracle under Eq. 7 gives its value)
+    ref = H.run_oracle(cfg, lay, x, x, [0, cfg.N], 5e-5)
+    lam_abs = float(ref["lam"])
+    errs = []
+    for refine in (0, 1):
+        got = gpu_build(B, cfg, lay, x, x, [0, cfg.N], lam_abs, B.ENGINE_AUTO, mode=B.LAMBDA_ABSOLUTE, refine=refine)
+        errs.append(H.rel_fro(got["dW"], ref["dW"]))
+        assert got["stats"]["cond_warning"] == 1
+        if refine:
+            assert H.rel_fro(got["xC_next"], ref["xC_next"]) <= 1e-3
+            gap = got["xF_next"].astype(np.float64) - got["xC_next"]
+            np.testing.assert_allclose(got["stats"]["resid_fro2"], np.sum(gap * gap), rtol=1e-2)
+            np.testing.assert_allclose(got["stats"]["dW_fro2"], np.sum(ref["dW"] ** 2), rtol=2e-2)
+    print("block, absolute lambda (5e-5 of the eigenvalue mean), cond lower bound %.1e: dW error %.2e plain, %.2e with one correction" %
+          (got["stats"]["cond_lower_bound"], errs[0], errs[1]))
+    assert errs[1] <= DW_TOL and errs[1] <= errs[0]
+    nl = 3
+    cfg = small_cfg("bf16", n_layers=nl, N=64, hd=128, Hq=4, Hkv=2)
+    lays = [H.make_problem(cfg, layer=l) for l in range(nl)]
+    x0 = lays[0]["x0"]
+    xF, xC = x0.astype(np.float64), x0.astype(np.float64)
+    refs = []
+    for l in range(nl):
+        refs.append(H.run_oracle(cfg, lays[l], xF, xC, [0, cfg.N], 1e-3))
+        xF, xC = refs[-1]["xF_next"], refs[-1]["xC_next"]
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    ctx.set_refinement(1)
+    dl = []
+    for l in range(nl):
+        off, idx = gen.kept_to_csr(lays[l]["kept"])
+        kv = B.to_device({"K": lays[l]["K"], "V": lays[l]["V"]}, cfg.dtype)
+        dl.append({"w": B.to_device(lays[l]["weights"], cfg.dtype), "K": kv["K"], "V": kv["V"], "head_off": off,
+                   "idx": torch.from_numpy(idx).cuda()})
+    xt = torch.from_numpy(x0).cuda()
+    out = ctx.build_stack(dl, xt, xt, [0, cfg.N], cfg.L, 1e-3)
+    for l in range(nl):
+        assert H.rel_fro(out["dW"][l].cpu().numpy(), refs[l]["dW"]) <= DW_TOL, l
+    assert H.rel_fro(out["xC_final"].cpu().numpy(), refs[-1]["xC_next"]) <= 2e-3
+    ctx.close()
 
 
 def test_identical_caches_give_zero_patch(B):
