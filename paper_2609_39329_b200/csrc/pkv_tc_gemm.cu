@@ -362,6 +362,208 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
     if (threadIdx.x == 0) gemm_stamp(p, 7);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// CTA-pair variant (cta_group::2): a cluster of two CTAs computes one 256 x 256 tile.  Each CTA loads its own 128
+// rows of every A part and its own 128-row half of every B part (no load is shared or multicast), the leader's
+// single MMA thread issues M = 256, N = 256 instructions that read both CTAs' shared memory, and each CTA's epilogue
+// warps store the 128 rows its tensor memory holds.  Against 128 x 256 tiles of single CTAs this halves the B bytes
+// an SM pulls from L2 per flop (a two-pass stage is 48 KB instead of 64 KB), which is what bounds the long products.
+// Taken for plain dense products whose M and N are multiples of 256 (the launcher decides); everything else stays
+// on k_gemm_tc.  Barriers per CTA: full[s] (used in the leader only: it counts the bytes of BOTH CTAs' loads of stage
+// s - the peer's loads name the leader's barrier -, so one wait tells the MMA thread that the whole stage is
+// there), empty[s] and the accumulator barrier (both arrived on by the leader's commits, in both CTAs).
+// ---------------------------------------------------------------------------------------------
+constexpr int kPairBarBytes = (3 * kGemmMaxStages + 1) * 8 + 32;
+
+__global__ void __launch_bounds__(192) k_gemm_tc_pair(const __grid_constant__ GemmTcParams p) {
+    constexpr int BN = 256;
+    const uint32_t rank = cluster_ctarank();          // 0: leader, 1: peer
+    const int ntn = (int)(gridDim.x >> 1);
+    const int tn = (p.k_tri == 1) ? ntn - 1 - (int)(blockIdx.x >> 1) : (int)(blockIdx.x >> 1);
+    const int m0 = (int)blockIdx.y * 256 + (int)rank * 128, n0 = tn * BN, z = blockIdx.z;
+    const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
+
+    constexpr int kT = 128 * 64 * 2;                  // every operand tile of a CTA: 128 rows x 64 bf16
+    const int stage_bytes = (p.nA + p.nB) * kT;
+    const int STAGES = p.stages;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - raw);
+    const uint32_t bars = base + STAGES * stage_bytes;        // full[S], empty[S], (unused [S]), accumulator
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * STAGES, bar_acc = bars + 24 * STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sm + STAGES * stage_bytes + (3 * STAGES + 1) * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* skip_flag = reinterpret_cast<volatile int*>(tmem_slot + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int kt_begin = 0, kt_end = (p.K + 63) / 64;
+    if (p.k_tri == 1) kt_end = min(kt_end, (n0 + BN + 63) / 64);
+    if (p.k_tri == 2) kt_begin = min(kt_end, n0 / 64);
+    const int ktiles = kt_end - kt_begin;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < STAGES; ++i) {
+            mbar_init(bar_full + 8 * i, 1);
+            mbar_init(bar_empty + 8 * i, 1);
+        }
+        mbar_init(bar_acc, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        // an earlier stage already failed: the leader reads the status word once and both CTAs take its branch
+        // (the peer reads the leader's copy after the cluster barrier below)
+        *skip_flag = p.status->code;
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(tmem_slot), (uint32_t)BN);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tbase = *tmem_slot;
+    const bool skip = ld_shared_cluster_u32(mapa_shared(smem_u32(const_cast<int*>(skip_flag)), 0)) != 0u;
+
+    if (skip) {
+        // nothing to do: fall through to the teardown
+    } else if (warp == 0) {
+        if (lane == 0) {
+            const int ar = p.a_row0 + z * p.a_zrow + m0, ac = p.a_col0 + z * p.a_zcol;
+            int br = p.b_row0 + z * p.b_zrow + n0;
+            const int bc = p.b_col0 + z * p.b_zcol;
+            int gsel = 0;
+            if (p.ngrp > 1) {
+                while (gsel + 1 < p.ngrp && n0 >= p.grp_end[gsel]) ++gsel;
+                if (gsel > 0) br -= p.grp_end[gsel - 1];
+            }
+            br += (int)rank * 128;                    // this CTA's half of the B tile
+            const uint32_t leader_full = mapa_shared(bar_full, 0);
+            for (int it = 0; it < ktiles; ++it) {
+                const int s = it % STAGES;
+                if (!mbar_wait_cluster(bar_empty + 8 * s, ((it / STAGES) & 1) ^ 1, abort_flag, p.status, 11)) break;
+                const int kt = kt_begin + it;
+                const uint32_t full = leader_full + 8 * s;
+                const uint32_t sa = base + s * stage_bytes;
+                // the leader announces both CTAs' bytes (the peer's may be counted before this: the phase cannot
+                // complete before the leader's arrival)
+                if (rank == 0) mbar_expect_tx(bar_full + 8 * s, 2 * stage_bytes);
+                for (int i = 0; i < p.nA; ++i) tma_load_2d_pair(sa + i * kT, &p.mapA[i], full, ac + kt * 64, ar);
+                for (int i = 0; i < p.nB; ++i)
+                    tma_load_2d_pair(sa + (p.nA + i) * kT, &p.mapB[p.ngrp > 1 ? gsel : i], full, bc + kt * 64, br);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = p.f16 ? idesc_f16(256, BN) : idesc_bf16(256, BN);
+            const uint32_t peer_empty = mapa_shared(bar_empty, 1), peer_acc = mapa_shared(bar_acc, 1);
+            bool ok = true;
+            uint32_t used = 0u;
+            for (int it = 0; it < ktiles; ++it) {
+                const int s = it % STAGES;
+                if (!mbar_wait_cluster(bar_full + 8 * s, (it / STAGES) & 1, abort_flag, p.status, 13)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t sa = base + s * stage_bytes;
+                for (int ps = 0; ps < p.npass; ++ps) {
+                    const uint64_t da = smem_desc_sw128(sa + p.pa[ps] * kT);
+                    const uint64_t db = smem_desc_sw128(sa + (p.nA + p.pb[ps]) * kT);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        mma_f16_ss_pair(tbase, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, used);
+                        used = 1u;
+                    }
+                }
+                // the stage is free again in both CTAs once these MMAs have read it
+                mma_commit_pair(bar_empty + 8 * s);
+                mma_commit_pair(peer_empty + 8 * s);
+            }
+            if (ok) {
+                mma_commit_pair(bar_acc);
+                mma_commit_pair(peer_acc);
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        const int rl0 = m0 + q * 32;
+        const int rowa0 = crow0 + q * 32;
+        const int nrows = max(0, min(32, min(p.M - rl0, p.c_rows - rowa0)));
+        float* const Cp = p.C_ind ? *p.C_ind : p.C;
+        bool ok = true;
+        if (ktiles > 0) {
+            ok = mbar_wait_cluster(bar_acc, 0, abort_flag, p.status, 15);
+            tc_fence_after();
+        }
+        if (ok) {
+            float alpha = p.alpha;
+            if (p.amax_a) alpha *= f16_inv_scale_from_max(*p.amax_a);
+            if (p.amax_b) alpha *= f16_inv_scale_from_max(*p.amax_b);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                if (ktiles > 0) {
+                    tmem_ld32(tbase + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;
+                }
+                const int col = ccol0 + c0;
+                if (min(p.N - (n0 + c0), p.c_cols - col) < 32) break;      // (the launcher only sends whole tiles)
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = alpha * __uint_as_float(r[j]);
+                const size_t row = (size_t)(rowa0 + min(lane, max(nrows - 1, 0)));
+                if (Cp && lane < nrows) {
+                    float* crow = Cp + row * p.ldc + col;
+                    if (p.addend) {
+                        const float* arow = p.addend + row * p.ldadd + col;
+                        float4 a4[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) a4[j] = *reinterpret_cast<const float4*>(arow + 4 * j);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            v[4 * j] += a4[j].x; v[4 * j + 1] += a4[j].y; v[4 * j + 2] += a4[j].z; v[4 * j + 3] += a4[j].w;
+                        }
+                    }
+                    if (p.accumulate && p.nout == 0) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(crow + 4 * j), "f"(v[4 * j]),
+                                         "f"(v[4 * j + 1]), "f"(v[4 * j + 2]), "f"(v[4 * j + 3])
+                                         : "memory");
+                    } else {
+                        if (p.accumulate) {
+                            float4 c4[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) c4[j] = *reinterpret_cast<const float4*>(crow + 4 * j);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                v[4 * j] += c4[j].x; v[4 * j + 1] += c4[j].y; v[4 * j + 2] += c4[j].z; v[4 * j + 3] += c4[j].w;
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            *reinterpret_cast<float4*>(crow + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    }
+                }
+                if (p.nout > 0 && lane < nrows) store_parts_row(p, v, row * p.ldo + (col - p.out_col_off));
+                __syncwarp();
+            }
+        }
+    }
+    // teardown: neither CTA may leave (its shared memory is read by the leader's MMAs, its barriers are arrived on
+    // from the other CTA) before both are done; after an abort give copies in flight time to land first
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tbase, (uint32_t)BN);
+    }
+}
+
 // Self-test of the bounded wait: the barrier below is initialised and never arrived on.
 __global__ void k_selftest_wait(DevStatus* status) {
     __shared__ uint64_t bar_mem;
@@ -530,6 +732,46 @@ static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     return PKV_OK;
 }
 
+static bool pair_enabled() {
+    static const bool v = [] { const char* e = getenv("PKV_GEMM_PAIR"); return !e || atoi(e) != 0; }();
+    return v;
+}
+
+static int launch_gemm_pair(const Lc& lc, GemmTcParams& p, int batch) {
+    static PerDeviceOnce once;
+    constexpr int kMaxSmem = 227 * 1024;
+    int dev;
+    if (once.needed(&dev)) {
+        if (cudaFuncSetAttribute(k_gemm_tc_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem) != cudaSuccess)
+            return PKV_ERR_CUDA;
+        once.mark(dev);
+    }
+    const int stage_bytes = (p.nA + p.nB) * 128 * 128;
+    const int fixed = kPairBarBytes + 1024;
+    const int ktiles = (p.K + 63) / 64;
+    int stages = (kMaxSmem - fixed) / stage_bytes;
+    if (stages > kGemmMaxStages) stages = kGemmMaxStages;
+    if (stages > ktiles) stages = ktiles > 0 ? ktiles : 1;
+    if (stages < 1) return PKV_ERR_UNSUPPORTED;
+    p.stages = stages;
+    const int smem = stages * stage_bytes + fixed;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (p.N / 256), p.M / 256, batch);
+    cfg.blockDim = dim3(192);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = lc.st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, k_gemm_tc_pair, p) != cudaSuccess) return PKV_ERR_CUDA;
+    lc.count();
+    return PKV_OK;
+}
+
 // (A persistent variant - one CTA per SM walking over the tiles with a second accumulator buffer so that one tile's
 // epilogue overlaps the next tile's MMAs - was built and measured: statistics at d = F = 5120 1.12 vs 1.20 ms, a
 // whole config-2 block 4.54 vs 4.39 ms.  The split-bf16 products are bound by operand traffic from L2 and, at few
@@ -544,6 +786,17 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     const long long tiles256 = (long long)((g.N + 255) / 256) * ((g.M + 127) / 128) * g.batch;
     const bool wide = g.N >= 512 && tiles256 >= 120 && !g.lower_only && g.nacc < 4;
     const int BN = (g.skip_tile00 || g.out_col0_only) ? 128 : ((g.N <= 64) ? 64 : (wide ? 256 : 128));
+    // CTA pairs on 256 x 256 tiles for plain dense products of whole tiles (see k_gemm_tc_pair)
+    bool pair = pair_enabled() && BN == 256 && !lc.pdl && g.M % 256 == 0 && g.N % 256 == 0 && g.a_tri == 0 && g.nacc <= 1 &&
+                !g.stamps && g.c_rows >= g.c_row0 + (g.batch - 1) * g.c_zrow + g.M && g.c_cols >= g.c_col0 + (g.batch - 1) * g.c_zcol + g.N &&
+                (long long)(g.M / 256) * (g.N / 256) * g.batch >= 60;
+    // (its epilogue has the 16-byte paths only)
+    const bool c_vec = g.C && ((uintptr_t)g.C & 15) == 0 && g.ldc % 4 == 0 && g.c_col0 % 4 == 0 && g.c_zcol % 4 == 0 &&
+                       (!g.addend || (((uintptr_t)g.addend & 15) == 0 && g.ldadd % 4 == 0));
+    bool o_vec = g.nout > 0 && g.ldo % 8 == 0 && (g.c_col0 - g.out_col_off) % 8 == 0 && g.c_zcol % 8 == 0;
+    for (int i = 0; i < g.nout; ++i) o_vec = o_vec && (((uintptr_t)g.out[i]) & 15) == 0;
+    pair = pair && (c_vec || !g.C) && (g.nout == 0 || o_vec) && !g.lower_only;
+    const int boxB = pair ? 128 : BN;
     MapCache* cache = (MapCache*)lc.map_cache;
     // distinct operands
     const __nv_bfloat16* da[3];
@@ -562,7 +815,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
         }
         if (ib < 0) {
             if (p.nB == 3) return PKV_ERR_INVALID_ARG;
-            int rc = cached_map(cache, &p.mapB[p.nB], g.B[i].p, g.B[i].rows, g.B[i].cols, g.B[i].ld, BN);
+            int rc = cached_map(cache, &p.mapB[p.nB], g.B[i].p, g.B[i].rows, g.B[i].cols, g.B[i].ld, boxB);
             if (rc != PKV_OK) return rc;
             db[p.nB] = g.B[i].p;
             ib = p.nB++;
@@ -577,7 +830,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
         int end = 0;
         for (int k = 0; k < g.ngrp; ++k) {
             if (g.grp_n[k] <= 0 || g.grp_n[k] % BN != 0) return PKV_ERR_INVALID_ARG;
-            int rc = cached_map(cache, &p.mapB[k], g.Bgrp[k].p, g.Bgrp[k].rows, g.Bgrp[k].cols, g.Bgrp[k].ld, BN);
+            int rc = cached_map(cache, &p.mapB[k], g.Bgrp[k].p, g.Bgrp[k].rows, g.Bgrp[k].cols, g.Bgrp[k].ld, boxB);
             if (rc != PKV_OK) return rc;
             end += g.grp_n[k];
             p.grp_end[k] = end;
@@ -618,6 +871,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
         // every row offset (c_row0 + z c_zrow + ...) * ldo is then a multiple of 8 elements as well
         p.out_vec = ok ? 1 : 0;
     }
+    if (pair) return launch_gemm_pair(lc, p, g.batch);
     if (BN == 64) return launch_gemm<64>(lc, p, g.batch);
     if (BN == 256) return launch_gemm<256>(lc, p, g.batch);
     return launch_gemm<128>(lc, p, g.batch);

@@ -565,6 +565,29 @@ def test_fp32_equivalent_product_and_its_accumulation_bias(B, M, N, K):
     ctx.close()
 
 
+@pytest.mark.parametrize("M,N,K", [(2048, 2048, 512), (4096, 1024, 200), (2048, 2048, 64)])
+def test_product_on_cta_pairs_matches_fp64(B, M, N, K):
+    """Products whose M and N are multiples of 256 and that fill the machine run on pairs of CTAs (256 x 256 tiles,
+    each CTA loading its own half of the operands): against an fp64 product of the same fp32 operands, per 128 x 128
+    block so that a misplaced half tile cannot hide in a norm; ragged K; overwrite and accumulate."""
+    import torch
+    cfg = small_cfg("bf16", hd=128, Hq=16, Hkv=2, d=2048, F=2048, L=256, N=64)
+    ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+    r = np.random.default_rng(33)
+    A = r.standard_normal((M, K)).astype(np.float32)
+    Bm = r.standard_normal((N, K)).astype(np.float32)
+    want = A.astype(np.float64) @ Bm.astype(np.float64).T
+    tA, tB = torch.from_numpy(A).cuda(), torch.from_numpy(Bm).cuda()
+    got = ctx.fp32_product(tA, tB, passes=3, accumulators=1).cpu().numpy().astype(np.float64)
+    blk = np.abs(got - want).reshape(M // 128, 128, N // 128, 128).max(axis=(1, 3)) / np.abs(want).max()
+    assert blk.max() <= 3e-5, (blk.max(), np.unravel_index(blk.argmax(), blk.shape))
+    C0 = r.standard_normal((M, N)).astype(np.float32)
+    tC = torch.from_numpy(C0).cuda()
+    ctx.fp32_product(tA, tB, alpha=-0.5, C_out=tC, accumulate=True, passes=3, accumulators=1)
+    np.testing.assert_allclose(tC.cpu().numpy(), C0 - 0.5 * want, rtol=0, atol=3e-5 * np.abs(want).max())
+    ctx.close()
+
+
 @pytest.mark.parametrize("d,F,n,r", [(256, 192, 500, 32), (128, 128, 60, 8)])
 def test_low_rank_patch_matches_oracle(B, d, F, n, r):
     """Appendix, low-rank weight patches: dW_r = U_r U_r^T dW with U_r the leading eigenvectors of dW S_H dW^T,
