@@ -382,6 +382,9 @@ __global__ void __launch_bounds__(192) k_gemm_tc_pair(const __grid_constant__ Ge
     const int ntn = (int)(gridDim.x >> 1);
     const int tn = (p.k_tri == 1) ? ntn - 1 - (int)(blockIdx.x >> 1) : (int)(blockIdx.x >> 1);
     const int m0 = (int)blockIdx.y * 256 + (int)rank * 128, n0 = tn * BN, z = blockIdx.z;
+    // symmetric products: tiles entirely above the diagonal are not computed (both CTAs of the pair leave together,
+    // before anything is shared between them)
+    if (p.lower_only && tn > (int)blockIdx.y) return;
     const int crow0 = p.c_row0 + z * p.c_zrow + m0, ccol0 = p.c_col0 + z * p.c_zcol + n0;
 
     constexpr int kT = 128 * 64 * 2;                  // every operand tile of a CTA: 128 rows x 64 bf16
@@ -784,18 +787,20 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     // of the SMs once (measured, three-pass products: 4096 x 2048 x 2048 607 vs 449 TFLOP/s executed, 4096 x 1024 x
     // 1024 358 vs 278; the earlier rule asked for two full waves)
     const long long tiles256 = (long long)((g.N + 255) / 256) * ((g.M + 127) / 128) * g.batch;
-    const bool wide = g.N >= 512 && tiles256 >= 120 && !g.lower_only && g.nacc < 4;
-    const int BN = (g.skip_tile00 || g.out_col0_only) ? 128 : ((g.N <= 64) ? 64 : (wide ? 256 : 128));
-    // CTA pairs on 256 x 256 tiles for plain dense products of whole tiles (see k_gemm_tc_pair)
-    bool pair = pair_enabled() && BN == 256 && !lc.pdl && g.M % 256 == 0 && g.N % 256 == 0 && g.a_tri == 0 && g.nacc <= 1 &&
-                !g.stamps && g.c_rows >= g.c_row0 + (g.batch - 1) * g.c_zrow + g.M && g.c_cols >= g.c_col0 + (g.batch - 1) * g.c_zcol + g.N &&
-                (long long)(g.M / 256) * (g.N / 256) * g.batch >= 60;
-    // (its epilogue has the 16-byte paths only)
+    // CTA pairs on 256 x 256 tiles for plain dense products of whole tiles (see k_gemm_tc_pair; its epilogue has the
+    // 16-byte paths only); a lower-triangle-only product counts the tiles on and below the diagonal
     const bool c_vec = g.C && ((uintptr_t)g.C & 15) == 0 && g.ldc % 4 == 0 && g.c_col0 % 4 == 0 && g.c_zcol % 4 == 0 &&
                        (!g.addend || (((uintptr_t)g.addend & 15) == 0 && g.ldadd % 4 == 0));
     bool o_vec = g.nout > 0 && g.ldo % 8 == 0 && (g.c_col0 - g.out_col_off) % 8 == 0 && g.c_zcol % 8 == 0;
     for (int i = 0; i < g.nout; ++i) o_vec = o_vec && (((uintptr_t)g.out[i]) & 15) == 0;
-    pair = pair && (c_vec || !g.C) && (g.nout == 0 || o_vec) && !g.lower_only;
+    const long long tm = g.M / 256, tnn = g.N / 256;
+    const long long pair_tiles = (g.lower_only ? (tm == tnn ? tm * (tm + 1) / 2 : 0) : tm * tnn) * g.batch;
+    const bool pair = pair_enabled() && !lc.pdl && g.M % 256 == 0 && g.N % 256 == 0 && g.N >= 512 && g.a_tri == 0 && g.nacc <= 1 &&
+                      !g.stamps && !g.skip_tile00 && !g.out_col0_only && (!g.lower_only || g.k_tri == 0) &&
+                      g.c_rows >= g.c_row0 + (g.batch - 1) * g.c_zrow + g.M && g.c_cols >= g.c_col0 + (g.batch - 1) * g.c_zcol + g.N &&
+                      pair_tiles >= 60 && (c_vec || !g.C) && (g.nout == 0 || o_vec);
+    const bool wide = g.N >= 512 && tiles256 >= 120 && !g.lower_only && g.nacc < 4;
+    const int BN = pair ? 256 : ((g.skip_tile00 || g.out_col0_only) ? 128 : ((g.N <= 64) ? 64 : (wide ? 256 : 128)));
     const int boxB = pair ? 128 : BN;
     MapCache* cache = (MapCache*)lc.map_cache;
     // distinct operands
