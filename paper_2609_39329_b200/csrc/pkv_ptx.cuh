@@ -87,7 +87,7 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 }
 // The same load issued by a CTA of a pair: the tile still lands in the issuing CTA's shared memory only, but the
 // mbarrier that counts its bytes may be the peer CTA's (given by its address in the cluster's shared window), which
-// is how the leader's MMA thread learns that both halves of a stage are there.  Not a multicast: one destination.
+// is how the leader's MMA thread learns that both halves of a stage are there.  One destination per load.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int c0, int c1) {
     asm volatile(
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"

@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(192) k_gemm_tc(const __grid_constant__ GemmTcP
 
 // ---------------------------------------------------------------------------------------------
 // CTA-pair variant (cta_group::2): a cluster of two CTAs computes one 256 x 256 tile.  Each CTA loads its own 128
-// rows of every A part and its own 128-row half of every B part (no load is shared or multicast), the leader's
+// rows of every A part and its own 128-row half of every B part (every load lands in the issuing CTA only), the leader's
 // single MMA thread issues M = 256, N = 256 instructions that read both CTAs' shared memory, and each CTA's epilogue
 // warps store the 128 rows its tensor memory holds.  Against 128 x 256 tiles of single CTAs this halves the B bytes
 // an SM pulls from L2 per flop (a two-pass stage is 48 KB instead of 64 KB), which is what bounds the long products.
