@@ -997,6 +997,42 @@ def test_alternate_paths_selected_by_environment(env):
         assert "build timeline" in r.stderr
 
 
+_PAIR_CASE = '''
+import sys
+sys.path.insert(0, %r)
+import numpy as np, torch
+from paper_2609_39329_b200 import binding as B
+from tests import test_gpu_parity as T
+cfg = T.small_cfg("bf16", hd=128, Hq=16, Hkv=2, d=2048, F=2048, L=256, N=64)
+ctx = B.PkvContext(B.dims_from_config(cfg), engine=B.ENGINE_AUTO)
+r = np.random.default_rng(34)
+A = r.standard_normal((2048, 320)).astype(np.float32)
+Bm = r.standard_normal((2048, 320)).astype(np.float32)
+got = ctx.fp32_product(torch.from_numpy(A).cuda(), torch.from_numpy(Bm).cuda(), passes=3, accumulators=1).cpu().numpy()
+want = A.astype(np.float64) @ Bm.astype(np.float64).T
+print("PAIR_CASE %%.9e %%s" %% (np.abs(got - want).max() / np.abs(want).max(), got.tobytes()[:64].hex()))
+'''
+
+
+def test_products_agree_with_and_without_cta_pairs():
+    """PKV_GEMM_PAIR=0 sends every product to single CTAs: the same 2048 x 2048 x 320 product in two processes, one per
+    setting, both against fp64 and against each other (same passes in the same order on the same accumulator width:
+    the two kernels give the same bits)."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    outs = []
+    for v in ("1", "0"):
+        r = subprocess.run([sys.executable, "-c", _PAIR_CASE % root], env={**os.environ, "PKV_GEMM_PAIR": v}, capture_output=True,
+                           text=True, timeout=600, cwd=root)
+        assert r.returncode == 0 and "PAIR_CASE" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
+        line = [x for x in r.stdout.splitlines() if x.startswith("PAIR_CASE")][-1].split()
+        assert float(line[1]) <= 3e-5
+        outs.append(line[2])
+    assert outs[0] == outs[1]
+
+
 def test_boundary_rejects_bad_arguments(B):
     import torch
     cfg = small_cfg("bf16")
