@@ -735,9 +735,12 @@ static int launch_gemm(const Lc& lc, GemmTcParams& p, int batch) {
     return PKV_OK;
 }
 
+// PKV_GEMM_PAIR=0 keeps every product on single CTAs; so does a cluster launch that the driver refused once (a
+// device or an SM partition that cannot co-schedule two CTAs of this size).
+static bool g_pair_refused = false;
 static bool pair_enabled() {
     static const bool v = [] { const char* e = getenv("PKV_GEMM_PAIR"); return !e || atoi(e) != 0; }();
-    return v;
+    return v && !g_pair_refused;
 }
 
 static int launch_gemm_pair(const Lc& lc, GemmTcParams& p, int batch) {
@@ -876,7 +879,13 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
         // every row offset (c_row0 + z c_zrow + ...) * ldo is then a multiple of 8 elements as well
         p.out_vec = ok ? 1 : 0;
     }
-    if (pair) return launch_gemm_pair(lc, p, g.batch);
+    if (pair) {
+        const int rc = launch_gemm_pair(lc, p, g.batch);
+        if (rc != PKV_ERR_CUDA) return rc;
+        cudaGetLastError();                 // the launch was refused: nothing ran; from now on single CTAs
+        g_pair_refused = true;
+        return gemm_tc(lc, g, status);
+    }
     if (BN == 64) return launch_gemm<64>(lc, p, g.batch);
     if (BN == 256) return launch_gemm<256>(lc, p, g.batch);
     return launch_gemm<128>(lc, p, g.batch);
