@@ -117,7 +117,7 @@ void make_ridge_matrix(const Lc& lc, const float* S_H, int F, float lam0, int mo
 void sub_f32(const Lc& lc, const float* a, const float* b, int64_t n, float* out);
 // P <- S_T - status->lam * dW - P (n elements), P = dW S_H on entry; status->dw_fro2 (and res_fro2) are reset.
 void refine_residual(const Lc& lc, const float* S_T, const float* dW, float* P, int64_t n, DevStatus* status, bool clear_res);
-// G [F][F] full symmetric from the lower triangle of S [F][F] (G != S).
+// G [F][F] full symmetric from the lower triangle of S [F][F]; G may be S (the upper part is then filled in place).
 void symmetric_from_lower(const Lc& lc, const float* S, float* G, int F);
 void merge_weights(const Lc& lc, void* W, int w_dtype, const float* dW, int64_t count);
 int fma_peak_tflops(cudaStream_t st, float* scratch, size_t scratch_floats, int sm_count, double* tflops);

@@ -817,8 +817,9 @@ void refine_residual(const Lc& lc, const float* S_T, const float* dW, float* P, 
     lc.count(2);
 }
 
-// G (full symmetric) from the lower triangle of S: G[i][j] = S[max(i,j)][min(i,j)].
-__global__ void k_symmetric_from_lower(const float* __restrict__ S, float* __restrict__ G, int F) {
+// G (full symmetric) from the lower triangle of S: G[i][j] = S[max(i,j)][min(i,j)].  G may be S itself (no entry
+// above the diagonal is read).
+__global__ void k_symmetric_from_lower(const float* S, float* G, int F) {
     __shared__ float t[32][33];
     const int bi = blockIdx.y, bj = blockIdx.x;
     if (bj > bi) return;

@@ -531,17 +531,28 @@ void tc_gram(const Lc& lc, TcBuffers* t, const pkv_dims* d, const float* X, cons
     t->stats_f16 = 0;
     transpose_split(lc, X, n, F, t->ldT, t->XT, precise ? t->XT3 : nullptr);
     transpose_split(lc, R, n, dm, t->ldT, t->RT, precise ? t->RT3 : nullptr);
+    // S_H is symmetric: the tiles on and below the diagonal are computed (and, for a running sum, added to), the
+    // upper part is then copied from the lower one, so that the caller still gets the full matrix
+    TcGemm h = plain_gemm(F, F, n, S_H, F, 1.f, nullptr, 0, accumulate);
+    TcGemm g = plain_gemm(dm, F, n, S_T, F, 1.f, nullptr, 0, accumulate);
     if (precise) {
-        TcGemm h = plain_gemm(F, F, n, S_H, F, 1.f, nullptr, 0, accumulate);
         six_pass_stats(h, t->XT, t->XT3, F, t->XT, t->XT3, F, t->ldT, n);
-        gemm_tc(lc, h, status);
-        TcGemm g = plain_gemm(dm, F, n, S_T, F, 1.f, nullptr, 0, accumulate);
         six_pass_stats(g, t->RT, t->RT3, dm, t->XT, t->XT3, F, t->ldT, n);
-        gemm_tc(lc, g, status);
-        return;
+    } else {
+        const Pair hp[2] = {t->XT, t->RT};
+        TcGemm* gs[2] = {&h, &g};
+        const int rows[2] = {F, dm};
+        for (int i = 0; i < 2; ++i) {
+            gs[i]->A[0] = TcMat{hp[i].hi, t->ldT, rows[i], n}; gs[i]->B[0] = TcMat{t->XT.hi, t->ldT, F, n};
+            gs[i]->A[1] = TcMat{hp[i].hi, t->ldT, rows[i], n}; gs[i]->B[1] = TcMat{t->XT.lo, t->ldT, F, n};
+            gs[i]->A[2] = TcMat{hp[i].lo, t->ldT, rows[i], n}; gs[i]->B[2] = TcMat{t->XT.hi, t->ldT, F, n};
+            gs[i]->npass = 3;
+        }
     }
-    gemm_pair_pair(lc, t->XT, t->ldT, t->XT, t->ldT, S_H, F, F, F, n, 1.f, nullptr, 0, accumulate, status);
-    gemm_pair_pair(lc, t->RT, t->ldT, t->XT, t->ldT, S_T, F, dm, F, n, 1.f, nullptr, 0, accumulate, status);
+    h.lower_only = true;
+    gemm_tc(lc, h, status);
+    symmetric_from_lower(lc, S_H, S_H, F);
+    gemm_tc(lc, g, status);
 }
 
 static bool side_stream_on() {
