@@ -400,7 +400,7 @@ def run_stack(args, cfg, B, torch, dist, world, rank, local, peaks):
     work = stage_work(cfg, sum(b_list))
     dom = int(np.argmax(stage_ms))
     name, fl, by, bound = work[dom]
-    dur_ms = s8_timed_schedule if (dom == 7 and s8_timed_schedule > 0) else stage_ms[dom]
+    dur_ms = stage_ms[dom]      # stage times of a stack come from the block-by-block driver's own pass
     dur = dur_ms * 1e-3
     fl *= cfg.n_layers
     if bound == "tensor":
