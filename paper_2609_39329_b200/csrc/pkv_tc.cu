@@ -23,6 +23,23 @@ __device__ __forceinline__ void split2(float v, __nv_bfloat16& hi, __nv_bfloat16
     lo = __float2bfloat16_rn(v - __bfloat162float(hi));
 }
 
+// The element-wise kernels below are bound by HBM: every thread moves four consecutive elements (16-byte loads of
+// fp32, 8-byte stores of bf16 parts).  Row lengths (d, F) are multiples of 8 and every buffer is 16-byte aligned.
+__device__ __forceinline__ uint32_t pack_bf16x2(__nv_bfloat16 a, __nv_bfloat16 b) {
+    return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
+}
+// hi/lo parts of four consecutive values at element index i (a multiple of 4)
+__device__ __forceinline__ void store_pair4(__nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo, size_t i, float4 v) {
+    __nv_bfloat16 h0, h1, h2, h3, l0, l1, l2, l3;
+    split2(v.x, h0, l0); split2(v.y, h1, l1); split2(v.z, h2, l2); split2(v.w, h3, l3);
+    *reinterpret_cast<uint2*>(hi + i) = make_uint2(pack_bf16x2(h0, h1), pack_bf16x2(h2, h3));
+    *reinterpret_cast<uint2*>(lo + i) = make_uint2(pack_bf16x2(l0, l1), pack_bf16x2(l2, l3));
+}
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ void st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ float4 sub4(float4 a, float4 b) { return make_float4(a.x - b.x, a.y - b.y, a.z - b.z, a.w - b.w); }
+__device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+
 // rows [row0, row0 + gridDim.x) of the stacked input (rows [0,N) from x0, rows [N,2N) from x1)
 __global__ void __launch_bounds__(256) k_rmsnorm_split(const float* __restrict__ x0, const float* __restrict__ x1,
                                                        int N, int d, const float* __restrict__ gain, float eps,
@@ -31,10 +48,11 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const float* __restrict__
     __shared__ float red[32];
     int r = blockIdx.x + row0;
     const float* x = (r < N) ? x0 + (size_t)r * d : x1 + (size_t)(r - N) * d;
+    const int d4 = d >> 2;
     float ss = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) {
-        float v = x[c];
-        ss += v * v;
+    for (int c = threadIdx.x; c < d4; c += blockDim.x) {
+        const float4 v = ld4(x + 4 * c);
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
@@ -46,75 +64,72 @@ __global__ void __launch_bounds__(256) k_rmsnorm_split(const float* __restrict__
     }
     __syncthreads();
     float inv = 1.0f / sqrtf(red[0] / (float)d + eps);
-    for (int c = threadIdx.x; c < d; c += blockDim.x) {
-        float v = x[c] * gain[c] * inv;
-        __nv_bfloat16 h, l;
-        split2(v, h, l);
-        hi[(size_t)r * d + c] = h;
-        lo[(size_t)r * d + c] = l;
+    for (int c = threadIdx.x; c < d4; c += blockDim.x) {
+        const float4 v = ld4(x + 4 * c), g = ld4(gain + 4 * c);
+        store_pair4(hi, lo, (size_t)r * d + 4 * c, make_float4(v.x * g.x * inv, v.y * g.y * inv, v.z * g.z * inv, v.w * g.w * inv));
     }
 }
 
 __device__ __forceinline__ float silu_f(float t) { return t / (1.0f + expf(-t)); }
+// silu(gate) * up for four consecutive features of the row a [2F] (gate | up)
+__device__ __forceinline__ float4 swiglu4(const float* __restrict__ a, size_t c, int F) {
+    const float4 g = ld4(a + c), u = ld4(a + F + c);
+    return make_float4(silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w);
+}
 
-// gu [2N][2F] (gate | up) -> hF, hC (fp32 + pairs), dh = hF - hC (pair)
+// gu [2N][2F] (gate | up) -> hF, hC (fp32 + pairs), dh = hF - hC (pair); one thread per four features
 __global__ void __launch_bounds__(256) k_swiglu_split(const float* __restrict__ gu, int N, int F,
                                                       float* __restrict__ hF32, float* __restrict__ hC32, Pair hF,
                                                       Pair hC, Pair dh) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    size_t n = (size_t)N * F;
-    if (i >= n) return;
-    size_t r = i / F, c = i % F;
-    const float* a = gu + r * 2 * F;
-    const float* b = gu + (r + N) * 2 * F;
-    float f = silu_f(a[c]) * a[F + c];
-    float s = silu_f(b[c]) * b[F + c];
-    hF32[i] = f;
-    hC32[i] = s;
-    split2(f, hF.hi[i], hF.lo[i]);
-    split2(s, hC.hi[i], hC.lo[i]);
-    split2(f - s, dh.hi[i], dh.lo[i]);
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i >= (size_t)N * F) return;
+    const size_t r = i / F, c = i % F;
+    const float4 f = swiglu4(gu + r * 2 * F, c, F);
+    const float4 s = swiglu4(gu + (r + N) * 2 * F, c, F);
+    st4(hF32 + i, f);
+    st4(hC32 + i, s);
+    store_pair4(hF.hi, hF.lo, i, f);
+    store_pair4(hC.hi, hC.lo, i, s);
+    store_pair4(dh.hi, dh.lo, i, sub4(f, s));
 }
 
 // teacher half: hF (fp32 + pair) from gu rows [0,N)
 __global__ void __launch_bounds__(256) k_swiglu_teacher(const float* __restrict__ gu, int N, int F,
                                                         float* __restrict__ hF32, Pair hF) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= (size_t)N * F) return;
-    size_t r = i / F, c = i % F;
-    const float* a = gu + r * 2 * F;
-    float f = silu_f(a[c]) * a[F + c];
-    hF32[i] = f;
-    split2(f, hF.hi[i], hF.lo[i]);
+    const size_t r = i / F, c = i % F;
+    const float4 f = swiglu4(gu + r * 2 * F, c, F);
+    st4(hF32 + i, f);
+    store_pair4(hF.hi, hF.lo, i, f);
 }
 // student half: hC (fp32 + pair) from gu rows [N,2N), dh = hF - hC (pair) with the teacher's hF
 __global__ void __launch_bounds__(256) k_swiglu_student(const float* __restrict__ gu, int N, int F,
                                                         const float* __restrict__ hF32, float* __restrict__ hC32,
                                                         Pair hC, Pair dh) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= (size_t)N * F) return;
-    size_t r = i / F, c = i % F;
-    const float* b = gu + (r + N) * 2 * F;
-    float s = silu_f(b[c]) * b[F + c];
-    hC32[i] = s;
-    split2(s, hC.hi[i], hC.lo[i]);
-    split2(hF32[i] - s, dh.hi[i], dh.lo[i]);
+    const size_t r = i / F, c = i % F;
+    const float4 s = swiglu4(gu + (r + N) * 2 * F, c, F);
+    st4(hC32 + i, s);
+    store_pair4(hC.hi, hC.lo, i, s);
+    store_pair4(dh.hi, dh.lo, i, sub4(ld4(hF32 + i), s));
 }
-// teacher half of the o-projection epilogue: zF = xF + o[0:N]
+// teacher half of the o-projection epilogue: zF = xF + o[0:N]   (n elements, four per thread)
 __global__ void k_oproj_teacher(const float* __restrict__ xF, const float* __restrict__ o, size_t n,
                                 float* __restrict__ zF) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) zF[i] = xF[i] + o[i];
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+    if (i < n) st4(zF + i, add4(ld4(xF + i), ld4(o + i)));
 }
 // student half: dz = dx + o[N:2N] (dx = xF - xC entering the block, o[N:2N] the projection of dA); zC = zF - dz
 __global__ void k_oproj_student(const float* __restrict__ dx, const float* __restrict__ o,
                                 const float* __restrict__ zF, size_t n, float* __restrict__ zC,
                                 float* __restrict__ dz) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= n) return;
-    float dd = dx[i] + o[n + i];
-    dz[i] = dd;
-    zC[i] = zF[i] - dd;
+    const float4 dd = add4(ld4(dx + i), ld4(o + n + i));
+    st4(dz + i, dd);
+    st4(zC + i, sub4(ld4(zF + i), dd));
 }
 
 // teacher half after the student's: dz = (xF - xC) + o[0:N] (the projection of dA), zF = zC + dz; dx, if given, is
@@ -123,24 +138,23 @@ __global__ void k_oproj_teacher_diff(const float* __restrict__ xF, const float* 
                                      const float* __restrict__ dx, const float* __restrict__ o,
                                      const float* __restrict__ zC, size_t n, float* __restrict__ zF,
                                      float* __restrict__ dz) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= n) return;
-    float dd = (dx ? dx[i] : xF[i] - xC[i]) + o[i];
-    dz[i] = dd;
-    zF[i] = zC[i] + dd;
+    const float4 dd = add4(dx ? ld4(dx + i) : sub4(ld4(xF + i), ld4(xC + i)), ld4(o + i));
+    st4(dz + i, dd);
+    st4(zF + i, add4(ld4(zC + i), dd));
 }
 // teacher half after the student's: hF (fp32 + pair) from gu rows [0,N), dh = hF - hC (pair) with the student's hC
 __global__ void __launch_bounds__(256) k_swiglu_teacher_diff(const float* __restrict__ gu, int N, int F,
                                                              const float* __restrict__ hC32, float* __restrict__ hF32,
                                                              Pair hF, Pair dh) {
-    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
     if (i >= (size_t)N * F) return;
-    size_t r = i / F, c = i % F;
-    const float* a = gu + r * 2 * F;
-    float f = silu_f(a[c]) * a[F + c];
-    hF32[i] = f;
-    split2(f, hF.hi[i], hF.lo[i]);
-    split2(f - hC32[i], dh.hi[i], dh.lo[i]);
+    const size_t r = i / F, c = i % F;
+    const float4 f = swiglu4(gu + r * 2 * F, c, F);
+    st4(hF32 + i, f);
+    store_pair4(hF.hi, hF.lo, i, f);
+    store_pair4(dh.hi, dh.lo, i, sub4(f, ld4(hC32 + i)));
 }
 
 // in [rows][cols] fp32 -> out pair [cols][ldo] (token-contiguous operands of the statistics)
@@ -705,7 +719,7 @@ int tc_teacher_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     if ((rc = gemm_act_weight(lc, t->a, Dq, w->Wo, Dq, t->o, d, N, d, Dq, 1.f, nullptr, 0, st))) return rc;
     {
         size_t n = (size_t)N * d;
-        k_oproj_teacher<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(a.xF, t->o, n, a.zF);
+        k_oproj_teacher<<<(unsigned)((n / 4 + 255) / 256), 256, 0, lc.st>>>(a.xF, t->o, n, a.zF);
         lc.count();
     }
     markT(3);
@@ -718,7 +732,7 @@ int tc_teacher_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     }
     {
         size_t n = (size_t)N * F;
-        k_swiglu_teacher<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, t->hF);
+        k_swiglu_teacher<<<(unsigned)((n / 4 + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, t->hF);
         lc.count();
     }
     markT(4);
@@ -755,7 +769,7 @@ int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     if ((rc = gemm_act_weight(lc, aS, Dq, w->Wo, Dq, t->o + uo, d, N, d, Dq, 1.f, nullptr, 0, st))) return rc;
     {
         size_t n = (size_t)N * d;
-        k_oproj_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(a.dx, t->o, a.zF, n, a.zC, a.dz);
+        k_oproj_student<<<(unsigned)((n / 4 + 255) / 256), 256, 0, lc.st>>>(a.dx, t->o, a.zF, n, a.zC, a.dz);
         lc.count();
     }
     mark(a, lc, 4);
@@ -769,7 +783,7 @@ int tc_student_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcFo
     }
     {
         size_t n = (size_t)N * F;
-        k_swiglu_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hC, t->dh);
+        k_swiglu_student<<<(unsigned)((n / 4 + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hC, t->dh);
         lc.count();
     }
     mark(a, lc, 5);
@@ -806,7 +820,7 @@ int tc_student_propagate(const Lc& lc, TcBuffers* t, const pkv_dims* D, const Tc
     if ((rc = gemm_act_weight(lc, aS, Dq, w->Wo, Dq, t->o + uo, d, N, d, Dq, 1.f, nullptr, 0, st))) return rc;
     {
         size_t n = (size_t)N * d;
-        k_oproj_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(zero_nd, t->o, a.xC, n, a.zC, a.dz);
+        k_oproj_student<<<(unsigned)((n / 4 + 255) / 256), 256, 0, lc.st>>>(zero_nd, t->o, a.xC, n, a.zC, a.dz);
         lc.count();
     }
     k_rmsnorm_split<<<N, 256, 0, lc.st>>>(a.zC, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, N);
@@ -819,7 +833,7 @@ int tc_student_propagate(const Lc& lc, TcBuffers* t, const pkv_dims* D, const Tc
     }
     {
         size_t n = (size_t)N * F;
-        k_swiglu_student<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hC, t->dh);
+        k_swiglu_student<<<(unsigned)((n / 4 + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hC, t->dh);
         lc.count();
     }
     // xC_next = z' + h' W^T + h' dW^T
@@ -872,7 +886,7 @@ int tc_forward(const Lc& lc, TcBuffers* t, const pkv_dims* D, const TcForwardArg
     }
     {
         size_t n = (size_t)N * F;
-        k_swiglu_split<<<(unsigned)((n + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hF, t->hC, t->dh);
+        k_swiglu_split<<<(unsigned)((n / 4 + 255) / 256), 256, 0, lc.st>>>(t->gu, N, F, a.hF, a.hC, t->hF, t->hC, t->dh);
         lc.count();
     }
     mark(a, lc, 5);
@@ -935,7 +949,7 @@ int tc_forward_overlapped(const Lc& lc, TcBuffers* t, const pkv_dims* D, const T
         cudaEventRecord(t->evq[1], lf.st);
         Pair aS{t->a.hi + (size_t)N * Dq, t->a.lo + (size_t)N * Dq};
         if ((rc = gemm_act_weight(lf, aS, Dq, w->Wo, Dq, t->o + uo, d, N, d, Dq, 1.f, nullptr, 0, st))) return rc;
-        k_oproj_teacher<<<(unsigned)((uo + 255) / 256), 256, 0, lf.st>>>(a.xC, t->o + uo, uo, a.zC);      // zC = xC + aC Wo^T
+        k_oproj_teacher<<<(unsigned)((uo / 4 + 255) / 256), 256, 0, lf.st>>>(a.xC, t->o + uo, uo, a.zC);      // zC = xC + aC Wo^T
         lf.count();
         cudaEventRecord(t->evq[2], lf.st);
         k_rmsnorm_split<<<N, 256, 0, lf.st>>>(a.zC, a.zC, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, N);
@@ -943,7 +957,7 @@ int tc_forward_overlapped(const Lc& lc, TcBuffers* t, const pkv_dims* D, const T
         float* guS = t->gu + (size_t)N * 2 * F;
         if ((rc = gemm_act_weights(lf, uS, d, Wgu, wgu, 2, d, guS, 2 * F, N, d, st))) return rc;
         const size_t n = (size_t)N * F;
-        k_swiglu_teacher<<<(unsigned)((n + 255) / 256), 256, 0, lf.st>>>(guS, N, F, a.hC, t->hC);
+        k_swiglu_teacher<<<(unsigned)((n / 4 + 255) / 256), 256, 0, lf.st>>>(guS, N, F, a.hC, t->hC);
         lf.count();
         cudaEventRecord(t->evq[3], lf.st);
         stats_operand(lf, t, a.hC, N, F, 0, precise);
@@ -973,7 +987,7 @@ int tc_forward_overlapped(const Lc& lc, TcBuffers* t, const pkv_dims* D, const T
         if (rc == PKV_OK) {
             const size_t n = (size_t)N * d;
             cudaStreamWaitEvent(ls.st, t->evq[2], 0);
-            k_oproj_teacher_diff<<<(unsigned)((n + 255) / 256), 256, 0, ls.st>>>(a.xF, a.xC, a.dx, t->o, a.zC, n, a.zF, a.dz);
+            k_oproj_teacher_diff<<<(unsigned)((n / 4 + 255) / 256), 256, 0, ls.st>>>(a.xF, a.xC, a.dx, t->o, a.zC, n, a.zF, a.dz);
             ls.count();
             k_rmsnorm_split<<<N, 256, 0, ls.st>>>(a.zF, a.zF, N, d, w->g_mlp, D->eps, t->u.hi, t->u.lo, 0);
             ls.count();
@@ -982,7 +996,7 @@ int tc_forward_overlapped(const Lc& lc, TcBuffers* t, const pkv_dims* D, const T
         if (rc == PKV_OK) {
             const size_t n = (size_t)N * F;
             cudaStreamWaitEvent(ls.st, t->evq[3], 0);
-            k_swiglu_teacher_diff<<<(unsigned)((n + 255) / 256), 256, 0, ls.st>>>(t->gu, N, F, a.hC, a.hF, t->hF, t->dh);
+            k_swiglu_teacher_diff<<<(unsigned)((n / 4 + 255) / 256), 256, 0, ls.st>>>(t->gu, N, F, a.hC, a.hF, t->hF, t->dh);
             ls.count();
             // S6 (Eq. 5), S_T (Eq. 9)
             rc = gemm_act_weight(ls, t->dh, F, w->Wdown, F, a.R, d, N, d, F, 1.f, a.dz, d, st);
