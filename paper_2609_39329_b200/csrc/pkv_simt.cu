@@ -488,8 +488,54 @@ void attention_simt(const Lc& lc, const AttnArgs& a) {
 }
 
 // Split-K combine and residual epilogue: one warp per (kv head, query row); merges the
-// (m, l, O) partials of each stream and writes aF, aC and dA = aF - aC in fp32.
+// (m, l, O) partials of each stream and writes aF, aC and dA = aF - aC in fp32.  A lane owns PER = hd / 32
+// consecutive columns and moves them as one vector (16 bytes of fp32 at hd = 128, 8 bytes of bf16 parts).
+template <int PER>
+struct VecF;
+template <>
+struct VecF<4> {
+    static __device__ __forceinline__ void ld(const float* p, float (&v)[4]) {
+        const float4 t = *reinterpret_cast<const float4*>(p);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+    static __device__ __forceinline__ void st(float* p, const float (&v)[4]) {
+        *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+    static __device__ __forceinline__ void st_pair(__nv_bfloat16* hi, __nv_bfloat16* lo, const float (&v)[4]) {
+        unsigned short h[4], l[4];
+        for (int c = 0; c < 4; ++c) {
+            const __nv_bfloat16 hh = __float2bfloat16_rn(v[c]);
+            h[c] = __bfloat16_as_ushort(hh);
+            l[c] = __bfloat16_as_ushort(__float2bfloat16_rn(v[c] - __bfloat162float(hh)));
+        }
+        *reinterpret_cast<uint2*>(hi) = make_uint2(h[0] | ((unsigned)h[1] << 16), h[2] | ((unsigned)h[3] << 16));
+        *reinterpret_cast<uint2*>(lo) = make_uint2(l[0] | ((unsigned)l[1] << 16), l[2] | ((unsigned)l[3] << 16));
+    }
+};
+template <>
+struct VecF<2> {
+    static __device__ __forceinline__ void ld(const float* p, float (&v)[2]) {
+        const float2 t = *reinterpret_cast<const float2*>(p);
+        v[0] = t.x; v[1] = t.y;
+    }
+    static __device__ __forceinline__ void st(float* p, const float (&v)[2]) {
+        *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]);
+    }
+    static __device__ __forceinline__ void st_pair(__nv_bfloat16* hi, __nv_bfloat16* lo, const float (&v)[2]) {
+        unsigned short h[2], l[2];
+        for (int c = 0; c < 2; ++c) {
+            const __nv_bfloat16 hh = __float2bfloat16_rn(v[c]);
+            h[c] = __bfloat16_as_ushort(hh);
+            l[c] = __bfloat16_as_ushort(__float2bfloat16_rn(v[c] - __bfloat162float(hh)));
+        }
+        *reinterpret_cast<unsigned*>(hi) = h[0] | ((unsigned)h[1] << 16);
+        *reinterpret_cast<unsigned*>(lo) = l[0] | ((unsigned)l[1] << 16);
+    }
+};
+
+template <int PER>
 __global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
+    using V = VecF<PER>;
     int g = a.Hq / a.Hkv;
     int rows = a.N * g;
     int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -497,77 +543,61 @@ __global__ void __launch_bounds__(256) k_attn_combine(AttnArgs a) {
     if (w >= a.Hkv * rows) return;
     int kh = w / rows, r = w % rows;
     int tok = r / g, hg = r % g;
-    int hd = a.hd;
-    int per = hd / 32;                       // 2 or 4 columns per lane
-    float res[2][4];
-    const size_t o = (size_t)tok * a.Hq * hd + (size_t)(kh * g + hg) * hd + lane * per;
-    if (a.mode == 2 && !a.student_first) {      // the teacher's output was produced earlier
-        for (int c = 0; c < per; ++c) res[0][c] = a.aF[o + c];
-    }
+    constexpr int hd = PER * 32;
+    float res[2][PER];
+    const size_t o = (size_t)tok * a.Hq * hd + (size_t)(kh * g + hg) * hd + lane * PER;
+    const size_t o2 = o + (size_t)a.N * a.Hq * hd;      // the same entry of rows [N,2N) of the stacked pair
+    if (a.mode == 2 && !a.student_first) V::ld(a.aF + o, res[0]);      // the teacher's output was produced earlier
     for (int s = (a.mode == 2 ? 1 : 0); s < (a.mode == 1 ? 1 : 2); ++s) {
         int z0 = s ? a.zoffC : 0;
         int ns = s ? a.nsplitC : a.nsplitF;
         float M = -INFINITY;
         for (int i = 0; i < ns; ++i) M = fmaxf(M, a.part_m[((size_t)(z0 + i) * a.Hkv + kh) * rows + r]);
-        float den = 0.f, num[4] = {0.f, 0.f, 0.f, 0.f};
+        float den = 0.f, num[PER];
+#pragma unroll
+        for (int c = 0; c < PER; ++c) num[c] = 0.f;
         for (int i = 0; i < ns; ++i) {
             size_t pr = ((size_t)(z0 + i) * a.Hkv + kh) * rows + r;
             float mi = a.part_m[pr];
             if (mi == -INFINITY) continue;
             float wgt = expf(mi - M);
             den += wgt * a.part_l[pr];
-            const float* po = a.part_O + pr * hd + lane * per;
-            for (int c = 0; c < per; ++c) num[c] += wgt * po[c];
+            float po[PER];
+            V::ld(a.part_O + pr * hd + lane * PER, po);
+#pragma unroll
+            for (int c = 0; c < PER; ++c) num[c] += wgt * po[c];
         }
         float inv = (den > 0.f) ? 1.f / den : 0.f;
-        for (int c = 0; c < per; ++c) res[s][c] = num[c] * inv;
+#pragma unroll
+        for (int c = 0; c < PER; ++c) res[s][c] = num[c] * inv;
     }
     if (a.student_first) {
-        for (int c = 0; c < per; ++c) {
-            if (a.mode == 2) {          // student alone: aC and its pair in rows [N,2N)
-                const float v = res[1][c];
-                a.aC[o + c] = v;
-                if (a.pair_hi) {
-                    const size_t o2 = o + c + (size_t)a.N * a.Hq * hd;
-                    __nv_bfloat16 h = __float2bfloat16_rn(v);
-                    a.pair_hi[o2] = h;
-                    a.pair_lo[o2] = __float2bfloat16_rn(v - __bfloat162float(h));
-                }
-            } else {                    // teacher after the student: aF, dA = aF - aC, pair of dA in rows [0,N)
-                const float f = res[0][c];
-                const float dd = f - a.aC[o + c];
-                a.aF[o + c] = f;
-                a.dA[o + c] = dd;
-                if (a.pair_hi) {
-                    __nv_bfloat16 h = __float2bfloat16_rn(dd);
-                    a.pair_hi[o + c] = h;
-                    a.pair_lo[o + c] = __float2bfloat16_rn(dd - __bfloat162float(h));
-                }
-            }
+        if (a.mode == 2) {          // student alone: aC and its pair in rows [N,2N)
+            V::st(a.aC + o, res[1]);
+            if (a.pair_hi) V::st_pair(a.pair_hi + o2, a.pair_lo + o2, res[1]);
+        } else {                    // teacher after the student: aF, dA = aF - aC, pair of dA in rows [0,N)
+            float ac[PER], dd[PER];
+            V::ld(a.aC + o, ac);
+#pragma unroll
+            for (int c = 0; c < PER; ++c) dd[c] = res[0][c] - ac[c];
+            V::st(a.aF + o, res[0]);
+            V::st(a.dA + o, dd);
+            if (a.pair_hi) V::st_pair(a.pair_hi + o, a.pair_lo + o, dd);
         }
         return;
     }
-    for (int c = 0; c < per; ++c) {
-        const float f = res[0][c];
-        if (a.mode != 2) {
-            a.aF[o + c] = f;
-            if (a.pair_hi) {    // operands of the o-projection: rows [0,N) aF, rows [N,2N) dA
-                __nv_bfloat16 h = __float2bfloat16_rn(f);
-                a.pair_hi[o + c] = h;
-                a.pair_lo[o + c] = __float2bfloat16_rn(f - __bfloat162float(h));
-            }
-        }
-        if (a.mode != 1) {
-            const float dd = f - res[1][c];
-            a.aC[o + c] = res[1][c];
-            a.dA[o + c] = dd;
-            if (a.pair_hi) {
-                const size_t o2 = o + c + (size_t)a.N * a.Hq * hd;
-                __nv_bfloat16 h = __float2bfloat16_rn(dd);
-                a.pair_hi[o2] = h;
-                a.pair_lo[o2] = __float2bfloat16_rn(dd - __bfloat162float(h));
-            }
-        }
+    if (a.mode != 2) {
+        V::st(a.aF + o, res[0]);
+        // operands of the o-projection: rows [0,N) aF, rows [N,2N) dA
+        if (a.pair_hi) V::st_pair(a.pair_hi + o, a.pair_lo + o, res[0]);
+    }
+    if (a.mode != 1) {
+        float dd[PER];
+#pragma unroll
+        for (int c = 0; c < PER; ++c) dd[c] = res[0][c] - res[1][c];
+        V::st(a.aC + o, res[1]);
+        V::st(a.dA + o, dd);
+        if (a.pair_hi) V::st_pair(a.pair_hi + o2, a.pair_lo + o2, dd);
     }
 }
 
@@ -575,7 +605,8 @@ void attention_combine(const Lc& lc, const AttnArgs& a) {
     int g = a.Hq / a.Hkv;
     long long warps = (long long)a.Hkv * a.N * g;
     if (a.combine_wait) cudaStreamWaitEvent(lc.st, (cudaEvent_t)a.combine_wait, 0);
-    k_attn_combine<<<(unsigned)((warps + 7) / 8), 256, 0, lc.st>>>(a);
+    if (a.hd == 128) k_attn_combine<4><<<(unsigned)((warps + 7) / 8), 256, 0, lc.st>>>(a);
+    else k_attn_combine<2><<<(unsigned)((warps + 7) / 8), 256, 0, lc.st>>>(a);
     lc.count();
 }
 
