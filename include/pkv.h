@@ -278,7 +278,7 @@ int pkv_dequant_cache(pkv_ctx* ctx, const pkv_kv_compressed* cb, void* Kc, void*
 
 /* Dual-cache attention alone (Sec. 2.2, teacher and student forward passes over the reference
  * tokens).  q: device fp32 [2][N][Hq*hd] rotated queries of the teacher (0) and student (1)
- * stream; k_new, v_new: device fp32 [2][N][Hkv*hd] the reference tokens' own keys/values.
+ * stream; k_new, v_new: device fp32 [2][N][Hkv*hd] the reference tokens' own keys/values (all 16-byte aligned).
  * Outputs device fp32 [N][Hq*hd], 16-byte aligned: aF, aC and dA = aF - aC (formed before any rounding). */
 int pkv_attention(pkv_ctx* ctx, const float* q, const float* k_new, const float* v_new,
                   const pkv_kv* full, const pkv_kv_compressed* cb, int32_t N, int32_t n_chunks,

@@ -1289,7 +1289,9 @@ extern "C" int pkv_attention(pkv_ctx* c, const float* q, const float* k_new, con
                              const pkv_kv* full, const pkv_kv_compressed* cb, int32_t N, int32_t n_chunks,
                              const int32_t* chunk_off, float* aF, float* aC, float* dA) {
     if (!c || !q || !k_new || !v_new || !full || !cb || !aF || !aC || !dA) return PKV_ERR_INVALID_ARG;
-    if (((uintptr_t)aF & 15) || ((uintptr_t)aC & 15) || ((uintptr_t)dA & 15)) return PKV_ERR_INVALID_ARG;      // vector stores
+    const void* vec_ptrs[] = {q, k_new, v_new, aF, aC, dA};      // 16-byte loads and stores
+    for (const void* vp : vec_ptrs)
+        if ((uintptr_t)vp & 15) return PKV_ERR_INVALID_ARG;
     int rc = check_chunks(c, N, n_chunks, chunk_off);
     if (rc != PKV_OK) return rc;
     int total = 0, max_b = 0;

@@ -36,6 +36,16 @@ using namespace ptx;
 // ---------------------------------------------------------------------------------------------
 // q  -> hi/lo [2][Hkv][N*g][hd] (row = token*g + head-in-group), scaled by log2(e)/sqrt(hd)
 // k,v-> bf16  [2][Hkv][N][hd]
+// One thread per four consecutive rotation pairs (c .. c+3 and their partners at + hd/2): 16-byte loads, 8-byte
+// stores.  All row strides are multiples of 4 floats and every base pointer is 16-byte aligned.
+__device__ __forceinline__ uint2 pack4_f16(float a, float b, float c, float d) {
+    const __half2 x = __floats2half2_rn(a, b), y = __floats2half2_rn(c, d);
+    return make_uint2(*reinterpret_cast<const uint32_t*>(&x), *reinterpret_cast<const uint32_t*>(&y));
+}
+__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
+    const __nv_bfloat162 x = __floats2bfloat162_rn(a, b), y = __floats2bfloat162_rn(c, d);
+    return make_uint2(*reinterpret_cast<const uint32_t*>(&x), *reinterpret_cast<const uint32_t*>(&y));
+}
 __global__ void __launch_bounds__(256) k_attn_prep(const float* __restrict__ q, long long ldq,
                                                    const float* __restrict__ k, const float* __restrict__ v,
                                                    long long ldkv, const float* __restrict__ rope_tab, int N, int Hq,
@@ -43,59 +53,78 @@ __global__ void __launch_bounds__(256) k_attn_prep(const float* __restrict__ q, 
                                                    __nv_bfloat16* __restrict__ qhi,
                                                    __nv_bfloat16* __restrict__ qlo, __nv_bfloat16* __restrict__ kn,
                                                    __nv_bfloat16* __restrict__ vn) {
-    const int half = hd / 2;
+    const int half = hd / 2, quads = half / 4;
     const int heads = Hq + 2 * Hkv;
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    size_t total = (size_t)s_count * N * heads * half;
+    size_t total = (size_t)s_count * N * heads * quads;
     if (i >= total) return;
-    int c = (int)(i % half);
-    int h = (int)((i / half) % heads);
-    int row = (int)(i / ((size_t)half * heads)) + s_begin * N;
+    int c = (int)(i % quads) * 4;
+    int h = (int)((i / quads) % heads);
+    int row = (int)(i / ((size_t)quads * heads)) + s_begin * N;
     int s = row / N, tok = row % N;
-    float co = 1.f, si = 0.f;
-    if (rope_tab) {
-        co = rope_tab[2 * ((size_t)tok * half + c)];
-        si = rope_tab[2 * ((size_t)tok * half + c) + 1];
+    float co[4] = {1.f, 1.f, 1.f, 1.f}, si[4] = {0.f, 0.f, 0.f, 0.f};
+    if (rope_tab) {      // (cos, sin) interleaved per pair
+        const float4 t0 = *reinterpret_cast<const float4*>(rope_tab + 2 * ((size_t)tok * half + c));
+        const float4 t1 = *reinterpret_cast<const float4*>(rope_tab + 2 * ((size_t)tok * half + c) + 4);
+        co[0] = t0.x; si[0] = t0.y; co[1] = t0.z; si[1] = t0.w;
+        co[2] = t1.x; si[2] = t1.y; co[3] = t1.z; si[3] = t1.w;
     }
     if (h < Hq) {
         const int g = Hq / Hkv;
         const float* p = q + (size_t)row * ldq + (size_t)h * hd + c;
-        float lo = p[0], hi = p[half];
+        const float4 l4 = *reinterpret_cast<const float4*>(p), h4 = *reinterpret_cast<const float4*>(p + half);
+        const float lo[4] = {l4.x, l4.y, l4.z, l4.w}, hi[4] = {h4.x, h4.y, h4.z, h4.w};
         const float sc = 1.4426950408889634f * rsqrtf((float)hd);
-        float a = (lo * co - hi * si) * sc, b = (hi * co + lo * si) * sc;
+        float a[4], b[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            a[e] = (lo[e] * co[e] - hi[e] * si[e]) * sc;
+            b[e] = (hi[e] * co[e] + lo[e] * si[e]) * sc;
+        }
         int kh = h / g, hg = h % g;
         size_t o = (((size_t)s * Hkv + kh) * ((size_t)N * g) + (size_t)tok * g + hg) * hd + c;
         if (q_f16) {
-            // one fp16 part (11 significant bits): the attention kernel multiplies it with the bf16 keys in one pass
-            __half* qh = reinterpret_cast<__half*>(qhi);
-            qh[o] = __float2half_rn(a);
-            qh[o + half] = __float2half_rn(b);
+            // one fp16 part (11 significant bits): the attention kernel multiplies it with the fp16 keys in one pass
+            *reinterpret_cast<uint2*>(qhi + o) = pack4_f16(a[0], a[1], a[2], a[3]);
+            *reinterpret_cast<uint2*>(qhi + o + half) = pack4_f16(b[0], b[1], b[2], b[3]);
         } else {
-            __nv_bfloat16 ah = __float2bfloat16_rn(a), bh = __float2bfloat16_rn(b);
-            qhi[o] = ah;
-            qhi[o + half] = bh;
-            qlo[o] = __float2bfloat16_rn(a - __bfloat162float(ah));
-            qlo[o + half] = __float2bfloat16_rn(b - __bfloat162float(bh));
+            float ar[4], br[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                ar[e] = a[e] - __bfloat162float(__float2bfloat16_rn(a[e]));
+                br[e] = b[e] - __bfloat162float(__float2bfloat16_rn(b[e]));
+            }
+            *reinterpret_cast<uint2*>(qhi + o) = pack4_bf16(a[0], a[1], a[2], a[3]);
+            *reinterpret_cast<uint2*>(qhi + o + half) = pack4_bf16(b[0], b[1], b[2], b[3]);
+            *reinterpret_cast<uint2*>(qlo + o) = pack4_bf16(ar[0], ar[1], ar[2], ar[3]);
+            *reinterpret_cast<uint2*>(qlo + o + half) = pack4_bf16(br[0], br[1], br[2], br[3]);
         }
     } else if (h < Hq + Hkv) {
         int kh = h - Hq;
         const float* p = k + (size_t)row * ldkv + (size_t)kh * hd + c;
-        float lo = p[0], hi = p[half];
+        const float4 l4 = *reinterpret_cast<const float4*>(p), h4 = *reinterpret_cast<const float4*>(p + half);
+        const float lo[4] = {l4.x, l4.y, l4.z, l4.w}, hi[4] = {h4.x, h4.y, h4.z, h4.w};
+        float a[4], b[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            a[e] = lo[e] * co[e] - hi[e] * si[e];
+            b[e] = hi[e] * co[e] + lo[e] * si[e];
+        }
         size_t o = (((size_t)s * Hkv + kh) * N + tok) * hd + c;
         if (q_f16) {
-            __half* kh16 = reinterpret_cast<__half*>(kn);
-            kh16[o] = __float2half_rn(lo * co - hi * si);
-            kh16[o + half] = __float2half_rn(hi * co + lo * si);
+            *reinterpret_cast<uint2*>(kn + o) = pack4_f16(a[0], a[1], a[2], a[3]);
+            *reinterpret_cast<uint2*>(kn + o + half) = pack4_f16(b[0], b[1], b[2], b[3]);
         } else {
-            kn[o] = __float2bfloat16_rn(lo * co - hi * si);
-            kn[o + half] = __float2bfloat16_rn(hi * co + lo * si);
+            *reinterpret_cast<uint2*>(kn + o) = pack4_bf16(a[0], a[1], a[2], a[3]);
+            *reinterpret_cast<uint2*>(kn + o + half) = pack4_bf16(b[0], b[1], b[2], b[3]);
         }
     } else {
         int kh = h - Hq - Hkv;
         const float* p = v + (size_t)row * ldkv + (size_t)kh * hd + c;
+        const float4 l4 = *reinterpret_cast<const float4*>(p), h4 = *reinterpret_cast<const float4*>(p + half);
         size_t o = (((size_t)s * Hkv + kh) * N + tok) * hd + c;
-        vn[o] = __float2bfloat16_rn(p[0]);
-        vn[o + half] = __float2bfloat16_rn(p[half]);
+        *reinterpret_cast<uint2*>(vn + o) = pack4_bf16(l4.x, l4.y, l4.z, l4.w);
+        *reinterpret_cast<uint2*>(vn + o + half) = pack4_bf16(h4.x, h4.y, h4.z, h4.w);
     }
 }
 
@@ -688,7 +717,7 @@ int attention_tc(const Lc& lc, TcBuffers* t, const pkv_dims* d, const AttnArgs& 
     const int rows = N * g;
     const int s_begin = (a.mode == 2) ? 1 : 0, s_count = (a.mode == 0) ? 2 : 1;
     {
-        size_t total = (size_t)s_count * N * (d->Hq + 2 * Hkv) * (hd / 2);
+        size_t total = (size_t)s_count * N * (d->Hq + 2 * Hkv) * (hd / 8);      // four rotation pairs per thread
         k_attn_prep<<<(unsigned)((total + 255) / 256), 256, 0, lc.st>>>(a.q, a.ldq, a.k_new, a.v_new, a.ldkv, rope_tab, N,
                                                                         d->Hq, Hkv, hd, s_begin, s_count,
                                                                         (hd == 128 && attn_q_f16()) ? 1 : 0, t->q.hi, t->q.lo,
