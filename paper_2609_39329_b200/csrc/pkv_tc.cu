@@ -157,25 +157,38 @@ __global__ void __launch_bounds__(256) k_swiglu_teacher_diff(const float* __rest
     store_pair4(dh.hi, dh.lo, i, sub4(f, ld4(hC32 + i)));
 }
 
-// in [rows][cols] fp32 -> out pair [cols][ldo] (token-contiguous operands of the statistics)
+// in [rows][cols] fp32 -> out pair [cols][ldo] (token-contiguous operands of the statistics).  A block transposes a
+// tile of 64 rows x 32 columns; on the way out a thread stores two consecutive tokens of one feature (4 bytes).
+// ldo is even, and rows beyond the matrix are left alone (their bytes are never read: the contraction stops at n).
 __global__ void k_transpose_split(const float* __restrict__ in, int rows, int cols, int ldo, Pair out,
                                   __nv_bfloat16* __restrict__ out3) {
-    __shared__ float t[32][33];
-    int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-    for (int j = threadIdx.y; j < 32; j += 8) {
+    __shared__ float t[64][33];
+    int c0 = blockIdx.x * 32, r0 = blockIdx.y * 64;
+    for (int j = threadIdx.y; j < 64; j += 8) {
         int r = r0 + j, c = c0 + threadIdx.x;
-        if (r < rows && c < cols) t[j][threadIdx.x] = in[(size_t)r * cols + c];
+        t[j][threadIdx.x] = (r < rows && c < cols) ? in[(size_t)r * cols + c] : 0.f;
     }
     __syncthreads();
     for (int j = threadIdx.y; j < 32; j += 8) {
-        int c = c0 + j, r = r0 + threadIdx.x;
+        int c = c0 + j, r = r0 + 2 * threadIdx.x;
         if (r < rows && c < cols) {
-            __nv_bfloat16 h, l;
-            const float v = t[threadIdx.x][j];
-            split2(v, h, l);
-            out.hi[(size_t)c * ldo + r] = h;
-            out.lo[(size_t)c * ldo + r] = l;
-            if (out3) out3[(size_t)c * ldo + r] = __float2bfloat16_rn((v - __bfloat162float(h)) - __bfloat162float(l));
+            const float v0 = t[2 * threadIdx.x][j], v1 = t[2 * threadIdx.x + 1][j];
+            __nv_bfloat16 h0, l0, h1, l1;
+            split2(v0, h0, l0);
+            split2(v1, h1, l1);
+            const size_t o = (size_t)c * ldo + r;
+            if (r + 1 < rows) {
+                *reinterpret_cast<uint32_t*>(out.hi + o) = pack_bf16x2(h0, h1);
+                *reinterpret_cast<uint32_t*>(out.lo + o) = pack_bf16x2(l0, l1);
+                if (out3)
+                    *reinterpret_cast<uint32_t*>(out3 + o) =
+                        pack_bf16x2(__float2bfloat16_rn((v0 - __bfloat162float(h0)) - __bfloat162float(l0)),
+                                    __float2bfloat16_rn((v1 - __bfloat162float(h1)) - __bfloat162float(l1)));
+            } else {
+                out.hi[o] = h0;
+                out.lo[o] = l0;
+                if (out3) out3[o] = __float2bfloat16_rn((v0 - __bfloat162float(h0)) - __bfloat162float(l0));
+            }
         }
     }
 }
@@ -192,20 +205,25 @@ __global__ void __launch_bounds__(256) k_absmax(const float4* __restrict__ x, si
     for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
     if ((threadIdx.x & 31) == 0 && m) atomicMax(out, m);
 }
-// in [rows][cols] fp32 -> out [cols][ldo] fp16 of in * 2^e, e from the array's maximum (f16_scale_from_max)
+// in [rows][cols] fp32 -> out [cols][ldo] fp16 of in * 2^e, e from the array's maximum (f16_scale_from_max); tiles and
+// stores as in k_transpose_split
 __global__ void k_transpose_f16(const float* __restrict__ in, int rows, int cols, int ldo, __half* __restrict__ out,
                                 const unsigned* __restrict__ amax) {
-    __shared__ float t[32][33];
+    __shared__ float t[64][33];
     const float sc = ptx::f16_scale_from_max(*amax);
-    int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-    for (int j = threadIdx.y; j < 32; j += 8) {
+    int c0 = blockIdx.x * 32, r0 = blockIdx.y * 64;
+    for (int j = threadIdx.y; j < 64; j += 8) {
         int r = r0 + j, c = c0 + threadIdx.x;
-        if (r < rows && c < cols) t[j][threadIdx.x] = in[(size_t)r * cols + c];
+        t[j][threadIdx.x] = (r < rows && c < cols) ? in[(size_t)r * cols + c] : 0.f;
     }
     __syncthreads();
     for (int j = threadIdx.y; j < 32; j += 8) {
-        int c = c0 + j, r = r0 + threadIdx.x;
-        if (r < rows && c < cols) out[(size_t)c * ldo + r] = __float2half_rn(t[threadIdx.x][j] * sc);
+        int c = c0 + j, r = r0 + 2 * threadIdx.x;
+        if (r < rows && c < cols) {
+            const size_t o = (size_t)c * ldo + r;
+            if (r + 1 < rows) *reinterpret_cast<__half2*>(out + o) = __floats2half2_rn(t[2 * threadIdx.x][j] * sc, t[2 * threadIdx.x + 1][j] * sc);
+            else out[o] = __float2half_rn(t[2 * threadIdx.x][j] * sc);
+        }
     }
 }
 
@@ -226,21 +244,21 @@ static void stats_operand(const Lc& lc, TcBuffers* t, const float* X, int rows, 
         const size_t nb = (n4 + 255) / 256;
         k_absmax<<<(unsigned)(nb < 1184 ? nb : 1184), 256, 0, lc.st>>>(reinterpret_cast<const float4*>(X), n4, t->stat + which);
         lc.count();
-        dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
+        dim3 grid((cols + 31) / 32, (rows + 63) / 64), block(32, 8);
         k_transpose_f16<<<grid, block, 0, lc.st>>>(X, rows, cols, t->ldT, reinterpret_cast<__half*>(out.hi), t->stat + which);
         lc.count();
         if (which == 0) t->stats_f16 = 1;
         return;
     }
     if (which == 0) t->stats_f16 = 0;
-    dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
+    dim3 grid((cols + 31) / 32, (rows + 63) / 64), block(32, 8);
     k_transpose_split<<<grid, block, 0, lc.st>>>(X, rows, cols, t->ldT, out, precise ? (which ? t->RT3 : t->XT3) : nullptr);
     lc.count();
 }
 
 static void transpose_split(const Lc& lc, const float* in, int rows, int cols, int ldo, Pair out,
                             __nv_bfloat16* out3 = nullptr) {
-    dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
+    dim3 grid((cols + 31) / 32, (rows + 63) / 64), block(32, 8);
     k_transpose_split<<<grid, block, 0, lc.st>>>(in, rows, cols, ldo, out, out3);
     lc.count();
 }
