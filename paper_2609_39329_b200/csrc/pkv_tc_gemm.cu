@@ -743,6 +743,13 @@ static bool pair_enabled() {
     return v && !g_pair_refused;
 }
 
+// Fewest 256 x 256 tiles for which a product goes to CTA pairs (PKV_GEMM_PAIR_MIN overrides).  Measured on the
+// config-2 block, whose 512-row halves give 32 - 48 tiles per projection: 2.71 ms with 24, 2.72 - 2.73 with 60.
+static int pair_min_tiles() {
+    static const int v = [] { const char* e = getenv("PKV_GEMM_PAIR_MIN"); return e ? atoi(e) : 24; }();
+    return v;
+}
+
 static int launch_gemm_pair(const Lc& lc, GemmTcParams& p, int batch) {
     static PerDeviceOnce once;
     constexpr int kMaxSmem = 227 * 1024;
@@ -801,7 +808,7 @@ int gemm_tc(const Lc& lc, const TcGemm& g, DevStatus* status) {
     const bool pair = pair_enabled() && !lc.pdl && g.M % 256 == 0 && g.N % 256 == 0 && g.N >= 512 && g.a_tri == 0 && g.nacc <= 1 &&
                       !g.stamps && !g.skip_tile00 && !g.out_col0_only && (!g.lower_only || g.k_tri == 0) &&
                       g.c_rows >= g.c_row0 + (g.batch - 1) * g.c_zrow + g.M && g.c_cols >= g.c_col0 + (g.batch - 1) * g.c_zcol + g.N &&
-                      pair_tiles >= 60 && (c_vec || !g.C) && (g.nout == 0 || o_vec);
+                      pair_tiles >= pair_min_tiles() && (c_vec || !g.C) && (g.nout == 0 || o_vec);
     const bool wide = g.N >= 512 && tiles256 >= 120 && !g.lower_only && g.nacc < 4;
     const int BN = pair ? 256 : ((g.skip_tile00 || g.out_col0_only) ? 128 : ((g.N <= 64) ? 64 : (wide ? 256 : 128)));
     const int boxB = pair ? 128 : BN;
