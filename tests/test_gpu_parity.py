@@ -860,6 +860,16 @@ def test_streamed_reference_set_equals_one_call_and_the_oracle(B, engine_name, l
     assert H.rel_fro(dW2.cpu().numpy(), ref["dW"]) <= DW_TOL
     with pytest.raises(B.PkvError):                      # no stream open
         ctx.stream_finish()
+    # the streamed solve with one correction of iterative refinement (the sums are kept as a full symmetric matrix)
+    if engine_name == "tc":
+        ctx.set_refinement(1)
+        ctx.stream_begin(lam0)
+        for a, e, co in parts:
+            ctx.stream_add(w, kv["K"], kv["V"], off, idx_t, tF[a:e].contiguous(), tC[a:e].contiguous(), co, cfg.L)
+        dW3, _ = ctx.stream_finish()
+        e3 = H.rel_fro(dW3.cpu().numpy(), ref["dW"])
+        print("   with one correction: dW vs oracle %.3e" % e3)
+        assert e3 <= DW_TOL and e3 <= e_or * 1.05 + 1e-5
     ctx.close()
 
 
